@@ -1,0 +1,197 @@
+/*
+ * spectre.h - C ABI of the B200 (sm_100a) SPECTRE spectral-mixer library.
+ *
+ * The library implements the per-head spectral token mixer of SPECTRE
+ * (arXiv 2502.18394): real FFT along the sequence axis, multiplication of the
+ * floor(n/2)+1 bins by a content-adaptive complex gate, inverse real FFT
+ * (Sec. 3.2, Eq. 1-4), the Prefix-FFT cache for decoding (Sec. 3.3, Eq. 5,
+ * Alg. 1) and the optional Haar wavelet refinement (Sec. 3.5).
+ *
+ * Conventions
+ *   - Every tensor argument is CALLER-OWNED DEVICE memory unless a comment says
+ *     "host".  The library never allocates or frees device memory in the calls
+ *     below (spectre_create allocates host memory only); scratch is passed in as
+ *     `workspace`, sized by the matching *_workspace_bytes query.
+ *   - All work is enqueued on the caller's stream (`stream` is a cudaStream_t
+ *     passed as void*; NULL = the default stream).  No call synchronises.
+ *   - Activations are [B, L, H, D] with D contiguous; strides are in elements.
+ *     The base pointer and every stride must keep each D-row 16-byte aligned.
+ *   - Complex numbers are interleaved (re, im) float32.
+ *   - n = n_fft is the transform length, K = n/2 + 1 (integer division) the
+ *     number of bins.  Supported n: 2^a for 0 <= a <= 17, and any
+ *     n = 2^a 3^b 5^c 7^e <= 2048.  D must be a multiple of 8.
+ *   - Every function returns a spectre_status; nothing throws or aborts.
+ *     Arguments are validated on the host before anything is launched.  There is
+ *     no CPU fallback: without a CUDA device every compute call fails.
+ */
+#ifndef SPECTRE_H_
+#define SPECTRE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPECTRE_OK = 0,
+  SPECTRE_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad shape, bad dtype      */
+  SPECTRE_ERR_UNSUPPORTED = 2,   /* valid request outside the supported set              */
+  SPECTRE_ERR_WORKSPACE = 3,     /* workspace missing or smaller than the query result   */
+  SPECTRE_ERR_CUDA = 4           /* a CUDA runtime call or launch failed                 */
+} spectre_status;
+
+typedef enum { SPECTRE_F32 = 0, SPECTRE_BF16 = 1 } spectre_dtype;
+
+typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch limits */
+
+/* Creates a context for CUDA device `device` (host allocation only). */
+int spectre_create(spectre_ctx** out, int device);
+int spectre_destroy(spectre_ctx* ctx);
+/* Static description of a status code. */
+const char* spectre_status_string(int status);
+/* Text of the most recent failure on the calling thread ("" if none). */
+const char* spectre_last_error(void);
+
+/* A [B, L, H, D] activation; D contiguous; strides in elements. */
+typedef struct {
+  void* ptr;
+  int32_t dtype;                 /* spectre_dtype */
+  int32_t B, L, H, D;
+  int64_t stride_b, stride_l, stride_h;
+} spectre_act;
+
+/* Parameters of the gate network (Sec. 3.2 step 3).  All arrays are per head
+ * ([H, ...]); with shared_across_heads != 0 they hold a single head's worth
+ * that every head uses (Sec. 3.6: gates shared across heads). */
+typedef struct {
+  int32_t wdtype;                /* spectre_dtype of W1 and W2                        */
+  int32_t hidden;                /* MLP hidden width (1..1024)                        */
+  int32_t toeplitz_r;            /* 0 = Toeplitz update off; else bandwidth 2r+1      */
+  int32_t shared_across_heads;
+  const float* ln_gamma;         /* [H, D]                                            */
+  const float* ln_beta;          /* [H, D]                                            */
+  float ln_eps;
+  const void* W1;                /* [H, D, hidden]                                    */
+  const float* b1;               /* [H, hidden]                                       */
+  const void* W2;                /* [H, hidden, 2K]  (re, im) interleaved per bin     */
+  const float* b2;               /* [H, 2K]                                           */
+  const float* modrelu_bias;     /* [H, K] or NULL (= 0)                              */
+  const float* toeplitz;         /* [H, 2r+1, 2] complex taps t_{-r..r}, or NULL      */
+} spectre_gate_params;
+
+/*
+ * spectre_gate - content-adaptive spectral gate (Sec. 3.2 step 3; Sec. 3.3.2
+ * steps c-d; Alg. 1 DecodeStep).
+ *   (a) mu = inv_count * sum_i q_i ; q_bar = LayerNorm_D(mu) ;
+ *       o = GELU(q_bar W1 + b1) W2 + b2 ; g_k = o_{2k} + j o_{2k+1}
+ *   (b) if toeplitz_r > 0: g_k <- g_k + sum_{m=-r..r} t_m g_{k-m} (zero boundary)
+ *   (c) modReLU: g_k <- max(|g_k| + bias_k, 0) g_k / |g_k|
+ *   then the positional phase g_k <- g_k exp(+j 2 pi k p / n), p = shift_all +
+ *   shift[b] ("Positional Awareness"; decode uses p = t).
+ * Either `q` (a [B, L, H, D] activation: the sum over L is computed here, and
+ * inv_count <= 0 means 1/L) or `sum_q` ([B, H, D] float32, e.g. the cache's
+ * running sum with inv_count = 1/N_max) must be given, not both.  B, H, D are
+ * always passed (and must match q when q is given).
+ *   shift      [B] int64 on the DEVICE, or NULL
+ *   g_out      [B, H, K, 2] float32
+ *   qbar_out   [B, H, D] float32 or NULL (input of the wavelet level-gate MLP)
+ *   workspace  spectre_gate_workspace_bytes(...) bytes, 16-byte aligned
+ */
+size_t spectre_gate_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
+                                    int32_t n_fft, int32_t toeplitz_r);
+int spectre_gate(spectre_ctx* ctx, void* stream,
+                 const spectre_act* q, const float* sum_q,
+                 int32_t B, int32_t H, int32_t D, float inv_count,
+                 const spectre_gate_params* params, int32_t n_fft,
+                 const int64_t* shift, int64_t shift_all,
+                 float* g_out, float* qbar_out,
+                 void* workspace, size_t workspace_bytes);
+
+/* Wavelet refinement parameters (Sec. 3.5).  Either level_gates is given, or it
+ * is NULL and the gates are computed from qbar by the two-layer MLP
+ * s = GELU(qbar Ww1 + bw1) Ww2 + bw2 (linear output). */
+typedef struct {
+  int32_t levels;                /* J >= 1; 2^J must divide L; J <= 10              */
+  int32_t hidden;                /* MLP hidden width (1..1024)                       */
+  int32_t wdtype;                /* spectre_dtype of Ww1, Ww2                        */
+  int32_t shared_across_heads;
+  const float* level_gates;      /* [B, H, J+1, D] order a_J, d_J, ..., d_1; or NULL */
+  const float* qbar;             /* [B, H, D]                                        */
+  const void* Ww1;               /* [H, D, hidden]                                   */
+  const float* bw1;              /* [H, hidden]                                      */
+  const void* Ww2;               /* [H, hidden, (J+1) D]                             */
+  const float* bw2;              /* [H, (J+1) D]                                     */
+} spectre_wavelet;
+
+/*
+ * spectre_mixer_forward - Y = R_n^{-1}( diag(g) R_n(V) ) per (batch, head)
+ * (Sec. 3.2 steps 2 and 4, Eq. 1, 3, 4); heads are written side by side in
+ * [B, L, H, D], which is the concatenation of step 4.
+ *   v, y     activations of identical shape and dtype; y may alias v only when
+ *            spectre_mixer_workspace_bytes(...) == 0 (single-pass path)
+ *   g        [B, H, K, 2] float32, K = n_fft/2 + 1; one gain per bin per head,
+ *            applied to all D columns; Im of the DC / Nyquist gains is ignored
+ *   n_fft    == L: exact circular transform of Eq. 1;  > L: rows L..n_fft-1 are
+ *            zero (the pad(.) of Sec. 3.3.1) and only rows 0..L-1 are written
+ *   wrm      NULL, or the wavelet refinement applied to Y afterwards (Sec. 3.5)
+ *   workspace  >= spectre_mixer_workspace_bytes(...) bytes, 16-byte aligned
+ *              (0 bytes / NULL allowed when the query returns 0)
+ */
+size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t L, int32_t H,
+                                     int32_t D, int32_t n_fft, int32_t dtype);
+int spectre_mixer_forward(spectre_ctx* ctx, void* stream,
+                          const spectre_act* v, const float* g, const spectre_act* y,
+                          int32_t n_fft, const spectre_wavelet* wrm,
+                          void* workspace, size_t workspace_bytes);
+
+/*
+ * spectre_wavelet_refine - Y_out = Y_in + W^{-1}( s * W Y_in ) with the
+ * orthonormal Haar transform W over aligned blocks of 2^J tokens (Sec. 3.5
+ * steps a, c, d); y_out may alias y_in.
+ */
+int spectre_wavelet_refine(spectre_ctx* ctx, void* stream,
+                           const spectre_act* y_in, const spectre_act* y_out,
+                           const spectre_wavelet* wrm);
+
+/* Prefix-FFT cache state (Alg. 1 "persistent state"), all caller-owned. */
+typedef struct {
+  int32_t B, H, D, N_max;
+  int32_t buf_dtype;             /* spectre_dtype of V_buf, Q_buf and of the tokens */
+  int32_t reserved;
+  float* prefix_fft;             /* [B, H, K, D, 2] float32, K = N_max/2 + 1        */
+  void* V_buf;                   /* [B, N_max, H, D] ring buffer                    */
+  void* Q_buf;                   /* [B, N_max, H, D] ring buffer                    */
+  float* sum_q;                  /* [B, H, D] float32 running sum of queries        */
+} spectre_cache;
+
+/*
+ * spectre_prefix_cache_prefill - PreFill of Alg. 1 (Sec. 3.3.1):
+ * prefix_fft = R_{N_max}(pad(V, N_max)) (unnormalised, Eq. 1), ring buffers
+ * rows 0..L-1 <- tokens and rows L..N_max-1 <- 0, sum_q = sum_i q_i.
+ * q, v: [B, L, H, D] with L <= N_max, dtype == buf_dtype.  N_max must be a
+ * supported n.  workspace >= spectre_prefill_workspace_bytes(...) bytes.
+ */
+size_t spectre_prefill_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
+                                       int32_t N_max);
+int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, const spectre_cache* cache,
+                                 const spectre_act* q, const spectre_act* v,
+                                 void* workspace, size_t workspace_bytes);
+
+/*
+ * spectre_prefix_cache_append - DecodeStep of Alg. 1, steps (a)-(b) of
+ * Sec. 3.3.2: with i = t mod N_max and (v_old, q_old) = ring-buffer row i if
+ * t >= N_max else 0, for every bin k
+ *   prefix_fft[k] += (v_t - v_old) exp(-j 2 pi k t / N_max)            (Eq. 5)
+ * then V_buf[i] <- v_t, Q_buf[i] <- q_t, sum_q += q_t - q_old.
+ * q_t, v_t: [B, H, D] contiguous, dtype buf_dtype.  t >= 0 is the absolute
+ * position of the new token; N_max may be any integer >= 2 here.
+ */
+int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const spectre_cache* cache,
+                                const void* q_t, const void* v_t, int64_t t);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SPECTRE_H_ */

@@ -1,0 +1,282 @@
+"""Thin ctypes binding over the C ABI of libspectre.so.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.
+Function names are those of include/spectre.h.  PyTorch appears here for device
+memory (tensors, workspace) and the current stream, nothing else.  If the
+shared library is missing the import of any entry point raises: there is no CPU
+or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspectre.so")
+_lib = None
+
+SPECTRE_OK = 0
+SPECTRE_ERR_INVALID_ARG = 1
+SPECTRE_ERR_UNSUPPORTED = 2
+SPECTRE_ERR_WORKSPACE = 3
+SPECTRE_ERR_CUDA = 4
+SPECTRE_F32 = 0
+SPECTRE_BF16 = 1
+
+EXPORTS = [
+    "spectre_create", "spectre_destroy", "spectre_status_string", "spectre_last_error",
+    "spectre_gate_workspace_bytes", "spectre_gate",
+    "spectre_mixer_workspace_bytes", "spectre_mixer_forward",
+    "spectre_wavelet_refine",
+    "spectre_prefill_workspace_bytes", "spectre_prefix_cache_prefill", "spectre_prefix_cache_append",
+]
+
+
+class SpectreError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"spectre status {status}: {msg}")
+        self.status = status
+
+
+class Act(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("dtype", C.c_int32), ("B", C.c_int32), ("L", C.c_int32),
+                ("H", C.c_int32), ("D", C.c_int32), ("stride_b", C.c_int64), ("stride_l", C.c_int64),
+                ("stride_h", C.c_int64)]
+
+
+class GateParams(C.Structure):
+    _fields_ = [("wdtype", C.c_int32), ("hidden", C.c_int32), ("toeplitz_r", C.c_int32),
+                ("shared_across_heads", C.c_int32), ("ln_gamma", C.c_void_p), ("ln_beta", C.c_void_p),
+                ("ln_eps", C.c_float), ("W1", C.c_void_p), ("b1", C.c_void_p), ("W2", C.c_void_p),
+                ("b2", C.c_void_p), ("modrelu_bias", C.c_void_p), ("toeplitz", C.c_void_p)]
+
+
+class Wavelet(C.Structure):
+    _fields_ = [("levels", C.c_int32), ("hidden", C.c_int32), ("wdtype", C.c_int32),
+                ("shared_across_heads", C.c_int32), ("level_gates", C.c_void_p), ("qbar", C.c_void_p),
+                ("Ww1", C.c_void_p), ("bw1", C.c_void_p), ("Ww2", C.c_void_p), ("bw2", C.c_void_p)]
+
+
+class Cache(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("N_max", C.c_int32),
+                ("buf_dtype", C.c_int32), ("reserved", C.c_int32), ("prefix_fft", C.c_void_p),
+                ("V_buf", C.c_void_p), ("Q_buf", C.c_void_p), ("sum_q", C.c_void_p)]
+
+
+def lib():
+    """Loads libspectre.so (built in-tree by paper_2502_18394_b200.build); fails loudly if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2502_18394_b200.build` "
+                           "(there is no CPU fallback)")
+    L = C.CDLL(_LIB_PATH)
+    L.spectre_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
+    L.spectre_destroy.argtypes = [C.c_void_p]
+    L.spectre_status_string.argtypes = [C.c_int]
+    L.spectre_status_string.restype = C.c_char_p
+    L.spectre_last_error.restype = C.c_char_p
+    L.spectre_gate_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 5
+    L.spectre_gate_workspace_bytes.restype = C.c_size_t
+    L.spectre_gate.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                               C.c_float, C.POINTER(GateParams), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p,
+                               C.c_void_p, C.c_void_p, C.c_size_t]
+    L.spectre_mixer_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 6
+    L.spectre_mixer_workspace_bytes.restype = C.c_size_t
+    L.spectre_mixer_forward.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.c_void_p, C.POINTER(Act), C.c_int32,
+                                        C.POINTER(Wavelet), C.c_void_p, C.c_size_t]
+    L.spectre_wavelet_refine.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.POINTER(Act), C.POINTER(Wavelet)]
+    L.spectre_prefill_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 4
+    L.spectre_prefill_workspace_bytes.restype = C.c_size_t
+    L.spectre_prefix_cache_prefill.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.POINTER(Act), C.POINTER(Act),
+                                               C.c_void_p, C.c_size_t]
+    L.spectre_prefix_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
+                                              C.c_int64]
+    _lib = L
+    return L
+
+
+def _check(status: int):
+    if status != SPECTRE_OK:
+        L = lib()
+        raise SpectreError(status, f"{L.spectre_status_string(status).decode()}: {L.spectre_last_error().decode()}")
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SPECTRE_F32
+    if t.dtype == torch.bfloat16:
+        return SPECTRE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def act(t: torch.Tensor) -> Act:
+    """Descriptor of a [B, L, H, D] tensor (any strides with D contiguous)."""
+    if t.dim() != 4 or t.stride(3) != 1:
+        raise ValueError("activation must be [B, L, H, D] with D contiguous")
+    return Act(t.data_ptr(), _dtype_code(t), t.shape[0], t.shape[1], t.shape[2], t.shape[3],
+               t.stride(0), t.stride(1), t.stride(2))
+
+
+class Context:
+    """Owns a spectre_ctx*; `device` is the CUDA device index."""
+
+    def __init__(self, device: int = 0):
+        self.handle = C.c_void_p()
+        _check(lib().spectre_create(C.byref(self.handle), device))
+        self.device = device
+
+    def close(self):
+        if self.handle:
+            lib().spectre_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _gate_struct(p: dict, keep: list) -> GateParams:
+    tz = p.get("toeplitz")
+    r = 0 if tz is None else (tz.shape[-2] - 1) // 2
+    keep.extend([p["ln_gamma"], p["ln_beta"], p["W1"], p["b1"], p["W2"], p["b2"], p.get("modrelu_bias"), tz])
+    return GateParams(_dtype_code(p["W1"]), int(p["hidden"]), r, int(p.get("shared_across_heads", 0)),
+                      p["ln_gamma"].data_ptr(), p["ln_beta"].data_ptr(), float(p["ln_eps"]),
+                      p["W1"].data_ptr(), p["b1"].data_ptr(), p["W2"].data_ptr(), p["b2"].data_ptr(),
+                      None if p.get("modrelu_bias") is None else p["modrelu_bias"].data_ptr(),
+                      None if tz is None else tz.data_ptr())
+
+
+def _wavelet_struct(w: dict | None, keep: list):
+    if w is None:
+        return None
+    keep.append(w)
+    g = w.get("level_gates")
+    wd = SPECTRE_F32 if w.get("Ww1") is None else _dtype_code(w["Ww1"])
+    return Wavelet(int(w["levels"]), int(w.get("hidden", 0)), wd, int(w.get("shared_across_heads", 0)),
+                   None if g is None else g.data_ptr(),
+                   None if w.get("qbar") is None else w["qbar"].data_ptr(),
+                   None if w.get("Ww1") is None else w["Ww1"].data_ptr(),
+                   None if w.get("bw1") is None else w["bw1"].data_ptr(),
+                   None if w.get("Ww2") is None else w["Ww2"].data_ptr(),
+                   None if w.get("bw2") is None else w["bw2"].data_ptr())
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor | None:
+    return torch.empty(max(nbytes, 16), dtype=torch.uint8, device=device) if nbytes > 0 else None
+
+
+def spectre_gate_workspace_bytes(ctx: Context, B, H, D, n_fft, toeplitz_r=0) -> int:
+    return lib().spectre_gate_workspace_bytes(ctx.handle, B, H, D, n_fft, toeplitz_r)
+
+
+def spectre_gate(ctx: Context, params: dict, n_fft: int, q: torch.Tensor | None = None,
+                 sum_q: torch.Tensor | None = None, inv_count: float = 0.0, shift: torch.Tensor | None = None,
+                 shift_all: int = 0, g_out: torch.Tensor | None = None, qbar_out: torch.Tensor | None = None,
+                 workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """g[B,H,K,2] = gate(...) (Sec. 3.2 step 3).  Allocates g_out / workspace with torch when not given."""
+    ref = q if q is not None else sum_q
+    if q is not None:
+        B, _, H, D = q.shape
+    else:
+        B, H, D = sum_q.shape
+    K = n_fft // 2 + 1
+    keep: list = []
+    gp = _gate_struct(params, keep)
+    if g_out is None:
+        g_out = torch.empty((B, H, K, 2), dtype=torch.float32, device=ref.device)
+    if workspace is None:
+        workspace = _workspace(spectre_gate_workspace_bytes(ctx, B, H, D, n_fft, gp.toeplitz_r), ref.device)
+    a = act(q) if q is not None else None
+    _check(lib().spectre_gate(ctx.handle, _stream(stream), None if a is None else C.byref(a), _ptr(sum_q), B, H, D,
+                              float(inv_count), C.byref(gp), n_fft, _ptr(shift), int(shift_all), _ptr(g_out),
+                              _ptr(qbar_out), _ptr(workspace), 0 if workspace is None else workspace.numel()))
+    return g_out
+
+
+def spectre_mixer_workspace_bytes(ctx: Context, B, L, H, D, n_fft, dtype_code) -> int:
+    return lib().spectre_mixer_workspace_bytes(ctx.handle, B, L, H, D, n_fft, dtype_code)
+
+
+def spectre_mixer_forward(ctx: Context, v: torch.Tensor, g: torch.Tensor, y: torch.Tensor | None = None,
+                          n_fft: int | None = None, wrm: dict | None = None,
+                          workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Y = irfft(g * rfft(V)) per head (Sec. 3.2 steps 2, 4)."""
+    B, L, H, D = v.shape
+    n = L if n_fft is None else n_fft
+    if y is None:
+        y = torch.empty_like(v)
+    if workspace is None:
+        workspace = _workspace(spectre_mixer_workspace_bytes(ctx, B, L, H, D, n, _dtype_code(v)), v.device)
+    keep: list = []
+    w = _wavelet_struct(wrm, keep)
+    av, ay = act(v), act(y)
+    _check(lib().spectre_mixer_forward(ctx.handle, _stream(stream), C.byref(av), _ptr(g), C.byref(ay), n,
+                                       None if w is None else C.byref(w), _ptr(workspace),
+                                       0 if workspace is None else workspace.numel()))
+    return y
+
+
+def spectre_wavelet_refine(ctx: Context, y_in: torch.Tensor, wrm: dict, y_out: torch.Tensor | None = None,
+                           stream=None) -> torch.Tensor:
+    """Y_out = Y_in + W^-1(s * W Y_in) (Sec. 3.5)."""
+    if y_out is None:
+        y_out = torch.empty_like(y_in)
+    keep: list = []
+    w = _wavelet_struct(wrm, keep)
+    ai, ao = act(y_in), act(y_out)
+    _check(lib().spectre_wavelet_refine(ctx.handle, _stream(stream), C.byref(ai), C.byref(ao), C.byref(w)))
+    return y_out
+
+
+class PrefixCache:
+    """Caller-owned cache tensors of Alg. 1 (allocated with torch) plus their C descriptor."""
+
+    def __init__(self, B, H, D, N_max, dtype=torch.bfloat16, device="cuda"):
+        K = N_max // 2 + 1
+        self.B, self.H, self.D, self.N_max = B, H, D, N_max
+        self.prefix_fft = torch.zeros((B, H, K, D, 2), dtype=torch.float32, device=device)
+        self.V_buf = torch.zeros((B, N_max, H, D), dtype=dtype, device=device)
+        self.Q_buf = torch.zeros((B, N_max, H, D), dtype=dtype, device=device)
+        self.sum_q = torch.zeros((B, H, D), dtype=torch.float32, device=device)
+
+    def struct(self) -> Cache:
+        return Cache(self.B, self.H, self.D, self.N_max, _dtype_code(self.V_buf), 0, self.prefix_fft.data_ptr(),
+                     self.V_buf.data_ptr(), self.Q_buf.data_ptr(), self.sum_q.data_ptr())
+
+
+def spectre_prefill_workspace_bytes(ctx: Context, B, H, D, N_max) -> int:
+    return lib().spectre_prefill_workspace_bytes(ctx.handle, B, H, D, N_max)
+
+
+def spectre_prefix_cache_prefill(ctx: Context, cache: PrefixCache, q: torch.Tensor, v: torch.Tensor,
+                                 workspace: torch.Tensor | None = None, stream=None) -> None:
+    """PreFill of Alg. 1."""
+    if workspace is None:
+        workspace = _workspace(spectre_prefill_workspace_bytes(ctx, cache.B, cache.H, cache.D, cache.N_max), v.device)
+    cs = cache.struct()
+    aq, av = act(q), act(v)
+    _check(lib().spectre_prefix_cache_prefill(ctx.handle, _stream(stream), C.byref(cs), C.byref(aq), C.byref(av),
+                                              _ptr(workspace), 0 if workspace is None else workspace.numel()))
+
+
+def spectre_prefix_cache_append(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t: torch.Tensor, t: int,
+                                stream=None) -> None:
+    """DecodeStep of Alg. 1, steps (a)-(b)."""
+    if not (q_t.is_contiguous() and v_t.is_contiguous()):
+        raise ValueError("q_t and v_t must be contiguous [B, H, D]")
+    cs = cache.struct()
+    _check(lib().spectre_prefix_cache_append(ctx.handle, _stream(stream), C.byref(cs), _ptr(q_t), _ptr(v_t), int(t)))

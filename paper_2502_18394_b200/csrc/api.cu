@@ -1,0 +1,109 @@
+// Context, status strings and host-side argument checks of the C ABI.
+#include <cstdio>
+#include <new>
+
+#include "common.cuh"
+
+namespace spectre {
+
+static thread_local std::string g_last_error;
+
+int fail(int status, const std::string& msg) {
+  g_last_error = msg;
+  return status;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  g_last_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return SPECTRE_ERR_CUDA;
+}
+
+bool is_pow2(int64_t x) { return x > 0 && (x & (x - 1)) == 0; }
+
+int radix_plan(int n, int* radices) {
+  if (n < 1) return -1;
+  int cnt = 0;
+  int rem = n;
+  const int odd[3] = {7, 5, 3};
+  for (int i = 0; i < 3; ++i) {
+    while (rem % odd[i] == 0) {
+      if (cnt >= 8) return -1;
+      radices[cnt++] = odd[i];
+      rem /= odd[i];
+    }
+  }
+  if (!is_pow2(rem)) return -1;
+  int a = 0;
+  while ((1 << a) < rem) ++a;
+  int q = a / 4, r = a % 4;
+  if (r == 1 && q >= 1) {          // 16 * 2 -> 8 * 4 keeps the stages balanced
+    for (int i = 0; i < q - 1; ++i) { if (cnt >= 8) return -1; radices[cnt++] = 16; }
+    if (cnt + 2 > 8) return -1;
+    radices[cnt++] = 8;
+    radices[cnt++] = 4;
+  } else {
+    for (int i = 0; i < q; ++i) { if (cnt >= 8) return -1; radices[cnt++] = 16; }
+    if (r > 0) { if (cnt >= 8) return -1; radices[cnt++] = 1 << r; }
+  }
+  return cnt;
+}
+
+int check_act(const spectre_act* a, const char* name) {
+  std::string nm(name);
+  if (!a) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": descriptor is NULL");
+  if (!a->ptr) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": data pointer is NULL");
+  if (a->dtype != SPECTRE_F32 && a->dtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": unknown dtype");
+  if (a->B < 1 || a->L < 1 || a->H < 1 || a->D < 1) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": non-positive extent");
+  if (a->D % 8 != 0) return fail(SPECTRE_ERR_UNSUPPORTED, nm + ": D must be a multiple of 8");
+  const int64_t es = a->dtype == SPECTRE_BF16 ? 2 : 4;
+  if (reinterpret_cast<uintptr_t>(a->ptr) & 15) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": pointer not 16-byte aligned");
+  if ((a->stride_b * es) % 16 || (a->stride_l * es) % 16 || (a->stride_h * es) % 16)
+    return fail(SPECTRE_ERR_INVALID_ARG, nm + ": strides must keep rows 16-byte aligned");
+  if (a->stride_h < a->D && a->H > 1) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": head stride smaller than D");
+  return SPECTRE_OK;
+}
+
+}  // namespace spectre
+
+using namespace spectre;
+
+extern "C" int spectre_create(spectre_ctx** out, int device) {
+  if (!out) return fail(SPECTRE_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  int count = 0;
+  cudaError_t e = cudaGetDeviceCount(&count);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDeviceCount (no CUDA device: there is no CPU fallback)");
+  if (device < 0 || device >= count) return fail(SPECTRE_ERR_INVALID_ARG, "device index out of range");
+  cudaDeviceProp prop;
+  SPECTRE_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+  if (prop.major < 10) return fail(SPECTRE_ERR_UNSUPPORTED, "built for sm_100a; this device is older");
+  spectre_ctx* c = new (std::nothrow) spectre_ctx();
+  if (!c) return fail(SPECTRE_ERR_INVALID_ARG, "out of host memory");
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  c->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+  int cl = 0;
+  cudaDeviceGetAttribute(&cl, cudaDevAttrClusterLaunch, device);
+  c->cluster_ok = cl;
+  c->l2_bytes = (size_t)prop.l2CacheSize;
+  *out = c;
+  return SPECTRE_OK;
+}
+
+extern "C" int spectre_destroy(spectre_ctx* ctx) {
+  delete ctx;
+  return SPECTRE_OK;
+}
+
+extern "C" const char* spectre_status_string(int status) {
+  switch (status) {
+    case SPECTRE_OK: return "ok";
+    case SPECTRE_ERR_INVALID_ARG: return "invalid argument";
+    case SPECTRE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SPECTRE_ERR_WORKSPACE: return "workspace missing or too small";
+    case SPECTRE_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+extern "C" const char* spectre_last_error(void) { return g_last_error.c_str(); }

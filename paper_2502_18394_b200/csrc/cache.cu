@@ -1,0 +1,246 @@
+// Prefix-FFT cache (Sec. 3.3, Eq. 5, Alg. 1): prefill and per-token append.
+#include "common.cuh"
+
+namespace spectre {
+
+// from mixer.cu / gate.cu
+int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
+                     float2* ws, int* N1_out, int* M_out);
+bool transform_supported(const spectre_ctx* ctx, int n);
+size_t transform_slab_bytes(int n, int D);
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums);
+
+// ---- prefill -----------------------------------------------------------------
+// The forward pass leaves Z = fft_n(a + jb) for each column pair (a, b) in
+// ws[slab_local][k1][kM][D/2], bin k = k1 + N1 kM.  The half spectra of the two
+// real columns follow from Hermitian symmetry (App. B):
+//   A_k = (Z_k + conj(Z_{n-k})) / 2,   B_k = (Z_k - conj(Z_{n-k})) / (2j).
+__global__ void __launch_bounds__(256) split_kernel(const float2* __restrict__ ws, float* __restrict__ prefix, int n,
+                                                    int K, int D, int N1, int M, int slab0, int nslab) {
+  const int half = D / 2;
+  const size_t total = (size_t)nslab * K * half;
+  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int c = (int)(idx % half);
+  size_t r = idx / half;
+  int k = (int)(r % K);
+  int slab_local = (int)(r / K);
+  int km = (n - k) % n;
+  size_t rk = ((size_t)slab_local * N1 + (k % N1)) * M + k / N1;
+  size_t rm = ((size_t)slab_local * N1 + (km % N1)) * M + km / N1;
+  float2 z = ws[rk * half + c], zm = ws[rm * half + c];
+  float4 out;
+  out.x = 0.5f * (z.x + zm.x);
+  out.y = 0.5f * (z.y - zm.y);
+  out.z = 0.5f * (z.y + zm.y);
+  out.w = -0.5f * (z.x - zm.x);
+  size_t o = (((size_t)(slab0 + slab_local) * K + k) * D + 2 * c) * 2;
+  *reinterpret_cast<float4*>(prefix + o) = out;
+}
+
+// Ring buffers: rows 0..L-1 <- tokens, rows L..N-1 <- 0 (Alg. 1 PreFill).
+template <typename T>
+__global__ void __launch_bounds__(256) ring_fill_kernel(const T* __restrict__ src, int64_t sb, int64_t sl, int64_t sh,
+                                                        T* __restrict__ buf, int B, int N, int H, int D, int L) {
+  constexpr int V = 16 / sizeof(T);
+  const int vec_per_row = H * D / V;
+  const size_t total = (size_t)B * N * vec_per_row;
+  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int vi = (int)(idx % vec_per_row);
+  size_t r = idx / vec_per_row;
+  int row = (int)(r % N);
+  int b = (int)(r / N);
+  int e = vi * V, h = e / D, c = e - h * D;
+  uint4 val = make_uint4(0u, 0u, 0u, 0u);
+  if (row < L) val = *reinterpret_cast<const uint4*>(src + b * sb + (int64_t)row * sl + h * sh + c);
+  *reinterpret_cast<uint4*>(buf + (((size_t)b * N + row) * H + h) * D + c) = val;
+}
+
+// ---- append ------------------------------------------------------------------
+// A warp owns 32 consecutive bins of one (batch, head): lane l evaluates the
+// twiddle of bin k0 + l once, then the warp walks the 32 bins with every lane
+// updating 2 channels (one 16-byte complex pair) of the bin's contiguous row.
+template <typename T>
+__global__ void __launch_bounds__(256) append_spectrum_kernel(float* __restrict__ prefix, const T* __restrict__ V_buf,
+                                                              const T* __restrict__ v_t, int H, int D, int N, int K,
+                                                              int slot, unsigned tm, int evict, int warps_per_slab,
+                                                              size_t nwarps_total) {
+  const size_t wid = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= nwarps_total) return;
+  const int slab = (int)(wid / warps_per_slab);
+  const int k0 = (int)(wid % warps_per_slab) * 32;
+  const int b = slab / H, h = slab - b * H;
+  // twiddle exp(-j 2 pi k t / N) of bin k0 + lane, angle reduced in integers
+  float2 my = make_float2(1.f, 0.f);
+  if (k0 + lane < K) {
+    unsigned kk = (unsigned)(((unsigned long long)(k0 + lane) * tm) % (unsigned)N);
+    my = twiddle_fwd(kk, (unsigned)N);
+  }
+  const int nb = min(32, K - k0);
+  const int half = D / 2;
+  float* base = prefix + (((size_t)slab * K + k0) * D) * 2;
+  for (int c0 = 0; c0 < half; c0 += 32) {      // uniform trip count: every lane takes part in the shuffles
+    const int c = c0 + lane;
+    const bool live = c < half;
+    float d0 = 0.f, d1 = 0.f;
+    if (live) {
+      d0 = io<T>::load1(v_t + (size_t)slab * D + 2 * c);
+      d1 = io<T>::load1(v_t + (size_t)slab * D + 2 * c + 1);
+      if (evict) {
+        const T* old = V_buf + (((size_t)b * N + slot) * H + h) * D + 2 * c;
+        d0 -= io<T>::load1(old);
+        d1 -= io<T>::load1(old + 1);
+      }
+    }
+    for (int i = 0; i < nb; ++i) {
+      float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
+      if (live) {
+        float4* p = reinterpret_cast<float4*>(base + ((size_t)i * D + 2 * c) * 2);
+        float4 v = *p;
+        v.x = fmaf(d0, wr, v.x); v.y = fmaf(d0, wi, v.y);
+        v.z = fmaf(d1, wr, v.z); v.w = fmaf(d1, wi, v.w);
+        *p = v;
+      }
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) append_ring_kernel(T* __restrict__ V_buf, T* __restrict__ Q_buf,
+                                                          float* __restrict__ sum_q, const T* __restrict__ q_t,
+                                                          const T* __restrict__ v_t, int B, int H, int D, int N,
+                                                          int slot, int evict) {
+  const int total = B * H * D;
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int b = idx / (H * D), hd = idx - b * (H * D);
+  size_t o = ((size_t)b * N + slot) * H * D + hd;
+  float qn = io<T>::load1(q_t + idx);
+  float qo = evict ? io<T>::load1(Q_buf + o) : 0.f;
+  sum_q[idx] += qn - qo;
+  Q_buf[o] = q_t[idx];
+  V_buf[o] = v_t[idx];
+}
+
+static int check_cache(const spectre_cache* c) {
+  if (!c) return fail(SPECTRE_ERR_INVALID_ARG, "cache descriptor is NULL");
+  if (c->B < 1 || c->H < 1 || c->D < 1 || c->N_max < 2) return fail(SPECTRE_ERR_INVALID_ARG, "cache extents");
+  if (c->D % 8) return fail(SPECTRE_ERR_UNSUPPORTED, "cache D must be a multiple of 8");
+  if (c->buf_dtype != SPECTRE_F32 && c->buf_dtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, "cache dtype");
+  if (!c->prefix_fft || !c->V_buf || !c->Q_buf || !c->sum_q) return fail(SPECTRE_ERR_INVALID_ARG, "cache pointer is NULL");
+  if ((reinterpret_cast<uintptr_t>(c->prefix_fft) | reinterpret_cast<uintptr_t>(c->V_buf) |
+       reinterpret_cast<uintptr_t>(c->Q_buf)) & 15)
+    return fail(SPECTRE_ERR_INVALID_ARG, "cache buffers must be 16-byte aligned");
+  return SPECTRE_OK;
+}
+
+static const size_t kPrefillWsCap = (size_t)256 << 20;   // group size cap for the prefill scratch
+
+}  // namespace spectre
+
+using namespace spectre;
+
+extern "C" size_t spectre_prefill_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D, int32_t N_max) {
+  if (!ctx || B < 1 || H < 1 || D < 8 || !transform_supported(ctx, N_max)) return 0;
+  size_t per = transform_slab_bytes(N_max, D);
+  size_t g = kPrefillWsCap / per;
+  if (g < 1) g = 1;
+  if (g > (size_t)B * H) g = (size_t)B * H;
+  return g * per;
+}
+
+extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, const spectre_cache* cache,
+                                            const spectre_act* q, const spectre_act* v, void* workspace,
+                                            size_t workspace_bytes) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  int rc = check_cache(cache);
+  if (rc != SPECTRE_OK) return rc;
+  rc = check_act(q, "q");
+  if (rc != SPECTRE_OK) return rc;
+  rc = check_act(v, "v");
+  if (rc != SPECTRE_OK) return rc;
+  const int B = cache->B, H = cache->H, D = cache->D, N = cache->N_max;
+  if (q->B != B || q->H != H || q->D != D || v->B != B || v->H != H || v->D != D || q->L != v->L)
+    return fail(SPECTRE_ERR_INVALID_ARG, "q / v shape differs from the cache");
+  if (q->dtype != cache->buf_dtype || v->dtype != cache->buf_dtype)
+    return fail(SPECTRE_ERR_INVALID_ARG, "q / v dtype differs from buf_dtype");
+  if (v->L > N) return fail(SPECTRE_ERR_INVALID_ARG, "prompt longer than N_max");
+  if (!transform_supported(ctx, N)) return fail(SPECTRE_ERR_UNSUPPORTED, "N_max outside the supported transform lengths");
+  const size_t per = transform_slab_bytes(N, D);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15))
+    return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
+  if (workspace_bytes < per) return fail(SPECTRE_ERR_WORKSPACE, "prefill workspace smaller than one (batch, head) slab");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int nslab = B * H, K = N / 2 + 1;
+  size_t gmax = workspace_bytes / per;
+  int group = gmax > (size_t)nslab ? nslab : (int)gmax;
+  float2* ws = reinterpret_cast<float2*>(workspace);
+  for (int s0 = 0; s0 < nslab; s0 += group) {
+    int cnt = nslab - s0 < group ? nslab - s0 : group;
+    int N1 = 1, M = N;
+    rc = forward_spectrum(ctx, st, v, N, s0, cnt, ws, &N1, &M);
+    if (rc != SPECTRE_OK) return rc;
+    size_t total = (size_t)cnt * K * (D / 2);
+    split_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, cache->prefix_fft, N, K, D, N1, M, s0, cnt);
+    SPECTRE_LAUNCH_OK("split_kernel");
+  }
+  const bool bf = cache->buf_dtype == SPECTRE_BF16;
+  const int V = bf ? 8 : 4;
+  size_t total = (size_t)B * N * (H * D / V);
+  unsigned blocks = (unsigned)((total + 255) / 256);
+  if (bf) {
+    ring_fill_kernel<bf16><<<blocks, 256, 0, st>>>(reinterpret_cast<const bf16*>(v->ptr), v->stride_b, v->stride_l,
+                                                    v->stride_h, reinterpret_cast<bf16*>(cache->V_buf), B, N, H, D, v->L);
+    ring_fill_kernel<bf16><<<blocks, 256, 0, st>>>(reinterpret_cast<const bf16*>(q->ptr), q->stride_b, q->stride_l,
+                                                    q->stride_h, reinterpret_cast<bf16*>(cache->Q_buf), B, N, H, D, q->L);
+  } else {
+    ring_fill_kernel<float><<<blocks, 256, 0, st>>>(reinterpret_cast<const float*>(v->ptr), v->stride_b, v->stride_l,
+                                                     v->stride_h, reinterpret_cast<float*>(cache->V_buf), B, N, H, D, v->L);
+    ring_fill_kernel<float><<<blocks, 256, 0, st>>>(reinterpret_cast<const float*>(q->ptr), q->stride_b, q->stride_l,
+                                                     q->stride_h, reinterpret_cast<float*>(cache->Q_buf), B, N, H, D, q->L);
+  }
+  SPECTRE_LAUNCH_OK("ring_fill_kernel");
+  return pool_sum(ctx, st, q, cache->sum_q);
+}
+
+extern "C" int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const spectre_cache* cache, const void* q_t,
+                                           const void* v_t, int64_t t) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  int rc = check_cache(cache);
+  if (rc != SPECTRE_OK) return rc;
+  if (!q_t || !v_t) return fail(SPECTRE_ERR_INVALID_ARG, "token pointer is NULL");
+  if (t < 0) return fail(SPECTRE_ERR_INVALID_ARG, "t must be >= 0");
+  const int B = cache->B, H = cache->H, D = cache->D, N = cache->N_max;
+  if ((size_t)B * H * D > (size_t)1 << 30) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H*D too large");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int K = N / 2 + 1;
+  const int slot = (int)(t % N);
+  const int evict = t >= N ? 1 : 0;
+  const int wps = (K + 31) / 32;
+  const size_t nwarps = (size_t)B * H * wps;
+  const unsigned blocks = (unsigned)((nwarps * 32 + 255) / 256);
+  const unsigned blocks2 = (unsigned)(((size_t)B * H * D + 255) / 256);
+  if (cache->buf_dtype == SPECTRE_BF16) {
+    append_spectrum_kernel<bf16><<<blocks, 256, 0, st>>>(cache->prefix_fft, reinterpret_cast<const bf16*>(cache->V_buf),
+                                                         reinterpret_cast<const bf16*>(v_t), H, D, N, K, slot,
+                                                         (unsigned)slot, evict, wps, nwarps);
+    append_ring_kernel<bf16><<<blocks2, 256, 0, st>>>(reinterpret_cast<bf16*>(cache->V_buf),
+                                                      reinterpret_cast<bf16*>(cache->Q_buf), cache->sum_q,
+                                                      reinterpret_cast<const bf16*>(q_t),
+                                                      reinterpret_cast<const bf16*>(v_t), B, H, D, N, slot, evict);
+  } else {
+    append_spectrum_kernel<float><<<blocks, 256, 0, st>>>(cache->prefix_fft, reinterpret_cast<const float*>(cache->V_buf),
+                                                          reinterpret_cast<const float*>(v_t), H, D, N, K, slot,
+                                                          (unsigned)slot, evict, wps, nwarps);
+    append_ring_kernel<float><<<blocks2, 256, 0, st>>>(reinterpret_cast<float*>(cache->V_buf),
+                                                       reinterpret_cast<float*>(cache->Q_buf), cache->sum_q,
+                                                       reinterpret_cast<const float*>(q_t),
+                                                       reinterpret_cast<const float*>(v_t), B, H, D, N, slot, evict);
+  }
+  SPECTRE_LAUNCH_OK("append kernels");
+  return SPECTRE_OK;
+}

@@ -1,0 +1,314 @@
+// Content-adaptive spectral gate (Sec. 3.2 step 3; Sec. 3.3.2 steps c-d).
+//   pool_kernel      sum of the query tokens over the sequence (bandwidth-bound)
+//   gate_mlp_kernel  LayerNorm + two-layer MLP; with the Toeplitz update off it
+//                    also applies modReLU and the positional phase
+//   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
+#include "common.cuh"
+
+namespace spectre {
+
+// ---- pooled sum over the sequence --------------------------------------------
+// Grid (chunks, B).  A thread owns one 8-channel vector of the [H*D] row and
+// walks the chunk's rows; partial sums are combined with float atomics into
+// sums[B,H,D] (zeroed by the caller on the same stream).
+template <typename T>
+__global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
+                                                   int H, int D, int rows_per, float* __restrict__ sums) {
+  const int b = blockIdx.y;
+  const int r0 = blockIdx.x * rows_per;
+  const int r1 = min(L, r0 + rows_per);
+  const int vec_per_head = D / 8;
+  const int nvec = H * vec_per_head;
+  for (int vi = threadIdx.x; vi < nvec; vi += blockDim.x) {
+    int h = vi / vec_per_head, c = (vi - h * vec_per_head) * 8;
+    const T* base = q + b * sb + h * sh + c;
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    int r = r0;
+    for (; r + 4 <= r1; r += 4) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        v[2 * u] = io<T>::load4(base + (int64_t)(r + u) * sl);
+        v[2 * u + 1] = io<T>::load4(base + (int64_t)(r + u) * sl + 4);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        acc[0] += v[2 * u].x; acc[1] += v[2 * u].y; acc[2] += v[2 * u].z; acc[3] += v[2 * u].w;
+        acc[4] += v[2 * u + 1].x; acc[5] += v[2 * u + 1].y; acc[6] += v[2 * u + 1].z; acc[7] += v[2 * u + 1].w;
+      }
+    }
+    for (; r < r1; ++r) {
+      float4 v0 = io<T>::load4(base + (int64_t)r * sl), v1 = io<T>::load4(base + (int64_t)r * sl + 4);
+      acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+      acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+    }
+    float* dst = sums + ((size_t)b * H + h) * D + c;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) atomicAdd(dst + i, acc[i]);
+  }
+}
+
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums) {
+  SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, (size_t)q->B * q->H * q->D * sizeof(float), st));
+  int target = (4 * ctx->sm_count + q->B - 1) / q->B;
+  if (target < 1) target = 1;
+  int rows_per = (q->L + target - 1) / target;
+  if (rows_per < 16) rows_per = 16;
+  dim3 grid((q->L + rows_per - 1) / rows_per, q->B);
+  if (q->dtype == SPECTRE_BF16)
+    pool_kernel<bf16><<<grid, 256, 0, st>>>(reinterpret_cast<const bf16*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
+                                             q->L, q->H, q->D, rows_per, sums);
+  else
+    pool_kernel<float><<<grid, 256, 0, st>>>(reinterpret_cast<const float*>(q->ptr), q->stride_b, q->stride_l,
+                                              q->stride_h, q->L, q->H, q->D, rows_per, sums);
+  SPECTRE_LAUNCH_OK("pool_kernel");
+  return SPECTRE_OK;
+}
+
+// ---- MLP ---------------------------------------------------------------------
+template <typename WT> __device__ __forceinline__ float wload(const WT* p);
+template <> __device__ __forceinline__ float wload<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float wload<bf16>(const bf16* p) { return __bfloat162float(*p); }
+template <typename WT> __device__ __forceinline__ float2 wload2(const WT* p);
+template <> __device__ __forceinline__ float2 wload2<float>(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
+template <> __device__ __forceinline__ float2 wload2<bf16>(const bf16* p) {
+  unsigned r = __ldg(reinterpret_cast<const unsigned*>(p));
+  return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u));
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < nw; ++i) t += red[i];
+  return t;
+}
+
+// q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the
+// hidden layer u = GELU(q_bar W1 + b1).
+template <typename WT>
+__device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, float inv_count, int D, int hidden,
+                                                      const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                      float eps, const WT* __restrict__ W1, const float* __restrict__ b1,
+                                                      float* qbar, float* u, float* red) {
+  float part = 0.f;
+  for (int c = threadIdx.x; c < D; c += blockDim.x) {
+    float m = sums[c] * inv_count;
+    qbar[c] = m;
+    part += m;
+  }
+  const float mean = block_sum(part, red) / (float)D;
+  part = 0.f;
+  for (int c = threadIdx.x; c < D; c += blockDim.x) {
+    float dlt = qbar[c] - mean;
+    part += dlt * dlt;
+  }
+  const float var = block_sum(part, red) / (float)D;
+  const float rstd = 1.0f / sqrtf(var + eps);
+  for (int c = threadIdx.x; c < D; c += blockDim.x) qbar[c] = gamma[c] * (qbar[c] - mean) * rstd + beta[c];
+  __syncthreads();
+  for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
+    float acc = b1[j];
+    for (int c = 0; c < D; ++c) acc = fmaf(qbar[c], wload<WT>(W1 + (size_t)c * hidden + j), acc);
+    u[j] = gelu_erf(acc);
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ float2 modrelu_phase(float2 gk, float bias, int k, int n, unsigned pm) {
+  // modReLU: max(|z| + b, 0) z / |z|   (0 at z = 0)
+  float mag = hypotf(gk.x, gk.y);
+  float sc = mag > 0.f ? fmaxf(mag + bias, 0.f) / mag : 0.f;
+  gk = cscale(gk, sc);
+  // positional phase exp(+j 2 pi k p / n), angle reduced in integers
+  if (pm != 0u) {
+    unsigned kp = (unsigned)(((unsigned long long)k * pm) % (unsigned)n);
+    float2 w = twiddle_fwd(kp, (unsigned)n);      // exp(-j ...)
+    gk = cmulc(gk, w);                            // times its conjugate
+  }
+  return gk;
+}
+
+struct GateMlpParams {
+  const float* sums;      // [B,H,D]
+  float inv_count;
+  int H, D, hidden, n, K;
+  size_t hs_ln, hs_w1, hs_b1, hs_w2, hs_b2, hs_mb;   // per-head strides (0 when shared)
+  const float* gamma; const float* beta; float eps;
+  const void* W1; const float* b1; const void* W2; const float* b2;
+  const float* modrelu_bias;
+  const long long* shift; long long shift_all;
+  float2* g_out;          // final gate, or the raw MLP output when post != 0
+  float* qbar_out;
+  int post;               // 1: Toeplitz follows, skip modReLU/phase here
+};
+
+template <typename WT>
+__global__ void __launch_bounds__(256) gate_mlp_kernel(const GateMlpParams p) {
+  extern __shared__ float smf[];
+  float* qbar = smf;                 // [D]
+  float* u = smf + p.D;              // [hidden]
+  float* red = u + p.hidden;         // [32]
+  const int bh = blockIdx.y, b = bh / p.H, h = bh - b * p.H;
+  const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
+  const WT* W2 = reinterpret_cast<const WT*>(p.W2) + h * p.hs_w2;
+  descriptor_and_hidden<WT>(p.sums + (size_t)bh * p.D, p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln,
+                            p.beta + h * p.hs_ln, p.eps, W1, p.b1 + h * p.hs_b1, qbar, u, red);
+  if (p.qbar_out && blockIdx.x == 0)
+    for (int c = threadIdx.x; c < p.D; c += blockDim.x) p.qbar_out[(size_t)bh * p.D + c] = qbar[c];
+
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= p.K) return;
+  const float* b2 = p.b2 + h * p.hs_b2;
+  float2 acc = make_float2(b2[2 * k], b2[2 * k + 1]);
+  const size_t ld = 2 * (size_t)p.K;
+  const WT* col = W2 + 2 * (size_t)k;
+  int j = 0;
+  for (; j + 8 <= p.hidden; j += 8) {
+    float2 w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = wload2<WT>(col + (size_t)(j + i) * ld);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { acc.x = fmaf(u[j + i], w[i].x, acc.x); acc.y = fmaf(u[j + i], w[i].y, acc.y); }
+  }
+  for (; j < p.hidden; ++j) {
+    float2 w = wload2<WT>(col + (size_t)j * ld);
+    acc.x = fmaf(u[j], w.x, acc.x); acc.y = fmaf(u[j], w.y, acc.y);
+  }
+  if (!p.post) {
+    long long sh = p.shift_all + (p.shift ? p.shift[b] : 0);
+    long long pm = sh % p.n; if (pm < 0) pm += p.n;
+    float bias = p.modrelu_bias ? p.modrelu_bias[h * p.hs_mb + k] : 0.f;
+    acc = modrelu_phase(acc, bias, k, p.n, (unsigned)pm);
+  }
+  p.g_out[(size_t)bh * p.K + k] = acc;
+}
+
+struct GatePostParams {
+  const float2* g_raw; float2* g_out;
+  const float2* taps; size_t hs_t; int r;
+  const float* modrelu_bias; size_t hs_mb;
+  const long long* shift; long long shift_all;
+  int H, K, n;
+};
+
+// Toeplitz update along the bin axis ('same' window, zero boundary, reads the
+// pre-update gate), then modReLU and phase (Sec. 3.2 steps 3b-3c).
+__global__ void __launch_bounds__(256) gate_post_kernel(const GatePostParams p) {
+  const int bh = blockIdx.y, b = bh / p.H, h = bh - b * p.H;
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= p.K) return;
+  const float2* g = p.g_raw + (size_t)bh * p.K;
+  const float2* t = p.taps + h * p.hs_t;
+  float2 acc = g[k];
+  for (int m = -p.r; m <= p.r; ++m) {
+    int src = k - m;
+    if (src >= 0 && src < p.K) acc = cadd(acc, cmul(t[m + p.r], g[src]));
+  }
+  long long sh = p.shift_all + (p.shift ? p.shift[b] : 0);
+  long long pm = sh % p.n; if (pm < 0) pm += p.n;
+  float bias = p.modrelu_bias ? p.modrelu_bias[h * p.hs_mb + k] : 0.f;
+  p.g_out[(size_t)bh * p.K + k] = modrelu_phase(acc, bias, k, p.n, (unsigned)pm);
+}
+
+static size_t gate_ws_layout(int B, int H, int D, int n_fft, int r, size_t* raw_off) {
+  size_t sums = align_up((size_t)B * H * D * sizeof(float), 256);
+  *raw_off = sums;
+  size_t raw = r > 0 ? align_up((size_t)B * H * (n_fft / 2 + 1) * sizeof(float2), 256) : 0;
+  return sums + raw;
+}
+
+}  // namespace spectre
+
+using namespace spectre;
+
+extern "C" size_t spectre_gate_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D, int32_t n_fft,
+                                               int32_t toeplitz_r) {
+  (void)ctx;
+  if (B < 1 || H < 1 || D < 1 || n_fft < 1 || toeplitz_r < 0) return 0;
+  size_t off;
+  return gate_ws_layout(B, H, D, n_fft, toeplitz_r, &off);
+}
+
+extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q, const float* sum_q, int32_t B,
+                            int32_t H, int32_t D, float inv_count, const spectre_gate_params* gp, int32_t n_fft,
+                            const int64_t* shift, int64_t shift_all, float* g_out, float* qbar_out, void* workspace,
+                            size_t workspace_bytes) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  if (!gp) return fail(SPECTRE_ERR_INVALID_ARG, "gate parameters are NULL");
+  if ((q != nullptr) == (sum_q != nullptr)) return fail(SPECTRE_ERR_INVALID_ARG, "give exactly one of q and sum_q");
+  if (!g_out || (reinterpret_cast<uintptr_t>(g_out) & 7)) return fail(SPECTRE_ERR_INVALID_ARG, "g_out is NULL or misaligned");
+  if (B < 1 || H < 1 || D < 1 || D > 1024) return fail(SPECTRE_ERR_INVALID_ARG, "B, H, D must be positive (D <= 1024)");
+  if (n_fft < 1 || n_fft > (1 << 24)) return fail(SPECTRE_ERR_INVALID_ARG, "n_fft out of range");
+  if (gp->hidden < 1 || gp->hidden > 1024) return fail(SPECTRE_ERR_UNSUPPORTED, "hidden width must be in 1..1024");
+  if (gp->toeplitz_r < 0 || gp->toeplitz_r > 64) return fail(SPECTRE_ERR_UNSUPPORTED, "toeplitz_r must be in 0..64");
+  if (gp->wdtype != SPECTRE_F32 && gp->wdtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, "unknown weight dtype");
+  if (!gp->ln_gamma || !gp->ln_beta || !gp->W1 || !gp->b1 || !gp->W2 || !gp->b2)
+    return fail(SPECTRE_ERR_INVALID_ARG, "a gate parameter array is NULL");
+  if (gp->toeplitz_r > 0 && !gp->toeplitz) return fail(SPECTRE_ERR_INVALID_ARG, "toeplitz taps are NULL");
+  if (reinterpret_cast<uintptr_t>(gp->W2) & 7) return fail(SPECTRE_ERR_INVALID_ARG, "W2 not 8-byte aligned");
+  if (!(gp->ln_eps >= 0.f)) return fail(SPECTRE_ERR_INVALID_ARG, "ln_eps must be >= 0");
+  if (q) {
+    int rc = check_act(q, "q");
+    if (rc != SPECTRE_OK) return rc;
+    if (q->B != B || q->H != H || q->D != D) return fail(SPECTRE_ERR_INVALID_ARG, "q shape differs from B, H, D");
+    if (!(inv_count > 0.f)) inv_count = 1.0f / (float)q->L;
+  } else if (!(inv_count > 0.f)) {
+    return fail(SPECTRE_ERR_INVALID_ARG, "inv_count must be positive with sum_q");
+  }
+  const int K = n_fft / 2 + 1;
+  const int r = gp->toeplitz_r;
+  size_t raw_off;
+  const size_t need = gate_ws_layout(B, H, D, n_fft, r, &raw_off);
+  const bool need_ws = (q != nullptr) || r > 0;
+  if (need_ws) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15))
+      return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
+    if (workspace_bytes < need) return fail(SPECTRE_ERR_WORKSPACE, "gate workspace too small");
+  }
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const float* sums = sum_q;
+  if (q) {
+    float* pooled = reinterpret_cast<float*>(workspace);
+    int rc = pool_sum(ctx, st, q, pooled);
+    if (rc != SPECTRE_OK) return rc;
+    sums = pooled;
+  }
+  const size_t one = gp->shared_across_heads ? 0 : 1;
+  GateMlpParams mp = {};
+  mp.sums = sums; mp.inv_count = inv_count;
+  mp.H = H; mp.D = D; mp.hidden = gp->hidden; mp.n = n_fft; mp.K = K;
+  mp.hs_ln = one * D; mp.hs_w1 = one * (size_t)D * gp->hidden; mp.hs_b1 = one * gp->hidden;
+  mp.hs_w2 = one * (size_t)gp->hidden * 2 * K; mp.hs_b2 = one * 2 * (size_t)K; mp.hs_mb = one * K;
+  mp.gamma = gp->ln_gamma; mp.beta = gp->ln_beta; mp.eps = gp->ln_eps;
+  mp.W1 = gp->W1; mp.b1 = gp->b1; mp.W2 = gp->W2; mp.b2 = gp->b2;
+  mp.modrelu_bias = gp->modrelu_bias;
+  mp.shift = reinterpret_cast<const long long*>(shift); mp.shift_all = shift_all;
+  mp.qbar_out = qbar_out;
+  mp.post = r > 0;
+  float2* raw = r > 0 ? reinterpret_cast<float2*>(reinterpret_cast<char*>(workspace) + raw_off) : nullptr;
+  mp.g_out = r > 0 ? raw : reinterpret_cast<float2*>(g_out);
+  dim3 grid((K + 255) / 256, B * H);
+  if (grid.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H exceeds 65535");
+  size_t smem = (size_t)(D + gp->hidden + 32) * sizeof(float);
+  if (gp->wdtype == SPECTRE_BF16) gate_mlp_kernel<bf16><<<grid, 256, smem, st>>>(mp);
+  else gate_mlp_kernel<float><<<grid, 256, smem, st>>>(mp);
+  SPECTRE_LAUNCH_OK("gate_mlp_kernel");
+  if (r > 0) {
+    GatePostParams pp = {};
+    pp.g_raw = raw; pp.g_out = reinterpret_cast<float2*>(g_out);
+    pp.taps = reinterpret_cast<const float2*>(gp->toeplitz); pp.hs_t = one * (2 * r + 1); pp.r = r;
+    pp.modrelu_bias = gp->modrelu_bias; pp.hs_mb = one * K;
+    pp.shift = mp.shift; pp.shift_all = shift_all;
+    pp.H = H; pp.K = K; pp.n = n_fft;
+    gate_post_kernel<<<grid, 256, 0, st>>>(pp);
+    SPECTRE_LAUNCH_OK("gate_post_kernel");
+  }
+  return SPECTRE_OK;
+}

@@ -1,0 +1,620 @@
+// Spectral mixer kernels: Y = R_n^{-1}( diag(g) R_n(V) )  (Sec. 3.2 steps 2 and 4).
+//
+// Formulation.  Two adjacent real columns a, b of a head are carried as ONE
+// complex sequence z = a + jb.  With G the Hermitian extension of the half
+// spectrum gate g (G_k = g_k for k <= n/2, conj(g_{n-k}) above, Im G_0 =
+// Im G_{n/2} = 0), ifft_n(G * fft_n(z)) = irfft(g * rfft a) + j irfft(g * rfft b),
+// so a head is D/2 complex transforms with no real/complex split or merge.
+//
+// The forward transform is decimation-in-frequency (natural order in,
+// digit-reversed order out), the gate is applied in digit-reversed order, and
+// the inverse is the mirrored decimation-in-time network, so no reordering pass
+// exists.  A tile is 8 complex pairs (16 real columns) of one (batch, head).
+//
+//   onchip kernel   whole transform of a tile in shared memory; optionally a
+//                   cluster of C CTAs splits the sequence and exchanges one
+//                   radix-C stage through distributed shared memory.
+//   strided kernels the outer factor N1 of a four-step transform n = N1 * M for
+//                   n beyond the on-chip range, with the twiddles fused.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace spectre {
+
+constexpr int kMaxStages = 8;
+constexpr int kLocalMax = 2048;      // rows of a tile one CTA keeps in shared memory
+
+struct OnchipParams {
+  const void* src;       // real [B,L,H,D] tensor (src_ws = 0)
+  void* dst;             // real [B,L,H,D] tensor (dst_ws = 0)
+  float2* ws;            // complex workspace [slab_local][N1][M][D/2]
+  const float2* g;       // gate [B*H][K]
+  int64_t s_sb, s_sl, s_sh;
+  int64_t d_sb, d_sl, d_sh;
+  int H, D, L;
+  int n, K;              // full transform length, bins
+  int M, Mloc, C;        // this kernel's transform: M = C * Mloc
+  int N1;                // outer factor of the four-step split (1 = none)
+  int slab0;             // first (b*H + h) slab handled by this launch
+  int ntile;             // 16-column tiles per slab
+  int nstage;
+  int radix[kMaxStages];
+  int prefix[kMaxStages];   // prefix[i] = radix[0] * ... * radix[i-1]
+  int mode;              // 0: forward, gate, inverse   1: forward only -> spectrum in ws
+  int src_ws, dst_ws;
+  float scale;           // 1/n, folded into the gate
+};
+
+struct TileCoord {
+  int rank, tile, k1, slab_local, b, h;
+};
+
+__device__ __forceinline__ TileCoord tile_coord(const OnchipParams& p) {
+  TileCoord t;
+  int u = blockIdx.x;
+  t.rank = u % p.C;  u /= p.C;
+  t.tile = u % p.ntile;  u /= p.ntile;
+  t.k1 = u % p.N1;  u /= p.N1;
+  t.slab_local = u;
+  int slab = p.slab0 + u;
+  t.b = slab / p.H;
+  t.h = slab - t.b * p.H;
+  return t;
+}
+
+// Element j of the length-M sequence, pair group pg (4 real columns / 2 pairs).
+template <typename T>
+__device__ __forceinline__ float4 load_elem(const OnchipParams& p, const TileCoord& tc, int j, int pg) {
+  int col = tc.tile * 16 + pg * 4;
+  if (col >= p.D) return make_float4(0.f, 0.f, 0.f, 0.f);
+  if (p.src_ws) {
+    size_t row = ((size_t)tc.slab_local * p.N1 + tc.k1) * p.M + j;
+    return *reinterpret_cast<const float4*>(p.ws + row * (p.D / 2) + col / 2);
+  }
+  if (j >= p.L) return make_float4(0.f, 0.f, 0.f, 0.f);
+  const T* ptr = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + (int64_t)j * p.s_sl + tc.h * p.s_sh + col;
+  return io<T>::load4(ptr);
+}
+
+template <typename T>
+__device__ __forceinline__ void store_elem(const OnchipParams& p, const TileCoord& tc, int j, int pg, float4 v) {
+  int col = tc.tile * 16 + pg * 4;
+  if (col >= p.D) return;
+  if (p.dst_ws) {
+    size_t row = ((size_t)tc.slab_local * p.N1 + tc.k1) * p.M + j;
+    *reinterpret_cast<float4*>(p.ws + row * (p.D / 2) + col / 2) = v;
+    return;
+  }
+  if (j >= p.L) return;
+  T* ptr = reinterpret_cast<T*>(p.dst) + tc.b * p.d_sb + (int64_t)j * p.d_sl + tc.h * p.d_sh + col;
+  io<T>::store4(ptr, v);
+}
+
+// Hermitian extension of the half-spectrum gate at full-spectrum index k.
+__device__ __forceinline__ float2 gate_at(const float2* __restrict__ g, int k, int n) {
+  int kk = (2 * k <= n) ? k : n - k;
+  float2 v = __ldg(g + kk);
+  if (kk != k) v.y = -v.y;
+  if (k == 0 || 2 * k == n) v.y = 0.f;
+  return v;
+}
+
+// One radix-R stage on block size S of the tile in shared memory.
+//   forward (decimation in frequency): y_q'[m] = W_S^{m q'} sum_q x[m + q S/R] W_R^{q q'}
+//   inverse (decimation in time):      x[m + q S/R] = sum_q' conj(W_R^{q q'}) conj(W_S^{m q'}) y_q'[m]
+template <int R, bool INV>
+__device__ __forceinline__ void stage(float4* sm, const float2* tw, int Mloc, int S) {
+  const int sub = S / R;
+  const int step = Mloc / S;
+  const int nwork = (Mloc / R) * 4;
+  for (int w = threadIdx.x; w < nwork; w += blockDim.x) {
+    int pg = w & 3, bf = w >> 2;
+    int blk = bf / sub, m = bf - blk * sub;
+    float4* base = sm + ((size_t)(blk * S + m) * 4 + pg);
+    float2 xa[R], xb[R];
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+      float4 v = base[(size_t)q * sub * 4];
+      xa[q] = make_float2(v.x, v.y);
+      xb[q] = make_float2(v.z, v.w);
+    }
+    if (INV) {
+#pragma unroll
+      for (int q = 1; q < R; ++q) {
+        float2 t = tw[m * q * step];
+        xa[q] = cmulc(xa[q], t);
+        xb[q] = cmulc(xb[q], t);
+      }
+    }
+    Dft<R, INV>::run(xa);
+    Dft<R, INV>::run(xb);
+    if (!INV) {
+#pragma unroll
+      for (int q = 1; q < R; ++q) {
+        float2 t = tw[m * q * step];
+        xa[q] = cmul(xa[q], t);
+        xb[q] = cmul(xb[q], t);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < R; ++q) base[(size_t)q * sub * 4] = make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y);
+  }
+}
+
+template <bool INV>
+__device__ __forceinline__ void run_stage(int R, float4* sm, const float2* tw, int Mloc, int S) {
+  switch (R) {
+    case 16: stage<16, INV>(sm, tw, Mloc, S); break;
+    case 8: stage<8, INV>(sm, tw, Mloc, S); break;
+    case 4: stage<4, INV>(sm, tw, Mloc, S); break;
+    case 2: stage<2, INV>(sm, tw, Mloc, S); break;
+    case 7: stage<7, INV>(sm, tw, Mloc, S); break;
+    case 5: stage<5, INV>(sm, tw, Mloc, S); break;
+    case 3: stage<3, INV>(sm, tw, Mloc, S); break;
+    default: break;
+  }
+}
+
+// Last forward stage (block size = radix, no twiddles) fused with the gate and,
+// in mode 0, the first inverse stage.  Local position blk*R + q' holds local
+// frequency kl = rev(blk) + (Mloc/R) q'.
+template <typename T, int R>
+__device__ __forceinline__ void middle(const OnchipParams& p, const TileCoord& tc, float4* sm) {
+  const int nwork = (p.Mloc / R) * 4;
+  const int nst = p.nstage;
+  const float2* g = p.g + (size_t)(p.slab0 + tc.slab_local) * p.K;
+  for (int w = threadIdx.x; w < nwork; w += blockDim.x) {
+    int pg = w & 3, blk = w >> 2;
+    float4* base = sm + ((size_t)blk * R * 4 + pg);
+    float2 xa[R], xb[R];
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+      float4 v = base[q * 4];
+      xa[q] = make_float2(v.x, v.y);
+      xb[q] = make_float2(v.z, v.w);
+    }
+    Dft<R, false>::run(xa);
+    Dft<R, false>::run(xb);
+    int rev = 0, tmp = blk;
+    for (int i = nst - 2; i >= 0; --i) {
+      int d = tmp % p.radix[i];
+      tmp /= p.radix[i];
+      rev += d * p.prefix[i];
+    }
+    const int kstep = p.Mloc / R;
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+      int kl = rev + kstep * q;
+      int kM = tc.rank + p.C * kl;
+      if (p.mode == 0) {
+        int k = tc.k1 + p.N1 * kM;
+        float2 G = cscale(gate_at(g, k, p.n), p.scale);
+        xa[q] = cmul(xa[q], G);
+        xb[q] = cmul(xb[q], G);
+      } else {
+        store_elem<T>(p, tc, kM, pg, make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y));
+      }
+    }
+    if (p.mode == 0) {
+      Dft<R, true>::run(xa);
+      Dft<R, true>::run(xb);
+#pragma unroll
+      for (int q = 0; q < R; ++q) base[q * 4] = make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y);
+    }
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void run_middle(int R, const OnchipParams& p, const TileCoord& tc, float4* sm) {
+  switch (R) {
+    case 16: middle<T, 16>(p, tc, sm); break;
+    case 8: middle<T, 8>(p, tc, sm); break;
+    case 4: middle<T, 4>(p, tc, sm); break;
+    case 2: middle<T, 2>(p, tc, sm); break;
+    case 7: middle<T, 7>(p, tc, sm); break;
+    case 5: middle<T, 5>(p, tc, sm); break;
+    case 3: middle<T, 3>(p, tc, sm); break;
+    default: middle<T, 1>(p, tc, sm); break;
+  }
+}
+
+// Radix-C stage across the CTAs of a cluster.  CTA `rank` computes the
+// butterflies of rows m in [rank*Mloc/C, (rank+1)*Mloc/C): forward reads
+// x[m + q Mloc] from global memory and writes y_q'[m] into CTA q' (remote
+// shared memory); inverse reads y_q'[m] from CTA q' and writes x[m + q Mloc].
+template <typename T, int C, bool INV>
+__device__ __forceinline__ void cross_stage(const OnchipParams& p, const TileCoord& tc, float4* sm,
+                                            cg::cluster_group& cluster) {
+  const int per = p.Mloc / C;
+  const int nwork = per * 4;
+  float4* remote[C];
+#pragma unroll
+  for (int q = 0; q < C; ++q) remote[q] = cluster.map_shared_rank(sm, q);
+  for (int w = threadIdx.x; w < nwork; w += blockDim.x) {
+    int pg = w & 3, m = tc.rank * per + (w >> 2);
+    float2 xa[C], xb[C];
+    float2 w1 = twiddle_fwd((unsigned)m, (unsigned)p.M);
+    float2 wq[C];
+    wq[0] = make_float2(1.f, 0.f);
+#pragma unroll
+    for (int q = 1; q < C; ++q) wq[q] = (q == 1) ? w1 : cmul(wq[q / 2], wq[q - q / 2]);
+#pragma unroll
+    for (int q = 0; q < C; ++q) {
+      float4 v = INV ? remote[q][(size_t)m * 4 + pg] : load_elem<T>(p, tc, m + q * p.Mloc, pg);
+      xa[q] = make_float2(v.x, v.y);
+      xb[q] = make_float2(v.z, v.w);
+      if (INV && q > 0) {
+        xa[q] = cmulc(xa[q], wq[q]);
+        xb[q] = cmulc(xb[q], wq[q]);
+      }
+    }
+    Dft<C, INV>::run(xa);
+    Dft<C, INV>::run(xb);
+#pragma unroll
+    for (int q = 0; q < C; ++q) {
+      if (!INV && q > 0) {
+        xa[q] = cmul(xa[q], wq[q]);
+        xb[q] = cmul(xb[q], wq[q]);
+      }
+      float4 v = make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y);
+      if (INV) store_elem<T>(p, tc, m + q * p.Mloc, pg, v);
+      else remote[q][(size_t)m * 4 + pg] = v;
+    }
+  }
+}
+
+template <typename T, int C>
+__global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float4* sm = reinterpret_cast<float4*>(smem_raw);                       // [Mloc][4] (8 complex pairs per row)
+  float2* tw = reinterpret_cast<float2*>(smem_raw + (size_t)p.Mloc * 64);  // [Mloc] exp(-j 2 pi i / Mloc)
+  const TileCoord tc = tile_coord(p);
+  const int Mloc = p.Mloc;
+
+  for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = twiddle_fwd((unsigned)i, (unsigned)Mloc);
+
+  if (C == 1) {
+    for (int i = threadIdx.x; i < Mloc * 4; i += blockDim.x) sm[i] = load_elem<T>(p, tc, i >> 2, i & 3);
+    __syncthreads();
+  } else {
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();                       // every CTA of the cluster is resident before remote writes
+    cross_stage<T, C, false>(p, tc, sm, cluster);
+    cluster.sync();
+  }
+
+  // forward stages (all but the last), the fused middle, inverse stages mirrored
+  int S = Mloc;
+  for (int s = 0; s + 1 < p.nstage; ++s) {
+    run_stage<false>(p.radix[s], sm, tw, Mloc, S);
+    S /= p.radix[s];
+    __syncthreads();
+  }
+  run_middle<T>(p.nstage > 0 ? p.radix[p.nstage - 1] : 1, p, tc, sm);
+  if (p.mode != 0) return;                // forward only: spectrum already written
+  __syncthreads();
+  for (int s = p.nstage - 2; s >= 0; --s) {
+    S *= p.radix[s];
+    run_stage<true>(p.radix[s], sm, tw, Mloc, S);
+    __syncthreads();
+  }
+
+  if (C == 1) {
+    for (int i = threadIdx.x; i < Mloc * 4; i += blockDim.x) store_elem<T>(p, tc, i >> 2, i & 3, sm[i]);
+  } else {
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();
+    cross_stage<T, C, true>(p, tc, sm, cluster);
+    cluster.sync();                       // no CTA exits while a peer still reads its shared memory
+  }
+}
+
+// ---- four-step outer factor -------------------------------------------------
+// n = N1 * M, t = n1 M + n2, k = k1 + N1 k2.  Forward: for each n2 an N1-point
+// DFT over n1, times W_n^{n2 k1}, stored at ws[k1][n2].  Inverse: the mirror.
+struct StridedParams {
+  const void* src;
+  void* dst;
+  float2* ws;
+  int64_t s_sb, s_sl, s_sh;
+  int64_t d_sb, d_sl, d_sh;
+  int H, D, L, n, M, slab0, nslab;
+};
+
+template <typename T, int N1, bool INV>
+__global__ void __launch_bounds__(256) strided_kernel(const StridedParams p) {
+  const int npg = p.D / 4;
+  const size_t total = (size_t)p.nslab * p.M * npg;
+  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int pg = (int)(idx % npg);
+  size_t r = idx / npg;
+  int n2 = (int)(r % p.M);
+  int slab_local = (int)(r / p.M);
+  int slab = p.slab0 + slab_local;
+  int b = slab / p.H, h = slab - b * p.H;
+  const int col = pg * 4;
+
+  float2 w1 = twiddle_fwd((unsigned)n2, (unsigned)p.n);
+  float2 wq[N1];
+  wq[0] = make_float2(1.f, 0.f);
+#pragma unroll
+  for (int q = 1; q < N1; ++q) wq[q] = (q == 1) ? w1 : cmul(wq[q / 2], wq[q - q / 2]);
+
+  float2 xa[N1], xb[N1];
+  if (!INV) {
+    const T* src = reinterpret_cast<const T*>(p.src) + b * p.s_sb + h * p.s_sh + col;
+#pragma unroll
+    for (int n1 = 0; n1 < N1; ++n1) {
+      int t = n1 * p.M + n2;
+      float4 v = (t < p.L) ? io<T>::load4(src + (int64_t)t * p.s_sl) : make_float4(0.f, 0.f, 0.f, 0.f);
+      xa[n1] = make_float2(v.x, v.y);
+      xb[n1] = make_float2(v.z, v.w);
+    }
+  } else {
+#pragma unroll
+    for (int k1 = 0; k1 < N1; ++k1) {
+      size_t row = ((size_t)slab_local * N1 + k1) * p.M + n2;
+      float4 v = *reinterpret_cast<const float4*>(p.ws + row * (p.D / 2) + col / 2);
+      xa[k1] = make_float2(v.x, v.y);
+      xb[k1] = make_float2(v.z, v.w);
+      if (k1 > 0) {
+        xa[k1] = cmulc(xa[k1], wq[k1]);
+        xb[k1] = cmulc(xb[k1], wq[k1]);
+      }
+    }
+  }
+  Dft<N1, INV>::run(xa);
+  Dft<N1, INV>::run(xb);
+  if (!INV) {
+#pragma unroll
+    for (int k1 = 0; k1 < N1; ++k1) {
+      if (k1 > 0) {
+        xa[k1] = cmul(xa[k1], wq[k1]);
+        xb[k1] = cmul(xb[k1], wq[k1]);
+      }
+      size_t row = ((size_t)slab_local * N1 + k1) * p.M + n2;
+      *reinterpret_cast<float4*>(p.ws + row * (p.D / 2) + col / 2) = make_float4(xa[k1].x, xa[k1].y, xb[k1].x, xb[k1].y);
+    }
+  } else {
+    T* dst = reinterpret_cast<T*>(p.dst) + b * p.d_sb + h * p.d_sh + col;
+#pragma unroll
+    for (int n1 = 0; n1 < N1; ++n1) {
+      int t = n1 * p.M + n2;
+      if (t < p.L) io<T>::store4(dst + (int64_t)t * p.d_sl, make_float4(xa[n1].x, xa[n1].y, xb[n1].x, xb[n1].y));
+    }
+  }
+}
+
+// ---- host side ----------------------------------------------------------------
+struct TransformPlan {
+  int n, M, Mloc, C, N1;
+  int nstage, radix[kMaxStages], prefix[kMaxStages];
+  int threads;
+  size_t smem;
+};
+
+// Chooses the decomposition for transform length n; false if unsupported.
+static bool make_plan(const spectre_ctx* ctx, int n, TransformPlan* pl) {
+  pl->n = n;
+  pl->N1 = 1;
+  pl->C = 1;
+  if (n < 1) return false;
+  int M = n;
+  if (n > kLocalMax) {
+    if (!is_pow2(n) || n > (1 << 17) || !ctx->cluster_ok) return false;
+    if (n <= 4 * kLocalMax) {
+      pl->C = n / kLocalMax;
+    } else {
+      pl->C = 4;
+      pl->N1 = n / (4 * kLocalMax);
+      M = 4 * kLocalMax;
+    }
+  }
+  pl->M = M;
+  pl->Mloc = M / pl->C;
+  pl->nstage = radix_plan(pl->Mloc, pl->radix);
+  if (pl->nstage < 0) return false;
+  int pre = 1;
+  for (int i = 0; i < pl->nstage; ++i) { pl->prefix[i] = pre; pre *= pl->radix[i]; }
+  int want = pl->Mloc * 4 / 8;
+  int thr = (want + 31) / 32 * 32;
+  pl->threads = thr < 64 ? 64 : (thr > 512 ? 512 : thr);
+  pl->smem = (size_t)pl->Mloc * 64 + (size_t)pl->Mloc * 8;
+  return pl->smem <= (size_t)ctx->max_smem_optin;
+}
+
+template <typename T, int C>
+static int launch_onchip_c(const OnchipParams& p, const TransformPlan& pl, int nslab, cudaStream_t st) {
+  auto kern = onchip_kernel<T, C>;
+  if (pl.smem > 48 * 1024)
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((size_t)nslab * pl.N1 * p.ntile * C), 1, 1);
+  cfg.blockDim = dim3(pl.threads, 1, 1);
+  cfg.dynamicSmemBytes = pl.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (C > 1) ? 1 : 0;
+  SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
+  return SPECTRE_OK;
+}
+
+template <typename T>
+static int launch_onchip(const OnchipParams& p, const TransformPlan& pl, int nslab, cudaStream_t st) {
+  switch (pl.C) {
+    case 1: return launch_onchip_c<T, 1>(p, pl, nslab, st);
+    case 2: return launch_onchip_c<T, 2>(p, pl, nslab, st);
+    case 4: return launch_onchip_c<T, 4>(p, pl, nslab, st);
+    default: return fail(SPECTRE_ERR_UNSUPPORTED, "cluster size not supported");
+  }
+}
+
+template <typename T, bool INV>
+static int launch_strided(const StridedParams& p, int N1, cudaStream_t st) {
+  size_t total = (size_t)p.nslab * p.M * (p.D / 4);
+  unsigned blocks = (unsigned)((total + 255) / 256);
+  switch (N1) {
+    case 2: strided_kernel<T, 2, INV><<<blocks, 256, 0, st>>>(p); break;
+    case 4: strided_kernel<T, 4, INV><<<blocks, 256, 0, st>>>(p); break;
+    case 8: strided_kernel<T, 8, INV><<<blocks, 256, 0, st>>>(p); break;
+    case 16: strided_kernel<T, 16, INV><<<blocks, 256, 0, st>>>(p); break;
+    default: return fail(SPECTRE_ERR_UNSUPPORTED, "outer factor not supported");
+  }
+  SPECTRE_LAUNCH_OK("strided_kernel");
+  return SPECTRE_OK;
+}
+
+static void fill_common(OnchipParams& p, const TransformPlan& pl, int H, int D, int L) {
+  p.H = H; p.D = D; p.L = L;
+  p.n = pl.n; p.K = pl.n / 2 + 1;
+  p.M = pl.M; p.Mloc = pl.Mloc; p.C = pl.C; p.N1 = pl.N1;
+  p.ntile = (D + 15) / 16;
+  p.nstage = pl.nstage;
+  for (int i = 0; i < kMaxStages; ++i) { p.radix[i] = i < pl.nstage ? pl.radix[i] : 1; p.prefix[i] = i < pl.nstage ? pl.prefix[i] : 1; }
+  p.scale = 1.0f / (float)pl.n;
+}
+
+static size_t slab_ws_bytes(int n, int D) { return (size_t)n * (D / 2) * sizeof(float2); }
+
+// Number of (batch, head) slabs whose four-step intermediates are processed per
+// group of launches: few enough that the group's workspace stays L2-resident.
+static int preferred_group(const spectre_ctx* ctx, int n, int D, int nslab_total) {
+  size_t per = slab_ws_bytes(n, D);
+  size_t budget = ctx->l2_bytes / 2;
+  int g = (int)(budget / per);
+  if (g < 1) g = 1;
+  if (g > nslab_total) g = nslab_total;
+  return g;
+}
+
+template <typename T>
+static int mixer_typed(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                       const spectre_act* y, const TransformPlan& pl, void* ws, size_t ws_bytes) {
+  const int nslab = v->B * v->H;
+  OnchipParams p = {};
+  fill_common(p, pl, v->H, v->D, v->L);
+  p.src = v->ptr; p.dst = y->ptr;
+  p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
+  p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
+  p.g = reinterpret_cast<const float2*>(g);
+  p.mode = 0;
+  if (pl.N1 == 1) {
+    p.slab0 = 0; p.src_ws = 0; p.dst_ws = 0; p.ws = nullptr;
+    return launch_onchip<T>(p, pl, nslab, st);
+  }
+  const size_t per = slab_ws_bytes(pl.n, v->D);
+  int group = (int)(ws_bytes / per);
+  int pref = preferred_group(ctx, pl.n, v->D, nslab);
+  if (group > pref) group = pref;
+  if (group < 1) return fail(SPECTRE_ERR_WORKSPACE, "mixer workspace smaller than one (batch, head) slab");
+  StridedParams sp = {};
+  sp.src = v->ptr; sp.dst = y->ptr; sp.ws = reinterpret_cast<float2*>(ws);
+  sp.s_sb = v->stride_b; sp.s_sl = v->stride_l; sp.s_sh = v->stride_h;
+  sp.d_sb = y->stride_b; sp.d_sl = y->stride_l; sp.d_sh = y->stride_h;
+  sp.H = v->H; sp.D = v->D; sp.L = v->L; sp.n = pl.n; sp.M = pl.M;
+  p.ws = sp.ws; p.src_ws = 1; p.dst_ws = 1;
+  for (int s0 = 0; s0 < nslab; s0 += group) {
+    int cnt = nslab - s0 < group ? nslab - s0 : group;
+    sp.slab0 = s0; sp.nslab = cnt;
+    p.slab0 = s0;
+    int rc = launch_strided<T, false>(sp, pl.N1, st);
+    if (rc != SPECTRE_OK) return rc;
+    rc = launch_onchip<T>(p, pl, cnt, st);
+    if (rc != SPECTRE_OK) return rc;
+    rc = launch_strided<T, true>(sp, pl.N1, st);
+    if (rc != SPECTRE_OK) return rc;
+  }
+  return SPECTRE_OK;
+}
+
+// Forward transform only (used by the cache prefill): complex spectrum of the
+// pair-packed columns for slabs [slab0, slab0+cnt) into ws, laid out
+// ws[slab_local][k1][kM][D/2] with bin k = k1 + N1 * kM.
+int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
+                     float2* ws, int* N1_out, int* M_out) {
+  TransformPlan pl;
+  if (!make_plan(ctx, n, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
+  *N1_out = pl.N1; *M_out = pl.M;
+  OnchipParams p = {};
+  fill_common(p, pl, v->H, v->D, v->L);
+  p.src = v->ptr;
+  p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
+  p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
+  const bool bf = v->dtype == SPECTRE_BF16;
+  if (pl.N1 == 1) {
+    p.src_ws = 0;
+    return bf ? launch_onchip<bf16>(p, pl, cnt, st) : launch_onchip<float>(p, pl, cnt, st);
+  }
+  StridedParams sp = {};
+  sp.src = v->ptr; sp.ws = ws;
+  sp.s_sb = v->stride_b; sp.s_sl = v->stride_l; sp.s_sh = v->stride_h;
+  sp.H = v->H; sp.D = v->D; sp.L = v->L; sp.n = pl.n; sp.M = pl.M;
+  sp.slab0 = slab0; sp.nslab = cnt;
+  int rc = bf ? launch_strided<bf16, false>(sp, pl.N1, st) : launch_strided<float, false>(sp, pl.N1, st);
+  if (rc != SPECTRE_OK) return rc;
+  p.src_ws = 1;
+  return bf ? launch_onchip<bf16>(p, pl, cnt, st) : launch_onchip<float>(p, pl, cnt, st);
+}
+
+bool transform_supported(const spectre_ctx* ctx, int n) {
+  TransformPlan pl;
+  return make_plan(ctx, n, &pl);
+}
+
+size_t transform_slab_bytes(int n, int D) { return slab_ws_bytes(n, D); }
+
+}  // namespace spectre
+
+using namespace spectre;
+
+extern "C" size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t L, int32_t H, int32_t D,
+                                                int32_t n_fft, int32_t dtype) {
+  (void)L; (void)dtype;
+  TransformPlan pl;
+  if (!ctx || B < 1 || H < 1 || D < 8 || !make_plan(ctx, n_fft, &pl)) return 0;
+  if (pl.N1 == 1) return 0;
+  return (size_t)preferred_group(ctx, n_fft, D, B * H) * slab_ws_bytes(n_fft, D);
+}
+
+extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spectre_act* v, const float* g,
+                                     const spectre_act* y, int32_t n_fft, const spectre_wavelet* wrm,
+                                     void* workspace, size_t workspace_bytes) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  int rc = check_act(v, "v");
+  if (rc != SPECTRE_OK) return rc;
+  rc = check_act(y, "y");
+  if (rc != SPECTRE_OK) return rc;
+  if (!g || (reinterpret_cast<uintptr_t>(g) & 7)) return fail(SPECTRE_ERR_INVALID_ARG, "g is NULL or not 8-byte aligned");
+  if (v->B != y->B || v->L != y->L || v->H != y->H || v->D != y->D || v->dtype != y->dtype)
+    return fail(SPECTRE_ERR_INVALID_ARG, "v and y differ in shape or dtype");
+  if (n_fft < v->L) return fail(SPECTRE_ERR_INVALID_ARG, "n_fft smaller than L");
+  TransformPlan pl;
+  if (!make_plan(ctx, n_fft, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "n_fft outside the supported set");
+  if (pl.N1 > 1) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15))
+      return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
+    if (workspace_bytes < slab_ws_bytes(n_fft, v->D))
+      return fail(SPECTRE_ERR_WORKSPACE, "mixer workspace smaller than one (batch, head) slab");
+    if (v->ptr == y->ptr) return fail(SPECTRE_ERR_INVALID_ARG, "y may not alias v on the multi-pass path");
+  }
+  if (wrm) {
+    if (wrm->levels < 1 || wrm->levels > 10 || (v->L % (1 << wrm->levels)) != 0)
+      return fail(SPECTRE_ERR_INVALID_ARG, "wavelet levels: 2^J must divide L");
+  }
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  rc = (v->dtype == SPECTRE_BF16) ? mixer_typed<bf16>(ctx, st, v, g, y, pl, workspace, workspace_bytes)
+                                  : mixer_typed<float>(ctx, st, v, g, y, pl, workspace, workspace_bytes);
+  if (rc != SPECTRE_OK) return rc;
+  if (wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
+  return SPECTRE_OK;
+}

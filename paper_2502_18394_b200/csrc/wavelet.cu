@@ -1,0 +1,165 @@
+// Wavelet refinement (Sec. 3.5): Y_out = Y + W^{-1}( s * W Y ), orthonormal Haar
+// over aligned blocks of 2^J tokens, level gates s broadcast over each band.
+// By linearity this equals W^{-1}( (1 + s) * W Y ), which is what the kernel
+// evaluates: analysis, scale by 1 + s, synthesis, all in shared memory.
+#include "common.cuh"
+
+namespace spectre {
+
+template <typename WT> __device__ __forceinline__ float wl(const WT* p);
+template <> __device__ __forceinline__ float wl<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float wl<bf16>(const bf16* p) { return __bfloat162float(*p); }
+
+struct WaveletParams {
+  const void* src; void* dst;
+  int64_t s_sb, s_sl, s_sh, d_sb, d_sl, d_sh;
+  int B, L, H, D, J, rows, chunks;
+  const float* level_gates;       // [B,H,J+1,D] or NULL
+  const float* qbar; const void* Ww1; const float* bw1; const void* Ww2; const float* bw2;
+  int hidden; size_t hs_w1, hs_b1, hs_w2, hs_b2;
+};
+
+template <typename T, typename WT>
+__global__ void __launch_bounds__(256) wavelet_kernel(const WaveletParams p) {
+  extern __shared__ float smw[];
+  float* tile = smw;                               // [rows][D]
+  float* sg = tile + (size_t)p.rows * p.D;         // [(J+1)][D]  holds 1 + s
+  float* u = sg + (size_t)(p.J + 1) * p.D;         // [hidden]
+  const int chunk = blockIdx.x % p.chunks;
+  const int bh = blockIdx.x / p.chunks, b = bh / p.H, h = bh - b * p.H;
+  const int D = p.D, J = p.J;
+  const int r0 = chunk * p.rows;
+  const int nr = min(p.rows, p.L - r0);
+  // level gates (step b): given, or the two-layer MLP on q_bar
+  if (p.level_gates) {
+    for (int i = threadIdx.x; i < (J + 1) * D; i += blockDim.x) sg[i] = 1.0f + p.level_gates[(size_t)bh * (J + 1) * D + i];
+  } else {
+    const WT* W1 = reinterpret_cast<const WT*>(p.Ww1) + h * p.hs_w1;
+    const WT* W2 = reinterpret_cast<const WT*>(p.Ww2) + h * p.hs_w2;
+    const float* qb = p.qbar + (size_t)bh * D;
+    for (int j = threadIdx.x; j < p.hidden; j += blockDim.x) {
+      float acc = p.bw1[h * p.hs_b1 + j];
+      for (int c = 0; c < D; ++c) acc = fmaf(qb[c], wl<WT>(W1 + (size_t)c * p.hidden + j), acc);
+      u[j] = gelu_erf(acc);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < (J + 1) * D; i += blockDim.x) {
+      float acc = p.bw2[h * p.hs_b2 + i];
+      for (int j = 0; j < p.hidden; ++j) acc = fmaf(u[j], wl<WT>(W2 + (size_t)j * (J + 1) * D + i), acc);
+      sg[i] = 1.0f + acc;
+    }
+  }
+  // load the tile
+  const T* src = reinterpret_cast<const T*>(p.src) + b * p.s_sb + h * p.s_sh;
+  const int nv = D / 4;
+  for (int i = threadIdx.x; i < nr * nv; i += blockDim.x) {
+    int r = i / nv, c = (i - r * nv) * 4;
+    float4 v = io<T>::load4(src + (int64_t)(r0 + r) * p.s_sl + c);
+    *reinterpret_cast<float4*>(tile + (size_t)r * D + c) = v;
+  }
+  __syncthreads();
+  const float s = 0.70710678118654752440f;
+  // analysis, in place: after level l the slots i*2^l hold a_l, i*2^l + 2^(l-1) hold d_l
+  for (int l = 1; l <= J; ++l) {
+    const int span = 1 << l, hs = span >> 1;
+    const int nwork = (nr / span) * D;
+    for (int i = threadIdx.x; i < nwork; i += blockDim.x) {
+      int blk = i / D, c = i - blk * D;
+      float* x0 = tile + (size_t)(blk * span) * D + c;
+      float* x1 = x0 + (size_t)hs * D;
+      float a = *x0, d = *x1;
+      *x0 = (a + d) * s;
+      *x1 = (a - d) * s;
+    }
+    __syncthreads();
+  }
+  // modulate: slot p of a 2^J block is a_J (p = 0) or d_l with l = ctz(p) + 1
+  const int mask = (1 << J) - 1;
+  for (int i = threadIdx.x; i < nr * D; i += blockDim.x) {
+    int r = i / D, c = i - r * D;
+    int pos = r & mask;
+    int lev = pos == 0 ? 0 : 1 + (J - (__ffs(pos)));     // gate order a_J, d_J, ..., d_1
+    tile[i] *= sg[lev * D + c];
+  }
+  __syncthreads();
+  // synthesis
+  for (int l = J; l >= 1; --l) {
+    const int span = 1 << l, hs = span >> 1;
+    const int nwork = (nr / span) * D;
+    for (int i = threadIdx.x; i < nwork; i += blockDim.x) {
+      int blk = i / D, c = i - blk * D;
+      float* x0 = tile + (size_t)(blk * span) * D + c;
+      float* x1 = x0 + (size_t)hs * D;
+      float a = *x0, d = *x1;
+      *x0 = (a + d) * s;
+      *x1 = (a - d) * s;
+    }
+    __syncthreads();
+  }
+  T* dst = reinterpret_cast<T*>(p.dst) + b * p.d_sb + h * p.d_sh;
+  for (int i = threadIdx.x; i < nr * nv; i += blockDim.x) {
+    int r = i / nv, c = (i - r * nv) * 4;
+    io<T>::store4(dst + (int64_t)(r0 + r) * p.d_sl + c, *reinterpret_cast<float4*>(tile + (size_t)r * D + c));
+  }
+}
+
+}  // namespace spectre
+
+using namespace spectre;
+
+extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spectre_act* y_in, const spectre_act* y_out,
+                                      const spectre_wavelet* w) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  if (!w) return fail(SPECTRE_ERR_INVALID_ARG, "wavelet parameters are NULL");
+  int rc = check_act(y_in, "y_in");
+  if (rc != SPECTRE_OK) return rc;
+  rc = check_act(y_out, "y_out");
+  if (rc != SPECTRE_OK) return rc;
+  if (y_in->B != y_out->B || y_in->L != y_out->L || y_in->H != y_out->H || y_in->D != y_out->D ||
+      y_in->dtype != y_out->dtype)
+    return fail(SPECTRE_ERR_INVALID_ARG, "y_in and y_out differ in shape or dtype");
+  const int J = w->levels, L = y_in->L, D = y_in->D;
+  if (J < 1 || J > 10) return fail(SPECTRE_ERR_INVALID_ARG, "wavelet levels must be in 1..10");
+  if (L % (1 << J)) return fail(SPECTRE_ERR_INVALID_ARG, "2^J must divide L");
+  if (!w->level_gates) {
+    if (!w->qbar || !w->Ww1 || !w->bw1 || !w->Ww2 || !w->bw2)
+      return fail(SPECTRE_ERR_INVALID_ARG, "level_gates is NULL and the MLP inputs are incomplete");
+    if (w->hidden < 1 || w->hidden > 1024) return fail(SPECTRE_ERR_UNSUPPORTED, "wavelet hidden width must be in 1..1024");
+    if (w->wdtype != SPECTRE_F32 && w->wdtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, "unknown weight dtype");
+  }
+  const int span = 1 << J;
+  int rows = (8192 / D) / span * span;      // about 32 KB of fp32 per CTA
+  if (rows < span) rows = span;
+  if (rows > L) rows = L;
+  const int hidden = w->level_gates ? 0 : w->hidden;
+  size_t smem = ((size_t)rows * D + (size_t)(J + 1) * D + hidden) * sizeof(float);
+  if (smem > (size_t)ctx->max_smem_optin) return fail(SPECTRE_ERR_UNSUPPORTED, "2^J * D exceeds the shared-memory tile");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  WaveletParams p = {};
+  p.src = y_in->ptr; p.dst = y_out->ptr;
+  p.s_sb = y_in->stride_b; p.s_sl = y_in->stride_l; p.s_sh = y_in->stride_h;
+  p.d_sb = y_out->stride_b; p.d_sl = y_out->stride_l; p.d_sh = y_out->stride_h;
+  p.B = y_in->B; p.L = L; p.H = y_in->H; p.D = D; p.J = J; p.rows = rows; p.chunks = (L + rows - 1) / rows;
+  p.level_gates = w->level_gates; p.qbar = w->qbar; p.Ww1 = w->Ww1; p.bw1 = w->bw1; p.Ww2 = w->Ww2; p.bw2 = w->bw2;
+  p.hidden = hidden;
+  const size_t one = w->shared_across_heads ? 0 : 1;
+  p.hs_w1 = one * (size_t)D * hidden; p.hs_b1 = one * hidden;
+  p.hs_w2 = one * (size_t)hidden * (J + 1) * D; p.hs_b2 = one * (size_t)(J + 1) * D;
+  const unsigned grid = (unsigned)((size_t)p.B * p.H * p.chunks);
+  const bool bf = y_in->dtype == SPECTRE_BF16, wbf = w->wdtype == SPECTRE_BF16;
+#define SPECTRE_WAVELET_LAUNCH(T, WT)                                                                           \
+  do {                                                                                                          \
+    if (smem > 48 * 1024)                                                                                       \
+      SPECTRE_CUDA_OK(cudaFuncSetAttribute(wavelet_kernel<T, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
+                                           (int)smem));                                                         \
+    wavelet_kernel<T, WT><<<grid, 256, smem, st>>>(p);                                                          \
+  } while (0)
+  if (bf && wbf) SPECTRE_WAVELET_LAUNCH(bf16, bf16);
+  else if (bf) SPECTRE_WAVELET_LAUNCH(bf16, float);
+  else if (wbf) SPECTRE_WAVELET_LAUNCH(float, bf16);
+  else SPECTRE_WAVELET_LAUNCH(float, float);
+#undef SPECTRE_WAVELET_LAUNCH
+  SPECTRE_LAUNCH_OK("wavelet_kernel");
+  return SPECTRE_OK;
+}

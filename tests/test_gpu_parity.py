@@ -1,0 +1,331 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle on
+the same seeded inputs, element by element.  Tolerances: max relative L2 error
+per (batch, head) slab <= 1e-5 for fp32 I/O, <= 1e-2 for bf16 I/O."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spectre_oracle as O
+from paper_2502_18394_b200 import binding as S
+from paper_2502_18394_b200 import workloads as W
+from util import TOL, gate_params_np, gate_to_complex, rel_err, slab_err, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = S.Context(0)
+    yield c
+    c.close()
+
+
+def run_mixer(ctx, w, structured=False, n_fft=None):
+    x = W.activations(w, structured=structured)
+    g = W.random_gate(w)
+    y = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=n_fft)
+    torch.cuda.synchronize()
+    ref = O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=n_fft)
+    return slab_err(W.to_f64(y), ref)
+
+
+# lengths: single CTA (<= 2048, all radices), 2- and 4-CTA clusters, four-step
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 7, 8, 12, 16, 30, 49, 64, 128, 196, 256, 512, 1000, 1024, 2048])
+def test_mixer_f32_single_cta(ctx, n):
+    w = W.Workload("t", B=2, L=n, H=3, D=16, dtype="f32", seed=100 + n)
+    assert run_mixer(ctx, w) < TOL["f32"]
+
+
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_mixer_f32_cluster(ctx, n):
+    w = W.Workload("t", B=1, L=n, H=2, D=32, dtype="f32", seed=n)
+    assert run_mixer(ctx, w) < TOL["f32"]
+
+
+@pytest.mark.parametrize("n", [16384, 32768, 131072])
+def test_mixer_f32_four_step(ctx, n):
+    w = W.Workload("t", B=1, L=n, H=2, D=16, dtype="f32", seed=n)
+    assert run_mixer(ctx, w) < TOL["f32"]
+
+
+@pytest.mark.parametrize("n,D", [(196, 64), (1024, 64), (8192, 64), (65536, 16), (2048, 8), (512, 24), (8192, 40)])
+def test_mixer_bf16(ctx, n, D):
+    w = W.Workload("t", B=2, L=n, H=2, D=D, dtype="bf16", seed=7 * n + D)
+    assert run_mixer(ctx, w) < TOL["bf16"]
+
+
+def test_mixer_structured_inputs(ctx):
+    # per-channel offsets and x30 outlier channels
+    for dt in ("f32", "bf16"):
+        w = W.Workload("t", B=1, L=2048, H=2, D=32, dtype=dt, seed=5)
+        assert run_mixer(ctx, w, structured=True) < TOL[dt]
+
+
+@pytest.mark.parametrize("L,n", [(100, 128), (196, 256), (3000, 4096), (5000, 8192), (20000, 32768)])
+def test_mixer_zero_pad_variant(ctx, L, n):
+    w = W.Workload("t", B=1, L=L, H=2, D=16, dtype="f32", n_fft=n, seed=L)
+    assert run_mixer(ctx, w, n_fft=n) < TOL["f32"]
+
+
+def test_mixer_strided_views_and_in_place(ctx):
+    w = W.Workload("t", B=2, L=256, H=4, D=16, dtype="f32", seed=9)
+    big = W.activations(W.scaled(w, H=8)).cuda()
+    x = big[:, :, 2:6, :]                                  # non-contiguous head slice
+    g = W.random_gate(w).cuda()
+    y = torch.zeros_like(big)
+    S.spectre_mixer_forward(ctx, x, g, y=y[:, :, 1:5, :])
+    ref = O.mixer(W.to_f64(x), gate_to_complex(g))
+    assert slab_err(W.to_f64(y[:, :, 1:5, :]), ref) < TOL["f32"]
+    assert float(y[:, :, 0].abs().max()) == 0.0 and float(y[:, :, 5:].abs().max()) == 0.0
+    xc = x.contiguous()
+    S.spectre_mixer_forward(ctx, xc, g, y=xc)              # in place on the single-pass path
+    assert slab_err(W.to_f64(xc), ref) < TOL["f32"]
+
+
+def test_mixer_special_inputs(ctx):
+    n, H, D = 1024, 1, 16
+    K = n // 2 + 1
+    g = W.random_gate(W.Workload("t", B=1, L=n, H=H, D=D, seed=3))
+    x = torch.zeros(1, n, H, D)
+    x[0, 0, 0, 3] = 1.0                      # impulse -> kernel irfft(g) in that column only
+    x[0, :, 0, 4] = 1.0                      # constant -> only bin 0
+    x[0, :, 0, 5] = torch.tensor([(-1.0) ** t for t in range(n)])   # alternating -> only bin n/2
+    y = W.to_f64(S.spectre_mixer_forward(ctx, x.cuda(), g.cuda()))
+    gc = gate_to_complex(g)[0, 0]
+    assert rel_err(y[0, :, 0, 3], O.irfft(gc, n)) < 1e-5
+    assert np.allclose(y[0, :, 0, 4], gc[0].real, atol=1e-5)
+    assert np.allclose(y[0, :, 0, 5], gc[K - 1].real * W.to_f64(x)[0, :, 0, 5], atol=1e-5)
+    assert np.abs(y[0, :, 0, 6:]).max() == 0.0
+    ones = torch.zeros(1, H, K, 2); ones[..., 0] = 1.0
+    xr = W.activations(W.Workload("t", B=1, L=n, H=H, D=D, dtype="f32", seed=4))
+    yi = S.spectre_mixer_forward(ctx, xr.cuda(), ones.cuda())
+    assert slab_err(W.to_f64(yi), W.to_f64(xr)) < 1e-6        # all-ones gate returns the input
+
+
+def run_gate(ctx, w, **kw):
+    x = W.activations(w)
+    p = W.gate_params(w, **{k: v for k, v in kw.items() if k in ("modrelu_bias_std", "toeplitz_r", "bias_std")})
+    shift = kw.get("shift")
+    sh_dev = None if shift is None else torch.tensor(shift, dtype=torch.int64).cuda()
+    qbar = torch.empty(w.B, w.H, w.D, device="cuda")
+    g = S.spectre_gate(ctx, to_dev(p), w.n, q=x.cuda(), shift=sh_dev, shift_all=kw.get("shift_all", 0), qbar_out=qbar)
+    pn = gate_params_np(p)
+    total_shift = None
+    if shift is not None or kw.get("shift_all", 0):
+        total_shift = np.array(shift if shift is not None else [0] * w.B) + kw.get("shift_all", 0)
+    sum_q = W.to_f64(x).sum(axis=1)
+    gref, qref = O.gate(sum_q, 1.0 / w.L, w.n, shift=total_shift, return_qbar=True, **pn)
+    return rel_err(gate_to_complex(g), gref), rel_err(W.to_f64(qbar), qref), g, p, x
+
+
+def test_gate_c1(ctx):
+    eg, eq, *_ = run_gate(ctx, W.CONFIGS["c1"])
+    assert eg < 1e-5 and eq < 1e-5
+
+
+def test_gate_bf16_weights_full_options(ctx):
+    w = W.Workload("t", B=3, L=777, H=4, D=64, dtype="bf16", wdtype="bf16", n_fft=1024, seed=11)
+    eg, eq, *_ = run_gate(ctx, w, modrelu_bias_std=0.05, toeplitz_r=2, bias_std=0.1, shift=[5, 0, 1030], shift_all=7)
+    assert eg < 1e-4 and eq < 1e-4
+    w = W.Workload("t", B=2, L=196, H=3, D=64, dtype="bf16", wdtype="f32", seed=12)
+    eg, eq, *_ = run_gate(ctx, w, modrelu_bias_std=0.05, bias_std=0.1, shift=[3, 100])
+    assert eg < 1e-4 and eq < 1e-4
+
+
+def test_gate_from_running_sum_and_shared_heads(ctx):
+    w = W.Workload("t", B=2, L=64, H=4, D=32, dtype="f32", wdtype="f32", n_fft=64, seed=13)
+    p = W.gate_params(w)
+    sum_q = torch.randn(w.B, w.H, w.D, generator=torch.Generator().manual_seed(1)) * 9
+    g = S.spectre_gate(ctx, to_dev(p), w.n, sum_q=sum_q.cuda(), inv_count=1.0 / 64, shift_all=70)
+    gref = O.gate(W.to_f64(sum_q), 1.0 / 64, w.n, shift=np.array([70, 70]), **gate_params_np(p))
+    assert rel_err(gate_to_complex(g), gref) < 1e-5
+    shared = {k: (v[:1].contiguous() if isinstance(v, torch.Tensor) else v) for k, v in p.items()}
+    shared["shared_across_heads"] = 1
+    g = S.spectre_gate(ctx, to_dev(shared), w.n, sum_q=sum_q.cuda(), inv_count=1.0 / 64)
+    pn = gate_params_np(p)
+    pn = {k: (np.repeat(v[:1], w.H, axis=0) if isinstance(v, np.ndarray) else v) for k, v in pn.items()}
+    assert rel_err(gate_to_complex(g), O.gate(W.to_f64(sum_q), 1.0 / 64, w.n, **pn)) < 1e-5
+
+
+def test_c1_end_to_end(ctx):
+    w = W.CONFIGS["c1"]
+    x = W.activations(w)
+    p = W.gate_params(w)
+    xd = x.cuda()
+    g = S.spectre_gate(ctx, to_dev(p), w.n, q=xd)
+    y = S.spectre_mixer_forward(ctx, xd, g)
+    gref = O.gate(W.to_f64(x).sum(axis=1), 1.0 / w.L, w.n, **gate_params_np(p))
+    ref = O.mixer(W.to_f64(x), gref)
+    assert slab_err(W.to_f64(y), ref) < TOL["f32"]
+
+
+def test_c2_reduced_heads_end_to_end(ctx):
+    w = W.scaled(W.CONFIGS["c2"], H=4)
+    x = W.activations(w)
+    p = W.gate_params(w)
+    xd = x.cuda()
+    g = S.spectre_gate(ctx, to_dev(p), w.n, q=xd)
+    y = S.spectre_mixer_forward(ctx, xd, g)
+    gref = O.gate(W.to_f64(x).sum(axis=1), 1.0 / w.L, w.n, **gate_params_np(p))
+    assert rel_err(gate_to_complex(g), gref) < 1e-4
+    assert slab_err(W.to_f64(y), O.mixer(W.to_f64(x), gref)) < TOL["bf16"]
+
+
+# ------------------------------------------------------------------ wavelet
+@pytest.mark.parametrize("dt,L,J,D", [("f32", 196, 2, 64), ("bf16", 196, 2, 64), ("f32", 64, 4, 16), ("f32", 1024, 1, 8),
+                                     ("bf16", 4096, 3, 64)])
+def test_wavelet_refine(ctx, dt, L, J, D):
+    w = W.Workload("t", B=2, L=L, H=3, D=D, dtype=dt, wdtype="f32", seed=L + J, wavelet_levels=J)
+    y = W.activations(w)
+    gates = torch.randn(w.B, w.H, J + 1, D, generator=torch.Generator().manual_seed(2))
+    out = S.spectre_wavelet_refine(ctx, y.cuda(), {"levels": J, "level_gates": gates.cuda()})
+    ref = O.wavelet_refine(W.to_f64(y), W.to_f64(gates), J)
+    assert slab_err(W.to_f64(out), ref) < TOL[dt]
+    # gates from q_bar through the MLP, in place
+    wp = W.wavelet_params(w)
+    qbar = torch.randn(w.B, w.H, D, generator=torch.Generator().manual_seed(3))
+    yd = y.cuda()
+    S.spectre_wavelet_refine(ctx, yd, dict(to_dev(wp), qbar=qbar.cuda()), y_out=yd)
+    s = O.wavelet_level_gates(W.to_f64(qbar), W.to_f64(wp["Ww1"]), W.to_f64(wp["bw1"]), W.to_f64(wp["Ww2"]),
+                              W.to_f64(wp["bw2"]), J)
+    assert slab_err(W.to_f64(yd), O.wavelet_refine(W.to_f64(y), s, J)) < TOL[dt]
+
+
+def test_c5_reduced_batch_with_wavelet(ctx):
+    w = W.scaled(W.CONFIGS["c5"], B=4)
+    x = W.activations(w)
+    p, wp = W.gate_params(w), W.wavelet_params(w)
+    xd = x.cuda()
+    qbar = torch.empty(w.B, w.H, w.D, device="cuda")
+    g = S.spectre_gate(ctx, to_dev(p), w.n, q=xd, qbar_out=qbar)
+    y = S.spectre_mixer_forward(ctx, xd, g, wrm=dict(to_dev(wp), qbar=qbar))
+    x64 = W.to_f64(x)
+    gref, qref = O.gate(x64.sum(axis=1), 1.0 / w.L, w.n, return_qbar=True, **gate_params_np(p))
+    s = O.wavelet_level_gates(qref, W.to_f64(wp["Ww1"]), W.to_f64(wp["bw1"]), W.to_f64(wp["Ww2"]), W.to_f64(wp["bw2"]), 2)
+    ref = O.wavelet_refine(O.mixer(x64, gref), s, 2)
+    assert slab_err(W.to_f64(y), ref) < TOL["bf16"]
+
+
+# ------------------------------------------------------------------ cache
+def cache_err(cache, st):
+    P = W.to_f64(cache.prefix_fft)
+    P = P[..., 0] + 1j * P[..., 1]                          # [B,H,K,D]
+    num = np.sqrt((np.abs(P - st["prefix_fft"]) ** 2).sum(axis=(2, 3)))
+    den = np.sqrt((np.abs(st["prefix_fft"]) ** 2).sum(axis=(2, 3)))
+    e_p = float((num / np.where(den > 0, den, 1)).max())
+    e_s = rel_err(W.to_f64(cache.sum_q), st["sum_q"])
+    return e_p, e_s
+
+
+@pytest.mark.parametrize("dt,N,L,steps", [("f32", 64, 20, 150), ("bf16", 256, 256, 300), ("f32", 4096, 1000, 40),
+                                         ("bf16", 16384, 16000, 500)])
+def test_cache_prefill_and_append(ctx, dt, N, L, steps):
+    w = W.Workload("t", B=2, L=L, H=2, D=16, dtype=dt, seed=N + L, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    cache = S.PrefixCache(w.B, w.H, w.D, N, dtype=W.torch_dtype(dt))
+    cache.V_buf.fill_(7.0); cache.Q_buf.fill_(7.0)          # prefill must zero the tail itself
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    st = O.cache_prefill(W.to_f64(q), W.to_f64(v), N)
+    tol = 1e-5 if dt == "f32" else 1e-5                     # spectrum is fp32 for both dtypes
+    e_p, e_s = cache_err(cache, st)
+    assert e_p < tol and e_s < tol
+    assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
+    qs, vs = W.decode_tokens(w, steps)
+    qd, vd = qs.cuda(), vs.cuda()
+    for i in range(steps):
+        t = L + i
+        S.spectre_prefix_cache_append(ctx, cache, qd[i], vd[i], t)
+        O.cache_append(st, t, W.to_f64(qs[i]), W.to_f64(vs[i]))
+        if (i + 1) % 50 == 0 or i == steps - 1:
+            e_p, e_s = cache_err(cache, st)
+            assert e_p < 2e-5 and e_s < 2e-5, (i, e_p, e_s)
+            ref = O.cache_recompute(st)                      # cached prefix == full recompute
+            P = W.to_f64(cache.prefix_fft); P = P[..., 0] + 1j * P[..., 1]
+            assert rel_err(P, ref["prefix_fft"]) < 2e-5
+    assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
+
+
+def test_cache_non_power_of_two_window_append(ctx):
+    # append works for any window length; prefill the state by hand (zeros)
+    N = 100
+    w = W.Workload("t", B=1, L=1, H=2, D=8, dtype="f32", seed=1, N_max=N)
+    cache = S.PrefixCache(1, 2, 8, N, dtype=torch.float32)
+    st = O.cache_prefill(np.zeros((1, 1, 2, 8)), np.zeros((1, 1, 2, 8)), N)
+    qs, vs = W.decode_tokens(w, 250)
+    for i in range(250):
+        S.spectre_prefix_cache_append(ctx, cache, qs[i].cuda(), vs[i].cuda(), 1 + i)
+        O.cache_append(st, 1 + i, W.to_f64(qs[i]), W.to_f64(vs[i]))
+    e_p, e_s = cache_err(cache, st)
+    assert e_p < 2e-5 and e_s < 2e-5
+
+
+def test_cache_snapshot_restore_is_bit_exact(ctx):
+    N, L = 128, 100
+    w = W.Workload("t", B=1, L=L, H=2, D=16, dtype="bf16", seed=77, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    qs, vs = W.decode_tokens(w, 80)
+    def run(snapshot_at=None):
+        cache = S.PrefixCache(1, 2, 16, N)
+        S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+        for i in range(80):
+            if snapshot_at == i:
+                saved = [t.clone() for t in (cache.prefix_fft, cache.V_buf, cache.Q_buf, cache.sum_q)]
+                cache = S.PrefixCache(1, 2, 16, N)
+                for dst, src in zip((cache.prefix_fft, cache.V_buf, cache.Q_buf, cache.sum_q), saved):
+                    dst.copy_(src)
+            S.spectre_prefix_cache_append(ctx, cache, qs[i].cuda(), vs[i].cuda(), L + i)
+        return cache
+    a, b = run(), run(snapshot_at=40)
+    assert torch.equal(a.prefix_fft, b.prefix_fft) and torch.equal(a.sum_q, b.sum_q) and torch.equal(a.V_buf, b.V_buf)
+
+
+def test_decode_step_equals_full_recompute(ctx):
+    # Sec. 3.3.2 (c)-(e): gate from sum_q / N_max with phase t applied to the cached
+    # spectrum equals the mixer on the ring buffer rotated by t.
+    N, L = 256, 200
+    w = W.Workload("t", B=2, L=L, H=2, D=16, dtype="bf16", wdtype="f32", n_fft=N, seed=21, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    p = W.gate_params(w)
+    cache = S.PrefixCache(w.B, w.H, w.D, N)
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    qs, vs = W.decode_tokens(w, 130)
+    for i in range(130):
+        S.spectre_prefix_cache_append(ctx, cache, qs[i].cuda(), vs[i].cuda(), L + i)
+    t = L + 129
+    g = S.spectre_gate(ctx, to_dev(p), N, sum_q=cache.sum_q, inv_count=1.0 / N, shift_all=t)
+    y = S.spectre_mixer_forward(ctx, cache.V_buf, g)        # full recompute on the ring buffer, same gate
+    st = {"prefix_fft": None, "N": N}
+    P = W.to_f64(cache.prefix_fft); st["prefix_fft"] = P[..., 0] + 1j * P[..., 1]
+    out = O.decode_readout(st, gate_to_complex(g))          # inverse of the cached spectrum
+    assert slab_err(W.to_f64(y), out) < TOL["bf16"]
+
+
+# ------------------------------------------------------------------ errors
+def test_invalid_arguments_are_rejected_before_launch(ctx):
+    x = torch.zeros(1, 64, 2, 16, device="cuda")
+    g = torch.zeros(1, 2, 33, 2, device="cuda")
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_mixer_forward(ctx, x, g, n_fft=32)          # n_fft < L
+    assert e.value.status == S.SPECTRE_ERR_INVALID_ARG
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_mixer_forward(ctx, x[:, :62], g[:, :, :32], n_fft=62)   # 62 = 2 * 31: unsupported prime
+    assert e.value.status == S.SPECTRE_ERR_UNSUPPORTED
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_mixer_forward(ctx, torch.zeros(1, 64, 2, 12, device="cuda"), g)   # D % 8
+    assert e.value.status == S.SPECTRE_ERR_UNSUPPORTED
+    big = torch.zeros(1, 16384, 1, 16, device="cuda")
+    gb = torch.zeros(1, 1, 8193, 2, device="cuda")
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_mixer_forward(ctx, big, gb, workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == S.SPECTRE_ERR_WORKSPACE
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_mixer_forward(ctx, big, gb, y=big)          # aliasing on the multi-pass path
+    assert e.value.status == S.SPECTRE_ERR_INVALID_ARG
+    cache = S.PrefixCache(1, 2, 16, 32, dtype=torch.float32)
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_prefix_cache_prefill(ctx, cache, x, x)      # L = 64 > N_max = 32
+    assert e.value.status == S.SPECTRE_ERR_INVALID_ARG
+    with pytest.raises(S.SpectreError):
+        S.spectre_wavelet_refine(ctx, x[:, :62].contiguous(), {"levels": 2, "level_gates": torch.zeros(1, 2, 3, 16, device="cuda")})
+    torch.cuda.synchronize()                                   # context still healthy
+    assert float(S.spectre_mixer_forward(ctx, x, g).abs().max()) == 0.0
