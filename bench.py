@@ -1,0 +1,433 @@
+#!/usr/bin/env python
+"""Benchmark of the SPECTRE spectral-mixer hot path on B200.
+
+A "step" is one pass of the hot path over one batch of synthetic input: the gate
+(pool + LayerNorm + MLP + modReLU) followed by the mixer (rFFT -> gate -> irFFT)
+for the mixer workloads, one cache append for the decode workload.  Inputs are
+resident in HBM when the timed region starts; `e2e` repeats the measurement with
+host buffers and the copies inside the timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c1]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores
+
+The path does not shard (every (batch, head) slab is independent, no exchange step):
+--gpus N runs N independent replicas, one process per GPU, no data-path collective.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2502_18394_b200 import replicas as R  # noqa: E402
+from paper_2502_18394_b200 import workloads as W  # noqa: E402
+
+METRIC = "mixer tokens/s and achieved HBM GB/s (% of B200 peak) at L=8k and 128k, 1 GPU"
+L2_BYTES = 126e6
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None until a capture exists for that workload).
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": None, "c3": None, "c4": None, "c5": None}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+               0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period: float = 0.004):
+        self.samples, self.reasons, self.ok, self.max_mhz = [], set(), False, None
+        self._stop = threading.Event()
+        self._period = period
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if vis:
+                try:
+                    phys = int(vis.split(",")[index])
+                except ValueError:
+                    phys = index
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+        self._thr = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def start(self):
+        if self.ok:
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self.ok and self._thr.is_alive():
+            self._thr.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- workloads
+def describe(w: W.Workload) -> str:
+    if w.N_max:
+        return (f"{w.name}: Prefix-FFT cache append, B={w.B} H={w.H} d={w.D} N_max={w.N_max}, "
+                f"{w.dtype} tokens, fp32 spectrum")
+    s = f"{w.name}: gate + mixer, B={w.B} H={w.H} d={w.D} L={w.L}, {w.dtype} I/O, fp32 accumulate"
+    if w.wavelet_levels:
+        s += f", Haar J={w.wavelet_levels}"
+    return s
+
+
+def mixer_algorithmic_bytes(w: W.Workload) -> int:
+    es = 2 if w.dtype == "bf16" else 4
+    return 2 * w.B * w.L * w.H * w.D * es + w.B * w.H * w.K * 8          # read V, write Y, read g
+
+
+def append_algorithmic_bytes(w: W.Workload) -> int:
+    K = w.N_max // 2 + 1
+    return 2 * w.B * w.H * K * w.D * 8                                    # read + write the spectrum
+
+
+class MixerBench:
+    """gate + mixer (+ wavelet) over rotating buffer sets."""
+
+    def __init__(self, w: W.Workload, dev, nsets: int | None):
+        from paper_2502_18394_b200 import binding as S
+        self.S, self.w, self.dev = S, w, dev
+        self.ctx = S.Context(dev.index)
+        per_set = 2 * w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
+        if nsets is None:
+            nsets = 1 if per_set > 2 * L2_BYTES else max(2, int(4 * L2_BYTES / per_set) + 1)
+        self.nsets = nsets
+        self.x_host = [W.activations(w, stream=i) for i in range(nsets)]
+        params = W.gate_params(w)
+        self.sets = []
+        ws_gate = S.spectre_gate_workspace_bytes(self.ctx, w.B, w.H, w.D, w.n, 0)
+        ws_mix = S.spectre_mixer_workspace_bytes(self.ctx, w.B, w.L, w.H, w.D, w.n, S.SPECTRE_BF16 if w.dtype == "bf16" else S.SPECTRE_F32)
+        self.ws_mix = torch.empty(max(ws_mix, 16), dtype=torch.uint8, device=dev) if ws_mix else None
+        wp = W.wavelet_params(w) if w.wavelet_levels else None
+        for i in range(nsets):
+            d = {"x": self.x_host[i].to(dev), "y": torch.empty((w.B, w.L, w.H, w.D), dtype=W.torch_dtype(w.dtype), device=dev),
+                 "g": torch.empty((w.B, w.H, w.K, 2), dtype=torch.float32, device=dev),
+                 "qbar": torch.empty((w.B, w.H, w.D), dtype=torch.float32, device=dev),
+                 "wsg": torch.empty(max(ws_gate, 16), dtype=torch.uint8, device=dev),
+                 # each set has its own copy of the weights, as each layer of a model would
+                 "p": {k: (v.to(dev).clone() if isinstance(v, torch.Tensor) else v) for k, v in params.items()}}
+            wrm = None
+            if wp is not None:
+                wrm = {k: (v.to(dev).clone() if isinstance(v, torch.Tensor) else v) for k, v in wp.items()}
+                wrm["qbar"] = d["qbar"]
+            d["gate"] = S.prepare_gate(self.ctx, d["p"], w.n, d["x"], d["g"], d["wsg"], qbar_out=d["qbar"])
+            d["mix"] = S.prepare_mixer_forward(self.ctx, d["x"], d["g"], d["y"], n_fft=w.n, wrm=wrm, workspace=self.ws_mix)
+            self.sets.append(d)
+        self.units_per_step = w.B * w.L                                  # tokens
+        self.alg_bytes = mixer_algorithmic_bytes(w)
+        self.kernel_name = "mixer (onchip_kernel)" if ws_mix == 0 else "mixer (strided + onchip + strided, per group)"
+        # kernels per step: pool, gate_mlp, mixer kernel(s), wavelet
+        import math
+        groups = 1
+        nk = 1
+        if ws_mix:
+            per = w.n * (w.D // 2) * 8
+            groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
+            nk = 3 * groups
+        self.launches_per_step = 2 + nk + (1 if w.wavelet_levels else 0)
+        self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
+        self.d2h = self.h2d
+
+    def step(self, k: int, e0=None, e1=None):
+        d = self.sets[k % self.nsets]
+        d["gate"]()
+        if e0 is not None:
+            e0.record()
+        d["mix"]()
+        if e1 is not None:
+            e1.record()
+
+    def e2e_prepare(self):
+        self.pin_x = [x.pin_memory() for x in self.x_host[:2]]
+        self.pin_y = torch.empty_like(self.pin_x[0]).pin_memory()
+
+    def e2e_step(self, k: int):
+        d = self.sets[k % self.nsets]
+        d["x"].copy_(self.pin_x[k % len(self.pin_x)], non_blocking=True)
+        d["gate"]()
+        d["mix"]()
+        self.pin_y.copy_(d["y"], non_blocking=True)
+
+    def cpu_step(self):
+        from oracle import spectre_oracle as O
+        w = self.w
+        x = W.to_f64(self.x_host[0])
+        p = W.gate_params(w)
+        pn = dict(ln_gamma=W.to_f64(p["ln_gamma"]), ln_beta=W.to_f64(p["ln_beta"]), ln_eps=p["ln_eps"],
+                  W1=W.to_f64(p["W1"]), b1=W.to_f64(p["b1"]), W2=W.to_f64(p["W2"]), b2=W.to_f64(p["b2"]))
+        t0 = time.perf_counter()
+        g, qbar = O.gate(x.sum(axis=1), 1.0 / w.L, w.n, return_qbar=True, **pn)
+        y = O.mixer(x, g, n_fft=w.n)
+        if w.wavelet_levels:
+            wp = W.wavelet_params(w)
+            s = O.wavelet_level_gates(qbar, W.to_f64(wp["Ww1"]), W.to_f64(wp["bw1"]), W.to_f64(wp["Ww2"]),
+                                      W.to_f64(wp["bw2"]), w.wavelet_levels)
+            y = O.wavelet_refine(y, s, w.wavelet_levels)
+        return time.perf_counter() - t0, w.B * w.L
+
+
+class AppendBench:
+    """One Prefix-FFT cache append per step (decode)."""
+
+    def __init__(self, w: W.Workload, dev, nsets=None):
+        from paper_2502_18394_b200 import binding as S
+        self.S, self.w, self.dev = S, w, dev
+        self.ctx = S.Context(dev.index)
+        self.cache = S.PrefixCache(w.B, w.H, w.D, w.N_max, dtype=W.torch_dtype(w.dtype), device=dev)
+        # state: a full window of random tokens (prefill through the library)
+        half = W.scaled(w, B=1)
+        ws = torch.empty(max(S.spectre_prefill_workspace_bytes(self.ctx, w.B, w.H, w.D, w.N_max), 16), dtype=torch.uint8, device=dev)
+        q = torch.cat([W.activations(half, stream=10 + b) for b in range(w.B)], dim=0).to(dev)
+        S.spectre_prefix_cache_prefill(self.ctx, self.cache, q, q, workspace=ws)
+        del ws, q
+        self.nsets = 1
+        qs, vs = W.decode_tokens(w, 64)
+        self.q_host, self.v_host = qs, vs
+        self.qd, self.vd = qs.to(dev), vs.to(dev)
+        self.t0 = w.L
+        self.units_per_step = w.B                                         # tokens appended
+        self.alg_bytes = append_algorithmic_bytes(w)
+        self.kernel_name = "append_spectrum_kernel"
+        self.launches_per_step = 2
+        es = 2 if w.dtype == "bf16" else 4
+        self.h2d = 2 * w.B * w.H * w.D * es
+        self.d2h = w.B * w.H * w.D * 4
+
+    def _call(self, k):
+        i = k % 64
+        return self.S.prepare_append(self.ctx, self.cache, self.qd[i], self.vd[i], self.t0 + k)
+
+    def step(self, k: int, e0=None, e1=None):
+        c = self._call(k)
+        if e0 is not None:
+            e0.record()
+        c()
+        if e1 is not None:
+            e1.record()
+
+    def e2e_prepare(self):
+        self.pin_q = self.q_host.pin_memory()
+        self.pin_v = self.v_host.pin_memory()
+        self.pin_s = torch.empty((self.w.B, self.w.H, self.w.D), dtype=torch.float32).pin_memory()
+
+    def e2e_step(self, k: int):
+        i = k % 64
+        self.qd[i].copy_(self.pin_q[i], non_blocking=True)
+        self.vd[i].copy_(self.pin_v[i], non_blocking=True)
+        self._call(100000 + k)()
+        self.pin_s.copy_(self.cache.sum_q, non_blocking=True)
+
+    def cpu_step(self):
+        # bounded sample: one (batch) row of the cache, all heads; scaled to tokens/s
+        from oracle import spectre_oracle as O
+        import numpy as np
+        w = self.w
+        rng = np.random.default_rng(0)
+        N, K = w.N_max, w.N_max // 2 + 1
+        st = {"N": N, "prefix_fft": np.zeros((1, w.H, K, w.D), dtype=np.complex128),
+              "V_buf": rng.standard_normal((1, N, w.H, w.D)), "Q_buf": rng.standard_normal((1, N, w.H, w.D)),
+              "sum_q": np.zeros((1, w.H, w.D))}
+        q = W.to_f64(self.q_host[0][:1]); v = W.to_f64(self.v_host[0][:1])
+        t0 = time.perf_counter()
+        O.cache_append(st, N + 5, q, v)
+        return time.perf_counter() - t0, 1
+
+
+def make_bench(w, dev, nsets):
+    return AppendBench(w, dev, nsets) if w.N_max else MixerBench(w, dev, nsets)
+
+
+# --------------------------------------------------------------------------- arms
+def run_reference(args, w):
+    """The oracle, as it stands, on the host cores; rank 0 only."""
+    rank, _, ws = R.world()
+    if rank != 0:
+        return
+    torch.set_num_threads(1)
+    bench = _cpu_only_bench(w)
+    for _ in range(min(args.warmup, 1)):
+        bench.cpu_step()
+    tot, units = 0.0, 0
+    for _ in range(args.steps):
+        dt, u = bench.cpu_step()
+        tot += dt
+        units += u
+    val = units / tot
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": describe(w)},
+           "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                            "sample": bench.sample_note},
+           "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def _cpu_only_bench(w):
+    """A bench object whose GPU side is never built (the reference arm runs without the library)."""
+    cls = AppendBench if w.N_max else MixerBench
+    b = cls.__new__(cls)
+    b.w = w
+    if w.N_max:
+        qs, vs = W.decode_tokens(w, 1)
+        b.q_host, b.v_host = qs, vs
+        b.sample_note = "one batch row (all heads) of one append, scaled to tokens/s"
+    else:
+        b.x_host = [W.activations(w, stream=0)]
+        b.sample_note = "the full workload, once per step" if w.L * w.B * w.H <= (1 << 20) * 4 else \
+            "the full workload, once per step (numpy FFT, single thread)"
+    return b
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--sets", type=int, default=None, help="rotating buffer sets (default: enough to exceed L2)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = W.CONFIGS[args.workload]
+    rank, local_rank, world = R.world()
+
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 3
+        args.warmup = args.warmup if args.warmup is not None else 1
+        if w.name == "c3" and args.steps > 2:
+            args.steps = 2
+        run_reference(args, w)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    default_steps = {"c1": 2000, "c2": 2000, "c3": 100, "c4": 200, "c5": 500}[w.name]
+    K = args.steps if args.steps is not None else default_steps
+    Wm = max(3, args.warmup if args.warmup is not None else 10)
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    R.init()
+    bench = make_bench(w, dev, args.sets)
+
+    for k in range(Wm):
+        bench.step(k)
+    torch.cuda.synchronize()
+
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    R.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev_a.record()
+    for k in range(K):
+        bench.step(Wm + k, e0[k], e1[k])
+    ev_b.record()
+    torch.cuda.synchronize()
+    R.barrier()
+    clocks = sampler.stop()
+    elapsed_ms = ev_a.elapsed_time(ev_b)
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(e0, e1))
+    tot_ms, tot_units = R.aggregate(elapsed_ms, bench.units_per_step * K, dev)
+
+    # end to end: host buffers, copies inside the timed region
+    Ke = max(3, min(K, 30))
+    bench.e2e_prepare()
+    for k in range(3):
+        bench.e2e_step(k)
+    torch.cuda.synchronize()
+    R.barrier()
+    ev_a.record()
+    for k in range(Ke):
+        bench.e2e_step(3 + k)
+    ev_b.record()
+    torch.cuda.synchronize()
+    R.barrier()
+    e2e_ms, e2e_units = R.aggregate(ev_a.elapsed_time(ev_b), bench.units_per_step * Ke, dev)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        torch.set_num_threads(1)
+        reps = 1 if w.name in ("c3",) else 3
+        tot, units = 0.0, 0
+        for _ in range(reps):
+            dt, u = bench.cpu_step()
+            tot += dt
+            units += u
+        note = _cpu_only_bench(w).sample_note + f", {reps} repetition(s)"
+        cpu = {"value": units / tot, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": note}
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        achieved = bench.alg_bytes / (kern_ms * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+                       "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
+                       "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
+                             if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": bench.h2d,
+                    "d2h_bytes_per_step": bench.d2h, "steps": Ke},
+            "gpu_launches": bench.launches_per_step * K,
+            "roofline": {"bound": "hbm", "kernel": bench.kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": bench.alg_bytes,
+                         "kernel_ms": kern_ms, "frac_of_8000": achieved / 8000.0,
+                         "kernel_tokens_per_s": bench.units_per_step / (kern_ms * 1e-3),
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(out))
+    R.finish()
+
+
+if __name__ == "__main__":
+    main()

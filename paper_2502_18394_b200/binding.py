@@ -280,3 +280,49 @@ def spectre_prefix_cache_append(ctx: Context, cache: PrefixCache, q_t: torch.Ten
         raise ValueError("q_t and v_t must be contiguous [B, H, D]")
     cs = cache.struct()
     _check(lib().spectre_prefix_cache_append(ctx.handle, _stream(stream), C.byref(cs), _ptr(q_t), _ptr(v_t), int(t)))
+
+
+# ---- pre-marshalled calls ---------------------------------------------------------------
+# A launch loop that rebuilds ctypes structures every step spends more host time than the
+# kernels take.  These objects marshal once and replay the identical C call.
+class PreparedCall:
+    def __init__(self, fn, args, keep):
+        self._fn, self._args, self._keep = fn, args, keep
+
+    def __call__(self):
+        st = self._fn(*self._args)
+        if st != SPECTRE_OK:
+            _check(st)
+
+
+def prepare_gate(ctx: Context, params: dict, n_fft: int, q: torch.Tensor, g_out: torch.Tensor,
+                 workspace: torch.Tensor, qbar_out: torch.Tensor | None = None, shift_all: int = 0,
+                 stream=None) -> PreparedCall:
+    B, _, H, D = q.shape
+    keep: list = [q, g_out, workspace, qbar_out]
+    gp = _gate_struct(params, keep)
+    a = act(q)
+    keep += [gp, a]
+    args = (ctx.handle, _stream(stream), C.byref(a), None, B, H, D, C.c_float(0.0), C.byref(gp), n_fft, None,
+            int(shift_all), _ptr(g_out), _ptr(qbar_out), _ptr(workspace), workspace.numel())
+    return PreparedCall(lib().spectre_gate, args, keep)
+
+
+def prepare_mixer_forward(ctx: Context, v: torch.Tensor, g: torch.Tensor, y: torch.Tensor, n_fft: int | None = None,
+                          wrm: dict | None = None, workspace: torch.Tensor | None = None, stream=None) -> PreparedCall:
+    n = v.shape[1] if n_fft is None else n_fft
+    keep: list = [v, g, y, workspace]
+    w = _wavelet_struct(wrm, keep)
+    av, ay = act(v), act(y)
+    keep += [w, av, ay]
+    args = (ctx.handle, _stream(stream), C.byref(av), _ptr(g), C.byref(ay), n, None if w is None else C.byref(w),
+            _ptr(workspace), 0 if workspace is None else workspace.numel())
+    return PreparedCall(lib().spectre_mixer_forward, args, keep)
+
+
+def prepare_append(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t: torch.Tensor, t: int,
+                   stream=None) -> PreparedCall:
+    cs = cache.struct()
+    keep = [cache, q_t, v_t, cs]
+    args = (ctx.handle, _stream(stream), C.byref(cs), _ptr(q_t), _ptr(v_t), int(t))
+    return PreparedCall(lib().spectre_prefix_cache_append, args, keep)
