@@ -109,6 +109,44 @@ int spectre_gate(spectre_ctx* ctx, void* stream,
                  float* g_out, float* qbar_out,
                  void* workspace, size_t workspace_bytes);
 
+/*
+ * spectre_gate_static - spectre_gate for callers that cannot provide scratch.
+ * (The paper has no counterpart; this is a deployment convenience.)
+ *
+ * Some hosts of this library may not allocate device memory at all at the point
+ * where the gate runs: an inference-engine plugin whose enqueue hook is handed
+ * inputs and outputs only and whose host owns every byte of the memory pool, a
+ * serving loop that must stay free of the implicit device-wide synchronisation
+ * cudaMalloc/cudaFree bring, or a process pinned to a fixed memory budget.  For
+ * them this entry point computes exactly what spectre_gate computes, with the
+ * same kernels, but keeps its scratch (the pooled sum of the queries and, with
+ * the Toeplitz update on, the pre-update gate) in an array compiled into the
+ * library: spectre_gate_static_max_bytes() bytes (1 MiB) of device memory that
+ * every GPU which loads the library holds until the process exits.  It calls no
+ * cudaMalloc, cudaFree or any allocating routine; inputs and outputs are still
+ * the caller's.
+ *
+ *   - Shapes whose spectre_gate_workspace_bytes(...) exceeds the array are
+ *     rejected with SPECTRE_ERR_UNSUPPORTED and a message that names both sizes
+ *     (with the Toeplitz update off the need is 4*B*H*D bytes rounded up to 256).
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress); make that first call before starting any stream
+ *     capture on that device.
+ *   - All calls on a device share the one array.  Each call clears the part it
+ *     accumulates into, so leftovers of earlier calls are harmless, but two calls
+ *     whose kernels may overlap on the GPU (different streams, no dependency
+ *     between them) race on it and give wrong gates: serialise them, or use
+ *     spectre_gate with separate workspaces.
+ * Arguments and results are those of spectre_gate without the workspace pair.
+ */
+size_t spectre_gate_static_max_bytes(void);
+int spectre_gate_static(spectre_ctx* ctx, void* stream,
+                        const spectre_act* q, const float* sum_q,
+                        int32_t B, int32_t H, int32_t D, float inv_count,
+                        const spectre_gate_params* params, int32_t n_fft,
+                        const int64_t* shift, int64_t shift_all,
+                        float* g_out, float* qbar_out);
+
 /* Wavelet refinement parameters (Sec. 3.5).  Either level_gates is given, or it
  * is NULL and the gates are computed from qbar by the two-layer MLP
  * s = GELU(qbar Ww1 + bw1) Ww2 + bw2 (linear output). */

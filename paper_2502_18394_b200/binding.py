@@ -26,7 +26,7 @@ SPECTRE_BF16 = 1
 
 EXPORTS = [
     "spectre_create", "spectre_destroy", "spectre_status_string", "spectre_last_error",
-    "spectre_gate_workspace_bytes", "spectre_gate",
+    "spectre_gate_workspace_bytes", "spectre_gate", "spectre_gate_static_max_bytes", "spectre_gate_static",
     "spectre_mixer_workspace_bytes", "spectre_mixer_forward",
     "spectre_wavelet_refine",
     "spectre_prefill_workspace_bytes", "spectre_prefix_cache_prefill", "spectre_prefix_cache_append",
@@ -83,6 +83,8 @@ def lib():
     L.spectre_gate.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                C.c_float, C.POINTER(GateParams), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p,
                                C.c_void_p, C.c_void_p, C.c_size_t]
+    L.spectre_gate_static_max_bytes.restype = C.c_size_t
+    L.spectre_gate_static.argtypes = L.spectre_gate.argtypes[:-2]
     L.spectre_mixer_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 6
     L.spectre_mixer_workspace_bytes.restype = C.c_size_t
     L.spectre_mixer_forward.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.c_void_p, C.POINTER(Act), C.c_int32,
@@ -204,6 +206,30 @@ def spectre_gate(ctx: Context, params: dict, n_fft: int, q: torch.Tensor | None 
     _check(lib().spectre_gate(ctx.handle, _stream(stream), None if a is None else C.byref(a), _ptr(sum_q), B, H, D,
                               float(inv_count), C.byref(gp), n_fft, _ptr(shift), int(shift_all), _ptr(g_out),
                               _ptr(qbar_out), _ptr(workspace), 0 if workspace is None else workspace.numel()))
+    return g_out
+
+
+def spectre_gate_static_max_bytes() -> int:
+    return lib().spectre_gate_static_max_bytes()
+
+
+def spectre_gate_static(ctx: Context, params: dict, n_fft: int, g_out: torch.Tensor, q: torch.Tensor | None = None,
+                        sum_q: torch.Tensor | None = None, inv_count: float = 0.0,
+                        shift: torch.Tensor | None = None, shift_all: int = 0,
+                        qbar_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """spectre_gate with the scratch inside the library: for callers that may not allocate device
+    memory where the gate runs.  Nothing is allocated here either, so the output tensor g_out
+    [B,H,K,2] is a required argument.  Calls on one device share the scratch: do not overlap them."""
+    if q is not None:
+        B, _, H, D = q.shape
+    else:
+        B, H, D = sum_q.shape
+    keep: list = []
+    gp = _gate_struct(params, keep)
+    a = act(q) if q is not None else None
+    _check(lib().spectre_gate_static(ctx.handle, _stream(stream), None if a is None else C.byref(a), _ptr(sum_q),
+                                     B, H, D, float(inv_count), C.byref(gp), n_fft, _ptr(shift), int(shift_all),
+                                     _ptr(g_out), _ptr(qbar_out)))
     return g_out
 
 

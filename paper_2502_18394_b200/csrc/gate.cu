@@ -312,3 +312,54 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   }
   return SPECTRE_OK;
 }
+
+// ---- gate without any caller- or library-side allocation -----------------------
+// Scratch of spectre_gate_static: one fixed array per GPU that loads this library,
+// resident until the process exits.  Host code must not hand this name to a kernel
+// (on the host it is only a stand-in for the symbol); the device address is looked
+// up once per device below.
+#define SPECTRE_GATE_STATIC_BYTES (1u << 20)
+static __device__ __align__(256) unsigned char g_gate_static_scratch[SPECTRE_GATE_STATIC_BYTES];
+
+namespace spectre {
+static const int kMaxDevices = 64;
+static void* g_static_ptr[kMaxDevices] = {};     // device address of the array, per device ordinal
+
+// With `device` current: resolves (once) the device address of the static scratch.
+static int static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return fail(SPECTRE_ERR_UNSUPPORTED, "device ordinal beyond 63");
+  if (!g_static_ptr[device]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_gate_static_scratch);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(gate static scratch)");
+    if (!p) return fail(SPECTRE_ERR_CUDA, "static scratch has no device address");
+    g_static_ptr[device] = p;
+  }
+  *out = g_static_ptr[device];
+  return SPECTRE_OK;
+}
+}  // namespace spectre
+
+extern "C" size_t spectre_gate_static_max_bytes(void) { return SPECTRE_GATE_STATIC_BYTES; }
+
+extern "C" int spectre_gate_static(spectre_ctx* ctx, void* stream, const spectre_act* q, const float* sum_q, int32_t B,
+                                   int32_t H, int32_t D, float inv_count, const spectre_gate_params* gp, int32_t n_fft,
+                                   const int64_t* shift, int64_t shift_all, float* g_out, float* qbar_out) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  if (!gp) return fail(SPECTRE_ERR_INVALID_ARG, "gate parameters are NULL");
+  if (B < 1 || H < 1 || D < 1 || n_fft < 1 || gp->toeplitz_r < 0)
+    return fail(SPECTRE_ERR_INVALID_ARG, "B, H, D, n_fft must be positive");
+  const size_t need = spectre_gate_workspace_bytes(ctx, B, H, D, n_fft, gp->toeplitz_r);
+  if (need > SPECTRE_GATE_STATIC_BYTES)
+    return fail(SPECTRE_ERR_UNSUPPORTED,
+                "spectre_gate_static: this shape needs " + std::to_string(need) + " bytes of scratch, the built-in array holds " +
+                    std::to_string((size_t)SPECTRE_GATE_STATIC_BYTES) + "; use spectre_gate with a workspace");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  void* scratch = nullptr;
+  int rc = static_scratch_address(ctx->device, &scratch);
+  if (rc != SPECTRE_OK) return rc;
+  // Same kernels as spectre_gate; the pooled sum is cleared inside (cudaMemsetAsync on the
+  // caller's stream), so what an earlier call left in the array does not matter.
+  return spectre_gate(ctx, stream, q, sum_q, B, H, D, inv_count, gp, n_fft, shift, shift_all, g_out, qbar_out, scratch,
+                      SPECTRE_GATE_STATIC_BYTES);
+}
