@@ -10,7 +10,7 @@
  * Conventions
  *   - Every tensor argument is CALLER-OWNED DEVICE memory unless a comment says
  *     "host".  The library never allocates or frees device memory in the calls
- *     below (spectre_create allocates host memory only); scratch is passed in as
+ *     below (spectre_create owns one small device table); scratch is passed in as
  *     `workspace`, sized by the matching *_workspace_bytes query.
  *   - All work is enqueued on the caller's stream (`stream` is a cudaStream_t
  *     passed as void*; NULL = the default stream).  No call synchronises.
@@ -39,16 +39,24 @@ typedef enum {
   SPECTRE_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad shape, bad dtype      */
   SPECTRE_ERR_UNSUPPORTED = 2,   /* valid request outside the supported set              */
   SPECTRE_ERR_WORKSPACE = 3,     /* workspace missing or smaller than the query result   */
-  SPECTRE_ERR_CUDA = 4           /* a CUDA runtime call or launch failed                 */
+  SPECTRE_ERR_CUDA = 4,          /* a CUDA runtime call or launch failed                 */
+  SPECTRE_ERR_TIMEOUT = 5        /* a bounded on-chip wait ran out (spectre_poll_status) */
 } spectre_status;
 
 typedef enum { SPECTRE_F32 = 0, SPECTRE_BF16 = 1 } spectre_dtype;
 
 typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch limits */
 
-/* Creates a context for CUDA device `device` (host allocation only). */
+/* Creates a context for CUDA device `device`.  Besides host memory it owns one 32 KiB
+ * device table (the 64-point DFT matrix of the tensor-core mixer) and one pinned status
+ * word; both are released by spectre_destroy.  No other call allocates. */
 int spectre_create(spectre_ctx** out, int device);
 int spectre_destroy(spectre_ctx* ctx);
+/* The tensor-core mixer hands tiles between its warps through on-chip barriers whose waits
+ * are bounded; a wait that runs out makes the kernel finish early and record it.  Call this
+ * after synchronising the stream: SPECTRE_OK, or SPECTRE_ERR_TIMEOUT (and the record is
+ * cleared) if any kernel since the last poll gave up, in which case its output is invalid. */
+int spectre_poll_status(spectre_ctx* ctx);
 /* Static description of a status code. */
 const char* spectre_status_string(int status);
 /* Text of the most recent failure on the calling thread ("" if none). */

@@ -21,11 +21,12 @@ SPECTRE_ERR_INVALID_ARG = 1
 SPECTRE_ERR_UNSUPPORTED = 2
 SPECTRE_ERR_WORKSPACE = 3
 SPECTRE_ERR_CUDA = 4
+SPECTRE_ERR_TIMEOUT = 5
 SPECTRE_F32 = 0
 SPECTRE_BF16 = 1
 
 EXPORTS = [
-    "spectre_create", "spectre_destroy", "spectre_status_string", "spectre_last_error",
+    "spectre_create", "spectre_destroy", "spectre_status_string", "spectre_last_error", "spectre_poll_status",
     "spectre_gate_workspace_bytes", "spectre_gate", "spectre_gate_static_max_bytes", "spectre_gate_static",
     "spectre_mixer_workspace_bytes", "spectre_mixer_forward",
     "spectre_wavelet_refine",
@@ -75,6 +76,7 @@ def lib():
     L = C.CDLL(_LIB_PATH)
     L.spectre_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
     L.spectre_destroy.argtypes = [C.c_void_p]
+    L.spectre_poll_status.argtypes = [C.c_void_p]
     L.spectre_status_string.argtypes = [C.c_int]
     L.spectre_status_string.restype = C.c_char_p
     L.spectre_last_error.restype = C.c_char_p
@@ -138,6 +140,10 @@ class Context:
         self.handle = C.c_void_p()
         _check(lib().spectre_create(C.byref(self.handle), device))
         self.device = device
+
+    def poll_status(self):
+        """Raises SpectreError(SPECTRE_ERR_TIMEOUT) if a kernel gave up on a bounded wait (call after a sync)."""
+        _check(lib().spectre_poll_status(self.handle))
 
     def close(self):
         if self.handle:

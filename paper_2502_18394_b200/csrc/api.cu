@@ -4,7 +4,11 @@
 
 #include "common.cuh"
 
+#include <cuda_fp16.h>
+
 namespace spectre {
+
+int build_dft64(__half* F, cudaStream_t st);   // mixer_tc.cu
 
 static thread_local std::string g_last_error;
 
@@ -86,12 +90,45 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
   cudaDeviceGetAttribute(&cl, cudaDevAttrClusterLaunch, device);
   c->cluster_ok = cl;
   c->l2_bytes = (size_t)prop.l2CacheSize;
+  c->dft64 = nullptr;
+  c->status_host = nullptr;
+  c->status_dev = nullptr;
+  cudaError_t e2 = cudaSetDevice(device);
+  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft64, 128 * 128 * sizeof(__half));
+  if (e2 == cudaSuccess) e2 = cudaHostAlloc(reinterpret_cast<void**>(&c->status_host), sizeof(int), cudaHostAllocMapped);
+  if (e2 == cudaSuccess) {
+    *c->status_host = 0;
+    e2 = cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->status_dev), c->status_host, 0);
+  }
+  if (e2 == cudaSuccess) {
+    int rc = build_dft64(reinterpret_cast<__half*>(c->dft64), 0);
+    if (rc == SPECTRE_OK) e2 = cudaStreamSynchronize(0);
+    else e2 = cudaErrorUnknown;
+  }
+  if (e2 != cudaSuccess) {
+    spectre_destroy(c);
+    return cuda_fail(e2, "spectre_create: device table set-up");
+  }
   *out = c;
   return SPECTRE_OK;
 }
 
 extern "C" int spectre_destroy(spectre_ctx* ctx) {
+  if (ctx) {
+    if (ctx->dft64) cudaFree(ctx->dft64);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+  }
   delete ctx;
+  return SPECTRE_OK;
+}
+
+extern "C" int spectre_poll_status(spectre_ctx* ctx) {
+  if (!ctx || !ctx->status_host) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  int v = *reinterpret_cast<volatile int*>(ctx->status_host);
+  if (v != 0) {
+    *reinterpret_cast<volatile int*>(ctx->status_host) = 0;
+    return fail(SPECTRE_ERR_TIMEOUT, "a kernel gave up on a bounded on-chip wait; its outputs are undefined");
+  }
   return SPECTRE_OK;
 }
 
@@ -102,6 +139,7 @@ extern "C" const char* spectre_status_string(int status) {
     case SPECTRE_ERR_UNSUPPORTED: return "unsupported configuration";
     case SPECTRE_ERR_WORKSPACE: return "workspace missing or too small";
     case SPECTRE_ERR_CUDA: return "CUDA error";
+    case SPECTRE_ERR_TIMEOUT: return "device-side wait timed out";
     default: return "unknown status";
   }
 }

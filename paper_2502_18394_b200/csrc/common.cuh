@@ -16,6 +16,9 @@ struct spectre_ctx {
   int max_smem_optin;     // bytes of dynamic shared memory a CTA may opt in to
   int cluster_ok;         // thread-block clusters usable on this device
   size_t l2_bytes;
+  void* dft64;            // device: 64-point DFT matrix (fp16, MMA operand layout), 32 KiB
+  int* status_host;       // pinned, device-mapped status word written by kernels whose waits ran out
+  int* status_dev;
 };
 
 namespace spectre {

@@ -22,7 +22,19 @@
 
 namespace cg = cooperative_groups;
 
+#include <cstdlib>
+#include <cstring>
+
 namespace spectre {
+
+int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                        const spectre_act* y);   // mixer_tc.cu
+
+// SPECTRE_FORCE_PATH=alu keeps every transform on the fp32 ALU kernels (tests use it).
+static bool tensor_path_allowed() {
+  const char* e = std::getenv("SPECTRE_FORCE_PATH");
+  return !(e && std::strcmp(e, "alu") == 0);
+}
 
 constexpr int kMaxStages = 8;
 constexpr int kLocalMax = 2048;      // rows of a tile one CTA keeps in shared memory
@@ -612,6 +624,12 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   }
   SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (v->dtype == SPECTRE_BF16 && n_fft == 8192 && ctx->dft64 && tensor_path_allowed()) {
+    rc = launch_mixer_tc8192(ctx, st, v, g, y);
+    if (rc != SPECTRE_OK) return rc;
+    if (wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
+    return SPECTRE_OK;
+  }
   rc = (v->dtype == SPECTRE_BF16) ? mixer_typed<bf16>(ctx, st, v, g, y, pl, workspace, workspace_bytes)
                                   : mixer_typed<float>(ctx, st, v, g, y, pl, workspace, workspace_bytes);
   if (rc != SPECTRE_OK) return rc;
