@@ -106,6 +106,7 @@ __device__ __forceinline__ float2 mul_root(float2 x, int J, int R) {
   // reduce to sixteenths / odd radices; after unrolling J and R are constants
   J %= R;
   if (J == 0) return x;
+  while ((J & 1) == 0 && (R & 1) == 0) { J >>= 1; R >>= 1; }     // lowest terms (folds after unrolling)
   if ((4 * J) % R == 0) {                 // multiples of a quarter turn
     int q = (4 * J) / R;                  // 1,2,3
     if (q == 2) return make_float2(-x.x, -x.y);
@@ -147,6 +148,22 @@ __device__ __forceinline__ float2 mul_root(float2 x, int J, int R) {
     case 228: c = -0.90096886790241915f; s = -0.43388373911755801f; break;
     case 229: c = -0.22252093395631459f; s = -0.97492791218182362f; break;
     case 230: c = 0.62348980185873337f; s = -0.78183148246802991f; break;
+    case 1025: c = 0.98078528040323043f; s = 0.19509032201612825f; break;
+    case 1027: c = 0.83146961230254524f; s = 0.55557023301960218f; break;
+    case 1029: c = 0.55557023301960229f; s = 0.83146961230254524f; break;
+    case 1031: c = 0.19509032201612833f; s = 0.98078528040323043f; break;
+    case 1033: c = -0.19509032201612819f; s = 0.98078528040323043f; break;
+    case 1035: c = -0.55557023301960196f; s = 0.83146961230254546f; break;
+    case 1037: c = -0.83146961230254535f; s = 0.55557023301960218f; break;
+    case 1039: c = -0.98078528040323043f; s = 0.19509032201612861f; break;
+    case 1041: c = -0.98078528040323043f; s = -0.19509032201612836f; break;
+    case 1043: c = -0.83146961230254546f; s = -0.55557023301960196f; break;
+    case 1045: c = -0.55557023301960218f; s = -0.83146961230254524f; break;
+    case 1047: c = -0.19509032201612866f; s = -0.98078528040323032f; break;
+    case 1049: c = 0.1950903220161283f; s = -0.98078528040323043f; break;
+    case 1051: c = 0.55557023301960184f; s = -0.83146961230254546f; break;
+    case 1053: c = 0.83146961230254524f; s = -0.55557023301960218f; break;
+    case 1055: c = 0.98078528040323032f; s = -0.19509032201612872f; break;
     default: break;
   }
   if (INV) s = -s;
@@ -211,6 +228,9 @@ template <bool INV> struct Dft<8, INV> {
 };
 template <bool INV> struct Dft<16, INV> {
   static __device__ __forceinline__ void run(float2 (&x)[16]) { dft_ct<4, 4, INV>(x); }
+};
+template <bool INV> struct Dft<32, INV> {
+  static __device__ __forceinline__ void run(float2 (&x)[32]) { dft_ct<4, 8, INV>(x); }
 };
 // Odd radices: the defining sum with constant roots.
 template <int R, bool INV>

@@ -30,10 +30,24 @@ namespace spectre {
 int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                         const spectre_act* y);   // mixer_tc.cu
 
-// SPECTRE_FORCE_PATH=alu keeps every transform on the fp32 ALU kernels (tests use it).
-static bool tensor_path_allowed() {
+bool tc4k_supported(int n, int D);                                                     // mixer_tc4k.cu
+size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
+size_t tc4k_min_workspace(int n, int D);
+int launch_mixer_tc4k(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                      const spectre_act* y, int n, void* ws, size_t ws_bytes);
+
+// Path choice for bf16 transforms.  SPECTRE_FORCE_PATH = alu | fused | staged overrides it (tests):
+//   alu     fp32 butterflies only
+//   fused   the single-kernel tensor-core mixer (n = 8192 only)
+//   staged  transpose-in / tensor-core units / transpose-out (n = 4096 ... 131072, needs workspace)
+enum { kPathAuto = 0, kPathAlu = 1, kPathFused = 2, kPathStaged = 3 };
+static int forced_path() {
   const char* e = std::getenv("SPECTRE_FORCE_PATH");
-  return !(e && std::strcmp(e, "alu") == 0);
+  if (!e) return kPathAuto;
+  if (std::strcmp(e, "alu") == 0) return kPathAlu;
+  if (std::strcmp(e, "fused") == 0) return kPathFused;
+  if (std::strcmp(e, "staged") == 0) return kPathStaged;
+  return kPathAuto;
 }
 
 constexpr int kMaxStages = 8;
@@ -590,9 +604,13 @@ using namespace spectre;
 
 extern "C" size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t L, int32_t H, int32_t D,
                                                 int32_t n_fft, int32_t dtype) {
-  (void)L; (void)dtype;
+  (void)L;
   TransformPlan pl;
   if (!ctx || B < 1 || H < 1 || D < 8 || !make_plan(ctx, n_fft, &pl)) return 0;
+  const int force = forced_path();
+  if (dtype == SPECTRE_BF16 && ctx->dft64 && tc4k_supported(n_fft, D) && force != kPathAlu && force != kPathFused &&
+      (n_fft != 8192 || force == kPathStaged))               // n = 8192 defaults to the single-kernel path
+    return tc4k_workspace_bytes(ctx, n_fft, D, B * H);
   if (pl.N1 == 1) return 0;
   return (size_t)preferred_group(ctx, n_fft, D, B * H) * slab_ws_bytes(n_fft, D);
 }
@@ -611,21 +629,28 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   if (n_fft < v->L) return fail(SPECTRE_ERR_INVALID_ARG, "n_fft smaller than L");
   TransformPlan pl;
   if (!make_plan(ctx, n_fft, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "n_fft outside the supported set");
-  if (pl.N1 > 1) {
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15))
-      return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
+  const int force = forced_path();
+  const bool tc_ok = v->dtype == SPECTRE_BF16 && ctx->dft64 != nullptr && force != kPathAlu;
+  const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 15);
+  const bool fused = tc_ok && n_fft == 8192 && force != kPathStaged;
+  const bool staged = !fused && tc_ok && force != kPathFused && tc4k_supported(n_fft, v->D) && ws_ok &&
+                      workspace_bytes >= tc4k_min_workspace(n_fft, v->D);
+  if (!staged && !fused && pl.N1 > 1) {
+    if (!ws_ok) return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
     if (workspace_bytes < slab_ws_bytes(n_fft, v->D))
       return fail(SPECTRE_ERR_WORKSPACE, "mixer workspace smaller than one (batch, head) slab");
-    if (v->ptr == y->ptr) return fail(SPECTRE_ERR_INVALID_ARG, "y may not alias v on the multi-pass path");
   }
+  if ((staged || pl.N1 > 1) && v->ptr == y->ptr)
+    return fail(SPECTRE_ERR_INVALID_ARG, "y may not alias v on the multi-pass path");
   if (wrm) {
     if (wrm->levels < 1 || wrm->levels > 10 || (v->L % (1 << wrm->levels)) != 0)
       return fail(SPECTRE_ERR_INVALID_ARG, "wavelet levels: 2^J must divide L");
   }
   SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (v->dtype == SPECTRE_BF16 && n_fft == 8192 && ctx->dft64 && tensor_path_allowed()) {
-    rc = launch_mixer_tc8192(ctx, st, v, g, y);
+  if (staged || fused) {
+    rc = staged ? launch_mixer_tc4k(ctx, st, v, g, y, n_fft, workspace, workspace_bytes)
+                : launch_mixer_tc8192(ctx, st, v, g, y);
     if (rc != SPECTRE_OK) return rc;
     if (wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
     return SPECTRE_OK;

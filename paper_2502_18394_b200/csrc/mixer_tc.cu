@@ -32,8 +32,18 @@ constexpr int kTcSbo = 2320;                   // bytes between 8-column groups 
 constexpr int kTcBBytes = 32 * kTcSbo;         // one 256-column B operand
 constexpr int kTcFBytes = 128 * 128 * 2;
 constexpr int kTcSmem = kTcFBytes + 2 * kTcBBytes + 64;
-constexpr int kTcThreads = 288;                // 8 epilogue warps + 1 MMA-issuing warp
+constexpr int kTcEpiWarps = 16;                // 4 per TMEM lane quadrant, one column quarter each
+constexpr int kTcEpiThreads = 32 * kTcEpiWarps;
+constexpr int kTcThreads = kTcEpiThreads + 32; // + 1 MMA-issuing warp
 constexpr uint32_t kSpinLimit = 1u << 24;
+
+// Optional phase stamps (SM clock), compiled in only for profiling builds.
+#ifdef SPECTRE_TC_TIMING
+__device__ long long g_tc_timing[1024][16];
+#define TC_STAMP(slot) do { if (T == 0 && warp == 0 && blockIdx.x < 1024) g_tc_timing[blockIdx.x][slot] = clock64(); } while (0)
+#else
+#define TC_STAMP(slot) do { } while (0)
+#endif
 
 struct TcParams {
   const bf16* src;
@@ -104,49 +114,73 @@ __device__ __forceinline__ float2 gate8192(const float2* __restrict__ g, int k) 
   return v;
 }
 
-// Epilogue between two MMA stages of one half.
+// Epilogue between two MMA stages of one half, for one warp: TMEM lane quadrant q, column
+// quarter cq (64 of the 256 columns).  A thread owns rows (digit) 16 q' + T/4 for the two lane
+// groups q' = 2q, 2q+1 and, per 8-column group, the column digit 2*group + p with the column
+// pair c = 2cp, 2cp+1.  TMEM loads run one 32-column chunk ahead of the arithmetic.
 //   MODE 1: twiddle W_4096^{row * col}, write transposed (row digit -> column index of B, col digit -> K)
 //   MODE 2: gate (and conjugate for the inverse), write straight (col digit -> column index, row digit -> K)
 template <int MODE>
-__device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm, int q, int chalf, int T,
-                                             const float2* __restrict__ g, int parity, float ginv) {
+__device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm, int q, int cq, int T,
+                                             const float2 (&G)[16], float ginv) {
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
-#pragma unroll 1
-  for (int j = 0; j < 2; ++j) {
-    const int row = 8 * (2 * q + j) + i;                      // digit held by this thread's TMEM rows
-    float2 w = make_float2(1.f, 0.f), wstep = w;
-    if (MODE == 1) {
-      w = twiddle_fwd((unsigned)((row * (32 * chalf + p)) & 4095), 4096u);
+  uint32_t r[2][16];
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
+  tmem_ld_16x256b_x4(taddr0, r[0]);
+  float2 w = make_float2(1.f, 0.f), wstep = w;
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {                      // step = 2 j + chunk
+    const int j = step >> 1, chunk = step & 1;
+    const int row = 8 * (2 * q + j) + i;
+    if (MODE == 1 && chunk == 0) {
+      w = twiddle_fwd((unsigned)((row * (16 * cq + p)) & 4095), 4096u);
       wstep = twiddle_fwd((unsigned)((2 * row) & 4095), 4096u);
     }
-    const uint32_t taddr = tmem_d + ((uint32_t)(32 * q + 16 * j) << 16) + 128 * chalf;
-#pragma unroll 1
-    for (int chunk = 0; chunk < 4; ++chunk) {
-      uint32_t r[16];
-      tmem_ld_16x256b_x4(taddr + 32 * chunk, r);
-      tmem_ld_wait();
+    tmem_ld_wait();
+    if (step < 3) {
+      const int nj = (step + 1) >> 1, nchunk = (step + 1) & 1;
+      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * nj) << 16) + 32 * nchunk, r[(step + 1) & 1]);
+    }
+    const uint32_t (&rr)[16] = r[step & 1];
+    // byte offset of this thread's first element of the chunk in the next operand
+    uint32_t base;
+    if (MODE == 1) base = (uint32_t)((row >> 1) * kTcSbo + (4 * (row & 1) + 2 * cp) * 16 + (4 * cq + 2 * chunk) * kTcLbo + 4 * p);
+    else base = (uint32_t)((8 * cq + 4 * chunk) * kTcSbo + (4 * p + 2 * cp) * 16 + (row >> 2) * kTcLbo + (row & 3) * 4);
 #pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        const int col = 2 * (16 * chalf + 4 * chunk + x) + p;  // digit held by this column group
-        float2 v0 = make_float2(__uint_as_float(r[4 * x]), __uint_as_float(r[4 * x + 2]));
-        float2 v1 = make_float2(__uint_as_float(r[4 * x + 1]), __uint_as_float(r[4 * x + 3]));
-        uint32_t off;
-        if (MODE == 1) {
-          v0 = cmul(v0, w);
-          v1 = cmul(v1, w);
-          w = cmul(w, wstep);
-          off = b_off(4 * row + 2 * cp, 2 * col);
-        } else {
-          float2 G = cscale(gate8192(g, 2 * (col + 64 * row) + parity), ginv);
-          v0 = cmul(v0, G);
-          v1 = cmul(v1, G);
-          v0.y = -v0.y;
-          v1.y = -v1.y;
-          off = b_off(4 * col + 2 * cp, 2 * row);
-        }
-        *reinterpret_cast<uint32_t*>(Bsm + off) = pack_h2(v0.x, v0.y);
-        *reinterpret_cast<uint32_t*>(Bsm + off + 16) = pack_h2(v1.x, v1.y);
+    for (int x = 0; x < 4; ++x) {
+      float2 v0 = make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
+      float2 v1 = make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
+      uint32_t off;
+      if (MODE == 1) {
+        v0 = cmul(v0, w);
+        v1 = cmul(v1, w);
+        w = cmul(w, wstep);
+        off = base + (x >> 1) * kTcLbo + (x & 1) * 8;
+      } else {
+        const float2 g = cscale(G[4 * step + x], ginv);
+        v0 = cmul(v0, g);
+        v1 = cmul(v1, g);
+        v0.y = -v0.y;
+        v1.y = -v1.y;
+        off = base + x * kTcSbo;
       }
+      *reinterpret_cast<uint32_t*>(Bsm + off) = pack_h2(v0.x, v0.y);
+      *reinterpret_cast<uint32_t*>(Bsm + off + 16) = pack_h2(v1.x, v1.y);
+    }
+  }
+}
+
+// Gate values one thread needs in the MODE 2 epilogue of one half: bin 2 (col + 64 row) + parity.
+__device__ __forceinline__ void fetch_gate(const float2* __restrict__ g, int q, int cq, int T, int parity,
+                                           float2 (&G)[16]) {
+  const int i = T >> 2, p = (T >> 1) & 1;
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    const int row = 8 * (2 * q + (step >> 1)) + i;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int col = 2 * (8 * cq + 4 * (step & 1) + x) + p;
+      G[4 * step + x] = gate8192(g, 2 * (col + 64 * row) + parity);
     }
   }
 }
@@ -165,7 +199,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
   unsigned char* Bsm[2] = {smem + kTcFBytes, smem + kTcFBytes + kTcBBytes};
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + 2 * kTcBBytes);   // [0,1] B ready, [2,3] D ready
   __shared__ uint32_t tmem_slot;
-  __shared__ float red[8];
+  __shared__ float red[kTcEpiWarps];
 
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
   const int tile = blockIdx.x % p.ntile, slab = blockIdx.x / p.ntile;
@@ -173,23 +207,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
   const int col0 = tile * 8;
   const float2* g = p.g + (size_t)slab * 4097;
 
-  if (warp == 8) {
+  TC_STAMP(0);
+  if (warp == kTcEpiWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(512));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[0])), "r"(256));
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[1])), "r"(256));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[0])), "r"(kTcEpiThreads));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[1])), "r"(kTcEpiThreads));
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[2])), "r"(1));
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[3])), "r"(1));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // DFT matrix -> smem; max |g| of this head (fp16 range management)
   float gmax = 0.f;
-  if (tid < 256) {
+  if (tid < kTcEpiThreads) {
     const uint4* Fg = reinterpret_cast<const uint4*>(p.F);
-    for (int i = tid; i < kTcFBytes / 16; i += 256) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
-    for (int k = tid; k <= 4096; k += 256) {
+    for (int i = tid; i < kTcFBytes / 16; i += kTcEpiThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
+    for (int k = tid; k <= 4096; k += kTcEpiThreads) {
       float2 v = __ldg(g + k);
       gmax = fmaxf(gmax, fmaxf(fabsf(v.x), fabsf(v.y)));
     }
@@ -201,11 +236,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = tmem_slot;
   gmax = 0.f;
-  for (int i = 0; i < 8; ++i) gmax = fmaxf(gmax, red[i]);
+  for (int i = 0; i < kTcEpiWarps; ++i) gmax = fmaxf(gmax, red[i]);
   gmax *= 1.41421356f;                                   // bound on |g_k|
   const float ginv = gmax > 0.f ? 1.0f / gmax : 0.f;
+  TC_STAMP(1);
 
-  if (warp == 8) {
+  if (warp == kTcEpiWarps) {
     // ---- MMA issuer: 4 stages x 2 halves, 8 K-steps each ----
     const uint32_t idesc = umma_idesc_128x256();
     bool ok = true;
@@ -237,14 +273,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
     {
       const bf16* src = p.src + b * p.s_sb + h * p.s_sh + col0;
       const int t1 = tid & 63, t2base = tid >> 6;          // 32 lanes = 32 consecutive t1: conflict-free stores
+      constexpr int kIter = 64 / (kTcEpiThreads / 64);
       float2 w = twiddle_fwd((unsigned)(64 * t1 + t2base), 8192u);
-      const float2 wstep = twiddle_fwd(4u, 8192u);
-#pragma unroll 2
-      for (int it = 0; it < 16; ++it) {
-        const int t2 = t2base + 4 * it, t = 64 * t1 + t2;
+      const float2 wstep = twiddle_fwd((unsigned)(kTcEpiThreads / 64), 8192u);
+#pragma unroll 4
+      for (int it = 0; it < kIter; ++it) {
+        const int t2 = t2base + (kTcEpiThreads / 64) * it, t = 64 * t1 + t2;
         uint4 ra = make_uint4(0u, 0u, 0u, 0u), rb = ra;
-        if (t < p.L) ra = *reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl);
-        if (t + 4096 < p.L) rb = *reinterpret_cast<const uint4*>(src + (int64_t)(t + 4096) * p.s_sl);
+        if (t < p.L) ra = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl));
+        if (t + 4096 < p.L) rb = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)(t + 4096) * p.s_sl));
         const uint32_t ua[4] = {ra.x, ra.y, ra.z, ra.w}, ub[4] = {rb.x, rb.y, rb.z, rb.w};
         const uint32_t off = b_off(4 * t2, 2 * t1);
 #pragma unroll
@@ -259,68 +296,83 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
       }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    TC_STAMP(2);
     mbar_arrive(smem_u32(&bars[0]));
     mbar_arrive(smem_u32(&bars[1]));
 
-    const int q = warp & 3, chalf = warp >> 2;
+    const int q = warp & 3, cq = warp >> 2;
     bool ok = true;
+    float2 G[16];
     // ---- stages 1..3: wait for D, transform, hand the next operand to the issuer ----
+#pragma unroll 1
     for (int stage = 0; stage < 3 && ok; ++stage) {
+#pragma unroll 1
       for (int half = 0; half < 2 && ok; ++half) {
+        if (stage == 1) fetch_gate(g, q, cq, T, half, G);   // in flight while the MMAs finish
         ok = mbar_wait(smem_u32(&bars[2 + half]), stage & 1);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t td = tmem + 256 * half;
-        if (stage == 1) epilogue_mid<2>(td, Bsm[half], q, chalf, T, g, half, ginv);
-        else epilogue_mid<1>(td, Bsm[half], q, chalf, T, g, half, ginv);
+        if (stage == 1) epilogue_mid<2>(td, Bsm[half], q, cq, T, G, ginv);
+        else epilogue_mid<1>(td, Bsm[half], q, cq, T, G, ginv);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        TC_STAMP(3 + 2 * stage + half);
         mbar_arrive(smem_u32(&bars[half]));
       }
     }
     // ---- final: y[t], y[t+4096] = (gmax/2) conj(D_e +- W_8192^t D_o), bf16 ----
     if (ok) ok = mbar_wait(smem_u32(&bars[2]), 1);
     if (ok) ok = mbar_wait(smem_u32(&bars[3]), 1);
+    TC_STAMP(9);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int i = T >> 2, pp = (T >> 1) & 1, cp = T & 1;
       const float gs = 0.5f * gmax;
       bf16* dst = p.dst + b * p.d_sb + h * p.d_sh + col0 + 4 * cp;
-#pragma unroll 1
-      for (int j = 0; j < 2; ++j) {
-        const int t1 = 8 * (2 * q + j) + i;
-        float2 w = twiddle_fwd((unsigned)(64 * t1 + 32 * chalf + pp), 8192u);
-        const float2 wstep = twiddle_fwd(2u, 8192u);
-        const uint32_t taddr = tmem + ((uint32_t)(32 * q + 16 * j) << 16) + 128 * chalf;
-#pragma unroll 1
-        for (int chunk = 0; chunk < 4; ++chunk) {
-          uint32_t re[16], ro[16];
-          tmem_ld_16x256b_x4(taddr + 32 * chunk, re);
-          tmem_ld_16x256b_x4(taddr + 256 + 32 * chunk, ro);
-          tmem_ld_wait();
+      const float2 wstep = twiddle_fwd(2u, 8192u);
+      const uint32_t taddr0 = tmem + ((uint32_t)(32 * q) << 16) + 64 * cq;
+      uint32_t re[2][16], ro[2][16];
+      tmem_ld_16x256b_x4(taddr0, re[0]);
+      tmem_ld_16x256b_x4(taddr0 + 256, ro[0]);
+      float2 w = make_float2(1.f, 0.f);
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const int t2 = 2 * (16 * chalf + 4 * chunk + x) + pp, t = 64 * t1 + t2;
-            float2 e0 = make_float2(__uint_as_float(re[4 * x]), __uint_as_float(re[4 * x + 2]));
-            float2 e1 = make_float2(__uint_as_float(re[4 * x + 1]), __uint_as_float(re[4 * x + 3]));
-            float2 o0 = cmul(make_float2(__uint_as_float(ro[4 * x]), __uint_as_float(ro[4 * x + 2])), w);
-            float2 o1 = cmul(make_float2(__uint_as_float(ro[4 * x + 1]), __uint_as_float(ro[4 * x + 3])), w);
-            w = cmul(w, wstep);
-            if (t < p.L)
-              *reinterpret_cast<uint2*>(dst + (int64_t)t * p.d_sl) =
-                  pack_bf16x4(gs * (e0.x + o0.x), -gs * (e0.y + o0.y), gs * (e1.x + o1.x), -gs * (e1.y + o1.y));
-            if (t + 4096 < p.L)
-              *reinterpret_cast<uint2*>(dst + (int64_t)(t + 4096) * p.d_sl) =
-                  pack_bf16x4(gs * (e0.x - o0.x), -gs * (e0.y - o0.y), gs * (e1.x - o1.x), -gs * (e1.y - o1.y));
-          }
+      for (int step = 0; step < 4; ++step) {
+        const int j = step >> 1, chunk = step & 1;
+        const int t1 = 8 * (2 * q + j) + i;
+        if (chunk == 0) w = twiddle_fwd((unsigned)(64 * t1 + 16 * cq + pp), 8192u);
+        tmem_ld_wait();
+        if (step < 3) {
+          const uint32_t ta = taddr0 + ((uint32_t)(16 * ((step + 1) >> 1)) << 16) + 32 * ((step + 1) & 1);
+          tmem_ld_16x256b_x4(ta, re[(step + 1) & 1]);
+          tmem_ld_16x256b_x4(ta + 256, ro[(step + 1) & 1]);
+        }
+        const uint32_t (&xe)[16] = re[step & 1];
+        const uint32_t (&xo)[16] = ro[step & 1];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const int t2 = 2 * (8 * cq + 4 * chunk + x) + pp, t = 64 * t1 + t2;
+          float2 e0 = make_float2(__uint_as_float(xe[4 * x]), __uint_as_float(xe[4 * x + 2]));
+          float2 e1 = make_float2(__uint_as_float(xe[4 * x + 1]), __uint_as_float(xe[4 * x + 3]));
+          float2 o0 = cmul(make_float2(__uint_as_float(xo[4 * x]), __uint_as_float(xo[4 * x + 2])), w);
+          float2 o1 = cmul(make_float2(__uint_as_float(xo[4 * x + 1]), __uint_as_float(xo[4 * x + 3])), w);
+          w = cmul(w, wstep);
+          if (t < p.L)
+            *reinterpret_cast<uint2*>(dst + (int64_t)t * p.d_sl) =
+                pack_bf16x4(gs * (e0.x + o0.x), -gs * (e0.y + o0.y), gs * (e1.x + o1.x), -gs * (e1.y + o1.y));
+          if (t + 4096 < p.L)
+            *reinterpret_cast<uint2*>(dst + (int64_t)(t + 4096) * p.d_sl) =
+                pack_bf16x4(gs * (e0.x - o0.x), -gs * (e0.y - o0.y), gs * (e1.x - o1.x), -gs * (e1.y - o1.y));
         }
       }
     }
+    TC_STAMP(10);
     if (!ok && T == 0) atomicExch(p.status, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 8) {
+  TC_STAMP(11);
+  if (warp == kTcEpiWarps) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(512));
   }

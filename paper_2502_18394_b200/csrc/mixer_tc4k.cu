@@ -1,0 +1,537 @@
+// Tensor-core spectral mixer for n = 4096 * R, R in {1, 2, 4, 8, 16, 32}, bf16 I/O
+// (Sec. 3.2 steps 2 and 4; covers n = 4096 ... 131072).
+//
+// Four-step split n = R * 4096 with t = n1 * 4096 + t', k = k1 + R * kM:
+//
+//   tc_in_kernel    reads whole 128-byte rows of [B, L, H, D] (coalesced), does the radix-R
+//                   DFT over n1 and the twiddle W_n^{k1 t'} on the ALUs, rounds to fp16 and
+//                   writes, for every unit (head, k1, 4 column pairs), the first tensor-core
+//                   operand as an image of its shared-memory layout (transposed through
+//                   shared memory so that the workspace writes are whole lines too)
+//   tc_gate_kernel  per (head, k1): the 4096 gate values the unit needs (Hermitian extension,
+//                   normalised by their maximum, fp16) in the order the core reads them
+//   tc_core_kernel  persistent; every SM runs two independent pipelines, each taking a unit
+//                   through   bulk copy -> [MMA -> epilogue] x 4   with the 64-point DFT
+//                   matrix as the A operand (see mixer_tc.cu for the formulation); while one
+//                   pipeline's epilogue occupies the ALUs the other's MMAs occupy the tensor
+//                   core.  Result: the unit's 4096 x 4 complex outputs in fp16, tile-major
+//   tc_out_kernel   inverse radix-R over k1 with conj twiddles, 1/n and gate scale, bf16,
+//                   transposed through shared memory into whole-row stores
+//
+// The workspace between the kernels is sized so that a group of heads stays in L2.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace spectre {
+
+// ---- shared with mixer_tc.cu (same conventions) ------------------------------------
+constexpr int k4Lbo = 128;                       // bytes between core matrices along K
+constexpr int k4Sbo = 2064;                      // bytes between 8-column groups (2048 + 16 pad)
+constexpr int k4BBytes = 32 * k4Sbo;             // one 256-column operand in shared memory
+constexpr int k4ImgBytes = 65536;                // the same operand in the workspace (unpadded)
+constexpr int k4FBytes = 128 * 128 * 2;
+constexpr int k4GStride = 72;                    // gate table: entry (row, col) at row + 72 col
+constexpr int k4GBytes = 64 * k4GStride * 4;
+constexpr int k4OutBytes = 4096 * 4 * 4;         // unit result: [t'][4 pairs] half2
+constexpr int k4GroupThreads = 256;
+constexpr int k4CoreThreads = 2 * k4GroupThreads;
+constexpr int k4CoreSmem = k4FBytes + 2 * k4BBytes + 2 * k4GBytes + 64;
+constexpr uint32_t k4SpinLimit = 1u << 24;
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t desc4(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = (uint64_t)((saddr >> 4) & 0x3fff);
+  d |= (uint64_t)((lbo >> 4) & 0x3fff) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3fff) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+__device__ __forceinline__ bool wait4(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < k4SpinLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ uint32_t h2pack(float lo, float hi) {
+  __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ float2 h2unpack(uint32_t u) {
+  __half2 h = *reinterpret_cast<__half2*>(&u);
+  return __half22float2(h);
+}
+__device__ __forceinline__ void ld16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void ld_wait4() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// XOR skew of a tile's words inside a 32-word line: the 8 tiles a warp touches at once land in
+// 8 different bank groups (flips the t1 % 4 and t2 % 2 bits of the word index)
+__device__ __forceinline__ int tile_skew(int tile) { return (tile & 3) | (((tile >> 2) & 1) << 4); }
+
+// forward-scale of the radix-R step (keeps fp16 magnitudes near the input's)
+__host__ __device__ constexpr float in_scale(int R) {
+  return R <= 2 ? 1.0f : (R <= 8 ? 0.5f : (R == 16 ? 0.25f : 0.125f));
+}
+
+// =====================================================================================
+// transpose-in
+// =====================================================================================
+struct TcInParams {
+  const bf16* src;
+  int64_t s_sb, s_sl, s_sh;
+  unsigned char* ws_in;       // [unit][65536]
+  int H, D, L, n, ntile, slab0;
+};
+
+// CTA = (slab, group of 4 consecutive t1, block of NT2 values of t2); t' = 64 t1 + t2.
+// A warp takes one (t1, t2) at a time with lane = column pair; staging holds, for every
+// (k1, tile), the core matrices (8 operand columns x 16 bytes) of this CTA's slice.
+template <int R>
+__global__ void __launch_bounds__(256) tc_in_kernel(const TcInParams p) {
+  constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
+  constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
+  extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][NT2/2][32 words]
+  const int t2blocks = 64 / NT2;
+  int u = blockIdx.x;
+  const int t2b = u % t2blocks;  u /= t2blocks;
+  const int t1g = u % 16;  u /= 16;
+  const int slab_local = u, slab = p.slab0 + u;
+  const int b = slab / p.H, h = slab - b * p.H;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int npair = p.D / 2;
+  const bf16* src = p.src + b * p.s_sb + h * p.s_sh;
+  const float sc = in_scale(R);
+
+  for (int cb = 0; cb < npair; cb += 32) {                     // column blocks of 32 pairs (D = 64: one)
+    const int c = cb + lane;
+    const bool live = c < npair;
+    const int tile = c >> 2, c4 = c & 3;
+#pragma unroll UNR
+    for (int rs = warp; rs < 4 * NT2; rs += 8) {
+      const int t1m = rs & 3, t2l = rs >> 2;
+      const int t1 = 4 * t1g + t1m, t2 = t2b * NT2 + t2l, tp = 64 * t1 + t2;
+      float2 x[R];
+#pragma unroll
+      for (int n1 = 0; n1 < R; ++n1) {
+        const int row = n1 * 4096 + tp;
+        uint32_t v = 0u;
+        if (live && row < p.L) v = __ldg(reinterpret_cast<const uint32_t*>(src + (int64_t)row * p.s_sl + 2 * c));
+        x[n1] = make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+      }
+      Dft<R, false>::run(x);
+      const float2 w1 = twiddle_fwd((unsigned)tp, (unsigned)p.n);
+      if (live) {
+        // word inside the 128-byte core matrix: (t2 % 2, c4, t1 % 4), XOR-skewed by the tile
+        const int wl = ((t2l & 1) * 16 + c4 * 4 + t1m) ^ tile_skew(tile);
+        float2 w = make_float2(sc, 0.f);                          // sc * W_n^{k1 t'}
+#pragma unroll
+        for (int k1 = 0; k1 < R; ++k1) {
+          const float2 v = cmul(x[k1], w);
+          stage[(((size_t)k1 * p.ntile + tile) * (NT2 / 2) + (t2l >> 1)) * 32 + wl] = h2pack(v.x, v.y);
+          w = cmul(w, w1);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  // copy out: one 128-byte line per (k1, tile, t2 pair)
+  const int nlines = R * p.ntile * (NT2 / 2);
+  for (int line = warp; line < nlines; line += 8) {
+    int l = line;
+    const int t2p = l % (NT2 / 2);  l /= (NT2 / 2);
+    const int tile = l % p.ntile, k1 = l / p.ntile;
+    const uint32_t v = stage[(size_t)line * 32 + (lane ^ tile_skew(tile))];
+    const size_t unit = ((size_t)slab_local * R + k1) * p.ntile + tile;
+    const int t2pair = t2b * (NT2 / 2) + t2p;                  // operand column group nu / 8
+    unsigned char* dst = p.ws_in + unit * k4ImgBytes + (size_t)t2pair * 2048 + (size_t)t1g * 128;
+    reinterpret_cast<uint32_t*>(dst)[lane] = v;
+  }
+}
+
+// =====================================================================================
+// gate images
+// =====================================================================================
+struct TcGateParams {
+  const float2* g;          // [B*H][K]
+  unsigned char* gimg;      // [slab_local * R + k1][k4GBytes]
+  float* gscale;            // [slab_local * R + k1]
+  int n, K, R, slab0;
+};
+
+__global__ void __launch_bounds__(256) tc_gate_kernel(const TcGateParams p) {
+  __shared__ float2 vals[4096];
+  __shared__ float red[8];
+  const int sk = blockIdx.x, slab_local = sk / p.R, k1 = sk - slab_local * p.R;
+  const float2* g = p.g + (size_t)(p.slab0 + slab_local) * p.K;
+  float m = 0.f;
+  for (int kM = threadIdx.x; kM < 4096; kM += 256) {
+    const int k = k1 + p.R * kM;
+    const int kk = (2 * k <= p.n) ? k : p.n - k;
+    float2 v = __ldg(g + kk);
+    if (kk != k) v.y = -v.y;
+    if (k == 0 || 2 * k == p.n) v.y = 0.f;
+    vals[kM] = v;
+    m = fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y)));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = 0.f;
+  for (int i = 0; i < 8; ++i) m = fmaxf(m, red[i]);
+  m *= 1.41421356f;
+  const float inv = m > 0.f ? 1.0f / m : 0.f;
+  if (threadIdx.x == 0) p.gscale[sk] = m;
+  uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * k4GBytes);
+  for (int idx = threadIdx.x; idx < 64 * k4GStride; idx += 256) {
+    const int col = idx / k4GStride, row = idx - col * k4GStride;     // kM = col + 64 row
+    uint32_t v = 0u;
+    if (row < 64) {
+      const float2 gv = vals[col + 64 * row];
+      v = h2pack(gv.x * inv, gv.y * inv);
+    }
+    img[idx] = v;
+  }
+}
+
+// =====================================================================================
+// core: 4096-point units on the tensor cores
+// =====================================================================================
+struct TcCoreParams {
+  const unsigned char* ws_in;
+  const unsigned char* gimg;
+  unsigned char* ws_out;
+  const __half* F;
+  int nunits, ntile;
+  int* status;
+};
+
+// Epilogue of one MMA stage for one warp (TMEM lane quadrant q, 128-column half ch).
+//   MODE 1: twiddle W_4096^{row col}; next operand gets (row digit -> column, col digit -> K)
+//   MODE 2: gate, conjugate;           next operand gets (col digit -> column, row digit -> K)
+//   MODE 3: final: store the unit's result [t' = 64 row + col][pair] as half2
+template <int MODE>
+__device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bsm, const uint32_t* Gsm,
+                                              unsigned char* out, int q, int ch, int T) {
+  const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
+  uint32_t r[2][16];
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 128 * ch;
+  ld16x256b_x4(taddr0, r[0]);
+  float2 w = make_float2(1.f, 0.f), wstep = w;
+#pragma unroll
+  for (int step = 0; step < 8; ++step) {                        // step = 4 j + chunk
+    const int j = step >> 2, chunk = step & 3;
+    const int row = 8 * (2 * q + j) + i;
+    if (MODE == 1 && chunk == 0) {
+      w = twiddle_fwd((unsigned)((row * (32 * ch + p)) & 4095), 4096u);
+      wstep = twiddle_fwd((unsigned)((2 * row) & 4095), 4096u);
+    }
+    ld_wait4();
+    if (step < 7) {
+      const int ns = step + 1;
+      ld16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 2)) << 16) + 32 * (ns & 3), r[ns & 1]);
+    }
+    const uint32_t (&rr)[16] = r[step & 1];
+    const int grp0 = 16 * ch + 4 * chunk;                       // first 8-column group of the chunk
+    uint32_t base;
+    if (MODE == 1) base = (uint32_t)((row >> 1) * k4Sbo + (4 * (row & 1) + 2 * cp) * 16 + (grp0 >> 1) * k4Lbo + 4 * p);
+    else if (MODE == 2) base = (uint32_t)(grp0 * k4Sbo + (4 * p + 2 * cp) * 16 + (row >> 2) * k4Lbo + (row & 3) * 4);
+    else base = (uint32_t)(((64 * row + 2 * grp0 + p) * 4 + 2 * cp) * 4);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      float2 v0 = make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
+      float2 v1 = make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
+      if (MODE == 1) {
+        v0 = cmul(v0, w);
+        v1 = cmul(v1, w);
+        w = cmul(w, wstep);
+        const uint32_t off = base + (x >> 1) * k4Lbo + (x & 1) * 8;
+        *reinterpret_cast<uint32_t*>(Bsm + off) = h2pack(v0.x, v0.y);
+        *reinterpret_cast<uint32_t*>(Bsm + off + 16) = h2pack(v1.x, v1.y);
+      } else if (MODE == 2) {
+        const int col = 2 * (grp0 + x) + p;
+        const float2 g = h2unpack(Gsm[row + k4GStride * col]);
+        v0 = cmul(v0, g);
+        v1 = cmul(v1, g);
+        const uint32_t off = base + x * k4Sbo;
+        *reinterpret_cast<uint32_t*>(Bsm + off) = h2pack(v0.x, -v0.y);
+        *reinterpret_cast<uint32_t*>(Bsm + off + 16) = h2pack(v1.x, -v1.y);
+      } else {
+        uint2 o;
+        o.x = h2pack(v0.x, v0.y);
+        o.y = h2pack(v1.x, v1.y);
+        *reinterpret_cast<uint2*>(out + base + x * 32) = o;
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* Fsm = smem;
+  __shared__ uint32_t tmem_slot;
+
+  const int tid = threadIdx.x, grp = tid / k4GroupThreads, gt = tid - grp * k4GroupThreads;
+  const int warp = gt >> 5, T = gt & 31;
+  unsigned char* Bsm = smem + k4FBytes + grp * k4BBytes;
+  uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + k4FBytes + 2 * k4BBytes + grp * k4GBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + k4FBytes + 2 * k4BBytes + 2 * k4GBytes) + 2 * grp;  // [0] load, [1] MMA
+  const uint32_t barL = s_u32(&bars[0]), barD = s_u32(&bars[1]);
+
+  if (tid < 32) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s_u32(&tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  if (gt == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barL), "r"(1));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barD), "r"(1));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  {
+    const uint4* Fg = reinterpret_cast<const uint4*>(p.F);
+    for (int i = tid; i < k4FBytes / 16; i += k4CoreThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = tmem_slot + 256 * grp;
+  const uint32_t idesc = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+  const int q = warp & 3, ch = warp >> 2;
+
+  __shared__ int gave_up[2];
+  if (gt == 0) gave_up[grp] = 0;
+  asm volatile("bar.sync %0, %1;" :: "r"(1 + grp), "r"(k4GroupThreads) : "memory");
+  bool ok = true;
+  uint32_t phaseL = 0, phaseD = 0;
+  // A wait that runs out is recorded in gave_up[grp]; every thread of the group still reaches every
+  // group barrier, reads the flag there and leaves the loops together.
+  for (int unit = blockIdx.x * 2 + grp; unit < p.nunits && ok; unit += 2 * gridDim.x) {
+    // ---- operand and gate table: bulk async copies, completion counted on barL ----
+    if (gt == 0) {
+      const unsigned char* img = p.ws_in + (size_t)unit * k4ImgBytes;
+      const unsigned char* gim = p.gimg + (size_t)(unit / p.ntile) * k4GBytes;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL), "r"(k4ImgBytes + k4GBytes) : "memory");
+      for (int m = 0; m < 32; ++m)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     :: "r"(s_u32(Bsm + m * k4Sbo)), "l"(img + (size_t)m * 2048), "r"(2048), "r"(barL) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   :: "r"(s_u32(Gsm)), "l"(gim), "r"(k4GBytes), "r"(barL) : "memory");
+    }
+    if (!wait4(barL, phaseL)) gave_up[grp] = 1;
+    phaseL ^= 1;
+    asm volatile("bar.sync %0, %1;" :: "r"(1 + grp), "r"(k4GroupThreads) : "memory");
+    ok = gave_up[grp] == 0;
+#pragma unroll 1
+    for (int stage = 0; stage < 4 && ok; ++stage) {
+      if (gt == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a0 = s_u32(Fsm), b0 = s_u32(Bsm);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint64_t da = desc4(a0 + ks * 256, 128, 2048);
+          const uint64_t db = desc4(b0 + ks * 2 * k4Lbo, k4Lbo, k4Sbo);
+          const uint32_t acc = ks > 0;
+          asm volatile(
+              "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+              :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barD) : "memory");
+      }
+      const bool good = wait4(barD, phaseD);
+      phaseD ^= 1;
+      if (!good) gave_up[grp] = 1;
+      if (good) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (stage == 1) core_epilogue<2>(tmem_d, Bsm, Gsm, nullptr, q, ch, T);
+        else if (stage == 3) core_epilogue<3>(tmem_d, Bsm, Gsm, p.ws_out + (size_t)unit * k4OutBytes, q, ch, T);
+        else core_epilogue<1>(tmem_d, Bsm, Gsm, nullptr, q, ch, T);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      }
+      asm volatile("bar.sync %0, %1;" :: "r"(1 + grp), "r"(k4GroupThreads) : "memory");   // the group's 256 threads
+      ok = gave_up[grp] == 0;
+    }
+  }
+  if (!ok && gt == 0) atomicExch(p.status, 1);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (tid < 32) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_slot), "r"(512));
+  }
+}
+
+// =====================================================================================
+// transpose-out
+// =====================================================================================
+struct TcOutParams {
+  const unsigned char* ws_out;   // [unit][t'][4] half2
+  const float* gscale;           // [slab_local * R + k1]
+  bf16* dst;
+  int64_t d_sb, d_sl, d_sh;
+  int H, D, L, n, ntile, slab0;
+};
+
+// CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.
+template <int R>
+__global__ void __launch_bounds__(256) tc_out_kernel(const TcOutParams p) {
+  constexpr int NT = 512 / R;
+  extern __shared__ __align__(128) uint32_t stage[];            // [R][NT][D/2 words]
+  const int nblk = 4096 / NT;
+  const int tb = blockIdx.x % nblk, slab_local = blockIdx.x / nblk, slab = p.slab0 + slab_local;
+  const int b = slab / p.H, h = slab - b * p.H;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t8 = lane >> 2, c4 = lane & 3;
+  const int npair = p.D / 2;
+  const float base_scale = 1.0f / ((float)R * in_scale(R));
+  const int skew_mask = (p.ntile & (p.ntile - 1)) == 0 ? min(p.ntile, 8) - 1 : 0;   // XOR stays inside the row
+
+  // phase 1: a warp takes (tile, 8 consecutive t'); lane = (t' % 8, pair within the tile)
+  const int nitems = p.ntile * (NT / 8);
+  for (int item = warp; item < nitems; item += 8) {
+    const int tile = item % p.ntile, tl = (item / p.ntile) * 8 + t8;
+    const int tp = tb * NT + tl;
+    float2 x[R];
+#pragma unroll
+    for (int k1 = 0; k1 < R; ++k1) {
+      const size_t unit = ((size_t)slab_local * R + k1) * p.ntile + tile;
+      const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(p.ws_out + unit * k4OutBytes) + tp * 4 + c4);
+      float2 f = h2unpack(v);
+      f.y = -f.y;                                               // result of conj(FFT(conj(.)))
+      x[k1] = cscale(f, __ldg(p.gscale + slab_local * R + k1) * base_scale);
+    }
+    const float2 w1 = twiddle_fwd((unsigned)tp, (unsigned)p.n);
+    float2 w = w1;
+#pragma unroll
+    for (int k = 1; k < R; ++k) {
+      x[k] = cmulc(x[k], w);                                    // times conj(W_n^{k1 t'})
+      w = cmul(w, w1);
+    }
+    Dft<R, true>::run(x);
+#pragma unroll
+    for (int n1 = 0; n1 < R; ++n1) {
+      __nv_bfloat162 o = __floats2bfloat162_rn(x[n1].x, x[n1].y);
+      const int word = (tile * 4 + c4) ^ ((tl & skew_mask) << 2);   // skew: the 8 rows of a warp hit 8 bank groups
+      stage[((size_t)n1 * NT + tl) * npair + word] = *reinterpret_cast<uint32_t*>(&o);
+    }
+  }
+  __syncthreads();
+  // phase 2: whole rows
+  bf16* dst = p.dst + b * p.d_sb + h * p.d_sh;
+  for (int r = warp; r < R * NT; r += 8) {
+    const int n1 = r / NT, tl = r - n1 * NT;
+    const int row = n1 * 4096 + tb * NT + tl;
+    if (row >= p.L) continue;
+    for (int c = lane; c < npair; c += 32) {
+      const uint32_t v = stage[(size_t)r * npair + (c ^ ((tl & skew_mask) << 2))];
+      *reinterpret_cast<uint32_t*>(dst + (int64_t)row * p.d_sl + 2 * c) = v;
+    }
+  }
+}
+
+// =====================================================================================
+// host
+// =====================================================================================
+static size_t tc4k_slab_bytes(int R, int D) {
+  const int ntile = D / 8;
+  return (size_t)R * ntile * (k4ImgBytes + k4OutBytes) + (size_t)R * k4GBytes + 256;
+}
+
+bool tc4k_supported(int n, int D) {
+  if (n < 4096 || n > 131072 || (n & (n - 1))) return false;
+  return D % 8 == 0 && D <= 128;
+}
+
+// Workspace for `group` heads: operand images, unit results, gate images, gate scales.
+size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
+  const int R = n / 4096;
+  size_t per = tc4k_slab_bytes(R, D);
+  size_t budget = (ctx->l2_bytes * 3) / 4;
+  size_t g = budget / per;
+  if (g < 1) g = 1;
+  if (g > (size_t)nslab) g = nslab;
+  return g * per;
+}
+
+template <int R>
+static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                      const spectre_act* y, int n, int slab0, int cnt, unsigned char* ws) {
+  const int D = v->D, ntile = D / 8;
+  const size_t nunits = (size_t)cnt * R * ntile;
+  unsigned char* ws_in = ws;
+  unsigned char* ws_out = ws_in + nunits * k4ImgBytes;
+  unsigned char* gimg = ws_out + nunits * k4OutBytes;
+  float* gscale = reinterpret_cast<float*>(gimg + (size_t)cnt * R * k4GBytes);
+
+  TcGateParams gp = {reinterpret_cast<const float2*>(g), gimg, gscale, n, n / 2 + 1, R, slab0};
+  tc_gate_kernel<<<cnt * R, 256, 0, st>>>(gp);
+  SPECTRE_LAUNCH_OK("tc_gate_kernel");
+
+  constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
+  TcInParams ip = {reinterpret_cast<const bf16*>(v->ptr), v->stride_b, v->stride_l, v->stride_h, ws_in,
+                   v->H, D, v->L, n, ntile, slab0};
+  const size_t smem_in = (size_t)R * ntile * (NT2 / 2) * 128;
+  if (smem_in > 48 * 1024)
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_in));
+  tc_in_kernel<R><<<cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip);
+  SPECTRE_LAUNCH_OK("tc_in_kernel");
+
+  TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64), (int)nunits, ntile,
+                     ctx->status_dev};
+  SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
+  int grid = (int)((nunits + 1) / 2);
+  if (grid > ctx->sm_count) grid = ctx->sm_count;
+  tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
+  SPECTRE_LAUNCH_OK("tc_core_kernel");
+
+  constexpr int NT = 512 / R;
+  TcOutParams op = {ws_out, gscale, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
+                    y->H, D, y->L, n, ntile, slab0};
+  const size_t smem_out = (size_t)R * NT * (D / 2) * 4;
+  if (smem_out > 48 * 1024)
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_out));
+  tc_out_kernel<R><<<cnt * (4096 / NT), 256, smem_out, st>>>(op);
+  SPECTRE_LAUNCH_OK("tc_out_kernel");
+  return SPECTRE_OK;
+}
+
+int launch_mixer_tc4k(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                      const spectre_act* y, int n, void* ws, size_t ws_bytes) {
+  const int R = n / 4096, nslab = v->B * v->H;
+  const size_t per = tc4k_slab_bytes(R, v->D);
+  int group = (int)(ws_bytes / per);
+  const int pref = (int)(tc4k_workspace_bytes(ctx, n, v->D, nslab) / per);
+  if (group > pref) group = pref;
+  if (group < 1) return fail(SPECTRE_ERR_WORKSPACE, "mixer workspace smaller than one (batch, head) slab");
+  unsigned char* w = reinterpret_cast<unsigned char*>(ws);
+  for (int s0 = 0; s0 < nslab; s0 += group) {
+    const int cnt = nslab - s0 < group ? nslab - s0 : group;
+    int rc;
+    switch (R) {
+      case 1: rc = tc4k_group<1>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      case 2: rc = tc4k_group<2>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      case 4: rc = tc4k_group<4>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      case 8: rc = tc4k_group<8>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      case 16: rc = tc4k_group<16>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      case 32: rc = tc4k_group<32>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      default: return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported by the tensor-core path");
+    }
+    if (rc != SPECTRE_OK) return rc;
+  }
+  return SPECTRE_OK;
+}
+
+size_t tc4k_min_workspace(int n, int D) { return tc4k_slab_bytes(n / 4096, D); }
+
+}  // namespace spectre

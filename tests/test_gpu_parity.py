@@ -54,6 +54,38 @@ def test_mixer_bf16(ctx, n, D):
     assert run_mixer(ctx, w) < TOL["bf16"]
 
 
+@pytest.mark.parametrize("path", ["alu", "fused", "staged"])
+def test_mixer_bf16_8192_every_path(ctx, path, monkeypatch):
+    monkeypatch.setenv("SPECTRE_FORCE_PATH", path)
+    w = W.Workload("t", B=1, L=8192, H=3, D=64, dtype="bf16", seed=808)
+    assert run_mixer(ctx, w, structured=True) < TOL["bf16"]
+    torch.cuda.synchronize()
+    ctx.poll_status()                                        # no bounded wait ran out
+
+
+@pytest.mark.parametrize("n,H,D", [(4096, 2, 64), (16384, 2, 64), (32768, 1, 32), (65536, 1, 64), (131072, 1, 16),
+                                   (8192, 2, 40), (4096, 3, 8)])
+def test_mixer_bf16_tensor_core_staged_lengths(ctx, n, H, D):
+    w = W.Workload("t", B=1, L=n, H=H, D=D, dtype="bf16", seed=n + D)
+    assert run_mixer(ctx, w) < TOL["bf16"]
+    torch.cuda.synchronize()
+    ctx.poll_status()
+
+
+def test_mixer_bf16_tensor_core_zero_pad_and_strides(ctx):
+    w = W.Workload("t", B=2, L=6000, H=2, D=64, dtype="bf16", n_fft=8192, seed=61)
+    assert run_mixer(ctx, w, n_fft=8192) < TOL["bf16"]
+    w = W.Workload("t", B=1, L=8192, H=2, D=64, dtype="bf16", seed=62)
+    big = W.activations(W.scaled(w, H=4)).cuda()
+    x = big[:, :, 1:3, :]
+    g = W.random_gate(w).cuda()
+    y = torch.zeros_like(big)
+    S.spectre_mixer_forward(ctx, x, g, y=y[:, :, 2:4, :])
+    ref = O.mixer(W.to_f64(x), gate_to_complex(g))
+    assert slab_err(W.to_f64(y[:, :, 2:4, :]), ref) < TOL["bf16"]
+    assert float(y[:, :, :2].abs().max()) == 0.0
+
+
 def test_mixer_structured_inputs(ctx):
     # per-channel offsets and x30 outlier channels
     for dt in ("f32", "bf16"):
