@@ -105,7 +105,11 @@ typedef struct {
  *   shift      [B] int64 on the DEVICE, or NULL
  *   g_out      [B, H, K, 2] float32
  *   qbar_out   [B, H, D] float32 or NULL (input of the wavelet level-gate MLP)
- *   workspace  spectre_gate_workspace_bytes(...) bytes, 16-byte aligned
+ *   workspace  16-byte aligned; spectre_gate_workspace_bytes(...) is the size at which the
+ *              pooling runs fastest (16 partial copies of the [B, H, D] sums); any size down
+ *              to one copy (4*B*H*D bytes of sums, 4*B*H*hidden of hidden activations, plus
+ *              8*B*H*K with the Toeplitz update on, each rounded up to 256) is accepted;
+ *              with sum_q given the sums part is still counted but unused
  */
 size_t spectre_gate_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
                                     int32_t n_fft, int32_t toeplitz_r);
@@ -134,9 +138,10 @@ int spectre_gate(spectre_ctx* ctx, void* stream,
  * cudaMalloc, cudaFree or any allocating routine; inputs and outputs are still
  * the caller's.
  *
- *   - Shapes whose spectre_gate_workspace_bytes(...) exceeds the array are
- *     rejected with SPECTRE_ERR_UNSUPPORTED and a message that names both sizes
- *     (with the Toeplitz update off the need is 4*B*H*D bytes rounded up to 256).
+ *   - Shapes whose minimum gate scratch (one copy of the sums; see spectre_gate)
+ *     exceeds the array are rejected with SPECTRE_ERR_UNSUPPORTED and a message
+ *     that names both sizes (with the Toeplitz update off the need is 4*B*H*D
+ *     plus 4*B*H*hidden bytes, each rounded up to 256).
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress); make that first call before starting any stream
  *     capture on that device.

@@ -8,7 +8,7 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
                      float2* ws, int* N1_out, int* M_out);
 bool transform_supported(const spectre_ctx* ctx, int n);
 size_t transform_slab_bytes(int n, int D);
-int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums);
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy);
 
 // ---- prefill -----------------------------------------------------------------
 // The forward pass leaves Z = fft_n(a + jb) for each column pair (a, b) in
@@ -203,7 +203,7 @@ extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, cons
                                                      q->stride_h, reinterpret_cast<float*>(cache->Q_buf), B, N, H, D, q->L);
   }
   SPECTRE_LAUNCH_OK("ring_fill_kernel");
-  return pool_sum(ctx, st, q, cache->sum_q);
+  return pool_sum(ctx, st, q, cache->sum_q, 1);
 }
 
 extern "C" int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const spectre_cache* cache, const void* q_t,

@@ -1,68 +1,85 @@
 // Content-adaptive spectral gate (Sec. 3.2 step 3; Sec. 3.3.2 steps c-d).
 //   pool_kernel      sum of the query tokens over the sequence (bandwidth-bound)
-//   gate_mlp_kernel  LayerNorm + two-layer MLP; with the Toeplitz update off it
-//                    also applies modReLU and the positional phase
+//   gate_hidden_kernel LayerNorm + hidden layer, once per (batch, head)
+//   gate_out_kernel    output layer as a stream over W2; with the Toeplitz update off
+//                      it also applies modReLU and the positional phase
 //   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
 #include "common.cuh"
 
 namespace spectre {
 
 // ---- pooled sum over the sequence --------------------------------------------
-// Grid (chunks, B).  A thread owns one 8-channel vector of the [H*D] row and
-// walks the chunk's rows; partial sums are combined with float atomics into
-// sums[B,H,D] (zeroed by the caller on the same stream).
+// Grid (slices, B).  A thread owns one 8-channel vector of the [H*D] row (several rows are in
+// flight when the row is narrower than the CTA) and walks the slice's rows with 8 loads in
+// flight; partial sums go with float atomics into copy (slice mod ncopy) of sums[ncopy][B,H,D]
+// (zeroed by the caller on the same stream), which keeps the contention per address low.
+template <typename T> struct vec8;
+template <> struct vec8<bf16> {
+  static __device__ __forceinline__ void add(const bf16* p, float (&a)[8]) {
+    const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      a[2 * i] += __uint_as_float(u[i] << 16);
+      a[2 * i + 1] += __uint_as_float(u[i] & 0xffff0000u);
+    }
+  }
+};
+template <> struct vec8<float> {
+  static __device__ __forceinline__ void add(const float* p, float (&a)[8]) {
+    const float4 lo = __ldg(reinterpret_cast<const float4*>(p)), hi = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    a[0] += lo.x; a[1] += lo.y; a[2] += lo.z; a[3] += lo.w;
+    a[4] += hi.x; a[5] += hi.y; a[6] += hi.z; a[7] += hi.w;
+  }
+};
+
 template <typename T>
 __global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
-                                                   int H, int D, int rows_per, float* __restrict__ sums) {
+                                                   int H, int D, int rows_per, int ncopy, size_t copy_stride,
+                                                   float* __restrict__ sums) {
   const int b = blockIdx.y;
   const int r0 = blockIdx.x * rows_per;
   const int r1 = min(L, r0 + rows_per);
   const int vec_per_head = D / 8;
   const int nvec = H * vec_per_head;
-  for (int vi = threadIdx.x; vi < nvec; vi += blockDim.x) {
-    int h = vi / vec_per_head, c = (vi - h * vec_per_head) * 8;
+  const int rif = nvec >= 256 ? 1 : 256 / nvec;              // rows in flight across the CTA
+  const int ro = nvec >= 256 ? 0 : (int)threadIdx.x / nvec;
+  if (ro >= rif) return;
+  float* dst_copy = sums + (size_t)(blockIdx.x % ncopy) * copy_stride + (size_t)b * H * D;
+  for (int vi = nvec >= 256 ? threadIdx.x : (int)threadIdx.x - ro * nvec; vi < nvec; vi += 256) {
+    const int h = vi / vec_per_head, c = (vi - h * vec_per_head) * 8;
     const T* base = q + b * sb + h * sh + c;
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    int r = r0;
-    for (; r + 4 <= r1; r += 4) {
-      float4 v[8];
+    int r = r0 + ro;
+    for (; r + 7 * rif < r1; r += 8 * rif) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        v[2 * u] = io<T>::load4(base + (int64_t)(r + u) * sl);
-        v[2 * u + 1] = io<T>::load4(base + (int64_t)(r + u) * sl + 4);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        acc[0] += v[2 * u].x; acc[1] += v[2 * u].y; acc[2] += v[2 * u].z; acc[3] += v[2 * u].w;
-        acc[4] += v[2 * u + 1].x; acc[5] += v[2 * u + 1].y; acc[6] += v[2 * u + 1].z; acc[7] += v[2 * u + 1].w;
-      }
+      for (int u = 0; u < 8; ++u) vec8<T>::add(base + (int64_t)(r + u * rif) * sl, acc);
     }
-    for (; r < r1; ++r) {
-      float4 v0 = io<T>::load4(base + (int64_t)r * sl), v1 = io<T>::load4(base + (int64_t)r * sl + 4);
-      acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
-      acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
-    }
-    float* dst = sums + ((size_t)b * H + h) * D + c;
+    for (; r < r1; r += rif) vec8<T>::add(base + (int64_t)r * sl, acc);
+    float* dst = dst_copy + h * D + c;
 #pragma unroll
     for (int i = 0; i < 8; ++i) atomicAdd(dst + i, acc[i]);
+    if (nvec < 256) break;
   }
 }
 
-int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums) {
-  SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, (size_t)q->B * q->H * q->D * sizeof(float), st));
-  int target = (4 * ctx->sm_count + q->B - 1) / q->B;
+// Sums of q over the sequence into `ncopy` partial copies (the consumer adds them up).
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy) {
+  const size_t copy_stride = (size_t)q->B * q->H * q->D;
+  SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, copy_stride * ncopy * sizeof(float), st));
+  int target = (2 * ctx->sm_count + q->B - 1) / q->B;
   if (target < 1) target = 1;
   int rows_per = (q->L + target - 1) / target;
-  if (rows_per < 16) rows_per = 16;
+  if (rows_per < 32) rows_per = 32;
   dim3 grid((q->L + rows_per - 1) / rows_per, q->B);
   if (q->dtype == SPECTRE_BF16)
     pool_kernel<bf16><<<grid, 256, 0, st>>>(reinterpret_cast<const bf16*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
-                                             q->L, q->H, q->D, rows_per, sums);
+                                             q->L, q->H, q->D, rows_per, ncopy, copy_stride, sums);
   else
     pool_kernel<float><<<grid, 256, 0, st>>>(reinterpret_cast<const float*>(q->ptr), q->stride_b, q->stride_l,
-                                              q->stride_h, q->L, q->H, q->D, rows_per, sums);
+                                              q->stride_h, q->L, q->H, q->D, rows_per, ncopy, copy_stride, sums);
   SPECTRE_LAUNCH_OK("pool_kernel");
   return SPECTRE_OK;
 }
@@ -92,13 +109,22 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the
 // hidden layer u = GELU(q_bar W1 + b1).
 template <typename WT>
-__device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, float inv_count, int D, int hidden,
+__device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, int ncopy, size_t copy_stride,
+                                                      float inv_count, int D, int hidden,
                                                       const float* __restrict__ gamma, const float* __restrict__ beta,
                                                       float eps, const WT* __restrict__ W1, const float* __restrict__ b1,
                                                       float* qbar, float* u, float* red) {
   float part = 0.f;
   for (int c = threadIdx.x; c < D; c += blockDim.x) {
-    float m = sums[c] * inv_count;
+    float m = 0.f;
+    for (int k0 = 0; k0 < ncopy; k0 += 16) {        // all copies in flight at once
+      float v[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) v[k] = (k0 + k < ncopy) ? sums[(size_t)(k0 + k) * copy_stride + c] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) m += v[k];
+    }
+    m *= inv_count;
     qbar[c] = m;
     part += m;
   }
@@ -114,7 +140,15 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
   __syncthreads();
   for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
     float acc = b1[j];
-    for (int c = 0; c < D; ++c) acc = fmaf(qbar[c], wload<WT>(W1 + (size_t)c * hidden + j), acc);
+    int c = 0;
+    for (; c + 32 <= D; c += 32) {                  // 32 independent loads in flight
+      float wv[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + j);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc = fmaf(qbar[c + i], wv[i], acc);
+    }
+    for (; c < D; ++c) acc = fmaf(qbar[c], wload<WT>(W1 + (size_t)c * hidden + j), acc);
     u[j] = gelu_erf(acc);
   }
   __syncthreads();
@@ -135,7 +169,8 @@ __device__ __forceinline__ float2 modrelu_phase(float2 gk, float bias, int k, in
 }
 
 struct GateMlpParams {
-  const float* sums;      // [B,H,D]
+  const float* sums;      // [ncopy][B,H,D]
+  int ncopy; size_t copy_stride;
   float inv_count;
   int H, D, hidden, n, K;
   size_t hs_ln, hs_w1, hs_b1, hs_w2, hs_b2, hs_mb;   // per-head strides (0 when shared)
@@ -145,40 +180,80 @@ struct GateMlpParams {
   const long long* shift; long long shift_all;
   float2* g_out;          // final gate, or the raw MLP output when post != 0
   float* qbar_out;
+  float* u_ws;            // [B,H,hidden] hidden activations (workspace)
   int post;               // 1: Toeplitz follows, skip modReLU/phase here
 };
 
+// LayerNorm + hidden layer once per (batch, head): u[B,H,hidden] (and q_bar for the caller).
 template <typename WT>
-__global__ void __launch_bounds__(256) gate_mlp_kernel(const GateMlpParams p) {
+__global__ void __launch_bounds__(128) gate_hidden_kernel(const GateMlpParams p) {
   extern __shared__ float smf[];
   float* qbar = smf;                 // [D]
   float* u = smf + p.D;              // [hidden]
   float* red = u + p.hidden;         // [32]
-  const int bh = blockIdx.y, b = bh / p.H, h = bh - b * p.H;
+  const int bh = blockIdx.x, h = bh % p.H;
   const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-  const WT* W2 = reinterpret_cast<const WT*>(p.W2) + h * p.hs_w2;
-  descriptor_and_hidden<WT>(p.sums + (size_t)bh * p.D, p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln,
-                            p.beta + h * p.hs_ln, p.eps, W1, p.b1 + h * p.hs_b1, qbar, u, red);
-  if (p.qbar_out && blockIdx.x == 0)
+  descriptor_and_hidden<WT>(p.sums + (size_t)bh * p.D, p.ncopy, p.copy_stride, p.inv_count, p.D, p.hidden,
+                            p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1, p.b1 + h * p.hs_b1, qbar, u, red);
+  if (p.qbar_out)
     for (int c = threadIdx.x; c < p.D; c += blockDim.x) p.qbar_out[(size_t)bh * p.D + c] = qbar[c];
+  for (int j = threadIdx.x; j < p.hidden; j += blockDim.x) p.u_ws[(size_t)bh * p.hidden + j] = u[j];
+}
 
+// raw (re, im) weight pair of one bin in one hidden row
+template <typename WT> struct wraw;
+template <> struct wraw<bf16> {
+  typedef unsigned type;
+  static __device__ __forceinline__ type load(const bf16* p) { return __ldg(reinterpret_cast<const unsigned*>(p)); }
+  static __device__ __forceinline__ float2 cvt(type r) { return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u)); }
+  static constexpr int kRows = 64;
+};
+template <> struct wraw<float> {
+  typedef float2 type;
+  static __device__ __forceinline__ type load(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
+  static __device__ __forceinline__ float2 cvt(type r) { return r; }
+  static constexpr int kRows = 32;
+};
+
+// Output layer: grid (ceil(K / 256), B*H), one bin per thread.  A thread issues the loads of up
+// to kRows hidden rows of its W2 column before it uses any of them, so the whole column is one
+// memory round trip; the kernel is a pure stream over W2.
+template <typename WT>
+__global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
+  extern __shared__ float u[];       // [hidden]
+  constexpr int R = wraw<WT>::kRows;
+  const int bh = blockIdx.y, b = bh / p.H, h = bh - b * p.H;
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= p.K) return;
+  const bool live = k < p.K;
+  const WT* col = reinterpret_cast<const WT*>(p.W2) + h * p.hs_w2 + 2 * (size_t)(live ? k : 0);
+  const size_t ld = 2 * (size_t)p.K;
+  typename wraw<WT>::type w[R];
+  const int n0 = min(R, p.hidden);
+  if (live) {
+#pragma unroll
+    for (int i = 0; i < R; ++i)
+      if (i < n0) w[i] = wraw<WT>::load(col + (size_t)i * ld);
+  }
+  for (int j = threadIdx.x; j < p.hidden; j += blockDim.x) u[j] = p.u_ws[(size_t)bh * p.hidden + j];
+  __syncthreads();
+  if (!live) return;
   const float* b2 = p.b2 + h * p.hs_b2;
   float2 acc = make_float2(b2[2 * k], b2[2 * k + 1]);
-  const size_t ld = 2 * (size_t)p.K;
-  const WT* col = W2 + 2 * (size_t)k;
-  int j = 0;
-  for (; j + 8 <= p.hidden; j += 8) {
-    float2 w[8];
+  for (int j = 0; j < p.hidden; j += R) {
+    const int nb = min(R, p.hidden - j);
+    if (j > 0) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] = wload2<WT>(col + (size_t)(j + i) * ld);
+      for (int i = 0; i < R; ++i)
+        if (i < nb) w[i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
+    }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { acc.x = fmaf(u[j + i], w[i].x, acc.x); acc.y = fmaf(u[j + i], w[i].y, acc.y); }
-  }
-  for (; j < p.hidden; ++j) {
-    float2 w = wload2<WT>(col + (size_t)j * ld);
-    acc.x = fmaf(u[j], w.x, acc.x); acc.y = fmaf(u[j], w.y, acc.y);
+    for (int i = 0; i < R; ++i) {
+      if (i < nb) {
+        const float2 wv = wraw<WT>::cvt(w[i]);
+        acc.x = fmaf(u[j + i], wv.x, acc.x);
+        acc.y = fmaf(u[j + i], wv.y, acc.y);
+      }
+    }
   }
   if (!p.post) {
     long long sh = p.shift_all + (p.shift ? p.shift[b] : 0);
@@ -216,11 +291,15 @@ __global__ void __launch_bounds__(256) gate_post_kernel(const GatePostParams p) 
   p.g_out[(size_t)bh * p.K + k] = modrelu_phase(acc, bias, k, p.n, (unsigned)pm);
 }
 
-static size_t gate_ws_layout(int B, int H, int D, int n_fft, int r, size_t* raw_off) {
-  size_t sums = align_up((size_t)B * H * D * sizeof(float), 256);
-  *raw_off = sums;
+constexpr int kPoolCopies = 16;      // partial copies of the pooled sum in a full-size workspace
+
+// Layout: [raw gate (Toeplitz only)] [hidden activations] [ncopy x pooled sums].  ncopy = 1 is the minimum.
+static size_t gate_ws_layout(int B, int H, int D, int n_fft, int r, int hidden, int ncopy, size_t* u_off,
+                             size_t* sums_off) {
   size_t raw = r > 0 ? align_up((size_t)B * H * (n_fft / 2 + 1) * sizeof(float2), 256) : 0;
-  return sums + raw;
+  *u_off = raw;
+  *sums_off = raw + align_up((size_t)B * H * hidden * sizeof(float), 256);
+  return *sums_off + align_up((size_t)ncopy * B * H * D * sizeof(float), 256);
 }
 
 }  // namespace spectre
@@ -231,8 +310,8 @@ extern "C" size_t spectre_gate_workspace_bytes(const spectre_ctx* ctx, int32_t B
                                                int32_t toeplitz_r) {
   (void)ctx;
   if (B < 1 || H < 1 || D < 1 || n_fft < 1 || toeplitz_r < 0) return 0;
-  size_t off;
-  return gate_ws_layout(B, H, D, n_fft, toeplitz_r, &off);
+  size_t off, off2;
+  return gate_ws_layout(B, H, D, n_fft, toeplitz_r, 1024, kPoolCopies, &off, &off2);   // any hidden width
 }
 
 extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q, const float* sum_q, int32_t B,
@@ -263,9 +342,9 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   }
   const int K = n_fft / 2 + 1;
   const int r = gp->toeplitz_r;
-  size_t raw_off;
-  const size_t need = gate_ws_layout(B, H, D, n_fft, r, &raw_off);
-  const bool need_ws = (q != nullptr) || r > 0;
+  size_t sums_off, u_off;
+  const size_t need = gate_ws_layout(B, H, D, n_fft, r, gp->hidden, 1, &u_off, &sums_off);   // one copy is enough
+  const bool need_ws = true;
   if (need_ws) {
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15))
       return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
@@ -274,15 +353,19 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const float* sums = sum_q;
+  int ncopy = 1;
   if (q) {
-    float* pooled = reinterpret_cast<float*>(workspace);
-    int rc = pool_sum(ctx, st, q, pooled);
+    float* pooled = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + sums_off);
+    const size_t one_copy = (size_t)B * H * D * sizeof(float);
+    size_t fit = (workspace_bytes - sums_off) / one_copy;
+    ncopy = fit > (size_t)kPoolCopies ? kPoolCopies : (int)fit;
+    int rc = pool_sum(ctx, st, q, pooled, ncopy);
     if (rc != SPECTRE_OK) return rc;
     sums = pooled;
   }
   const size_t one = gp->shared_across_heads ? 0 : 1;
   GateMlpParams mp = {};
-  mp.sums = sums; mp.inv_count = inv_count;
+  mp.sums = sums; mp.ncopy = ncopy; mp.copy_stride = (size_t)B * H * D; mp.inv_count = inv_count;
   mp.H = H; mp.D = D; mp.hidden = gp->hidden; mp.n = n_fft; mp.K = K;
   mp.hs_ln = one * D; mp.hs_w1 = one * (size_t)D * gp->hidden; mp.hs_b1 = one * gp->hidden;
   mp.hs_w2 = one * (size_t)gp->hidden * 2 * K; mp.hs_b2 = one * 2 * (size_t)K; mp.hs_mb = one * K;
@@ -291,15 +374,21 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   mp.modrelu_bias = gp->modrelu_bias;
   mp.shift = reinterpret_cast<const long long*>(shift); mp.shift_all = shift_all;
   mp.qbar_out = qbar_out;
+  mp.u_ws = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + u_off);
   mp.post = r > 0;
-  float2* raw = r > 0 ? reinterpret_cast<float2*>(reinterpret_cast<char*>(workspace) + raw_off) : nullptr;
+  float2* raw = r > 0 ? reinterpret_cast<float2*>(workspace) : nullptr;
   mp.g_out = r > 0 ? raw : reinterpret_cast<float2*>(g_out);
   dim3 grid((K + 255) / 256, B * H);
   if (grid.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H exceeds 65535");
   size_t smem = (size_t)(D + gp->hidden + 32) * sizeof(float);
-  if (gp->wdtype == SPECTRE_BF16) gate_mlp_kernel<bf16><<<grid, 256, smem, st>>>(mp);
-  else gate_mlp_kernel<float><<<grid, 256, smem, st>>>(mp);
-  SPECTRE_LAUNCH_OK("gate_mlp_kernel");
+  if (gp->wdtype == SPECTRE_BF16) {
+    gate_hidden_kernel<bf16><<<B * H, 128, smem, st>>>(mp);
+    gate_out_kernel<bf16><<<grid, 256, gp->hidden * sizeof(float), st>>>(mp);
+  } else {
+    gate_hidden_kernel<float><<<B * H, 128, smem, st>>>(mp);
+    gate_out_kernel<float><<<grid, 256, gp->hidden * sizeof(float), st>>>(mp);
+  }
+  SPECTRE_LAUNCH_OK("gate_hidden_kernel / gate_out_kernel");
   if (r > 0) {
     GatePostParams pp = {};
     pp.g_raw = raw; pp.g_out = reinterpret_cast<float2*>(g_out);
@@ -349,7 +438,8 @@ extern "C" int spectre_gate_static(spectre_ctx* ctx, void* stream, const spectre
   if (!gp) return fail(SPECTRE_ERR_INVALID_ARG, "gate parameters are NULL");
   if (B < 1 || H < 1 || D < 1 || n_fft < 1 || gp->toeplitz_r < 0)
     return fail(SPECTRE_ERR_INVALID_ARG, "B, H, D, n_fft must be positive");
-  const size_t need = spectre_gate_workspace_bytes(ctx, B, H, D, n_fft, gp->toeplitz_r);
+  size_t off_a, off_b;
+  const size_t need = gate_ws_layout(B, H, D, n_fft, gp->toeplitz_r, gp->hidden, 1, &off_a, &off_b);   // one copy of the sums
   if (need > SPECTRE_GATE_STATIC_BYTES)
     return fail(SPECTRE_ERR_UNSUPPORTED,
                 "spectre_gate_static: this shape needs " + std::to_string(need) + " bytes of scratch, the built-in array holds " +

@@ -31,7 +31,9 @@ constexpr int kTcLbo = 144;                    // bytes between core matrices al
 constexpr int kTcSbo = 2320;                   // bytes between 8-column groups (16 * 144 + 16 pad)
 constexpr int kTcBBytes = 32 * kTcSbo;         // one 256-column B operand
 constexpr int kTcFBytes = 128 * 128 * 2;
-constexpr int kTcSmem = kTcFBytes + 2 * kTcBBytes + 64;
+constexpr int kTcGStride = 72;                 // gate table: entry (row, col) at row + 72 col (conflict-free reads)
+constexpr int kTcGBytes = 64 * kTcGStride * 4; // per half, fp16 (re, im)
+constexpr int kTcSmem = kTcFBytes + 2 * kTcBBytes + 2 * kTcGBytes + 64;
 constexpr int kTcEpiWarps = 16;                // 4 per TMEM lane quadrant, one column quarter each
 constexpr int kTcEpiThreads = 32 * kTcEpiWarps;
 constexpr int kTcThreads = kTcEpiThreads + 32; // + 1 MMA-issuing warp
@@ -122,7 +124,7 @@ __device__ __forceinline__ float2 gate8192(const float2* __restrict__ g, int k) 
 //   MODE 2: gate (and conjugate for the inverse), write straight (col digit -> column index, row digit -> K)
 template <int MODE>
 __device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm, int q, int cq, int T,
-                                             const float2 (&G)[16], float ginv) {
+                                             const uint32_t* __restrict__ Gtab) {
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
@@ -157,7 +159,9 @@ __device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm
         w = cmul(w, wstep);
         off = base + (x >> 1) * kTcLbo + (x & 1) * 8;
       } else {
-        const float2 g = cscale(G[4 * step + x], ginv);
+        const int col = 2 * (8 * cq + 4 * chunk + x) + p;
+        const uint32_t gu = Gtab[row + kTcGStride * col];
+        const float2 g = __half22float2(*reinterpret_cast<const __half2*>(&gu));
         v0 = cmul(v0, g);
         v1 = cmul(v1, g);
         v0.y = -v0.y;
@@ -166,21 +170,6 @@ __device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm
       }
       *reinterpret_cast<uint32_t*>(Bsm + off) = pack_h2(v0.x, v0.y);
       *reinterpret_cast<uint32_t*>(Bsm + off + 16) = pack_h2(v1.x, v1.y);
-    }
-  }
-}
-
-// Gate values one thread needs in the MODE 2 epilogue of one half: bin 2 (col + 64 row) + parity.
-__device__ __forceinline__ void fetch_gate(const float2* __restrict__ g, int q, int cq, int T, int parity,
-                                           float2 (&G)[16]) {
-  const int i = T >> 2, p = (T >> 1) & 1;
-#pragma unroll
-  for (int step = 0; step < 4; ++step) {
-    const int row = 8 * (2 * q + (step >> 1)) + i;
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const int col = 2 * (8 * cq + 4 * (step & 1) + x) + p;
-      G[4 * step + x] = gate8192(g, 2 * (col + 64 * row) + parity);
     }
   }
 }
@@ -197,7 +186,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* Fsm = smem;
   unsigned char* Bsm[2] = {smem + kTcFBytes, smem + kTcFBytes + kTcBBytes};
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + 2 * kTcBBytes);   // [0,1] B ready, [2,3] D ready
+  uint32_t* Gsm[2] = {reinterpret_cast<uint32_t*>(smem + kTcFBytes + 2 * kTcBBytes),
+                      reinterpret_cast<uint32_t*>(smem + kTcFBytes + 2 * kTcBBytes + kTcGBytes)};
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + 2 * kTcBBytes + 2 * kTcGBytes);   // [0,1] B ready, [2,3] D ready
   __shared__ uint32_t tmem_slot;
   __shared__ float red[kTcEpiWarps];
 
@@ -219,26 +210,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[3])), "r"(1));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // DFT matrix -> smem; max |g| of this head (fp16 range management)
-  float gmax = 0.f;
+  // DFT matrix -> smem
   if (tid < kTcEpiThreads) {
     const uint4* Fg = reinterpret_cast<const uint4*>(p.F);
     for (int i = tid; i < kTcFBytes / 16; i += kTcEpiThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
-    for (int k = tid; k <= 4096; k += kTcEpiThreads) {
-      float2 v = __ldg(g + k);
-      gmax = fmaxf(gmax, fmaxf(fabsf(v.x), fabsf(v.y)));
-    }
-    for (int o = 16; o > 0; o >>= 1) gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
-    if (T == 0) red[warp] = gmax;
   }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = tmem_slot;
-  gmax = 0.f;
-  for (int i = 0; i < kTcEpiWarps; ++i) gmax = fmaxf(gmax, red[i]);
-  gmax *= 1.41421356f;                                   // bound on |g_k|
-  const float ginv = gmax > 0.f ? 1.0f / gmax : 0.f;
   TC_STAMP(1);
 
   if (warp == kTcEpiWarps) {
@@ -280,8 +261,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
       for (int it = 0; it < kIter; ++it) {
         const int t2 = t2base + (kTcEpiThreads / 64) * it, t = 64 * t1 + t2;
         uint4 ra = make_uint4(0u, 0u, 0u, 0u), rb = ra;
-        if (t < p.L) ra = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl));
-        if (t + 4096 < p.L) rb = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)(t + 4096) * p.s_sl));
+        if (t < p.L) ra = __ldcg(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl));
+        if (t + 4096 < p.L) rb = __ldcg(reinterpret_cast<const uint4*>(src + (int64_t)(t + 4096) * p.s_sl));
         const uint32_t ua[4] = {ra.x, ra.y, ra.z, ra.w}, ub[4] = {rb.x, rb.y, rb.z, rb.w};
         const uint32_t off = b_off(4 * t2, 2 * t1);
 #pragma unroll
@@ -300,21 +281,42 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
     mbar_arrive(smem_u32(&bars[0]));
     mbar_arrive(smem_u32(&bars[1]));
 
+    // ---- gate tables (while the first MMAs run): Hermitian extension, normalised by a bound on
+    //      max |g| so that the gated spectrum stays in fp16 range; entry for bin 2 (col + 64 row) + parity
+    float gmax = 0.f;
+    constexpr int kGIter = 8192 / kTcEpiThreads;                 // table entries per thread
+    float2 gv[kGIter];
+#pragma unroll
+    for (int i = 0; i < kGIter; ++i) gv[i] = gate8192(g, tid + i * kTcEpiThreads);   // all loads in flight
+#pragma unroll
+    for (int i = 0; i < kGIter; ++i) gmax = fmaxf(gmax, fmaxf(fabsf(gv[i].x), fabsf(gv[i].y)));
+    for (int o = 16; o > 0; o >>= 1) gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
+    if (T == 0) red[warp] = gmax;
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+    gmax = 0.f;
+    for (int i = 0; i < kTcEpiWarps; ++i) gmax = fmaxf(gmax, red[i]);
+    gmax *= 1.41421356f;
+    const float ginv = gmax > 0.f ? 1.0f / gmax : 0.f;
+#pragma unroll
+    for (int i = 0; i < kGIter; ++i) {
+      const int k = tid + i * kTcEpiThreads, m = k >> 1;
+      Gsm[k & 1][(m >> 6) + kTcGStride * (m & 63)] = pack_h2(gv[i].x * ginv, gv[i].y * ginv);
+    }
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+
     const int q = warp & 3, cq = warp >> 2;
     bool ok = true;
-    float2 G[16];
     // ---- stages 1..3: wait for D, transform, hand the next operand to the issuer ----
 #pragma unroll 1
     for (int stage = 0; stage < 3 && ok; ++stage) {
 #pragma unroll 1
       for (int half = 0; half < 2 && ok; ++half) {
-        if (stage == 1) fetch_gate(g, q, cq, T, half, G);   // in flight while the MMAs finish
         ok = mbar_wait(smem_u32(&bars[2 + half]), stage & 1);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t td = tmem + 256 * half;
-        if (stage == 1) epilogue_mid<2>(td, Bsm[half], q, cq, T, G, ginv);
-        else epilogue_mid<1>(td, Bsm[half], q, cq, T, G, ginv);
+        if (stage == 1) epilogue_mid<2>(td, Bsm[half], q, cq, T, Gsm[half]);
+        else epilogue_mid<1>(td, Bsm[half], q, cq, T, Gsm[half]);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         TC_STAMP(3 + 2 * stage + half);

@@ -21,6 +21,8 @@
 // The workspace between the kernels is sized so that a group of heads stays in L2.
 #include <cuda_fp16.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace spectre {
@@ -29,13 +31,14 @@ namespace spectre {
 constexpr int k4Lbo = 128;                       // bytes between core matrices along K
 constexpr int k4Sbo = 2064;                      // bytes between 8-column groups (2048 + 16 pad)
 constexpr int k4BBytes = 32 * k4Sbo;             // one 256-column operand in shared memory
-constexpr int k4ImgBytes = 65536;                // the same operand in the workspace (unpadded)
+constexpr int k4ImgBytes = k4BBytes;             // the workspace holds the same image, padding included
 constexpr int k4FBytes = 128 * 128 * 2;
 constexpr int k4GStride = 72;                    // gate table: entry (row, col) at row + 72 col
 constexpr int k4GBytes = 64 * k4GStride * 4;
 constexpr int k4OutBytes = 4096 * 4 * 4;         // unit result: [t'][4 pairs] half2
-constexpr int k4GroupThreads = 256;
-constexpr int k4CoreThreads = 2 * k4GroupThreads;
+constexpr int k4EpiWarps = 16;
+constexpr int k4EpiThreads = 32 * k4EpiWarps;
+constexpr int k4CoreThreads = k4EpiThreads + 32;    // + producer / MMA-issuing warp
 constexpr int k4CoreSmem = k4FBytes + 2 * k4BBytes + 2 * k4GBytes + 64;
 constexpr uint32_t k4SpinLimit = 1u << 24;
 
@@ -98,7 +101,7 @@ struct TcInParams {
 // A warp takes one (t1, t2) at a time with lane = column pair; staging holds, for every
 // (k1, tile), the core matrices (8 operand columns x 16 bytes) of this CTA's slice.
 template <int R>
-__global__ void __launch_bounds__(256) tc_in_kernel(const TcInParams p) {
+__global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
   extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][NT2/2][32 words]
@@ -120,13 +123,15 @@ __global__ void __launch_bounds__(256) tc_in_kernel(const TcInParams p) {
 #pragma unroll UNR
     for (int rs = warp; rs < 4 * NT2; rs += 8) {
       const int t1m = rs & 3, t2l = rs >> 2;
-      const int t1 = 4 * t1g + t1m, t2 = t2b * NT2 + t2l, tp = 64 * t1 + t2;
+      const int tp = 64 * (4 * t1g + t1m) + t2b * NT2 + t2l;
+      // rows n1 * 4096 + t' are a constant stride apart; rows >= L read as zero
+      const uint32_t* pl = reinterpret_cast<const uint32_t*>(src + (int64_t)tp * p.s_sl + 2 * c);
+      const int64_t lstride = 2048 * p.s_sl;                     // 4096 rows, in 32-bit words
+      const int nvalid = live ? (p.L - tp + 4095) >> 12 : 0;     // number of n1 with a row below L
       float2 x[R];
 #pragma unroll
       for (int n1 = 0; n1 < R; ++n1) {
-        const int row = n1 * 4096 + tp;
-        uint32_t v = 0u;
-        if (live && row < p.L) v = __ldg(reinterpret_cast<const uint32_t*>(src + (int64_t)row * p.s_sl + 2 * c));
+        const uint32_t v = n1 < nvalid ? __ldg(pl + n1 * lstride) : 0u;
         x[n1] = make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
       }
       Dft<R, false>::run(x);
@@ -134,11 +139,13 @@ __global__ void __launch_bounds__(256) tc_in_kernel(const TcInParams p) {
       if (live) {
         // word inside the 128-byte core matrix: (t2 % 2, c4, t1 % 4), XOR-skewed by the tile
         const int wl = ((t2l & 1) * 16 + c4 * 4 + t1m) ^ tile_skew(tile);
+        uint32_t* ps = stage + (tile * (NT2 / 2) + (t2l >> 1)) * 32 + wl;
+        const int sstride = p.ntile * (NT2 / 2) * 32;             // words between consecutive k1
         float2 w = make_float2(sc, 0.f);                          // sc * W_n^{k1 t'}
 #pragma unroll
         for (int k1 = 0; k1 < R; ++k1) {
           const float2 v = cmul(x[k1], w);
-          stage[(((size_t)k1 * p.ntile + tile) * (NT2 / 2) + (t2l >> 1)) * 32 + wl] = h2pack(v.x, v.y);
+          ps[k1 * sstride] = h2pack(v.x, v.y);
           w = cmul(w, w1);
         }
       }
@@ -147,15 +154,22 @@ __global__ void __launch_bounds__(256) tc_in_kernel(const TcInParams p) {
   __syncthreads();
   // copy out: one 128-byte line per (k1, tile, t2 pair)
   const int nlines = R * p.ntile * (NT2 / 2);
-  for (int line = warp; line < nlines; line += 8) {
-    int l = line;
-    const int t2p = l % (NT2 / 2);  l /= (NT2 / 2);
-    const int tile = l % p.ntile, k1 = l / p.ntile;
-    const uint32_t v = stage[(size_t)line * 32 + (lane ^ tile_skew(tile))];
-    const size_t unit = ((size_t)slab_local * R + k1) * p.ntile + tile;
-    const int t2pair = t2b * (NT2 / 2) + t2p;                  // operand column group nu / 8
-    unsigned char* dst = p.ws_in + unit * k4ImgBytes + (size_t)t2pair * 2048 + (size_t)t1g * 128;
-    reinterpret_cast<uint32_t*>(dst)[lane] = v;
+  // 16-byte chunks: chunk index = line * 8 + q; (k1, tile) pairs are consecutive units, so
+  // line -> unit is a shift.  The tile skew permutes words inside a chunk (low two bits) and
+  // swaps the two 64-byte halves of the line (bit 4).
+  unsigned char* img0 = p.ws_in + (size_t)slab_local * R * p.ntile * k4ImgBytes + (size_t)(t2b * (NT2 / 2)) * k4Sbo +
+                        (size_t)t1g * k4Lbo;
+  const bool pow2 = (p.ntile & (p.ntile - 1)) == 0;
+  for (int idx = threadIdx.x; idx < nlines * 8; idx += 256) {
+    const int line = idx >> 3, q16 = idx & 7;
+    const int t2p = line & (NT2 / 2 - 1), ut = line / (NT2 / 2);     // ut = k1 * ntile + tile
+    const int tile = pow2 ? (ut & (p.ntile - 1)) : (ut % p.ntile);
+    const int sk = tile_skew(tile);
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + line * 32 + ((q16 ^ (sk >> 2)) << 2));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint4 o;
+    o.x = w[0 ^ (sk & 3)]; o.y = w[1 ^ (sk & 3)]; o.z = w[2 ^ (sk & 3)]; o.w = w[3 ^ (sk & 3)];
+    *reinterpret_cast<uint4*>(img0 + (size_t)ut * k4ImgBytes + t2p * k4Sbo + q16 * 16) = o;
   }
 }
 
@@ -175,14 +189,20 @@ __global__ void __launch_bounds__(256) tc_gate_kernel(const TcGateParams p) {
   const int sk = blockIdx.x, slab_local = sk / p.R, k1 = sk - slab_local * p.R;
   const float2* g = p.g + (size_t)(p.slab0 + slab_local) * p.K;
   float m = 0.f;
-  for (int kM = threadIdx.x; kM < 4096; kM += 256) {
-    const int k = k1 + p.R * kM;
+  float2 gv[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {                                 // 16 strided loads in flight per thread
+    const int k = k1 + p.R * (threadIdx.x + 256 * i);
     const int kk = (2 * k <= p.n) ? k : p.n - k;
     float2 v = __ldg(g + kk);
     if (kk != k) v.y = -v.y;
     if (k == 0 || 2 * k == p.n) v.y = 0.f;
-    vals[kM] = v;
-    m = fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y)));
+    gv[i] = v;
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    vals[threadIdx.x + 256 * i] = gv[i];
+    m = fmaxf(m, fmaxf(fabsf(gv[i].x), fabsf(gv[i].y)));
   }
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
@@ -204,6 +224,13 @@ __global__ void __launch_bounds__(256) tc_gate_kernel(const TcGateParams p) {
   }
 }
 
+#ifdef SPECTRE_TC_TIMING
+__device__ long long g_core_timing[256][16];
+#define CORE_STAMP(slot) do { if (T == 0 && warp == 0 && blockIdx.x < 256) g_core_timing[blockIdx.x][slot] = clock64(); } while (0)
+#else
+#define CORE_STAMP(slot) do { } while (0)
+#endif
+
 // =====================================================================================
 // core: 4096-point units on the tensor cores
 // =====================================================================================
@@ -216,33 +243,34 @@ struct TcCoreParams {
   int* status;
 };
 
-// Epilogue of one MMA stage for one warp (TMEM lane quadrant q, 128-column half ch).
+// Epilogue of one MMA stage for one warp (TMEM lane quadrant q, 64-column quarter cq); TMEM loads
+// run one 32-column chunk ahead of the arithmetic.
 //   MODE 1: twiddle W_4096^{row col}; next operand gets (row digit -> column, col digit -> K)
 //   MODE 2: gate, conjugate;           next operand gets (col digit -> column, row digit -> K)
 //   MODE 3: final: store the unit's result [t' = 64 row + col][pair] as half2
 template <int MODE>
 __device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bsm, const uint32_t* Gsm,
-                                              unsigned char* out, int q, int ch, int T) {
+                                              unsigned char* out, int q, int cq, int T) {
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
   uint32_t r[2][16];
-  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 128 * ch;
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
   ld16x256b_x4(taddr0, r[0]);
   float2 w = make_float2(1.f, 0.f), wstep = w;
 #pragma unroll
-  for (int step = 0; step < 8; ++step) {                        // step = 4 j + chunk
-    const int j = step >> 2, chunk = step & 3;
+  for (int step = 0; step < 4; ++step) {                        // step = 2 j + chunk
+    const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
     if (MODE == 1 && chunk == 0) {
-      w = twiddle_fwd((unsigned)((row * (32 * ch + p)) & 4095), 4096u);
+      w = twiddle_fwd((unsigned)((row * (16 * cq + p)) & 4095), 4096u);
       wstep = twiddle_fwd((unsigned)((2 * row) & 4095), 4096u);
     }
     ld_wait4();
-    if (step < 7) {
+    if (step < 3) {
       const int ns = step + 1;
-      ld16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 2)) << 16) + 32 * (ns & 3), r[ns & 1]);
+      ld16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 1)) << 16) + 32 * (ns & 1), r[ns & 1]);
     }
     const uint32_t (&rr)[16] = r[step & 1];
-    const int grp0 = 16 * ch + 4 * chunk;                       // first 8-column group of the chunk
+    const int grp0 = 8 * cq + 4 * chunk;                        // first 8-column group of the chunk
     uint32_t base;
     if (MODE == 1) base = (uint32_t)((row >> 1) * k4Sbo + (4 * (row & 1) + 2 * cp) * 16 + (grp0 >> 1) * k4Lbo + 4 * p);
     else if (MODE == 2) base = (uint32_t)(grp0 * k4Sbo + (4 * p + 2 * cp) * 16 + (row >> 2) * k4Lbo + (row & 3) * 4);
@@ -276,99 +304,145 @@ __device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bs
   }
 }
 
+__device__ __forceinline__ void arrive4(uint32_t bar) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" :: "r"(bar) : "memory");
+}
+
+// Persistent: a CTA takes pairs of units (2 pair, 2 pair + 1).  16 epilogue warps alternate
+// between the two units of the pair; one more warp fetches operands and issues the MMAs, so
+// while the ALUs run one unit's epilogue the tensor core runs the other unit's stage.
+//   barL[s]  operand + gate table of slot s landed (bulk copies, transaction count)
+//   barD[s]  the stage's MMAs of slot s completed                    (4 phases per pair)
+//   barB[s]  all epilogue threads finished with slot s: next operand written (stages 0-2) or
+//            result stored and the slot free again (stage 3)         (4 phases per pair)
 __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* Fsm = smem;
+  unsigned char* Bsm[2] = {smem + k4FBytes, smem + k4FBytes + k4BBytes};
+  uint32_t* Gsm[2] = {reinterpret_cast<uint32_t*>(smem + k4FBytes + 2 * k4BBytes),
+                      reinterpret_cast<uint32_t*>(smem + k4FBytes + 2 * k4BBytes + k4GBytes)};
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + k4FBytes + 2 * k4BBytes + 2 * k4GBytes);
   __shared__ uint32_t tmem_slot;
+  const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
+  uint32_t barL[2], barD[2], barB[2];
+  for (int s2 = 0; s2 < 2; ++s2) { barL[s2] = s_u32(&bars[s2]); barD[s2] = s_u32(&bars[2 + s2]); barB[s2] = s_u32(&bars[4 + s2]); }
 
-  const int tid = threadIdx.x, grp = tid / k4GroupThreads, gt = tid - grp * k4GroupThreads;
-  const int warp = gt >> 5, T = gt & 31;
-  unsigned char* Bsm = smem + k4FBytes + grp * k4BBytes;
-  uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + k4FBytes + 2 * k4BBytes + grp * k4GBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + k4FBytes + 2 * k4BBytes + 2 * k4GBytes) + 2 * grp;  // [0] load, [1] MMA
-  const uint32_t barL = s_u32(&bars[0]), barD = s_u32(&bars[1]);
-
-  if (tid < 32) {
+  if (warp == k4EpiWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s_u32(&tmem_slot)), "r"(512));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
-  if (gt == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barL), "r"(1));
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barD), "r"(1));
+  if (tid == 0) {
+    for (int s2 = 0; s2 < 2; ++s2) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barL[s2]), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barD[s2]), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barB[s2]), "r"(k4EpiThreads));
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  {
+  if (tid < k4EpiThreads) {
     const uint4* Fg = reinterpret_cast<const uint4*>(p.F);
-    for (int i = tid; i < k4FBytes / 16; i += k4CoreThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
+    for (int i = tid; i < k4FBytes / 16; i += k4EpiThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_d = tmem_slot + 256 * grp;
-  const uint32_t idesc = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
-  const int q = warp & 3, ch = warp >> 2;
-
-  __shared__ int gave_up[2];
-  if (gt == 0) gave_up[grp] = 0;
-  asm volatile("bar.sync %0, %1;" :: "r"(1 + grp), "r"(k4GroupThreads) : "memory");
+  const uint32_t tmem = tmem_slot;
+  const int npairs = (p.nunits + 1) / 2;
   bool ok = true;
-  uint32_t phaseL = 0, phaseD = 0;
-  // A wait that runs out is recorded in gave_up[grp]; every thread of the group still reaches every
-  // group barrier, reads the flag there and leaves the loops together.
-  for (int unit = blockIdx.x * 2 + grp; unit < p.nunits && ok; unit += 2 * gridDim.x) {
-    // ---- operand and gate table: bulk async copies, completion counted on barL ----
-    if (gt == 0) {
-      const unsigned char* img = p.ws_in + (size_t)unit * k4ImgBytes;
-      const unsigned char* gim = p.gimg + (size_t)(unit / p.ntile) * k4GBytes;
-      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL), "r"(k4ImgBytes + k4GBytes) : "memory");
-      for (int m = 0; m < 32; ++m)
+  CORE_STAMP(0);
+
+  if (warp == k4EpiWarps) {
+    // ---- producer + MMA issuer ----
+    const uint32_t idesc = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+    // fetch(pair, slot): one bulk copy for the operand image, one for the gate table
+    auto fetch = [&](int pair, int s2) {
+      const int unit = 2 * pair + s2;
+      if (unit < p.nunits) {
+        const unsigned char* img = p.ws_in + (size_t)unit * k4ImgBytes;
+        const unsigned char* gim = p.gimg + (size_t)(unit / p.ntile) * k4GBytes;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL[s2]), "r"(k4ImgBytes + k4GBytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(s_u32(Bsm + m * k4Sbo)), "l"(img + (size_t)m * 2048), "r"(2048), "r"(barL) : "memory");
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   :: "r"(s_u32(Gsm)), "l"(gim), "r"(k4GBytes), "r"(barL) : "memory");
-    }
-    if (!wait4(barL, phaseL)) gave_up[grp] = 1;
-    phaseL ^= 1;
-    asm volatile("bar.sync %0, %1;" :: "r"(1 + grp), "r"(k4GroupThreads) : "memory");
-    ok = gave_up[grp] == 0;
-#pragma unroll 1
-    for (int stage = 0; stage < 4 && ok; ++stage) {
-      if (gt == 0) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a0 = s_u32(Fsm), b0 = s_u32(Bsm);
+                     :: "r"(s_u32(Bsm[s2])), "l"(img), "r"(k4ImgBytes), "r"(barL[s2]) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     :: "r"(s_u32(Gsm[s2])), "l"(gim), "r"(k4GBytes), "r"(barL[s2]) : "memory");
+      } else {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(barL[s2]) : "memory");   // odd tail: nothing to fetch
+      }
+    };
+    int iter = 0;
+    if (T == 0 && blockIdx.x < npairs) { fetch(blockIdx.x, 0); fetch(blockIdx.x, 1); }
+    __syncwarp();
+    for (int pair = blockIdx.x; pair < npairs && ok; pair += gridDim.x, ++iter) {
+      for (int stage = 0; stage < 4 && ok; ++stage) {
+        for (int s2 = 0; s2 < 2 && ok; ++s2) {
+          if (stage == 0) {
+            ok = wait4(barL[s2], iter & 1);                         // operand landed
+            if (ok && iter > 0) ok = wait4(barB[s2], 1);            // previous result of this slot left TMEM
+          } else {
+            ok = wait4(barB[s2], (stage - 1) & 1);
+          }
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          if (T == 0) {
+            const uint32_t a0 = s_u32(Fsm), b0 = s_u32(Bsm[s2]);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t da = desc4(a0 + ks * 256, 128, 2048);
-          const uint64_t db = desc4(b0 + ks * 2 * k4Lbo, k4Lbo, k4Sbo);
-          const uint32_t acc = ks > 0;
-          asm volatile(
-              "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-              :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint64_t da = desc4(a0 + ks * 256, 128, 2048);
+              const uint64_t db = desc4(b0 + ks * 2 * k4Lbo, k4Lbo, k4Sbo);
+              const uint32_t acc = ks > 0;
+              asm volatile(
+                  "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                  :: "r"(tmem + 256 * s2), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barD[s2]) : "memory");
+          }
+          __syncwarp();
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barD) : "memory");
       }
-      const bool good = wait4(barD, phaseD);
-      phaseD ^= 1;
-      if (!good) gave_up[grp] = 1;
-      if (good) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (stage == 1) core_epilogue<2>(tmem_d, Bsm, Gsm, nullptr, q, ch, T);
-        else if (stage == 3) core_epilogue<3>(tmem_d, Bsm, Gsm, p.ws_out + (size_t)unit * k4OutBytes, q, ch, T);
-        else core_epilogue<1>(tmem_d, Bsm, Gsm, nullptr, q, ch, T);
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      // the slot's shared memory is free once its last MMAs completed: prefetch the next pair
+      // while the epilogue warps still drain the accumulators
+      const int next = pair + gridDim.x;
+      if (next < npairs) {
+        for (int s2 = 0; s2 < 2 && ok; ++s2) {
+          ok = wait4(barD[s2], 1);
+          if (ok && T == 0) fetch(next, s2);
+          __syncwarp();
+        }
       }
-      asm volatile("bar.sync %0, %1;" :: "r"(1 + grp), "r"(k4GroupThreads) : "memory");   // the group's 256 threads
-      ok = gave_up[grp] == 0;
+    }
+  } else {
+    // ---- epilogue warps ----
+    const int q = warp & 3, cq = warp >> 2;
+    for (int pair = blockIdx.x; pair < npairs && ok; pair += gridDim.x) {
+#pragma unroll 1
+      for (int stage = 0; stage < 4 && ok; ++stage) {
+#pragma unroll 1
+        for (int s2 = 0; s2 < 2 && ok; ++s2) {
+          ok = wait4(barD[s2], stage & 1);
+          if (!ok) break;
+          if (pair == blockIdx.x && stage == 0 && s2 == 0) CORE_STAMP(1);
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t td = tmem + 256 * s2;
+          const int unit = 2 * pair + s2;
+          if (stage == 1) core_epilogue<2>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T);
+          else if (stage == 3) {
+            if (unit < p.nunits) core_epilogue<3>(td, Bsm[s2], Gsm[s2], p.ws_out + (size_t)unit * k4OutBytes, q, cq, T);
+          } else core_epilogue<1>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T);
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          if (pair == blockIdx.x) CORE_STAMP(2 + 2 * stage + s2);
+          arrive4(barB[s2]);
+        }
+      }
     }
   }
-  if (!ok && gt == 0) atomicExch(p.status, 1);
+  if (!ok && T == 0) atomicExch(p.status, 1);
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (tid < 32) {
+  if (warp == k4EpiWarps) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_slot), "r"(512));
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(512));
   }
 }
 
@@ -385,7 +459,7 @@ struct TcOutParams {
 
 // CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.
 template <int R>
-__global__ void __launch_bounds__(256) tc_out_kernel(const TcOutParams p) {
+__global__ void __launch_bounds__(256, 2) tc_out_kernel(const TcOutParams p) {
   constexpr int NT = 512 / R;
   extern __shared__ __align__(128) uint32_t stage[];            // [R][NT][D/2 words]
   const int nblk = 4096 / NT;
@@ -397,19 +471,23 @@ __global__ void __launch_bounds__(256) tc_out_kernel(const TcOutParams p) {
   const float base_scale = 1.0f / ((float)R * in_scale(R));
   const int skew_mask = (p.ntile & (p.ntile - 1)) == 0 ? min(p.ntile, 8) - 1 : 0;   // XOR stays inside the row
 
+  // gate scales of this head's R units, times 1 / (R s_in)
+  __shared__ float gsc[R];
+  if (threadIdx.x < R) gsc[threadIdx.x] = __ldg(p.gscale + slab_local * R + threadIdx.x) * base_scale;
+  __syncthreads();
   // phase 1: a warp takes (tile, 8 consecutive t'); lane = (t' % 8, pair within the tile)
   const int nitems = p.ntile * (NT / 8);
+  const uint32_t* wsl = reinterpret_cast<const uint32_t*>(p.ws_out + (size_t)slab_local * R * p.ntile * k4OutBytes);
+  const int ustride = p.ntile * (k4OutBytes / 4);               // words between consecutive k1 (same tile)
   for (int item = warp; item < nitems; item += 8) {
     const int tile = item % p.ntile, tl = (item / p.ntile) * 8 + t8;
     const int tp = tb * NT + tl;
+    const uint32_t* pu = wsl + tile * (k4OutBytes / 4) + tp * 4 + c4;
     float2 x[R];
 #pragma unroll
     for (int k1 = 0; k1 < R; ++k1) {
-      const size_t unit = ((size_t)slab_local * R + k1) * p.ntile + tile;
-      const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(p.ws_out + unit * k4OutBytes) + tp * 4 + c4);
-      float2 f = h2unpack(v);
-      f.y = -f.y;                                               // result of conj(FFT(conj(.)))
-      x[k1] = cscale(f, __ldg(p.gscale + slab_local * R + k1) * base_scale);
+      float2 f = h2unpack(__ldg(pu + k1 * ustride));
+      x[k1] = make_float2(f.x * gsc[k1], -f.y * gsc[k1]);       // result of conj(FFT(conj(.))), scaled
     }
     const float2 w1 = twiddle_fwd((unsigned)tp, (unsigned)p.n);
     float2 w = w1;
@@ -419,24 +497,25 @@ __global__ void __launch_bounds__(256) tc_out_kernel(const TcOutParams p) {
       w = cmul(w, w1);
     }
     Dft<R, true>::run(x);
+    const int word = (tile * 4 + c4) ^ ((tl & skew_mask) << 2);   // skew: the 8 rows of a warp hit 8 bank groups
+    uint32_t* ps = stage + tl * npair + word;
 #pragma unroll
     for (int n1 = 0; n1 < R; ++n1) {
       __nv_bfloat162 o = __floats2bfloat162_rn(x[n1].x, x[n1].y);
-      const int word = (tile * 4 + c4) ^ ((tl & skew_mask) << 2);   // skew: the 8 rows of a warp hit 8 bank groups
-      stage[((size_t)n1 * NT + tl) * npair + word] = *reinterpret_cast<uint32_t*>(&o);
+      ps[n1 * NT * npair] = *reinterpret_cast<uint32_t*>(&o);
     }
   }
   __syncthreads();
   // phase 2: whole rows
   bf16* dst = p.dst + b * p.d_sb + h * p.d_sh;
-  for (int r = warp; r < R * NT; r += 8) {
-    const int n1 = r / NT, tl = r - n1 * NT;
+  const int cpr = npair / 4;                                    // 16-byte chunks per row
+  for (int idx = threadIdx.x; idx < R * NT * cpr; idx += 256) {
+    const int r = idx / cpr, q16 = idx - r * cpr;
+    const int n1 = r / NT, tl = r & (NT - 1);                   // NT is a power of two
     const int row = n1 * 4096 + tb * NT + tl;
     if (row >= p.L) continue;
-    for (int c = lane; c < npair; c += 32) {
-      const uint32_t v = stage[(size_t)r * npair + (c ^ ((tl & skew_mask) << 2))];
-      *reinterpret_cast<uint32_t*>(dst + (int64_t)row * p.d_sl + 2 * c) = v;
-    }
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + r * npair + ((q16 ^ (tl & skew_mask)) << 2));
+    *reinterpret_cast<uint4*>(dst + (int64_t)row * p.d_sl + 8 * q16) = v;
   }
 }
 
@@ -457,7 +536,10 @@ bool tc4k_supported(int n, int D) {
 size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
   const int R = n / 4096;
   size_t per = tc4k_slab_bytes(R, D);
-  size_t budget = (ctx->l2_bytes * 3) / 4;
+  // heads per group: measured on B200, larger groups win (fewer, fuller launches) although the
+  // intermediates then no longer stay in L2; the preferred workspace is capped at 1.25 GiB
+  size_t budget = (size_t)1280 << 20;
+  if (const char* e = std::getenv("SPECTRE_TC_L2_FRACTION_PCT")) budget = ctx->l2_bytes / 100 * (size_t)atoi(e);
   size_t g = budget / per;
   if (g < 1) g = 1;
   if (g > (size_t)nslab) g = nslab;
@@ -490,7 +572,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64), (int)nunits, ntile,
                      ctx->status_dev};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
-  int grid = (int)((nunits + 1) / 2);
+  int grid = (int)((nunits + 1) / 2);               // pairs of units
   if (grid > ctx->sm_count) grid = ctx->sm_count;
   tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
   SPECTRE_LAUNCH_OK("tc_core_kernel");
