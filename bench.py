@@ -37,7 +37,11 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": None, "c3": None, "c4": None, "c5": None}
+# c2: mixer_tc8192_kernel 35.0 MB read + 1.2 MB written inside the launch (its 33.6 MB output was still
+#     dirty in L2 when the launch ended, so this understates the traffic; nothing is re-read)
+# c3: the four kernels of one staged mixer call at full size (intermediates spill from L2)
+# c4: append_spectrum_kernel measured at B = 2 (1015.3 MB), scaled by 4 to B = 8
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": 36.2e6, "c3": 3126e6, "c4": 4061e6, "c5": None}
 
 
 def measured_peak():
@@ -159,16 +163,24 @@ class MixerBench:
             self.sets.append(d)
         self.units_per_step = w.B * w.L                                  # tokens
         self.alg_bytes = mixer_algorithmic_bytes(w)
-        self.kernel_name = "mixer (onchip_kernel)" if ws_mix == 0 else "mixer (strided + onchip + strided, per group)"
-        # kernels per step: pool, gate_mlp, mixer kernel(s), wavelet
+        # kernels per step: gate = pool + hidden + output layer; mixer = 1 (single-kernel paths) or
+        # gate images + transpose-in + core + transpose-out per group of heads (staged tensor-core
+        # path) or strided + on-chip + strided per group (fp32 four-step path); + wavelet
         import math
-        groups = 1
-        nk = 1
-        if ws_mix:
+        if w.dtype == "bf16" and w.n == 8192:
+            self.kernel_name, nk = "mixer_tc8192_kernel (single-kernel tcgen05 mixer)", 1
+        elif w.dtype == "bf16" and ws_mix and w.n >= 4096:
+            R, ntile = w.n // 4096, w.D // 8
+            per = R * ntile * (32 * 2064 + 65536) + R * 18432 + 256
+            groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
+            self.kernel_name, nk = "mixer, staged tcgen05 path (tc_gate + tc_in + tc_core + tc_out per group)", 4 * groups
+        elif ws_mix:
             per = w.n * (w.D // 2) * 8
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
-            nk = 3 * groups
-        self.launches_per_step = 2 + nk + (1 if w.wavelet_levels else 0)
+            self.kernel_name, nk = "mixer (strided + onchip + strided per group)", 3 * groups
+        else:
+            self.kernel_name, nk = "mixer (onchip_kernel)", 1
+        self.launches_per_step = 3 + nk + (1 if w.wavelet_levels else 0)
         self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         self.d2h = self.h2d
 
@@ -332,21 +344,28 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(W.CONFIGS))
     ap.add_argument("--sets", type=int, default=None, help="rotating buffer sets (default: enough to exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
+    ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
+    if args.heads:
+        w = W.scaled(w, H=args.heads, name=f"{w.name} reduced to H={args.heads}")
+    if args.batch:
+        w = W.scaled(w, B=args.batch, name=f"{w.name} reduced to B={args.batch}")
     rank, local_rank, world = R.world()
 
     if args.impl == "reference":
         args.steps = args.steps if args.steps is not None else 3
         args.warmup = args.warmup if args.warmup is not None else 1
-        if w.name == "c3" and args.steps > 2:
+        if args.workload == "c3" and args.steps > 2:
             args.steps = 2
         run_reference(args, w)
         return
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
-    default_steps = {"c1": 2000, "c2": 2000, "c3": 100, "c4": 200, "c5": 500}[w.name]
+    base = args.workload
+    default_steps = {"c1": 2000, "c2": 2000, "c3": 100, "c4": 200, "c5": 500}[base]
     K = args.steps if args.steps is not None else default_steps
     Wm = max(3, args.warmup if args.warmup is not None else 10)
     dev = torch.device("cuda", local_rank)
@@ -394,7 +413,7 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         torch.set_num_threads(1)
-        reps = 1 if w.name in ("c3",) else 3
+        reps = 1 if base in ("c3",) else 3
         tot, units = 0.0, 0
         for _ in range(reps):
             dt, u = bench.cpu_step()
@@ -422,7 +441,7 @@ def main():
                          "frac": achieved / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": bench.alg_bytes,
                          "kernel_ms": kern_ms, "frac_of_8000": achieved / 8000.0,
                          "kernel_tokens_per_s": bench.units_per_step / (kern_ms * 1e-3),
-                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},   # None for reduced cases
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))

@@ -1,0 +1,107 @@
+"""Parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times
+(same shapes, strides, workspace sizes and default path selection).  The oracle cannot run a whole
+workload in seconds, so it recomputes a seeded sample of (batch, head) slabs (columns of different
+heads are independent given the gate) and, for the cache, a sample of bins with the closed form."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spectre_oracle as O
+from paper_2502_18394_b200 import binding as S
+from paper_2502_18394_b200 import workloads as W
+from util import TOL, gate_params_np, gate_to_complex, rel_err, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = S.Context(0)
+    yield c
+    c.close()
+
+
+def slab_error(y, ref):
+    return float(np.linalg.norm(y - ref) / np.linalg.norm(ref))
+
+
+def run_full(ctx, name, sample):
+    w = W.CONFIGS[name]
+    x = W.activations(w)
+    p = W.gate_params(w)
+    xd = x.cuda()
+    pd = to_dev(p)
+    qbar = torch.empty(w.B, w.H, w.D, device="cuda")
+    g = S.spectre_gate(ctx, pd, w.n, q=xd, qbar_out=qbar)
+    wrm = None
+    if w.wavelet_levels:
+        wp = W.wavelet_params(w)
+        wrm = dict(to_dev(wp), qbar=qbar)
+    y = S.spectre_mixer_forward(ctx, xd, g, wrm=wrm)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    pn = gate_params_np(p)
+    worst_g = worst_y = 0.0
+    for (b, h) in sample:
+        xs = W.to_f64(x[b:b + 1, :, h:h + 1, :])
+        ph = {k: (v[h:h + 1] if isinstance(v, np.ndarray) else v) for k, v in pn.items()}
+        gref, qref = O.gate(xs.sum(axis=1), 1.0 / w.L, w.n, return_qbar=True, **ph)
+        worst_g = max(worst_g, rel_err(gate_to_complex(g[b:b + 1, h:h + 1]), gref))
+        ref = O.mixer(xs, gref)
+        if w.wavelet_levels:
+            wp = W.wavelet_params(w)
+            s = O.wavelet_level_gates(qref, W.to_f64(wp["Ww1"][h:h + 1]), W.to_f64(wp["bw1"][h:h + 1]),
+                                      W.to_f64(wp["Ww2"][h:h + 1]), W.to_f64(wp["bw2"][h:h + 1]), w.wavelet_levels)
+            ref = O.wavelet_refine(ref, s, w.wavelet_levels)
+        worst_y = max(worst_y, slab_error(W.to_f64(y[b:b + 1, :, h:h + 1, :]), ref))
+    return worst_g, worst_y, w
+
+
+def test_c2_full_size_sampled_heads(ctx):
+    eg, ey, w = run_full(ctx, "c2", [(0, 0), (0, 13), (0, 31)])
+    assert eg < 1e-4 and ey < TOL["bf16"]
+
+
+def test_c3_full_size_sampled_heads(ctx):
+    eg, ey, w = run_full(ctx, "c3", [(0, 5), (0, 31)])
+    assert eg < 1e-3 and ey < TOL["bf16"]      # gate: 131072-token mean in fp32 with atomics
+
+
+def test_c5_full_size_sampled_heads(ctx):
+    eg, ey, w = run_full(ctx, "c5", [(0, 0), (100, 7), (255, 11)])
+    assert eg < 1e-4 and ey < TOL["bf16"]
+
+
+def test_c1_full_size(ctx):
+    eg, ey, w = run_full(ctx, "c1", [(0, 0), (0, 1)])
+    assert eg < 1e-5 and ey < TOL["f32"]
+
+
+def test_c4_full_size_append_sampled_bins(ctx):
+    # B = 8, H = 32, d = 64, N_max = 32768: prefill a full window, append 1024 tokens (every append
+    # evicts), compare sampled (b, h) spectra with a from-scratch transform of the ring buffer at
+    # every 128th step, and the running sum of queries throughout.
+    w = W.CONFIGS["c4"]
+    N = w.N_max
+    cache = S.PrefixCache(w.B, w.H, w.D, N)
+    one = W.scaled(w, B=1)
+    q = torch.cat([W.activations(one, stream=10 + b) for b in range(w.B)], dim=0).cuda()
+    v = torch.cat([W.activations(one, stream=30 + b) for b in range(w.B)], dim=0).cuda()
+    S.spectre_prefix_cache_prefill(ctx, cache, q, v)
+    del q, v
+    steps = w.appends
+    qs, vs = W.decode_tokens(w, steps)
+    qd, vd = qs.cuda(), vs.cuda()
+    sample = [(0, 0), (3, 17), (7, 31)]
+    for i in range(steps):
+        S.spectre_prefix_cache_append(ctx, cache, qd[i], vd[i], N + i)
+        if (i + 1) % 128 == 0:
+            torch.cuda.synchronize()
+            for (b, h) in sample:
+                P = W.to_f64(cache.prefix_fft[b, h])
+                P = P[..., 0] + 1j * P[..., 1]                           # [K, D]
+                ref = O.rfft(W.to_f64(cache.V_buf[b, :, h, :]), N)       # full recompute of the window
+                assert rel_err(P, ref) < 2e-5, (i, b, h)
+                assert rel_err(W.to_f64(cache.sum_q[b, h]), W.to_f64(cache.Q_buf[b, :, h, :]).sum(axis=0)) < 2e-5
+    # the ring buffer holds the last N tokens: slot (N + i) mod N = i was overwritten by append i
+    assert torch.equal(cache.V_buf[:, :steps], vd.permute(1, 0, 2, 3))
