@@ -17,6 +17,7 @@ struct spectre_ctx {
   int cluster_ok;         // thread-block clusters usable on this device
   size_t l2_bytes;
   void* dft64;            // device: 64-point DFT matrix (fp16, MMA operand layout), 32 KiB
+  void* tw8192;           // device: (cos, sin)(2 pi r / 8192), r = 0..2048 (quarter wave), 16 KiB
   int* status_host;       // pinned, device-mapped status word written by kernels whose waits ran out
   int* status_dev;
 };
@@ -66,6 +67,14 @@ __device__ __forceinline__ float2 twiddle_fwd(unsigned num, unsigned den) {
   float s, c;
   sincospif(2.0f * (float)num / (float)den, &s, &c);
   return make_float2(c, -s);
+}
+
+// exp(-j 2 pi m / 8192) from the quarter-wave table (cos, sin)(2 pi r / 8192), r = 0..2048
+__device__ __forceinline__ float2 twiddle8192(const float2* __restrict__ tab, unsigned m) {
+  const unsigned q = (m >> 11) & 3u, r = m & 2047u;
+  const float2 t = __ldg(tab + r);
+  const float c = (q & 1u) ? -t.y : t.x, s = (q & 1u) ? t.x : t.y;    // rotate by q quarter turns
+  return (q & 2u) ? make_float2(-c, s) : make_float2(c, -s);
 }
 
 // ---- loads / stores of 4 adjacent real columns as two complex pairs ----------

@@ -53,6 +53,7 @@ struct TcParams {
   int64_t s_sb, s_sl, s_sh, d_sb, d_sl, d_sh;
   const float2* g;        // [B*H][4097]
   const __half* F;        // 64-point DFT matrix, canonical smem layout
+  const float2* tw;       // quarter-wave twiddle table (8192nds)
   int H, D, L, ntile;
   int* status;            // host-mapped status word (0 = fine)
 };
@@ -124,7 +125,7 @@ __device__ __forceinline__ float2 gate8192(const float2* __restrict__ g, int k) 
 //   MODE 2: gate (and conjugate for the inverse), write straight (col digit -> column index, row digit -> K)
 template <int MODE>
 __device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm, int q, int cq, int T,
-                                             const uint32_t* __restrict__ Gtab) {
+                                             const uint32_t* __restrict__ Gtab, const float2* __restrict__ tw) {
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
@@ -135,8 +136,8 @@ __device__ __forceinline__ void epilogue_mid(uint32_t tmem_d, unsigned char* Bsm
     const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
     if (MODE == 1 && chunk == 0) {
-      w = twiddle_fwd((unsigned)((row * (16 * cq + p)) & 4095), 4096u);
-      wstep = twiddle_fwd((unsigned)((2 * row) & 4095), 4096u);
+      w = twiddle8192(tw, 2u * (unsigned)((row * (16 * cq + p)) & 4095));
+      wstep = twiddle8192(tw, 4u * (unsigned)row);
     }
     tmem_ld_wait();
     if (step < 3) {
@@ -255,8 +256,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
       const bf16* src = p.src + b * p.s_sb + h * p.s_sh + col0;
       const int t1 = tid & 63, t2base = tid >> 6;          // 32 lanes = 32 consecutive t1: conflict-free stores
       constexpr int kIter = 64 / (kTcEpiThreads / 64);
-      float2 w = twiddle_fwd((unsigned)(64 * t1 + t2base), 8192u);
-      const float2 wstep = twiddle_fwd((unsigned)(kTcEpiThreads / 64), 8192u);
+      float2 w = twiddle8192(p.tw, (unsigned)(64 * t1 + t2base));
+      const float2 wstep = twiddle8192(p.tw, (unsigned)(kTcEpiThreads / 64));
 #pragma unroll 4
       for (int it = 0; it < kIter; ++it) {
         const int t2 = t2base + (kTcEpiThreads / 64) * it, t = 64 * t1 + t2;
@@ -315,8 +316,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t td = tmem + 256 * half;
-        if (stage == 1) epilogue_mid<2>(td, Bsm[half], q, cq, T, Gsm[half]);
-        else epilogue_mid<1>(td, Bsm[half], q, cq, T, Gsm[half]);
+        if (stage == 1) epilogue_mid<2>(td, Bsm[half], q, cq, T, Gsm[half], p.tw);
+        else epilogue_mid<1>(td, Bsm[half], q, cq, T, Gsm[half], p.tw);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         TC_STAMP(3 + 2 * stage + half);
@@ -332,7 +333,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
       const int i = T >> 2, pp = (T >> 1) & 1, cp = T & 1;
       const float gs = 0.5f * gmax;
       bf16* dst = p.dst + b * p.d_sb + h * p.d_sh + col0 + 4 * cp;
-      const float2 wstep = twiddle_fwd(2u, 8192u);
+      const float2 wstep = twiddle8192(p.tw, 2u);
       const uint32_t taddr0 = tmem + ((uint32_t)(32 * q) << 16) + 64 * cq;
       uint32_t re[2][16], ro[2][16];
       tmem_ld_16x256b_x4(taddr0, re[0]);
@@ -342,7 +343,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc8192_kernel(const TcPar
       for (int step = 0; step < 4; ++step) {
         const int j = step >> 1, chunk = step & 1;
         const int t1 = 8 * (2 * q + j) + i;
-        if (chunk == 0) w = twiddle_fwd((unsigned)(64 * t1 + 16 * cq + pp), 8192u);
+        if (chunk == 0) w = twiddle8192(p.tw, (unsigned)(64 * t1 + 16 * cq + pp));
         tmem_ld_wait();
         if (step < 3) {
           const uint32_t ta = taddr0 + ((uint32_t)(16 * ((step + 1) >> 1)) << 16) + 32 * ((step + 1) & 1);
@@ -397,6 +398,21 @@ __global__ void build_dft64_kernel(__half* F) {
   *reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(F) + off) = __float2half_rn(0.125f * v);
 }
 
+// (cos, sin)(2 pi r / 8192) for r = 0..2048
+__global__ void build_tw8192_kernel(float2* tab) {
+  int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r > 2048) return;
+  float s, c;
+  sincospif((float)r / 4096.0f, &s, &c);
+  tab[r] = make_float2(c, s);
+}
+
+int build_tw8192(float2* tab, cudaStream_t st) {
+  build_tw8192_kernel<<<9, 256, 0, st>>>(tab);
+  SPECTRE_LAUNCH_OK("build_tw8192_kernel");
+  return SPECTRE_OK;
+}
+
 int build_dft64(__half* F, cudaStream_t st) {
   build_dft64_kernel<<<64, 256, 0, st>>>(F);
   SPECTRE_LAUNCH_OK("build_dft64_kernel");
@@ -412,6 +428,7 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
   p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
   p.g = reinterpret_cast<const float2*>(g);
   p.F = reinterpret_cast<const __half*>(ctx->dft64);
+  p.tw = reinterpret_cast<const float2*>(ctx->tw8192);
   p.H = v->H; p.D = v->D; p.L = v->L; p.ntile = v->D / 8;
   p.status = ctx->status_dev;
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));

@@ -29,7 +29,7 @@ namespace spectre {
 
 // ---- shared with mixer_tc.cu (same conventions) ------------------------------------
 constexpr int k4Lbo = 128;                       // bytes between core matrices along K
-constexpr int k4Sbo = 2064;                      // bytes between 8-column groups (2048 + 16 pad)
+constexpr int k4Sbo = 2064;                      // bytes between 8-column groups (2048 + 16 pad; 144 / 2320 measured slower)
 constexpr int k4BBytes = 32 * k4Sbo;             // one 256-column operand in shared memory
 constexpr int k4ImgBytes = k4BBytes;             // the workspace holds the same image, padding included
 constexpr int k4FBytes = 128 * 128 * 2;
@@ -239,6 +239,7 @@ struct TcCoreParams {
   const unsigned char* gimg;
   unsigned char* ws_out;
   const __half* F;
+  const float2* tw;         // quarter-wave twiddle table (8192nds)
   int nunits, ntile;
   int* status;
 };
@@ -250,7 +251,8 @@ struct TcCoreParams {
 //   MODE 3: final: store the unit's result [t' = 64 row + col][pair] as half2
 template <int MODE>
 __device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bsm, const uint32_t* Gsm,
-                                              unsigned char* out, int q, int cq, int T) {
+                                              unsigned char* out, int q, int cq, int T,
+                                              const float2* __restrict__ tw) {
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
@@ -261,8 +263,8 @@ __device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bs
     const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
     if (MODE == 1 && chunk == 0) {
-      w = twiddle_fwd((unsigned)((row * (16 * cq + p)) & 4095), 4096u);
-      wstep = twiddle_fwd((unsigned)((2 * row) & 4095), 4096u);
+      w = twiddle8192(tw, 2u * (unsigned)((row * (16 * cq + p)) & 4095));
+      wstep = twiddle8192(tw, 4u * (unsigned)row);
     }
     ld_wait4();
     if (step < 3) {
@@ -425,10 +427,10 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t td = tmem + 256 * s2;
           const int unit = 2 * pair + s2;
-          if (stage == 1) core_epilogue<2>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T);
+          if (stage == 1) core_epilogue<2>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T, p.tw);
           else if (stage == 3) {
-            if (unit < p.nunits) core_epilogue<3>(td, Bsm[s2], Gsm[s2], p.ws_out + (size_t)unit * k4OutBytes, q, cq, T);
-          } else core_epilogue<1>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T);
+            if (unit < p.nunits) core_epilogue<3>(td, Bsm[s2], Gsm[s2], p.ws_out + (size_t)unit * k4OutBytes, q, cq, T, p.tw);
+          } else core_epilogue<1>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T, p.tw);
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           if (pair == blockIdx.x) CORE_STAMP(2 + 2 * stage + s2);
@@ -569,8 +571,8 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   tc_in_kernel<R><<<cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip);
   SPECTRE_LAUNCH_OK("tc_in_kernel");
 
-  TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64), (int)nunits, ntile,
-                     ctx->status_dev};
+  TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
+                     reinterpret_cast<const float2*>(ctx->tw8192), (int)nunits, ntile, ctx->status_dev};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
   int grid = (int)((nunits + 1) / 2);               // pairs of units
   if (grid > ctx->sm_count) grid = ctx->sm_count;
