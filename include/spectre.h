@@ -47,10 +47,10 @@ typedef enum { SPECTRE_F32 = 0, SPECTRE_BF16 = 1 } spectre_dtype;
 
 typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch limits */
 
-/* Creates a context for CUDA device `device`.  Besides host memory it owns two small device
- * tables (the 64-point DFT matrix of the tensor-core mixer, 32 KiB, and a quarter-wave twiddle
- * table, 16 KiB) and one pinned status word, all released by spectre_destroy.  No other call
- * allocates. */
+/* Creates a context for CUDA device `device`.  Besides host memory it owns three small device
+ * tables (the 64-point and 49-point DFT matrices of the tensor-core mixers, 32 KiB each, and a
+ * quarter-wave twiddle table, 16 KiB) and one pinned status word, all released by
+ * spectre_destroy.  No other call allocates. */
 int spectre_create(spectre_ctx** out, int device);
 int spectre_destroy(spectre_ctx* ctx);
 /* The tensor-core mixer hands tiles between its warps through on-chip barriers whose waits

@@ -17,6 +17,7 @@ struct spectre_ctx {
   int cluster_ok;         // thread-block clusters usable on this device
   size_t l2_bytes;
   void* dft64;            // device: 64-point DFT matrix (fp16, MMA operand layout), 32 KiB
+  void* dft49;            // device: 49-point DFT matrix, same format (n = 196 path), 32 KiB
   void* tw8192;           // device: (cos, sin)(2 pi r / 8192), r = 0..2048 (quarter wave), 16 KiB
   int* status_host;       // pinned, device-mapped status word written by kernels whose waits ran out
   int* status_dev;

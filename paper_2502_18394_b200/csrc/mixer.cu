@@ -29,6 +29,8 @@ namespace spectre {
 
 int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                         const spectre_act* y);   // mixer_tc.cu
+int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                       const spectre_act* y);
 
 bool tc4k_supported(int n, int D);                                                     // mixer_tc4k.cu
 size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
@@ -632,6 +634,7 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   const int force = forced_path();
   const bool tc_ok = v->dtype == SPECTRE_BF16 && ctx->dft64 != nullptr && force != kPathAlu;
   const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 15);
+  const bool tc196 = tc_ok && n_fft == 196 && v->D == 64 && ctx->dft49 != nullptr;
   const bool fused = tc_ok && n_fft == 8192 && force != kPathStaged;
   const bool staged = !fused && tc_ok && force != kPathFused && tc4k_supported(n_fft, v->D) && ws_ok &&
                       workspace_bytes >= tc4k_min_workspace(n_fft, v->D);
@@ -648,9 +651,10 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   }
   SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (staged || fused) {
-    rc = staged ? launch_mixer_tc4k(ctx, st, v, g, y, n_fft, workspace, workspace_bytes)
-                : launch_mixer_tc8192(ctx, st, v, g, y);
+  if (staged || fused || tc196) {
+    rc = tc196 ? launch_mixer_tc196(ctx, st, v, g, y)
+               : (staged ? launch_mixer_tc4k(ctx, st, v, g, y, n_fft, workspace, workspace_bytes)
+                         : launch_mixer_tc8192(ctx, st, v, g, y));
     if (rc != SPECTRE_OK) return rc;
     if (wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
     return SPECTRE_OK;

@@ -438,4 +438,311 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
   return SPECTRE_OK;
 }
 
+
+// =====================================================================================
+// n = 196 (14 x 14 patch grids), bf16 I/O, D = 64: 196 = 4 * 49.
+//
+// t = 49 n1 + t', k = k1 + 4 kM.  The radix-4 DFT over n1 and the twiddle W_196^{k1 t'} run on
+// the ALUs while whole 128-byte head rows are loaded; each 49-point DFT over t' is ONE tensor-core
+// stage with the 49-point DFT matrix in real form (98 x 98, zero-padded to 128 x 112) as the A
+// operand; the gate is applied to the accumulator, one more stage does the inverse 49-point DFT
+// (conj trick), and the final epilogue does the inverse radix-4 and stores bf16 rows.
+// A CTA takes 4 heads: columns (head, k1, pair) = 4 x 4 x 32 = 512 = the whole TMEM; the two
+// 2-head halves ping-pong between tensor core and ALUs like the halves of the 8192 kernel.
+// =====================================================================================
+constexpr int k196Heads = 4;
+constexpr int k196KSteps = 7;                 // K = 112 >= 98
+constexpr int k196Smem = kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4 + 64;
+
+struct Tc196Params {
+  const bf16* src;
+  bf16* dst;
+  int64_t s_sb, s_sl, s_sh, d_sb, d_sl, d_sh;
+  const float2* g;        // [B*H][99]
+  const __half* F;        // 49-point DFT matrix (real form, padded), canonical smem layout
+  int H, L, nheads;       // nheads = B * H
+  int* status;
+};
+
+__device__ __forceinline__ void tmem_ld_16x256b_x1(uint32_t taddr, uint32_t (&r)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x1.b32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr));
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196Params p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* Fsm = smem;
+  unsigned char* Bsm[2] = {smem + kTcFBytes, smem + kTcFBytes + kTcBBytes};
+  uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + kTcFBytes + 2 * kTcBBytes);        // [4 heads][k1 * 64 + kM]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4);
+  __shared__ uint32_t tmem_slot;
+  __shared__ float red[kTcEpiWarps];
+  __shared__ float gmax_s[k196Heads];
+
+  const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
+  const int head0 = blockIdx.x * k196Heads;
+
+  if (warp == kTcEpiWarps) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[0])), "r"(kTcEpiThreads));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[1])), "r"(kTcEpiThreads));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[2])), "r"(1));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[3])), "r"(1));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < kTcEpiThreads) {
+    const uint4* Fg = reinterpret_cast<const uint4*>(p.F);
+    for (int i = tid; i < kTcFBytes / 16; i += kTcEpiThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
+    // zero the operands once: K rows 98..127 and the columns of absent heads must read as zero
+    for (int i = tid; i < 2 * kTcBBytes / 16; i += kTcEpiThreads) reinterpret_cast<uint4*>(Bsm[0])[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = tmem_slot;
+
+  if (warp == kTcEpiWarps) {
+    // ---- MMA issuer: 2 stages x 2 halves, 7 K-steps each ----
+    const uint32_t idesc = umma_idesc_128x256();
+    bool ok = true;
+    for (int stage = 0; stage < 2 && ok; ++stage) {
+      for (int half = 0; half < 2 && ok; ++half) {
+        ok = mbar_wait(smem_u32(&bars[half]), stage & 1);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (T == 0) {
+          const uint32_t a0 = smem_u32(Fsm), b0 = smem_u32(Bsm[half]);
+#pragma unroll
+          for (int ks = 0; ks < k196KSteps; ++ks) {
+            uint64_t da = umma_desc(a0 + ks * 256, 128, 2048);
+            uint64_t db = umma_desc(b0 + ks * 2 * kTcLbo, kTcLbo, kTcSbo);
+            uint32_t acc = ks > 0;
+            asm volatile(
+                "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                :: "r"(tmem + 256 * half), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+          }
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                       :: "r"(smem_u32(&bars[2 + half])) : "memory");
+        }
+        __syncwarp();
+      }
+    }
+    if (!ok && T == 0) atomicExch(p.status, 1);
+  } else {
+    // ---- load: rows t' + 49 n1 of each head, radix-4 over n1, twiddle, fp16, operand (K = t', column = (head, k1, pair)) ----
+    // a warp takes 4 consecutive t' x 8 chunks of 16 bytes (conflict-free operand stores)
+    for (int item = warp; item < k196Heads * 13; item += kTcEpiWarps) {
+      const int hl = item / 13, tg = item - hl * 13;
+      const int tp = 4 * tg + (T >> 3), chunk = T & 7;
+      const int hg = head0 + hl;
+      if (tp >= 49 || hg >= p.nheads) continue;
+      const int b = hg / p.H, h = hg - b * p.H;
+      const bf16* src = p.src + b * p.s_sb + h * p.s_sh + 8 * chunk;
+      uint4 rr[4];
+#pragma unroll
+      for (int n1 = 0; n1 < 4; ++n1) {
+        const int row = tp + 49 * n1;
+        rr[n1] = row < p.L ? __ldcg(reinterpret_cast<const uint4*>(src + (int64_t)row * p.s_sl)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+      const float2 w1 = twiddle_fwd((unsigned)tp, 196u);
+      const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
+      unsigned char* Bh = Bsm[hl >> 1];
+      const int nu0 = (hl & 1) * 128 + 4 * chunk;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float2 x[4];
+#pragma unroll
+        for (int n1 = 0; n1 < 4; ++n1) {
+          const uint32_t u = j == 0 ? rr[n1].x : (j == 1 ? rr[n1].y : (j == 2 ? rr[n1].z : rr[n1].w));
+          x[n1] = make_float2(0.5f * __uint_as_float(u << 16), 0.5f * __uint_as_float(u & 0xffff0000u));
+        }
+        Dft<4, false>::run(x);
+        x[1] = cmul(x[1], w1);
+        x[2] = cmul(x[2], w2);
+        x[3] = cmul(x[3], w3);
+#pragma unroll
+        for (int k1 = 0; k1 < 4; ++k1)
+          *reinterpret_cast<uint32_t*>(Bh + b_off(nu0 + 32 * k1 + j, 2 * tp)) = pack_h2(x[k1].x, x[k1].y);
+      }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_arrive(smem_u32(&bars[0]));
+    mbar_arrive(smem_u32(&bars[1]));
+
+    // ---- gate tables: head hl, entry k1 * 64 + kM holds G_ext[k1 + 4 kM] / gmax(head) as fp16 ----
+    float2 gv[2];
+    float gm[2];
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int e = tid + it * kTcEpiThreads, hl = e >> 8, idx = e & 255, k1 = idx >> 6, kM = idx & 63;
+      const int hg = head0 + hl;
+      float2 v = make_float2(0.f, 0.f);
+      if (kM < 49 && hg < p.nheads) {
+        const int k = k1 + 4 * kM, kk = k <= 98 ? k : 196 - k;
+        v = __ldg(p.g + (size_t)hg * 99 + kk);
+        if (kk != k) v.y = -v.y;
+        if (k == 0 || k == 98) v.y = 0.f;
+      }
+      gv[it] = v;
+      float m = fmaxf(fabsf(v.x), fabsf(v.y));
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      gm[it] = m;
+    }
+    // warps 0-7 hold head 0 (it = 0) and head 2 (it = 1); warps 8-15 heads 1 and 3
+    if (T == 0) red[warp] = gm[0];
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+    if (tid < 2) { float m = 0.f; for (int i = 0; i < 8; ++i) m = fmaxf(m, red[8 * tid + i]); gmax_s[tid] = 1.41421356f * m; }
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+    if (T == 0) red[warp] = gm[1];
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+    if (tid < 2) { float m = 0.f; for (int i = 0; i < 8; ++i) m = fmaxf(m, red[8 * tid + i]); gmax_s[2 + tid] = 1.41421356f * m; }
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int e = tid + it * kTcEpiThreads, hl = e >> 8;
+      const float gmx = gmax_s[hl], inv = gmx > 0.f ? 1.0f / gmx : 0.f;
+      Gsm[e] = pack_h2(gv[it].x * inv, gv[it].y * inv);
+    }
+    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+
+    const int q = warp & 3, cq = warp >> 2;
+    const int i = T >> 2, t4 = T & 3;
+    bool ok = true;
+    // ---- gate epilogue: rows kM, columns (head, k1, pair) unchanged; next operand has K = kM ----
+#pragma unroll 1
+    for (int half = 0; half < 2 && ok; ++half) {
+      ok = mbar_wait(smem_u32(&bars[2 + half]), 0);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t taddr0 = tmem + 256 * half + ((uint32_t)(32 * q) << 16) + 64 * cq;
+      const int hl = 2 * half + (cq >> 1);
+      uint32_t r[2][16];
+      tmem_ld_16x256b_x4(taddr0, r[0]);
+#pragma unroll
+      for (int step = 0; step < 4; ++step) {
+        const int j = step >> 1, chunk = step & 1;
+        const int kM = 8 * (2 * q + j) + i, k1 = 2 * (cq & 1) + chunk;
+        tmem_ld_wait();
+        if (step < 3) tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * ((step + 1) >> 1)) << 16) + 32 * ((step + 1) & 1), r[(step + 1) & 1]);
+        const uint32_t (&rr)[16] = r[step & 1];
+        const uint32_t gu = Gsm[hl * 256 + k1 * 64 + kM];
+        const float2 g = __half22float2(*reinterpret_cast<const __half2*>(&gu));
+        const uint32_t base = (uint32_t)((8 * cq + 4 * chunk) * kTcSbo + (2 * t4) * 16 + (kM >> 2) * kTcLbo + (kM & 3) * 4);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), g);
+          float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), g);
+          *reinterpret_cast<uint32_t*>(Bsm[half] + base + x * kTcSbo) = pack_h2(v0.x, -v0.y);
+          *reinterpret_cast<uint32_t*>(Bsm[half] + base + x * kTcSbo + 16) = pack_h2(v1.x, -v1.y);
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&bars[half]));
+    }
+    // ---- final: rows t', inverse radix-4 over k1 (columns 32 apart), bf16 rows t' + 49 n1 ----
+#pragma unroll 1
+    for (int half = 0; half < 2 && ok; ++half) {
+      ok = mbar_wait(smem_u32(&bars[2 + half]), 1);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int hl = 2 * half + (cq >> 1), hg = head0 + hl;
+      if (hg >= p.nheads) continue;
+      const int b = hg / p.H, h = hg - b * p.H;
+      const float gs = 0.5f * gmax_s[hl];
+      bf16* dst = p.dst + b * p.d_sb + h * p.d_sh;
+#pragma unroll 1
+      for (int j = 0; j < 2; ++j) {
+        const int tp = 8 * (2 * q + j) + i;
+        if (8 * (2 * q + j) >= 49) continue;                         // warp-uniform: no valid rows in this lane group
+        const float2 w1 = twiddle_fwd((unsigned)(tp < 49 ? tp : 0), 196u);
+        const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
+#pragma unroll 1
+        for (int g8 = 0; g8 < 2; ++g8) {
+          const int cbase = 16 * (cq & 1) + 8 * g8;                 // first pair of this 8-column group
+          uint32_t rk[4][4];
+#pragma unroll
+          for (int k1 = 0; k1 < 4; ++k1)
+            tmem_ld_16x256b_x1(tmem + 256 * half + ((uint32_t)(32 * q + 16 * j) << 16) + 128 * (cq >> 1) + 32 * k1 + cbase, rk[k1]);
+          tmem_ld_wait();
+          if (tp < 49) {
+            float2 y0[4], y1[4];
+#pragma unroll
+            for (int k1 = 0; k1 < 4; ++k1) {                         // conj of the accumulator = IDFT49 (conj trick)
+              y0[k1] = make_float2(__uint_as_float(rk[k1][0]), -__uint_as_float(rk[k1][2]));
+              y1[k1] = make_float2(__uint_as_float(rk[k1][1]), -__uint_as_float(rk[k1][3]));
+            }
+            y0[1] = cmulc(y0[1], w1); y0[2] = cmulc(y0[2], w2); y0[3] = cmulc(y0[3], w3);
+            y1[1] = cmulc(y1[1], w1); y1[2] = cmulc(y1[2], w2); y1[3] = cmulc(y1[3], w3);
+            Dft<4, true>::run(y0);
+            Dft<4, true>::run(y1);
+            const int col = 2 * (cbase + 2 * t4);
+#pragma unroll
+            for (int n1 = 0; n1 < 4; ++n1) {
+              const int row = tp + 49 * n1;
+              if (row < p.L)
+                __stcs(reinterpret_cast<uint2*>(dst + (int64_t)row * p.d_sl + col),
+                       pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y));
+            }
+          }
+        }
+      }
+    }
+    if (!ok && T == 0) atomicExch(p.status, 1);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == kTcEpiWarps) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(512));
+  }
+}
+
+// 49-point DFT matrix in real form, scaled by 1/7, zero-padded to 128 x 128, same layout and row
+// order as the 64-point matrix (row 16 g + 8 part + i is bin 8 g + i).
+__global__ void build_dft49_kernel(__half* F) {
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= 128 * 128) return;
+  int m = idx >> 7, kappa = idx & 127;
+  int kd = 8 * (m >> 4) + (m & 7), part_out = (m >> 3) & 1;
+  int t = kappa >> 1, part_in = kappa & 1;
+  float v = 0.f;
+  if (kd < 49 && t < 49) {
+    float s, c;
+    sincospif(2.0f * (float)((kd * t) % 49) / 49.0f, &s, &c);
+    v = part_out == 0 ? (part_in == 0 ? c : s) : (part_in == 0 ? -s : c);
+    v *= 0.14285714285714285f;
+  }
+  size_t off = (size_t)(m >> 3) * 2048 + (size_t)(kappa >> 3) * 128 + (m & 7) * 16 + (kappa & 7) * 2;
+  *reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(F) + off) = __float2half_rn(v);
+}
+
+int build_dft49(__half* F, cudaStream_t st) {
+  build_dft49_kernel<<<64, 256, 0, st>>>(F);
+  SPECTRE_LAUNCH_OK("build_dft49_kernel");
+  return SPECTRE_OK;
+}
+
+int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
+                       const spectre_act* y) {
+  Tc196Params p = {};
+  p.src = reinterpret_cast<const bf16*>(v->ptr);
+  p.dst = reinterpret_cast<bf16*>(y->ptr);
+  p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
+  p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
+  p.g = reinterpret_cast<const float2*>(g);
+  p.F = reinterpret_cast<const __half*>(ctx->dft49);
+  p.H = v->H; p.L = v->L; p.nheads = v->B * v->H;
+  p.status = ctx->status_dev;
+  SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k196Smem));
+  const unsigned grid = (unsigned)((p.nheads + k196Heads - 1) / k196Heads);
+  mixer_tc196_kernel<<<grid, kTcThreads, k196Smem, st>>>(p);
+  SPECTRE_LAUNCH_OK("mixer_tc196_kernel");
+  return SPECTRE_OK;
+}
+
 }  // namespace spectre

@@ -103,6 +103,108 @@ __global__ void __launch_bounds__(256) wavelet_kernel(const WaveletParams p) {
   }
 }
 
+
+// Register-resident variant for J <= 4: a thread owns one aligned block of 2^J tokens of two
+// adjacent channels (4-byte bf16 pairs / 8-byte fp32 pairs), so the refinement is a single
+// streaming pass with no shared-memory tile.  CTA = (batch, head): the level gates are computed
+// (or fetched) once into shared memory, then threads sweep the head's blocks.
+template <typename T> struct pair_io;
+template <> struct pair_io<bf16> {
+  static __device__ __forceinline__ float2 load(const bf16* p) {
+    const uint32_t u = *reinterpret_cast<const uint32_t*>(p);
+    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+  }
+  static __device__ __forceinline__ void store(bf16* p, float2 v) {
+    __nv_bfloat162 o = __floats2bfloat162_rn(v.x, v.y);
+    *reinterpret_cast<uint32_t*>(p) = *reinterpret_cast<uint32_t*>(&o);
+  }
+};
+template <> struct pair_io<float> {
+  static __device__ __forceinline__ float2 load(const float* p) { return *reinterpret_cast<const float2*>(p); }
+  static __device__ __forceinline__ void store(float* p, float2 v) { *reinterpret_cast<float2*>(p) = v; }
+};
+
+template <typename T, typename WT, int J>
+__global__ void __launch_bounds__(256) wavelet_reg_kernel(const WaveletParams p) {
+  extern __shared__ float smw[];
+  float* sg = smw;                                 // [(J+1)][D]  holds 1 + s
+  float* u = sg + (size_t)(J + 1) * p.D;           // [hidden]
+  const int bh = blockIdx.x, b = bh / p.H, h = bh - b * p.H;
+  const int D = p.D;
+  if (p.level_gates) {
+    for (int i = threadIdx.x; i < (J + 1) * D; i += blockDim.x) sg[i] = 1.0f + p.level_gates[(size_t)bh * (J + 1) * D + i];
+  } else {
+    const WT* W1 = reinterpret_cast<const WT*>(p.Ww1) + h * p.hs_w1;
+    const WT* W2 = reinterpret_cast<const WT*>(p.Ww2) + h * p.hs_w2;
+    const float* qb = p.qbar + (size_t)bh * D;
+    for (int j = threadIdx.x; j < p.hidden; j += blockDim.x) {
+      float acc = p.bw1[h * p.hs_b1 + j];
+      for (int c = 0; c < D; ++c) acc = fmaf(qb[c], wl<WT>(W1 + (size_t)c * p.hidden + j), acc);
+      u[j] = gelu_erf(acc);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < (J + 1) * D; i += blockDim.x) {
+      float acc = p.bw2[h * p.hs_b2 + i];
+      for (int j = 0; j < p.hidden; ++j) acc = fmaf(u[j], wl<WT>(W2 + (size_t)j * (J + 1) * D + i), acc);
+      sg[i] = 1.0f + acc;
+    }
+  }
+  __syncthreads();
+  constexpr int S = 1 << J;
+  const float r2 = 0.70710678118654752440f;
+  const int npair = D / 2, nblk = p.L / S;
+  const T* src = reinterpret_cast<const T*>(p.src) + b * p.s_sb + h * p.s_sh;
+  T* dst = reinterpret_cast<T*>(p.dst) + b * p.d_sb + h * p.d_sh;
+  for (int item = threadIdx.x; item < nblk * npair; item += blockDim.x) {
+    const int blk = item / npair, c = 2 * (item - blk * npair);
+    float2 x[S];
+#pragma unroll
+    for (int r = 0; r < S; ++r) x[r] = pair_io<T>::load(src + (int64_t)(blk * S + r) * p.s_sl + c);
+    // analysis in place: after level l, slot i * 2^l holds a_l and slot i * 2^l + 2^(l-1) holds d_l
+#pragma unroll
+    for (int l = 1; l <= J; ++l) {
+      const int span = 1 << l, hs = span >> 1;
+#pragma unroll
+      for (int i = 0; i < S; i += span) {
+        const float2 a = x[i], d = x[i + hs];
+        x[i] = make_float2((a.x + d.x) * r2, (a.y + d.y) * r2);
+        x[i + hs] = make_float2((a.x - d.x) * r2, (a.y - d.y) * r2);
+      }
+    }
+    // modulate: slot 0 is a_J, slot r > 0 is d_l with l = ctz(r) + 1; gate order a_J, d_J, ..., d_1
+#pragma unroll
+    for (int r = 0; r < S; ++r) {
+      const int lev = r == 0 ? 0 : 1 + (J - (__ffs(r)));
+      x[r].x *= sg[lev * D + c];
+      x[r].y *= sg[lev * D + c + 1];
+    }
+#pragma unroll
+    for (int l = J; l >= 1; --l) {
+      const int span = 1 << l, hs = span >> 1;
+#pragma unroll
+      for (int i = 0; i < S; i += span) {
+        const float2 a = x[i], d = x[i + hs];
+        x[i] = make_float2((a.x + d.x) * r2, (a.y + d.y) * r2);
+        x[i + hs] = make_float2((a.x - d.x) * r2, (a.y - d.y) * r2);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < S; ++r) pair_io<T>::store(dst + (int64_t)(blk * S + r) * p.d_sl + c, x[r]);
+  }
+}
+
+template <typename T, typename WT>
+static int launch_wavelet_reg(const WaveletParams& p, int J, unsigned grid, size_t smem, cudaStream_t st) {
+  switch (J) {
+    case 1: wavelet_reg_kernel<T, WT, 1><<<grid, 256, smem, st>>>(p); break;
+    case 2: wavelet_reg_kernel<T, WT, 2><<<grid, 256, smem, st>>>(p); break;
+    case 3: wavelet_reg_kernel<T, WT, 3><<<grid, 256, smem, st>>>(p); break;
+    default: wavelet_reg_kernel<T, WT, 4><<<grid, 256, smem, st>>>(p); break;
+  }
+  SPECTRE_LAUNCH_OK("wavelet_reg_kernel");
+  return SPECTRE_OK;
+}
+
 }  // namespace spectre
 
 using namespace spectre;
@@ -126,6 +228,28 @@ extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spec
       return fail(SPECTRE_ERR_INVALID_ARG, "level_gates is NULL and the MLP inputs are incomplete");
     if (w->hidden < 1 || w->hidden > 1024) return fail(SPECTRE_ERR_UNSUPPORTED, "wavelet hidden width must be in 1..1024");
     if (w->wdtype != SPECTRE_F32 && w->wdtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, "unknown weight dtype");
+  }
+  if (J <= 4) {                              // register-resident streaming kernel
+    SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+    cudaStream_t st0 = reinterpret_cast<cudaStream_t>(stream);
+    const int hidden0 = w->level_gates ? 0 : w->hidden;
+    WaveletParams p0 = {};
+    p0.src = y_in->ptr; p0.dst = y_out->ptr;
+    p0.s_sb = y_in->stride_b; p0.s_sl = y_in->stride_l; p0.s_sh = y_in->stride_h;
+    p0.d_sb = y_out->stride_b; p0.d_sl = y_out->stride_l; p0.d_sh = y_out->stride_h;
+    p0.B = y_in->B; p0.L = L; p0.H = y_in->H; p0.D = D; p0.J = J;
+    p0.level_gates = w->level_gates; p0.qbar = w->qbar; p0.Ww1 = w->Ww1; p0.bw1 = w->bw1; p0.Ww2 = w->Ww2; p0.bw2 = w->bw2;
+    p0.hidden = hidden0;
+    const size_t one0 = w->shared_across_heads ? 0 : 1;
+    p0.hs_w1 = one0 * (size_t)D * hidden0; p0.hs_b1 = one0 * hidden0;
+    p0.hs_w2 = one0 * (size_t)hidden0 * (J + 1) * D; p0.hs_b2 = one0 * (size_t)(J + 1) * D;
+    const size_t smem0 = ((size_t)(J + 1) * D + hidden0) * sizeof(float);
+    const unsigned grid0 = (unsigned)((size_t)p0.B * p0.H);
+    const bool bf0 = y_in->dtype == SPECTRE_BF16, wbf0 = w->wdtype == SPECTRE_BF16;
+    if (bf0 && wbf0) return launch_wavelet_reg<bf16, bf16>(p0, J, grid0, smem0, st0);
+    if (bf0) return launch_wavelet_reg<bf16, float>(p0, J, grid0, smem0, st0);
+    if (wbf0) return launch_wavelet_reg<float, bf16>(p0, J, grid0, smem0, st0);
+    return launch_wavelet_reg<float, float>(p0, J, grid0, smem0, st0);
   }
   const int span = 1 << J;
   int rows = (8192 / D) / span * span;      // about 32 KB of fp32 per CTA

@@ -86,6 +86,18 @@ def test_mixer_bf16_tensor_core_zero_pad_and_strides(ctx):
     assert float(y[:, :, :2].abs().max()) == 0.0
 
 
+@pytest.mark.parametrize("B,H,L", [(1, 3, 196), (3, 5, 196), (2, 2, 150), (64, 12, 196)])
+def test_mixer_bf16_196_tensor_core(ctx, B, H, L, monkeypatch):
+    # 196 = 4 x 49 on the tensor cores (D = 64); head counts that do not fill a CTA, zero-padded rows
+    w = W.Workload("t", B=B, L=L, H=H, D=64, dtype="bf16", n_fft=196, seed=B * 100 + H)
+    e_tc = run_mixer(ctx, w, structured=True, n_fft=196)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    assert e_tc < TOL["bf16"]
+    monkeypatch.setenv("SPECTRE_FORCE_PATH", "alu")          # the fp32 butterfly path must agree too
+    assert run_mixer(ctx, w, structured=True, n_fft=196) < TOL["bf16"]
+
+
 def test_mixer_structured_inputs(ctx):
     # per-channel offsets and x30 outlier channels
     for dt in ("f32", "bf16"):
