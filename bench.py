@@ -163,7 +163,7 @@ class MixerBench:
             self.sets.append(d)
         self.units_per_step = w.B * w.L                                  # tokens
         self.alg_bytes = mixer_algorithmic_bytes(w)
-        # kernels per step: gate = pool + hidden + output layer; mixer = 1 (single-kernel paths) or
+        # kernels per step: gate = pool + output layer; mixer = 1 (single-kernel paths) or
         # gate images + transpose-in + core + transpose-out per group of heads (staged tensor-core
         # path) or strided + on-chip + strided per group (fp32 four-step path); + wavelet
         import math
@@ -180,7 +180,7 @@ class MixerBench:
             self.kernel_name, nk = "mixer (strided + onchip + strided per group)", 3 * groups
         else:
             self.kernel_name, nk = "mixer (onchip_kernel)", 1
-        self.launches_per_step = 3 + nk + (1 if w.wavelet_levels else 0)
+        self.launches_per_step = 2 + nk + (1 if w.wavelet_levels else 0)
         self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         self.d2h = self.h2d
 

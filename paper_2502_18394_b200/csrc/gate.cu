@@ -1,8 +1,8 @@
 // Content-adaptive spectral gate (Sec. 3.2 step 3; Sec. 3.3.2 steps c-d).
 //   pool_kernel      sum of the query tokens over the sequence (bandwidth-bound)
-//   gate_hidden_kernel LayerNorm + hidden layer, once per (batch, head)
-//   gate_out_kernel    output layer as a stream over W2; with the Toeplitz update off
-//                      it also applies modReLU and the positional phase
+//   gate_out_kernel    LayerNorm + hidden layer (per CTA) and the output layer as a stream
+//                      over W2; with the Toeplitz update off it also applies modReLU and
+//                      the positional phase
 //   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
 #include "common.cuh"
 
@@ -184,22 +184,6 @@ struct GateMlpParams {
   int post;               // 1: Toeplitz follows, skip modReLU/phase here
 };
 
-// LayerNorm + hidden layer once per (batch, head): u[B,H,hidden] (and q_bar for the caller).
-template <typename WT>
-__global__ void __launch_bounds__(128) gate_hidden_kernel(const GateMlpParams p) {
-  extern __shared__ float smf[];
-  float* qbar = smf;                 // [D]
-  float* u = smf + p.D;              // [hidden]
-  float* red = u + p.hidden;         // [32]
-  const int bh = blockIdx.x, h = bh % p.H;
-  const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-  descriptor_and_hidden<WT>(p.sums + (size_t)bh * p.D, p.ncopy, p.copy_stride, p.inv_count, p.D, p.hidden,
-                            p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1, p.b1 + h * p.hs_b1, qbar, u, red);
-  if (p.qbar_out)
-    for (int c = threadIdx.x; c < p.D; c += blockDim.x) p.qbar_out[(size_t)bh * p.D + c] = qbar[c];
-  for (int j = threadIdx.x; j < p.hidden; j += blockDim.x) p.u_ws[(size_t)bh * p.hidden + j] = u[j];
-}
-
 // raw (re, im) weight pair of one bin in one hidden row
 template <typename WT> struct wraw;
 template <> struct wraw<bf16> {
@@ -234,8 +218,17 @@ __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
     for (int i = 0; i < R; ++i)
       if (i < n0) w[i] = wraw<WT>::load(col + (size_t)i * ld);
   }
-  for (int j = threadIdx.x; j < p.hidden; j += blockDim.x) u[j] = p.u_ws[(size_t)bh * p.hidden + j];
-  __syncthreads();
+  // LayerNorm + hidden layer, repeated by every CTA of the head (a few thousand FLOPs, two short
+  // round trips) while this thread's W2 column is already on its way
+  {
+    float* qbar = u + p.hidden;        // [D]
+    float* red = qbar + p.D;           // [32]
+    const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
+    descriptor_and_hidden<WT>(p.sums + (size_t)bh * p.D, p.ncopy, p.copy_stride, p.inv_count, p.D, p.hidden,
+                              p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1, p.b1 + h * p.hs_b1, qbar, u, red);
+    if (p.qbar_out && blockIdx.x == 0)
+      for (int c = threadIdx.x; c < p.D; c += blockDim.x) p.qbar_out[(size_t)bh * p.D + c] = qbar[c];
+  }
   if (!live) return;
   const float* b2 = p.b2 + h * p.hs_b2;
   float2 acc = make_float2(b2[2 * k], b2[2 * k + 1]);
@@ -381,14 +374,12 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   dim3 grid((K + 255) / 256, B * H);
   if (grid.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H exceeds 65535");
   size_t smem = (size_t)(D + gp->hidden + 32) * sizeof(float);
-  if (gp->wdtype == SPECTRE_BF16) {
-    gate_hidden_kernel<bf16><<<B * H, 128, smem, st>>>(mp);
-    gate_out_kernel<bf16><<<grid, 256, gp->hidden * sizeof(float), st>>>(mp);
-  } else {
-    gate_hidden_kernel<float><<<B * H, 128, smem, st>>>(mp);
-    gate_out_kernel<float><<<grid, 256, gp->hidden * sizeof(float), st>>>(mp);
-  }
-  SPECTRE_LAUNCH_OK("gate_hidden_kernel / gate_out_kernel");
+  // block sized to the bin count for short transforms (K = 99 does not need 256 threads)
+  const int thr_out = K >= 256 ? 256 : ((K + 31) / 32 * 32 < 64 ? 64 : (K + 31) / 32 * 32);
+  dim3 grid_out((K + thr_out - 1) / thr_out, B * H);
+  if (gp->wdtype == SPECTRE_BF16) gate_out_kernel<bf16><<<grid_out, thr_out, smem, st>>>(mp);
+  else gate_out_kernel<float><<<grid_out, thr_out, smem, st>>>(mp);
+  SPECTRE_LAUNCH_OK("gate_out_kernel");
   if (r > 0) {
     GatePostParams pp = {};
     pp.g_raw = raw; pp.g_out = reinterpret_cast<float2*>(g_out);

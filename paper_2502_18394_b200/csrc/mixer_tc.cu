@@ -481,6 +481,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
 
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
   const int head0 = blockIdx.x * k196Heads;
+  TC_STAMP(0);
 
   if (warp == kTcEpiWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(512));
@@ -504,6 +505,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = tmem_slot;
+  TC_STAMP(1);
 
   if (warp == kTcEpiWarps) {
     // ---- MMA issuer: 2 stages x 2 halves, 7 K-steps each ----
@@ -534,42 +536,54 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
     if (!ok && T == 0) atomicExch(p.status, 1);
   } else {
     // ---- load: rows t' + 49 n1 of each head, radix-4 over n1, twiddle, fp16, operand (K = t', column = (head, k1, pair)) ----
-    // a warp takes 4 consecutive t' x 8 chunks of 16 bytes (conflict-free operand stores)
-    for (int item = warp; item < k196Heads * 13; item += kTcEpiWarps) {
+    // a warp takes 4 consecutive t' x 8 chunks of 16 bytes (conflict-free operand stores); all of
+    // a warp's rows (up to 4 items x 4 rows) are requested before the first one is used
+    constexpr int kItems = (k196Heads * 13 + kTcEpiWarps - 1) / kTcEpiWarps;
+    uint4 rr[kItems][4];
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const int item = warp + it * kTcEpiWarps;
       const int hl = item / 13, tg = item - hl * 13;
-      const int tp = 4 * tg + (T >> 3), chunk = T & 7;
-      const int hg = head0 + hl;
-      if (tp >= 49 || hg >= p.nheads) continue;
-      const int b = hg / p.H, h = hg - b * p.H;
-      const bf16* src = p.src + b * p.s_sb + h * p.s_sh + 8 * chunk;
-      uint4 rr[4];
+      const int tp = 4 * tg + (T >> 3), hg = head0 + hl;
+      const bool live = item < k196Heads * 13 && tp < 49 && hg < p.nheads;
+      const int b = live ? hg / p.H : 0, h = live ? hg - b * p.H : 0;
+      const bf16* src = p.src + b * p.s_sb + h * p.s_sh + 8 * (T & 7);
 #pragma unroll
       for (int n1 = 0; n1 < 4; ++n1) {
         const int row = tp + 49 * n1;
-        rr[n1] = row < p.L ? __ldcg(reinterpret_cast<const uint4*>(src + (int64_t)row * p.s_sl)) : make_uint4(0u, 0u, 0u, 0u);
+        rr[it][n1] = (live && row < p.L) ? __ldcg(reinterpret_cast<const uint4*>(src + (int64_t)row * p.s_sl))
+                                         : make_uint4(0u, 0u, 0u, 0u);
       }
+    }
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const int item = warp + it * kTcEpiWarps;
+      const int hl = item / 13, tg = item - hl * 13;
+      const int tp = 4 * tg + (T >> 3), chunk = T & 7, hg = head0 + hl;
+      if (item >= k196Heads * 13 || tp >= 49 || hg >= p.nheads) continue;
       const float2 w1 = twiddle_fwd((unsigned)tp, 196u);
       const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
-      unsigned char* Bh = Bsm[hl >> 1];
-      const int nu0 = (hl & 1) * 128 + 4 * chunk;
+      unsigned char* Bh = Bsm[hl >> 1] + b_off((hl & 1) * 128 + 4 * chunk, 2 * tp);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         float2 x[4];
 #pragma unroll
         for (int n1 = 0; n1 < 4; ++n1) {
-          const uint32_t u = j == 0 ? rr[n1].x : (j == 1 ? rr[n1].y : (j == 2 ? rr[n1].z : rr[n1].w));
+          const uint32_t u = j == 0 ? rr[it][n1].x : (j == 1 ? rr[it][n1].y : (j == 2 ? rr[it][n1].z : rr[it][n1].w));
           x[n1] = make_float2(0.5f * __uint_as_float(u << 16), 0.5f * __uint_as_float(u & 0xffff0000u));
         }
         Dft<4, false>::run(x);
         x[1] = cmul(x[1], w1);
         x[2] = cmul(x[2], w2);
         x[3] = cmul(x[3], w3);
+        // column (head, k1, pair): k1 moves 32 columns = 4 groups of 8, j moves one row of 16 bytes
 #pragma unroll
         for (int k1 = 0; k1 < 4; ++k1)
-          *reinterpret_cast<uint32_t*>(Bh + b_off(nu0 + 32 * k1 + j, 2 * tp)) = pack_h2(x[k1].x, x[k1].y);
+          *reinterpret_cast<uint32_t*>(Bh + 4 * k1 * kTcSbo + 16 * j) = pack_h2(x[k1].x, x[k1].y);
       }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    TC_STAMP(2);
     mbar_arrive(smem_u32(&bars[0]));
     mbar_arrive(smem_u32(&bars[1]));
 
@@ -612,6 +626,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
     const int q = warp & 3, cq = warp >> 2;
     const int i = T >> 2, t4 = T & 3;
     bool ok = true;
+    TC_STAMP(3);
     // ---- gate epilogue: rows kM, columns (head, k1, pair) unchanged; next operand has K = kM ----
 #pragma unroll 1
     for (int half = 0; half < 2 && ok; ++half) {
@@ -642,6 +657,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      TC_STAMP(4 + half);
       mbar_arrive(smem_u32(&bars[half]));
     }
     // ---- final: rows t', inverse radix-4 over k1 (columns 32 apart), bf16 rows t' + 49 n1 ----
@@ -655,32 +671,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       const int b = hg / p.H, h = hg - b * p.H;
       const float gs = 0.5f * gmax_s[hl];
       bf16* dst = p.dst + b * p.d_sb + h * p.d_sh;
-#pragma unroll 1
-      for (int j = 0; j < 2; ++j) {
-        const int tp = 8 * (2 * q + j) + i;
-        if (8 * (2 * q + j) >= 49) continue;                         // warp-uniform: no valid rows in this lane group
-        const float2 w1 = twiddle_fwd((unsigned)(tp < 49 ? tp : 0), 196u);
-        const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
-#pragma unroll 1
-        for (int g8 = 0; g8 < 2; ++g8) {
-          const int cbase = 16 * (cq & 1) + 8 * g8;                 // first pair of this 8-column group
-          uint32_t rk[4][4];
+      const uint32_t tbase = tmem + 256 * half + ((uint32_t)(32 * q) << 16) + 128 * (cq >> 1) + 16 * (cq & 1);
+      const int nstep = (16 * q >= 49) ? 0 : ((16 * q + 8 >= 49) ? 2 : 4);    // lane groups with valid rows (warp-uniform)
+      uint32_t rk[2][4][4];
+      if (nstep > 0) {
 #pragma unroll
-          for (int k1 = 0; k1 < 4; ++k1)
-            tmem_ld_16x256b_x1(tmem + 256 * half + ((uint32_t)(32 * q + 16 * j) << 16) + 128 * (cq >> 1) + 32 * k1 + cbase, rk[k1]);
+        for (int k1 = 0; k1 < 4; ++k1) tmem_ld_16x256b_x1(tbase + 32 * k1, rk[0][k1]);
+      }
+#pragma unroll
+      for (int step = 0; step < 4; ++step) {                       // step = 2 j + g8; accumulator reads run one step ahead
+        if (step < nstep) {
+          const int j = step >> 1, g8 = step & 1;
+          const int tp = 8 * (2 * q + j) + i;
           tmem_ld_wait();
+          if (step + 1 < nstep) {
+            const int nj = (step + 1) >> 1, ng = (step + 1) & 1;
+#pragma unroll
+            for (int k1 = 0; k1 < 4; ++k1)
+              tmem_ld_16x256b_x1(tbase + ((uint32_t)(16 * nj) << 16) + 32 * k1 + 8 * ng, rk[(step + 1) & 1][k1]);
+          }
           if (tp < 49) {
+            const float2 w1 = twiddle_fwd((unsigned)tp, 196u);
+            const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
             float2 y0[4], y1[4];
 #pragma unroll
             for (int k1 = 0; k1 < 4; ++k1) {                         // conj of the accumulator = IDFT49 (conj trick)
-              y0[k1] = make_float2(__uint_as_float(rk[k1][0]), -__uint_as_float(rk[k1][2]));
-              y1[k1] = make_float2(__uint_as_float(rk[k1][1]), -__uint_as_float(rk[k1][3]));
+              y0[k1] = make_float2(__uint_as_float(rk[step & 1][k1][0]), -__uint_as_float(rk[step & 1][k1][2]));
+              y1[k1] = make_float2(__uint_as_float(rk[step & 1][k1][1]), -__uint_as_float(rk[step & 1][k1][3]));
             }
             y0[1] = cmulc(y0[1], w1); y0[2] = cmulc(y0[2], w2); y0[3] = cmulc(y0[3], w3);
             y1[1] = cmulc(y1[1], w1); y1[2] = cmulc(y1[2], w2); y1[3] = cmulc(y1[3], w3);
             Dft<4, true>::run(y0);
             Dft<4, true>::run(y1);
-            const int col = 2 * (cbase + 2 * t4);
+            const int col = 2 * (16 * (cq & 1) + 8 * g8 + 2 * t4);
 #pragma unroll
             for (int n1 = 0; n1 < 4; ++n1) {
               const int row = tp + 49 * n1;
@@ -692,6 +715,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
         }
       }
     }
+    TC_STAMP(6);
     if (!ok && T == 0) atomicExch(p.status, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
