@@ -115,6 +115,11 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
   const int npair = p.D / 2;
   const bf16* src = p.src + b * p.s_sb + h * p.s_sh;
   const float sc = in_scale(R);
+  // W_n^{t'} of this CTA's 4 NT2 values of t', once (index = row set)
+  __shared__ float2 tws[4 * NT2];
+  for (int rs = threadIdx.x; rs < 4 * NT2; rs += 256)
+    tws[rs] = twiddle_fwd((unsigned)(64 * (4 * t1g + (rs & 3)) + t2b * NT2 + (rs >> 2)), (unsigned)p.n);
+  __syncthreads();
 
   for (int cb = 0; cb < npair; cb += 32) {                     // column blocks of 32 pairs (D = 64: one)
     const int c = cb + lane;
@@ -135,7 +140,7 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
         x[n1] = make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
       }
       Dft<R, false>::run(x);
-      const float2 w1 = twiddle_fwd((unsigned)tp, (unsigned)p.n);
+      const float2 w1 = tws[rs];
       if (live) {
         // word inside the 128-byte core matrix: (t2 % 2, c4, t1 % 4), XOR-skewed by the tile
         const int wl = ((t2l & 1) * 16 + c4 * 4 + t1m) ^ tile_skew(tile);
@@ -475,7 +480,9 @@ __global__ void __launch_bounds__(256, 2) tc_out_kernel(const TcOutParams p) {
 
   // gate scales of this head's R units, times 1 / (R s_in)
   __shared__ float gsc[R];
+  __shared__ float2 tws[NT];                                   // W_n^{t'} of this CTA's t'
   if (threadIdx.x < R) gsc[threadIdx.x] = __ldg(p.gscale + slab_local * R + threadIdx.x) * base_scale;
+  for (int tl = threadIdx.x; tl < NT; tl += 256) tws[tl] = twiddle_fwd((unsigned)(tb * NT + tl), (unsigned)p.n);
   __syncthreads();
   // phase 1: a warp takes (tile, 8 consecutive t'); lane = (t' % 8, pair within the tile)
   const int nitems = p.ntile * (NT / 8);
@@ -491,7 +498,7 @@ __global__ void __launch_bounds__(256, 2) tc_out_kernel(const TcOutParams p) {
       float2 f = h2unpack(__ldg(pu + k1 * ustride));
       x[k1] = make_float2(f.x * gsc[k1], -f.y * gsc[k1]);       // result of conj(FFT(conj(.))), scaled
     }
-    const float2 w1 = twiddle_fwd((unsigned)tp, (unsigned)p.n);
+    const float2 w1 = tws[tl];
     float2 w = w1;
 #pragma unroll
     for (int k = 1; k < R; ++k) {
