@@ -10,15 +10,17 @@
 //                   shared memory so that the workspace writes are whole lines too)
 //   tc_gate_kernel  per (head, k1): the 4096 gate values the unit needs (Hermitian extension,
 //                   normalised by their maximum, fp16) in the order the core reads them
-//   tc_core_kernel  persistent; every SM runs two independent pipelines, each taking a unit
-//                   through   bulk copy -> [MMA -> epilogue] x 4   with the 64-point DFT
-//                   matrix as the A operand (see mixer_tc.cu for the formulation); while one
-//                   pipeline's epilogue occupies the ALUs the other's MMAs occupy the tensor
-//                   core.  Result: the unit's 4096 x 4 complex outputs in fp16, tile-major
+//   tc_core_kernel  persistent, one CTA per SM, units taken in pairs: 16 epilogue warps alternate
+//                   between the two units while a producer warp fetches the operand images with
+//                   bulk async copies and issues the MMAs (64-point DFT matrix as the A operand,
+//                   see mixer_tc.cu for the formulation), so one unit's epilogue on the ALUs
+//                   overlaps the other unit's stage on the tensor core; 4 x [MMA -> epilogue] per
+//                   unit.  Result: the unit's 4096 x 4 complex outputs in fp16, tile-major
 //   tc_out_kernel   inverse radix-R over k1 with conj twiddles, 1/n and gate scale, bf16,
 //                   transposed through shared memory into whole-row stores
 //
-// The workspace between the kernels is sized so that a group of heads stays in L2.
+// Heads are processed in groups sized by the workspace (operand images + unit results + gate
+// images per head); larger groups measured faster than groups small enough to stay in L2.
 #include <cuda_fp16.h>
 
 #include <cstdlib>
@@ -93,7 +95,7 @@ __host__ __device__ constexpr float in_scale(int R) {
 struct TcInParams {
   const bf16* src;
   int64_t s_sb, s_sl, s_sh;
-  unsigned char* ws_in;       // [unit][65536]
+  unsigned char* ws_in;       // [unit][k4ImgBytes]
   int H, D, L, n, ntile, slab0;
 };
 
