@@ -29,6 +29,7 @@ namespace spectre {
 
 int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                         const spectre_act* y);   // mixer_tc.cu
+bool tc8192_supported(const spectre_act* v, const spectre_act* y);                     // mixer_tc8k.cu
 int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                        const spectre_act* y);
 
@@ -635,7 +636,7 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   const bool tc_ok = v->dtype == SPECTRE_BF16 && ctx->dft64 != nullptr && force != kPathAlu;
   const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 15);
   const bool tc196 = tc_ok && n_fft == 196 && v->D == 64 && ctx->dft49 != nullptr;
-  const bool fused = tc_ok && n_fft == 8192 && force != kPathStaged;
+  const bool fused = tc_ok && n_fft == 8192 && force != kPathStaged && tc8192_supported(v, y);
   const bool staged = !fused && tc_ok && force != kPathFused && tc4k_supported(n_fft, v->D) && ws_ok &&
                       workspace_bytes >= tc4k_min_workspace(n_fft, v->D);
   if (!staged && !fused && pl.N1 > 1) {
