@@ -41,7 +41,7 @@ L2_BYTES = 126e6
 #     dirty in L2 when the launch ended, so this understates the traffic; nothing is re-read)
 # c3: the four kernels of one staged mixer call at full size (intermediates spill from L2)
 # c4: append_spectrum_kernel measured at B = 2 (1015.3 MB), scaled by 4 to B = 8
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": 36.2e6, "c3": 3126e6, "c4": 4061e6, "c5": None}
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": 36.9e6, "c3": 3126e6, "c4": 4061e6, "c5": None}
 
 
 def measured_peak():

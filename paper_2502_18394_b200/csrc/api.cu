@@ -11,6 +11,7 @@ namespace spectre {
 int build_dft64(__half* F, cudaStream_t st);   // mixer_tc.cu
 int build_tw8192(float2* tab, cudaStream_t st);
 int build_dft49(__half* F, cudaStream_t st);
+int build_tw64x64(float4* tab, cudaStream_t st);
 
 static thread_local std::string g_last_error;
 
@@ -95,12 +96,14 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
   c->dft64 = nullptr;
   c->tw8192 = nullptr;
   c->dft49 = nullptr;
+  c->tw64x64 = nullptr;
   c->status_host = nullptr;
   c->status_dev = nullptr;
   cudaError_t e2 = cudaSetDevice(device);
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft64, 128 * 128 * sizeof(__half));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw8192, 2049 * sizeof(float2));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft49, 128 * 128 * sizeof(__half));
+  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw64x64, 2048 * sizeof(float4));
   if (e2 == cudaSuccess) e2 = cudaHostAlloc(reinterpret_cast<void**>(&c->status_host), sizeof(int), cudaHostAllocMapped);
   if (e2 == cudaSuccess) {
     *c->status_host = 0;
@@ -110,6 +113,7 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
     int rc = build_dft64(reinterpret_cast<__half*>(c->dft64), 0);
     if (rc == SPECTRE_OK) rc = build_tw8192(reinterpret_cast<float2*>(c->tw8192), 0);
     if (rc == SPECTRE_OK) rc = build_dft49(reinterpret_cast<__half*>(c->dft49), 0);
+    if (rc == SPECTRE_OK) rc = build_tw64x64(reinterpret_cast<float4*>(c->tw64x64), 0);
     if (rc == SPECTRE_OK) e2 = cudaStreamSynchronize(0);
     else e2 = cudaErrorUnknown;
   }
@@ -126,6 +130,7 @@ extern "C" int spectre_destroy(spectre_ctx* ctx) {
     if (ctx->dft64) cudaFree(ctx->dft64);
     if (ctx->tw8192) cudaFree(ctx->tw8192);
     if (ctx->dft49) cudaFree(ctx->dft49);
+    if (ctx->tw64x64) cudaFree(ctx->tw64x64);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
   }
   delete ctx;

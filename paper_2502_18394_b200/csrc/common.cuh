@@ -19,6 +19,7 @@ struct spectre_ctx {
   void* dft64;            // device: 64-point DFT matrix (fp16, MMA operand layout), 32 KiB
   void* dft49;            // device: 49-point DFT matrix, same format (n = 196 path), 32 KiB
   void* tw8192;           // device: (cos, sin)(2 pi r / 8192), r = 0..2048 (quarter wave), 16 KiB
+  void* tw64x64;          // device: W_4096^{row d} pairs in the epilogue threads' own order (float4), 32 KiB
   int* status_host;       // pinned, device-mapped status word written by kernels whose waits ran out
   int* status_dev;
 };

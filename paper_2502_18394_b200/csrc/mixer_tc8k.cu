@@ -61,6 +61,7 @@ struct Tc8kParams {
   const float2* g;        // [B*H][4097]
   const __half* F;        // 64-point DFT matrix, canonical smem layout
   const float2* tw;       // quarter-wave twiddle table (8192nds)
+  const float4* tw64;     // stage twiddles W_4096^{row d} in epilogue order
   int H, ntile;
   int* status;            // host-mapped status word (0 = fine)
 };
@@ -89,27 +90,25 @@ __device__ __forceinline__ void tma_store_rows(const CUtensorMap* tm, int col, i
 // Epilogue after a stage whose accumulator has columns 64 c + d (d = the digit still to be
 // contracted), for one warp: TMEM lane quadrant q, pair c.  A thread owns rows (new digit)
 // 16 q' + T/4 for the two lane groups q' = 2q, 2q+1 and the columns d = 32 chunk + 8 x + 2 (T%4)
-// + {0, 1}.  It multiplies by W_4096^{row d} and writes the transposed operand (row -> column
-// index, d -> K) as one 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
+// + {0, 1}.  It multiplies by W_4096^{row d} (read from a table laid out in this thread order, one
+// 16-byte load per x) and writes the transposed operand (row -> column index, d -> K) as one
+// 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
 //   COLS64: output columns 64 c + row (else 4 row + c).
 template <int LBO, int SBO, bool COLS64>
 __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
-                                                 const float2* __restrict__ tw) {
+                                                 const float4* __restrict__ tw) {
   const int i = T >> 2, tq = T & 3;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * c;
   tmem_ld_16x256b_x4(taddr0, r[0]);
-  float2 wrow = make_float2(1.f, 0.f), wstep = wrow;
+  tw += q * 512 + T;
 #pragma unroll
   for (int step = 0; step < 4; ++step) {                      // step = 2 j + chunk
     const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
-    if (chunk == 0) {
-      wrow = twiddle8192(tw, 2u * (unsigned)row);
-      wstep = twiddle8192(tw, 16u * (unsigned)row);
-    }
-    float2 wa = twiddle8192(tw, 2u * (unsigned)((row * (32 * chunk + 2 * tq)) & 4095));
-    float2 wb = cmul(wa, wrow);
+    float4 w[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) w[x] = __ldg(tw + (4 * step + x) * 32);
     tmem_ld_wait();
     if (step < 3) {
       const int nj = (step + 1) >> 1, nchunk = (step + 1) & 1;
@@ -121,13 +120,9 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
     const uint32_t base = colpart + (uint32_t)((8 * chunk + (tq >> 1)) * LBO + 8 * (tq & 1));
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
-      const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), wa);
-      const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), wb);
+      const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), make_float2(w[x].x, w[x].y));
+      const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), make_float2(w[x].z, w[x].w));
       *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
-      if (x < 3) {
-        wa = cmul(wa, wstep);
-        wb = cmul(wb, wstep);
-      }
     }
   }
 }
@@ -328,9 +323,9 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t td = tmem + 256 * half;
         unsigned char* Bh = Bsm[0] + half * k8BBytes;
-        if (stage == 0) epilogue_twiddle<k8Lbo1, k8Sbo1, true>(td, Bh, q, cq, T, p.tw);
+        if (stage == 0) epilogue_twiddle<k8Lbo1, k8Sbo1, true>(td, Bh, q, cq, T, p.tw64);
         else if (stage == 1) epilogue_gate(td, Bh, q, cq, T, Gsm[0] + half * (k8GBytes / 4));
-        else epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bh, q, cq, T, p.tw);
+        else epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bh, q, cq, T, p.tw64);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         TC8K_STAMP(4 + 2 * stage + half);
@@ -460,6 +455,7 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
   p.g = reinterpret_cast<const float2*>(g);
   p.F = reinterpret_cast<const __half*>(ctx->dft64);
   p.tw = reinterpret_cast<const float2*>(ctx->tw8192);
+  p.tw64 = reinterpret_cast<const float4*>(ctx->tw64x64);
   p.H = v->H; p.ntile = v->D / 8;
   p.status = ctx->status_dev;
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k8Smem));
