@@ -39,6 +39,7 @@ __all__ = [
     "dft_direct", "rfft_direct", "irfft_direct", "rfft", "irfft",
     "layer_norm", "gelu_erf", "gate", "hermitian_extend", "mixer",
     "cache_prefill", "cache_append", "cache_recompute", "decode_readout",
+    "decode_readout_rows", "decode_step",
     "haar_forward", "haar_inverse", "wavelet_level_gates", "wavelet_refine",
     "expand_level_gates",
 ]
@@ -288,6 +289,49 @@ def decode_readout(state: dict, g: np.ndarray) -> np.ndarray:
         for h in range(H):
             out[b, :, h, :] = irfft(g[b, h].reshape(K, 1) * P[b, h], N)
     return out
+
+
+def decode_readout_rows(state: dict, g: np.ndarray, rows) -> np.ndarray:
+    """Selected rows of Sec. 3.3.2 step (e), each from the definition of the
+    inverse real transform at one output index (App. B, Corollary 1), with
+    ``X_k = g_k prefix_fft[k]``:
+
+        V~[r] = (1/N) ( Re X_0 + [N even] (-1)^r Re X_{N/2}
+                        + 2 sum_{0 < k < N/2} Re( X_k exp(+j 2 pi k r / N) ) )
+
+    which is the O(K d) per-row cost quoted at the end of Sec. 3.3.2.
+    g [B,H,K] complex, rows: integers in [0, N).  Returns [B, len(rows), H, d]."""
+    N = state["N"]
+    P = state["prefix_fft"]
+    B, H, K, d = P.shape
+    out = np.zeros((B, len(rows), H, d))
+    k = np.arange(K, dtype=np.int64)
+    weight = np.full(K, 2.0)
+    weight[0] = 1.0
+    if N % 2 == 0:
+        weight[N // 2] = 1.0
+    for i, r in enumerate(rows):
+        assert 0 <= int(r) < N
+        ang = 2.0 * np.pi * ((k * int(r)) % N).astype(np.float64) / N
+        e = np.cos(ang) + 1j * np.sin(ang)
+        for b in range(B):
+            for h in range(H):
+                X = g[b, h].reshape(K, 1) * P[b, h]                     # [K,d]
+                out[b, i, h, :] = np.sum(weight.reshape(K, 1) * np.real(X * e.reshape(K, 1)), axis=0) / N
+    return out
+
+
+def decode_step(state: dict, t: int, q_t: np.ndarray, v_t: np.ndarray, gate_params: dict, rows) -> tuple:
+    """DecodeStep of Alg. 1 in the printed order: (a)-(b) update prefix_fft,
+    the ring buffers and sum_q with token t; (c) gate from ``sum_q / N_max``;
+    (d) positional phase ``p = t``; (e) read-out, here for the listed rows.
+    gate_params: keyword arguments of :func:`gate` other than the descriptor,
+    count, length and shift.  Returns (rows [B,len(rows),H,d], g [B,H,K])."""
+    N = state["N"]
+    cache_append(state, t, q_t, v_t)
+    B = state["sum_q"].shape[0]
+    g = gate(state["sum_q"], 1.0 / N, N, shift=[t] * B, **gate_params)
+    return decode_readout_rows(state, g, rows), g
 
 
 # --------------------------------------------------------------------------

@@ -86,6 +86,24 @@ def test_mixer_bf16_tensor_core_zero_pad_and_strides(ctx):
     assert float(y[:, :, :2].abs().max()) == 0.0
 
 
+@pytest.mark.parametrize("L", [64, 4160, 8128])
+def test_mixer_bf16_8192_short_sequences_through_the_tensor_maps(ctx, L):
+    # whole 64-row blocks shorter than n: rows beyond L read as zero and are not written;
+    # y is a view into a longer buffer whose tail must stay untouched; then in place
+    w = W.Workload("t", B=2, L=L, H=2, D=64, dtype="bf16", n_fft=8192, seed=L)
+    x = W.activations(w, structured=True).cuda()
+    g = W.random_gate(w).cuda()
+    ybig = torch.full((2, L + 64, 2, 64), 7.0, dtype=torch.bfloat16, device="cuda")
+    S.spectre_mixer_forward(ctx, x, g, y=ybig[:, :L], n_fft=8192)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ref = O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=8192)
+    assert slab_err(W.to_f64(ybig[:, :L]), ref) < TOL["bf16"]
+    assert bool((ybig[:, L:] == 7.0).all())
+    S.spectre_mixer_forward(ctx, x, g, y=x, n_fft=8192)
+    assert slab_err(W.to_f64(x), ref) < TOL["bf16"]
+
+
 @pytest.mark.parametrize("B,H,L", [(1, 3, 196), (3, 5, 196), (2, 2, 150), (64, 12, 196)])
 def test_mixer_bf16_196_tensor_core(ctx, B, H, L, monkeypatch):
     # 196 = 4 x 49 on the tensor cores (D = 64); head counts that do not fill a CTA, zero-padded rows

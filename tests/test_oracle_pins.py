@@ -359,6 +359,60 @@ def test_decode_readout_equals_rotated_full_recompute():
     assert rel(out, np.roll(ref, -t, axis=1)) < 1e-10
 
 
+@pytest.mark.parametrize("N", [16, 15, 2, 3])
+def test_single_row_readout_is_the_inverse_transform_row(N):
+    # written-out inverse DFT of the Hermitian completion (irfft_direct) and the library irfft,
+    # with complex DC / Nyquist products whose imaginary parts must drop out
+    B, H, d = 2, 2, 3
+    K = N // 2 + 1
+    st = {"N": N, "prefix_fft": RNG.standard_normal((B, H, K, d)) + 1j * RNG.standard_normal((B, H, K, d))}
+    g = RNG.standard_normal((B, H, K)) + 1j * RNG.standard_normal((B, H, K))
+    rows = list(range(N))[::-1]
+    out = O.decode_readout_rows(st, g, rows)
+    full = O.decode_readout(st, g)
+    assert rel(out, full[:, rows]) < 1e-12
+    brute = O.irfft_direct(g[1, 0].reshape(K, 1) * st["prefix_fft"][1, 0], N)
+    assert rel(out[1, :, 0, :], brute[rows]) < 1e-12
+
+
+def test_single_row_readout_closed_forms():
+    # one token v at slot s, gate = 1: the window reads back v at row s and 0 elsewhere;
+    # a pure phase exp(+j 2 pi k p / N) moves it to row s - p
+    N, s, p = 12, 7, 3
+    K = N // 2 + 1
+    k = np.arange(K)
+    v = np.array([2.0, -1.0, 0.5])
+    st = {"N": N, "prefix_fft": (np.exp(-2j * np.pi * k * s / N)[:, None] * v[None, :]).reshape(1, 1, K, 3)}
+    ones = np.ones((1, 1, K), dtype=np.complex128)
+    out = O.decode_readout_rows(st, ones, list(range(N)))[0, :, 0, :]
+    expect = np.zeros((N, 3)); expect[s] = v
+    assert np.allclose(out, expect, atol=1e-13)
+    phase = np.exp(2j * np.pi * k * p / N).reshape(1, 1, K)
+    out = O.decode_readout_rows(st, phase, list(range(N)))[0, :, 0, :]
+    expect = np.zeros((N, 3)); expect[s - p] = v
+    assert np.allclose(out, expect, atol=1e-13)
+    # DC-only gate: every row is the window mean of each channel
+    dc = np.zeros((1, 1, K), dtype=np.complex128); dc[0, 0, 0] = 1.0
+    assert np.allclose(O.decode_readout_rows(st, dc, [0, 5])[0, :, 0, :], np.tile(v / N, (2, 1)))
+
+
+def test_decode_step_equals_recompute_on_the_window():
+    # the whole DecodeStep against a from-scratch mixer on the ring buffer: gate from the window's
+    # queries, no phase, then the rotation by t that the phase stands for
+    N, L, B, H, d, hid = 8, 3, 2, 2, 4, 5
+    K = N // 2 + 1
+    p = _gate_params(H, d, hid, K)
+    q = RNG.standard_normal((B, L, H, d)); v = RNG.standard_normal((B, L, H, d))
+    st = O.cache_prefill(q, v, N)
+    rows = [N - 1, 0, 3]
+    for t in range(L, L + 20):
+        out, g = O.decode_step(st, t, RNG.standard_normal((B, H, d)), RNG.standard_normal((B, H, d)), p, rows)
+        g0 = O.gate(st["Q_buf"].sum(axis=1), 1.0 / N, N, **p)
+        ref = np.roll(O.mixer(st["V_buf"], g0), -t, axis=1)
+        assert rel(out, ref[:, rows]) < 1e-10
+        assert np.allclose(np.abs(g), np.abs(g0))
+
+
 # ---------------------------------------------------------------- wavelet
 def test_haar_worked_example():
     w = O.haar_forward(np.array([1.0, 2.0, 3.0, 4.0]), 2)
