@@ -225,9 +225,9 @@ class MixerBench:
 class AppendBench:
     """One Prefix-FFT cache append per step (decode)."""
 
-    def __init__(self, w: W.Workload, dev, nsets=None):
+    def __init__(self, w: W.Workload, dev, nsets=None, decode=False):
         from paper_2502_18394_b200 import binding as S
-        self.S, self.w, self.dev = S, w, dev
+        self.S, self.w, self.dev, self.decode = S, w, dev, decode
         self.ctx = S.Context(dev.index)
         self.cache = S.PrefixCache(w.B, w.H, w.D, w.N_max, dtype=W.torch_dtype(w.dtype), device=dev)
         # state: a full window of random tokens (prefill through the library)
@@ -248,9 +248,27 @@ class AppendBench:
         es = 2 if w.dtype == "bf16" else 4
         self.h2d = 2 * w.B * w.H * w.D * es
         self.d2h = w.B * w.H * w.D * 4
+        if decode:
+            # the whole DecodeStep: ring buffers, gate from the running sum (phase t), and one pass over
+            # the spectrum doing the rank-one update and the read-out of the newest live row
+            N, K = w.N_max, w.N_max // 2 + 1
+            self.params = {k: (v.to(dev) if isinstance(v, torch.Tensor) else v)
+                           for k, v in W.gate_params(W.scaled(w, n_fft=N)).items()}
+            self.rows = [N - 1]
+            self.y_rows = torch.empty((w.B, 1, w.H, w.D), dtype=W.torch_dtype(w.dtype), device=dev)
+            self.g_out = torch.empty((w.B, w.H, K, 2), dtype=torch.float32, device=dev)
+            self.dws = torch.empty(S.spectre_decode_workspace_bytes(self.ctx, w.B, w.H, w.D, N, 1, 0), dtype=torch.uint8, device=dev)
+            wbytes = 2 if w.wdtype == "bf16" else 4
+            self.alg_bytes += w.H * w.hidden * 2 * K * wbytes + 2 * w.B * w.H * K * 8   # + W2 stream, gate write + read
+            self.kernel_name = "decode step (decode_spectrum_kernel dominant)"
+            self.launches_per_step = 5      # ring, gate_out, gate_post, decode_spectrum, decode_reduce
+            self.d2h = w.B * w.H * w.D * es
 
     def _call(self, k):
         i = k % 64
+        if self.decode:
+            return self.S.prepare_decode_step(self.ctx, self.cache, self.qd[i], self.vd[i], self.t0 + k, self.params,
+                                              self.rows, self.y_rows, self.g_out, self.dws)
         return self.S.prepare_append(self.ctx, self.cache, self.qd[i], self.vd[i], self.t0 + k)
 
     def step(self, k: int, e0=None, e1=None):
@@ -265,13 +283,15 @@ class AppendBench:
         self.pin_q = self.q_host.pin_memory()
         self.pin_v = self.v_host.pin_memory()
         self.pin_s = torch.empty((self.w.B, self.w.H, self.w.D), dtype=torch.float32).pin_memory()
+        if self.decode:
+            self.pin_s = torch.empty_like(self.y_rows, device="cpu").pin_memory()
 
     def e2e_step(self, k: int):
         i = k % 64
         self.qd[i].copy_(self.pin_q[i], non_blocking=True)
         self.vd[i].copy_(self.pin_v[i], non_blocking=True)
         self._call(100000 + k)()
-        self.pin_s.copy_(self.cache.sum_q, non_blocking=True)
+        self.pin_s.copy_(self.y_rows if self.decode else self.cache.sum_q, non_blocking=True)
 
     def cpu_step(self):
         # bounded sample: one (batch) row of the cache, all heads; scaled to tokens/s
@@ -284,13 +304,20 @@ class AppendBench:
               "V_buf": rng.standard_normal((1, N, w.H, w.D)), "Q_buf": rng.standard_normal((1, N, w.H, w.D)),
               "sum_q": np.zeros((1, w.H, w.D))}
         q = W.to_f64(self.q_host[0][:1]); v = W.to_f64(self.v_host[0][:1])
+        if getattr(self, "decode", False):
+            gp = W.gate_params(W.scaled(w, n_fft=N))
+            pn = {k: (W.to_f64(a) if isinstance(a, torch.Tensor) else a) for k, a in gp.items()
+                  if k in ("ln_gamma", "ln_beta", "ln_eps", "W1", "b1", "W2", "b2")}
+            t0 = time.perf_counter()
+            O.decode_step(st, N + 5, q, v, pn, [N - 1])
+            return time.perf_counter() - t0, 1
         t0 = time.perf_counter()
         O.cache_append(st, N + 5, q, v)
         return time.perf_counter() - t0, 1
 
 
-def make_bench(w, dev, nsets):
-    return AppendBench(w, dev, nsets) if w.N_max else MixerBench(w, dev, nsets)
+def make_bench(w, dev, nsets, decode=False):
+    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets)
 
 
 # --------------------------------------------------------------------------- arms
@@ -346,6 +373,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
     ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
+    ap.add_argument("--decode", action="store_true", help="c4: time the whole decode step (gate + fused update/read-out)")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
     if args.heads:
@@ -371,7 +399,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
-    bench = make_bench(w, dev, args.sets)
+    bench = make_bench(w, dev, args.sets, args.decode)
 
     for k in range(Wm):
         bench.step(k)
@@ -429,7 +457,7 @@ def main():
             "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(w), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
                        "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
                        "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
                              if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},

@@ -243,6 +243,43 @@ int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, const spectre_c
 int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const spectre_cache* cache,
                                 const void* q_t, const void* v_t, int64_t t);
 
+/* Largest number of read-out rows one decode step returns. */
+#define SPECTRE_DECODE_MAX_ROWS 4
+
+/*
+ * spectre_prefix_cache_decode_step - the whole DecodeStep of Alg. 1 for one
+ * token (Sec. 3.3.2 steps a-e), returning selected rows of the read-out:
+ *   (a)-(b) exactly what spectre_prefix_cache_append does for (q_t, v_t, t);
+ *   (c)-(d) g = gate of sum_q / N_max with the positional phase p = t
+ *           (spectre_gate with the cache's running sum, inv_count = 1/N_max);
+ *   (e)     for each listed row r, the entry r of
+ *           V~ = R^{-1}_{N_max}( diag(g) prefix_fft ) by its definition,
+ *             V~[r] = (1/N) sum_k w_k Re( g_k prefix_fft[k] exp(+j 2 pi k r / N) ),
+ *           w_0 = w_{N/2} = 1 and w_k = 2 otherwise (Im of the DC / Nyquist
+ *           products drops out), N = N_max: O(K D) per row, the per-token cost
+ *           quoted at the end of Sec. 3.3.2, instead of a full inverse transform.
+ * The spectrum is read and written once: the rank-one update of Eq. 5 and the
+ * row sums run in the same pass (the gate needs only sum_q, so it is computed
+ * first).  With the phase p = t, row r of V~ is row (r + t) mod N_max of the
+ * un-phased window, i.e. ring-buffer slot (r + t) mod N_max; Alg. 1 returns rows
+ * N_max - L' .. N_max - 1.
+ *   q_t, v_t  [B, H, D] contiguous, dtype buf_dtype (device)
+ *   params    gate network; K = N_max/2 + 1 bins
+ *   rows      HOST array of nrows indices in [0, N_max), 1 <= nrows <= SPECTRE_DECODE_MAX_ROWS
+ *   y_rows    [B, nrows, H, D] contiguous, dtype buf_dtype (device), written
+ *   g_out     [B, H, K, 2] float32 (device), written: the gate of this step
+ *   workspace >= spectre_decode_workspace_bytes(...) bytes, 16-byte aligned
+ * Errors: as spectre_prefix_cache_append and spectre_gate; a row outside the
+ * window or nrows out of range is SPECTRE_ERR_INVALID_ARG before any launch.
+ */
+size_t spectre_decode_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
+                                      int32_t N_max, int32_t nrows, int32_t toeplitz_r);
+int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, const spectre_cache* cache,
+                                     const void* q_t, const void* v_t, int64_t t,
+                                     const spectre_gate_params* params,
+                                     const int32_t* rows, int32_t nrows, void* y_rows, float* g_out,
+                                     void* workspace, size_t workspace_bytes);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,7 +31,9 @@ EXPORTS = [
     "spectre_mixer_workspace_bytes", "spectre_mixer_forward",
     "spectre_wavelet_refine",
     "spectre_prefill_workspace_bytes", "spectre_prefix_cache_prefill", "spectre_prefix_cache_append",
+    "spectre_decode_workspace_bytes", "spectre_prefix_cache_decode_step",
 ]
+DECODE_MAX_ROWS = 4
 
 
 class SpectreError(RuntimeError):
@@ -98,6 +100,11 @@ def lib():
                                                C.c_void_p, C.c_size_t]
     L.spectre_prefix_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
                                               C.c_int64]
+    L.spectre_decode_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 6
+    L.spectre_decode_workspace_bytes.restype = C.c_size_t
+    L.spectre_prefix_cache_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
+                                                   C.c_int64, C.POINTER(GateParams), C.POINTER(C.c_int32), C.c_int32,
+                                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t]
     _lib = L
     return L
 
@@ -314,6 +321,37 @@ def spectre_prefix_cache_append(ctx: Context, cache: PrefixCache, q_t: torch.Ten
     _check(lib().spectre_prefix_cache_append(ctx.handle, _stream(stream), C.byref(cs), _ptr(q_t), _ptr(v_t), int(t)))
 
 
+def spectre_decode_workspace_bytes(ctx: Context, B, H, D, N_max, nrows, toeplitz_r=0) -> int:
+    return lib().spectre_decode_workspace_bytes(ctx.handle, B, H, D, N_max, nrows, toeplitz_r)
+
+
+def spectre_prefix_cache_decode_step(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t: torch.Tensor, t: int,
+                                     params: dict, rows, y_rows: torch.Tensor | None = None,
+                                     g_out: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                                     stream=None):
+    """Whole DecodeStep of Alg. 1 with the listed read-out rows.  Returns (y_rows [B,len(rows),H,D], g [B,H,K,2])."""
+    if not (q_t.is_contiguous() and v_t.is_contiguous()):
+        raise ValueError("q_t and v_t must be contiguous [B, H, D]")
+    rows = [int(r) for r in rows]
+    keep: list = []
+    gp = _gate_struct(params, keep)
+    K = cache.N_max // 2 + 1
+    if y_rows is None:
+        y_rows = torch.empty((cache.B, len(rows), cache.H, cache.D), dtype=v_t.dtype, device=v_t.device)
+    if g_out is None:
+        g_out = torch.empty((cache.B, cache.H, K, 2), dtype=torch.float32, device=v_t.device)
+    if workspace is None:
+        workspace = _workspace(spectre_decode_workspace_bytes(ctx, cache.B, cache.H, cache.D, cache.N_max,
+                                                              max(1, min(len(rows), DECODE_MAX_ROWS)), gp.toeplitz_r),
+                               v_t.device)
+    cs = cache.struct()
+    arr = (C.c_int32 * max(1, len(rows)))(*rows)
+    _check(lib().spectre_prefix_cache_decode_step(ctx.handle, _stream(stream), C.byref(cs), _ptr(q_t), _ptr(v_t), int(t),
+                                                  C.byref(gp), arr, len(rows), _ptr(y_rows), _ptr(g_out),
+                                                  _ptr(workspace), 0 if workspace is None else workspace.numel()))
+    return y_rows, g_out
+
+
 # ---- pre-marshalled calls ---------------------------------------------------------------
 # A launch loop that rebuilds ctypes structures every step spends more host time than the
 # kernels take.  These objects marshal once and replay the identical C call.
@@ -350,6 +388,19 @@ def prepare_mixer_forward(ctx: Context, v: torch.Tensor, g: torch.Tensor, y: tor
     args = (ctx.handle, _stream(stream), C.byref(av), _ptr(g), C.byref(ay), n, None if w is None else C.byref(w),
             _ptr(workspace), 0 if workspace is None else workspace.numel())
     return PreparedCall(lib().spectre_mixer_forward, args, keep)
+
+
+def prepare_decode_step(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t: torch.Tensor, t: int, params: dict,
+                        rows, y_rows: torch.Tensor, g_out: torch.Tensor, workspace: torch.Tensor,
+                        stream=None) -> PreparedCall:
+    cs = cache.struct()
+    keep: list = [cache, q_t, v_t, cs, y_rows, g_out, workspace]
+    gp = _gate_struct(params, keep)
+    arr = (C.c_int32 * len(rows))(*[int(r) for r in rows])
+    keep += [gp, arr]
+    args = (ctx.handle, _stream(stream), C.byref(cs), _ptr(q_t), _ptr(v_t), int(t), C.byref(gp), arr, len(rows),
+            _ptr(y_rows), _ptr(g_out), _ptr(workspace), workspace.numel())
+    return PreparedCall(lib().spectre_prefix_cache_decode_step, args, keep)
 
 
 def prepare_append(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t: torch.Tensor, t: int,

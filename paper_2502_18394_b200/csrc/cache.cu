@@ -1,4 +1,5 @@
-// Prefix-FFT cache (Sec. 3.3, Eq. 5, Alg. 1): prefill and per-token append.
+// Prefix-FFT cache (Sec. 3.3, Eq. 5, Alg. 1): prefill, per-token append, and the whole decode
+// step with single-row read-out.
 #include "common.cuh"
 
 namespace spectre {
@@ -9,6 +10,7 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
 bool transform_supported(const spectre_ctx* ctx, int n);
 size_t transform_slab_bytes(int n, int D);
 int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy);
+size_t gate_min_workspace(int B, int H, int D, int n_fft, int r);
 
 // ---- prefill -----------------------------------------------------------------
 // The forward pass leaves Z = fft_n(a + jb) for each column pair (a, b) in
@@ -122,6 +124,124 @@ __global__ void __launch_bounds__(256) append_ring_kernel(T* __restrict__ V_buf,
   sum_q[idx] += qn - qo;
   Q_buf[o] = q_t[idx];
   V_buf[o] = v_t[idx];
+}
+
+
+// ---- decode step -------------------------------------------------------------
+// Ring buffers and running sum as in the append, plus delta = v_t - v_old in fp32 for the
+// spectrum pass (which then no longer needs the ring buffer).
+template <typename T>
+__global__ void __launch_bounds__(256) decode_ring_kernel(T* __restrict__ V_buf, T* __restrict__ Q_buf,
+                                                          float* __restrict__ sum_q, float* __restrict__ delta,
+                                                          const T* __restrict__ q_t, const T* __restrict__ v_t, int B,
+                                                          int H, int D, int N, int slot, int evict) {
+  const int total = B * H * D;
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int b = idx / (H * D), hd = idx - b * (H * D);
+  size_t o = ((size_t)b * N + slot) * H * D + hd;
+  float qn = io<T>::load1(q_t + idx), vn = io<T>::load1(v_t + idx);
+  float qo = evict ? io<T>::load1(Q_buf + o) : 0.f;
+  float vo = evict ? io<T>::load1(V_buf + o) : 0.f;
+  sum_q[idx] += qn - qo;
+  delta[idx] = vn - vo;
+  Q_buf[o] = q_t[idx];
+  V_buf[o] = v_t[idx];
+}
+
+struct DecodeRows { int r[SPECTRE_DECODE_MAX_ROWS]; };
+
+// One pass over the spectrum: P_k += delta exp(-j 2 pi k t / N) (Eq. 5) and, from the updated
+// value, the NR read-out rows  V~[r] = (1/N) sum_k w_k Re(g_k P_k exp(+j 2 pi k r / N)),
+// w_0 = w_{N/2} = 1, else 2 (Sec. 3.3.2 step e at one output index).  A CTA takes 256
+// consecutive bins of one (batch, head), a warp 32 of them: lane l evaluates bin k0 + l's
+// update twiddle and its NR read-out coefficients once, then the warp walks the 32 bins with
+// every lane holding 2 channels.  Row sums are reduced over the CTA and written as one
+// partial per (slab, bin block); decode_reduce_kernel adds the partials in a fixed order.
+template <int NR>
+__global__ void __launch_bounds__(256) decode_spectrum_kernel(float* __restrict__ prefix, const float* __restrict__ delta,
+                                                              const float2* __restrict__ g, float* __restrict__ partial,
+                                                              int D, int N, int K, unsigned tm, DecodeRows rows,
+                                                              int nblk) {
+  __shared__ float red[8][NR][64];
+  const int slab = blockIdx.x / nblk, blk = blockIdx.x - slab * nblk;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k0 = (blk * 8 + warp) * 32, k = k0 + lane;
+  float2 my = make_float2(1.f, 0.f);
+  float2 coef[NR];
+#pragma unroll
+  for (int r = 0; r < NR; ++r) coef[r] = make_float2(0.f, 0.f);
+  if (k < K) {
+    my = twiddle_fwd((unsigned)(((unsigned long long)k * tm) % (unsigned)N), (unsigned)N);
+    const float2 gk = __ldg(g + (size_t)slab * K + k);
+    const float wk = ((k == 0 || 2 * k == N) ? 1.0f : 2.0f) / (float)N;
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      const float2 e = twiddle_fwd((unsigned)(((unsigned long long)k * (unsigned)rows.r[r]) % (unsigned)N), (unsigned)N);
+      coef[r] = cscale(cmulc(gk, e), wk);               // g_k exp(+j theta) w_k / N
+    }
+  }
+  const int nb = max(0, min(32, K - k0));
+  const int half = D / 2;
+  float* base = prefix + (((size_t)slab * K + k0) * D) * 2;
+  for (int c0 = 0; c0 < half; c0 += 32) {               // uniform trip count: every lane takes part in the shuffles
+    const int c = c0 + lane;
+    const bool live = c < half;
+    float d0 = 0.f, d1 = 0.f;
+    if (live) {
+      d0 = delta[(size_t)slab * D + 2 * c];
+      d1 = delta[(size_t)slab * D + 2 * c + 1];
+    }
+    float acc[NR][2];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) acc[r][0] = acc[r][1] = 0.f;
+    for (int i = 0; i < nb; ++i) {
+      const float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (live) {
+        float4* p = reinterpret_cast<float4*>(base + ((size_t)i * D + 2 * c) * 2);
+        v = *p;
+        v.x = fmaf(d0, wr, v.x); v.y = fmaf(d0, wi, v.y);
+        v.z = fmaf(d1, wr, v.z); v.w = fmaf(d1, wi, v.w);
+        *p = v;
+      }
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {
+        const float cr = __shfl_sync(0xffffffffu, coef[r].x, i), ci = __shfl_sync(0xffffffffu, coef[r].y, i);
+        acc[r][0] = fmaf(cr, v.x, fmaf(-ci, v.y, acc[r][0]));
+        acc[r][1] = fmaf(cr, v.z, fmaf(-ci, v.w, acc[r][1]));
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      red[warp][r][2 * lane] = acc[r][0];
+      red[warp][r][2 * lane + 1] = acc[r][1];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < NR * 64; e += 256) {
+      const int r = e >> 6, cc = e & 63;
+      if (2 * c0 + cc < D) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += red[w][r][cc];
+        partial[(((size_t)slab * nblk + blk) * NR + r) * D + 2 * c0 + cc] = s;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) decode_reduce_kernel(const float* __restrict__ partial, T* __restrict__ y, int B, int H,
+                                                            int D, int nblk, int NR, int nrows) {
+  const int total = B * nrows * H * D;
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int c = idx % D, h = (idx / D) % H, r = (idx / (D * H)) % nrows, b = idx / (D * H * nrows);
+  const float* p = partial + (((size_t)(b * H + h) * nblk) * NR + r) * D + c;
+  float s = 0.f;
+  for (int blk = 0; blk < nblk; ++blk) s += p[(size_t)blk * NR * D];
+  io<T>::store1(y + idx, s);
 }
 
 static int check_cache(const spectre_cache* c) {
@@ -242,5 +362,80 @@ extern "C" int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const
                                                        reinterpret_cast<const float*>(v_t), B, H, D, N, slot, evict);
   }
   SPECTRE_LAUNCH_OK("append kernels");
+  return SPECTRE_OK;
+}
+
+static size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+static int decode_nr(int nrows) { return nrows <= 1 ? 1 : (nrows <= 2 ? 2 : SPECTRE_DECODE_MAX_ROWS); }
+
+extern "C" size_t spectre_decode_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D, int32_t N_max,
+                                                 int32_t nrows, int32_t toeplitz_r) {
+  (void)ctx;
+  if (B < 1 || H < 1 || D < 1 || N_max < 2 || nrows < 1 || nrows > SPECTRE_DECODE_MAX_ROWS || toeplitz_r < 0) return 0;
+  const int K = N_max / 2 + 1, nblk = (K + 255) / 256;
+  return round256((size_t)B * H * D * 4) + round256((size_t)B * H * nblk * decode_nr(nrows) * D * 4) +
+         gate_min_workspace(B, H, D, N_max, toeplitz_r);
+}
+
+extern "C" int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, const spectre_cache* cache, const void* q_t,
+                                                const void* v_t, int64_t t, const spectre_gate_params* params,
+                                                const int32_t* rows, int32_t nrows, void* y_rows, float* g_out,
+                                                void* workspace, size_t workspace_bytes) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  int rc = check_cache(cache);
+  if (rc != SPECTRE_OK) return rc;
+  if (!q_t || !v_t || !y_rows || !g_out) return fail(SPECTRE_ERR_INVALID_ARG, "token, output or gate pointer is NULL");
+  if (!params) return fail(SPECTRE_ERR_INVALID_ARG, "gate parameters are NULL");
+  if (t < 0) return fail(SPECTRE_ERR_INVALID_ARG, "t must be >= 0");
+  if (!rows || nrows < 1 || nrows > SPECTRE_DECODE_MAX_ROWS)
+    return fail(SPECTRE_ERR_INVALID_ARG, "rows is NULL or nrows outside 1..SPECTRE_DECODE_MAX_ROWS");
+  const int B = cache->B, H = cache->H, D = cache->D, N = cache->N_max;
+  for (int i = 0; i < nrows; ++i)
+    if (rows[i] < 0 || rows[i] >= N) return fail(SPECTRE_ERR_INVALID_ARG, "read-out row outside [0, N_max)");
+  if ((size_t)B * H * D > (size_t)1 << 30) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H*D too large");
+  const int K = N / 2 + 1, nblk = (K + 255) / 256, NR = decode_nr(nrows);
+  if ((size_t)B * H * nblk > (size_t)0x7fffffff) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H*K too large");
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15))
+    return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
+  const size_t delta_bytes = round256((size_t)B * H * D * 4);
+  const size_t part_bytes = round256((size_t)B * H * nblk * NR * D * 4);
+  const size_t gate_bytes = gate_min_workspace(B, H, D, N, params->toeplitz_r < 0 ? 0 : params->toeplitz_r);
+  if (workspace_bytes < delta_bytes + part_bytes + gate_bytes) return fail(SPECTRE_ERR_WORKSPACE, "decode workspace too small");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  float* delta = reinterpret_cast<float*>(workspace);
+  float* partial = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + delta_bytes);
+  void* gate_ws = reinterpret_cast<unsigned char*>(workspace) + delta_bytes + part_bytes;
+  const int slot = (int)(t % N);
+  const int evict = t >= N ? 1 : 0;
+  const bool bf = cache->buf_dtype == SPECTRE_BF16;
+  // (a)-(b) ring buffers, running sum, delta
+  const unsigned blocks_r = (unsigned)(((size_t)B * H * D + 255) / 256);
+  if (bf)
+    decode_ring_kernel<bf16><<<blocks_r, 256, 0, st>>>(reinterpret_cast<bf16*>(cache->V_buf), reinterpret_cast<bf16*>(cache->Q_buf),
+                                                       cache->sum_q, delta, reinterpret_cast<const bf16*>(q_t),
+                                                       reinterpret_cast<const bf16*>(v_t), B, H, D, N, slot, evict);
+  else
+    decode_ring_kernel<float><<<blocks_r, 256, 0, st>>>(reinterpret_cast<float*>(cache->V_buf), reinterpret_cast<float*>(cache->Q_buf),
+                                                        cache->sum_q, delta, reinterpret_cast<const float*>(q_t),
+                                                        reinterpret_cast<const float*>(v_t), B, H, D, N, slot, evict);
+  SPECTRE_LAUNCH_OK("decode_ring_kernel");
+  // (c)-(d) gate from the running sum with phase p = t
+  rc = spectre_gate(ctx, stream, nullptr, cache->sum_q, B, H, D, 1.0f / (float)N, params, N, nullptr, t, g_out, nullptr,
+                    gate_ws, gate_bytes);
+  if (rc != SPECTRE_OK) return rc;
+  // (b) + (e) one pass over the spectrum
+  DecodeRows dr;
+  for (int i = 0; i < SPECTRE_DECODE_MAX_ROWS; ++i) dr.r[i] = rows[i < nrows ? i : nrows - 1];
+  const unsigned blocks_s = (unsigned)((size_t)B * H * nblk);
+  const float2* g2 = reinterpret_cast<const float2*>(g_out);
+  if (NR == 1) decode_spectrum_kernel<1><<<blocks_s, 256, 0, st>>>(cache->prefix_fft, delta, g2, partial, D, N, K, (unsigned)slot, dr, nblk);
+  else if (NR == 2) decode_spectrum_kernel<2><<<blocks_s, 256, 0, st>>>(cache->prefix_fft, delta, g2, partial, D, N, K, (unsigned)slot, dr, nblk);
+  else decode_spectrum_kernel<SPECTRE_DECODE_MAX_ROWS><<<blocks_s, 256, 0, st>>>(cache->prefix_fft, delta, g2, partial, D, N, K, (unsigned)slot, dr, nblk);
+  SPECTRE_LAUNCH_OK("decode_spectrum_kernel");
+  const unsigned blocks_y = (unsigned)(((size_t)B * nrows * H * D + 255) / 256);
+  if (bf) decode_reduce_kernel<bf16><<<blocks_y, 256, 0, st>>>(partial, reinterpret_cast<bf16*>(y_rows), B, H, D, nblk, NR, nrows);
+  else decode_reduce_kernel<float><<<blocks_y, 256, 0, st>>>(partial, reinterpret_cast<float*>(y_rows), B, H, D, nblk, NR, nrows);
+  SPECTRE_LAUNCH_OK("decode_reduce_kernel");
   return SPECTRE_OK;
 }

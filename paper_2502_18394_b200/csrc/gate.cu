@@ -299,6 +299,14 @@ static size_t gate_ws_layout(int B, int H, int D, int n_fft, int r, int hidden, 
 
 using namespace spectre;
 
+namespace spectre {
+// Smallest gate scratch (one copy of the sums, any hidden width); used by the decode step.
+size_t gate_min_workspace(int B, int H, int D, int n_fft, int r) {
+  size_t off, off2;
+  return gate_ws_layout(B, H, D, n_fft, r, 1024, 1, &off, &off2);
+}
+}  // namespace spectre
+
 extern "C" size_t spectre_gate_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D, int32_t n_fft,
                                                int32_t toeplitz_r) {
   (void)ctx;

@@ -105,3 +105,39 @@ def test_c4_full_size_append_sampled_bins(ctx):
                 assert rel_err(W.to_f64(cache.sum_q[b, h]), W.to_f64(cache.Q_buf[b, :, h, :]).sum(axis=0)) < 2e-5
     # the ring buffer holds the last N tokens: slot (N + i) mod N = i was overwritten by append i
     assert torch.equal(cache.V_buf[:, :steps], vd.permute(1, 0, 2, 3))
+
+
+def test_c4_full_size_decode_step_sampled_heads(ctx):
+    # the whole DecodeStep at B = 8, H = 32, d = 64, N_max = 32768 on a full window: after a few
+    # steps, sampled (b, h): read-out rows and gate against the oracle evaluated on the window
+    # (the ring buffers hold the input tokens bit for bit), spectrum against a fresh transform
+    w = W.CONFIGS["c4"]
+    N = w.N_max
+    cache = S.PrefixCache(w.B, w.H, w.D, N)
+    one = W.scaled(w, B=1)
+    q = torch.cat([W.activations(one, stream=10 + b) for b in range(w.B)], dim=0).cuda()
+    v = torch.cat([W.activations(one, stream=30 + b) for b in range(w.B)], dim=0).cuda()
+    S.spectre_prefix_cache_prefill(ctx, cache, q, v)
+    del q, v
+    wg = W.scaled(w, n_fft=N)
+    p = W.gate_params(wg, modrelu_bias_std=0.05)
+    pd, pn = to_dev(p), gate_params_np(p)
+    steps, rows = 5, [N - 1, N - 2]
+    qs, vs = W.decode_tokens(w, steps)
+    qd, vd = qs.cuda(), vs.cuda()
+    for i in range(steps):
+        y, g = S.spectre_prefix_cache_decode_step(ctx, cache, qd[i], vd[i], N + i, pd, rows)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    t = N + steps - 1
+    for (b, h) in [(0, 0), (5, 13), (7, 31)]:
+        win = W.to_f64(cache.V_buf[b, :, h, :])
+        P = O.rfft(win, N)
+        Pg = W.to_f64(cache.prefix_fft[b, h]); Pg = Pg[..., 0] + 1j * Pg[..., 1]
+        assert rel_err(Pg, P) < 2e-5
+        sq = W.to_f64(cache.Q_buf[b, :, h, :]).sum(axis=0)
+        head = {k: (a[h:h + 1] if isinstance(a, np.ndarray) else a) for k, a in pn.items()}
+        g_ref = O.gate(sq.reshape(1, 1, -1), 1.0 / N, N, shift=[t], **head)
+        assert rel_err(gate_to_complex(g[b, h]), g_ref[0, 0]) < 2e-5
+        ref = O.decode_readout_rows({"N": N, "prefix_fft": P.reshape(1, 1, *P.shape)}, g_ref, rows)
+        assert rel_err(W.to_f64(y[b, :, h, :]), ref[0, :, 0, :]) < TOL["bf16"], (b, h)

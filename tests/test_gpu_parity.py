@@ -362,6 +362,72 @@ def test_decode_step_equals_full_recompute(ctx):
     assert slab_err(W.to_f64(y), out) < TOL["bf16"]
 
 
+@pytest.mark.parametrize("dt,N,L,steps,rows", [("f32", 64, 20, 150, [63]), ("bf16", 256, 256, 300, [255, 0, 100]),
+                                               ("f32", 100, 40, 130, [99, 98]), ("bf16", 16384, 16000, 40, [16383, 16382, 5, 8000]),
+                                               ("f32", 1024, 1000, 60, [1023, 1022, 1021])])
+def test_decode_step_rows_against_oracle(ctx, dt, N, L, steps, rows):
+    # the whole DecodeStep of Alg. 1 (cache update, gate with phase t, read-out rows) against the
+    # oracle's, step by step on the same tokens; afterwards the cache equals the oracle's state
+    w = W.Workload("t", B=2, L=L, H=2, D=16, dtype=dt, wdtype="f32", n_fft=N, seed=N + 3 * L, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    p = W.gate_params(w, modrelu_bias_std=0.05, toeplitz_r=2 if N == 256 else 0, bias_std=0.1)
+    pd, pn = to_dev(p), gate_params_np(p)
+    cache = S.PrefixCache(w.B, w.H, w.D, N, dtype=W.torch_dtype(dt))
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    st = O.cache_prefill(W.to_f64(q), W.to_f64(v), N)
+    qs, vs = W.decode_tokens(w, steps)
+    qd, vd = qs.cuda(), vs.cuda()
+    tol_y = 5e-5 if dt == "f32" else TOL["bf16"]
+    for i in range(steps):
+        t = L + i
+        y, g = S.spectre_prefix_cache_decode_step(ctx, cache, qd[i], vd[i], t, pd, rows)
+        ref, g_ref = O.decode_step(st, t, W.to_f64(qs[i]), W.to_f64(vs[i]), pn, rows)
+        if i % 7 == 0 or i == steps - 1:
+            yy = W.to_f64(y)                                             # [B, nrows, H, D]
+            assert yy.shape == ref.shape
+            err = max(rel_err(yy[b, :, h], ref[b, :, h]) for b in range(w.B) for h in range(w.H))
+            assert err < tol_y, (i, err)
+            assert rel_err(gate_to_complex(g), g_ref) < 1e-5
+    e_p, e_s = cache_err(cache, st)
+    assert e_p < 2e-5 and e_s < 2e-5
+    assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
+
+
+def test_decode_step_leaves_the_same_state_as_append(ctx):
+    # steps (a)-(b) inside the fused step are the append's arithmetic: bit-identical state
+    N, L = 512, 500
+    w = W.Workload("t", B=2, L=L, H=3, D=24, dtype="bf16", wdtype="f32", n_fft=N, seed=5, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    pd = to_dev(W.gate_params(w))
+    qs, vs = W.decode_tokens(w, 40)
+    a, b = S.PrefixCache(w.B, w.H, w.D, N), S.PrefixCache(w.B, w.H, w.D, N)
+    S.spectre_prefix_cache_prefill(ctx, a, q.cuda(), v.cuda())
+    for dst, src in zip((b.prefix_fft, b.V_buf, b.Q_buf, b.sum_q), (a.prefix_fft, a.V_buf, a.Q_buf, a.sum_q)):
+        dst.copy_(src)                                               # (the prefill's pooled sum uses float atomics)
+    for i in range(40):
+        S.spectre_prefix_cache_append(ctx, a, qs[i].cuda(), vs[i].cuda(), L + i)
+        S.spectre_prefix_cache_decode_step(ctx, b, qs[i].cuda(), vs[i].cuda(), L + i, pd, [N - 1])
+    assert torch.equal(a.prefix_fft, b.prefix_fft) and torch.equal(a.sum_q, b.sum_q)
+    assert torch.equal(a.V_buf, b.V_buf) and torch.equal(a.Q_buf, b.Q_buf)
+
+
+def test_decode_step_rejects_bad_rows(ctx):
+    N = 64
+    w = W.Workload("t", B=1, L=8, H=2, D=16, dtype="f32", wdtype="f32", n_fft=N, seed=2, N_max=N)
+    pd = to_dev(W.gate_params(w))
+    cache = S.PrefixCache(1, 2, 16, N, dtype=torch.float32)
+    tok = torch.zeros(1, 2, 16, device="cuda")
+    for rows in ([], [0, 1, 2, 3, 4], [64], [-1]):
+        with pytest.raises(S.SpectreError) as e:
+            S.spectre_prefix_cache_decode_step(ctx, cache, tok, tok, 8, pd, rows)
+        assert e.value.status == S.SPECTRE_ERR_INVALID_ARG
+    with pytest.raises(S.SpectreError) as e:
+        S.spectre_prefix_cache_decode_step(ctx, cache, tok, tok, 8, pd, [0],
+                                           workspace=torch.empty(64, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == S.SPECTRE_ERR_WORKSPACE
+    assert float(cache.prefix_fft.abs().max()) == 0.0               # nothing ran
+
+
 # ------------------------------------------------------------------ errors
 def test_invalid_arguments_are_rejected_before_launch(ctx):
     x = torch.zeros(1, 64, 2, 16, device="cuda")
