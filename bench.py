@@ -180,7 +180,8 @@ class MixerBench:
             self.kernel_name, nk = "mixer (strided + onchip + strided per group)", 3 * groups
         else:
             self.kernel_name, nk = "mixer (onchip_kernel)", 1
-        self.launches_per_step = 2 + nk + (1 if w.wavelet_levels else 0)
+        # pool, gate_out (+ gate_hidden when a head's bins span >= 32 CTAs), mixer kernels, wavelet
+        self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels else 0)
         self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         self.d2h = self.h2d
 
@@ -261,7 +262,7 @@ class AppendBench:
             wbytes = 2 if w.wdtype == "bf16" else 4
             self.alg_bytes += w.H * w.hidden * 2 * K * wbytes + 2 * w.B * w.H * K * 8   # + W2 stream, gate write + read
             self.kernel_name = "decode step (decode_spectrum_kernel dominant)"
-            self.launches_per_step = 5      # ring, gate_out, gate_post, decode_spectrum, decode_reduce
+            self.launches_per_step = 5      # ring, gate_hidden, gate_out, decode_spectrum, decode_reduce
             self.d2h = w.B * w.H * w.D * es
 
     def _call(self, k):

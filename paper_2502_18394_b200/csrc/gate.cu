@@ -1,7 +1,8 @@
 // Content-adaptive spectral gate (Sec. 3.2 step 3; Sec. 3.3.2 steps c-d).
 //   pool_kernel      sum of the query tokens over the sequence (bandwidth-bound)
-//   gate_out_kernel    LayerNorm + hidden layer (per CTA) and the output layer as a stream
-//                      over W2; with the Toeplitz update off it also applies modReLU and
+//   gate_hidden_kernel LayerNorm + hidden layer once per (head, batch group), long transforms only
+//   gate_out_kernel    LayerNorm + hidden layer (per CTA, short transforms) and the output layer as a
+//                      stream over W2, 1-8 batch entries per pass; with the Toeplitz update off it also applies modReLU and
 //                      the positional phase
 //   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
 #include "common.cuh"
@@ -106,65 +107,83 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
-// q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the
-// hidden layer u = GELU(q_bar W1 + b1).
+// q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the hidden layer
+// u = GELU(q_bar W1 + b1), for nb batch entries of one head at once: a warp normalises one
+// entry (no block-wide reduction), then the nb x hidden outputs are spread over the CTA.
+// sums points at the first entry's [D] row, bstride is the distance between batch entries;
+// u is written as [hidden][ustride] (batch entry fastest).
 template <typename WT>
-__device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, int ncopy, size_t copy_stride,
-                                                      float inv_count, int D, int hidden,
+__device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, size_t bstride, int nb, int ncopy,
+                                                      size_t copy_stride, float inv_count, int D, int hidden,
                                                       const float* __restrict__ gamma, const float* __restrict__ beta,
                                                       float eps, const WT* __restrict__ W1, const float* __restrict__ b1,
-                                                      float* qbar, float* u, float* red) {
-  float part = 0.f;
-  for (int c = threadIdx.x; c < D; c += blockDim.x) {
-    float m = 0.f;
-    for (int k0 = 0; k0 < ncopy; k0 += 16) {        // all copies in flight at once
-      float v[16];
+                                                      float* qbar, float* u, int ustride) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  for (int bb = warp; bb < nb; bb += nw) {
+    const float* sb = sums + (size_t)bb * bstride;
+    float* qb = qbar + bb * D;
+    float part = 0.f;
+    for (int c = lane; c < D; c += 32) {
+      float m = 0.f;
+      for (int k0 = 0; k0 < ncopy; k0 += 16) {        // all copies in flight at once
+        float v[16];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) v[k] = (k0 + k < ncopy) ? sums[(size_t)(k0 + k) * copy_stride + c] : 0.f;
+        for (int k = 0; k < 16; ++k) v[k] = (k0 + k < ncopy) ? sb[(size_t)(k0 + k) * copy_stride + c] : 0.f;
 #pragma unroll
-      for (int k = 0; k < 16; ++k) m += v[k];
+        for (int k = 0; k < 16; ++k) m += v[k];
+      }
+      m *= inv_count;
+      qb[c] = m;
+      part += m;
     }
-    m *= inv_count;
-    qbar[c] = m;
-    part += m;
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    const float mean = part / (float)D;
+    part = 0.f;
+    for (int c = lane; c < D; c += 32) {
+      float dlt = qb[c] - mean;
+      part += dlt * dlt;
+    }
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    const float rstd = 1.0f / sqrtf(part / (float)D + eps);
+    for (int c = lane; c < D; c += 32) qb[c] = gamma[c] * (qb[c] - mean) * rstd + beta[c];
   }
-  const float mean = block_sum(part, red) / (float)D;
-  part = 0.f;
-  for (int c = threadIdx.x; c < D; c += blockDim.x) {
-    float dlt = qbar[c] - mean;
-    part += dlt * dlt;
-  }
-  const float var = block_sum(part, red) / (float)D;
-  const float rstd = 1.0f / sqrtf(var + eps);
-  for (int c = threadIdx.x; c < D; c += blockDim.x) qbar[c] = gamma[c] * (qbar[c] - mean) * rstd + beta[c];
   __syncthreads();
-  for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
-    float acc = b1[j];
+  for (int item = threadIdx.x; item < nb * hidden; item += blockDim.x) {
+    const int bb = item / hidden, jj = item - bb * hidden;
+    const float* qb = qbar + bb * D;
+    float acc = b1[jj];
     int c = 0;
     for (; c + 32 <= D; c += 32) {                  // 32 independent loads in flight
       float wv[32];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + j);
+      for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + jj);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) acc = fmaf(qbar[c + i], wv[i], acc);
+      for (int i = 0; i < 32; ++i) acc = fmaf(qb[c + i], wv[i], acc);
     }
-    for (; c < D; ++c) acc = fmaf(qbar[c], wload<WT>(W1 + (size_t)c * hidden + j), acc);
-    u[j] = gelu_erf(acc);
+    for (; c < D; ++c) acc = fmaf(qb[c], wload<WT>(W1 + (size_t)c * hidden + jj), acc);
+    u[jj * ustride + bb] = gelu_erf(acc);            // [hidden][ustride]: one row = all batch entries
   }
   __syncthreads();
 }
 
+// modReLU: max(|z| + b, 0) z / |z|   (0 at z = 0)
+__device__ __forceinline__ float2 modrelu(float2 gk, float bias) {
+  const float mag = sqrtf(fmaf(gk.x, gk.x, gk.y * gk.y));
+  const float sc = mag > 0.f ? fmaxf(mag + bias, 0.f) / mag : 0.f;
+  return cscale(gk, sc);
+}
+// positional phase exp(+j 2 pi k p / n), angle reduced in integers
+__device__ __forceinline__ float2 phase_factor(int k, int n, long long shift) {
+  long long pm = shift % n;
+  if (pm < 0) pm += n;
+  if (pm == 0) return make_float2(1.f, 0.f);
+  const unsigned kp = (unsigned)(((unsigned long long)k * (unsigned long long)pm) % (unsigned)n);
+  const float2 w = twiddle_fwd(kp, (unsigned)n);  // exp(-j ...)
+  return make_float2(w.x, -w.y);
+}
 __device__ __forceinline__ float2 modrelu_phase(float2 gk, float bias, int k, int n, unsigned pm) {
-  // modReLU: max(|z| + b, 0) z / |z|   (0 at z = 0)
-  float mag = hypotf(gk.x, gk.y);
-  float sc = mag > 0.f ? fmaxf(mag + bias, 0.f) / mag : 0.f;
-  gk = cscale(gk, sc);
-  // positional phase exp(+j 2 pi k p / n), angle reduced in integers
-  if (pm != 0u) {
-    unsigned kp = (unsigned)(((unsigned long long)k * pm) % (unsigned)n);
-    float2 w = twiddle_fwd(kp, (unsigned)n);      // exp(-j ...)
-    gk = cmulc(gk, w);                            // times its conjugate
-  }
+  gk = modrelu(gk, bias);
+  if (pm != 0u) gk = cmul(gk, phase_factor(k, n, (long long)pm));
   return gk;
 }
 
@@ -172,7 +191,7 @@ struct GateMlpParams {
   const float* sums;      // [ncopy][B,H,D]
   int ncopy; size_t copy_stride;
   float inv_count;
-  int H, D, hidden, n, K;
+  int B, H, D, hidden, n, K;
   size_t hs_ln, hs_w1, hs_b1, hs_w2, hs_b2, hs_mb;   // per-head strides (0 when shared)
   const float* gamma; const float* beta; float eps;
   const void* W1; const float* b1; const void* W2; const float* b2;
@@ -199,14 +218,42 @@ template <> struct wraw<float> {
   static constexpr int kRows = 32;
 };
 
-// Output layer: grid (ceil(K / 256), B*H), one bin per thread.  A thread issues the loads of up
-// to kRows hidden rows of its W2 column before it uses any of them, so the whole column is one
-// memory round trip; the kernel is a pure stream over W2.
-template <typename WT>
+// Output layer: grid (ceil(K / threads), H * ceil(B / BB)), one bin per thread for BB batch
+// entries of one head: W2 is shared by the batch, so a column fetched once serves all of them.
+// A thread issues the loads of up to kRows hidden rows of its W2 column before it uses any of
+// them, so the whole column is one memory round trip; the kernel is a pure stream over W2.
+// Hidden activations of BB batch entries of one head, once: grid H * ceil(B / BB).
+template <typename WT, int BB>
+__global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p) {
+  extern __shared__ __align__(16) float u[];       // [hidden][BB], then q_bar [BB][D]
+  const int nbg = (p.B + BB - 1) / BB;
+  const int h = blockIdx.x / nbg, b0 = (blockIdx.x - h * nbg) * BB;
+  const int nb = min(BB, p.B - b0);
+  float* qbar = u + BB * p.hidden;
+  const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
+  descriptor_and_hidden<WT>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+                            p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
+                            p.b1 + h * p.hs_b1, qbar, u, BB);
+  for (int e = threadIdx.x; e < nb * p.hidden; e += blockDim.x) {
+    const int bb = e / p.hidden, jj = e - bb * p.hidden;
+    p.u_ws[((size_t)(b0 + bb) * p.H + h) * p.hidden + jj] = u[jj * BB + bb];
+  }
+  if (p.qbar_out)
+    for (int e = threadIdx.x; e < nb * p.D; e += blockDim.x) {
+      const int bb = e / p.D, c = e - bb * p.D;
+      p.qbar_out[((size_t)(b0 + bb) * p.H + h) * p.D + c] = qbar[e];
+    }
+}
+
+// PRE: the hidden activations were computed once per (head, batch entry) by gate_hidden_kernel
+// (long transforms: hundreds of CTAs per head would otherwise repeat that work).
+template <typename WT, int BB, bool PRE>
 __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
-  extern __shared__ float u[];       // [hidden]
+  extern __shared__ __align__(16) float u[];       // [hidden][BB], then q_bar [BB][D]
   constexpr int R = wraw<WT>::kRows;
-  const int bh = blockIdx.y, b = bh / p.H, h = bh - b * p.H;
+  const int nbg = (p.B + BB - 1) / BB;
+  const int h = blockIdx.y / nbg, b0 = (blockIdx.y - h * nbg) * BB;
+  const int nb = min(BB, p.B - b0);
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
   const bool live = k < p.K;
   const WT* col = reinterpret_cast<const WT*>(p.W2) + h * p.hs_w2 + 2 * (size_t)(live ? k : 0);
@@ -218,43 +265,78 @@ __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
     for (int i = 0; i < R; ++i)
       if (i < n0) w[i] = wraw<WT>::load(col + (size_t)i * ld);
   }
-  // LayerNorm + hidden layer, repeated by every CTA of the head (a few thousand FLOPs, two short
-  // round trips) while this thread's W2 column is already on its way
-  {
-    float* qbar = u + p.hidden;        // [D]
-    float* red = qbar + p.D;           // [32]
+  if (PRE) {
+    for (int e = threadIdx.x; e < nb * p.hidden; e += blockDim.x) {
+      const int bb = e / p.hidden, jj = e - bb * p.hidden;
+      u[jj * BB + bb] = p.u_ws[((size_t)(b0 + bb) * p.H + h) * p.hidden + jj];
+    }
+    __syncthreads();
+  } else {
+    // LayerNorm + hidden layer, repeated by every CTA of the head (a few thousand FLOPs per batch
+    // entry, two short round trips) while this thread's W2 column is already on its way
+    float* qbar = u + BB * p.hidden;   // [BB][D]
     const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-    descriptor_and_hidden<WT>(p.sums + (size_t)bh * p.D, p.ncopy, p.copy_stride, p.inv_count, p.D, p.hidden,
-                              p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1, p.b1 + h * p.hs_b1, qbar, u, red);
+    descriptor_and_hidden<WT>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+                              p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
+                              p.b1 + h * p.hs_b1, qbar, u, BB);
     if (p.qbar_out && blockIdx.x == 0)
-      for (int c = threadIdx.x; c < p.D; c += blockDim.x) p.qbar_out[(size_t)bh * p.D + c] = qbar[c];
+      for (int e = threadIdx.x; e < nb * p.D; e += blockDim.x) {
+        const int bb = e / p.D, c = e - bb * p.D;
+        p.qbar_out[((size_t)(b0 + bb) * p.H + h) * p.D + c] = qbar[e];
+      }
   }
   if (!live) return;
   const float* b2 = p.b2 + h * p.hs_b2;
-  float2 acc = make_float2(b2[2 * k], b2[2 * k + 1]);
+  float2 acc[BB];
+#pragma unroll
+  for (int bb = 0; bb < BB; ++bb) acc[bb] = make_float2(b2[2 * k], b2[2 * k + 1]);
   for (int j = 0; j < p.hidden; j += R) {
-    const int nb = min(R, p.hidden - j);
+    const int nr = min(R, p.hidden - j);
     if (j > 0) {
 #pragma unroll
       for (int i = 0; i < R; ++i)
-        if (i < nb) w[i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
+        if (i < nr) w[i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
     }
 #pragma unroll
     for (int i = 0; i < R; ++i) {
-      if (i < nb) {
+      if (i < nr) {
         const float2 wv = wraw<WT>::cvt(w[i]);
-        acc.x = fmaf(u[j + i], wv.x, acc.x);
-        acc.y = fmaf(u[j + i], wv.y, acc.y);
+        const float* ur = u + (j + i) * BB;             // entries of absent batch rows hold stale values, never stored
+        float ub[BB];
+        if (BB >= 4) {
+#pragma unroll
+          for (int v = 0; v < BB / 4; ++v) {
+            const float4 t = *reinterpret_cast<const float4*>(ur + 4 * v);
+            ub[4 * v] = t.x; ub[4 * v + 1] = t.y; ub[4 * v + 2] = t.z; ub[4 * v + 3] = t.w;
+          }
+        } else {
+#pragma unroll
+          for (int bb = 0; bb < BB; ++bb) ub[bb] = ur[bb];
+        }
+#pragma unroll
+        for (int bb = 0; bb < BB; ++bb) {
+          acc[bb].x = fmaf(ub[bb], wv.x, acc[bb].x);
+          acc[bb].y = fmaf(ub[bb], wv.y, acc[bb].y);
+        }
       }
     }
   }
-  if (!p.post) {
-    long long sh = p.shift_all + (p.shift ? p.shift[b] : 0);
-    long long pm = sh % p.n; if (pm < 0) pm += p.n;
-    float bias = p.modrelu_bias ? p.modrelu_bias[h * p.hs_mb + k] : 0.f;
-    acc = modrelu_phase(acc, bias, k, p.n, (unsigned)pm);
+  const float bias = (!p.post && p.modrelu_bias) ? p.modrelu_bias[h * p.hs_mb + k] : 0.f;
+  // one positional phase for the whole batch unless per-entry shifts are given
+  float2 ph = make_float2(1.f, 0.f);
+  if (!p.post && !p.shift) ph = phase_factor(k, p.n, p.shift_all);
+#pragma unroll
+  for (int bb = 0; bb < BB; ++bb) {
+    if (bb < nb) {
+      const int b = b0 + bb;
+      float2 a = acc[bb];
+      if (!p.post) {
+        a = modrelu(a, bias);
+        a = cmul(a, p.shift ? phase_factor(k, p.n, p.shift_all + p.shift[b]) : ph);
+      }
+      p.g_out[((size_t)b * p.H + h) * p.K + k] = a;
+    }
   }
-  p.g_out[(size_t)bh * p.K + k] = acc;
 }
 
 struct GatePostParams {
@@ -367,7 +449,7 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   const size_t one = gp->shared_across_heads ? 0 : 1;
   GateMlpParams mp = {};
   mp.sums = sums; mp.ncopy = ncopy; mp.copy_stride = (size_t)B * H * D; mp.inv_count = inv_count;
-  mp.H = H; mp.D = D; mp.hidden = gp->hidden; mp.n = n_fft; mp.K = K;
+  mp.B = B; mp.H = H; mp.D = D; mp.hidden = gp->hidden; mp.n = n_fft; mp.K = K;
   mp.hs_ln = one * D; mp.hs_w1 = one * (size_t)D * gp->hidden; mp.hs_b1 = one * gp->hidden;
   mp.hs_w2 = one * (size_t)gp->hidden * 2 * K; mp.hs_b2 = one * 2 * (size_t)K; mp.hs_mb = one * K;
   mp.gamma = gp->ln_gamma; mp.beta = gp->ln_beta; mp.eps = gp->ln_eps;
@@ -379,14 +461,31 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   mp.post = r > 0;
   float2* raw = r > 0 ? reinterpret_cast<float2*>(workspace) : nullptr;
   mp.g_out = r > 0 ? raw : reinterpret_cast<float2*>(g_out);
-  dim3 grid((K + 255) / 256, B * H);
-  if (grid.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H exceeds 65535");
-  size_t smem = (size_t)(D + gp->hidden + 32) * sizeof(float);
   // block sized to the bin count for short transforms (K = 99 does not need 256 threads)
   const int thr_out = K >= 256 ? 256 : ((K + 31) / 32 * 32 < 64 ? 64 : (K + 31) / 32 * 32);
-  dim3 grid_out((K + thr_out - 1) / thr_out, B * H);
-  if (gp->wdtype == SPECTRE_BF16) gate_out_kernel<bf16><<<grid_out, thr_out, smem, st>>>(mp);
-  else gate_out_kernel<float><<<grid_out, thr_out, smem, st>>>(mp);
+  // batch entries per CTA: the weights of a head are fetched once for all of them
+  const int BB = (gp->hidden > 256 || B < 2) ? 1 : (B < 4 ? 2 : (B < 8 ? 4 : 8));
+  dim3 grid_out((K + thr_out - 1) / thr_out, (unsigned)(H * ((B + BB - 1) / BB)));
+  if (grid_out.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "H * ceil(B / 8) exceeds 65535");
+  const size_t smem = (size_t)BB * (D + gp->hidden) * sizeof(float);
+  const bool wb = gp->wdtype == SPECTRE_BF16;
+  const bool pre = grid_out.x >= 32;               // many CTAs per head: compute the hidden layer once
+#define SPECTRE_GATE_LAUNCH(WT, NB)                                                              \
+  do {                                                                                           \
+    if (pre) {                                                                                   \
+      gate_hidden_kernel<WT, NB><<<grid_out.y, 256, smem, st>>>(mp);                             \
+      gate_out_kernel<WT, NB, true><<<grid_out, thr_out, smem, st>>>(mp);                        \
+    } else {                                                                                     \
+      gate_out_kernel<WT, NB, false><<<grid_out, thr_out, smem, st>>>(mp);                       \
+    }                                                                                            \
+  } while (0)
+  switch (BB) {
+    case 8: if (wb) SPECTRE_GATE_LAUNCH(bf16, 8); else SPECTRE_GATE_LAUNCH(float, 8); break;
+    case 4: if (wb) SPECTRE_GATE_LAUNCH(bf16, 4); else SPECTRE_GATE_LAUNCH(float, 4); break;
+    case 2: if (wb) SPECTRE_GATE_LAUNCH(bf16, 2); else SPECTRE_GATE_LAUNCH(float, 2); break;
+    default: if (wb) SPECTRE_GATE_LAUNCH(bf16, 1); else SPECTRE_GATE_LAUNCH(float, 1); break;
+  }
+#undef SPECTRE_GATE_LAUNCH
   SPECTRE_LAUNCH_OK("gate_out_kernel");
   if (r > 0) {
     GatePostParams pp = {};
@@ -395,6 +494,8 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
     pp.modrelu_bias = gp->modrelu_bias; pp.hs_mb = one * K;
     pp.shift = mp.shift; pp.shift_all = shift_all;
     pp.H = H; pp.K = K; pp.n = n_fft;
+    dim3 grid((K + 255) / 256, B * H);
+    if (grid.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B*H exceeds 65535");
     gate_post_kernel<<<grid, 256, 0, st>>>(pp);
     SPECTRE_LAUNCH_OK("gate_post_kernel");
   }
