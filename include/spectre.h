@@ -280,6 +280,26 @@ int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, const spect
                                      const int32_t* rows, int32_t nrows, void* y_rows, float* g_out,
                                      void* workspace, size_t workspace_bytes);
 
+/*
+ * spectre_prefix_cache_readout - step (e) of Sec. 3.3.2 for the whole window:
+ * y = R^{-1}_{N_max}( diag(g) prefix_fft ), rows 0..L-1 of it (L = y->L <= N_max;
+ * Alg. 1 returns rows N_max - L' .. N_max - 1, so pass L = N_max and slice).
+ * The inverse half of the mixer, entered with the cached half spectra instead of
+ * a forward transform; Im of the DC / Nyquist products is dropped (App. B).
+ *   g       [B, H, K, 2] float32, e.g. the g_out of spectre_prefix_cache_decode_step
+ *   y       [B, L, H, D] activation, any supported dtype; written
+ *   workspace >= spectre_readout_workspace_bytes(...) bytes, 16-byte aligned
+ *           (0 / NULL allowed when the query returns 0)
+ * N_max must be a supported transform length.  The same rows equal
+ * spectre_mixer_forward(V_buf, g) because prefix_fft = R(V_buf); this entry
+ * point does half the work and does not need the ring buffer.
+ */
+size_t spectre_readout_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
+                                       int32_t N_max);
+int spectre_prefix_cache_readout(spectre_ctx* ctx, void* stream, const spectre_cache* cache,
+                                 const float* g, const spectre_act* y,
+                                 void* workspace, size_t workspace_bytes);
+
 #ifdef __cplusplus
 }
 #endif

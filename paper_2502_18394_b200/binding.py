@@ -32,6 +32,7 @@ EXPORTS = [
     "spectre_wavelet_refine",
     "spectre_prefill_workspace_bytes", "spectre_prefix_cache_prefill", "spectre_prefix_cache_append",
     "spectre_decode_workspace_bytes", "spectre_prefix_cache_decode_step",
+    "spectre_readout_workspace_bytes", "spectre_prefix_cache_readout",
 ]
 DECODE_MAX_ROWS = 4
 
@@ -100,6 +101,10 @@ def lib():
                                                C.c_void_p, C.c_size_t]
     L.spectre_prefix_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
                                               C.c_int64]
+    L.spectre_readout_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 4
+    L.spectre_readout_workspace_bytes.restype = C.c_size_t
+    L.spectre_prefix_cache_readout.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.POINTER(Act),
+                                               C.c_void_p, C.c_size_t]
     L.spectre_decode_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 6
     L.spectre_decode_workspace_bytes.restype = C.c_size_t
     L.spectre_prefix_cache_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
@@ -350,6 +355,24 @@ def spectre_prefix_cache_decode_step(ctx: Context, cache: PrefixCache, q_t: torc
                                                   C.byref(gp), arr, len(rows), _ptr(y_rows), _ptr(g_out),
                                                   _ptr(workspace), 0 if workspace is None else workspace.numel()))
     return y_rows, g_out
+
+
+def spectre_readout_workspace_bytes(ctx: Context, B, H, D, N_max) -> int:
+    return lib().spectre_readout_workspace_bytes(ctx.handle, B, H, D, N_max)
+
+
+def spectre_prefix_cache_readout(ctx: Context, cache: PrefixCache, g: torch.Tensor, y: torch.Tensor | None = None,
+                                 workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Whole-window read-out irfft(g * prefix_fft) (Sec. 3.3.2 step e) -> [B, N_max, H, D]."""
+    if y is None:
+        y = torch.empty((cache.B, cache.N_max, cache.H, cache.D), dtype=cache.V_buf.dtype, device=g.device)
+    if workspace is None:
+        workspace = _workspace(spectre_readout_workspace_bytes(ctx, cache.B, cache.H, cache.D, cache.N_max), g.device)
+    cs = cache.struct()
+    ay = act(y)
+    _check(lib().spectre_prefix_cache_readout(ctx.handle, _stream(stream), C.byref(cs), _ptr(g), C.byref(ay),
+                                              _ptr(workspace), 0 if workspace is None else workspace.numel()))
+    return y
 
 
 # ---- pre-marshalled calls ---------------------------------------------------------------

@@ -11,6 +11,9 @@ bool transform_supported(const spectre_ctx* ctx, int n);
 size_t transform_slab_bytes(int n, int D);
 int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy);
 size_t gate_min_workspace(int B, int H, int D, int n_fft, int r);
+size_t inverse_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
+int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y,
+                          int n, void* ws, size_t ws_bytes);
 
 // ---- prefill -----------------------------------------------------------------
 // The forward pass leaves Z = fft_n(a + jb) for each column pair (a, b) in
@@ -438,4 +441,26 @@ extern "C" int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, 
   else decode_reduce_kernel<float><<<blocks_y, 256, 0, st>>>(partial, reinterpret_cast<float*>(y_rows), B, H, D, nblk, NR, nrows);
   SPECTRE_LAUNCH_OK("decode_reduce_kernel");
   return SPECTRE_OK;
+}
+
+extern "C" size_t spectre_readout_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D, int32_t N_max) {
+  if (!ctx || B < 1 || H < 1 || D < 8 || !transform_supported(ctx, N_max)) return 0;
+  return inverse_workspace_bytes(ctx, N_max, D, B * H);
+}
+
+extern "C" int spectre_prefix_cache_readout(spectre_ctx* ctx, void* stream, const spectre_cache* cache, const float* g,
+                                            const spectre_act* y, void* workspace, size_t workspace_bytes) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  int rc = check_cache(cache);
+  if (rc != SPECTRE_OK) return rc;
+  rc = check_act(y, "y");
+  if (rc != SPECTRE_OK) return rc;
+  if (!g || (reinterpret_cast<uintptr_t>(g) & 7)) return fail(SPECTRE_ERR_INVALID_ARG, "g is NULL or not 8-byte aligned");
+  const int N = cache->N_max;
+  if (y->B != cache->B || y->H != cache->H || y->D != cache->D || y->L > N || y->L < 1)
+    return fail(SPECTRE_ERR_INVALID_ARG, "y shape differs from the cache (rows 0..L-1 of the window, L <= N_max)");
+  if (!transform_supported(ctx, N)) return fail(SPECTRE_ERR_UNSUPPORTED, "N_max outside the supported transform lengths");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  return inverse_from_spectrum(ctx, reinterpret_cast<cudaStream_t>(stream), cache->prefix_fft, g, y, N, workspace,
+                               workspace_bytes);
 }

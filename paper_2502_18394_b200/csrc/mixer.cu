@@ -61,6 +61,7 @@ struct OnchipParams {
   void* dst;             // real [B,L,H,D] tensor (dst_ws = 0)
   float2* ws;            // complex workspace [slab_local][N1][M][D/2]
   const float2* g;       // gate [B*H][K]
+  const float2* spec;    // half spectra [B*H][K][D] (mode 2)
   int64_t s_sb, s_sl, s_sh;
   int64_t d_sb, d_sl, d_sh;
   int H, D, L;
@@ -73,6 +74,7 @@ struct OnchipParams {
   int radix[kMaxStages];
   int prefix[kMaxStages];   // prefix[i] = radix[0] * ... * radix[i-1]
   int mode;              // 0: forward, gate, inverse   1: forward only -> spectrum in ws
+                         // 2: inverse only, from the gated half spectra in `spec`
   int src_ws, dst_ws;
   float scale;           // 1/n, folded into the gate
 };
@@ -187,26 +189,40 @@ __device__ __forceinline__ void run_stage(int R, float4* sm, const float2* tw, i
   }
 }
 
+// Full-spectrum value of a column pair (a, b) from their half spectra and the gate (mode 2):
+// Z_k = X^a_k + j X^b_k with X = g * P completed by Hermitian symmetry; at DC and Nyquist only
+// the real parts of the two products survive the real inverse (App. B).
+__device__ __forceinline__ float2 pair_from_half(float2 gk, float4 ab, int k, int kk, int n) {
+  const float2 xa = cmul(gk, make_float2(ab.x, ab.y)), xb = cmul(gk, make_float2(ab.z, ab.w));
+  if (k == 0 || 2 * k == n) return make_float2(xa.x, xb.x);
+  if (kk == k) return make_float2(xa.x - xb.y, xa.y + xb.x);
+  return make_float2(xa.x + xb.y, xb.x - xa.y);
+}
+
 // Last forward stage (block size = radix, no twiddles) fused with the gate and,
 // in mode 0, the first inverse stage.  Local position blk*R + q' holds local
-// frequency kl = rev(blk) + (Mloc/R) q'.
+// frequency kl = rev(blk) + (Mloc/R) q'.  Mode 2 starts here: the values come from
+// the gated half spectra instead of the forward stages.
 template <typename T, int R>
 __device__ __forceinline__ void middle(const OnchipParams& p, const TileCoord& tc, float4* sm) {
   const int nwork = (p.Mloc / R) * 4;
   const int nst = p.nstage;
-  const float2* g = p.g + (size_t)(p.slab0 + tc.slab_local) * p.K;
+  const int slab = p.slab0 + tc.slab_local;
+  const float2* g = p.g + (size_t)slab * p.K;
   for (int w = threadIdx.x; w < nwork; w += blockDim.x) {
     int pg = w & 3, blk = w >> 2;
     float4* base = sm + ((size_t)blk * R * 4 + pg);
     float2 xa[R], xb[R];
+    if (p.mode != 2) {
 #pragma unroll
-    for (int q = 0; q < R; ++q) {
-      float4 v = base[q * 4];
-      xa[q] = make_float2(v.x, v.y);
-      xb[q] = make_float2(v.z, v.w);
+      for (int q = 0; q < R; ++q) {
+        float4 v = base[q * 4];
+        xa[q] = make_float2(v.x, v.y);
+        xb[q] = make_float2(v.z, v.w);
+      }
+      Dft<R, false>::run(xa);
+      Dft<R, false>::run(xb);
     }
-    Dft<R, false>::run(xa);
-    Dft<R, false>::run(xb);
     int rev = 0, tmp = blk;
     for (int i = nst - 2; i >= 0; --i) {
       int d = tmp % p.radix[i];
@@ -223,11 +239,21 @@ __device__ __forceinline__ void middle(const OnchipParams& p, const TileCoord& t
         float2 G = cscale(gate_at(g, k, p.n), p.scale);
         xa[q] = cmul(xa[q], G);
         xb[q] = cmul(xb[q], G);
-      } else {
+      } else if (p.mode == 1) {
         store_elem<T>(p, tc, kM, pg, make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y));
+      } else {
+        const int k = tc.k1 + p.N1 * kM, kk = (2 * k <= p.n) ? k : p.n - k;
+        const int col = tc.tile * 16 + pg * 4;
+        xa[q] = xb[q] = make_float2(0.f, 0.f);
+        if (col < p.D) {
+          const float2* row = p.spec + ((size_t)slab * p.K + kk) * p.D + col;
+          const float2 gk = cscale(__ldg(g + kk), p.scale);
+          xa[q] = pair_from_half(gk, *reinterpret_cast<const float4*>(row), k, kk, p.n);
+          xb[q] = pair_from_half(gk, *reinterpret_cast<const float4*>(row + 2), k, kk, p.n);
+        }
       }
     }
-    if (p.mode == 0) {
+    if (p.mode != 1) {
       Dft<R, true>::run(xa);
       Dft<R, true>::run(xb);
 #pragma unroll
@@ -305,25 +331,28 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
 
   for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = twiddle_fwd((unsigned)i, (unsigned)Mloc);
 
-  if (C == 1) {
-    for (int i = threadIdx.x; i < Mloc * 4; i += blockDim.x) sm[i] = load_elem<T>(p, tc, i >> 2, i & 3);
-    __syncthreads();
-  } else {
-    cg::cluster_group cluster = cg::this_cluster();
-    cluster.sync();                       // every CTA of the cluster is resident before remote writes
-    cross_stage<T, C, false>(p, tc, sm, cluster);
-    cluster.sync();
-  }
-
-  // forward stages (all but the last), the fused middle, inverse stages mirrored
   int S = Mloc;
-  for (int s = 0; s + 1 < p.nstage; ++s) {
-    run_stage<false>(p.radix[s], sm, tw, Mloc, S);
-    S /= p.radix[s];
-    __syncthreads();
+  if (p.mode == 2) {
+    for (int s = 0; s + 1 < p.nstage; ++s) S /= p.radix[s];     // where the forward stages would have left off
+  } else {
+    if (C == 1) {
+      for (int i = threadIdx.x; i < Mloc * 4; i += blockDim.x) sm[i] = load_elem<T>(p, tc, i >> 2, i & 3);
+      __syncthreads();
+    } else {
+      cg::cluster_group cluster = cg::this_cluster();
+      cluster.sync();                       // every CTA of the cluster is resident before remote writes
+      cross_stage<T, C, false>(p, tc, sm, cluster);
+      cluster.sync();
+    }
+    // forward stages (all but the last), the fused middle, inverse stages mirrored
+    for (int s = 0; s + 1 < p.nstage; ++s) {
+      run_stage<false>(p.radix[s], sm, tw, Mloc, S);
+      S /= p.radix[s];
+      __syncthreads();
+    }
   }
   run_middle<T>(p.nstage > 0 ? p.radix[p.nstage - 1] : 1, p, tc, sm);
-  if (p.mode != 0) return;                // forward only: spectrum already written
+  if (p.mode == 1) return;                // forward only: spectrum already written
   __syncthreads();
   for (int s = p.nstage - 2; s >= 0; --s) {
     S *= p.radix[s];
@@ -592,6 +621,63 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
   if (rc != SPECTRE_OK) return rc;
   p.src_ws = 1;
   return bf ? launch_onchip<bf16>(p, pl, cnt, st) : launch_onchip<float>(p, pl, cnt, st);
+}
+
+// Inverse transform only (read-out of the Prefix-FFT cache): y = R_n^{-1}(diag(g) spec) for all
+// slabs, spec = half spectra [B*H][K][D].  Same kernels as the mixer, entered after the gate.
+template <typename T>
+static int inverse_typed(const spectre_ctx* ctx, cudaStream_t st, const float2* spec, const float* g, const spectre_act* y,
+                         const TransformPlan& pl, void* ws, size_t ws_bytes) {
+  const int nslab = y->B * y->H;
+  OnchipParams p = {};
+  fill_common(p, pl, y->H, y->D, y->L);
+  p.dst = y->ptr;
+  p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
+  p.g = reinterpret_cast<const float2*>(g);
+  p.spec = spec;
+  p.mode = 2;
+  if (pl.N1 == 1) {
+    p.slab0 = 0; p.dst_ws = 0; p.ws = nullptr;
+    return launch_onchip<T>(p, pl, nslab, st);
+  }
+  const size_t per = slab_ws_bytes(pl.n, y->D);
+  int group = (int)(ws_bytes / per);
+  int pref = preferred_group(ctx, pl.n, y->D, nslab);
+  if (group > pref) group = pref;
+  if (group < 1) return fail(SPECTRE_ERR_WORKSPACE, "read-out workspace smaller than one (batch, head) slab");
+  StridedParams sp = {};
+  sp.dst = y->ptr; sp.ws = reinterpret_cast<float2*>(ws);
+  sp.d_sb = y->stride_b; sp.d_sl = y->stride_l; sp.d_sh = y->stride_h;
+  sp.H = y->H; sp.D = y->D; sp.L = y->L; sp.n = pl.n; sp.M = pl.M;
+  p.ws = sp.ws; p.dst_ws = 1;
+  for (int s0 = 0; s0 < nslab; s0 += group) {
+    int cnt = nslab - s0 < group ? nslab - s0 : group;
+    sp.slab0 = s0; sp.nslab = cnt;
+    p.slab0 = s0;
+    int rc = launch_onchip<T>(p, pl, cnt, st);
+    if (rc != SPECTRE_OK) return rc;
+    rc = launch_strided<T, true>(sp, pl.N1, st);
+    if (rc != SPECTRE_OK) return rc;
+  }
+  return SPECTRE_OK;
+}
+
+size_t inverse_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
+  TransformPlan pl;
+  if (!make_plan(ctx, n, &pl) || pl.N1 == 1) return 0;
+  return (size_t)preferred_group(ctx, n, D, nslab) * slab_ws_bytes(n, D);
+}
+
+int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y,
+                          int n, void* ws, size_t ws_bytes) {
+  TransformPlan pl;
+  if (!make_plan(ctx, n, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
+  if (pl.N1 > 1) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 15)) return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
+  }
+  const float2* sp = reinterpret_cast<const float2*>(spec);
+  return y->dtype == SPECTRE_BF16 ? inverse_typed<bf16>(ctx, st, sp, g, y, pl, ws, ws_bytes)
+                                  : inverse_typed<float>(ctx, st, sp, g, y, pl, ws, ws_bytes);
 }
 
 bool transform_supported(const spectre_ctx* ctx, int n) {

@@ -393,6 +393,39 @@ def test_decode_step_rows_against_oracle(ctx, dt, N, L, steps, rows):
     assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
 
 
+@pytest.mark.parametrize("dt,N", [("f32", 64), ("f32", 196), ("bf16", 1000), ("f32", 4096), ("bf16", 8192), ("f32", 32768)])
+def test_cache_readout_whole_window(ctx, dt, N):
+    # step (e) for the whole window from the cached spectrum: after a prefill and a few appends,
+    # against the oracle's inverse of its own gated spectrum; then a spectrum that is NOT that of a
+    # real window (complex DC / Nyquist bins), where the imaginary parts of those products must drop
+    L = N - 7
+    w = W.Workload("t", B=2, L=L, H=2, D=24 if N < 8192 else 16, dtype=dt, n_fft=N, seed=N + 1, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    cache = S.PrefixCache(w.B, w.H, w.D, N, dtype=W.torch_dtype(dt))
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    st = O.cache_prefill(W.to_f64(q), W.to_f64(v), N)
+    qs, vs = W.decode_tokens(w, 20)
+    for i in range(20):
+        S.spectre_prefix_cache_append(ctx, cache, qs[i].cuda(), vs[i].cuda(), L + i)
+        O.cache_append(st, L + i, W.to_f64(qs[i]), W.to_f64(vs[i]))
+    g = W.random_gate(w)
+    y = S.spectre_prefix_cache_readout(ctx, cache, g.cuda())
+    ref = O.decode_readout(st, gate_to_complex(g))
+    tol = 2e-5 if dt == "f32" else TOL["bf16"]
+    assert slab_err(W.to_f64(y), ref) < tol
+    # only the first rows, into a view of a larger buffer
+    ybig = torch.full((w.B, 40, w.H, w.D), 3.0, dtype=W.torch_dtype(dt), device="cuda")
+    S.spectre_prefix_cache_readout(ctx, cache, g.cuda(), y=ybig[:, :33])
+    assert slab_err(W.to_f64(ybig[:, :33]), ref[:, :33]) < tol and bool((ybig[:, 33:] == 3.0).all())
+    gen = torch.Generator().manual_seed(N)
+    P = torch.randn(cache.prefix_fft.shape, generator=gen)
+    cache.prefix_fft.copy_(P)
+    P64 = W.to_f64(P)
+    y = S.spectre_prefix_cache_readout(ctx, cache, g.cuda())
+    ref = O.decode_readout({"N": N, "prefix_fft": P64[..., 0] + 1j * P64[..., 1]}, gate_to_complex(g))
+    assert slab_err(W.to_f64(y), ref) < tol
+
+
 def test_decode_step_leaves_the_same_state_as_append(ctx):
     # steps (a)-(b) inside the fused step are the append's arithmetic: bit-identical state
     N, L = 512, 500
