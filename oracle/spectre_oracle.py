@@ -37,7 +37,7 @@ import numpy as np
 
 __all__ = [
     "dft_direct", "rfft_direct", "irfft_direct", "rfft", "irfft",
-    "layer_norm", "gelu_erf", "gate", "hermitian_extend", "mixer",
+    "layer_norm", "gelu_erf", "gate", "hermitian_extend", "mixer", "mixer_backward",
     "cache_prefill", "cache_append", "cache_recompute", "decode_readout",
     "decode_readout_rows", "decode_step",
     "haar_forward", "haar_inverse", "wavelet_level_gates", "wavelet_refine",
@@ -213,6 +213,36 @@ def mixer(v: np.ndarray, g: np.ndarray, n_fft: int | None = None) -> np.ndarray:
             Yhat = g[b, h].reshape(K, 1) * Vhat           # diag(g) Vhat
             y[b, :, h, :] = irfft(Yhat, n)[:L]            # step 4
     return y
+
+
+def mixer_backward(v: np.ndarray, dy: np.ndarray, g: np.ndarray, n_fft: int | None = None):
+    """Gradients of ``<dy, mixer(v, g)>`` (sum over all entries), which is what "fully
+    differentiable" (Sec. 3.7) asks of Eq. 3-4.  The mixer is real-linear in ``v`` and in
+    ``(Re g, Im g)``; with ``Vhat = R_n(pad v)``, ``Ghat = R_n(pad dy)`` and the inverse-transform
+    weights ``w_0 = w_{n/2} = 1``, ``w_k = 2`` otherwise (App. B, Corollary 1):
+
+        dv   = R_n^{-1}( conj(g) Ghat )[:L]                       (adjoint of a circular convolution)
+        dg_k = dL/dRe g_k + j dL/dIm g_k = (w_k / n) sum_c conj(Vhat_{k,c}) Ghat_{k,c}
+
+    Returns (dv [B,L,H,d], dg [B,H,K] complex).  Pinned by central differences of ``mixer`` itself."""
+    v = np.asarray(v, dtype=np.float64)
+    dy = np.asarray(dy, dtype=np.float64)
+    B, L, H, d = v.shape
+    n = L if n_fft is None else int(n_fft)
+    K = n // 2 + 1
+    w = np.full(K, 2.0)
+    w[0] = 1.0
+    if n % 2 == 0:
+        w[n // 2] = 1.0
+    dv = np.zeros_like(v)
+    dg = np.zeros((B, H, K), dtype=np.complex128)
+    for b in range(B):
+        for h in range(H):
+            Vhat = rfft(v[b, :, h, :], n)
+            Ghat = rfft(dy[b, :, h, :], n)
+            dv[b, :, h, :] = irfft(np.conj(g[b, h]).reshape(K, 1) * Ghat, n)[:L]
+            dg[b, h] = (w / n) * np.sum(np.conj(Vhat) * Ghat, axis=1)
+    return dv, dg
 
 
 # --------------------------------------------------------------------------

@@ -306,6 +306,43 @@ def test_gate_phase_rotates_output_and_commutes_with_modrelu():
     assert rel(y1[1], np.roll(y0[1], -3, axis=0)) < 1e-11          # p taken mod n
 
 
+# ---------------------------------------------------------------- backward
+@pytest.mark.parametrize("L,n", [(8, 8), (7, 7), (5, 8), (6, 9)])
+def test_mixer_backward_matches_central_differences(L, n):
+    # L(v, g) = <dy, mixer(v, g)> is linear in v and in (Re g, Im g): central differences are exact up
+    # to rounding; even and odd n, zero-padded variant; Im of the DC / Nyquist gains has zero gradient
+    B, H, d = 1, 2, 3
+    K = n // 2 + 1
+    v = RNG.standard_normal((B, L, H, d)); dy = RNG.standard_normal((B, L, H, d))
+    g = RNG.standard_normal((B, H, K)) + 1j * RNG.standard_normal((B, H, K))
+    dv, dg = O.mixer_backward(v, dy, g, n_fft=n)
+    loss = lambda vv, gg: float(np.sum(dy * O.mixer(vv, gg, n_fft=n)))
+    eps = 1e-3
+    for idx in [(0, 0, 0, 0), (0, L - 1, 1, 2), (0, L // 2, 0, 1)]:
+        e = np.zeros_like(v); e[idx] = eps
+        assert abs((loss(v + e, g) - loss(v - e, g)) / (2 * eps) - dv[idx]) < 1e-9
+    for k in range(K):
+        for part in (1.0, 1j):
+            e = np.zeros_like(g); e[0, 1, k] = eps * part
+            fd = (loss(v, g + e) - loss(v, g - e)) / (2 * eps)
+            want = dg[0, 1, k].real if part == 1.0 else dg[0, 1, k].imag
+            assert abs(fd - want) < 1e-9, (k, part)
+    assert abs(dg[0, 0, 0].imag) < 1e-12
+    if n % 2 == 0:
+        assert abs(dg[0, 0, n // 2].imag) < 1e-12
+
+
+def test_mixer_backward_is_the_adjoint():
+    # <dy, M v> = <M^T dy, v> for random pairs, and M^T is the mixer with the conjugate gate
+    B, L, H, d, n = 2, 12, 2, 4, 12
+    K = n // 2 + 1
+    v = RNG.standard_normal((B, L, H, d)); dy = RNG.standard_normal((B, L, H, d))
+    g = RNG.standard_normal((B, H, K)) + 1j * RNG.standard_normal((B, H, K))
+    dv, _ = O.mixer_backward(v, dy, g)
+    assert abs(np.sum(dy * O.mixer(v, g)) - np.sum(dv * v)) < 1e-10
+    assert rel(dv, O.mixer(dy, np.conj(g))) < 1e-13
+
+
 # ---------------------------------------------------------------- cache
 @pytest.mark.parametrize("N,L,steps", [(8, 3, 30), (8, 8, 9), (12, 1, 40)])
 def test_cache_equals_recompute_through_wraps(N, L, steps):
