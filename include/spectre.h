@@ -300,6 +300,27 @@ int spectre_prefix_cache_readout(spectre_ctx* ctx, void* stream, const spectre_c
                                  const float* g, const spectre_act* y,
                                  void* workspace, size_t workspace_bytes);
 
+/*
+ * spectre_mixer_backward - gradients of <dy, Y> for Y = spectre_mixer_forward(v, g)
+ * (Eq. 3-4 are real-linear in V and in (Re g, Im g); Sec. 3.7 "fully differentiable").
+ * With Vhat = R_n(pad v), Ghat = R_n(pad dy), w_0 = w_{n/2} = 1 and w_k = 2 otherwise:
+ *   dv   = R_n^{-1}( conj(g) Ghat ), rows 0..L-1        (the mixer on dy with the conjugate gate)
+ *   dg_k = dL/dRe g_k + j dL/dIm g_k = (w_k / n) sum_c conj(Vhat_{k,c}) Ghat_{k,c}
+ * v, dy, dv: activations of identical shape and dtype; dv may alias dy where
+ * spectre_mixer_forward allows y to alias v.  dv or dg may be NULL to skip that
+ * gradient (not both).  dg: [B, H, K, 2] float32.  dv runs on the same kernels as
+ * the forward pass; dg uses two forward-only fp32 transforms and a reduction.
+ * workspace >= spectre_mixer_backward_workspace_bytes(...), 16-byte aligned; any size
+ * down to the conjugate gate + the forward workspace + two (batch, head) slabs of
+ * spectrum (n_fft * D/2 * 8 bytes each) is accepted.
+ */
+size_t spectre_mixer_backward_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t L, int32_t H,
+                                              int32_t D, int32_t n_fft, int32_t dtype);
+int spectre_mixer_backward(spectre_ctx* ctx, void* stream,
+                           const spectre_act* v, const spectre_act* dy, const float* g,
+                           const spectre_act* dv, float* dg, int32_t n_fft,
+                           void* workspace, size_t workspace_bytes);
+
 #ifdef __cplusplus
 }
 #endif

@@ -33,6 +33,7 @@ EXPORTS = [
     "spectre_prefill_workspace_bytes", "spectre_prefix_cache_prefill", "spectre_prefix_cache_append",
     "spectre_decode_workspace_bytes", "spectre_prefix_cache_decode_step",
     "spectre_readout_workspace_bytes", "spectre_prefix_cache_readout",
+    "spectre_mixer_backward_workspace_bytes", "spectre_mixer_backward",
 ]
 DECODE_MAX_ROWS = 4
 
@@ -101,6 +102,10 @@ def lib():
                                                C.c_void_p, C.c_size_t]
     L.spectre_prefix_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
                                               C.c_int64]
+    L.spectre_mixer_backward_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 6
+    L.spectre_mixer_backward_workspace_bytes.restype = C.c_size_t
+    L.spectre_mixer_backward.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.POINTER(Act), C.c_void_p,
+                                         C.POINTER(Act), C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t]
     L.spectre_readout_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 4
     L.spectre_readout_workspace_bytes.restype = C.c_size_t
     L.spectre_prefix_cache_readout.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.POINTER(Act),
@@ -355,6 +360,28 @@ def spectre_prefix_cache_decode_step(ctx: Context, cache: PrefixCache, q_t: torc
                                                   C.byref(gp), arr, len(rows), _ptr(y_rows), _ptr(g_out),
                                                   _ptr(workspace), 0 if workspace is None else workspace.numel()))
     return y_rows, g_out
+
+
+def spectre_mixer_backward_workspace_bytes(ctx: Context, B, L, H, D, n_fft, dtype_code) -> int:
+    return lib().spectre_mixer_backward_workspace_bytes(ctx.handle, B, L, H, D, n_fft, dtype_code)
+
+
+def spectre_mixer_backward(ctx: Context, v: torch.Tensor, dy: torch.Tensor, g: torch.Tensor, n_fft: int | None = None,
+                           need_dv: bool = True, need_dg: bool = True, workspace: torch.Tensor | None = None,
+                           stream=None):
+    """Gradients of <dy, mixer(v, g)>: (dv like v or None, dg [B,H,K,2] float32 or None)."""
+    B, L, H, D = v.shape
+    n = L if n_fft is None else n_fft
+    dv = torch.empty_like(v) if need_dv else None
+    dg = torch.empty((B, H, n // 2 + 1, 2), dtype=torch.float32, device=v.device) if need_dg else None
+    if workspace is None:
+        workspace = _workspace(spectre_mixer_backward_workspace_bytes(ctx, B, L, H, D, n, _dtype_code(v)), v.device)
+    av, ady = act(v), act(dy)
+    adv = act(dv) if need_dv else None
+    _check(lib().spectre_mixer_backward(ctx.handle, _stream(stream), C.byref(av), C.byref(ady), _ptr(g),
+                                        None if adv is None else C.byref(adv), _ptr(dg), n, _ptr(workspace),
+                                        0 if workspace is None else workspace.numel()))
+    return dv, dg
 
 
 def spectre_readout_workspace_bytes(ctx: Context, B, H, D, N_max) -> int:

@@ -461,6 +461,27 @@ def test_decode_step_rejects_bad_rows(ctx):
     assert float(cache.prefix_fft.abs().max()) == 0.0               # nothing ran
 
 
+# ------------------------------------------------------------------ backward
+@pytest.mark.parametrize("dt,L,n,D", [("f32", 64, 64, 16), ("f32", 196, 196, 24), ("f32", 50, 64, 16), ("bf16", 1024, 1024, 32),
+                                      ("f32", 4096, 4096, 16), ("bf16", 8192, 8192, 64), ("f32", 16384, 16384, 16),
+                                      ("bf16", 3000, 4096, 64)])
+def test_mixer_backward(ctx, dt, L, n, D):
+    # dv = mixer(dy, conj g), dg_k = (w_k / n) sum_c conj(Vhat) Ghat against the oracle's gradients
+    w = W.Workload("t", B=2, L=L, H=2, D=D, dtype=dt, n_fft=n, seed=3 * n + L)
+    v, dy = W.activations(w, stream=0), W.activations(w, stream=5)
+    g = W.random_gate(w)
+    dv, dg = S.spectre_mixer_backward(ctx, v.cuda(), dy.cuda(), g.cuda(), n_fft=n)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    rv, rg = O.mixer_backward(W.to_f64(v), W.to_f64(dy), gate_to_complex(g), n_fft=n)
+    assert slab_err(W.to_f64(dv), rv) < TOL[dt]
+    dgc = gate_to_complex(dg)
+    err = max(rel_err(dgc[b, h], rg[b, h]) for b in range(2) for h in range(2))
+    assert err < 2e-5, err                                   # both spectra in fp32 whatever the I/O dtype
+    only_dg = S.spectre_mixer_backward(ctx, v.cuda(), dy.cuda(), g.cuda(), n_fft=n, need_dv=False)[1]
+    assert torch.equal(only_dg, dg)
+
+
 # ------------------------------------------------------------------ errors
 def test_invalid_arguments_are_rejected_before_launch(ctx):
     x = torch.zeros(1, 64, 2, 16, device="cuda")
