@@ -132,9 +132,9 @@ def append_algorithmic_bytes(w: W.Workload) -> int:
 class MixerBench:
     """gate + mixer (+ wavelet) over rotating buffer sets."""
 
-    def __init__(self, w: W.Workload, dev, nsets: int | None):
+    def __init__(self, w: W.Workload, dev, nsets: int | None, backward: bool = False):
         from paper_2502_18394_b200 import binding as S
-        self.S, self.w, self.dev = S, w, dev
+        self.S, self.w, self.dev, self.backward = S, w, dev, backward
         self.ctx = S.Context(dev.index)
         per_set = 2 * w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         if nsets is None:
@@ -160,6 +160,15 @@ class MixerBench:
                 wrm["qbar"] = d["qbar"]
             d["gate"] = S.prepare_gate(self.ctx, d["p"], w.n, d["x"], d["g"], d["wsg"], qbar_out=d["qbar"])
             d["mix"] = S.prepare_mixer_forward(self.ctx, d["x"], d["g"], d["y"], n_fft=w.n, wrm=wrm, workspace=self.ws_mix)
+            if backward:
+                # training-like step: the forward output stands in for the incoming gradient
+                if i == 0:
+                    nb = S.spectre_mixer_backward_workspace_bytes(self.ctx, w.B, w.L, w.H, w.D, w.n,
+                                                                  S.SPECTRE_BF16 if w.dtype == "bf16" else S.SPECTRE_F32)
+                    self.ws_bwd = torch.empty(max(nb, 16), dtype=torch.uint8, device=dev)
+                    self.dv = torch.empty_like(d["y"])
+                d["dg"] = torch.empty_like(d["g"])
+                d["bwd"] = S.prepare_mixer_backward(self.ctx, d["x"], d["y"], d["g"], self.dv, d["dg"], self.ws_bwd, n_fft=w.n)
             self.sets.append(d)
         self.units_per_step = w.B * w.L                                  # tokens
         self.alg_bytes = mixer_algorithmic_bytes(w)
@@ -184,13 +193,24 @@ class MixerBench:
         self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels else 0)
         self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         self.d2h = self.h2d
+        if backward:
+            # timed call = spectre_mixer_backward: dV (read dY, write dV, read g) + gate gradient (read V and dY, write dg)
+            self.kernel_name = "spectre_mixer_backward (dV through the forward kernels, dg through two fp32 transforms)"
+            self.alg_bytes = 2 * mixer_algorithmic_bytes(w)
+            per = w.n * (w.D // 2) * 8
+            gb = math.ceil(w.B * w.H / max(1, min(w.B * w.H, (128 << 20) // per)))
+            # conjugate gate + forward kernels on dY; per group of heads two forward-only transforms
+            # (one kernel each up to n = 8192, two beyond) and the reduction
+            self.launches_per_step += 1 + nk + gb * (3 if w.n <= 8192 else 5)
 
     def step(self, k: int, e0=None, e1=None):
         d = self.sets[k % self.nsets]
         d["gate"]()
+        if self.backward:
+            d["mix"]()
         if e0 is not None:
             e0.record()
-        d["mix"]()
+        (d["bwd"] if self.backward else d["mix"])()
         if e1 is not None:
             e1.record()
 
@@ -203,7 +223,9 @@ class MixerBench:
         d["x"].copy_(self.pin_x[k % len(self.pin_x)], non_blocking=True)
         d["gate"]()
         d["mix"]()
-        self.pin_y.copy_(d["y"], non_blocking=True)
+        if self.backward:
+            d["bwd"]()
+        self.pin_y.copy_(self.dv if self.backward else d["y"], non_blocking=True)
 
     def cpu_step(self):
         from oracle import spectre_oracle as O
@@ -317,8 +339,8 @@ class AppendBench:
         return time.perf_counter() - t0, 1
 
 
-def make_bench(w, dev, nsets, decode=False):
-    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets)
+def make_bench(w, dev, nsets, decode=False, backward=False):
+    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets, backward)
 
 
 # --------------------------------------------------------------------------- arms
@@ -374,6 +396,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
     ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
+    ap.add_argument("--backward", action="store_true", help="mixer workloads: step = gate + forward + backward; the timed call is the backward")
     ap.add_argument("--decode", action="store_true", help="c4: time the whole decode step (gate + fused update/read-out)")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
@@ -400,7 +423,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
-    bench = make_bench(w, dev, args.sets, args.decode)
+    bench = make_bench(w, dev, args.sets, args.decode, args.backward)
 
     for k in range(Wm):
         bench.step(k)
@@ -458,7 +481,7 @@ def main():
             "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" + backward" if args.backward else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
                        "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
                        "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
                              if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},

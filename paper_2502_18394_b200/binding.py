@@ -453,6 +453,17 @@ def prepare_decode_step(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t
     return PreparedCall(lib().spectre_prefix_cache_decode_step, args, keep)
 
 
+def prepare_mixer_backward(ctx: Context, v: torch.Tensor, dy: torch.Tensor, g: torch.Tensor, dv: torch.Tensor,
+                           dg: torch.Tensor, workspace: torch.Tensor, n_fft: int | None = None,
+                           stream=None) -> PreparedCall:
+    n = v.shape[1] if n_fft is None else n_fft
+    av, ady, adv = act(v), act(dy), act(dv)
+    keep = [v, dy, g, dv, dg, workspace, av, ady, adv]
+    args = (ctx.handle, _stream(stream), C.byref(av), C.byref(ady), _ptr(g), C.byref(adv), _ptr(dg), n,
+            _ptr(workspace), workspace.numel())
+    return PreparedCall(lib().spectre_mixer_backward, args, keep)
+
+
 def prepare_append(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t: torch.Tensor, t: int,
                    stream=None) -> PreparedCall:
     cs = cache.struct()
