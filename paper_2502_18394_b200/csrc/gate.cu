@@ -108,8 +108,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 // q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the hidden layer
-// u = GELU(q_bar W1 + b1), for nb batch entries of one head at once: a warp normalises one
-// entry (no block-wide reduction), then the nb x hidden outputs are spread over the CTA.
+// u = GELU(q_bar W1 + b1), for nb batch entries of one head at once: the means are spread over
+// the CTA, a warp normalises one entry, then the nb x hidden outputs are spread over the CTA.
 // sums points at the first entry's [D] row, bstride is the distance between batch entries;
 // u is written as [hidden][ustride] (batch entry fastest).
 template <typename WT>
@@ -119,23 +119,24 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
                                                       float eps, const WT* __restrict__ W1, const float* __restrict__ b1,
                                                       float* qbar, float* u, int ustride) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
-  for (int bb = warp; bb < nb; bb += nw) {
-    const float* sb = sums + (size_t)bb * bstride;
+  for (int e = threadIdx.x; e < nb * D; e += blockDim.x) {   // means: the whole CTA, one channel per thread
+    const int bb = e / D, c = e - bb * D;
+    const float* sb = sums + (size_t)bb * bstride + c;
+    float m = 0.f;
+    for (int k0 = 0; k0 < ncopy; k0 += 16) {                  // all copies in flight at once
+      float v[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) v[k] = (k0 + k < ncopy) ? sb[(size_t)(k0 + k) * copy_stride] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) m += v[k];
+    }
+    qbar[e] = m * inv_count;
+  }
+  __syncthreads();
+  for (int bb = warp; bb < nb; bb += nw) {                    // statistics: one warp per batch entry
     float* qb = qbar + bb * D;
     float part = 0.f;
-    for (int c = lane; c < D; c += 32) {
-      float m = 0.f;
-      for (int k0 = 0; k0 < ncopy; k0 += 16) {        // all copies in flight at once
-        float v[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) v[k] = (k0 + k < ncopy) ? sb[(size_t)(k0 + k) * copy_stride + c] : 0.f;
-#pragma unroll
-        for (int k = 0; k < 16; ++k) m += v[k];
-      }
-      m *= inv_count;
-      qb[c] = m;
-      part += m;
-    }
+    for (int c = lane; c < D; c += 32) part += qb[c];
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
     const float mean = part / (float)D;
     part = 0.f;
