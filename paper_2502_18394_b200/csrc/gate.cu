@@ -38,6 +38,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
                                                    int H, int D, int rows_per, int ncopy, size_t copy_stride,
                                                    float* __restrict__ sums) {
+  // the gate kernels behind this one may start early: they stream weights before they need the sums
+  asm volatile("griddepcontrol.launch_dependents;");
   const int b = blockIdx.y;
   const int r0 = blockIdx.x * rows_per;
   const int r1 = min(L, r0 + rows_per);
@@ -230,6 +232,8 @@ __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p)
   const int nbg = (p.B + BB - 1) / BB;
   const int h = blockIdx.x / nbg, b0 = (blockIdx.x - h * nbg) * BB;
   const int nb = min(BB, p.B - b0);
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");        // the sums come from the kernel before
   float* qbar = u + BB * p.hidden;
   const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
   descriptor_and_hidden<WT>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
@@ -266,6 +270,8 @@ __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
     for (int i = 0; i < R; ++i)
       if (i < n0) w[i] = wraw<WT>::load(col + (size_t)i * ld);
   }
+  // everything above reads only weights; the sums / hidden activations come from the kernel before
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (PRE) {
     for (int e = threadIdx.x; e < nb * p.hidden; e += blockDim.x) {
       const int bb = e / p.hidden, jj = e - bb * p.hidden;
@@ -471,13 +477,24 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   const size_t smem = (size_t)BB * (D + gp->hidden) * sizeof(float);
   const bool wb = gp->wdtype == SPECTRE_BF16;
   const bool pre = grid_out.x >= 32;               // many CTAs per head: compute the hidden layer once
+  // Programmatic dependent launch: the weight stream of the output layer may overlap the kernel
+  // before it (the pooling pass here, or whatever produced sum_q); each kernel waits for its
+  // predecessor (griddepcontrol.wait) before it touches the sums.
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg_out = {}, cfg_hid = {};
+  cfg_out.gridDim = grid_out; cfg_out.blockDim = dim3(thr_out, 1, 1); cfg_out.dynamicSmemBytes = smem; cfg_out.stream = st;
+  cfg_out.attrs = pdl; cfg_out.numAttrs = 1;
+  cfg_hid = cfg_out;
+  cfg_hid.gridDim = dim3(grid_out.y, 1, 1); cfg_hid.blockDim = dim3(256, 1, 1);
 #define SPECTRE_GATE_LAUNCH(WT, NB)                                                              \
   do {                                                                                           \
     if (pre) {                                                                                   \
-      gate_hidden_kernel<WT, NB><<<grid_out.y, 256, smem, st>>>(mp);                             \
-      gate_out_kernel<WT, NB, true><<<grid_out, thr_out, smem, st>>>(mp);                        \
+      SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg_hid, gate_hidden_kernel<WT, NB>, mp));             \
+      SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg_out, gate_out_kernel<WT, NB, true>, mp));          \
     } else {                                                                                     \
-      gate_out_kernel<WT, NB, false><<<grid_out, thr_out, smem, st>>>(mp);                       \
+      SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg_out, gate_out_kernel<WT, NB, false>, mp));         \
     }                                                                                            \
   } while (0)
   switch (BB) {
