@@ -190,7 +190,8 @@ class MixerBench:
         else:
             self.kernel_name, nk = "mixer (onchip_kernel)", 1
         # pool, gate_out (+ gate_hidden when a head's bins span >= 32 CTAs), mixer kernels, wavelet
-        self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels else 0)
+        fused_wrm = w.dtype == "bf16" and w.n == 196 and w.D == 64 and w.wavelet_levels in (1, 2) and w.wavelet_hidden <= 256
+        self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels and not fused_wrm else 0)
         self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         self.d2h = self.h2d
         if backward:

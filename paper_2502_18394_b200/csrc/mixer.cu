@@ -31,7 +31,8 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
                         const spectre_act* y);   // mixer_tc.cu
 bool tc8192_supported(const spectre_act* v, const spectre_act* y);                     // mixer_tc8k.cu
 int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
-                       const spectre_act* y);
+                       const spectre_act* y, const spectre_wavelet* wrm);
+bool tc196_fuses_wavelet(const spectre_wavelet* w);
 
 bool tc4k_supported(int n, int D);                                                     // mixer_tc4k.cu
 size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
@@ -739,11 +740,16 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (staged || fused || tc196) {
-    rc = tc196 ? launch_mixer_tc196(ctx, st, v, g, y)
+    // n = 196: the refinement rides in the kernel's store phase when it can
+    const bool fuse_wrm = tc196 && wrm && tc196_fuses_wavelet(wrm) &&
+                          (wrm->level_gates || (wrm->qbar && wrm->Ww1 && wrm->bw1 && wrm->Ww2 && wrm->bw2 &&
+                                                !((reinterpret_cast<uintptr_t>(wrm->Ww1) | reinterpret_cast<uintptr_t>(wrm->Ww2) | reinterpret_cast<uintptr_t>(wrm->bw2)) & 7) &&
+                                                (wrm->wdtype == SPECTRE_F32 || wrm->wdtype == SPECTRE_BF16)));
+    rc = tc196 ? launch_mixer_tc196(ctx, st, v, g, y, fuse_wrm ? wrm : nullptr)
                : (staged ? launch_mixer_tc4k(ctx, st, v, g, y, n_fft, workspace, workspace_bytes)
                          : launch_mixer_tc8192(ctx, st, v, g, y));
     if (rc != SPECTRE_OK) return rc;
-    if (wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
+    if (wrm && !fuse_wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
     return SPECTRE_OK;
   }
   rc = (v->dtype == SPECTRE_BF16) ? mixer_typed<bf16>(ctx, st, v, g, y, pl, workspace, workspace_bytes)

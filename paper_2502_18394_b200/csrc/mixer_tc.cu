@@ -99,7 +99,10 @@ int build_dft64(__half* F, cudaStream_t st) {
 // =====================================================================================
 constexpr int k196Heads = 4;
 constexpr int k196KSteps = 7;                 // K = 112 >= 98
-constexpr int k196Smem = kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4 + 64;
+constexpr int k196WHidden = 256;              // widest level-gate MLP the fused refinement handles
+constexpr int k196StageRow = 160;             // bytes per staged output row (128 + pad against bank conflicts)
+constexpr int k196Smem = kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4 + 64 + k196Heads * (k196WHidden + 3 * 64) * 4;
+static_assert(2 * 196 * k196StageRow <= kTcBBytes, "staged rows of two heads fit one operand buffer");
 
 struct Tc196Params {
   const bf16* src;
@@ -109,14 +112,38 @@ struct Tc196Params {
   const __half* F;        // 49-point DFT matrix (real form, padded), canonical smem layout
   int H, L, nheads;       // nheads = B * H
   int* status;
+  // wavelet refinement fused into the store (Sec. 3.5), J = 0: off
+  int J, whidden, w_bf16;
+  const float* level_gates;       // [B,H,J+1,64] or NULL
+  const float* qbar; const void* Ww1; const float* bw1; const void* Ww2; const float* bw2;
+  size_t hs_w1, hs_b1, hs_w2, hs_b2;
 };
 
+template <bool WBF> __device__ __forceinline__ float wload_rt(const void* w, size_t i) {
+  return WBF ? __bfloat162float(reinterpret_cast<const bf16*>(w)[i]) : __ldg(reinterpret_cast<const float*>(w) + i);
+}
+// two adjacent weights (i even), kept raw until used
+template <bool WBF> struct wpair;
+template <> struct wpair<true> {
+  typedef unsigned raw;
+  static __device__ __forceinline__ raw load(const void* w, size_t i) { return __ldg(reinterpret_cast<const unsigned*>(reinterpret_cast<const bf16*>(w) + i)); }
+  static __device__ __forceinline__ float2 cvt(raw r) { return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u)); }
+};
+template <> struct wpair<false> {
+  typedef float2 raw;
+  static __device__ __forceinline__ raw load(const void* w, size_t i) { return __ldg(reinterpret_cast<const float2*>(reinterpret_cast<const float*>(w) + i)); }
+  static __device__ __forceinline__ float2 cvt(raw r) { return r; }
+};
+
+template <int J, bool WBF>
 __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196Params p) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* Fsm = smem;
   unsigned char* Bsm[2] = {smem + kTcFBytes, smem + kTcFBytes + kTcBBytes};
   uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + kTcFBytes + 2 * kTcBBytes);        // [4 heads][k1 * 64 + kM]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4);
+  float* wu = reinterpret_cast<float*>(smem + kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4 + 64);   // [4][k196WHidden]
+  float* wsg = wu + k196Heads * k196WHidden;                                                         // [4][3][64] holds 1 + s
   __shared__ uint32_t tmem_slot;
   __shared__ float red[kTcEpiWarps];
   __shared__ float gmax_s[k196Heads];
@@ -263,6 +290,58 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       const float gmx = gmax_s[hl], inv = gmx > 0.f ? 1.0f / gmx : 0.f;
       Gsm[e] = pack_h2(gv[it].x * inv, gv[it].y * inv);
     }
+    if (J > 0) {
+      // level gates of the refinement: given, or s = GELU(q_bar Ww1 + bw1) Ww2 + bw2 per head (Sec. 3.5
+      // step b).  Every weight a thread needs for one output is requested before the first is used.
+      constexpr int NG = (J + 1) * 64;
+      if (!p.level_gates) {
+        for (int e = tid; e < k196Heads * p.whidden; e += kTcEpiThreads) {
+          const int hl = e / p.whidden, jj = e - hl * p.whidden, hg = head0 + hl;
+          float acc = 0.f;
+          if (hg < p.nheads) {
+            const int h = hg % p.H;
+            float wv[64];
+#pragma unroll
+            for (int c = 0; c < 64; ++c) wv[c] = wload_rt<WBF>(p.Ww1, h * p.hs_w1 + (size_t)c * p.whidden + jj);
+            acc = p.bw1[h * p.hs_b1 + jj];
+            const float* qb = p.qbar + (size_t)hg * 64;
+#pragma unroll
+            for (int c = 0; c < 64; ++c) acc = fmaf(qb[c], wv[c], acc);
+            acc = gelu_erf(acc);
+          }
+          wu[hl * k196WHidden + jj] = acc;
+        }
+        asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+      }
+      for (int e = tid; e < k196Heads * NG / 2; e += kTcEpiThreads) {       // two adjacent outputs per thread
+        const int hl = e / (NG / 2), ii = 2 * (e - hl * (NG / 2)), hg = head0 + hl;
+        float2 sv = make_float2(0.f, 0.f);
+        if (hg < p.nheads) {
+          if (p.level_gates) {
+            sv = *reinterpret_cast<const float2*>(p.level_gates + (size_t)hg * NG + ii);
+          } else {
+            const int h = hg % p.H;
+            sv = *reinterpret_cast<const float2*>(p.bw2 + h * p.hs_b2 + ii);
+            constexpr int NB = WBF ? 64 : 32;                     // rows of W2 in flight (one register each in bf16)
+            for (int j0 = 0; j0 < p.whidden; j0 += NB) {
+              typename wpair<WBF>::raw raw[NB];
+#pragma unroll
+              for (int u = 0; u < NB; ++u)
+                raw[u] = wpair<WBF>::load(p.Ww2, h * p.hs_w2 + (size_t)min(j0 + u, p.whidden - 1) * NG + ii);
+#pragma unroll
+              for (int u = 0; u < NB; ++u) {
+                const float uu = (j0 + u < p.whidden) ? wu[hl * k196WHidden + j0 + u] : 0.f;
+                const float2 wv = wpair<WBF>::cvt(raw[u]);
+                sv.x = fmaf(uu, wv.x, sv.x);
+                sv.y = fmaf(uu, wv.y, sv.y);
+              }
+            }
+          }
+        }
+        wsg[hl * 192 + ii] = 1.0f + sv.x;
+        wsg[hl * 192 + ii + 1] = 1.0f + sv.y;
+      }
+    }
     asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
 
     const int q = warp & 3, cq = warp >> 2;
@@ -349,15 +428,85 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
 #pragma unroll
             for (int n1 = 0; n1 < 4; ++n1) {
               const int row = tp + 49 * n1;
-              if (row < p.L)
-                __stcs(reinterpret_cast<uint2*>(dst + (int64_t)row * p.d_sl + col),
-                       pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y));
+              const uint2 out = pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y);
+              if (J > 0) *reinterpret_cast<uint2*>(Bsm[half] + ((hl & 1) * 196 + row) * k196StageRow + 2 * col) = out;
+              else if (row < p.L) __stcs(reinterpret_cast<uint2*>(dst + (int64_t)row * p.d_sl + col), out);
             }
           }
         }
       }
     }
     TC_STAMP(6);
+    if (J > 0) {
+      // ---- wavelet refinement on the staged bf16 rows (Sec. 3.5): Haar over aligned blocks of 2^J
+      //      tokens, bands scaled by 1 + s, synthesis; a thread takes 8 channels of one block and
+      //      writes whole 16-byte pieces, 8 lanes per 128-byte row ----
+      asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+      if (ok) {
+        constexpr int S = 1 << J;
+        const float r2 = 0.70710678118654752440f;
+        const int nblk = p.L / S;
+        for (int item = tid; item < k196Heads * nblk * 8; item += kTcEpiThreads) {
+          const int cch = item & 7, blk = (item >> 3) % nblk, hl = item / (8 * nblk), hg = head0 + hl;
+          if (hg >= p.nheads) continue;
+          const int b = hg / p.H, h = hg - b * p.H;
+          const unsigned char* st = Bsm[hl >> 1] + ((hl & 1) * 196 + blk * S) * k196StageRow + 16 * cch;
+          float x[S][8];
+#pragma unroll
+          for (int r = 0; r < S; ++r) {
+            const uint4 u4 = *reinterpret_cast<const uint4*>(st + r * k196StageRow);
+            const uint32_t w4[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              x[r][2 * e] = __uint_as_float(w4[e] << 16);
+              x[r][2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
+            }
+          }
+          // analysis in place: after level l, slot i 2^l holds a_l and slot i 2^l + 2^(l-1) holds d_l
+#pragma unroll
+          for (int l = 1; l <= J; ++l) {
+            const int span = 1 << l, hs = span >> 1;
+#pragma unroll
+            for (int i0 = 0; i0 < S; i0 += span)
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float a = x[i0][e], d = x[i0 + hs][e];
+                x[i0][e] = (a + d) * r2;
+                x[i0 + hs][e] = (a - d) * r2;
+              }
+          }
+          // slot 0 is a_J, slot r > 0 is d_l with l = ctz(r) + 1; gate order a_J, d_J, ..., d_1
+          const float* sg = wsg + hl * 192 + 8 * cch;
+#pragma unroll
+          for (int r = 0; r < S; ++r) {
+            const int lev = r == 0 ? 0 : 1 + (J - (__ffs(r)));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) x[r][e] *= sg[lev * 64 + e];
+          }
+#pragma unroll
+          for (int l = J; l >= 1; --l) {
+            const int span = 1 << l, hs = span >> 1;
+#pragma unroll
+            for (int i0 = 0; i0 < S; i0 += span)
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float a = x[i0][e], d = x[i0 + hs][e];
+                x[i0][e] = (a + d) * r2;
+                x[i0 + hs][e] = (a - d) * r2;
+              }
+          }
+          bf16* dst = p.dst + b * p.d_sb + h * p.d_sh + 8 * cch;
+#pragma unroll
+          for (int r = 0; r < S; ++r) {
+            uint4 o;
+            o.x = pack_bf2(x[r][0], x[r][1]); o.y = pack_bf2(x[r][2], x[r][3]);
+            o.z = pack_bf2(x[r][4], x[r][5]); o.w = pack_bf2(x[r][6], x[r][7]);
+            __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(blk * S + r) * p.d_sl), o);
+          }
+        }
+      }
+    }
+    TC_STAMP(7);
     if (!ok && T == 0) atomicExch(p.status, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -393,8 +542,15 @@ int build_dft49(__half* F, cudaStream_t st) {
   return SPECTRE_OK;
 }
 
+// The refinement can ride in the store phase when the block length divides 196 (J <= 2) and the
+// level-gate MLP fits the kernel's scratch.
+bool tc196_fuses_wavelet(const spectre_wavelet* w) {
+  return w && (w->levels == 1 || w->levels == 2) &&
+         (w->level_gates || (w->hidden >= 1 && w->hidden <= k196WHidden));
+}
+
 int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
-                       const spectre_act* y) {
+                       const spectre_act* y, const spectre_wavelet* wrm) {
   Tc196Params p = {};
   p.src = reinterpret_cast<const bf16*>(v->ptr);
   p.dst = reinterpret_cast<bf16*>(y->ptr);
@@ -404,9 +560,25 @@ int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_ac
   p.F = reinterpret_cast<const __half*>(ctx->dft49);
   p.H = v->H; p.L = v->L; p.nheads = v->B * v->H;
   p.status = ctx->status_dev;
-  SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k196Smem));
+  if (wrm) {
+    const int J = wrm->levels, hid = wrm->level_gates ? 0 : wrm->hidden;
+    const size_t one = wrm->shared_across_heads ? 0 : 1;
+    p.J = J; p.whidden = hid; p.w_bf16 = wrm->wdtype == SPECTRE_BF16;
+    p.level_gates = wrm->level_gates; p.qbar = wrm->qbar;
+    p.Ww1 = wrm->Ww1; p.bw1 = wrm->bw1; p.Ww2 = wrm->Ww2; p.bw2 = wrm->bw2;
+    p.hs_w1 = one * (size_t)64 * hid; p.hs_b1 = one * hid;
+    p.hs_w2 = one * (size_t)hid * (J + 1) * 64; p.hs_b2 = one * (size_t)(J + 1) * 64;
+  }
   const unsigned grid = (unsigned)((p.nheads + k196Heads - 1) / k196Heads);
-  mixer_tc196_kernel<<<grid, kTcThreads, k196Smem, st>>>(p);
+#define SPECTRE_TC196_LAUNCH(JJ, WB)                                                                              \
+  do {                                                                                                            \
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel<JJ, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, k196Smem)); \
+    mixer_tc196_kernel<JJ, WB><<<grid, kTcThreads, k196Smem, st>>>(p);                                            \
+  } while (0)
+  if (p.J == 2) { if (p.w_bf16) SPECTRE_TC196_LAUNCH(2, true); else SPECTRE_TC196_LAUNCH(2, false); }
+  else if (p.J == 1) { if (p.w_bf16) SPECTRE_TC196_LAUNCH(1, true); else SPECTRE_TC196_LAUNCH(1, false); }
+  else SPECTRE_TC196_LAUNCH(0, false);
+#undef SPECTRE_TC196_LAUNCH
   SPECTRE_LAUNCH_OK("mixer_tc196_kernel");
   return SPECTRE_OK;
 }

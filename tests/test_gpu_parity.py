@@ -268,6 +268,36 @@ def test_c5_reduced_batch_with_wavelet(ctx):
     assert slab_err(W.to_f64(y), ref) < TOL["bf16"]
 
 
+@pytest.mark.parametrize("J,L,B,H,wdt,hid,given", [(2, 196, 2, 3, "bf16", 64, False), (1, 196, 1, 5, "f32", 48, False),
+                                                 (2, 148, 3, 2, "bf16", 64, True), (1, 150, 2, 2, "f32", 64, True),
+                                                 (2, 196, 1, 2, "f32", 320, False)])
+def test_mixer_196_with_refinement_in_the_store_phase(ctx, J, L, B, H, wdt, hid, given):
+    # n = 196 on the tensor cores with the Haar refinement chained: level gates from the MLP (bf16 and
+    # fp32 weights, widths other than 64) or given; zero-padded rows; partial head groups; a hidden
+    # width the fused kernel does not take (320) must fall back to the separate refinement kernel.
+    w = W.Workload("t", B=B, L=L, H=H, D=64, dtype="bf16", wdtype=wdt, n_fft=196, seed=11 * J + L + H,
+                   wavelet_levels=J, wavelet_hidden=hid)
+    x = W.activations(w, structured=True)
+    g = W.random_gate(w)
+    wp = W.wavelet_params(w)
+    gen = torch.Generator().manual_seed(5)
+    wp["bw2"] = 0.3 * torch.randn(wp["bw2"].shape, generator=gen)
+    qbar = torch.randn(B, H, 64, generator=gen)
+    s_ref = O.wavelet_level_gates(W.to_f64(qbar), W.to_f64(wp["Ww1"]), W.to_f64(wp["bw1"]), W.to_f64(wp["Ww2"]),
+                                  W.to_f64(wp["bw2"]), J)                   # [B,H,J+1,D]
+    if given:
+        lg = torch.tensor(s_ref, dtype=torch.float32)
+        wrm = {"levels": J, "level_gates": lg.cuda()}
+        s_ref = W.to_f64(lg)
+    else:
+        wrm = dict(to_dev(wp), qbar=qbar.cuda())
+    y = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=196, wrm=wrm)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ref = O.wavelet_refine(O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=196), s_ref, J)
+    assert slab_err(W.to_f64(y), ref) < TOL["bf16"]
+
+
 # ------------------------------------------------------------------ cache
 def cache_err(cache, st):
     P = W.to_f64(cache.prefix_fft)
