@@ -98,17 +98,6 @@ template <> __device__ __forceinline__ float2 wload2<bf16>(const bf16* p) {
   return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u));
 }
 
-__device__ __forceinline__ float block_sum(float v, float* red) {
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
-  __syncthreads();
-  if (lane == 0) red[warp] = v;
-  __syncthreads();
-  float t = 0.f;
-  for (int i = 0; i < nw; ++i) t += red[i];
-  return t;
-}
-
 // q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the hidden layer
 // u = GELU(q_bar W1 + b1), for nb batch entries of one head at once: the means are spread over
 // the CTA, a warp normalises one entry, then the nb x hidden outputs are spread over the CTA.

@@ -9,9 +9,6 @@ constexpr int kTcLbo = 144;                    // bytes between core matrices al
 constexpr int kTcSbo = 2320;                   // bytes between 8-column groups (16 * 144 + 16 pad)
 constexpr int kTcBBytes = 32 * kTcSbo;         // one 256-column B operand
 constexpr int kTcFBytes = 128 * 128 * 2;
-constexpr int kTcGStride = 72;                 // gate table: entry (row, col) at row + 72 col (conflict-free reads)
-constexpr int kTcGBytes = 64 * kTcGStride * 4; // per half, fp16 (re, im)
-constexpr int kTcSmem = kTcFBytes + 2 * kTcBBytes + 2 * kTcGBytes + 64;
 constexpr int kTcEpiWarps = 16;                // 4 per TMEM lane quadrant, one column quarter each
 constexpr int kTcEpiThreads = 32 * kTcEpiWarps;
 constexpr int kTcThreads = kTcEpiThreads + 32; // + 1 MMA-issuing warp
