@@ -36,7 +36,7 @@ import math
 import numpy as np
 
 __all__ = [
-    "dft_direct", "rfft_direct", "irfft_direct", "rfft", "irfft",
+    "dft_direct", "rfft_direct", "irfft_direct", "rfft", "irfft", "project_qv",
     "layer_norm", "gelu_erf", "gate", "hermitian_extend", "mixer", "mixer_backward",
     "cache_prefill", "cache_append", "cache_recompute", "decode_readout",
     "decode_readout_rows", "decode_step",
@@ -99,6 +99,25 @@ def rfft(x: np.ndarray, n: int | None = None) -> np.ndarray:
 def irfft(Y: np.ndarray, n: int) -> np.ndarray:
     """Inverse real transform along axis 0 (Eq. 4's ``R_n^{-1}``), 1/n inside."""
     return np.fft.irfft(np.asarray(Y, dtype=np.complex128), n=n, axis=0)
+
+
+# --------------------------------------------------------------------------
+# Token projection (Sec. 3.2 step 1, Eq. 2)
+# --------------------------------------------------------------------------
+def project_qv(x: np.ndarray, Wq: np.ndarray, Wv: np.ndarray):
+    """Eq. 2 per head: ``Q = X W^(q)``, ``V = X W^(v)`` with ``X`` the head's
+    ``[n, d]`` slice and ``W`` of shape ``[d, d]`` (input channel first).
+    x [B,L,H,d]; Wq, Wv [H,d,d].  Returns (Q, V [B,L,H,d], sum_q [B,H,d] = sum of
+    Q over the sequence, the quantity the gate pools in step 3a)."""
+    x = np.asarray(x, dtype=np.float64)
+    B, L, H, d = x.shape
+    Q = np.zeros_like(x)
+    V = np.zeros_like(x)
+    for b in range(B):
+        for h in range(H):
+            Q[b, :, h, :] = x[b, :, h, :] @ np.asarray(Wq[h], dtype=np.float64)
+            V[b, :, h, :] = x[b, :, h, :] @ np.asarray(Wv[h], dtype=np.float64)
+    return Q, V, Q.sum(axis=1)
 
 
 # --------------------------------------------------------------------------

@@ -194,6 +194,23 @@ def test_hermitian_extension_equals_half_spectrum_gate():
     assert rel(z.real, y[0, :, 0, 0]) < 1e-12 and rel(z.imag, y[0, :, 0, 1]) < 1e-12
 
 
+# ---------------------------------------------------------------- projection
+def test_projection_written_out_and_special_cases():
+    B, L, H, d = 2, 5, 3, 4
+    x = RNG.standard_normal((B, L, H, d))
+    Wq = RNG.standard_normal((H, d, d)); Wv = RNG.standard_normal((H, d, d))
+    Q, V, sq = O.project_qv(x, Wq, Wv)
+    for (b, t, h, o) in [(0, 0, 0, 0), (1, 4, 2, 3), (0, 2, 1, 1)]:
+        assert abs(Q[b, t, h, o] - sum(x[b, t, h, i] * Wq[h, i, o] for i in range(d))) < 1e-12   # input channel first
+        assert abs(V[b, t, h, o] - sum(x[b, t, h, i] * Wv[h, i, o] for i in range(d))) < 1e-12
+    assert np.allclose(sq, Q.sum(axis=1))
+    eye = np.tile(np.eye(d), (H, 1, 1))
+    Qi, Vi, _ = O.project_qv(x, eye, 2 * eye)
+    assert np.array_equal(Qi, x) and np.array_equal(Vi, 2 * x)                                   # identity weights
+    Wz = Wq.copy(); Wz[1] = 0
+    assert np.all(O.project_qv(x, Wz, Wv)[0][:, :, 1] == 0) and np.allclose(O.project_qv(x, Wz, Wv)[0][:, :, 0], Q[:, :, 0])   # heads do not mix
+
+
 # ---------------------------------------------------------------- gate
 def _gate_params(H, d, hid, K, std=0.5):
     return dict(ln_gamma=1 + 0.1 * RNG.standard_normal((H, d)), ln_beta=0.1 * RNG.standard_normal((H, d)),
