@@ -321,6 +321,25 @@ int spectre_mixer_backward(spectre_ctx* ctx, void* stream,
                            const spectre_act* dv, float* dg, int32_t n_fft,
                            void* workspace, size_t workspace_bytes);
 
+/*
+ * spectre_project_qv - token projections of Sec. 3.2 step 1 (Eq. 2), per head:
+ *   Q = X W^(q),  V = X W^(v),  X the head's [L, D] slice, W [D, D] (input channel first),
+ * on the tensor cores (bf16 operands, fp32 accumulation), with the pooled query sum
+ *   sum_q[b, h, :] = sum_t Q[b, t, h, :]   (fp32, taken from the accumulators)
+ * of step 3a as a by-product, so that spectre_gate can be called with sum_q
+ * (inv_count = 1/L) instead of reading Q again.
+ *   x, q, v   [B, L, H, D] bf16 activations, D = 64, three distinct buffers
+ *   Wq, Wv    [H, D, D] of dtype wdtype (SPECTRE_F32 or SPECTRE_BF16; rounded to bf16)
+ *   sum_q     [B, H, D] float32, overwritten; or NULL
+ *   workspace >= spectre_project_workspace_bytes(ctx, H, D) bytes, 16-byte aligned
+ * Other dtypes or head widths: SPECTRE_ERR_UNSUPPORTED.
+ */
+size_t spectre_project_workspace_bytes(const spectre_ctx* ctx, int32_t H, int32_t D);
+int spectre_project_qv(spectre_ctx* ctx, void* stream, const spectre_act* x,
+                       const void* Wq, const void* Wv, int32_t wdtype,
+                       const spectre_act* q, const spectre_act* v, float* sum_q,
+                       void* workspace, size_t workspace_bytes);
+
 #ifdef __cplusplus
 }
 #endif

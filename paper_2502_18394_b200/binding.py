@@ -34,6 +34,7 @@ EXPORTS = [
     "spectre_decode_workspace_bytes", "spectre_prefix_cache_decode_step",
     "spectre_readout_workspace_bytes", "spectre_prefix_cache_readout",
     "spectre_mixer_backward_workspace_bytes", "spectre_mixer_backward",
+    "spectre_project_workspace_bytes", "spectre_project_qv",
 ]
 DECODE_MAX_ROWS = 4
 
@@ -102,6 +103,10 @@ def lib():
                                                C.c_void_p, C.c_size_t]
     L.spectre_prefix_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Cache), C.c_void_p, C.c_void_p,
                                               C.c_int64]
+    L.spectre_project_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    L.spectre_project_workspace_bytes.restype = C.c_size_t
+    L.spectre_project_qv.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.c_void_p, C.c_void_p, C.c_int32,
+                                     C.POINTER(Act), C.POINTER(Act), C.c_void_p, C.c_void_p, C.c_size_t]
     L.spectre_mixer_backward_workspace_bytes.argtypes = [C.c_void_p] + [C.c_int32] * 6
     L.spectre_mixer_backward_workspace_bytes.restype = C.c_size_t
     L.spectre_mixer_backward.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Act), C.POINTER(Act), C.c_void_p,
@@ -360,6 +365,30 @@ def spectre_prefix_cache_decode_step(ctx: Context, cache: PrefixCache, q_t: torc
                                                   C.byref(gp), arr, len(rows), _ptr(y_rows), _ptr(g_out),
                                                   _ptr(workspace), 0 if workspace is None else workspace.numel()))
     return y_rows, g_out
+
+
+def spectre_project_workspace_bytes(ctx: Context, H, D) -> int:
+    return lib().spectre_project_workspace_bytes(ctx.handle, H, D)
+
+
+def spectre_project_qv(ctx: Context, x: torch.Tensor, Wq: torch.Tensor, Wv: torch.Tensor, q: torch.Tensor | None = None,
+                       v: torch.Tensor | None = None, sum_q: torch.Tensor | None = None, need_sum: bool = True,
+                       workspace: torch.Tensor | None = None, stream=None):
+    """Q = X Wq, V = X Wv per head (Eq. 2) and sum_q = sum over the sequence of Q.  Returns (q, v, sum_q)."""
+    B, L, H, D = x.shape
+    if Wq.dtype != Wv.dtype or not (Wq.is_contiguous() and Wv.is_contiguous()):
+        raise ValueError("Wq and Wv must be contiguous and of one dtype")
+    q = torch.empty_like(x) if q is None else q
+    v = torch.empty_like(x) if v is None else v
+    if sum_q is None and need_sum:
+        sum_q = torch.empty((B, H, D), dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = _workspace(spectre_project_workspace_bytes(ctx, H, D), x.device)
+    ax, aq, av = act(x), act(q), act(v)
+    _check(lib().spectre_project_qv(ctx.handle, _stream(stream), C.byref(ax), _ptr(Wq), _ptr(Wv), _dtype_code(Wq),
+                                    C.byref(aq), C.byref(av), _ptr(sum_q), _ptr(workspace),
+                                    0 if workspace is None else workspace.numel()))
+    return q, v, sum_q
 
 
 def spectre_mixer_backward_workspace_bytes(ctx: Context, B, L, H, D, n_fft, dtype_code) -> int:

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libspectre.so")
 SOURCES = ["api.cu", "mixer.cu", "mixer_tc.cu", "mixer_tc8k.cu", "mixer_tc4k.cu", "gate.cu", "cache.cu", "wavelet.cu",
-           "backward.cu"]
+           "backward.cu", "project.cu"]
 FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "-shared"]
 

@@ -491,6 +491,33 @@ def test_decode_step_rejects_bad_rows(ctx):
     assert float(cache.prefix_fft.abs().max()) == 0.0               # nothing ran
 
 
+# ------------------------------------------------------------------ projections
+@pytest.mark.parametrize("B,L,H,wdt", [(1, 128, 1, "bf16"), (2, 1000, 3, "f32"), (1, 8192, 4, "bf16"), (3, 196, 2, "bf16"), (1, 50, 2, "f32")])
+def test_project_qv(ctx, B, L, H, wdt):
+    # Eq. 2 on the tensor cores against the oracle: bf16 operands, fp32 accumulation, bf16 outputs;
+    # ragged last tile; sum_q from the accumulators; strided output views
+    w = W.Workload("t", B=B, L=L, H=H, D=64, dtype="bf16", seed=L + H)
+    x = W.activations(w, structured=True)
+    gen = torch.Generator().manual_seed(L)
+    wd = W.torch_dtype(wdt)
+    Wq = (torch.randn(H, 64, 64, generator=gen) / 8).to(wd)
+    Wv = (torch.randn(H, 64, 64, generator=gen) / 8).to(wd)
+    big = torch.full((2, B, L, H + 1, 64), 5.0, dtype=torch.bfloat16, device="cuda")
+    q, v, sq = S.spectre_project_qv(ctx, x.cuda(), Wq.cuda(), Wv.cuda(), q=big[0, :, :, :H], v=big[1, :, :, 1:])
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    Wq64 = W.to_f64(Wq.to(torch.bfloat16)); Wv64 = W.to_f64(Wv.to(torch.bfloat16))      # the kernel's operands are bf16
+    rq, rv, rs = O.project_qv(W.to_f64(x), Wq64, Wv64)
+    assert slab_err(W.to_f64(q), rq) < TOL["bf16"] and slab_err(W.to_f64(v), rv) < TOL["bf16"]
+    assert rel_err(W.to_f64(sq), rs) < 1e-4
+    assert bool((big[0, :, :, H] == 5.0).all()) and bool((big[1, :, :, 0] == 5.0).all())
+    # the pooled sum feeds the gate without a second pass over Q
+    p = W.gate_params(w)
+    g1 = S.spectre_gate(ctx, to_dev(p), L, sum_q=sq, inv_count=1.0 / L)
+    g2 = S.spectre_gate(ctx, to_dev(p), L, q=q)
+    assert rel_err(gate_to_complex(g1), gate_to_complex(g2)) < 2e-2
+
+
 # ------------------------------------------------------------------ backward
 @pytest.mark.parametrize("dt,L,n,D", [("f32", 64, 64, 16), ("f32", 196, 196, 24), ("f32", 50, 64, 16), ("bf16", 1024, 1024, 32),
                                       ("f32", 4096, 4096, 16), ("bf16", 8192, 8192, 64), ("f32", 16384, 16384, 16),
