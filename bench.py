@@ -132,9 +132,9 @@ def append_algorithmic_bytes(w: W.Workload) -> int:
 class MixerBench:
     """gate + mixer (+ wavelet) over rotating buffer sets."""
 
-    def __init__(self, w: W.Workload, dev, nsets: int | None, backward: bool = False):
+    def __init__(self, w: W.Workload, dev, nsets: int | None, backward: bool = False, project: bool = False):
         from paper_2502_18394_b200 import binding as S
-        self.S, self.w, self.dev, self.backward = S, w, dev, backward
+        self.S, self.w, self.dev, self.backward, self.project = S, w, dev, backward, project
         self.ctx = S.Context(dev.index)
         per_set = 2 * w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         if nsets is None:
@@ -160,6 +160,17 @@ class MixerBench:
                 wrm["qbar"] = d["qbar"]
             d["gate"] = S.prepare_gate(self.ctx, d["p"], w.n, d["x"], d["g"], d["wsg"], qbar_out=d["qbar"])
             d["mix"] = S.prepare_mixer_forward(self.ctx, d["x"], d["g"], d["y"], n_fft=w.n, wrm=wrm, workspace=self.ws_mix)
+            if project:
+                # whole layer front: Q = X Wq, V = X Wv with sum_q as a by-product, gate from sum_q, mixer on V
+                gen = torch.Generator().manual_seed(100 + i)
+                d["Wq"] = (torch.randn(w.H, w.D, w.D, generator=gen) / 8).to(torch.bfloat16).to(dev)
+                d["Wv"] = (torch.randn(w.H, w.D, w.D, generator=gen) / 8).to(torch.bfloat16).to(dev)
+                d["q"], d["v"] = torch.empty_like(d["x"]), torch.empty_like(d["x"])
+                d["sq"] = torch.empty((w.B, w.H, w.D), dtype=torch.float32, device=dev)
+                d["wsp"] = torch.empty(S.spectre_project_workspace_bytes(self.ctx, w.H, w.D), dtype=torch.uint8, device=dev)
+                d["proj"] = S.prepare_project_qv(self.ctx, d["x"], d["Wq"], d["Wv"], d["q"], d["v"], d["sq"], d["wsp"])
+                d["gate"] = S.prepare_gate_from_sum(self.ctx, d["p"], w.n, d["sq"], 1.0 / w.L, d["g"], d["wsg"], qbar_out=d["qbar"])
+                d["mix"] = S.prepare_mixer_forward(self.ctx, d["v"], d["g"], d["y"], n_fft=w.n, wrm=wrm, workspace=self.ws_mix)
             if backward:
                 # training-like step: the forward output stands in for the incoming gradient
                 if i == 0:
@@ -194,6 +205,11 @@ class MixerBench:
         self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels and not fused_wrm else 0)
         self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
         self.d2h = self.h2d
+        if project:
+            es = 2
+            self.kernel_name = "spectre_project_qv (proj_weights_kernel + project_qv_kernel, tcgen05)"
+            self.alg_bytes = 3 * w.B * w.L * w.H * w.D * es + 2 * w.H * w.D * w.D * es     # read X, write Q and V, read weights
+            self.launches_per_step += 1          # weights transpose + projection replace the pooling pass
         if backward:
             # timed call = spectre_mixer_backward: dV (read dY, write dV, read g) + gate gradient (read V and dY, write dg)
             self.kernel_name = "spectre_mixer_backward (dV through the forward kernels, dg through two fp32 transforms)"
@@ -206,6 +222,15 @@ class MixerBench:
 
     def step(self, k: int, e0=None, e1=None):
         d = self.sets[k % self.nsets]
+        if self.project:                     # timed call = the projection
+            if e0 is not None:
+                e0.record()
+            d["proj"]()
+            if e1 is not None:
+                e1.record()
+            d["gate"]()
+            d["mix"]()
+            return
         d["gate"]()
         if self.backward:
             d["mix"]()
@@ -222,6 +247,8 @@ class MixerBench:
     def e2e_step(self, k: int):
         d = self.sets[k % self.nsets]
         d["x"].copy_(self.pin_x[k % len(self.pin_x)], non_blocking=True)
+        if self.project:
+            d["proj"]()
         d["gate"]()
         d["mix"]()
         if self.backward:
@@ -340,8 +367,8 @@ class AppendBench:
         return time.perf_counter() - t0, 1
 
 
-def make_bench(w, dev, nsets, decode=False, backward=False):
-    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets, backward)
+def make_bench(w, dev, nsets, decode=False, backward=False, project=False):
+    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets, backward, project)
 
 
 # --------------------------------------------------------------------------- arms
@@ -397,6 +424,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
     ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
+    ap.add_argument("--project", action="store_true", help="mixer workloads (bf16, d = 64): step = projections + gate from sum_q + mixer; the timed call is the projection")
     ap.add_argument("--backward", action="store_true", help="mixer workloads: step = gate + forward + backward; the timed call is the backward")
     ap.add_argument("--decode", action="store_true", help="c4: time the whole decode step (gate + fused update/read-out)")
     args = ap.parse_args()
@@ -424,7 +452,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
-    bench = make_bench(w, dev, args.sets, args.decode, args.backward)
+    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project)
 
     for k in range(Wm):
         bench.step(k)
@@ -482,7 +510,7 @@ def main():
             "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" + backward" if args.backward else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" + backward" if args.backward else "") + (" with token projections in front (gate from their sum_q)" if args.project else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
                        "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
                        "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
                              if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},
@@ -494,7 +522,7 @@ def main():
                          "frac": achieved / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": bench.alg_bytes,
                          "kernel_ms": kern_ms, "frac_of_8000": achieved / 8000.0,
                          "kernel_tokens_per_s": bench.units_per_step / (kern_ms * 1e-3),
-                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},   # None for reduced cases
+                         "traffic": None if (args.project or args.backward or args.decode) else NCU_TRAFFIC_BYTES.get(w.name)},   # None for reduced cases and variant legs
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))

@@ -482,6 +482,27 @@ def prepare_decode_step(ctx: Context, cache: PrefixCache, q_t: torch.Tensor, v_t
     return PreparedCall(lib().spectre_prefix_cache_decode_step, args, keep)
 
 
+def prepare_project_qv(ctx: Context, x: torch.Tensor, Wq: torch.Tensor, Wv: torch.Tensor, q: torch.Tensor,
+                       v: torch.Tensor, sum_q: torch.Tensor, workspace: torch.Tensor, stream=None) -> PreparedCall:
+    ax, aq, av = act(x), act(q), act(v)
+    keep = [x, Wq, Wv, q, v, sum_q, workspace, ax, aq, av]
+    args = (ctx.handle, _stream(stream), C.byref(ax), _ptr(Wq), _ptr(Wv), _dtype_code(Wq), C.byref(aq), C.byref(av),
+            _ptr(sum_q), _ptr(workspace), workspace.numel())
+    return PreparedCall(lib().spectre_project_qv, args, keep)
+
+
+def prepare_gate_from_sum(ctx: Context, params: dict, n_fft: int, sum_q: torch.Tensor, inv_count: float,
+                          g_out: torch.Tensor, workspace: torch.Tensor, qbar_out: torch.Tensor | None = None,
+                          shift_all: int = 0, stream=None) -> PreparedCall:
+    B, H, D = sum_q.shape
+    keep: list = [sum_q, g_out, workspace, qbar_out]
+    gp = _gate_struct(params, keep)
+    keep += [gp]
+    args = (ctx.handle, _stream(stream), None, _ptr(sum_q), B, H, D, C.c_float(inv_count), C.byref(gp), n_fft, None,
+            int(shift_all), _ptr(g_out), _ptr(qbar_out), _ptr(workspace), workspace.numel())
+    return PreparedCall(lib().spectre_gate, args, keep)
+
+
 def prepare_mixer_backward(ctx: Context, v: torch.Tensor, dy: torch.Tensor, g: torch.Tensor, dv: torch.Tensor,
                            dg: torch.Tensor, workspace: torch.Tensor, n_fft: int | None = None,
                            stream=None) -> PreparedCall:

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(256) proj_weights_kernel(const WT* __restrict_
   wt[idx] = __float2bfloat16_rn(w);
 }
 
-__global__ void __launch_bounds__(kPjThreads) project_qv_kernel(const ProjParams p) {
+__global__ void __launch_bounds__(kPjThreads, 3) project_qv_kernel(const ProjParams p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   unsigned char* Asm = smem;                         // X tile
