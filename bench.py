@@ -494,12 +494,13 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         torch.set_num_threads(1)
-        reps = 1 if base in ("c3",) else 3
-        tot, units = 0.0, 0
-        for _ in range(reps):
+        # bounded sample: repeat the oracle's step until about 10 s of CPU work have been timed
+        reps, tot, units = 0, 0.0, 0
+        while reps < 1 or (tot < 10.0 and reps < 200):
             dt, u = bench.cpu_step()
             tot += dt
             units += u
+            reps += 1
         note = _cpu_only_bench(w).sample_note + f", {reps} repetition(s)"
         cpu = {"value": units / tot, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": note}
 
