@@ -132,7 +132,8 @@ def append_algorithmic_bytes(w: W.Workload) -> int:
 class MixerBench:
     """gate + mixer (+ wavelet) over rotating buffer sets."""
 
-    def __init__(self, w: W.Workload, dev, nsets: int | None, backward: bool = False, project: bool = False):
+    def __init__(self, w: W.Workload, dev, nsets: int | None, backward: bool = False, project: bool = False,
+                 shared_gates: bool = False):
         from paper_2502_18394_b200 import binding as S
         self.S, self.w, self.dev, self.backward, self.project = S, w, dev, backward, project
         self.ctx = S.Context(dev.index)
@@ -142,6 +143,10 @@ class MixerBench:
         self.nsets = nsets
         self.x_host = [W.activations(w, stream=i) for i in range(nsets)]
         params = W.gate_params(w)
+        if shared_gates:
+            # one gate network for all heads (Sec. 3.6): head 0's parameters, shape [1, ...]
+            params = {k: (v[:1].contiguous() if isinstance(v, torch.Tensor) else v) for k, v in params.items()}
+            params["shared_across_heads"] = 1
         self.sets = []
         ws_gate = S.spectre_gate_workspace_bytes(self.ctx, w.B, w.H, w.D, w.n, 0)
         ws_mix = S.spectre_mixer_workspace_bytes(self.ctx, w.B, w.L, w.H, w.D, w.n, S.SPECTRE_BF16 if w.dtype == "bf16" else S.SPECTRE_F32)
@@ -367,8 +372,8 @@ class AppendBench:
         return time.perf_counter() - t0, 1
 
 
-def make_bench(w, dev, nsets, decode=False, backward=False, project=False):
-    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets, backward, project)
+def make_bench(w, dev, nsets, decode=False, backward=False, project=False, shared_gates=False):
+    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets, backward, project, shared_gates)
 
 
 # --------------------------------------------------------------------------- arms
@@ -424,6 +429,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
     ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
+    ap.add_argument("--shared-gates", action="store_true", help="mixer workloads: one gate network shared by all heads (Sec. 3.6)")
     ap.add_argument("--project", action="store_true", help="mixer workloads (bf16, d = 64): step = projections + gate from sum_q + mixer; the timed call is the projection")
     ap.add_argument("--backward", action="store_true", help="mixer workloads: step = gate + forward + backward; the timed call is the backward")
     ap.add_argument("--decode", action="store_true", help="c4: time the whole decode step (gate + fused update/read-out)")
@@ -452,7 +458,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
-    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project)
+    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project, args.shared_gates)
 
     for k in range(Wm):
         bench.step(k)
@@ -511,7 +517,7 @@ def main():
             "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" + backward" if args.backward else "") + (" with token projections in front (gate from their sum_q)" if args.project else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" + backward" if args.backward else "") + (" with token projections in front (gate from their sum_q)" if args.project else "") + (", gate shared across heads" if args.shared_gates else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
                        "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
                        "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
                              if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},

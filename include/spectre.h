@@ -175,6 +175,10 @@ typedef struct {
   const float* bw1;              /* [H, hidden]                                      */
   const void* Ww2;               /* [H, hidden, (J+1) D]                             */
   const float* bw2;              /* [H, (J+1) D]                                     */
+  const int32_t* skip;           /* [B] on the device, or NULL: batch entries with a
+                                    non-zero flag are passed through unrefined (the
+                                    module is "applied conditionally", Sec. 3.5; the
+                                    controller that sets the flags is the caller's)   */
 } spectre_wavelet;
 
 /*

@@ -448,13 +448,18 @@ def wavelet_level_gates(qbar, Ww1, bw1, Ww2, bw2, J):
     return out
 
 
-def wavelet_refine(y: np.ndarray, level_gates: np.ndarray, J: int) -> np.ndarray:
+def wavelet_refine(y: np.ndarray, level_gates: np.ndarray, J: int, skip=None) -> np.ndarray:
     """Sec. 3.5 steps (a),(c),(d): ``V_out = Y + W^{-1}( s * W Y )``.
-    y [B,n,H,d]; level_gates [B,H,J+1,d]."""
+    y [B,n,H,d]; level_gates [B,H,J+1,d].  ``skip`` [B] (optional): batch entries
+    with a true flag are returned unrefined (the module is applied conditionally;
+    the controller that decides is outside this function)."""
     y = np.asarray(y, dtype=np.float64)
     B, n, H, d = y.shape
     out = np.zeros_like(y)
     for b in range(B):
+        if skip is not None and skip[b]:
+            out[b] = y[b]
+            continue
         for h in range(H):
             col = y[b, :, h, :]
             w = haar_forward(col, J)

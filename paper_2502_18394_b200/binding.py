@@ -61,7 +61,8 @@ class GateParams(C.Structure):
 class Wavelet(C.Structure):
     _fields_ = [("levels", C.c_int32), ("hidden", C.c_int32), ("wdtype", C.c_int32),
                 ("shared_across_heads", C.c_int32), ("level_gates", C.c_void_p), ("qbar", C.c_void_p),
-                ("Ww1", C.c_void_p), ("bw1", C.c_void_p), ("Ww2", C.c_void_p), ("bw2", C.c_void_p)]
+                ("Ww1", C.c_void_p), ("bw1", C.c_void_p), ("Ww2", C.c_void_p), ("bw2", C.c_void_p),
+                ("skip", C.c_void_p)]
 
 
 class Cache(C.Structure):
@@ -202,7 +203,8 @@ def _wavelet_struct(w: dict | None, keep: list):
                    None if w.get("Ww1") is None else w["Ww1"].data_ptr(),
                    None if w.get("bw1") is None else w["bw1"].data_ptr(),
                    None if w.get("Ww2") is None else w["Ww2"].data_ptr(),
-                   None if w.get("bw2") is None else w["bw2"].data_ptr())
+                   None if w.get("bw2") is None else w["bw2"].data_ptr(),
+                   None if w.get("skip") is None else w["skip"].data_ptr())
 
 
 def _workspace(nbytes: int, device) -> torch.Tensor | None:

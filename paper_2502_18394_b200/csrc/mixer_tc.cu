@@ -114,6 +114,7 @@ struct Tc196Params {
   const float* level_gates;       // [B,H,J+1,64] or NULL
   const float* qbar; const void* Ww1; const float* bw1; const void* Ww2; const float* bw2;
   size_t hs_w1, hs_b1, hs_w2, hs_b2;
+  const int* skip;                // [B] or NULL: non-zero = no refinement for this batch entry
 };
 
 template <bool WBF> __device__ __forceinline__ float wload_rt(const void* w, size_t i) {
@@ -448,6 +449,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
           if (hg >= p.nheads) continue;
           const int b = hg / p.H, h = hg - b * p.H;
           const unsigned char* st = Bsm[hl >> 1] + ((hl & 1) * 196 + blk * S) * k196StageRow + 16 * cch;
+          if (p.skip && p.skip[b]) {                             // skipped batch entry: the mixer output as it is
+            bf16* dst0 = p.dst + b * p.d_sb + h * p.d_sh + 8 * cch;
+#pragma unroll
+            for (int r = 0; r < S; ++r)
+              __stcs(reinterpret_cast<uint4*>(dst0 + (int64_t)(blk * S + r) * p.d_sl), *reinterpret_cast<const uint4*>(st + r * k196StageRow));
+            continue;
+          }
           float x[S][8];
 #pragma unroll
           for (int r = 0; r < S; ++r) {
@@ -565,6 +573,7 @@ int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_ac
     p.Ww1 = wrm->Ww1; p.bw1 = wrm->bw1; p.Ww2 = wrm->Ww2; p.bw2 = wrm->bw2;
     p.hs_w1 = one * (size_t)64 * hid; p.hs_b1 = one * hid;
     p.hs_w2 = one * (size_t)hid * (J + 1) * 64; p.hs_b2 = one * (size_t)(J + 1) * 64;
+    p.skip = wrm->skip;
   }
   const unsigned grid = (unsigned)((p.nheads + k196Heads - 1) / k196Heads);
 #define SPECTRE_TC196_LAUNCH(JJ, WB)                                                                              \

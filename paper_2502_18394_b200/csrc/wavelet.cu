@@ -17,7 +17,22 @@ struct WaveletParams {
   const float* level_gates;       // [B,H,J+1,D] or NULL
   const float* qbar; const void* Ww1; const float* bw1; const void* Ww2; const float* bw2;
   int hidden; size_t hs_w1, hs_b1, hs_w2, hs_b2;
+  const int* skip;                // [B] or NULL: non-zero = pass this batch entry through
 };
+
+// Pass-through of one (batch, head) slab for a skipped batch entry (nothing to do in place).
+template <typename T>
+__device__ __forceinline__ void wavelet_pass_through(const WaveletParams& p, int b, int h, int r0, int nr) {
+  if (p.src == p.dst && p.s_sb == p.d_sb && p.s_sl == p.d_sl && p.s_sh == p.d_sh) return;
+  const T* src = reinterpret_cast<const T*>(p.src) + b * p.s_sb + h * p.s_sh;
+  T* dst = reinterpret_cast<T*>(p.dst) + b * p.d_sb + h * p.d_sh;
+  constexpr int V = 16 / sizeof(T);
+  const int nv = p.D / V;
+  for (int i = threadIdx.x; i < nr * nv; i += blockDim.x) {
+    const int r = i / nv, c = (i - r * nv) * V;
+    *reinterpret_cast<uint4*>(dst + (int64_t)(r0 + r) * p.d_sl + c) = *reinterpret_cast<const uint4*>(src + (int64_t)(r0 + r) * p.s_sl + c);
+  }
+}
 
 template <typename T, typename WT>
 __global__ void __launch_bounds__(256) wavelet_kernel(const WaveletParams p) {
@@ -30,6 +45,7 @@ __global__ void __launch_bounds__(256) wavelet_kernel(const WaveletParams p) {
   const int D = p.D, J = p.J;
   const int r0 = chunk * p.rows;
   const int nr = min(p.rows, p.L - r0);
+  if (p.skip && p.skip[b]) { wavelet_pass_through<T>(p, b, h, r0, nr); return; }
   // level gates (step b): given, or the two-layer MLP on q_bar
   if (p.level_gates) {
     for (int i = threadIdx.x; i < (J + 1) * D; i += blockDim.x) sg[i] = 1.0f + p.level_gates[(size_t)bh * (J + 1) * D + i];
@@ -131,6 +147,7 @@ __global__ void __launch_bounds__(256) wavelet_reg_kernel(const WaveletParams p)
   float* u = sg + (size_t)(J + 1) * p.D;           // [hidden]
   const int bh = blockIdx.x, b = bh / p.H, h = bh - b * p.H;
   const int D = p.D;
+  if (p.skip && p.skip[b]) { wavelet_pass_through<T>(p, b, h, 0, p.L); return; }
   if (p.level_gates) {
     for (int i = threadIdx.x; i < (J + 1) * D; i += blockDim.x) sg[i] = 1.0f + p.level_gates[(size_t)bh * (J + 1) * D + i];
   } else {
@@ -239,7 +256,7 @@ extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spec
     p0.d_sb = y_out->stride_b; p0.d_sl = y_out->stride_l; p0.d_sh = y_out->stride_h;
     p0.B = y_in->B; p0.L = L; p0.H = y_in->H; p0.D = D; p0.J = J;
     p0.level_gates = w->level_gates; p0.qbar = w->qbar; p0.Ww1 = w->Ww1; p0.bw1 = w->bw1; p0.Ww2 = w->Ww2; p0.bw2 = w->bw2;
-    p0.hidden = hidden0;
+    p0.hidden = hidden0; p0.skip = w->skip;
     const size_t one0 = w->shared_across_heads ? 0 : 1;
     p0.hs_w1 = one0 * (size_t)D * hidden0; p0.hs_b1 = one0 * hidden0;
     p0.hs_w2 = one0 * (size_t)hidden0 * (J + 1) * D; p0.hs_b2 = one0 * (size_t)(J + 1) * D;
@@ -266,7 +283,7 @@ extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spec
   p.d_sb = y_out->stride_b; p.d_sl = y_out->stride_l; p.d_sh = y_out->stride_h;
   p.B = y_in->B; p.L = L; p.H = y_in->H; p.D = D; p.J = J; p.rows = rows; p.chunks = (L + rows - 1) / rows;
   p.level_gates = w->level_gates; p.qbar = w->qbar; p.Ww1 = w->Ww1; p.bw1 = w->bw1; p.Ww2 = w->Ww2; p.bw2 = w->bw2;
-  p.hidden = hidden;
+  p.hidden = hidden; p.skip = w->skip;
   const size_t one = w->shared_across_heads ? 0 : 1;
   p.hs_w1 = one * (size_t)D * hidden; p.hs_b1 = one * hidden;
   p.hs_w2 = one * (size_t)hidden * (J + 1) * D; p.hs_b2 = one * (size_t)(J + 1) * D;

@@ -39,7 +39,7 @@ def test_struct_layouts_match_the_header():
     assert C.sizeof(b.Act) == 8 + 4 * 5 + 4 + 8 * 3        # ptr, dtype+BLHD, pad, strides
     assert C.sizeof(b.Cache) == 4 * 6 + 8 * 4
     assert b.GateParams.ln_eps.offset == 32 and b.GateParams.W1.offset == 40
-    assert C.sizeof(b.Wavelet) == 16 + 8 * 6
+    assert C.sizeof(b.Wavelet) == 16 + 8 * 7 and b.Wavelet.skip.offset == 16 + 8 * 6
 
 
 def test_null_arguments_fail_without_a_device(lib):

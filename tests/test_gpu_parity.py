@@ -298,6 +298,31 @@ def test_mixer_196_with_refinement_in_the_store_phase(ctx, J, L, B, H, wdt, hid,
     assert slab_err(W.to_f64(y), ref) < TOL["bf16"]
 
 
+@pytest.mark.parametrize("dt,L,J,D,fused", [("bf16", 196, 2, 64, True), ("f32", 64, 3, 16, False), ("bf16", 2048, 6, 32, False)])
+def test_wavelet_skip_mask(ctx, dt, L, J, D, fused):
+    # flagged batch entries come out unrefined, bit for bit; the others as before.  Register kernel,
+    # tile kernel (J > 4) and the refinement fused into the n = 196 mixer.
+    B, H = 4, 2
+    w = W.Workload("t", B=B, L=L, H=H, D=D, dtype=dt, n_fft=L, seed=J * 100 + L, wavelet_levels=J)
+    gen = torch.Generator().manual_seed(7)
+    lg = 0.5 * torch.randn(B, H, J + 1, D, generator=gen)
+    skip = torch.tensor([0, 1, 1, 0], dtype=torch.int32)
+    x = W.activations(w)
+    wrm = {"levels": J, "level_gates": lg.cuda(), "skip": skip.cuda()}
+    if fused:
+        g = W.random_gate(w)
+        y = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=L, wrm=wrm)
+        plain = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=L)
+        ref = O.wavelet_refine(O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=L), W.to_f64(lg), J, skip=skip.tolist())
+    else:
+        y = torch.empty_like(x, device="cuda")
+        S.spectre_wavelet_refine(ctx, x.cuda(), wrm, y_out=y)
+        plain = x.cuda()
+        ref = O.wavelet_refine(W.to_f64(x), W.to_f64(lg), J, skip=skip.tolist())
+    assert slab_err(W.to_f64(y), ref) < TOL[dt]
+    assert torch.equal(y[1], plain[1]) and torch.equal(y[2], plain[2]) and not torch.equal(y[0], plain[0])
+
+
 # ------------------------------------------------------------------ cache
 def cache_err(cache, st):
     P = W.to_f64(cache.prefix_fft)

@@ -536,3 +536,13 @@ def test_paper_facts_fixture():
         assert O.rfft(np.zeros(n)).shape[0] == expect
         seen += 1
     assert seen == 4
+
+
+def test_wavelet_skip_mask_passes_flagged_batch_entries_through():
+    B, n, H, d, J = 3, 8, 2, 2, 2
+    y = RNG.standard_normal((B, n, H, d))
+    s = RNG.standard_normal((B, H, J + 1, d))
+    full = O.wavelet_refine(y, s, J)
+    part = O.wavelet_refine(y, s, J, skip=[0, 1, 0])
+    assert np.array_equal(part[1], y[1]) and np.array_equal(part[0], full[0]) and np.array_equal(part[2], full[2])
+    assert np.array_equal(O.wavelet_refine(y, s, J, skip=[1, 1, 1]), y)
