@@ -247,18 +247,54 @@ class MixerBench:
 
     def e2e_prepare(self):
         self.pin_x = [x.pin_memory() for x in self.x_host[:2]]
-        self.pin_y = torch.empty_like(self.pin_x[0]).pin_memory()
+        self.pin_y = [torch.empty_like(self.pin_x[0]).pin_memory() for _ in range(2)]
+        # with two or more device buffer sets the copies of neighbouring steps run on their own
+        # streams beside the kernels (every step still copies its input in and its result out)
+        self.pipelined = self.nsets >= 2 and not self.backward
+        if self.pipelined:
+            self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+            self.ev_done, self.ev_out = {}, {}
 
-    def e2e_step(self, k: int):
-        d = self.sets[k % self.nsets]
-        d["x"].copy_(self.pin_x[k % len(self.pin_x)], non_blocking=True)
+    def _compute(self, d):
         if self.project:
             d["proj"]()
         d["gate"]()
         d["mix"]()
         if self.backward:
             d["bwd"]()
-        self.pin_y.copy_(self.dv if self.backward else d["y"], non_blocking=True)
+
+    def e2e_step(self, k: int):
+        i = k % self.nsets
+        d = self.sets[i]
+        if not self.pipelined:
+            d["x"].copy_(self.pin_x[k % len(self.pin_x)], non_blocking=True)
+            self._compute(d)
+            self.pin_y[0].copy_(self.dv if self.backward else d["y"], non_blocking=True)
+            return
+        cur = torch.cuda.current_stream()
+        with torch.cuda.stream(self.s_in):
+            if i in self.ev_done:
+                self.s_in.wait_event(self.ev_done[i])          # the kernels that last read this input buffer
+            d["x"].copy_(self.pin_x[k % len(self.pin_x)], non_blocking=True)
+            ev_in = torch.cuda.Event()
+            ev_in.record(self.s_in)
+        cur.wait_event(ev_in)
+        if i in self.ev_out:
+            cur.wait_event(self.ev_out[i])                     # this set's previous result has left the device
+        self._compute(d)
+        ev_done = torch.cuda.Event()
+        ev_done.record(cur)
+        self.ev_done[i] = ev_done
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(ev_done)
+            self.pin_y[k % 2].copy_(d["y"], non_blocking=True)
+            ev_out = torch.cuda.Event()
+            ev_out.record(self.s_out)
+        self.ev_out[i] = ev_out
+
+    def e2e_finish(self):
+        if self.pipelined:
+            torch.cuda.current_stream().wait_stream(self.s_out)
 
     def cpu_step(self):
         from oracle import spectre_oracle as O
@@ -348,6 +384,9 @@ class AppendBench:
         self.vd[i].copy_(self.pin_v[i], non_blocking=True)
         self._call(100000 + k)()
         self.pin_s.copy_(self.y_rows if self.decode else self.cache.sum_q, non_blocking=True)
+
+    def e2e_finish(self):
+        pass
 
     def cpu_step(self):
         # bounded sample: one (batch) row of the cache, all heads; scaled to tokens/s
@@ -492,6 +531,7 @@ def main():
     ev_a.record()
     for k in range(Ke):
         bench.e2e_step(3 + k)
+    bench.e2e_finish()
     ev_b.record()
     torch.cuda.synchronize()
     R.barrier()
