@@ -43,14 +43,15 @@ typedef enum {
   SPECTRE_ERR_TIMEOUT = 5        /* a bounded on-chip wait ran out (spectre_poll_status) */
 } spectre_status;
 
-typedef enum { SPECTRE_F32 = 0, SPECTRE_BF16 = 1 } spectre_dtype;
+/* Element types of activations and ring buffers; weights are SPECTRE_F32 or SPECTRE_BF16. */
+typedef enum { SPECTRE_F32 = 0, SPECTRE_BF16 = 1, SPECTRE_F16 = 2 } spectre_dtype;
 
 typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch limits */
 
-/* Creates a context for CUDA device `device`.  Besides host memory it owns three small device
- * tables (the 64-point and 49-point DFT matrices of the tensor-core mixers, 32 KiB each, and a
- * quarter-wave twiddle table, 16 KiB) and one pinned status word, all released by
- * spectre_destroy.  No other call allocates. */
+/* Creates a context for CUDA device `device`.  Besides host memory it owns four small device
+ * tables (the 64-point and 49-point DFT matrices of the tensor-core mixers and the twiddles
+ * between two 64-point stages, 32 KiB each, and a quarter-wave twiddle table, 16 KiB) and one
+ * pinned status word, all released by spectre_destroy.  No other call allocates. */
 int spectre_create(spectre_ctx** out, int device);
 int spectre_destroy(spectre_ctx* ctx);
 /* The tensor-core mixer hands tiles between its warps through on-chip barriers whose waits

@@ -24,6 +24,7 @@ SPECTRE_ERR_CUDA = 4
 SPECTRE_ERR_TIMEOUT = 5
 SPECTRE_F32 = 0
 SPECTRE_BF16 = 1
+SPECTRE_F16 = 2
 
 EXPORTS = [
     "spectre_create", "spectre_destroy", "spectre_status_string", "spectre_last_error", "spectre_poll_status",
@@ -136,6 +137,8 @@ def _dtype_code(t: torch.Tensor) -> int:
         return SPECTRE_F32
     if t.dtype == torch.bfloat16:
         return SPECTRE_BF16
+    if t.dtype == torch.float16:
+        return SPECTRE_F16
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 

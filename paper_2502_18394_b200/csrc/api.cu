@@ -59,10 +59,10 @@ int check_act(const spectre_act* a, const char* name) {
   std::string nm(name);
   if (!a) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": descriptor is NULL");
   if (!a->ptr) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": data pointer is NULL");
-  if (a->dtype != SPECTRE_F32 && a->dtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": unknown dtype");
+  if (!is_io_dtype(a->dtype)) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": unknown dtype");
   if (a->B < 1 || a->L < 1 || a->H < 1 || a->D < 1) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": non-positive extent");
   if (a->D % 8 != 0) return fail(SPECTRE_ERR_UNSUPPORTED, nm + ": D must be a multiple of 8");
-  const int64_t es = a->dtype == SPECTRE_BF16 ? 2 : 4;
+  const int64_t es = io_elem_bytes(a->dtype);
   if (reinterpret_cast<uintptr_t>(a->ptr) & 15) return fail(SPECTRE_ERR_INVALID_ARG, nm + ": pointer not 16-byte aligned");
   if ((a->stride_b * es) % 16 || (a->stride_l * es) % 16 || (a->stride_h * es) % 16)
     return fail(SPECTRE_ERR_INVALID_ARG, nm + ": strides must keep rows 16-byte aligned");

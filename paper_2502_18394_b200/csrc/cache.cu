@@ -251,7 +251,7 @@ static int check_cache(const spectre_cache* c) {
   if (!c) return fail(SPECTRE_ERR_INVALID_ARG, "cache descriptor is NULL");
   if (c->B < 1 || c->H < 1 || c->D < 1 || c->N_max < 2) return fail(SPECTRE_ERR_INVALID_ARG, "cache extents");
   if (c->D % 8) return fail(SPECTRE_ERR_UNSUPPORTED, "cache D must be a multiple of 8");
-  if (c->buf_dtype != SPECTRE_F32 && c->buf_dtype != SPECTRE_BF16) return fail(SPECTRE_ERR_INVALID_ARG, "cache dtype");
+  if (!is_io_dtype(c->buf_dtype)) return fail(SPECTRE_ERR_INVALID_ARG, "cache dtype");
   if (!c->prefix_fft || !c->V_buf || !c->Q_buf || !c->sum_q) return fail(SPECTRE_ERR_INVALID_ARG, "cache pointer is NULL");
   if ((reinterpret_cast<uintptr_t>(c->prefix_fft) | reinterpret_cast<uintptr_t>(c->V_buf) |
        reinterpret_cast<uintptr_t>(c->Q_buf)) & 15)
@@ -310,21 +310,15 @@ extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, cons
     split_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, cache->prefix_fft, N, K, D, N1, M, s0, cnt);
     SPECTRE_LAUNCH_OK("split_kernel");
   }
-  const bool bf = cache->buf_dtype == SPECTRE_BF16;
-  const int V = bf ? 8 : 4;
+  const int V = 16 / io_elem_bytes(cache->buf_dtype);
   size_t total = (size_t)B * N * (H * D / V);
   unsigned blocks = (unsigned)((total + 255) / 256);
-  if (bf) {
-    ring_fill_kernel<bf16><<<blocks, 256, 0, st>>>(reinterpret_cast<const bf16*>(v->ptr), v->stride_b, v->stride_l,
-                                                    v->stride_h, reinterpret_cast<bf16*>(cache->V_buf), B, N, H, D, v->L);
-    ring_fill_kernel<bf16><<<blocks, 256, 0, st>>>(reinterpret_cast<const bf16*>(q->ptr), q->stride_b, q->stride_l,
-                                                    q->stride_h, reinterpret_cast<bf16*>(cache->Q_buf), B, N, H, D, q->L);
-  } else {
-    ring_fill_kernel<float><<<blocks, 256, 0, st>>>(reinterpret_cast<const float*>(v->ptr), v->stride_b, v->stride_l,
-                                                     v->stride_h, reinterpret_cast<float*>(cache->V_buf), B, N, H, D, v->L);
-    ring_fill_kernel<float><<<blocks, 256, 0, st>>>(reinterpret_cast<const float*>(q->ptr), q->stride_b, q->stride_l,
-                                                     q->stride_h, reinterpret_cast<float*>(cache->Q_buf), B, N, H, D, q->L);
-  }
+  SPECTRE_IO_DISPATCH(cache->buf_dtype, {
+    ring_fill_kernel<T><<<blocks, 256, 0, st>>>(reinterpret_cast<const T*>(v->ptr), v->stride_b, v->stride_l, v->stride_h,
+                                                reinterpret_cast<T*>(cache->V_buf), B, N, H, D, v->L);
+    ring_fill_kernel<T><<<blocks, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
+                                                reinterpret_cast<T*>(cache->Q_buf), B, N, H, D, q->L);
+  });
   SPECTRE_LAUNCH_OK("ring_fill_kernel");
   return pool_sum(ctx, st, q, cache->sum_q, 1);
 }
@@ -347,23 +341,14 @@ extern "C" int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const
   const size_t nwarps = (size_t)B * H * wps;
   const unsigned blocks = (unsigned)((nwarps * 32 + 255) / 256);
   const unsigned blocks2 = (unsigned)(((size_t)B * H * D + 255) / 256);
-  if (cache->buf_dtype == SPECTRE_BF16) {
-    append_spectrum_kernel<bf16><<<blocks, 256, 0, st>>>(cache->prefix_fft, reinterpret_cast<const bf16*>(cache->V_buf),
-                                                         reinterpret_cast<const bf16*>(v_t), H, D, N, K, slot,
-                                                         (unsigned)slot, evict, wps, nwarps);
-    append_ring_kernel<bf16><<<blocks2, 256, 0, st>>>(reinterpret_cast<bf16*>(cache->V_buf),
-                                                      reinterpret_cast<bf16*>(cache->Q_buf), cache->sum_q,
-                                                      reinterpret_cast<const bf16*>(q_t),
-                                                      reinterpret_cast<const bf16*>(v_t), B, H, D, N, slot, evict);
-  } else {
-    append_spectrum_kernel<float><<<blocks, 256, 0, st>>>(cache->prefix_fft, reinterpret_cast<const float*>(cache->V_buf),
-                                                          reinterpret_cast<const float*>(v_t), H, D, N, K, slot,
-                                                          (unsigned)slot, evict, wps, nwarps);
-    append_ring_kernel<float><<<blocks2, 256, 0, st>>>(reinterpret_cast<float*>(cache->V_buf),
-                                                       reinterpret_cast<float*>(cache->Q_buf), cache->sum_q,
-                                                       reinterpret_cast<const float*>(q_t),
-                                                       reinterpret_cast<const float*>(v_t), B, H, D, N, slot, evict);
-  }
+  SPECTRE_IO_DISPATCH(cache->buf_dtype, {
+    append_spectrum_kernel<T><<<blocks, 256, 0, st>>>(cache->prefix_fft, reinterpret_cast<const T*>(cache->V_buf),
+                                                      reinterpret_cast<const T*>(v_t), H, D, N, K, slot, (unsigned)slot,
+                                                      evict, wps, nwarps);
+    append_ring_kernel<T><<<blocks2, 256, 0, st>>>(reinterpret_cast<T*>(cache->V_buf), reinterpret_cast<T*>(cache->Q_buf),
+                                                   cache->sum_q, reinterpret_cast<const T*>(q_t),
+                                                   reinterpret_cast<const T*>(v_t), B, H, D, N, slot, evict);
+  });
   SPECTRE_LAUNCH_OK("append kernels");
   return SPECTRE_OK;
 }
@@ -411,17 +396,12 @@ extern "C" int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, 
   void* gate_ws = reinterpret_cast<unsigned char*>(workspace) + delta_bytes + part_bytes;
   const int slot = (int)(t % N);
   const int evict = t >= N ? 1 : 0;
-  const bool bf = cache->buf_dtype == SPECTRE_BF16;
   // (a)-(b) ring buffers, running sum, delta
   const unsigned blocks_r = (unsigned)(((size_t)B * H * D + 255) / 256);
-  if (bf)
-    decode_ring_kernel<bf16><<<blocks_r, 256, 0, st>>>(reinterpret_cast<bf16*>(cache->V_buf), reinterpret_cast<bf16*>(cache->Q_buf),
-                                                       cache->sum_q, delta, reinterpret_cast<const bf16*>(q_t),
-                                                       reinterpret_cast<const bf16*>(v_t), B, H, D, N, slot, evict);
-  else
-    decode_ring_kernel<float><<<blocks_r, 256, 0, st>>>(reinterpret_cast<float*>(cache->V_buf), reinterpret_cast<float*>(cache->Q_buf),
-                                                        cache->sum_q, delta, reinterpret_cast<const float*>(q_t),
-                                                        reinterpret_cast<const float*>(v_t), B, H, D, N, slot, evict);
+  SPECTRE_IO_DISPATCH(cache->buf_dtype,
+                      decode_ring_kernel<T><<<blocks_r, 256, 0, st>>>(reinterpret_cast<T*>(cache->V_buf), reinterpret_cast<T*>(cache->Q_buf),
+                                                                      cache->sum_q, delta, reinterpret_cast<const T*>(q_t),
+                                                                      reinterpret_cast<const T*>(v_t), B, H, D, N, slot, evict));
   SPECTRE_LAUNCH_OK("decode_ring_kernel");
   // (c)-(d) gate from the running sum with phase p = t
   rc = spectre_gate(ctx, stream, nullptr, cache->sum_q, B, H, D, 1.0f / (float)N, params, N, nullptr, t, g_out, nullptr,
@@ -437,8 +417,8 @@ extern "C" int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, 
   else decode_spectrum_kernel<SPECTRE_DECODE_MAX_ROWS><<<blocks_s, 256, 0, st>>>(cache->prefix_fft, delta, g2, partial, D, N, K, (unsigned)slot, dr, nblk);
   SPECTRE_LAUNCH_OK("decode_spectrum_kernel");
   const unsigned blocks_y = (unsigned)(((size_t)B * nrows * H * D + 255) / 256);
-  if (bf) decode_reduce_kernel<bf16><<<blocks_y, 256, 0, st>>>(partial, reinterpret_cast<bf16*>(y_rows), B, H, D, nblk, NR, nrows);
-  else decode_reduce_kernel<float><<<blocks_y, 256, 0, st>>>(partial, reinterpret_cast<float*>(y_rows), B, H, D, nblk, NR, nrows);
+  SPECTRE_IO_DISPATCH(cache->buf_dtype,
+                      decode_reduce_kernel<T><<<blocks_y, 256, 0, st>>>(partial, reinterpret_cast<T*>(y_rows), B, H, D, nblk, NR, nrows));
   SPECTRE_LAUNCH_OK("decode_reduce_kernel");
   return SPECTRE_OK;
 }

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -52,6 +53,7 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 #ifdef __CUDACC__
 
 typedef __nv_bfloat16 bf16;
+typedef __half f16;
 
 __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
 __device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
@@ -109,6 +111,33 @@ template <> struct io<bf16> {
   static __device__ __forceinline__ float load1(const bf16* p) { return __bfloat162float(*p); }
   static __device__ __forceinline__ void store1(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
 };
+template <> struct io<f16> {
+  static __device__ __forceinline__ float4 load4(const f16* p) {
+    const uint2 r = *reinterpret_cast<const uint2*>(p);
+    const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&r.x));
+    const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&r.y));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+  }
+  static __device__ __forceinline__ void store4(f16* p, float4 v) {
+    const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
+    uint2 r;
+    r.x = *reinterpret_cast<const unsigned*>(&lo);
+    r.y = *reinterpret_cast<const unsigned*>(&hi);
+    *reinterpret_cast<uint2*>(p) = r;
+  }
+  static __device__ __forceinline__ float load1(const f16* p) { return __half2float(*p); }
+  static __device__ __forceinline__ void store1(f16* p, float v) { *p = __float2half_rn(v); }
+};
+
+// Runs the statement(s) with T bound to the element type of an activation dtype.
+#define SPECTRE_IO_DISPATCH(dtype, ...)                                        \
+  do {                                                                         \
+    if ((dtype) == SPECTRE_BF16) { using T = ::spectre::bf16; __VA_ARGS__; }   \
+    else if ((dtype) == SPECTRE_F16) { using T = ::spectre::f16; __VA_ARGS__; } \
+    else { using T = float; __VA_ARGS__; }                                     \
+  } while (0)
+inline bool is_io_dtype(int d) { return d == SPECTRE_F32 || d == SPECTRE_BF16 || d == SPECTRE_F16; }
+inline int io_elem_bytes(int d) { return d == SPECTRE_F32 ? 4 : 2; }
 
 // ---- constant roots of unity -----------------------------------------------
 // x * exp(-/+ j 2 pi J / R) for compile-time-foldable (J, R); INV conjugates.

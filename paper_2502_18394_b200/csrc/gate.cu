@@ -26,6 +26,18 @@ template <> struct vec8<bf16> {
     }
   }
 };
+template <> struct vec8<f16> {
+  static __device__ __forceinline__ void add(const f16* p, float (&a)[8]) {
+    const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&u[i]));
+      a[2 * i] += v.x;
+      a[2 * i + 1] += v.y;
+    }
+  }
+};
 template <> struct vec8<float> {
   static __device__ __forceinline__ void add(const float* p, float (&a)[8]) {
     const float4 lo = __ldg(reinterpret_cast<const float4*>(p)), hi = __ldg(reinterpret_cast<const float4*>(p) + 1);
@@ -77,12 +89,9 @@ int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, floa
   int rows_per = (q->L + target - 1) / target;
   if (rows_per < 32) rows_per = 32;
   dim3 grid((q->L + rows_per - 1) / rows_per, q->B);
-  if (q->dtype == SPECTRE_BF16)
-    pool_kernel<bf16><<<grid, 256, 0, st>>>(reinterpret_cast<const bf16*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
-                                             q->L, q->H, q->D, rows_per, ncopy, copy_stride, sums);
-  else
-    pool_kernel<float><<<grid, 256, 0, st>>>(reinterpret_cast<const float*>(q->ptr), q->stride_b, q->stride_l,
-                                              q->stride_h, q->L, q->H, q->D, rows_per, ncopy, copy_stride, sums);
+  SPECTRE_IO_DISPATCH(q->dtype, pool_kernel<T><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l,
+                                                                     q->stride_h, q->L, q->H, q->D, rows_per, ncopy,
+                                                                     copy_stride, sums));
   SPECTRE_LAUNCH_OK("pool_kernel");
   return SPECTRE_OK;
 }

@@ -608,20 +608,20 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
   p.src = v->ptr;
   p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
   p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
-  const bool bf = v->dtype == SPECTRE_BF16;
   if (pl.N1 == 1) {
     p.src_ws = 0;
-    return bf ? launch_onchip<bf16>(p, pl, cnt, st) : launch_onchip<float>(p, pl, cnt, st);
+    SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
   }
   StridedParams sp = {};
   sp.src = v->ptr; sp.ws = ws;
   sp.s_sb = v->stride_b; sp.s_sl = v->stride_l; sp.s_sh = v->stride_h;
   sp.H = v->H; sp.D = v->D; sp.L = v->L; sp.n = pl.n; sp.M = pl.M;
   sp.slab0 = slab0; sp.nslab = cnt;
-  int rc = bf ? launch_strided<bf16, false>(sp, pl.N1, st) : launch_strided<float, false>(sp, pl.N1, st);
+  int rc = SPECTRE_OK;
+  SPECTRE_IO_DISPATCH(v->dtype, rc = (launch_strided<T, false>(sp, pl.N1, st)));
   if (rc != SPECTRE_OK) return rc;
   p.src_ws = 1;
-  return bf ? launch_onchip<bf16>(p, pl, cnt, st) : launch_onchip<float>(p, pl, cnt, st);
+  SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
 }
 
 // Inverse transform only (read-out of the Prefix-FFT cache): y = R_n^{-1}(diag(g) spec) for all
@@ -677,8 +677,7 @@ int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* 
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 15)) return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
   }
   const float2* sp = reinterpret_cast<const float2*>(spec);
-  return y->dtype == SPECTRE_BF16 ? inverse_typed<bf16>(ctx, st, sp, g, y, pl, ws, ws_bytes)
-                                  : inverse_typed<float>(ctx, st, sp, g, y, pl, ws, ws_bytes);
+  SPECTRE_IO_DISPATCH(y->dtype, return inverse_typed<T>(ctx, st, sp, g, y, pl, ws, ws_bytes));
 }
 
 bool transform_supported(const spectre_ctx* ctx, int n) {
@@ -752,8 +751,7 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
     if (wrm && !fuse_wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
     return SPECTRE_OK;
   }
-  rc = (v->dtype == SPECTRE_BF16) ? mixer_typed<bf16>(ctx, st, v, g, y, pl, workspace, workspace_bytes)
-                                  : mixer_typed<float>(ctx, st, v, g, y, pl, workspace, workspace_bytes);
+  SPECTRE_IO_DISPATCH(v->dtype, rc = mixer_typed<T>(ctx, st, v, g, y, pl, workspace, workspace_bytes));
   if (rc != SPECTRE_OK) return rc;
   if (wrm) return spectre_wavelet_refine(ctx, stream, y, y, wrm);
   return SPECTRE_OK;

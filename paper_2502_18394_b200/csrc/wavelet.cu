@@ -135,6 +135,10 @@ template <> struct pair_io<bf16> {
     *reinterpret_cast<uint32_t*>(p) = *reinterpret_cast<uint32_t*>(&o);
   }
 };
+template <> struct pair_io<f16> {
+  static __device__ __forceinline__ float2 load(const f16* p) { return __half22float2(*reinterpret_cast<const __half2*>(p)); }
+  static __device__ __forceinline__ void store(f16* p, float2 v) { *reinterpret_cast<__half2*>(p) = __floats2half2_rn(v.x, v.y); }
+};
 template <> struct pair_io<float> {
   static __device__ __forceinline__ float2 load(const float* p) { return *reinterpret_cast<const float2*>(p); }
   static __device__ __forceinline__ void store(float* p, float2 v) { *reinterpret_cast<float2*>(p) = v; }
@@ -262,11 +266,11 @@ extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spec
     p0.hs_w2 = one0 * (size_t)hidden0 * (J + 1) * D; p0.hs_b2 = one0 * (size_t)(J + 1) * D;
     const size_t smem0 = ((size_t)(J + 1) * D + hidden0) * sizeof(float);
     const unsigned grid0 = (unsigned)((size_t)p0.B * p0.H);
-    const bool bf0 = y_in->dtype == SPECTRE_BF16, wbf0 = w->wdtype == SPECTRE_BF16;
-    if (bf0 && wbf0) return launch_wavelet_reg<bf16, bf16>(p0, J, grid0, smem0, st0);
-    if (bf0) return launch_wavelet_reg<bf16, float>(p0, J, grid0, smem0, st0);
-    if (wbf0) return launch_wavelet_reg<float, bf16>(p0, J, grid0, smem0, st0);
-    return launch_wavelet_reg<float, float>(p0, J, grid0, smem0, st0);
+    const bool wbf0 = w->wdtype == SPECTRE_BF16;
+    SPECTRE_IO_DISPATCH(y_in->dtype, {
+      if (wbf0) return launch_wavelet_reg<T, bf16>(p0, J, grid0, smem0, st0);
+      return launch_wavelet_reg<T, float>(p0, J, grid0, smem0, st0);
+    });
   }
   const int span = 1 << J;
   int rows = (8192 / D) / span * span;      // about 32 KB of fp32 per CTA
@@ -288,7 +292,7 @@ extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spec
   p.hs_w1 = one * (size_t)D * hidden; p.hs_b1 = one * hidden;
   p.hs_w2 = one * (size_t)hidden * (J + 1) * D; p.hs_b2 = one * (size_t)(J + 1) * D;
   const unsigned grid = (unsigned)((size_t)p.B * p.H * p.chunks);
-  const bool bf = y_in->dtype == SPECTRE_BF16, wbf = w->wdtype == SPECTRE_BF16;
+  const bool wbf = w->wdtype == SPECTRE_BF16;
 #define SPECTRE_WAVELET_LAUNCH(T, WT)                                                                           \
   do {                                                                                                          \
     if (smem > 48 * 1024)                                                                                       \
@@ -296,10 +300,10 @@ extern "C" int spectre_wavelet_refine(spectre_ctx* ctx, void* stream, const spec
                                            (int)smem));                                                         \
     wavelet_kernel<T, WT><<<grid, 256, smem, st>>>(p);                                                          \
   } while (0)
-  if (bf && wbf) SPECTRE_WAVELET_LAUNCH(bf16, bf16);
-  else if (bf) SPECTRE_WAVELET_LAUNCH(bf16, float);
-  else if (wbf) SPECTRE_WAVELET_LAUNCH(float, bf16);
-  else SPECTRE_WAVELET_LAUNCH(float, float);
+  SPECTRE_IO_DISPATCH(y_in->dtype, {
+    if (wbf) SPECTRE_WAVELET_LAUNCH(T, bf16);
+    else SPECTRE_WAVELET_LAUNCH(T, float);
+  });
 #undef SPECTRE_WAVELET_LAUNCH
   SPECTRE_LAUNCH_OK("wavelet_kernel");
   return SPECTRE_OK;

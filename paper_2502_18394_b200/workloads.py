@@ -28,7 +28,7 @@ class Workload:
     L: int
     H: int
     D: int
-    dtype: str = "bf16"          # I/O dtype of activations ("f32" | "bf16")
+    dtype: str = "bf16"          # I/O dtype of activations ("f32" | "bf16" | "f16")
     wdtype: str = "bf16"         # dtype of the gate MLP matrices
     hidden: int = 64             # gate-MLP hidden width
     n_fft: int = 0               # 0 -> n_fft = L (exact circular transform)
@@ -62,7 +62,7 @@ def scaled(w: Workload, **kw) -> Workload:
 
 
 def torch_dtype(name: str) -> torch.dtype:
-    return {"f32": torch.float32, "bf16": torch.bfloat16}[name]
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[name]
 
 
 def _gen(seed: int, stream: int) -> torch.Generator:

@@ -564,6 +564,55 @@ def test_mixer_backward(ctx, dt, L, n, D):
     assert torch.equal(only_dg, dg)
 
 
+# ------------------------------------------------------------------ fp16 I/O
+@pytest.mark.parametrize("n,L,D", [(64, 64, 16), (196, 196, 64), (1000, 1000, 24), (4096, 4096, 16), (8192, 8192, 64),
+                                   (8192, 6000, 64), (16384, 16384, 16), (65536, 65536, 64)])
+def test_mixer_fp16_io(ctx, n, L, D):
+    # the paper's inference precision: fp16 activations in and out
+    w = W.Workload("t", B=2, L=L, H=2, D=D, dtype="f16", n_fft=n, seed=n + D)
+    assert run_mixer(ctx, w, structured=True, n_fft=n) < TOL["f16"]
+    torch.cuda.synchronize()
+    ctx.poll_status()
+
+
+def test_fp16_io_gate_wavelet_cache_decode_backward(ctx):
+    N, L, B, H, D = 256, 200, 2, 2, 16
+    w = W.Workload("t", B=B, L=L, H=H, D=D, dtype="f16", wdtype="f32", n_fft=N, seed=99, N_max=N, wavelet_levels=2)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    p = W.gate_params(w, modrelu_bias_std=0.05)
+    pd, pn = to_dev(p), gate_params_np(p)
+    # gate from fp16 queries
+    g = S.spectre_gate(ctx, pd, N, q=q.cuda())
+    g_ref = O.gate(W.to_f64(q).sum(axis=1), 1.0 / L, N, **pn)
+    assert rel_err(gate_to_complex(g), g_ref) < 1e-5
+    # refinement
+    lg = 0.5 * torch.randn(B, H, 3, D, generator=torch.Generator().manual_seed(1))
+    y = S.spectre_wavelet_refine(ctx, v.cuda(), {"levels": 2, "level_gates": lg.cuda()})
+    assert slab_err(W.to_f64(y), O.wavelet_refine(W.to_f64(v), W.to_f64(lg), 2)) < TOL["f16"]
+    # cache: prefill, appends, decode step with read-out rows, whole-window read-out
+    cache = S.PrefixCache(B, H, D, N, dtype=torch.float16)
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    st = O.cache_prefill(W.to_f64(q), W.to_f64(v), N)
+    qs, vs = W.decode_tokens(w, 80)
+    for i in range(79):
+        S.spectre_prefix_cache_append(ctx, cache, qs[i].cuda(), vs[i].cuda(), L + i)
+        O.cache_append(st, L + i, W.to_f64(qs[i]), W.to_f64(vs[i]))
+    rows = [N - 1, 3]
+    yr, gd = S.spectre_prefix_cache_decode_step(ctx, cache, qs[79].cuda(), vs[79].cuda(), L + 79, pd, rows)
+    ref_rows, g_dec = O.decode_step(st, L + 79, W.to_f64(qs[79]), W.to_f64(vs[79]), pn, rows)
+    e_p, e_s = cache_err(cache, st)
+    assert e_p < 2e-5 and e_s < 2e-5
+    assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"])
+    assert rel_err(W.to_f64(yr), ref_rows) < TOL["f16"]
+    full = S.spectre_prefix_cache_readout(ctx, cache, gd)
+    assert slab_err(W.to_f64(full), O.decode_readout(st, g_dec)) < TOL["f16"]
+    # backward
+    dv, dg = S.spectre_mixer_backward(ctx, v.cuda(), q.cuda(), g, n_fft=N)
+    rv, rg = O.mixer_backward(W.to_f64(v), W.to_f64(q), gate_to_complex(g), n_fft=N)
+    assert slab_err(W.to_f64(dv), rv) < TOL["f16"]
+    assert max(rel_err(gate_to_complex(dg)[b, h], rg[b, h]) for b in range(B) for h in range(H)) < 2e-5
+
+
 # ------------------------------------------------------------------ errors
 def test_invalid_arguments_are_rejected_before_launch(ctx):
     x = torch.zeros(1, 64, 2, 16, device="cuda")

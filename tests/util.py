@@ -4,7 +4,8 @@ import torch
 
 from paper_2502_18394_b200 import workloads as W
 
-TOL = {"f32": 1e-5, "bf16": 1e-2}     # max relative L2 error per (batch, head) slab
+# max relative L2 error per (batch, head) slab; fp16 I/O (11-bit significand) sits three bits under bf16
+TOL = {"f32": 1e-5, "bf16": 1e-2, "f16": 2e-3}
 
 
 def slab_err(y_gpu, y_ref):
