@@ -120,7 +120,7 @@ def describe(w: W.Workload) -> str:
 
 
 def mixer_algorithmic_bytes(w: W.Workload) -> int:
-    es = 2 if w.dtype == "bf16" else 4
+    es = 4 if w.dtype == "f32" else 2
     return 2 * w.B * w.L * w.H * w.D * es + w.B * w.H * w.K * 8          # read V, write Y, read g
 
 
@@ -137,7 +137,7 @@ class MixerBench:
         from paper_2502_18394_b200 import binding as S
         self.S, self.w, self.dev, self.backward, self.project = S, w, dev, backward, project
         self.ctx = S.Context(dev.index)
-        per_set = 2 * w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
+        per_set = 2 * w.B * w.L * w.H * w.D * (4 if w.dtype == "f32" else 2)
         if nsets is None:
             nsets = 1 if per_set > 2 * L2_BYTES else max(2, int(4 * L2_BYTES / per_set) + 1)
         self.nsets = nsets
@@ -149,7 +149,7 @@ class MixerBench:
             params["shared_across_heads"] = 1
         self.sets = []
         ws_gate = S.spectre_gate_workspace_bytes(self.ctx, w.B, w.H, w.D, w.n, 0)
-        ws_mix = S.spectre_mixer_workspace_bytes(self.ctx, w.B, w.L, w.H, w.D, w.n, S.SPECTRE_BF16 if w.dtype == "bf16" else S.SPECTRE_F32)
+        ws_mix = S.spectre_mixer_workspace_bytes(self.ctx, w.B, w.L, w.H, w.D, w.n, {"f32": S.SPECTRE_F32, "bf16": S.SPECTRE_BF16, "f16": S.SPECTRE_F16}[w.dtype])
         self.ws_mix = torch.empty(max(ws_mix, 16), dtype=torch.uint8, device=dev) if ws_mix else None
         wp = W.wavelet_params(w) if w.wavelet_levels else None
         for i in range(nsets):
@@ -180,7 +180,7 @@ class MixerBench:
                 # training-like step: the forward output stands in for the incoming gradient
                 if i == 0:
                     nb = S.spectre_mixer_backward_workspace_bytes(self.ctx, w.B, w.L, w.H, w.D, w.n,
-                                                                  S.SPECTRE_BF16 if w.dtype == "bf16" else S.SPECTRE_F32)
+                                                                  {"f32": S.SPECTRE_F32, "bf16": S.SPECTRE_BF16, "f16": S.SPECTRE_F16}[w.dtype])
                     self.ws_bwd = torch.empty(max(nb, 16), dtype=torch.uint8, device=dev)
                     self.dv = torch.empty_like(d["y"])
                 d["dg"] = torch.empty_like(d["g"])
@@ -192,9 +192,9 @@ class MixerBench:
         # gate images + transpose-in + core + transpose-out per group of heads (staged tensor-core
         # path) or strided + on-chip + strided per group (fp32 four-step path); + wavelet
         import math
-        if w.dtype == "bf16" and w.n == 8192:
+        if w.dtype in ("bf16", "f16") and w.n == 8192:
             self.kernel_name, nk = "mixer_tc8192_kernel (single-kernel tcgen05 mixer)", 1
-        elif w.dtype == "bf16" and ws_mix and w.n >= 4096:
+        elif w.dtype in ("bf16", "f16") and ws_mix and w.n >= 4096:
             R, ntile = w.n // 4096, w.D // 8
             per = R * ntile * (32 * 2064 + 65536) + R * 18432 + 256
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
@@ -206,9 +206,9 @@ class MixerBench:
         else:
             self.kernel_name, nk = "mixer (onchip_kernel)", 1
         # pool, gate_out (+ gate_hidden when a head's bins span >= 32 CTAs), mixer kernels, wavelet
-        fused_wrm = w.dtype == "bf16" and w.n == 196 and w.D == 64 and w.wavelet_levels in (1, 2) and w.wavelet_hidden <= 256
+        fused_wrm = w.dtype in ("bf16", "f16") and w.n == 196 and w.D == 64 and w.wavelet_levels in (1, 2) and w.wavelet_hidden <= 256
         self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels and not fused_wrm else 0)
-        self.h2d = w.B * w.L * w.H * w.D * (2 if w.dtype == "bf16" else 4)
+        self.h2d = w.B * w.L * w.H * w.D * (4 if w.dtype == "f32" else 2)
         self.d2h = self.h2d
         if project:
             es = 2
@@ -337,7 +337,7 @@ class AppendBench:
         self.alg_bytes = append_algorithmic_bytes(w)
         self.kernel_name = "append_spectrum_kernel"
         self.launches_per_step = 2
-        es = 2 if w.dtype == "bf16" else 4
+        es = 4 if w.dtype == "f32" else 2
         self.h2d = 2 * w.B * w.H * w.D * es
         self.d2h = w.B * w.H * w.D * 4
         if decode:
@@ -468,6 +468,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
     ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
+    ap.add_argument("--io-dtype", default=None, choices=["bf16", "f16", "f32"], help="override the activation dtype (f16 = the paper's inference precision)")
     ap.add_argument("--shared-gates", action="store_true", help="mixer workloads: one gate network shared by all heads (Sec. 3.6)")
     ap.add_argument("--project", action="store_true", help="mixer workloads (bf16, d = 64): step = projections + gate from sum_q + mixer; the timed call is the projection")
     ap.add_argument("--backward", action="store_true", help="mixer workloads: step = gate + forward + backward; the timed call is the backward")
@@ -478,6 +479,8 @@ def main():
         w = W.scaled(w, H=args.heads, name=f"{w.name} reduced to H={args.heads}")
     if args.batch:
         w = W.scaled(w, B=args.batch, name=f"{w.name} reduced to B={args.batch}")
+    if args.io_dtype and args.io_dtype != w.dtype:
+        w = W.scaled(w, dtype=args.io_dtype, name=f"{w.name} with {args.io_dtype} activations")
     rank, local_rank, world = R.world()
 
     if args.impl == "reference":

@@ -697,7 +697,7 @@ extern "C" size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t 
   TransformPlan pl;
   if (!ctx || B < 1 || H < 1 || D < 8 || !make_plan(ctx, n_fft, &pl)) return 0;
   const int force = forced_path();
-  if (dtype == SPECTRE_BF16 && ctx->dft64 && tc4k_supported(n_fft, D) && force != kPathAlu && force != kPathFused &&
+  if ((dtype == SPECTRE_BF16 || dtype == SPECTRE_F16) && ctx->dft64 && tc4k_supported(n_fft, D) && force != kPathAlu && force != kPathFused &&
       (n_fft != 8192 || force == kPathStaged))               // n = 8192 defaults to the single-kernel path
     return tc4k_workspace_bytes(ctx, n_fft, D, B * H);
   if (pl.N1 == 1) return 0;
@@ -719,7 +719,7 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   TransformPlan pl;
   if (!make_plan(ctx, n_fft, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "n_fft outside the supported set");
   const int force = forced_path();
-  const bool tc_ok = v->dtype == SPECTRE_BF16 && ctx->dft64 != nullptr && force != kPathAlu;
+  const bool tc_ok = (v->dtype == SPECTRE_BF16 || v->dtype == SPECTRE_F16) && ctx->dft64 != nullptr && force != kPathAlu;
   const bool ws_ok = workspace && !(reinterpret_cast<uintptr_t>(workspace) & 15);
   const bool tc196 = tc_ok && n_fft == 196 && v->D == 64 && ctx->dft49 != nullptr;
   const bool fused = tc_ok && n_fft == 8192 && force != kPathStaged && tc8192_supported(v, y);

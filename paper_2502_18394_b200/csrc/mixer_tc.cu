@@ -133,7 +133,7 @@ template <> struct wpair<false> {
   static __device__ __forceinline__ float2 cvt(raw r) { return r; }
 };
 
-template <int J, bool WBF>
+template <int J, bool WBF, bool F16>
 __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196Params p) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* Fsm = smem;
@@ -237,7 +237,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
 #pragma unroll
         for (int n1 = 0; n1 < 4; ++n1) {
           const uint32_t u = j == 0 ? rr[it][n1].x : (j == 1 ? rr[it][n1].y : (j == 2 ? rr[it][n1].z : rr[it][n1].w));
-          x[n1] = make_float2(0.5f * __uint_as_float(u << 16), 0.5f * __uint_as_float(u & 0xffff0000u));
+          const float2 xv = F16 ? unpack_h2(u) : make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+          x[n1] = make_float2(0.5f * xv.x, 0.5f * xv.y);
         }
         Dft<4, false>::run(x);
         x[1] = cmul(x[1], w1);
@@ -426,7 +427,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
 #pragma unroll
             for (int n1 = 0; n1 < 4; ++n1) {
               const int row = tp + 49 * n1;
-              const uint2 out = pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y);
+              const uint2 out = F16 ? make_uint2(pack_h2(gs * y0[n1].x, gs * y0[n1].y), pack_h2(gs * y1[n1].x, gs * y1[n1].y))
+                                    : pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y);
               if (J > 0) *reinterpret_cast<uint2*>(Bsm[half] + ((hl & 1) * 196 + row) * k196StageRow + 2 * col) = out;
               else if (row < p.L) __stcs(reinterpret_cast<uint2*>(dst + (int64_t)row * p.d_sl + col), out);
             }
@@ -463,8 +465,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
             const uint32_t w4[4] = {u4.x, u4.y, u4.z, u4.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              x[r][2 * e] = __uint_as_float(w4[e] << 16);
-              x[r][2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
+              const float2 xv = F16 ? unpack_h2(w4[e]) : make_float2(__uint_as_float(w4[e] << 16), __uint_as_float(w4[e] & 0xffff0000u));
+              x[r][2 * e] = xv.x;
+              x[r][2 * e + 1] = xv.y;
             }
           }
           // analysis in place: after level l, slot i 2^l holds a_l and slot i 2^l + 2^(l-1) holds d_l
@@ -504,8 +507,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
 #pragma unroll
           for (int r = 0; r < S; ++r) {
             uint4 o;
-            o.x = pack_bf2(x[r][0], x[r][1]); o.y = pack_bf2(x[r][2], x[r][3]);
-            o.z = pack_bf2(x[r][4], x[r][5]); o.w = pack_bf2(x[r][6], x[r][7]);
+            if (F16) {
+              o.x = pack_h2(x[r][0], x[r][1]); o.y = pack_h2(x[r][2], x[r][3]);
+              o.z = pack_h2(x[r][4], x[r][5]); o.w = pack_h2(x[r][6], x[r][7]);
+            } else {
+              o.x = pack_bf2(x[r][0], x[r][1]); o.y = pack_bf2(x[r][2], x[r][3]);
+              o.z = pack_bf2(x[r][4], x[r][5]); o.w = pack_bf2(x[r][6], x[r][7]);
+            }
             __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(blk * S + r) * p.d_sl), o);
           }
         }
@@ -576,14 +584,19 @@ int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_ac
     p.skip = wrm->skip;
   }
   const unsigned grid = (unsigned)((p.nheads + k196Heads - 1) / k196Heads);
+#define SPECTRE_TC196_LAUNCH2(JJ, WB, FH)                                                                         \
+  do {                                                                                                            \
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel<JJ, WB, FH>, cudaFuncAttributeMaxDynamicSharedMemorySize, k196Smem)); \
+    mixer_tc196_kernel<JJ, WB, FH><<<grid, kTcThreads, k196Smem, st>>>(p);                                        \
+  } while (0)
 #define SPECTRE_TC196_LAUNCH(JJ, WB)                                                                              \
   do {                                                                                                            \
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel<JJ, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, k196Smem)); \
-    mixer_tc196_kernel<JJ, WB><<<grid, kTcThreads, k196Smem, st>>>(p);                                            \
+    if (v->dtype == SPECTRE_F16) SPECTRE_TC196_LAUNCH2(JJ, WB, true); else SPECTRE_TC196_LAUNCH2(JJ, WB, false);  \
   } while (0)
   if (p.J == 2) { if (p.w_bf16) SPECTRE_TC196_LAUNCH(2, true); else SPECTRE_TC196_LAUNCH(2, false); }
   else if (p.J == 1) { if (p.w_bf16) SPECTRE_TC196_LAUNCH(1, true); else SPECTRE_TC196_LAUNCH(1, false); }
   else SPECTRE_TC196_LAUNCH(0, false);
+#undef SPECTRE_TC196_LAUNCH2
 #undef SPECTRE_TC196_LAUNCH
   SPECTRE_LAUNCH_OK("mixer_tc196_kernel");
   return SPECTRE_OK;

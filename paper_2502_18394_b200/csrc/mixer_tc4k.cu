@@ -1,4 +1,4 @@
-// Tensor-core spectral mixer for n = 4096 * R, R in {1, 2, 4, 8, 16, 32}, bf16 I/O
+// Tensor-core spectral mixer for n = 4096 * R, R in {1, 2, 4, 8, 16, 32}, bf16 or fp16 I/O
 // (Sec. 3.2 steps 2 and 4; covers n = 4096 ... 131072).
 //
 // Four-step split n = R * 4096 with t = n1 * 4096 + t', k = k1 + R * kM:
@@ -102,7 +102,7 @@ struct TcInParams {
 // CTA = (slab, group of 4 consecutive t1, block of NT2 values of t2); t' = 64 t1 + t2.
 // A warp takes one (t1, t2) at a time with lane = column pair; staging holds, for every
 // (k1, tile), the core matrices (8 operand columns x 16 bytes) of this CTA's slice.
-template <int R>
+template <int R, bool F16>
 __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
 #pragma unroll
       for (int n1 = 0; n1 < R; ++n1) {
         const uint32_t v = n1 < nvalid ? __ldg(pl + n1 * lstride) : 0u;
-        x[n1] = make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+        x[n1] = F16 ? h2unpack(v) : make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
       }
       Dft<R, false>::run(x);
       const float2 w1 = tws[rs];
@@ -467,7 +467,7 @@ struct TcOutParams {
 };
 
 // CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.
-template <int R>
+template <int R, bool F16>
 __global__ void __launch_bounds__(256, 2) tc_out_kernel(const TcOutParams p) {
   constexpr int NT = 512 / R;
   extern __shared__ __align__(128) uint32_t stage[];            // [R][NT][D/2 words]
@@ -512,8 +512,12 @@ __global__ void __launch_bounds__(256, 2) tc_out_kernel(const TcOutParams p) {
     uint32_t* ps = stage + tl * npair + word;
 #pragma unroll
     for (int n1 = 0; n1 < R; ++n1) {
-      __nv_bfloat162 o = __floats2bfloat162_rn(x[n1].x, x[n1].y);
-      ps[n1 * NT * npair] = *reinterpret_cast<uint32_t*>(&o);
+      if (F16) {
+        ps[n1 * NT * npair] = h2pack(x[n1].x, x[n1].y);
+      } else {
+        __nv_bfloat162 o = __floats2bfloat162_rn(x[n1].x, x[n1].y);
+        ps[n1 * NT * npair] = *reinterpret_cast<uint32_t*>(&o);
+      }
     }
   }
   __syncthreads();
@@ -557,7 +561,7 @@ size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
   return g * per;
 }
 
-template <int R>
+template <int R, bool F16>
 static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                       const spectre_act* y, int n, int slab0, int cnt, unsigned char* ws) {
   const int D = v->D, ntile = D / 8;
@@ -576,8 +580,8 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
                    v->H, D, v->L, n, ntile, slab0};
   const size_t smem_in = (size_t)R * ntile * (NT2 / 2) * 128;
   if (smem_in > 48 * 1024)
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_in));
-  tc_in_kernel<R><<<cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip);
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in_kernel<R, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_in));
+  tc_in_kernel<R, F16><<<cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip);
   SPECTRE_LAUNCH_OK("tc_in_kernel");
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
@@ -593,8 +597,8 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
                     y->H, D, y->L, n, ntile, slab0};
   const size_t smem_out = (size_t)R * NT * (D / 2) * 4;
   if (smem_out > 48 * 1024)
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_out));
-  tc_out_kernel<R><<<cnt * (4096 / NT), 256, smem_out, st>>>(op);
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel<R, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_out));
+  tc_out_kernel<R, F16><<<cnt * (4096 / NT), 256, smem_out, st>>>(op);
   SPECTRE_LAUNCH_OK("tc_out_kernel");
   return SPECTRE_OK;
 }
@@ -611,15 +615,18 @@ int launch_mixer_tc4k(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   for (int s0 = 0; s0 < nslab; s0 += group) {
     const int cnt = nslab - s0 < group ? nslab - s0 : group;
     int rc;
+    const bool f16 = v->dtype == SPECTRE_F16;              // 16-bit activations: bf16 or fp16 (same kernels, other unpack / pack)
+#define SPECTRE_TC4K_GROUP(RR) (f16 ? tc4k_group<RR, true>(ctx, st, v, g, y, n, s0, cnt, w) : tc4k_group<RR, false>(ctx, st, v, g, y, n, s0, cnt, w))
     switch (R) {
-      case 1: rc = tc4k_group<1>(ctx, st, v, g, y, n, s0, cnt, w); break;
-      case 2: rc = tc4k_group<2>(ctx, st, v, g, y, n, s0, cnt, w); break;
-      case 4: rc = tc4k_group<4>(ctx, st, v, g, y, n, s0, cnt, w); break;
-      case 8: rc = tc4k_group<8>(ctx, st, v, g, y, n, s0, cnt, w); break;
-      case 16: rc = tc4k_group<16>(ctx, st, v, g, y, n, s0, cnt, w); break;
-      case 32: rc = tc4k_group<32>(ctx, st, v, g, y, n, s0, cnt, w); break;
+      case 1: rc = SPECTRE_TC4K_GROUP(1); break;
+      case 2: rc = SPECTRE_TC4K_GROUP(2); break;
+      case 4: rc = SPECTRE_TC4K_GROUP(4); break;
+      case 8: rc = SPECTRE_TC4K_GROUP(8); break;
+      case 16: rc = SPECTRE_TC4K_GROUP(16); break;
+      case 32: rc = SPECTRE_TC4K_GROUP(32); break;
       default: return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported by the tensor-core path");
     }
+#undef SPECTRE_TC4K_GROUP
     if (rc != SPECTRE_OK) return rc;
   }
   return SPECTRE_OK;

@@ -1,4 +1,4 @@
-// Tensor-core spectral mixer for n = 8192, bf16 I/O (Sec. 3.2 steps 2 and 4), one kernel.
+// Tensor-core spectral mixer for n = 8192, bf16 or fp16 I/O (Sec. 3.2 steps 2 and 4), one kernel.
 //
 // The length-8192 complex transform of a column pair z = a + jb (see mixer.cu for the pair
 // packing) is factored 8192 = 2 * 64 * 64.  The radix-2 step runs on the ALUs (even / odd output
@@ -87,6 +87,11 @@ __device__ __forceinline__ void tma_store_rows(const CUtensorMap* tm, int col, i
                :: "l"(tm), "r"(col), "r"(t1), "r"(t2), "r"(h), "r"(b), "r"(src) : "memory");
 }
 
+// four output values in the activation dtype (bf16 or fp16)
+template <bool F16> __device__ __forceinline__ uint2 pack_io4(float a, float b, float c, float d) {
+  return F16 ? make_uint2(pack_h2(a, b), pack_h2(c, d)) : pack_bf16x4(a, b, c, d);
+}
+
 // Epilogue after a stage whose accumulator has columns 64 c + d (d = the digit still to be
 // contracted), for one warp: TMEM lane quadrant q, pair c.  A thread owns rows (new digit)
 // 16 q' + T/4 for the two lane groups q' = 2q, 2q+1 and the columns d = 32 chunk + 8 x + 2 (T%4)
@@ -159,6 +164,7 @@ __device__ __forceinline__ void epilogue_gate(uint32_t tmem_d, unsigned char* Bo
   }
 }
 
+template <bool F16>
 __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid_constant__ CUtensorMap tm_in,
                                                                     const __grid_constant__ CUtensorMap tm_out,
                                                                     const Tc8kParams p) {
@@ -297,7 +303,7 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
           for (int u = 0; u < 4; ++u) {
             const uint32_t ua = c == 0 ? ra[u].x : (c == 1 ? ra[u].y : (c == 2 ? ra[u].z : ra[u].w));
             const uint32_t ub = c == 0 ? rb[u].x : (c == 1 ? rb[u].y : (c == 2 ? rb[u].z : rb[u].w));
-            const float2 va = unpack_bf2(ua), vb = unpack_bf2(ub);
+            const float2 va = F16 ? unpack_h2(ua) : unpack_bf2(ua), vb = F16 ? unpack_h2(ub) : unpack_bf2(ub);
             const float2 ve = cadd(va, vb), vo = cmul(csub(va, vb), w[u]);
             e[u] = pack_h2(ve.x, ve.y);
             o[u] = pack_h2(vo.x, vo.y);
@@ -370,9 +376,9 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
           const float2 o1 = cmul(make_float2(__uint_as_float(xo[4 * x + 1]), __uint_as_float(xo[4 * x + 3])), w);
           if (x < 3) w = cmul(w, wstep);
           *reinterpret_cast<uint2*>(Bsm[0] + base + 2048 * x) =
-              pack_bf16x4(gs * (e0.x + o0.x), -gs * (e0.y + o0.y), gs * (e1.x + o1.x), -gs * (e1.y + o1.y));
+              pack_io4<F16>(gs * (e0.x + o0.x), -gs * (e0.y + o0.y), gs * (e1.x + o1.x), -gs * (e1.y + o1.y));
           *reinterpret_cast<uint2*>(Bsm[1] + base + 2048 * x) =
-              pack_bf16x4(gs * (e0.x - o0.x), -gs * (e0.y - o0.y), gs * (e1.x - o1.x), -gs * (e1.y - o1.y));
+              pack_io4<F16>(gs * (e0.x - o0.x), -gs * (e0.y - o0.y), gs * (e1.x - o1.x), -gs * (e1.y - o1.y));
         }
         if (j == 1) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -437,7 +443,7 @@ static int make_row_map(CUtensorMap* tm, const spectre_act* a, bool t1_fastest, 
   }
   cuuint32_t box[5] = {8, box1, box2, 1, 1};
   cuuint32_t es[5] = {1, 1, 1, 1, 1};
-  CUresult r = encode_tiled_fn()(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr, dims, strides, box, es,
+  CUresult r = encode_tiled_fn()(tm, a->dtype == SPECTRE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr, dims, strides, box, es,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
@@ -458,9 +464,14 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
   p.tw64 = reinterpret_cast<const float4*>(ctx->tw64x64);
   p.H = v->H; p.ntile = v->D / 8;
   p.status = ctx->status_dev;
-  SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k8Smem));
   const unsigned grid = (unsigned)((size_t)v->B * v->H * p.ntile);
-  mixer_tc8192_kernel<<<grid, k8Threads, k8Smem, st>>>(tm_in, tm_out, p);
+  if (v->dtype == SPECTRE_F16) {
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k8Smem));
+    mixer_tc8192_kernel<true><<<grid, k8Threads, k8Smem, st>>>(tm_in, tm_out, p);
+  } else {
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k8Smem));
+    mixer_tc8192_kernel<false><<<grid, k8Threads, k8Smem, st>>>(tm_in, tm_out, p);
+  }
   SPECTRE_LAUNCH_OK("mixer_tc8192_kernel");
   return SPECTRE_OK;
 }

@@ -575,6 +575,21 @@ def test_mixer_fp16_io(ctx, n, L, D):
     ctx.poll_status()
 
 
+def test_fp16_io_196_with_refinement(ctx):
+    # ViT shape in fp16: tensor-core mixer with the refinement in its store phase
+    w = W.Workload("t", B=3, L=196, H=3, D=64, dtype="f16", wdtype="bf16", n_fft=196, seed=17, wavelet_levels=2)
+    x = W.activations(w)
+    g = W.random_gate(w)
+    wp = W.wavelet_params(w)
+    qbar = torch.randn(3, 3, 64, generator=torch.Generator().manual_seed(2))
+    y = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=196, wrm=dict(to_dev(wp), qbar=qbar.cuda()))
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    s = O.wavelet_level_gates(W.to_f64(qbar), W.to_f64(wp["Ww1"]), W.to_f64(wp["bw1"]), W.to_f64(wp["Ww2"]), W.to_f64(wp["bw2"]), 2)
+    ref = O.wavelet_refine(O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=196), s, 2)
+    assert slab_err(W.to_f64(y), ref) < TOL["f16"]
+
+
 def test_fp16_io_gate_wavelet_cache_decode_backward(ctx):
     N, L, B, H, D = 256, 200, 2, 2, 16
     w = W.Workload("t", B=B, L=L, H=H, D=D, dtype="f16", wdtype="f32", n_fft=N, seed=99, N_max=N, wavelet_levels=2)
