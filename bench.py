@@ -41,7 +41,9 @@ L2_BYTES = 126e6
 #     dirty in L2 when the launch ended, so this understates the traffic; nothing is re-read)
 # c3: the four kernels of one staged mixer call at full size (intermediates spill from L2)
 # c4: append_spectrum_kernel measured at B = 2 (1015.3 MB), scaled by 4 to B = 8
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": 36.9e6, "c3": 3126e6, "c4": 4061e6, "c5": None}
+# c5: mixer_tc196_kernel at full size: 82.0 MB read + 27.6 MB written by the end of the launch (the rest of
+#     the 77 MB output is still in L2 then)
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": 36.9e6, "c3": 3126e6, "c4": 4061e6, "c5": 109.6e6}
 
 
 def measured_peak():
@@ -192,8 +194,12 @@ class MixerBench:
         # gate images + transpose-in + core + transpose-out per group of heads (staged tensor-core
         # path) or strided + on-chip + strided per group (fp32 four-step path); + wavelet
         import math
+        fused_wrm = w.dtype in ("bf16", "f16") and w.n == 196 and w.D == 64 and w.wavelet_levels in (1, 2) and w.wavelet_hidden <= 256
         if w.dtype in ("bf16", "f16") and w.n == 8192:
             self.kernel_name, nk = "mixer_tc8192_kernel (single-kernel tcgen05 mixer)", 1
+        elif w.dtype in ("bf16", "f16") and w.n == 196 and w.D == 64:
+            # level gates of the fused refinement (own small kernel) + the persistent mixer kernel
+            self.kernel_name, nk = "mixer_tc196_kernel (single-kernel tcgen05 mixer, refinement in the store phase) + level_gates_kernel", (2 if fused_wrm else 1)
         elif w.dtype in ("bf16", "f16") and ws_mix and w.n >= 4096:
             R, ntile = w.n // 4096, w.D // 8
             per = R * ntile * (32 * 2064 + 65536) + R * 18432 + 256
@@ -206,7 +212,6 @@ class MixerBench:
         else:
             self.kernel_name, nk = "mixer (onchip_kernel)", 1
         # pool, gate_out (+ gate_hidden when a head's bins span >= 32 CTAs), mixer kernels, wavelet
-        fused_wrm = w.dtype in ("bf16", "f16") and w.n == 196 and w.D == 64 and w.wavelet_levels in (1, 2) and w.wavelet_hidden <= 256
         self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels and not fused_wrm else 0)
         self.h2d = w.B * w.L * w.H * w.D * (4 if w.dtype == "f32" else 2)
         self.d2h = self.h2d

@@ -186,15 +186,21 @@ typedef struct {
  * spectre_mixer_forward - Y = R_n^{-1}( diag(g) R_n(V) ) per (batch, head)
  * (Sec. 3.2 steps 2 and 4, Eq. 1, 3, 4); heads are written side by side in
  * [B, L, H, D], which is the concatenation of step 4.
- *   v, y     activations of identical shape and dtype; y may alias v only when
- *            spectre_mixer_workspace_bytes(...) == 0 (single-pass path)
+ *   v, y     activations of identical shape and dtype; y may alias v where the
+ *            transform is one kernel (the workspace query returns 0, and the
+ *            bf16 / fp16 tensor-core paths n_fft = 196 with D = 64 and
+ *            n_fft = 8192); on a multi-pass path an aliased call is refused
+ *            with SPECTRE_ERR_INVALID_ARG
  *   g        [B, H, K, 2] float32, K = n_fft/2 + 1; one gain per bin per head,
  *            applied to all D columns; Im of the DC / Nyquist gains is ignored
  *   n_fft    == L: exact circular transform of Eq. 1;  > L: rows L..n_fft-1 are
  *            zero (the pad(.) of Sec. 3.3.1) and only rows 0..L-1 are written
  *   wrm      NULL, or the wavelet refinement applied to Y afterwards (Sec. 3.5)
  *   workspace  >= spectre_mixer_workspace_bytes(...) bytes, 16-byte aligned
- *              (0 bytes / NULL allowed when the query returns 0)
+ *              (0 bytes / NULL allowed when the query returns 0).  For bf16 / fp16,
+ *              n_fft = 196, D = 64 the workspace only holds the level gates that
+ *              wrm's MLP produces for the refinement fused into the mixer kernel
+ *              (B H 3 D floats): with less, the refinement runs as its own kernel
  */
 size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t L, int32_t H,
                                      int32_t D, int32_t n_fft, int32_t dtype);

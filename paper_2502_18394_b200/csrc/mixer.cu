@@ -31,8 +31,9 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
                         const spectre_act* y);   // mixer_tc.cu
 bool tc8192_supported(const spectre_act* v, const spectre_act* y);                     // mixer_tc8k.cu
 int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
-                       const spectre_act* y, const spectre_wavelet* wrm);
+                       const spectre_act* y, const spectre_wavelet* wrm, float* level_gate_scratch);
 bool tc196_fuses_wavelet(const spectre_wavelet* w);
+size_t tc196_level_gate_bytes(int B, int H);
 
 bool tc4k_supported(int n, int D);                                                     // mixer_tc4k.cu
 size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
@@ -700,6 +701,8 @@ extern "C" size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t 
   if ((dtype == SPECTRE_BF16 || dtype == SPECTRE_F16) && ctx->dft64 && tc4k_supported(n_fft, D) && force != kPathAlu && force != kPathFused &&
       (n_fft != 8192 || force == kPathStaged))               // n = 8192 defaults to the single-kernel path
     return tc4k_workspace_bytes(ctx, n_fft, D, B * H);
+  if ((dtype == SPECTRE_BF16 || dtype == SPECTRE_F16) && n_fft == 196 && D == 64 && ctx->dft49 && force != kPathAlu)
+    return tc196_level_gate_bytes(B, H);                     // level gates of a fused refinement
   if (pl.N1 == 1) return 0;
   return (size_t)preferred_group(ctx, n_fft, D, B * H) * slab_ws_bytes(n_fft, D);
 }
@@ -740,11 +743,13 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (staged || fused || tc196) {
     // n = 196: the refinement rides in the kernel's store phase when it can
+    // (level gates given, 8-byte aligned; or the MLP's weights and room for its output in the workspace)
     const bool fuse_wrm = tc196 && wrm && tc196_fuses_wavelet(wrm) &&
-                          (wrm->level_gates || (wrm->qbar && wrm->Ww1 && wrm->bw1 && wrm->Ww2 && wrm->bw2 &&
-                                                !((reinterpret_cast<uintptr_t>(wrm->Ww1) | reinterpret_cast<uintptr_t>(wrm->Ww2) | reinterpret_cast<uintptr_t>(wrm->bw2)) & 7) &&
-                                                (wrm->wdtype == SPECTRE_F32 || wrm->wdtype == SPECTRE_BF16)));
-    rc = tc196 ? launch_mixer_tc196(ctx, st, v, g, y, fuse_wrm ? wrm : nullptr)
+                          (wrm->level_gates ? !(reinterpret_cast<uintptr_t>(wrm->level_gates) & 7)
+                                            : (wrm->qbar && wrm->Ww1 && wrm->bw1 && wrm->Ww2 && wrm->bw2 &&
+                                               (wrm->wdtype == SPECTRE_F32 || wrm->wdtype == SPECTRE_BF16) && ws_ok &&
+                                               workspace_bytes >= tc196_level_gate_bytes(v->B, v->H)));
+    rc = tc196 ? launch_mixer_tc196(ctx, st, v, g, y, fuse_wrm ? wrm : nullptr, reinterpret_cast<float*>(workspace))
                : (staged ? launch_mixer_tc4k(ctx, st, v, g, y, n_fft, workspace, workspace_bytes)
                          : launch_mixer_tc8192(ctx, st, v, g, y));
     if (rc != SPECTRE_OK) return rc;

@@ -94,11 +94,11 @@ int build_dft64(__half* F, cudaStream_t st) {
 // A CTA takes 4 heads: columns (head, k1, pair) = 4 x 4 x 32 = 512 = the whole TMEM; the two
 // 2-head halves ping-pong between tensor core and ALUs like the halves of the 8192 kernel.
 // =====================================================================================
-constexpr int k196Heads = 4;
+constexpr int k196Heads = 2;                  // heads per CTA the launcher uses: two CTAs per SM (4 per CTA measured slower)
 constexpr int k196KSteps = 7;                 // K = 112 >= 98
 constexpr int k196WHidden = 256;              // widest level-gate MLP the fused refinement handles
 constexpr int k196StageRow = 160;             // bytes per staged output row (128 + pad against bank conflicts)
-constexpr int k196Smem = kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4 + 64 + k196Heads * (k196WHidden + 3 * 64) * 4;
+constexpr int k196_smem(int NH) { return kTcFBytes + (NH / 2) * kTcBBytes + NH * 256 * 4 + 64 + NH * 3 * 64 * 4; }
 static_assert(2 * 196 * k196StageRow <= kTcBBytes, "staged rows of two heads fit one operand buffer");
 
 struct Tc196Params {
@@ -107,65 +107,153 @@ struct Tc196Params {
   int64_t s_sb, s_sl, s_sh, d_sb, d_sl, d_sh;
   const float2* g;        // [B*H][99]
   const __half* F;        // 49-point DFT matrix (real form, padded), canonical smem layout
-  int H, L, nheads;       // nheads = B * H
+  int H, L, B;
   int* status;
   // wavelet refinement fused into the store (Sec. 3.5), J = 0: off
-  int J, whidden, w_bf16;
-  const float* level_gates;       // [B,H,J+1,64] or NULL
-  const float* qbar; const void* Ww1; const float* bw1; const void* Ww2; const float* bw2;
-  size_t hs_w1, hs_b1, hs_w2, hs_b2;
+  int J;
+  const float* level_gates;       // [B,H,J+1,64]
   const int* skip;                // [B] or NULL: non-zero = no refinement for this batch entry
 };
 
-template <bool WBF> __device__ __forceinline__ float wload_rt(const void* w, size_t i) {
-  return WBF ? __bfloat162float(reinterpret_cast<const bf16*>(w)[i]) : __ldg(reinterpret_cast<const float*>(w) + i);
-}
-// two adjacent weights (i even), kept raw until used
-template <bool WBF> struct wpair;
-template <> struct wpair<true> {
-  typedef unsigned raw;
-  static __device__ __forceinline__ raw load(const void* w, size_t i) { return __ldg(reinterpret_cast<const unsigned*>(reinterpret_cast<const bf16*>(w) + i)); }
-  static __device__ __forceinline__ float2 cvt(raw r) { return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u)); }
-};
-template <> struct wpair<false> {
-  typedef float2 raw;
-  static __device__ __forceinline__ raw load(const void* w, size_t i) { return __ldg(reinterpret_cast<const float2*>(reinterpret_cast<const float*>(w) + i)); }
-  static __device__ __forceinline__ float2 cvt(raw r) { return r; }
+// Level gates of the refinement (Sec. 3.5 step b): s = GELU(q_bar Ww1 + bw1) Ww2 + bw2, [B,H,NG] with
+// NG = (J + 1) 64.  A CTA takes kLgBatch batch entries of one head index, so each weight is fetched
+// once per kLgBatch entries.  Hidden layer: an item is one hidden unit x a quarter of the 64 inputs
+// (partial sums meet in shared memory); output layer: a thread owns one output.  The first item's
+// weights and the first 32 rows of W2 are requested together at the start; three CTAs fit an SM, so
+// the grid of a ViT-sized batch is resident at once.  The mixer kernel launched next may start while this one runs.
+constexpr int kLgBatch = 8;
+struct LevelGateParams {
+  const float* qbar; const void* Ww1; const float* bw1; const void* Ww2; const float* bw2;
+  size_t hs_w1, hs_b1, hs_w2, hs_b2;     // per-head strides in elements (0: shared across heads)
+  float* out;
+  int B, H, hidden, NG;
 };
 
-template <int J, bool WBF, bool F16>
-__global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196Params p) {
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(bf16 x) { return __bfloat162float(x); }
+
+template <typename WT>
+__global__ void __launch_bounds__(256, 3) level_gates_kernel(const LevelGateParams p) {
+  __shared__ __align__(16) float qs[kLgBatch][64];
+  extern __shared__ float part_raw[];                        // [4][kLgBatch][hidden]: hidden-layer partial sums per input quarter
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int tid = threadIdx.x, h = blockIdx.x, b0 = blockIdx.y * kLgBatch;
+  const WT* W1 = reinterpret_cast<const WT*>(p.Ww1) + h * p.hs_w1;
+  const WT* W2 = reinterpret_cast<const WT*>(p.Ww2) + h * p.hs_w2;
+  const int nitems = 4 * p.hidden;
+  float qv[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int e = tid + 256 * i, b = b0 + (e >> 6);
+    qv[i] = b < p.B ? p.qbar[((size_t)b * p.H + h) * 64 + (e & 63)] : 0.f;
+  }
+  WT w1[16], w2[32];
+  {
+    const int it = min(tid, nitems - 1), jj = it % p.hidden, cq = it / p.hidden;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) w1[c] = W1[(size_t)(16 * cq + c) * p.hidden + jj];
+  }
+  const int ii = min(tid, p.NG - 1);
+#pragma unroll
+  for (int u = 0; u < 32; ++u) w2[u] = W2[(size_t)min(u, p.hidden - 1) * p.NG + ii];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) qs[(tid + 256 * i) >> 6][(tid + 256 * i) & 63] = qv[i];
+  __syncthreads();
+  for (int it = tid; it < nitems; it += 256) {
+    const int jj = it % p.hidden, cq = it / p.hidden;
+    if (it != tid) {
+#pragma unroll
+      for (int c = 0; c < 16; ++c) w1[c] = W1[(size_t)(16 * cq + c) * p.hidden + jj];
+    }
+    float acc[kLgBatch];
+#pragma unroll
+    for (int e = 0; e < kLgBatch; ++e) acc[e] = 0.f;
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) {
+#pragma unroll
+      for (int e = 0; e < kLgBatch; ++e) {
+        const float4 q4 = *reinterpret_cast<const float4*>(&qs[e][16 * cq + 4 * c4]);
+        acc[e] = fmaf(q4.x, to_float(w1[4 * c4]), acc[e]);
+        acc[e] = fmaf(q4.y, to_float(w1[4 * c4 + 1]), acc[e]);
+        acc[e] = fmaf(q4.z, to_float(w1[4 * c4 + 2]), acc[e]);
+        acc[e] = fmaf(q4.w, to_float(w1[4 * c4 + 3]), acc[e]);
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < kLgBatch; ++e) part_raw[(cq * kLgBatch + e) * p.hidden + jj] = acc[e];
+  }
+  __syncthreads();
+  for (int i = tid; i < kLgBatch * p.hidden; i += 256) {       // u = GELU(sum of the quarters + bias), kept in part[0]
+    const int e = i / p.hidden, jj = i - e * p.hidden;
+    const int st = kLgBatch * p.hidden;
+    part_raw[i] = gelu_erf(p.bw1[h * p.hs_b1 + jj] + ((part_raw[i] + part_raw[st + i]) + (part_raw[2 * st + i] + part_raw[3 * st + i])));
+  }
+  __syncthreads();
+  if (tid < p.NG) {
+    float acc[kLgBatch];
+    const float b2 = p.bw2[h * p.hs_b2 + ii];
+#pragma unroll
+    for (int e = 0; e < kLgBatch; ++e) acc[e] = b2;
+    for (int j0 = 0; j0 < p.hidden; j0 += 32) {
+      if (j0 > 0) {
+#pragma unroll
+        for (int u = 0; u < 32; ++u) w2[u] = W2[(size_t)min(j0 + u, p.hidden - 1) * p.NG + ii];
+      }
+#pragma unroll
+      for (int u = 0; u < 32; ++u) {
+        if (j0 + u < p.hidden) {
+          const float wv = to_float(w2[u]);
+#pragma unroll
+          for (int e = 0; e < kLgBatch; ++e) acc[e] = fmaf(part_raw[e * p.hidden + j0 + u], wv, acc[e]);
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < kLgBatch; ++e)
+      if (b0 + e < p.B) p.out[((size_t)(b0 + e) * p.H + h) * p.NG + ii] = acc[e];
+  }
+}
+
+// NH heads per CTA (2 or 4): NH / 2 operand buffers and accumulators of 256 columns, 4 NH epilogue
+// warps + the issuing warp.  With NH = 2 two CTAs share an SM, so one CTA's loads and weight fetches
+// run under the other's arithmetic.
+template <int NH, int J, bool F16>
+__global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_kernel(const Tc196Params p) {
+  constexpr int NHALF = NH / 2, EW = 4 * NH, ET = 32 * EW;        // halves, epilogue warps and threads
+  constexpr int HPI = NH / 2;                                     // heads per gate-table pass
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* Fsm = smem;
-  unsigned char* Bsm[2] = {smem + kTcFBytes, smem + kTcFBytes + kTcBBytes};
-  uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + kTcFBytes + 2 * kTcBBytes);        // [4 heads][k1 * 64 + kM]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4);
-  float* wu = reinterpret_cast<float*>(smem + kTcFBytes + 2 * kTcBBytes + k196Heads * 256 * 4 + 64);   // [4][k196WHidden]
-  float* wsg = wu + k196Heads * k196WHidden;                                                         // [4][3][64] holds 1 + s
+  unsigned char* Bsm[2] = {smem + kTcFBytes, smem + kTcFBytes + (NHALF - 1) * kTcBBytes};
+  uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + kTcFBytes + NHALF * kTcBBytes);        // [NH heads][k1 * 64 + kM]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTcFBytes + NHALF * kTcBBytes + NH * 256 * 4);
+  float* wsg = reinterpret_cast<float*>(smem + kTcFBytes + NHALF * kTcBBytes + NH * 256 * 4 + 64);  // [NH][3][64] holds 1 + s
   __shared__ uint32_t tmem_slot;
-  __shared__ float red[kTcEpiWarps];
-  __shared__ float gmax_s[k196Heads];
+  __shared__ float red[2 * EW];
+  __shared__ float gmax_s[NH];
+
+  __shared__ int abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
-  const int head0 = blockIdx.x * k196Heads;
+  const int nwork = p.H * ((p.B + NH - 1) / NH);     // work items: NH batch entries of one head index
   TC_STAMP(0);
 
-  if (warp == kTcEpiWarps) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(512));
+  if (warp == EW) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(256 * NHALF));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[0])), "r"(kTcEpiThreads));
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[1])), "r"(kTcEpiThreads));
+    abort_s = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[0])), "r"(ET));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[1])), "r"(ET));
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[2])), "r"(1));
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bars[3])), "r"(1));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (tid < kTcEpiThreads) {
+  if (tid < ET) {
     const uint4* Fg = reinterpret_cast<const uint4*>(p.F);
-    for (int i = tid; i < kTcFBytes / 16; i += kTcEpiThreads) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
+    for (int i = tid; i < kTcFBytes / 16; i += ET) reinterpret_cast<uint4*>(Fsm)[i] = __ldg(Fg + i);
     // zero the operands once: K rows 98..127 and the columns of absent heads must read as zero
-    for (int i = tid; i < 2 * kTcBBytes / 16; i += kTcEpiThreads) reinterpret_cast<uint4*>(Bsm[0])[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < NHALF * kTcBBytes / 16; i += ET) reinterpret_cast<uint4*>(Bsm[0])[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -174,12 +262,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
   const uint32_t tmem = tmem_slot;
   TC_STAMP(1);
 
-  if (warp == kTcEpiWarps) {
-    // ---- MMA issuer: 2 stages x 2 halves, 7 K-steps each ----
+  if (warp == EW) {
+    // ---- MMA issuer: per work item 2 stages x NH / 2 halves, 7 K-steps each ----
     const uint32_t idesc = umma_idesc_128x256();
     bool ok = true;
+    for (int work = blockIdx.x; work < nwork && ok; work += gridDim.x)
     for (int stage = 0; stage < 2 && ok; ++stage) {
-      for (int half = 0; half < 2 && ok; ++half) {
+      for (int half = 0; half < NHALF && ok; ++half) {
         ok = mbar_wait(smem_u32(&bars[half]), stage & 1);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -202,19 +291,44 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
     }
     if (!ok && T == 0) atomicExch(p.status, 1);
   } else {
+    // The CTA keeps its DFT matrix, accumulators and barriers over all its work items: the barriers
+    // complete two phases per item, so every item sees the same parities.
+    bool ok = true;
+#pragma unroll 1
+    for (int work = blockIdx.x; work < nwork; work += gridDim.x) {
+    // the item's heads are batch entries bg NH .. bg NH + NH - 1 of ONE head index hh: they share the
+    // level-gate weights, and neighbouring items read neighbouring 128-byte pieces of the same rows
+    const int hh = work % p.H, bg = work / p.H;
+    // per-thread indices re-derived from an opaque copy, so that the compiler keeps the item's index
+    // arithmetic and twiddles inside the loop instead of carrying them in registers across items
+    int tid_item = threadIdx.x;
+    asm volatile("" : "+r"(tid_item));
+    const int tid = tid_item, warp = tid >> 5, T = tid & 31;
+    if (J > 0 && work != (int)blockIdx.x) {
+      // the staged rows of the previous item covered K rows 98..111, which the MMA reads as zero padding:
+      // clear them again (bytes 4..15 of slot 12's rows, all of slot 13; the loads below write the rest)
+#pragma unroll
+      for (int half = 0; half < NHALF; ++half) {
+        for (int idx = tid; idx < 32 * 8; idx += ET) {               // (group of 8 columns, column)
+          unsigned char* z = Bsm[half] + (idx >> 3) * kTcSbo + 12 * kTcLbo + (idx & 7) * 16;
+          *reinterpret_cast<uint32_t*>(z + 4) = 0u;
+          *reinterpret_cast<uint2*>(z + 8) = make_uint2(0u, 0u);
+          *reinterpret_cast<uint4*>(z + kTcLbo) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    }
     // ---- load: rows t' + 49 n1 of each head, radix-4 over n1, twiddle, fp16, operand (K = t', column = (head, k1, pair)) ----
     // a warp takes 4 consecutive t' x 8 chunks of 16 bytes (conflict-free operand stores); all of
     // a warp's rows (up to 4 items x 4 rows) are requested before the first one is used
-    constexpr int kItems = (k196Heads * 13 + kTcEpiWarps - 1) / kTcEpiWarps;
+    constexpr int kItems = (NH * 13 + EW - 1) / EW;
     uint4 rr[kItems][4];
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
-      const int item = warp + it * kTcEpiWarps;
+      const int item = warp + it * EW;
       const int hl = item / 13, tg = item - hl * 13;
-      const int tp = 4 * tg + (T >> 3), hg = head0 + hl;
-      const bool live = item < k196Heads * 13 && tp < 49 && hg < p.nheads;
-      const int b = live ? hg / p.H : 0, h = live ? hg - b * p.H : 0;
-      const bf16* src = p.src + b * p.s_sb + h * p.s_sh + 8 * (T & 7);
+      const int tp = 4 * tg + (T >> 3), b = bg * NH + hl;
+      const bool live = item < NH * 13 && tp < 49 && b < p.B;
+      const bf16* src = p.src + (live ? b : 0) * p.s_sb + hh * p.s_sh + 8 * (T & 7);
 #pragma unroll
       for (int n1 = 0; n1 < 4; ++n1) {
         const int row = tp + 49 * n1;
@@ -224,10 +338,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
     }
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
-      const int item = warp + it * kTcEpiWarps;
+      const int item = warp + it * EW;
       const int hl = item / 13, tg = item - hl * 13;
-      const int tp = 4 * tg + (T >> 3), chunk = T & 7, hg = head0 + hl;
-      if (item >= k196Heads * 13 || tp >= 49 || hg >= p.nheads) continue;
+      const int tp = 4 * tg + (T >> 3), chunk = T & 7;
+      if (item >= NH * 13 || tp >= 49 || bg * NH + hl >= p.B) continue;
       const float2 w1 = twiddle_fwd((unsigned)tp, 196u);
       const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
       unsigned char* Bh = Bsm[hl >> 1] + b_off((hl & 1) * 128 + 4 * chunk, 2 * tp);
@@ -251,21 +365,34 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");     // the previous item's accumulator reads are done
     TC_STAMP(2);
     mbar_arrive(smem_u32(&bars[0]));
-    mbar_arrive(smem_u32(&bars[1]));
+    if (NHALF == 2) mbar_arrive(smem_u32(&bars[1]));
+
+    // ---- level gates of the refinement (Sec. 3.5 step b), [B,H,J+1,64]: requested here, used after the gate
+    //      tables.  They may come from the kernel launched just before this one (programmatic dependent
+    //      launch): griddepcontrol.wait returns once that grid's writes are visible ----
+    constexpr int NG = (J + 1) * 64;
+    float2 lgv = make_float2(0.f, 0.f);
+    const int lg_hl = tid / (NG / 2), lg_i = 2 * (tid % (NG / 2));
+    if (J > 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (lg_hl < NH && bg * NH + lg_hl < p.B)
+        lgv = *reinterpret_cast<const float2*>(p.level_gates + ((size_t)(bg * NH + lg_hl) * p.H + hh) * NG + lg_i);
+    }
 
     // ---- gate tables: head hl, entry k1 * 64 + kM holds G_ext[k1 + 4 kM] / gmax(head) as fp16 ----
     float2 gv[2];
     float gm[2];
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
-      const int e = tid + it * kTcEpiThreads, hl = e >> 8, idx = e & 255, k1 = idx >> 6, kM = idx & 63;
-      const int hg = head0 + hl;
+      const int e = tid + it * ET, hl = e >> 8, idx = e & 255, k1 = idx >> 6, kM = idx & 63;
+      const int b = bg * NH + hl;
       float2 v = make_float2(0.f, 0.f);
-      if (kM < 49 && hg < p.nheads) {
+      if (kM < 49 && b < p.B) {
         const int k = k1 + 4 * kM, kk = k <= 98 ? k : 196 - k;
-        v = __ldg(p.g + (size_t)hg * 99 + kk);
+        v = __ldg(p.g + ((size_t)b * p.H + hh) * 99 + kk);
         if (kk != k) v.y = -v.y;
         if (k == 0 || k == 98) v.y = 0.f;
       }
@@ -274,84 +401,41 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
       gm[it] = m;
     }
-    // warps 0-7 hold head 0 (it = 0) and head 2 (it = 1); warps 8-15 heads 1 and 3
-    if (T == 0) red[warp] = gm[0];
-    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
-    if (tid < 2) { float m = 0.f; for (int i = 0; i < 8; ++i) m = fmaxf(m, red[8 * tid + i]); gmax_s[tid] = 1.41421356f * m; }
-    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
-    if (T == 0) red[warp] = gm[1];
-    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
-    if (tid < 2) { float m = 0.f; for (int i = 0; i < 8; ++i) m = fmaxf(m, red[8 * tid + i]); gmax_s[2 + tid] = 1.41421356f * m; }
-    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+    // 8 consecutive warps hold one head per pass: pass `it` covers heads HPI * it .. HPI * it + HPI - 1
+    if (T == 0) { red[warp] = gm[0]; red[EW + warp] = gm[1]; }
+    asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");
+    if (tid < NH) {                                   // head tid = HPI * it + w: warps 8 w .. 8 w + 7 of pass it
+      const int it = tid / HPI, w8 = tid - it * HPI;
+      float m = 0.f;
+      for (int i = 0; i < 8; ++i) m = fmaxf(m, red[it * EW + 8 * w8 + i]);
+      gmax_s[tid] = 1.41421356f * m;
+    }
+    asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
-      const int e = tid + it * kTcEpiThreads, hl = e >> 8;
+      const int e = tid + it * ET, hl = e >> 8;
       const float gmx = gmax_s[hl], inv = gmx > 0.f ? 1.0f / gmx : 0.f;
       Gsm[e] = pack_h2(gv[it].x * inv, gv[it].y * inv);
     }
-    if (J > 0) {
-      // level gates of the refinement: given, or s = GELU(q_bar Ww1 + bw1) Ww2 + bw2 per head (Sec. 3.5
-      // step b).  Every weight a thread needs for one output is requested before the first is used.
-      constexpr int NG = (J + 1) * 64;
-      if (!p.level_gates) {
-        for (int e = tid; e < k196Heads * p.whidden; e += kTcEpiThreads) {
-          const int hl = e / p.whidden, jj = e - hl * p.whidden, hg = head0 + hl;
-          float acc = 0.f;
-          if (hg < p.nheads) {
-            const int h = hg % p.H;
-            float wv[64];
-#pragma unroll
-            for (int c = 0; c < 64; ++c) wv[c] = wload_rt<WBF>(p.Ww1, h * p.hs_w1 + (size_t)c * p.whidden + jj);
-            acc = p.bw1[h * p.hs_b1 + jj];
-            const float* qb = p.qbar + (size_t)hg * 64;
-#pragma unroll
-            for (int c = 0; c < 64; ++c) acc = fmaf(qb[c], wv[c], acc);
-            acc = gelu_erf(acc);
-          }
-          wu[hl * k196WHidden + jj] = acc;
-        }
-        asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
-      }
-      for (int e = tid; e < k196Heads * NG / 2; e += kTcEpiThreads) {       // two adjacent outputs per thread
-        const int hl = e / (NG / 2), ii = 2 * (e - hl * (NG / 2)), hg = head0 + hl;
-        float2 sv = make_float2(0.f, 0.f);
-        if (hg < p.nheads) {
-          if (p.level_gates) {
-            sv = *reinterpret_cast<const float2*>(p.level_gates + (size_t)hg * NG + ii);
-          } else {
-            const int h = hg % p.H;
-            sv = *reinterpret_cast<const float2*>(p.bw2 + h * p.hs_b2 + ii);
-            constexpr int NB = WBF ? 64 : 32;                     // rows of W2 in flight (one register each in bf16)
-            for (int j0 = 0; j0 < p.whidden; j0 += NB) {
-              typename wpair<WBF>::raw raw[NB];
-#pragma unroll
-              for (int u = 0; u < NB; ++u)
-                raw[u] = wpair<WBF>::load(p.Ww2, h * p.hs_w2 + (size_t)min(j0 + u, p.whidden - 1) * NG + ii);
-#pragma unroll
-              for (int u = 0; u < NB; ++u) {
-                const float uu = (j0 + u < p.whidden) ? wu[hl * k196WHidden + j0 + u] : 0.f;
-                const float2 wv = wpair<WBF>::cvt(raw[u]);
-                sv.x = fmaf(uu, wv.x, sv.x);
-                sv.y = fmaf(uu, wv.y, sv.y);
-              }
-            }
-          }
-        }
-        wsg[hl * 192 + ii] = 1.0f + sv.x;
-        wsg[hl * 192 + ii + 1] = 1.0f + sv.y;
-      }
+    if (J > 0 && lg_hl < NH) {
+      wsg[lg_hl * 192 + lg_i] = 1.0f + lgv.x;
+      wsg[lg_hl * 192 + lg_i + 1] = 1.0f + lgv.y;
     }
-    asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");
 
-    const int q = warp & 3, cq = warp >> 2;
+    // a warp owns TMEM lanes 32 q .. 32 q + 31; per unit it takes 64 columns: with 4 heads unit = half and
+    // the column quarter is fixed, with 2 heads the one half's quarters 2 (warp >> 2) + unit
+    const int q = warp & 3;
     const int i = T >> 2, t4 = T & 3;
-    bool ok = true;
     TC_STAMP(3);
     // ---- gate epilogue: rows kM, columns (head, k1, pair) unchanged; next operand has K = kM ----
 #pragma unroll 1
-    for (int half = 0; half < 2 && ok; ++half) {
-      ok = mbar_wait(smem_u32(&bars[2 + half]), 0);
-      if (!ok) break;
+    for (int unit = 0; unit < 2 && ok; ++unit) {
+      const int half = NH == 4 ? unit : 0, cq = NH == 4 ? (warp >> 2) : 2 * (warp >> 2) + unit;
+      if (NH == 4 || unit == 0) {
+        ok = mbar_wait(smem_u32(&bars[2 + half]), 0);
+        if (!ok) break;
+      }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t taddr0 = tmem + 256 * half + ((uint32_t)(32 * q) << 16) + 64 * cq;
       const int hl = 2 * half + (cq >> 1);
@@ -377,18 +461,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      TC_STAMP(4 + half);
-      mbar_arrive(smem_u32(&bars[half]));
+      TC_STAMP(4 + unit);
+      if (NH == 4 || unit == 1) mbar_arrive(smem_u32(&bars[half]));
     }
     // ---- final: rows t', inverse radix-4 over k1 (columns 32 apart), bf16 rows t' + 49 n1 ----
 #pragma unroll 1
-    for (int half = 0; half < 2 && ok; ++half) {
-      ok = mbar_wait(smem_u32(&bars[2 + half]), 1);
-      if (!ok) break;
+    for (int unit = 0; unit < 2 && ok; ++unit) {
+      const int half = NH == 4 ? unit : 0, cq = NH == 4 ? (warp >> 2) : 2 * (warp >> 2) + unit;
+      if (NH == 4 || unit == 0) {
+        ok = mbar_wait(smem_u32(&bars[2 + half]), 1);
+        if (!ok) break;
+      }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int hl = 2 * half + (cq >> 1), hg = head0 + hl;
-      if (hg >= p.nheads) continue;
-      const int b = hg / p.H, h = hg - b * p.H;
+      const int hl = 2 * half + (cq >> 1), b = bg * NH + hl, h = hh;
+      if (b >= p.B) continue;
       const float gs = 0.5f * gmax_s[hl];
       bf16* dst = p.dst + b * p.d_sb + h * p.d_sh;
       const uint32_t tbase = tmem + 256 * half + ((uint32_t)(32 * q) << 16) + 128 * (cq >> 1) + 16 * (cq & 1);
@@ -441,15 +527,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       // ---- wavelet refinement on the staged bf16 rows (Sec. 3.5): Haar over aligned blocks of 2^J
       //      tokens, bands scaled by 1 + s, synthesis; a thread takes 8 channels of one block and
       //      writes whole 16-byte pieces, 8 lanes per 128-byte row ----
-      asm volatile("bar.sync 1, %0;" :: "r"(kTcEpiThreads) : "memory");
+      asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");
       if (ok) {
         constexpr int S = 1 << J;
         const float r2 = 0.70710678118654752440f;
         const int nblk = p.L / S;
-        for (int item = tid; item < k196Heads * nblk * 8; item += kTcEpiThreads) {
-          const int cch = item & 7, blk = (item >> 3) % nblk, hl = item / (8 * nblk), hg = head0 + hl;
-          if (hg >= p.nheads) continue;
-          const int b = hg / p.H, h = hg - b * p.H;
+        for (int item = tid; item < NH * nblk * 8; item += ET) {
+          const int cch = item & 7, blk = (item >> 3) % nblk, hl = item / (8 * nblk), b = bg * NH + hl, h = hh;
+          if (b >= p.B) continue;
           const unsigned char* st = Bsm[hl >> 1] + ((hl & 1) * 196 + blk * S) * k196StageRow + 16 * cch;
           if (p.skip && p.skip[b]) {                             // skipped batch entry: the mixer output as it is
             bf16* dst0 = p.dst + b * p.d_sb + h * p.d_sh + 8 * cch;
@@ -520,13 +605,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) mixer_tc196_kernel(const Tc196P
       }
     }
     TC_STAMP(7);
+    // end of the item: the staged rows and level gates are free again; a wait that ran out ends the loop for all
+    if (!ok) abort_s = 1;
+    asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");
+    if (abort_s) break;
+    }
     if (!ok && T == 0) atomicExch(p.status, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == kTcEpiWarps) {
+  if (warp == EW) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(512));
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(256 * NHALF));
   }
 }
 
@@ -562,8 +652,11 @@ bool tc196_fuses_wavelet(const spectre_wavelet* w) {
          (w->level_gates || (w->hidden >= 1 && w->hidden <= k196WHidden));
 }
 
+size_t tc196_level_gate_bytes(int B, int H) { return (size_t)B * H * 3 * 64 * sizeof(float); }
+
+// level_gate_scratch: tc196_level_gate_bytes(B, H) bytes, needed when wrm carries the MLP weights
 int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
-                       const spectre_act* y, const spectre_wavelet* wrm) {
+                       const spectre_act* y, const spectre_wavelet* wrm, float* level_gate_scratch) {
   Tc196Params p = {};
   p.src = reinterpret_cast<const bf16*>(v->ptr);
   p.dst = reinterpret_cast<bf16*>(y->ptr);
@@ -571,32 +664,53 @@ int launch_mixer_tc196(const spectre_ctx* ctx, cudaStream_t st, const spectre_ac
   p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
   p.g = reinterpret_cast<const float2*>(g);
   p.F = reinterpret_cast<const __half*>(ctx->dft49);
-  p.H = v->H; p.L = v->L; p.nheads = v->B * v->H;
+  p.H = v->H; p.L = v->L; p.B = v->B;
   p.status = ctx->status_dev;
+  bool dependent = false;            // the mixer kernel follows a kernel of ours whose output it reads
   if (wrm) {
-    const int J = wrm->levels, hid = wrm->level_gates ? 0 : wrm->hidden;
-    const size_t one = wrm->shared_across_heads ? 0 : 1;
-    p.J = J; p.whidden = hid; p.w_bf16 = wrm->wdtype == SPECTRE_BF16;
-    p.level_gates = wrm->level_gates; p.qbar = wrm->qbar;
-    p.Ww1 = wrm->Ww1; p.bw1 = wrm->bw1; p.Ww2 = wrm->Ww2; p.bw2 = wrm->bw2;
-    p.hs_w1 = one * (size_t)64 * hid; p.hs_b1 = one * hid;
-    p.hs_w2 = one * (size_t)hid * (J + 1) * 64; p.hs_b2 = one * (size_t)(J + 1) * 64;
+    const int J = wrm->levels;
+    p.J = J;
     p.skip = wrm->skip;
+    p.level_gates = wrm->level_gates;
+    if (!wrm->level_gates) {
+      LevelGateParams lp = {};
+      const int hid = wrm->hidden;
+      const size_t one = wrm->shared_across_heads ? 0 : 1;
+      lp.qbar = wrm->qbar; lp.Ww1 = wrm->Ww1; lp.bw1 = wrm->bw1; lp.Ww2 = wrm->Ww2; lp.bw2 = wrm->bw2;
+      lp.hs_w1 = one * (size_t)64 * hid; lp.hs_b1 = one * hid;
+      lp.hs_w2 = one * (size_t)hid * (J + 1) * 64; lp.hs_b2 = one * (size_t)(J + 1) * 64;
+      lp.out = level_gate_scratch;
+      lp.B = v->B; lp.H = v->H; lp.hidden = hid; lp.NG = (J + 1) * 64;
+      const dim3 lgrid((unsigned)v->H, (unsigned)((v->B + kLgBatch - 1) / kLgBatch));
+      const size_t lsmem = (size_t)4 * kLgBatch * hid * sizeof(float);       // <= 32 KB
+      if (wrm->wdtype == SPECTRE_BF16) level_gates_kernel<bf16><<<lgrid, 256, lsmem, st>>>(lp);
+      else level_gates_kernel<float><<<lgrid, 256, lsmem, st>>>(lp);
+      SPECTRE_LAUNCH_OK("level_gates_kernel");
+      p.level_gates = level_gate_scratch;
+      dependent = true;
+    }
   }
-  const unsigned grid = (unsigned)((p.nheads + k196Heads - 1) / k196Heads);
-#define SPECTRE_TC196_LAUNCH2(JJ, WB, FH)                                                                         \
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  const unsigned nwork = (unsigned)(p.H * ((p.B + k196Heads - 1) / k196Heads)), slots = 2u * (unsigned)ctx->sm_count;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(nwork < slots ? nwork : slots);        // persistent: two CTAs per SM
+  cfg.blockDim = dim3(128 * k196Heads + 32);
+  cfg.dynamicSmemBytes = k196_smem(k196Heads);
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+#define SPECTRE_TC196_LAUNCH(JJ, FH)                                                                              \
   do {                                                                                                            \
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel<JJ, WB, FH>, cudaFuncAttributeMaxDynamicSharedMemorySize, k196Smem)); \
-    mixer_tc196_kernel<JJ, WB, FH><<<grid, kTcThreads, k196Smem, st>>>(p);                                        \
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc196_kernel<k196Heads, JJ, FH>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                         k196_smem(k196Heads)));                                                  \
+    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, mixer_tc196_kernel<k196Heads, JJ, FH>, p));                          \
   } while (0)
-#define SPECTRE_TC196_LAUNCH(JJ, WB)                                                                              \
-  do {                                                                                                            \
-    if (v->dtype == SPECTRE_F16) SPECTRE_TC196_LAUNCH2(JJ, WB, true); else SPECTRE_TC196_LAUNCH2(JJ, WB, false);  \
-  } while (0)
-  if (p.J == 2) { if (p.w_bf16) SPECTRE_TC196_LAUNCH(2, true); else SPECTRE_TC196_LAUNCH(2, false); }
-  else if (p.J == 1) { if (p.w_bf16) SPECTRE_TC196_LAUNCH(1, true); else SPECTRE_TC196_LAUNCH(1, false); }
-  else SPECTRE_TC196_LAUNCH(0, false);
-#undef SPECTRE_TC196_LAUNCH2
+  const bool f16 = v->dtype == SPECTRE_F16;
+  if (p.J == 2) { if (f16) SPECTRE_TC196_LAUNCH(2, true); else SPECTRE_TC196_LAUNCH(2, false); }
+  else if (p.J == 1) { if (f16) SPECTRE_TC196_LAUNCH(1, true); else SPECTRE_TC196_LAUNCH(1, false); }
+  else { if (f16) SPECTRE_TC196_LAUNCH(0, true); else SPECTRE_TC196_LAUNCH(0, false); }
 #undef SPECTRE_TC196_LAUNCH
   SPECTRE_LAUNCH_OK("mixer_tc196_kernel");
   return SPECTRE_OK;

@@ -270,11 +270,14 @@ def test_c5_reduced_batch_with_wavelet(ctx):
 
 @pytest.mark.parametrize("J,L,B,H,wdt,hid,given", [(2, 196, 2, 3, "bf16", 64, False), (1, 196, 1, 5, "f32", 48, False),
                                                  (2, 148, 3, 2, "bf16", 64, True), (1, 150, 2, 2, "f32", 64, True),
-                                                 (2, 196, 1, 2, "f32", 320, False)])
+                                                 (2, 196, 1, 2, "f32", 320, False), (2, 196, 11, 2, "bf16", 256, False),
+                                                 (2, 196, 9, 3, "f32", 37, False), (2, 196, 53, 12, "bf16", 64, False),
+                                                 (1, 196, 51, 12, "bf16", 64, True)])
 def test_mixer_196_with_refinement_in_the_store_phase(ctx, J, L, B, H, wdt, hid, given):
     # n = 196 on the tensor cores with the Haar refinement chained: level gates from the MLP (bf16 and
-    # fp32 weights, widths other than 64) or given; zero-padded rows; partial head groups; a hidden
-    # width the fused kernel does not take (320) must fall back to the separate refinement kernel.
+    # fp32 weights, widths 37 .. 256) or given; zero-padded rows; batch counts that leave a head pair
+    # and a level-gate batch partly empty; more head pairs than resident CTAs (each CTA loops); a hidden
+    # width the fused path does not take (320) must fall back to the separate refinement kernel.
     w = W.Workload("t", B=B, L=L, H=H, D=64, dtype="bf16", wdtype=wdt, n_fft=196, seed=11 * J + L + H,
                    wavelet_levels=J, wavelet_hidden=hid)
     x = W.activations(w, structured=True)
@@ -295,6 +298,23 @@ def test_mixer_196_with_refinement_in_the_store_phase(ctx, J, L, B, H, wdt, hid,
     torch.cuda.synchronize()
     ctx.poll_status()
     ref = O.wavelet_refine(O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=196), s_ref, J)
+    assert slab_err(W.to_f64(y), ref) < TOL["bf16"]
+
+
+def test_mixer_196_refinement_without_workspace(ctx):
+    # the MLP's level gates need scratch: without it the call must still be right (separate refinement kernel)
+    w = W.Workload("t", B=2, L=196, H=3, D=64, dtype="bf16", wdtype="bf16", n_fft=196, seed=31, wavelet_levels=2)
+    x = W.activations(w, structured=True)
+    g = W.random_gate(w)
+    wp = W.wavelet_params(w)
+    qbar = torch.randn(2, 3, 64, generator=torch.Generator().manual_seed(6))
+    s_ref = O.wavelet_level_gates(W.to_f64(qbar), W.to_f64(wp["Ww1"]), W.to_f64(wp["bw1"]), W.to_f64(wp["Ww2"]),
+                                  W.to_f64(wp["bw2"]), 2)
+    tiny = torch.empty(16, dtype=torch.uint8, device="cuda")
+    y = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=196, wrm=dict(to_dev(wp), qbar=qbar.cuda()), workspace=tiny)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ref = O.wavelet_refine(O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=196), s_ref, 2)
     assert slab_err(W.to_f64(y), ref) < TOL["bf16"]
 
 
