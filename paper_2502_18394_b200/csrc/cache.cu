@@ -9,7 +9,7 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
                      float2* ws, int* N1_out, int* M_out);
 bool transform_supported(const spectre_ctx* ctx, int n);
 size_t transform_slab_bytes(int n, int D);
-int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy);
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy_max, int* ncopy_used);
 size_t gate_min_workspace(int B, int H, int D, int n_fft, int r);
 size_t inverse_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
 int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y,
@@ -320,7 +320,8 @@ extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, cons
                                                 reinterpret_cast<T*>(cache->Q_buf), B, N, H, D, q->L);
   });
   SPECTRE_LAUNCH_OK("ring_fill_kernel");
-  return pool_sum(ctx, st, q, cache->sum_q, 1);
+  int used = 1;
+  return pool_sum(ctx, st, q, cache->sum_q, 1, &used);
 }
 
 extern "C" int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const spectre_cache* cache, const void* q_t,

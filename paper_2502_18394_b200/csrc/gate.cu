@@ -7,17 +7,23 @@
 //   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
 #include "common.cuh"
 
+#include <type_traits>
+
 namespace spectre {
 
 // ---- pooled sum over the sequence --------------------------------------------
-// Grid (slices, B).  A thread owns one 8-channel vector of the [H*D] row (several rows are in
-// flight when the row is narrower than the CTA) and walks the slice's rows with 8 loads in
-// flight; partial sums go with float atomics into copy (slice mod ncopy) of sums[ncopy][B,H,D]
-// (zeroed by the caller on the same stream), which keeps the contention per address low.
+// Grid (groups of 32 vectors, slices of the sequence, B).  A lane owns one 8-channel vector of the
+// [H*D] row, so a warp reads 512 contiguous bytes of a row; the CTA's 8 warps take rows 8 apart with
+// up to 16 rows per thread in flight.  The warps' partial sums meet in shared memory, and the CTA adds
+// one value per channel with float atomics into copy (slice mod ncopy) of sums[ncopy][B,H,D] (zeroed
+// by the caller on the same stream), which keeps the contention per address low.
 template <typename T> struct vec8;
 template <> struct vec8<bf16> {
-  static __device__ __forceinline__ void add(const bf16* p, float (&a)[8]) {
-    const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+  typedef uint4 raw;
+  static constexpr int kRows = 16;
+  static __device__ __forceinline__ raw load(const bf16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  static __device__ __forceinline__ raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
+  static __device__ __forceinline__ void add(const raw& r, float (&a)[8]) {
     const uint32_t u[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -27,8 +33,11 @@ template <> struct vec8<bf16> {
   }
 };
 template <> struct vec8<f16> {
-  static __device__ __forceinline__ void add(const f16* p, float (&a)[8]) {
-    const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+  typedef uint4 raw;
+  static constexpr int kRows = 16;
+  static __device__ __forceinline__ raw load(const f16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  static __device__ __forceinline__ raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
+  static __device__ __forceinline__ void add(const raw& r, float (&a)[8]) {
     const uint32_t u[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -39,10 +48,23 @@ template <> struct vec8<f16> {
   }
 };
 template <> struct vec8<float> {
-  static __device__ __forceinline__ void add(const float* p, float (&a)[8]) {
-    const float4 lo = __ldg(reinterpret_cast<const float4*>(p)), hi = __ldg(reinterpret_cast<const float4*>(p) + 1);
-    a[0] += lo.x; a[1] += lo.y; a[2] += lo.z; a[3] += lo.w;
-    a[4] += hi.x; a[5] += hi.y; a[6] += hi.z; a[7] += hi.w;
+  struct raw { float4 lo, hi; };
+  static constexpr int kRows = 8;
+  static __device__ __forceinline__ raw load(const float* p) {
+    raw r;
+    r.lo = __ldg(reinterpret_cast<const float4*>(p));
+    r.hi = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    return r;
+  }
+  static __device__ __forceinline__ raw zero() {
+    raw r;
+    r.lo = make_float4(0.f, 0.f, 0.f, 0.f);
+    r.hi = r.lo;
+    return r;
+  }
+  static __device__ __forceinline__ void add(const raw& r, float (&a)[8]) {
+    a[0] += r.lo.x; a[1] += r.lo.y; a[2] += r.lo.z; a[3] += r.lo.w;
+    a[4] += r.hi.x; a[5] += r.hi.y; a[6] += r.hi.z; a[7] += r.hi.w;
   }
 };
 
@@ -50,45 +72,57 @@ template <typename T>
 __global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
                                                    int H, int D, int rows_per, int ncopy, size_t copy_stride,
                                                    float* __restrict__ sums) {
+  __shared__ float red[8][8][32];                              // [warp][channel][lane]
   // the gate kernels behind this one may start early: they stream weights before they need the sums
   asm volatile("griddepcontrol.launch_dependents;");
-  const int b = blockIdx.y;
-  const int r0 = blockIdx.x * rows_per;
-  const int r1 = min(L, r0 + rows_per);
-  const int vec_per_head = D / 8;
-  const int nvec = H * vec_per_head;
-  const int rif = nvec >= 256 ? 1 : 256 / nvec;              // rows in flight across the CTA
-  const int ro = nvec >= 256 ? 0 : (int)threadIdx.x / nvec;
-  if (ro >= rif) return;
-  float* dst_copy = sums + (size_t)(blockIdx.x % ncopy) * copy_stride + (size_t)b * H * D;
-  for (int vi = nvec >= 256 ? threadIdx.x : (int)threadIdx.x - ro * nvec; vi < nvec; vi += 256) {
-    const int h = vi / vec_per_head, c = (vi - h * vec_per_head) * 8;
-    const T* base = q + b * sb + h * sh + c;
-    float acc[8];
+  constexpr int R = vec8<T>::kRows;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.z;
+  const int vec_per_head = D / 8, nvec = H * vec_per_head;
+  const int vi = blockIdx.x * 32 + lane;
+  const bool live = vi < nvec;
+  const int h = live ? vi / vec_per_head : 0, c = live ? (vi - h * vec_per_head) * 8 : 0;
+  const T* base = q + b * sb + h * sh + c;
+  const int r0 = blockIdx.y * rows_per, r1 = min(L, r0 + rows_per);
+  float acc[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    int r = r0 + ro;
-    for (; r + 7 * rif < r1; r += 8 * rif) {
+  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+  if (live) {
+    for (int r = r0 + warp; r < r1; r += 8 * R) {
+      typename vec8<T>::raw v[R];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) vec8<T>::add(base + (int64_t)(r + u * rif) * sl, acc);
+      for (int u = 0; u < R; ++u) v[u] = (r + 8 * u < r1) ? vec8<T>::load(base + (int64_t)(r + 8 * u) * sl) : vec8<T>::zero();
+#pragma unroll
+      for (int u = 0; u < R; ++u) vec8<T>::add(v[u], acc);
     }
-    for (; r < r1; r += rif) vec8<T>::add(base + (int64_t)r * sl, acc);
-    float* dst = dst_copy + h * D + c;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) atomicAdd(dst + i, acc[i]);
-    if (nvec < 256) break;
   }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) red[warp][i][lane] = acc[i];
+  __syncthreads();
+  float s = 0.f;                                               // thread (channel = warp, lane) adds up the 8 warps
+#pragma unroll
+  for (int w = 0; w < 8; ++w) s += red[w][warp][lane];
+  if (live) atomicAdd(sums + (size_t)(blockIdx.y % ncopy) * copy_stride + ((size_t)b * H + h) * D + c + warp, s);
 }
 
-// Sums of q over the sequence into `ncopy` partial copies (the consumer adds them up).
-int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy) {
+// Sums of q over the sequence into *ncopy_used <= ncopy_max partial copies (the consumer adds them up).
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy_max, int* ncopy_used) {
   const size_t copy_stride = (size_t)q->B * q->H * q->D;
+  const int groups = (q->H * (q->D / 8) + 31) / 32;
+  if (q->B > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B exceeds 65535");
+  // about 8 CTAs per SM in all, at least 8 rows (one per warp) per CTA
+  const long long per_slice = (long long)groups * q->B;
+  long long slices = (8LL * ctx->sm_count + per_slice - 1) / per_slice;
+  if (slices < 1) slices = 1;
+  int rows_per = (int)((q->L + slices - 1) / slices);
+  if (rows_per < 8) rows_per = 8;
+  const int nslice = (q->L + rows_per - 1) / rows_per;
+  int ncopy = (nslice + 15) / 16;                              // <= 16 CTAs add into one address
+  if (ncopy > ncopy_max) ncopy = ncopy_max;
+  if (ncopy < 1) ncopy = 1;
+  *ncopy_used = ncopy;
   SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, copy_stride * ncopy * sizeof(float), st));
-  int target = (2 * ctx->sm_count + q->B - 1) / q->B;
-  if (target < 1) target = 1;
-  int rows_per = (q->L + target - 1) / target;
-  if (rows_per < 32) rows_per = 32;
-  dim3 grid((q->L + rows_per - 1) / rows_per, q->B);
+  dim3 grid((unsigned)groups, (unsigned)nslice, (unsigned)q->B);
   SPECTRE_IO_DISPATCH(q->dtype, pool_kernel<T><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l,
                                                                      q->stride_h, q->L, q->H, q->D, rows_per, ncopy,
                                                                      copy_stride, sums));
@@ -99,7 +133,9 @@ int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, floa
 // ---- MLP ---------------------------------------------------------------------
 template <typename WT> __device__ __forceinline__ float wload(const WT* p);
 template <> __device__ __forceinline__ float wload<float>(const float* p) { return __ldg(p); }
-template <> __device__ __forceinline__ float wload<bf16>(const bf16* p) { return __bfloat162float(*p); }
+template <> __device__ __forceinline__ float wload<bf16>(const bf16* p) {
+  return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
+}
 template <typename WT> __device__ __forceinline__ float2 wload2(const WT* p);
 template <> __device__ __forceinline__ float2 wload2<float>(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
 template <> __device__ __forceinline__ float2 wload2<bf16>(const bf16* p) {
@@ -108,11 +144,12 @@ template <> __device__ __forceinline__ float2 wload2<bf16>(const bf16* p) {
 }
 
 // q_bar = LN(inv_count * sum) into shared memory (Sec. 3.2 step 3a), then the hidden layer
-// u = GELU(q_bar W1 + b1), for nb batch entries of one head at once: the means are spread over
-// the CTA, a warp normalises one entry, then the nb x hidden outputs are spread over the CTA.
+// u = GELU(q_bar W1 + b1), for nb <= NB batch entries of one head at once: the means are spread over
+// the CTA, a warp normalises one entry, then a thread takes one hidden unit for every g-th batch
+// entry (g = threads / hidden groups), so a weight column is fetched once per group, not per entry.
 // sums points at the first entry's [D] row, bstride is the distance between batch entries;
 // u is written as [hidden][ustride] (batch entry fastest).
-template <typename WT>
+template <typename WT, int NB>
 __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, size_t bstride, int nb, int ncopy,
                                                       size_t copy_stride, float inv_count, int D, int hidden,
                                                       const float* __restrict__ gamma, const float* __restrict__ beta,
@@ -149,20 +186,58 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
     for (int c = lane; c < D; c += 32) qb[c] = gamma[c] * (qb[c] - mean) * rstd + beta[c];
   }
   __syncthreads();
-  for (int item = threadIdx.x; item < nb * hidden; item += blockDim.x) {
-    const int bb = item / hidden, jj = item - bb * hidden;
-    const float* qb = qbar + bb * D;
-    float acc = b1[jj];
+  if constexpr (NB == 1) {
+    for (int jj = threadIdx.x; jj < hidden; jj += blockDim.x) {
+      float acc = b1[jj];
+      int c = 0;
+      for (; c + 32 <= D; c += 32) {                // 32 independent loads in flight
+        float wv[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + jj);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc = fmaf(qbar[c + i], wv[i], acc);
+      }
+      for (; c < D; ++c) acc = fmaf(qbar[c], wload<WT>(W1 + (size_t)c * hidden + jj), acc);
+      u[jj * ustride] = gelu_erf(acc);
+    }
+    __syncthreads();
+    return;
+  }
+  int groups = (int)blockDim.x / hidden;
+  groups = groups < 1 ? 1 : (groups > nb ? nb : groups);
+  for (int item = threadIdx.x; item < groups * hidden; item += blockDim.x) {
+    const int gi = item / hidden, jj = item - gi * hidden;
+    float acc[NB];                                  // slot s: batch entry gi + s * groups
+#pragma unroll
+    for (int sl = 0; sl < NB; ++sl) acc[sl] = b1[jj];
     int c = 0;
     for (; c + 32 <= D; c += 32) {                  // 32 independent loads in flight
       float wv[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + jj);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) acc = fmaf(qb[c + i], wv[i], acc);
+      for (int sl = 0; sl < NB; ++sl) {
+        const int bb = gi + sl * groups;
+        if (bb < nb) {
+          const float* qb = qbar + bb * D + c;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[sl] = fmaf(qb[i], wv[i], acc[sl]);
+        }
+      }
     }
-    for (; c < D; ++c) acc = fmaf(qb[c], wload<WT>(W1 + (size_t)c * hidden + jj), acc);
-    u[jj * ustride + bb] = gelu_erf(acc);            // [hidden][ustride]: one row = all batch entries
+    for (; c < D; ++c) {
+      const float wv = wload<WT>(W1 + (size_t)c * hidden + jj);
+#pragma unroll
+      for (int sl = 0; sl < NB; ++sl) {
+        const int bb = gi + sl * groups;
+        if (bb < nb) acc[sl] = fmaf(qbar[bb * D + c], wv, acc[sl]);
+      }
+    }
+#pragma unroll
+    for (int sl = 0; sl < NB; ++sl) {
+      const int bb = gi + sl * groups;
+      if (bb < nb) u[jj * ustride + bb] = gelu_erf(acc[sl]);   // [hidden][ustride]: one row = all batch entries
+    }
   }
   __syncthreads();
 }
@@ -174,13 +249,17 @@ __device__ __forceinline__ float2 modrelu(float2 gk, float bias) {
   return cscale(gk, sc);
 }
 // positional phase exp(+j 2 pi k p / n), angle reduced in integers
-__device__ __forceinline__ float2 phase_factor(int k, int n, long long shift) {
-  long long pm = shift % n;
-  if (pm < 0) pm += n;
-  if (pm == 0) return make_float2(1.f, 0.f);
+// pm = shift mod n in [0, n)
+__device__ __forceinline__ float2 phase_reduced(int k, int n, unsigned pm) {
+  if (pm == 0u) return make_float2(1.f, 0.f);
   const unsigned kp = (unsigned)(((unsigned long long)k * (unsigned long long)pm) % (unsigned)n);
   const float2 w = twiddle_fwd(kp, (unsigned)n);  // exp(-j ...)
   return make_float2(w.x, -w.y);
+}
+__device__ __forceinline__ float2 phase_factor(int k, int n, long long shift) {
+  long long pm = shift % n;
+  if (pm < 0) pm += n;
+  return phase_reduced(k, n, (unsigned)pm);
 }
 __device__ __forceinline__ float2 modrelu_phase(float2 gk, float bias, int k, int n, unsigned pm) {
   gk = modrelu(gk, bias);
@@ -198,6 +277,7 @@ struct GateMlpParams {
   const void* W1; const float* b1; const void* W2; const float* b2;
   const float* modrelu_bias;
   const long long* shift; long long shift_all;
+  unsigned pm_all;        // shift_all mod n in [0, n), reduced on the host
   float2* g_out;          // final gate, or the raw MLP output when post != 0
   float* qbar_out;
   float* u_ws;            // [B,H,hidden] hidden activations (workspace)
@@ -210,19 +290,21 @@ template <> struct wraw<bf16> {
   typedef unsigned type;
   static __device__ __forceinline__ type load(const bf16* p) { return __ldg(reinterpret_cast<const unsigned*>(p)); }
   static __device__ __forceinline__ float2 cvt(type r) { return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u)); }
-  static constexpr int kRows = 64;
+  static constexpr int kRows = 32;
 };
 template <> struct wraw<float> {
   typedef float2 type;
   static __device__ __forceinline__ type load(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
   static __device__ __forceinline__ float2 cvt(type r) { return r; }
-  static constexpr int kRows = 32;
+  static constexpr int kRows = 16;
 };
 
 // Output layer: grid (ceil(K / threads), H * ceil(B / BB)), one bin per thread for BB batch
 // entries of one head: W2 is shared by the batch, so a column fetched once serves all of them.
-// A thread issues the loads of up to kRows hidden rows of its W2 column before it uses any of
-// them, so the whole column is one memory round trip; the kernel is a pure stream over W2.
+// A thread issues the loads of kRows hidden rows of its W2 column before it uses any of them
+// (32 rows in bf16: two round trips for the usual 64-wide hidden layer) and needs few enough
+// registers for four CTAs per SM, so that the grid of an 8k-token transform is resident at once;
+// the kernel is a pure stream over W2.
 // Hidden activations of BB batch entries of one head, once: grid H * ceil(B / BB).
 template <typename WT, int BB>
 __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p) {
@@ -234,7 +316,7 @@ __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p)
   asm volatile("griddepcontrol.wait;" ::: "memory");        // the sums come from the kernel before
   float* qbar = u + BB * p.hidden;
   const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-  descriptor_and_hidden<WT>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+  descriptor_and_hidden<WT, BB>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
                             p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
                             p.b1 + h * p.hs_b1, qbar, u, BB);
   for (int e = threadIdx.x; e < nb * p.hidden; e += blockDim.x) {
@@ -251,7 +333,7 @@ __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p)
 // PRE: the hidden activations were computed once per (head, batch entry) by gate_hidden_kernel
 // (long transforms: hundreds of CTAs per head would otherwise repeat that work).
 template <typename WT, int BB, bool PRE>
-__global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
+__global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const GateMlpParams p) {
   extern __shared__ __align__(16) float u[];       // [hidden][BB], then q_bar [BB][D]
   constexpr int R = wraw<WT>::kRows;
   const int nbg = (p.B + BB - 1) / BB;
@@ -281,7 +363,7 @@ __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
     // entry, two short round trips) while this thread's W2 column is already on its way
     float* qbar = u + BB * p.hidden;   // [BB][D]
     const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-    descriptor_and_hidden<WT>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+    descriptor_and_hidden<WT, BB>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
                               p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
                               p.b1 + h * p.hs_b1, qbar, u, BB);
     if (p.qbar_out && blockIdx.x == 0)
@@ -295,16 +377,17 @@ __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
   float2 acc[BB];
 #pragma unroll
   for (int bb = 0; bb < BB; ++bb) acc[bb] = make_float2(b2[2 * k], b2[2 * k + 1]);
-  for (int j = 0; j < p.hidden; j += R) {
-    const int nr = min(R, p.hidden - j);
+  auto rows = [&](int j, auto full) {                    // rows j .. j + R - 1 (all present when `full`)
+    constexpr bool kFull = decltype(full)::value;
+    const int nr = kFull ? R : min(R, p.hidden - j);
     if (j > 0) {
 #pragma unroll
       for (int i = 0; i < R; ++i)
-        if (i < nr) w[i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
+        if (kFull || i < nr) w[i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
     }
 #pragma unroll
     for (int i = 0; i < R; ++i) {
-      if (i < nr) {
+      if (kFull || i < nr) {
         const float2 wv = wraw<WT>::cvt(w[i]);
         const float* ur = u + (j + i) * BB;             // entries of absent batch rows hold stale values, never stored
         float ub[BB];
@@ -325,11 +408,16 @@ __global__ void __launch_bounds__(256) gate_out_kernel(const GateMlpParams p) {
         }
       }
     }
+  };
+  if (p.hidden % R == 0) {
+    for (int j = 0; j < p.hidden; j += R) rows(j, std::true_type());
+  } else {
+    for (int j = 0; j < p.hidden; j += R) rows(j, std::false_type());
   }
   const float bias = (!p.post && p.modrelu_bias) ? p.modrelu_bias[h * p.hs_mb + k] : 0.f;
   // one positional phase for the whole batch unless per-entry shifts are given
   float2 ph = make_float2(1.f, 0.f);
-  if (!p.post && !p.shift) ph = phase_factor(k, p.n, p.shift_all);
+  if (!p.post && !p.shift) ph = phase_reduced(k, p.n, p.pm_all);
 #pragma unroll
   for (int bb = 0; bb < BB; ++bb) {
     if (bb < nb) {
@@ -446,8 +534,7 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
     float* pooled = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + sums_off);
     const size_t one_copy = (size_t)B * H * D * sizeof(float);
     size_t fit = (workspace_bytes - sums_off) / one_copy;
-    ncopy = fit > (size_t)kPoolCopies ? kPoolCopies : (int)fit;
-    int rc = pool_sum(ctx, st, q, pooled, ncopy);
+    int rc = pool_sum(ctx, st, q, pooled, fit > (size_t)kPoolCopies ? kPoolCopies : (int)fit, &ncopy);
     if (rc != SPECTRE_OK) return rc;
     sums = pooled;
   }
@@ -461,6 +548,11 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   mp.W1 = gp->W1; mp.b1 = gp->b1; mp.W2 = gp->W2; mp.b2 = gp->b2;
   mp.modrelu_bias = gp->modrelu_bias;
   mp.shift = reinterpret_cast<const long long*>(shift); mp.shift_all = shift_all;
+  {
+    long long pm = shift_all % n_fft;
+    if (pm < 0) pm += n_fft;
+    mp.pm_all = (unsigned)pm;
+  }
   mp.qbar_out = qbar_out;
   mp.u_ws = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + u_off);
   mp.post = r > 0;
