@@ -14,13 +14,14 @@ namespace spectre {
 // ---- pooled sum over the sequence --------------------------------------------
 // Grid (groups of 32 vectors, slices of the sequence, B).  A lane owns one 8-channel vector of the
 // [H*D] row, so a warp reads 512 contiguous bytes of a row; the CTA's 8 warps take rows 8 apart with
-// up to 16 rows per thread in flight.  The warps' partial sums meet in shared memory, and the CTA adds
+// up to 8 rows per thread in flight and four CTAs per SM.  The warps' partial sums meet in shared memory, and the CTA adds
 // one value per channel with float atomics into copy (slice mod ncopy) of sums[ncopy][B,H,D] (zeroed
-// by the caller on the same stream), which keeps the contention per address low.
+// by the caller on the same stream), which keeps the contention per address low; a CTA that holds the
+// whole sequence stores its sums instead.
 template <typename T> struct vec8;
 template <> struct vec8<bf16> {
   typedef uint4 raw;
-  static constexpr int kRows = 16;
+  static constexpr int kRows = 8;
   static __device__ __forceinline__ raw load(const bf16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
   static __device__ __forceinline__ raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
   static __device__ __forceinline__ void add(const raw& r, float (&a)[8]) {
@@ -34,7 +35,7 @@ template <> struct vec8<bf16> {
 };
 template <> struct vec8<f16> {
   typedef uint4 raw;
-  static constexpr int kRows = 16;
+  static constexpr int kRows = 8;
   static __device__ __forceinline__ raw load(const f16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
   static __device__ __forceinline__ raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
   static __device__ __forceinline__ void add(const raw& r, float (&a)[8]) {
@@ -49,7 +50,7 @@ template <> struct vec8<f16> {
 };
 template <> struct vec8<float> {
   struct raw { float4 lo, hi; };
-  static constexpr int kRows = 8;
+  static constexpr int kRows = 4;
   static __device__ __forceinline__ raw load(const float* p) {
     raw r;
     r.lo = __ldg(reinterpret_cast<const float4*>(p));
@@ -69,7 +70,7 @@ template <> struct vec8<float> {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
+__global__ void __launch_bounds__(256, 4) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
                                                    int H, int D, int rows_per, int ncopy, size_t copy_stride,
                                                    float* __restrict__ sums) {
   __shared__ float red[8][8][32];                              // [warp][channel][lane]
@@ -102,7 +103,11 @@ __global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ q, int6
   float s = 0.f;                                               // thread (channel = warp, lane) adds up the 8 warps
 #pragma unroll
   for (int w = 0; w < 8; ++w) s += red[w][warp][lane];
-  if (live) atomicAdd(sums + (size_t)(blockIdx.y % ncopy) * copy_stride + ((size_t)b * H + h) * D + c + warp, s);
+  if (live) {
+    float* dst = sums + (size_t)(blockIdx.y % ncopy) * copy_stride + ((size_t)b * H + h) * D + c + warp;
+    if (gridDim.y == 1) *dst = s;                              // the only slice: no other CTA adds to this address
+    else atomicAdd(dst, s);
+  }
 }
 
 // Sums of q over the sequence into *ncopy_used <= ncopy_max partial copies (the consumer adds them up).
@@ -110,18 +115,20 @@ int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, floa
   const size_t copy_stride = (size_t)q->B * q->H * q->D;
   const int groups = (q->H * (q->D / 8) + 31) / 32;
   if (q->B > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B exceeds 65535");
-  // about 8 CTAs per SM in all, at least 8 rows (one per warp) per CTA
+  // one resident wave (four CTAs per SM) of equal slices, never a few CTAs more than fit at once;
+  // at least 8 rows (one per warp) per CTA
   const long long per_slice = (long long)groups * q->B;
-  long long slices = (8LL * ctx->sm_count + per_slice - 1) / per_slice;
+  long long slices = (4LL * ctx->sm_count) / per_slice;
   if (slices < 1) slices = 1;
   int rows_per = (int)((q->L + slices - 1) / slices);
   if (rows_per < 8) rows_per = 8;
   const int nslice = (q->L + rows_per - 1) / rows_per;
   int ncopy = (nslice + 15) / 16;                              // <= 16 CTAs add into one address
+  if (ncopy > 8) ncopy = 8;                                    // one batch of loads for the consumer
   if (ncopy > ncopy_max) ncopy = ncopy_max;
   if (ncopy < 1) ncopy = 1;
   *ncopy_used = ncopy;
-  SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, copy_stride * ncopy * sizeof(float), st));
+  if (nslice > 1) SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, copy_stride * ncopy * sizeof(float), st));
   dim3 grid((unsigned)groups, (unsigned)nslice, (unsigned)q->B);
   SPECTRE_IO_DISPATCH(q->dtype, pool_kernel<T><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l,
                                                                      q->stride_h, q->L, q->H, q->D, rows_per, ncopy,
@@ -149,25 +156,51 @@ template <> __device__ __forceinline__ float2 wload2<bf16>(const bf16* p) {
 // entry (g = threads / hidden groups), so a weight column is fetched once per group, not per entry.
 // sums points at the first entry's [D] row, bstride is the distance between batch entries;
 // u is written as [hidden][ustride] (batch entry fastest).
-template <typename WT, int NB>
+// STAGED: W1 points at a copy of the head's weights in shared memory (made before the wait on the
+// producer of the sums), so the hidden layer adds no memory round trip behind the sums.
+template <typename WT> __device__ __forceinline__ float wvalue(WT x);
+template <> __device__ __forceinline__ float wvalue<float>(float x) { return x; }
+template <> __device__ __forceinline__ float wvalue<bf16>(bf16 x) { return __bfloat162float(x); }
+template <typename WT, bool STAGED> __device__ __forceinline__ float wget(const WT* p) {
+  if constexpr (STAGED) return wvalue<WT>(*p);
+  else return wload<WT>(p);
+}
+
+template <typename WT, int NB, bool STAGED>
 __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ sums, size_t bstride, int nb, int ncopy,
                                                       size_t copy_stride, float inv_count, int D, int hidden,
                                                       const float* __restrict__ gamma, const float* __restrict__ beta,
                                                       float eps, const WT* __restrict__ W1, const float* __restrict__ b1,
                                                       float* qbar, float* u, int ustride) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
-  for (int e = threadIdx.x; e < nb * D; e += blockDim.x) {   // means: the whole CTA, one channel per thread
-    const int bb = e / D, c = e - bb * D;
-    const float* sb = sums + (size_t)bb * bstride + c;
-    float m = 0.f;
-    for (int k0 = 0; k0 < ncopy; k0 += 16) {                  // all copies in flight at once
-      float v[16];
+  if (NB > 1 && ncopy == 1) {                                // means, one copy: up to 4 channels per thread in flight
+    for (int e0 = threadIdx.x; e0 < nb * D; e0 += 4 * blockDim.x) {
+      float v[4];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) v[k] = (k0 + k < ncopy) ? sb[(size_t)(k0 + k) * copy_stride] : 0.f;
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * (int)blockDim.x, bb = e / D, c = e - bb * D;
+        v[u] = e < nb * D ? sums[(size_t)bb * bstride + c] : 0.f;
+      }
 #pragma unroll
-      for (int k = 0; k < 16; ++k) m += v[k];
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * (int)blockDim.x;
+        if (e < nb * D) qbar[e] = v[u] * inv_count;
+      }
     }
-    qbar[e] = m * inv_count;
+  } else {
+    for (int e = threadIdx.x; e < nb * D; e += blockDim.x) {   // means: the whole CTA, one channel per thread
+      const int bb = e / D, c = e - bb * D;
+      const float* sb = sums + (size_t)bb * bstride + c;
+      float m = 0.f;
+      for (int k0 = 0; k0 < ncopy; k0 += 8) {                   // eight copies in flight at once
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = (k0 + k < ncopy) ? sb[(size_t)(k0 + k) * copy_stride] : 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) m += v[k];
+      }
+      qbar[e] = m * inv_count;
+    }
   }
   __syncthreads();
   for (int bb = warp; bb < nb; bb += nw) {                    // statistics: one warp per batch entry
@@ -193,11 +226,11 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
       for (; c + 32 <= D; c += 32) {                // 32 independent loads in flight
         float wv[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + jj);
+        for (int i = 0; i < 32; ++i) wv[i] = wget<WT, STAGED>(W1 + (size_t)(c + i) * hidden + jj);
 #pragma unroll
         for (int i = 0; i < 32; ++i) acc = fmaf(qbar[c + i], wv[i], acc);
       }
-      for (; c < D; ++c) acc = fmaf(qbar[c], wload<WT>(W1 + (size_t)c * hidden + jj), acc);
+      for (; c < D; ++c) acc = fmaf(qbar[c], wget<WT, STAGED>(W1 + (size_t)c * hidden + jj), acc);
       u[jj * ustride] = gelu_erf(acc);
     }
     __syncthreads();
@@ -214,7 +247,7 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
     for (; c + 32 <= D; c += 32) {                  // 32 independent loads in flight
       float wv[32];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) wv[i] = wload<WT>(W1 + (size_t)(c + i) * hidden + jj);
+      for (int i = 0; i < 32; ++i) wv[i] = wget<WT, STAGED>(W1 + (size_t)(c + i) * hidden + jj);
 #pragma unroll
       for (int sl = 0; sl < NB; ++sl) {
         const int bb = gi + sl * groups;
@@ -226,7 +259,7 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
       }
     }
     for (; c < D; ++c) {
-      const float wv = wload<WT>(W1 + (size_t)c * hidden + jj);
+      const float wv = wget<WT, STAGED>(W1 + (size_t)c * hidden + jj);
 #pragma unroll
       for (int sl = 0; sl < NB; ++sl) {
         const int bb = gi + sl * groups;
@@ -240,6 +273,21 @@ __device__ __forceinline__ void descriptor_and_hidden(const float* __restrict__ 
     }
   }
   __syncthreads();
+}
+
+// 16-byte copy of a head's W1 into shared memory, two pieces per thread in flight
+__device__ __forceinline__ void stage_weights(const void* src, void* dst, int bytes) {
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+  const int n16 = bytes >> 4;
+  for (int i0 = threadIdx.x; i0 < n16; i0 += 2 * blockDim.x) {
+    const int i1 = i0 + (int)blockDim.x;
+    const uint4 v0 = __ldg(s4 + i0);
+    uint4 v1 = make_uint4(0u, 0u, 0u, 0u);
+    if (i1 < n16) v1 = __ldg(s4 + i1);
+    d4[i0] = v0;
+    if (i1 < n16) d4[i1] = v1;
+  }
 }
 
 // modReLU: max(|z| + b, 0) z / |z|   (0 at z = 0)
@@ -282,6 +330,7 @@ struct GateMlpParams {
   float* qbar_out;
   float* u_ws;            // [B,H,hidden] hidden activations (workspace)
   int post;               // 1: Toeplitz follows, skip modReLU/phase here
+  int stage_w1;           // W1 of a head is copied to shared memory before the wait (size and alignment allow)
 };
 
 // raw (re, im) weight pair of one bin in one hidden row
@@ -313,12 +362,19 @@ __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p)
   const int h = blockIdx.x / nbg, b0 = (blockIdx.x - h * nbg) * BB;
   const int nb = min(BB, p.B - b0);
   asm volatile("griddepcontrol.launch_dependents;");
-  asm volatile("griddepcontrol.wait;" ::: "memory");        // the sums come from the kernel before
   float* qbar = u + BB * p.hidden;
   const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-  descriptor_and_hidden<WT, BB>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
-                            p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
-                            p.b1 + h * p.hs_b1, qbar, u, BB);
+  WT* w1s = reinterpret_cast<WT*>(u + ((BB * (p.hidden + p.D) + 3) & ~3));
+  if (p.stage_w1) stage_weights(W1, w1s, p.D * p.hidden * (int)sizeof(WT));
+  asm volatile("griddepcontrol.wait;" ::: "memory");        // the sums come from the kernel before
+  if (p.stage_w1)
+    descriptor_and_hidden<WT, BB, true>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+                                        p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, w1s,
+                                        p.b1 + h * p.hs_b1, qbar, u, BB);
+  else
+    descriptor_and_hidden<WT, BB, false>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+                                         p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
+                                         p.b1 + h * p.hs_b1, qbar, u, BB);
   for (int e = threadIdx.x; e < nb * p.hidden; e += blockDim.x) {
     const int bb = e / p.hidden, jj = e - bb * p.hidden;
     p.u_ws[((size_t)(b0 + bb) * p.H + h) * p.hidden + jj] = u[jj * BB + bb];
@@ -343,6 +399,8 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
   const bool live = k < p.K;
   const WT* col = reinterpret_cast<const WT*>(p.W2) + h * p.hs_w2 + 2 * (size_t)(live ? k : 0);
   const size_t ld = 2 * (size_t)p.K;
+  WT* w1s = reinterpret_cast<WT*>(u + ((BB * (p.hidden + p.D) + 3) & ~3));
+  if (!PRE && p.stage_w1) stage_weights(reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1, w1s, p.D * p.hidden * (int)sizeof(WT));
   typename wraw<WT>::type w[R];
   const int n0 = min(R, p.hidden);
   if (live) {
@@ -363,9 +421,14 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
     // entry, two short round trips) while this thread's W2 column is already on its way
     float* qbar = u + BB * p.hidden;   // [BB][D]
     const WT* W1 = reinterpret_cast<const WT*>(p.W1) + h * p.hs_w1;
-    descriptor_and_hidden<WT, BB>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
-                              p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
-                              p.b1 + h * p.hs_b1, qbar, u, BB);
+    if (p.stage_w1)
+      descriptor_and_hidden<WT, BB, true>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+                                          p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, w1s,
+                                          p.b1 + h * p.hs_b1, qbar, u, BB);
+    else
+      descriptor_and_hidden<WT, BB, false>(p.sums + ((size_t)b0 * p.H + h) * p.D, (size_t)p.H * p.D, nb, p.ncopy, p.copy_stride,
+                                           p.inv_count, p.D, p.hidden, p.gamma + h * p.hs_ln, p.beta + h * p.hs_ln, p.eps, W1,
+                                           p.b1 + h * p.hs_b1, qbar, u, BB);
     if (p.qbar_out && blockIdx.x == 0)
       for (int e = threadIdx.x; e < nb * p.D; e += blockDim.x) {
         const int bb = e / p.D, c = e - bb * p.D;
@@ -564,8 +627,10 @@ extern "C" int spectre_gate(spectre_ctx* ctx, void* stream, const spectre_act* q
   const int BB = (gp->hidden > 256 || B < 2) ? 1 : (B < 4 ? 2 : (B < 8 ? 4 : 8));
   dim3 grid_out((K + thr_out - 1) / thr_out, (unsigned)(H * ((B + BB - 1) / BB)));
   if (grid_out.y > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "H * ceil(B / 8) exceeds 65535");
-  const size_t smem = (size_t)BB * (D + gp->hidden) * sizeof(float);
   const bool wb = gp->wdtype == SPECTRE_BF16;
+  const size_t w1_bytes = (size_t)D * gp->hidden * (wb ? 2 : 4);
+  mp.stage_w1 = w1_bytes <= 16384 && w1_bytes % 16 == 0 && !(reinterpret_cast<uintptr_t>(gp->W1) & 15);
+  const size_t smem = (((size_t)BB * (D + gp->hidden) + 3) & ~(size_t)3) * sizeof(float) + (mp.stage_w1 ? w1_bytes : 0);
   const bool pre = grid_out.x >= 32;               // many CTAs per head: compute the hidden layer once
   // Programmatic dependent launch: the weight stream of the output layer may overlap the kernel
   // before it (the pooling pass here, or whatever produced sum_q); each kernel waits for its
