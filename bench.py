@@ -191,7 +191,7 @@ class MixerBench:
         self.units_per_step = w.B * w.L                                  # tokens
         self.alg_bytes = mixer_algorithmic_bytes(w)
         # kernels per step: gate = pool + output layer; mixer = 1 (single-kernel paths) or
-        # gate images + transpose-in + core + transpose-out per group of heads (staged tensor-core
+        # transpose-in (with the gate images) + core + transpose-out per group of heads (staged tensor-core
         # path) or strided + on-chip + strided per group (fp32 four-step path); + wavelet
         import math
         fused_wrm = w.dtype in ("bf16", "f16") and w.n == 196 and w.D == 64 and w.wavelet_levels in (1, 2) and w.wavelet_hidden <= 256
@@ -204,7 +204,7 @@ class MixerBench:
             R, ntile = w.n // 4096, w.D // 8
             per = R * ntile * (32 * 2064 + 65536) + R * 18432 + 256
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
-            self.kernel_name, nk = "mixer, staged tcgen05 path (tc_gate + tc_in + tc_core + tc_out per group)", 4 * groups
+            self.kernel_name, nk = "mixer, staged tcgen05 path (tc_in incl. gate images + tc_core + tc_out per group)", 3 * groups
         elif ws_mix:
             per = w.n * (w.D // 2) * 8
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))

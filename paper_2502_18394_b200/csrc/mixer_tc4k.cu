@@ -8,8 +8,9 @@
 //                   writes, for every unit (head, k1, 4 column pairs), the first tensor-core
 //                   operand as an image of its shared-memory layout (transposed through
 //                   shared memory so that the workspace writes are whole lines too)
-//   tc_gate_kernel  per (head, k1): the 4096 gate values the unit needs (Hermitian extension,
-//                   normalised by their maximum, fp16) in the order the core reads them
+//   (gate images)   per (head, k1): the 4096 gate values the unit needs (Hermitian extension,
+//                   normalised by their maximum, fp16) in the order the core reads them; written by
+//                   the first CTAs of the tc_in_kernel launch
 //   tc_core_kernel  persistent, one CTA per SM, units taken in pairs: 16 epilogue warps alternate
 //                   between the two units while a producer warp fetches the operand images with
 //                   bulk async copies and issues the MMAs (64-point DFT matrix as the A operand,
@@ -90,6 +91,60 @@ __host__ __device__ constexpr float in_scale(int R) {
 }
 
 // =====================================================================================
+// gate images: per (head, k1) the 4096 gate values the unit needs (Hermitian extension, normalised
+// by their maximum, fp16) in the order the core reads them.  Runs as the first CTAs of the
+// transpose-in launch (it depends on the gate only, the other CTAs on the activations only), so its
+// strided reads fill the gaps of that kernel instead of standing alone in the stream.
+// =====================================================================================
+struct TcGateParams {
+  const float2* g;          // [B*H][K]
+  unsigned char* gimg;      // [slab_local * R + k1][k4GBytes]
+  float* gscale;            // [slab_local * R + k1]
+  int n, K, R, slab0;
+};
+
+// vals: 4096 float2 of shared memory
+__device__ __forceinline__ void tc_gate_body(const TcGateParams& p, int sk, float2* vals) {
+  __shared__ float red[8];
+  const int slab_local = sk / p.R, k1 = sk - slab_local * p.R;
+  const float2* g = p.g + (size_t)(p.slab0 + slab_local) * p.K;
+  float m = 0.f;
+  float2 gv[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {                                 // 16 strided loads in flight per thread
+    const int k = k1 + p.R * (threadIdx.x + 256 * i);
+    const int kk = (2 * k <= p.n) ? k : p.n - k;
+    float2 v = __ldg(g + kk);
+    if (kk != k) v.y = -v.y;
+    if (k == 0 || 2 * k == p.n) v.y = 0.f;
+    gv[i] = v;
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    vals[threadIdx.x + 256 * i] = gv[i];
+    m = fmaxf(m, fmaxf(fabsf(gv[i].x), fabsf(gv[i].y)));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = 0.f;
+  for (int i = 0; i < 8; ++i) m = fmaxf(m, red[i]);
+  m *= 1.41421356f;
+  const float inv = m > 0.f ? 1.0f / m : 0.f;
+  if (threadIdx.x == 0) p.gscale[sk] = m;
+  uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * k4GBytes);
+  for (int idx = threadIdx.x; idx < 64 * k4GStride; idx += 256) {
+    const int col = idx / k4GStride, row = idx - col * k4GStride;     // kM = col + 64 row
+    uint32_t v = 0u;
+    if (row < 64) {
+      const float2 gv2 = vals[col + 64 * row];
+      v = h2pack(gv2.x * inv, gv2.y * inv);
+    }
+    img[idx] = v;
+  }
+}
+
+// =====================================================================================
 // transpose-in
 // =====================================================================================
 struct TcInParams {
@@ -102,13 +157,18 @@ struct TcInParams {
 // CTA = (slab, group of 4 consecutive t1, block of NT2 values of t2); t' = 64 t1 + t2.
 // A warp takes one (t1, t2) at a time with lane = column pair; staging holds, for every
 // (k1, tile), the core matrices (8 operand columns x 16 bytes) of this CTA's slice.
+// The first ngate CTAs write the gate images (tc_gate_body) instead.
 template <int R, bool F16>
-__global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
+__global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const TcGateParams gp, int ngate) {
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
-  extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][NT2/2][32 words]
+  extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][NT2/2][32 words]; >= 32 KB
+  if ((int)blockIdx.x < ngate) {
+    tc_gate_body(gp, (int)blockIdx.x, reinterpret_cast<float2*>(stage));
+    return;
+  }
   const int t2blocks = 64 / NT2;
-  int u = blockIdx.x;
+  int u = (int)blockIdx.x - ngate;
   const int t2b = u % t2blocks;  u /= t2blocks;
   const int t1g = u % 16;  u /= 16;
   const int slab_local = u, slab = p.slab0 + u;
@@ -177,57 +237,6 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p) {
     uint4 o;
     o.x = w[0 ^ (sk & 3)]; o.y = w[1 ^ (sk & 3)]; o.z = w[2 ^ (sk & 3)]; o.w = w[3 ^ (sk & 3)];
     *reinterpret_cast<uint4*>(img0 + (size_t)ut * k4ImgBytes + t2p * k4Sbo + q16 * 16) = o;
-  }
-}
-
-// =====================================================================================
-// gate images
-// =====================================================================================
-struct TcGateParams {
-  const float2* g;          // [B*H][K]
-  unsigned char* gimg;      // [slab_local * R + k1][k4GBytes]
-  float* gscale;            // [slab_local * R + k1]
-  int n, K, R, slab0;
-};
-
-__global__ void __launch_bounds__(256) tc_gate_kernel(const TcGateParams p) {
-  __shared__ float2 vals[4096];
-  __shared__ float red[8];
-  const int sk = blockIdx.x, slab_local = sk / p.R, k1 = sk - slab_local * p.R;
-  const float2* g = p.g + (size_t)(p.slab0 + slab_local) * p.K;
-  float m = 0.f;
-  float2 gv[16];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {                                 // 16 strided loads in flight per thread
-    const int k = k1 + p.R * (threadIdx.x + 256 * i);
-    const int kk = (2 * k <= p.n) ? k : p.n - k;
-    float2 v = __ldg(g + kk);
-    if (kk != k) v.y = -v.y;
-    if (k == 0 || 2 * k == p.n) v.y = 0.f;
-    gv[i] = v;
-  }
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    vals[threadIdx.x + 256 * i] = gv[i];
-    m = fmaxf(m, fmaxf(fabsf(gv[i].x), fabsf(gv[i].y)));
-  }
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
-  __syncthreads();
-  m = 0.f;
-  for (int i = 0; i < 8; ++i) m = fmaxf(m, red[i]);
-  m *= 1.41421356f;
-  const float inv = m > 0.f ? 1.0f / m : 0.f;
-  if (threadIdx.x == 0) p.gscale[sk] = m;
-  uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * k4GBytes);
-  for (int idx = threadIdx.x; idx < 64 * k4GStride; idx += 256) {
-    const int col = idx / k4GStride, row = idx - col * k4GStride;     // kM = col + 64 row
-    uint32_t v = 0u;
-    if (row < 64) {
-      const float2 gv = vals[col + 64 * row];
-      v = h2pack(gv.x * inv, gv.y * inv);
-    }
-    img[idx] = v;
   }
 }
 
@@ -572,16 +581,15 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   float* gscale = reinterpret_cast<float*>(gimg + (size_t)cnt * R * k4GBytes);
 
   TcGateParams gp = {reinterpret_cast<const float2*>(g), gimg, gscale, n, n / 2 + 1, R, slab0};
-  tc_gate_kernel<<<cnt * R, 256, 0, st>>>(gp);
-  SPECTRE_LAUNCH_OK("tc_gate_kernel");
 
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   TcInParams ip = {reinterpret_cast<const bf16*>(v->ptr), v->stride_b, v->stride_l, v->stride_h, ws_in,
                    v->H, D, v->L, n, ntile, slab0};
-  const size_t smem_in = (size_t)R * ntile * (NT2 / 2) * 128;
+  size_t smem_in = (size_t)R * ntile * (NT2 / 2) * 128;
+  if (smem_in < 4096 * sizeof(float2)) smem_in = 4096 * sizeof(float2);       // the gate CTAs' staging
   if (smem_in > 48 * 1024)
     SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in_kernel<R, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_in));
-  tc_in_kernel<R, F16><<<cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip);
+  tc_in_kernel<R, F16><<<cnt * R + cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip, gp, cnt * R);
   SPECTRE_LAUNCH_OK("tc_in_kernel");
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
