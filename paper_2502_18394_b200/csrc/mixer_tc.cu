@@ -9,9 +9,6 @@ constexpr int kTcLbo = 144;                    // bytes between core matrices al
 constexpr int kTcSbo = 2320;                   // bytes between 8-column groups (16 * 144 + 16 pad)
 constexpr int kTcBBytes = 32 * kTcSbo;         // one 256-column B operand
 constexpr int kTcFBytes = 128 * 128 * 2;
-constexpr int kTcEpiWarps = 16;                // 4 per TMEM lane quadrant, one column quarter each
-constexpr int kTcEpiThreads = 32 * kTcEpiWarps;
-constexpr int kTcThreads = kTcEpiThreads + 32; // + 1 MMA-issuing warp
 // Optional phase stamps (SM clock), compiled in only for profiling builds.
 #ifdef SPECTRE_TC_TIMING
 __device__ long long g_tc_timing[1024][16];
@@ -84,15 +81,18 @@ int build_dft64(__half* F, cudaStream_t st) {
 }
 
 // =====================================================================================
-// n = 196 (14 x 14 patch grids), bf16 I/O, D = 64: 196 = 4 * 49.
+// n = 196 (14 x 14 patch grids), bf16 or fp16 I/O, D = 64: 196 = 4 * 49.
 //
 // t = 49 n1 + t', k = k1 + 4 kM.  The radix-4 DFT over n1 and the twiddle W_196^{k1 t'} run on
 // the ALUs while whole 128-byte head rows are loaded; each 49-point DFT over t' is ONE tensor-core
 // stage with the 49-point DFT matrix in real form (98 x 98, zero-padded to 128 x 112) as the A
 // operand; the gate is applied to the accumulator, one more stage does the inverse 49-point DFT
 // (conj trick), and the final epilogue does the inverse radix-4 and stores bf16 rows.
-// A CTA takes 4 heads: columns (head, k1, pair) = 4 x 4 x 32 = 512 = the whole TMEM; the two
-// 2-head halves ping-pong between tensor core and ALUs like the halves of the 8192 kernel.
+// A work item is 2 heads (the same head index of two batch entries): columns (head, k1, pair) =
+// 2 x 4 x 32 = 256 TMEM columns and one operand buffer, so two CTAs share an SM and one's loads run
+// under the other's arithmetic; a CTA loops over its work items (persistent grid).  The kernel is
+// written for NH = 2 or 4 heads per item (4: two halves that ping-pong between tensor core and ALUs
+// like the halves of the 8192 kernel, one CTA per SM); 2 measured faster and is what is launched.
 // =====================================================================================
 constexpr int k196Heads = 2;                  // heads per CTA the launcher uses: two CTAs per SM (4 per CTA measured slower)
 constexpr int k196KSteps = 7;                 // K = 112 >= 98
@@ -232,6 +232,7 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
   __shared__ float gmax_s[NH];
 
   __shared__ int abort_s;
+  __shared__ float2 tw_s[3 * 49];                    // W_196^{m t'}, m = 1, 2, 3
 
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
   const int nwork = p.H * ((p.B + NH - 1) / NH);     // work items: NH batch entries of one head index
@@ -240,6 +241,13 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
   if (warp == EW) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(256 * NHALF));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  if (tid < 49) {
+    const float2 w1 = twiddle_fwd((unsigned)tid, 196u);
+    const float2 w2 = cmul(w1, w1);
+    tw_s[3 * tid] = w1;
+    tw_s[3 * tid + 1] = w2;
+    tw_s[3 * tid + 2] = cmul(w2, w1);
   }
   if (tid == 0) {
     abort_s = 0;
@@ -342,8 +350,7 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
       const int hl = item / 13, tg = item - hl * 13;
       const int tp = 4 * tg + (T >> 3), chunk = T & 7;
       if (item >= NH * 13 || tp >= 49 || bg * NH + hl >= p.B) continue;
-      const float2 w1 = twiddle_fwd((unsigned)tp, 196u);
-      const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
+      const float2 w1 = tw_s[3 * tp], w2 = tw_s[3 * tp + 1], w3 = tw_s[3 * tp + 2];
       unsigned char* Bh = Bsm[hl >> 1] + b_off((hl & 1) * 128 + 4 * chunk, 2 * tp);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -497,8 +504,7 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
               tmem_ld_16x256b_x1(tbase + ((uint32_t)(16 * nj) << 16) + 32 * k1 + 8 * ng, rk[(step + 1) & 1][k1]);
           }
           if (tp < 49) {
-            const float2 w1 = twiddle_fwd((unsigned)tp, 196u);
-            const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
+            const float2 w1 = tw_s[3 * tp], w2 = tw_s[3 * tp + 1], w3 = tw_s[3 * tp + 2];
             float2 y0[4], y1[4];
 #pragma unroll
             for (int k1 = 0; k1 < 4; ++k1) {                         // conj of the accumulator = IDFT49 (conj trick)
