@@ -391,6 +391,8 @@ __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p)
 template <typename WT, int BB, bool PRE>
 __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const GateMlpParams p) {
   extern __shared__ __align__(16) float u[];       // [hidden][BB], then q_bar [BB][D]
+  // a kernel launched behind this one as a programmatic dependent may do its set-up meanwhile
+  asm volatile("griddepcontrol.launch_dependents;");
   constexpr int R = wraw<WT>::kRows;
   const int nbg = (p.B + BB - 1) / BB;
   const int h = blockIdx.y / nbg, b0 = (blockIdx.y - h * nbg) * BB;
@@ -506,6 +508,7 @@ struct GatePostParams {
 // Toeplitz update along the bin axis ('same' window, zero boundary, reads the
 // pre-update gate), then modReLU and phase (Sec. 3.2 steps 3b-3c).
 __global__ void __launch_bounds__(256) gate_post_kernel(const GatePostParams p) {
+  asm volatile("griddepcontrol.launch_dependents;");
   const int bh = blockIdx.y, b = bh / p.H, h = bh - b * p.H;
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= p.K) return;

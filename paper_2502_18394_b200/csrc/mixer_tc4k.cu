@@ -163,6 +163,7 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
   extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][NT2/2][32 words]; >= 32 KB
+  asm volatile("griddepcontrol.wait;" ::: "memory");          // launched as a programmatic dependent
   if ((int)blockIdx.x < ngate) {
     tc_gate_body(gp, (int)blockIdx.x, reinterpret_cast<float2*>(stage));
     return;
@@ -589,7 +590,17 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   if (smem_in < 4096 * sizeof(float2)) smem_in = 4096 * sizeof(float2);       // the gate CTAs' staging
   if (smem_in > 48 * 1024)
     SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in_kernel<R, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_in));
-  tc_in_kernel<R, F16><<<cnt * R + cnt * 16 * (64 / NT2), 256, smem_in, st>>>(ip, gp, cnt * R);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(cnt * R + cnt * 16 * (64 / NT2)));
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = smem_in;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_in_kernel<R, F16>, ip, gp, cnt * R));
   SPECTRE_LAUNCH_OK("tc_in_kernel");
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),

@@ -199,6 +199,10 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = tmem_slot;
+  // Launched as a programmatic dependent of whatever precedes it in the stream: the set-up above may
+  // run while that kernel finishes (if it triggers early, as the gate kernels do); nothing of V or g
+  // is read before its writes are visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   TC8K_STAMP(1);
 
   if (warp == k8EpiWarps) {
@@ -465,12 +469,22 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
   p.H = v->H; p.ntile = v->D / 8;
   p.status = ctx->status_dev;
   const unsigned grid = (unsigned)((size_t)v->B * v->H * p.ntile);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(k8Threads);
+  cfg.dynamicSmemBytes = k8Smem;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (v->dtype == SPECTRE_F16) {
     SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k8Smem));
-    mixer_tc8192_kernel<true><<<grid, k8Threads, k8Smem, st>>>(tm_in, tm_out, p);
+    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, mixer_tc8192_kernel<true>, tm_in, tm_out, p));
   } else {
     SPECTRE_CUDA_OK(cudaFuncSetAttribute(mixer_tc8192_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k8Smem));
-    mixer_tc8192_kernel<false><<<grid, k8Threads, k8Smem, st>>>(tm_in, tm_out, p);
+    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, mixer_tc8192_kernel<false>, tm_in, tm_out, p));
   }
   SPECTRE_LAUNCH_OK("mixer_tc8192_kernel");
   return SPECTRE_OK;
