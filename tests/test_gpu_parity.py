@@ -194,6 +194,19 @@ def test_gate_bf16_weights_full_options(ctx):
     assert eg < 1e-4 and eq < 1e-4
 
 
+@pytest.mark.parametrize("B,L,H,D,hid,dt,wdt,n", [(5, 5, 1, 8, 16, "f32", "f32", 8), (2, 3000, 9, 40, 64, "bf16", "bf16", 4096),
+                                                  (1, 100, 2, 128, 300, "f32", "bf16", 128), (9, 333, 5, 64, 64, "f16", "bf16", 512),
+                                                  (3, 20000, 2, 64, 48, "bf16", "f32", 32768)])
+def test_gate_shapes(ctx, B, L, H, D, hid, dt, wdt, n):
+    # pooling: fewer rows than warps, row widths that are not a multiple of a warp's 512 bytes, one and
+    # many slices (store / atomics into several copies), several vector groups; output layer: hidden widths
+    # that are and are not a multiple of the rows in flight, W1 staged in shared memory or too large for
+    # it, all batch groupings
+    w = W.Workload("t", B=B, L=L, H=H, D=D, dtype=dt, wdtype=wdt, n_fft=n, hidden=hid, seed=B + L)
+    eg, eq, *_ = run_gate(ctx, w, modrelu_bias_std=0.05, bias_std=0.1, shift_all=3)
+    assert eg < 2e-4 and eq < 2e-4
+
+
 def test_gate_from_running_sum_and_shared_heads(ctx):
     w = W.Workload("t", B=2, L=64, H=4, D=32, dtype="f32", wdtype="f32", n_fft=64, seed=13)
     p = W.gate_params(w)
