@@ -244,8 +244,13 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const
 #ifdef SPECTRE_TC_TIMING
 __device__ long long g_core_timing[256][16];
 #define CORE_STAMP(slot) do { if (T == 0 && warp == 0 && blockIdx.x < 256) g_core_timing[blockIdx.x][slot] = clock64(); } while (0)
+__device__ long long g_core_wait[256][8];       // per CTA: cycles warp 0 spent waiting for the MMAs, per (stage, slot)
+#define CORE_WAIT_BEGIN() long long wt0_ = clock64()
+#define CORE_WAIT_END(idx) do { if (T == 0 && warp == 0 && blockIdx.x < 256) g_core_wait[blockIdx.x][idx] += clock64() - wt0_; } while (0)
 #else
 #define CORE_STAMP(slot) do { } while (0)
+#define CORE_WAIT_BEGIN() do { } while (0)
+#define CORE_WAIT_END(idx) do { } while (0)
 #endif
 
 // =====================================================================================
@@ -438,7 +443,9 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
       for (int stage = 0; stage < 4 && ok; ++stage) {
 #pragma unroll 1
         for (int s2 = 0; s2 < 2 && ok; ++s2) {
+          CORE_WAIT_BEGIN();
           ok = wait4(barD[s2], stage & 1);
+          CORE_WAIT_END(2 * stage + s2);
           if (!ok) break;
           if (pair == blockIdx.x && stage == 0 && s2 == 0) CORE_STAMP(1);
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
