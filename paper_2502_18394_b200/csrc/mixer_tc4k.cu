@@ -26,18 +26,16 @@
 
 #include <cstdlib>
 
-#include "common.cuh"
+#include "tc_stage.cuh"
 
 namespace spectre {
 
 // ---- shared with mixer_tc.cu (same conventions) ------------------------------------
-constexpr int k4Lbo = 128;                       // bytes between core matrices along K
-constexpr int k4Sbo = 2064;                      // bytes between 8-column groups (2048 + 16 pad; 144 / 2320 measured slower)
-constexpr int k4BBytes = 32 * k4Sbo;             // one 256-column operand in shared memory
-constexpr int k4ImgBytes = k4BBytes;             // the workspace holds the same image, padding included
+constexpr int k4BBytes = k8BBytes;               // one 256-column operand buffer (largest of the four stage layouts)
+constexpr int k4ImgBytes = 16 * k8Lbo0;          // stage-0 operand image in the workspace (dense: columns 64 c + t2, K = t1)
 constexpr int k4FBytes = 128 * 128 * 2;
-constexpr int k4GStride = 72;                    // gate table: entry (row, col) at row + 72 col
-constexpr int k4GBytes = 64 * k4GStride * 4;
+constexpr int k4GStride = k8GStride;             // gate table: entry (k1, k2) at 72 k2 + k1, bin kM = k1 + 64 k2
+constexpr int k4GBytes = k8GBytes;
 constexpr int k4OutBytes = 4096 * 4 * 4;         // unit result: [t'][4 pairs] half2
 constexpr int k4EpiWarps = 16;
 constexpr int k4EpiThreads = 32 * k4EpiWarps;
@@ -81,9 +79,9 @@ __device__ __forceinline__ void ld16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) 
 }
 __device__ __forceinline__ void ld_wait4() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// XOR skew of a tile's words inside a 32-word line: the 8 tiles a warp touches at once land in
-// 8 different bank groups (flips the t1 % 4 and t2 % 2 bits of the word index)
-__device__ __forceinline__ int tile_skew(int tile) { return (tile & 3) | (((tile >> 2) & 1) << 4); }
+// XOR skew of the low five bits of a staged word's index: the 8 tiles x 4 pairs a warp writes at once
+// land in 32 different banks
+__device__ __forceinline__ int stage_skew(int tile, int c4) { return (tile & 7) | (c4 << 3); }
 
 // forward-scale of the radix-R step (keeps fp16 magnitudes near the input's)
 __host__ __device__ constexpr float in_scale(int R) {
@@ -134,10 +132,10 @@ __device__ __forceinline__ void tc_gate_body(const TcGateParams& p, int sk, floa
   if (threadIdx.x == 0) p.gscale[sk] = m;
   uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * k4GBytes);
   for (int idx = threadIdx.x; idx < 64 * k4GStride; idx += 256) {
-    const int col = idx / k4GStride, row = idx - col * k4GStride;     // kM = col + 64 row
+    const int k2 = idx / k4GStride, k1 = idx - k2 * k4GStride;        // kM = k1 + 64 k2
     uint32_t v = 0u;
-    if (row < 64) {
-      const float2 gv2 = vals[col + 64 * row];
+    if (k1 < 64) {
+      const float2 gv2 = vals[k1 + 64 * k2];
       v = h2pack(gv2.x * inv, gv2.y * inv);
     }
     img[idx] = v;
@@ -162,7 +160,7 @@ template <int R, bool F16>
 __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const TcGateParams gp, int ngate) {
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
-  extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][NT2/2][32 words]; >= 32 KB
+  extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][4 pairs][NT2][4 t1] words (skewed); >= 32 KB
   asm volatile("griddepcontrol.wait;" ::: "memory");          // launched as a programmatic dependent
   if ((int)blockIdx.x < ngate) {
     tc_gate_body(gp, (int)blockIdx.x, reinterpret_cast<float2*>(stage));
@@ -205,10 +203,10 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const
       Dft<R, false>::run(x);
       const float2 w1 = tws[rs];
       if (live) {
-        // word inside the 128-byte core matrix: (t2 % 2, c4, t1 % 4), XOR-skewed by the tile
-        const int wl = ((t2l & 1) * 16 + c4 * 4 + t1m) ^ tile_skew(tile);
-        uint32_t* ps = stage + (tile * (NT2 / 2) + (t2l >> 1)) * 32 + wl;
-        const int sstride = p.ntile * (NT2 / 2) * 32;             // words between consecutive k1
+        // word of the unit's slice [c4][t2][t1 % 4], XOR-skewed in its low five bits
+        const int wl = ((c4 * NT2 + t2l) * 4 + t1m) ^ stage_skew(tile, c4);
+        uint32_t* ps = stage + tile * (16 * NT2) + wl;
+        const int sstride = p.ntile * (16 * NT2);                  // words between consecutive k1
         float2 w = make_float2(sc, 0.f);                          // sc * W_n^{k1 t'}
 #pragma unroll
         for (int k1 = 0; k1 < R; ++k1) {
@@ -220,24 +218,23 @@ __global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const
     }
   }
   __syncthreads();
-  // copy out: one 128-byte line per (k1, tile, t2 pair)
-  const int nlines = R * p.ntile * (NT2 / 2);
-  // 16-byte chunks: chunk index = line * 8 + q; (k1, tile) pairs are consecutive units, so
-  // line -> unit is a shift.  The tile skew permutes words inside a chunk (low two bits) and
-  // swaps the two 64-byte halves of the line (bit 4).
-  unsigned char* img0 = p.ws_in + (size_t)slab_local * R * p.ntile * k4ImgBytes + (size_t)(t2b * (NT2 / 2)) * k4Sbo +
-                        (size_t)t1g * k4Lbo;
+  // copy out: per (k1, tile) unit and pair c4 the CTA holds NT2 consecutive t2 x 4 t1 = NT2 16-byte
+  // chunks, contiguous in the unit's image (column 64 c4 + t2, K group t1g).  The skew permutes the
+  // words inside a chunk (low two bits) and the chunks among their neighbours (next three bits).
+  unsigned char* img0 = p.ws_in + (size_t)slab_local * R * p.ntile * k4ImgBytes + (size_t)t1g * k8Lbo0 +
+                        (size_t)(t2b * NT2) * 16;
   const bool pow2 = (p.ntile & (p.ntile - 1)) == 0;
-  for (int idx = threadIdx.x; idx < nlines * 8; idx += 256) {
-    const int line = idx >> 3, q16 = idx & 7;
-    const int t2p = line & (NT2 / 2 - 1), ut = line / (NT2 / 2);     // ut = k1 * ntile + tile
+  const int nchunk = R * p.ntile * 4 * NT2;
+  for (int idx = threadIdx.x; idx < nchunk; idx += 256) {
+    const int lc = idx & (4 * NT2 - 1), ut = idx / (4 * NT2);        // logical chunk c4 * NT2 + t2l; ut = k1 * ntile + tile
+    const int c4 = lc / NT2, t2l = lc - c4 * NT2;
     const int tile = pow2 ? (ut & (p.ntile - 1)) : (ut % p.ntile);
-    const int sk = tile_skew(tile);
-    const uint4 v = *reinterpret_cast<const uint4*>(stage + line * 32 + ((q16 ^ (sk >> 2)) << 2));
+    const int sk = stage_skew(tile, c4);
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + ut * (16 * NT2) + ((lc ^ (sk >> 2)) << 2));
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     uint4 o;
     o.x = w[0 ^ (sk & 3)]; o.y = w[1 ^ (sk & 3)]; o.z = w[2 ^ (sk & 3)]; o.w = w[3 ^ (sk & 3)];
-    *reinterpret_cast<uint4*>(img0 + (size_t)ut * k4ImgBytes + t2p * k4Sbo + q16 * 16) = o;
+    *reinterpret_cast<uint4*>(img0 + (size_t)ut * k4ImgBytes + c4 * 1024 + t2l * 16) = o;
   }
 }
 
@@ -261,33 +258,23 @@ struct TcCoreParams {
   const unsigned char* gimg;
   unsigned char* ws_out;
   const __half* F;
-  const float2* tw;         // quarter-wave twiddle table (8192nds)
+  const float4* tw64;       // stage twiddles W_4096^{row d} in epilogue order
   int nunits, ntile;
   int* status;
 };
 
-// Epilogue of one MMA stage for one warp (TMEM lane quadrant q, 64-column quarter cq); TMEM loads
-// run one 32-column chunk ahead of the arithmetic.
-//   MODE 1: twiddle W_4096^{row col}; next operand gets (row digit -> column, col digit -> K)
-//   MODE 2: gate, conjugate;           next operand gets (col digit -> column, row digit -> K)
-//   MODE 3: final: store the unit's result [t' = 64 row + col][pair] as half2
-template <int MODE>
-__device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bsm, const uint32_t* Gsm,
-                                              unsigned char* out, int q, int cq, int T,
-                                              const float2* __restrict__ tw) {
+// Last epilogue of a unit for one warp (TMEM lane quadrant q, 64-column quarter cq): the accumulator
+// has rows s2 and columns 4 s1 + c (tc_stage.cuh); the unit's result [t' = 64 row + s1][pair] goes to
+// the workspace as half2, two pairs per 8-byte store.  TMEM loads run one 32-column chunk ahead.
+__device__ __forceinline__ void core_store(uint32_t tmem_d, unsigned char* out, int q, int cq, int T) {
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
   ld16x256b_x4(taddr0, r[0]);
-  float2 w = make_float2(1.f, 0.f), wstep = w;
 #pragma unroll
   for (int step = 0; step < 4; ++step) {                        // step = 2 j + chunk
     const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
-    if (MODE == 1 && chunk == 0) {
-      w = twiddle8192(tw, 2u * (unsigned)((row * (16 * cq + p)) & 4095));
-      wstep = twiddle8192(tw, 4u * (unsigned)row);
-    }
     ld_wait4();
     if (step < 3) {
       const int ns = step + 1;
@@ -295,35 +282,13 @@ __device__ __forceinline__ void core_epilogue(uint32_t tmem_d, unsigned char* Bs
     }
     const uint32_t (&rr)[16] = r[step & 1];
     const int grp0 = 8 * cq + 4 * chunk;                        // first 8-column group of the chunk
-    uint32_t base;
-    if (MODE == 1) base = (uint32_t)((row >> 1) * k4Sbo + (4 * (row & 1) + 2 * cp) * 16 + (grp0 >> 1) * k4Lbo + 4 * p);
-    else if (MODE == 2) base = (uint32_t)(grp0 * k4Sbo + (4 * p + 2 * cp) * 16 + (row >> 2) * k4Lbo + (row & 3) * 4);
-    else base = (uint32_t)(((64 * row + 2 * grp0 + p) * 4 + 2 * cp) * 4);
+    const uint32_t base = (uint32_t)(((64 * row + 2 * grp0 + p) * 4 + 2 * cp) * 4);
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
-      float2 v0 = make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
-      float2 v1 = make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
-      if (MODE == 1) {
-        v0 = cmul(v0, w);
-        v1 = cmul(v1, w);
-        w = cmul(w, wstep);
-        const uint32_t off = base + (x >> 1) * k4Lbo + (x & 1) * 8;
-        *reinterpret_cast<uint32_t*>(Bsm + off) = h2pack(v0.x, v0.y);
-        *reinterpret_cast<uint32_t*>(Bsm + off + 16) = h2pack(v1.x, v1.y);
-      } else if (MODE == 2) {
-        const int col = 2 * (grp0 + x) + p;
-        const float2 g = h2unpack(Gsm[row + k4GStride * col]);
-        v0 = cmul(v0, g);
-        v1 = cmul(v1, g);
-        const uint32_t off = base + x * k4Sbo;
-        *reinterpret_cast<uint32_t*>(Bsm + off) = h2pack(v0.x, -v0.y);
-        *reinterpret_cast<uint32_t*>(Bsm + off + 16) = h2pack(v1.x, -v1.y);
-      } else {
-        uint2 o;
-        o.x = h2pack(v0.x, v0.y);
-        o.y = h2pack(v1.x, v1.y);
-        *reinterpret_cast<uint2*>(out + base + x * 32) = o;
-      }
+      uint2 o;
+      o.x = h2pack(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
+      o.y = h2pack(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
+      *reinterpret_cast<uint2*>(out + base + x * 32) = o;
     }
   }
 }
@@ -410,10 +375,12 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           if (T == 0) {
             const uint32_t a0 = s_u32(Fsm), b0 = s_u32(Bsm[s2]);
+            const uint32_t lbo = stage == 0 ? k8Lbo0 : (stage == 1 ? k8Lbo1 : (stage == 2 ? k8Lbo2 : k8Lbo3));
+            const uint32_t sbo = stage == 0 ? k8Sbo0 : (stage == 1 ? k8Sbo1 : (stage == 2 ? k8Sbo2 : k8Sbo3));
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
               const uint64_t da = desc4(a0 + ks * 256, 128, 2048);
-              const uint64_t db = desc4(b0 + ks * 2 * k4Lbo, k4Lbo, k4Sbo);
+              const uint64_t db = desc4(b0 + ks * 2 * lbo, lbo, sbo);
               const uint32_t acc = ks > 0;
               asm volatile(
                   "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
@@ -451,10 +418,10 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t td = tmem + 256 * s2;
           const int unit = 2 * pair + s2;
-          if (stage == 1) core_epilogue<2>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T, p.tw);
-          else if (stage == 3) {
-            if (unit < p.nunits) core_epilogue<3>(td, Bsm[s2], Gsm[s2], p.ws_out + (size_t)unit * k4OutBytes, q, cq, T, p.tw);
-          } else core_epilogue<1>(td, Bsm[s2], Gsm[s2], nullptr, q, cq, T, p.tw);
+          if (stage == 0) epilogue_twiddle<k8Lbo1, k8Sbo1, true>(td, Bsm[s2], q, cq, T, p.tw64);
+          else if (stage == 1) epilogue_gate(td, Bsm[s2], q, cq, T, Gsm[s2]);
+          else if (stage == 2) epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bsm[s2], q, cq, T, p.tw64);
+          else if (unit < p.nunits) core_store(td, p.ws_out + (size_t)unit * k4OutBytes, q, cq, T);
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           if (pair == blockIdx.x) CORE_STAMP(2 + 2 * stage + s2);
@@ -611,7 +578,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   SPECTRE_LAUNCH_OK("tc_in_kernel");
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
-                     reinterpret_cast<const float2*>(ctx->tw8192), (int)nunits, ntile, ctx->status_dev};
+                     reinterpret_cast<const float4*>(ctx->tw64x64), (int)nunits, ntile, ctx->status_dev};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
   int grid = (int)((nunits + 1) / 2);               // pairs of units
   if (grid > ctx->sm_count) grid = ctx->sm_count;

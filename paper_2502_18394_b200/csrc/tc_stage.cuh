@@ -1,0 +1,94 @@
+// The 64 x 64 stages of a 4096-point transform on the tensor cores, shared by the n = 8192 kernel
+// (two such problems per tile) and the core kernel of the longer transforms (one per unit): operand
+// strides per stage and the epilogues between the stages.  Conventions as in mixer_tc8k.cu: the
+// accumulator of a stage has the new digit along its rows and, along its columns, the column pair c
+// and the digit that is contracted next.
+#pragma once
+#include "tc_common.cuh"
+
+namespace spectre {
+
+// Operand strides (bytes) per stage: LBO between core matrices along K, SBO between 8-column
+// groups.  Stage 0 is the TMA landing image (dense).  The others are chosen so that the stores
+// of the epilogue that writes them spread over all 32 banks.
+constexpr int k8Lbo0 = 4096, k8Sbo0 = 128;       // columns 64 c + t2, K = t1
+constexpr int k8Lbo1 = 4160, k8Sbo1 = 128;       // columns 64 c + k1, K = t2
+constexpr int k8Lbo2 = 4112, k8Sbo2 = 128;       // columns 64 c + k1, K = k2
+constexpr int k8Lbo3 = 144, k8Sbo3 = 2336;       // columns 4 s1 + c,  K = k1
+constexpr int k8BBytes = 32 * k8Sbo3;            // largest of the four images (74752)
+constexpr int k8GStride = 72;                    // gate table: entry (k1, k2) at 72 k2 + k1
+constexpr int k8GBytes = 64 * k8GStride * 4;     // per half, fp16 (re, im)
+
+// Epilogue after a stage whose accumulator has columns 64 c + d (d = the digit still to be
+// contracted), for one warp: TMEM lane quadrant q, pair c.  A thread owns rows (new digit)
+// 16 q' + T/4 for the two lane groups q' = 2q, 2q+1 and the columns d = 32 chunk + 8 x + 2 (T%4)
+// + {0, 1}.  It multiplies by W_4096^{row d} (read from a table laid out in this thread order, one
+// 16-byte load per x) and writes the transposed operand (row -> column index, d -> K) as one
+// 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
+//   COLS64: output columns 64 c + row (else 4 row + c).
+template <int LBO, int SBO, bool COLS64>
+__device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
+                                                 const float4* __restrict__ tw) {
+  const int i = T >> 2, tq = T & 3;
+  uint32_t r[2][16];
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * c;
+  tmem_ld_16x256b_x4(taddr0, r[0]);
+  tw += q * 512 + T;
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {                      // step = 2 j + chunk
+    const int j = step >> 1, chunk = step & 1;
+    const int row = 8 * (2 * q + j) + i;
+    float4 w[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) w[x] = __ldg(tw + (4 * step + x) * 32);
+    tmem_ld_wait();
+    if (step < 3) {
+      const int nj = (step + 1) >> 1, nchunk = (step + 1) & 1;
+      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * nj) << 16) + 32 * nchunk, r[(step + 1) & 1]);
+    }
+    const uint32_t (&rr)[16] = r[step & 1];
+    const uint32_t colpart = COLS64 ? (uint32_t)((8 * c + (row >> 3)) * SBO + (row & 7) * 16)
+                                    : (uint32_t)((row >> 1) * SBO + (4 * (row & 1) + c) * 16);
+    const uint32_t base = colpart + (uint32_t)((8 * chunk + (tq >> 1)) * LBO + 8 * (tq & 1));
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), make_float2(w[x].x, w[x].y));
+      const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), make_float2(w[x].z, w[x].w));
+      *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
+    }
+  }
+}
+
+// Epilogue after the second forward stage: rows k2, columns 64 c + k1; bin 2 (k1 + 64 k2) + parity
+// of the half.  Gate, conjugate (for the inverse by the conj trick) and write the operand with
+// the same columns and K = k2.
+__device__ __forceinline__ void epilogue_gate(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
+                                              const uint32_t* __restrict__ Gtab) {
+  const int i = T >> 2, tq = T & 3;
+  uint32_t r[2][16];
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * c;
+  tmem_ld_16x256b_x4(taddr0, r[0]);
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    const int j = step >> 1, chunk = step & 1;
+    const int row = 8 * (2 * q + j) + i;
+    tmem_ld_wait();
+    if (step < 3) {
+      const int nj = (step + 1) >> 1, nchunk = (step + 1) & 1;
+      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * nj) << 16) + 32 * nchunk, r[(step + 1) & 1]);
+    }
+    const uint32_t (&rr)[16] = r[step & 1];
+    const uint32_t base = (uint32_t)((8 * c + 4 * chunk) * k8Sbo2 + (2 * tq) * 16 + (row >> 2) * k8Lbo2 + (row & 3) * 4);
+    const uint32_t* grow = Gtab + k8GStride * row + 32 * chunk + 2 * tq;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const uint2 gp = *reinterpret_cast<const uint2*>(grow + 8 * x);
+      const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), unpack_h2(gp.x));
+      const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), unpack_h2(gp.y));
+      *reinterpret_cast<uint32_t*>(Bout + base + x * k8Sbo2) = pack_h2(v0.x, -v0.y);
+      *reinterpret_cast<uint32_t*>(Bout + base + x * k8Sbo2 + 16) = pack_h2(v1.x, -v1.y);
+    }
+  }
+}
+
+}  // namespace spectre
