@@ -243,7 +243,13 @@ __global__ void __launch_bounds__(256) decode_reduce_kernel(const float* __restr
   int c = idx % D, h = (idx / D) % H, r = (idx / (D * H)) % nrows, b = idx / (D * H * nrows);
   const float* p = partial + (((size_t)(b * H + h) * nblk) * NR + r) * D + c;
   float s = 0.f;
-  for (int blk = 0; blk < nblk; ++blk) s += p[(size_t)blk * NR * D];
+  for (int blk0 = 0; blk0 < nblk; blk0 += 16) {              // 16 partials in flight; the order of the sum is fixed
+    float v[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) v[u] = blk0 + u < nblk ? __ldg(p + (size_t)(blk0 + u) * NR * D) : 0.f;
+#pragma unroll
+    for (int u = 0; u < 16; ++u) s += v[u];
+  }
   io<T>::store1(y + idx, s);
 }
 
