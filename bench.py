@@ -322,9 +322,9 @@ class MixerBench:
 class AppendBench:
     """One Prefix-FFT cache append per step (decode)."""
 
-    def __init__(self, w: W.Workload, dev, nsets=None, decode=False):
+    def __init__(self, w: W.Workload, dev, nsets=None, decode=False, prefill=False):
         from paper_2502_18394_b200 import binding as S
-        self.S, self.w, self.dev, self.decode = S, w, dev, decode
+        self.S, self.w, self.dev, self.decode, self.prefill = S, w, dev, decode, prefill
         self.ctx = S.Context(dev.index)
         self.cache = S.PrefixCache(w.B, w.H, w.D, w.N_max, dtype=W.torch_dtype(w.dtype), device=dev)
         # state: a full window of random tokens (prefill through the library)
@@ -332,8 +332,23 @@ class AppendBench:
         ws = torch.empty(max(S.spectre_prefill_workspace_bytes(self.ctx, w.B, w.H, w.D, w.N_max), 16), dtype=torch.uint8, device=dev)
         q = torch.cat([W.activations(half, stream=10 + b) for b in range(w.B)], dim=0).to(dev)
         S.spectre_prefix_cache_prefill(self.ctx, self.cache, q, q, workspace=ws)
-        del ws, q
         self.nsets = 1
+        if prefill:
+            # the timed call is the prefill of the whole window itself (prompt of N_max tokens per batch entry)
+            self.pf_q, self.pf_v, self.pf_ws = q, q.clone(), ws
+            es = 4 if w.dtype == "f32" else 2
+            K = w.N_max // 2 + 1
+            self.units_per_step = w.B * w.N_max
+            tok = w.B * w.N_max * w.H * w.D * es
+            self.alg_bytes = 4 * tok + w.B * w.H * K * w.D * 8            # read q, v; write both rings; write the spectrum
+            self.kernel_name = "spectre_prefix_cache_prefill (fp32 transforms per group of heads + split, ring fills, pooling)"
+            per = w.N_max * (w.D // 2) * 8
+            groups = -(-(w.B * w.H) // max(1, min(w.B * w.H, ws.numel() // per)))
+            self.launches_per_step = 3 * groups + 3                       # (strided, on-chip, split) per group; 2 ring fills; pooling
+            self.h2d, self.d2h = 2 * tok, w.B * w.H * w.D * 4
+            self.q_host = self.v_host = None
+            return
+        del ws, q
         qs, vs = W.decode_tokens(w, 64)
         self.q_host, self.v_host = qs, vs
         self.qd, self.vd = qs.to(dev), vs.to(dev)
@@ -369,6 +384,13 @@ class AppendBench:
         return self.S.prepare_append(self.ctx, self.cache, self.qd[i], self.vd[i], self.t0 + k)
 
     def step(self, k: int, e0=None, e1=None):
+        if self.prefill:
+            if e0 is not None:
+                e0.record()
+            self.S.spectre_prefix_cache_prefill(self.ctx, self.cache, self.pf_q, self.pf_v, workspace=self.pf_ws)
+            if e1 is not None:
+                e1.record()
+            return
         c = self._call(k)
         if e0 is not None:
             e0.record()
@@ -377,6 +399,11 @@ class AppendBench:
             e1.record()
 
     def e2e_prepare(self):
+        if self.prefill:
+            self.pin_q = self.pf_q.cpu().pin_memory()
+            self.pin_v = self.pf_v.cpu().pin_memory()
+            self.pin_s = torch.empty((self.w.B, self.w.H, self.w.D), dtype=torch.float32).pin_memory()
+            return
         self.pin_q = self.q_host.pin_memory()
         self.pin_v = self.v_host.pin_memory()
         self.pin_s = torch.empty((self.w.B, self.w.H, self.w.D), dtype=torch.float32).pin_memory()
@@ -384,6 +411,12 @@ class AppendBench:
             self.pin_s = torch.empty_like(self.y_rows, device="cpu").pin_memory()
 
     def e2e_step(self, k: int):
+        if self.prefill:
+            self.pf_q.copy_(self.pin_q, non_blocking=True)
+            self.pf_v.copy_(self.pin_v, non_blocking=True)
+            self.S.spectre_prefix_cache_prefill(self.ctx, self.cache, self.pf_q, self.pf_v, workspace=self.pf_ws)
+            self.pin_s.copy_(self.cache.sum_q, non_blocking=True)
+            return
         i = k % 64
         self.qd[i].copy_(self.pin_q[i], non_blocking=True)
         self.vd[i].copy_(self.pin_v[i], non_blocking=True)
@@ -403,6 +436,12 @@ class AppendBench:
         st = {"N": N, "prefix_fft": np.zeros((1, w.H, K, w.D), dtype=np.complex128),
               "V_buf": rng.standard_normal((1, N, w.H, w.D)), "Q_buf": rng.standard_normal((1, N, w.H, w.D)),
               "sum_q": np.zeros((1, w.H, w.D))}
+        if getattr(self, "prefill", False):
+            # bounded sample: the prefill of one head of one batch entry (N_max tokens), scaled to tokens/s
+            qs = rng.standard_normal((1, N, 1, w.D))
+            t0 = time.perf_counter()
+            O.cache_prefill(qs, qs, N)
+            return time.perf_counter() - t0, N / w.H
         q = W.to_f64(self.q_host[0][:1]); v = W.to_f64(self.v_host[0][:1])
         if getattr(self, "decode", False):
             gp = W.gate_params(W.scaled(w, n_fft=N))
@@ -416,8 +455,8 @@ class AppendBench:
         return time.perf_counter() - t0, 1
 
 
-def make_bench(w, dev, nsets, decode=False, backward=False, project=False, shared_gates=False):
-    return AppendBench(w, dev, nsets, decode) if w.N_max else MixerBench(w, dev, nsets, backward, project, shared_gates)
+def make_bench(w, dev, nsets, decode=False, backward=False, project=False, shared_gates=False, prefill=False):
+    return AppendBench(w, dev, nsets, decode, prefill) if w.N_max else MixerBench(w, dev, nsets, backward, project, shared_gates)
 
 
 # --------------------------------------------------------------------------- arms
@@ -427,7 +466,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     torch.set_num_threads(1)
-    bench = _cpu_only_bench(w)
+    bench = _cpu_only_bench(w, getattr(args, "prefill", False))
     for _ in range(min(args.warmup, 1)):
         bench.cpu_step()
     tot, units = 0.0, 0
@@ -446,12 +485,15 @@ def run_reference(args, w):
     print(json.dumps(out))
 
 
-def _cpu_only_bench(w):
+def _cpu_only_bench(w, prefill=False):
     """A bench object whose GPU side is never built (the reference arm runs without the library)."""
     cls = AppendBench if w.N_max else MixerBench
     b = cls.__new__(cls)
     b.w = w
-    if w.N_max:
+    b.prefill = prefill
+    if w.N_max and prefill:
+        b.sample_note = "the prefill of one head of one batch entry (N_max tokens), scaled to tokens/s"
+    elif w.N_max:
         qs, vs = W.decode_tokens(w, 1)
         b.q_host, b.v_host = qs, vs
         b.sample_note = "one batch row (all heads) of one append, scaled to tokens/s"
@@ -478,6 +520,7 @@ def main():
     ap.add_argument("--project", action="store_true", help="mixer workloads (bf16, d = 64): step = projections + gate from sum_q + mixer; the timed call is the projection")
     ap.add_argument("--backward", action="store_true", help="mixer workloads: step = gate + forward + backward; the timed call is the backward")
     ap.add_argument("--decode", action="store_true", help="c4: time the whole decode step (gate + fused update/read-out)")
+    ap.add_argument("--prefill", action="store_true", help="c4: time the prefill of the whole window (N_max tokens per batch entry)")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
     if args.heads:
@@ -500,12 +543,12 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     base = args.workload
     default_steps = {"c1": 2000, "c2": 2000, "c3": 100, "c4": 200, "c5": 500}[base]
-    K = args.steps if args.steps is not None else default_steps
+    K = args.steps if args.steps is not None else (30 if getattr(args, "prefill", False) else default_steps)
     Wm = max(3, args.warmup if args.warmup is not None else 10)
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
-    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project, args.shared_gates)
+    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project, args.shared_gates, args.prefill)
 
     for k in range(Wm):
         bench.step(k)
@@ -534,7 +577,7 @@ def main():
     tot_ms, tot_units = R.aggregate(elapsed_ms, bench.units_per_step * K, dev)
 
     # end to end: host buffers, copies inside the timed region
-    Ke = max(3, min(K, 30))
+    Ke = 3 if args.prefill else max(3, min(K, 30))
     bench.e2e_prepare()
     for k in range(3):
         bench.e2e_step(k)
@@ -559,7 +602,7 @@ def main():
             tot += dt
             units += u
             reps += 1
-        note = _cpu_only_bench(w).sample_note + f", {reps} repetition(s)"
+        note = _cpu_only_bench(w, args.prefill).sample_note + f", {reps} repetition(s)"
         cpu = {"value": units / tot, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": note}
 
     if rank == 0:
@@ -569,7 +612,7 @@ def main():
             "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" + backward" if args.backward else "") + (" with token projections in front (gate from their sum_q)" if args.project else "") + (", gate shared across heads" if args.shared_gates else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" - prefill of the whole window" if args.prefill else "") + (" + backward" if args.backward else "") + (" with token projections in front (gate from their sum_q)" if args.project else "") + (", gate shared across heads" if args.shared_gates else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
                        "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
                        "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
                              if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},
@@ -582,7 +625,7 @@ def main():
                          "kernel_ms": kern_ms, "kernel_timed_steps": len([e for e in e0 if e is not None]),
                          "frac_of_8000": achieved / 8000.0,
                          "kernel_tokens_per_s": bench.units_per_step / (kern_ms * 1e-3),
-                         "traffic": None if (args.project or args.backward or args.decode) else NCU_TRAFFIC_BYTES.get(w.name)},   # None for reduced cases and variant legs
+                         "traffic": None if (args.project or args.backward or args.decode or args.prefill) else NCU_TRAFFIC_BYTES.get(w.name)},   # None for reduced cases and variant legs
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
