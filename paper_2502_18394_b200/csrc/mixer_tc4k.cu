@@ -157,7 +157,7 @@ struct TcInParams {
 // (k1, tile), the core matrices (8 operand columns x 16 bytes) of this CTA's slice.
 // The first ngate CTAs write the gate images (tc_gate_body) instead.
 template <int R, bool F16>
-__global__ void __launch_bounds__(256, 2) tc_in_kernel(const TcInParams p, const TcGateParams gp, int ngate) {
+__global__ void __launch_bounds__(256, 3) tc_in_kernel(const TcInParams p, const TcGateParams gp, int ngate) {
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   constexpr int UNR = R <= 2 ? 4 : (R <= 8 ? 2 : 1);          // row sets in flight per warp
   extern __shared__ __align__(128) uint32_t stage[];          // [R][ntile][4 pairs][NT2][4 t1] words (skewed); >= 32 KB
@@ -452,7 +452,7 @@ struct TcOutParams {
 
 // CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.
 template <int R, bool F16>
-__global__ void __launch_bounds__(256, 2) tc_out_kernel(const TcOutParams p) {
+__global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
   constexpr int NT = 512 / R;
   extern __shared__ __align__(128) uint32_t stage[];            // [R][NT][D/2 words]
   const int nblk = 4096 / NT;
