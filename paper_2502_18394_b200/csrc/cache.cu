@@ -43,23 +43,28 @@ __global__ void __launch_bounds__(256) split_kernel(const float2* __restrict__ w
   *reinterpret_cast<float4*>(prefix + o) = out;
 }
 
-// Ring buffers: rows 0..L-1 <- tokens, rows L..N-1 <- 0 (Alg. 1 PreFill).
+// Ring buffers: rows 0..L-1 <- tokens, rows L..N-1 <- 0 (Alg. 1 PreFill).  A CTA copies kRingRows
+// consecutive rows of one batch entry, a thread one 16-byte piece of each with all of them in flight.
+constexpr int kRingRows = 8;
 template <typename T>
 __global__ void __launch_bounds__(256) ring_fill_kernel(const T* __restrict__ src, int64_t sb, int64_t sl, int64_t sh,
                                                         T* __restrict__ buf, int B, int N, int H, int D, int L) {
   constexpr int V = 16 / sizeof(T);
   const int vec_per_row = H * D / V;
-  const size_t total = (size_t)B * N * vec_per_row;
-  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= total) return;
-  int vi = (int)(idx % vec_per_row);
-  size_t r = idx / vec_per_row;
-  int row = (int)(r % N);
-  int b = (int)(r / N);
-  int e = vi * V, h = e / D, c = e - h * D;
-  uint4 val = make_uint4(0u, 0u, 0u, 0u);
-  if (row < L) val = *reinterpret_cast<const uint4*>(src + b * sb + (int64_t)row * sl + h * sh + c);
-  *reinterpret_cast<uint4*>(buf + (((size_t)b * N + row) * H + h) * D + c) = val;
+  const int chunks = (N + kRingRows - 1) / kRingRows;
+  const int b = blockIdx.x / chunks, r0 = (blockIdx.x - b * chunks) * kRingRows;
+  for (int vi = threadIdx.x; vi < vec_per_row; vi += blockDim.x) {
+    const int e = vi * V, h = e / D, c = e - h * D;
+    const T* s = src + b * sb + h * sh + c;
+    T* d = buf + (((size_t)b * N + r0) * H + h) * D + c;
+    uint4 val[kRingRows];
+#pragma unroll
+    for (int u = 0; u < kRingRows; ++u)
+      val[u] = (r0 + u < L) ? __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)(r0 + u) * sl)) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int u = 0; u < kRingRows; ++u)
+      if (r0 + u < N) __stcs(reinterpret_cast<uint4*>(d + (size_t)u * H * D), val[u]);
+  }
 }
 
 // ---- append ------------------------------------------------------------------
@@ -316,9 +321,9 @@ extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, cons
     split_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, cache->prefix_fft, N, K, D, N1, M, s0, cnt);
     SPECTRE_LAUNCH_OK("split_kernel");
   }
-  const int V = 16 / io_elem_bytes(cache->buf_dtype);
-  size_t total = (size_t)B * N * (H * D / V);
-  unsigned blocks = (unsigned)((total + 255) / 256);
+  const size_t nblocks = (size_t)B * ((N + kRingRows - 1) / kRingRows);
+  if (nblocks > 0x7fffffffu) return fail(SPECTRE_ERR_UNSUPPORTED, "B * N_max too large for the ring copy");
+  unsigned blocks = (unsigned)nblocks;
   SPECTRE_IO_DISPATCH(cache->buf_dtype, {
     ring_fill_kernel<T><<<blocks, 256, 0, st>>>(reinterpret_cast<const T*>(v->ptr), v->stride_b, v->stride_l, v->stride_h,
                                                 reinterpret_cast<T*>(cache->V_buf), B, N, H, D, v->L);
