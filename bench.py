@@ -433,15 +433,15 @@ class AppendBench:
         w = self.w
         rng = np.random.default_rng(0)
         N, K = w.N_max, w.N_max // 2 + 1
-        st = {"N": N, "prefix_fft": np.zeros((1, w.H, K, w.D), dtype=np.complex128),
-              "V_buf": rng.standard_normal((1, N, w.H, w.D)), "Q_buf": rng.standard_normal((1, N, w.H, w.D)),
-              "sum_q": np.zeros((1, w.H, w.D))}
         if getattr(self, "prefill", False):
             # bounded sample: the prefill of one head of one batch entry (N_max tokens), scaled to tokens/s
             qs = rng.standard_normal((1, N, 1, w.D))
             t0 = time.perf_counter()
             O.cache_prefill(qs, qs, N)
             return time.perf_counter() - t0, N / w.H
+        st = {"N": N, "prefix_fft": np.zeros((1, w.H, K, w.D), dtype=np.complex128),
+              "V_buf": rng.standard_normal((1, N, w.H, w.D)), "Q_buf": rng.standard_normal((1, N, w.H, w.D)),
+              "sum_q": np.zeros((1, w.H, w.D))}
         q = W.to_f64(self.q_host[0][:1]); v = W.to_f64(self.v_host[0][:1])
         if getattr(self, "decode", False):
             gp = W.gate_params(W.scaled(w, n_fft=N))
