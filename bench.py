@@ -43,7 +43,12 @@ L2_BYTES = 126e6
 # c4: append_spectrum_kernel measured at B = 2 (1015.3 MB), scaled by 4 to B = 8
 # c5: mixer_tc196_kernel at full size: 82.0 MB read + 27.6 MB written by the end of the launch (the rest of
 #     the 77 MB output is still in L2 then)
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": 36.9e6, "c3": 3126e6, "c4": 4061e6, "c5": 109.6e6}
+# Not measured by this run: each entry names the committed summary it was read from.
+NCU_TRAFFIC = {"c1": None,
+               "c2": (36.9e6, "profiles/mixer_tc8192_kernel_c2.md (ncu capture, not this run)"),
+               "c3": (3126e6, "profiles/launches_c3_gate_mixer.md (ncu capture, not this run)"),
+               "c4": (4061e6, "profiles/append_spectrum_kernel_c4_batch2.md (ncu capture at B = 2, x4; not this run)"),
+               "c5": (109.6e6, "profiles/launches_c5_and_kernels.md (ncu capture, not this run)")}
 
 
 def measured_peak():
@@ -115,7 +120,7 @@ def describe(w: W.Workload) -> str:
     if w.N_max:
         return (f"{w.name}: Prefix-FFT cache append, B={w.B} H={w.H} d={w.D} N_max={w.N_max}, "
                 f"{w.dtype} tokens, fp32 spectrum")
-    s = f"{w.name}: gate + mixer, B={w.B} H={w.H} d={w.D} L={w.L}, {w.dtype} I/O, fp32 accumulate"
+    s = f"{w.name}: gate + mixer, B={w.B} H={w.H} d={w.D} L={w.L}, {w.dtype} I/O"
     if w.wavelet_levels:
         s += f", Haar J={w.wavelet_levels}"
     return s
@@ -478,9 +483,11 @@ def run_reference(args, w):
     out = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": describe(w)},
+           "config": {"workload": describe(w), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+                      "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{args.gpus} (no sharding)"},
            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": 1, "kind": "oracle",
-                            "sample": bench.sample_note},
+                            "sample": bench.sample_note, "host_cores": os.cpu_count(),
+                            "host_cores_usable": len(os.sched_getaffinity(0))},
            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
 
@@ -513,6 +520,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(W.CONFIGS))
     ap.add_argument("--sets", type=int, default=None, help="rotating buffer sets (default: enough to exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true", help="default workload only: skip the L = 128k block")
     ap.add_argument("--heads", type=int, default=None, help="override H (reduced cases for profiler captures)")
     ap.add_argument("--batch", type=int, default=None, help="override B (reduced cases for profiler captures)")
     ap.add_argument("--io-dtype", default=None, choices=["bf16", "f16", "f32"], help="override the activation dtype (f16 = the paper's inference precision)")
@@ -548,49 +556,9 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
+    variant = args.decode or args.backward or args.project or args.shared_gates or args.prefill
     bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project, args.shared_gates, args.prefill)
-
-    for k in range(Wm):
-        bench.step(k)
-    torch.cuda.synchronize()
-
-    # The dominant call is bracketed by events on every ev_stride-th timed step only: an event between
-    # two kernels keeps the second from starting as the first one's programmatic dependent, so
-    # bracketing every step would change what is measured.
-    ev_stride = 8 if K >= 64 else 1
-    e0 = [torch.cuda.Event(enable_timing=True) if k % ev_stride == 0 else None for k in range(K)]
-    e1 = [torch.cuda.Event(enable_timing=True) if k % ev_stride == 0 else None for k in range(K)]
-    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
-    R.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    ev_a.record()
-    for k in range(K):
-        bench.step(Wm + k, e0[k], e1[k])
-    ev_b.record()
-    torch.cuda.synchronize()
-    R.barrier()
-    clocks = sampler.stop()
-    elapsed_ms = ev_a.elapsed_time(ev_b)
-    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(e0, e1) if a is not None)
-    tot_ms, tot_units = R.aggregate(elapsed_ms, bench.units_per_step * K, dev)
-
-    # end to end: host buffers, copies inside the timed region
-    Ke = 3 if args.prefill else max(3, min(K, 30))
-    bench.e2e_prepare()
-    for k in range(3):
-        bench.e2e_step(k)
-    torch.cuda.synchronize()
-    R.barrier()
-    ev_a.record()
-    for k in range(Ke):
-        bench.e2e_step(3 + k)
-    bench.e2e_finish()
-    ev_b.record()
-    torch.cuda.synchronize()
-    R.barrier()
-    e2e_ms, e2e_units = R.aggregate(ev_a.elapsed_time(ev_b), bench.units_per_step * Ke, dev)
+    m = measure(bench, K, Wm, local_rank, dev, e2e_steps=3 if args.prefill else max(3, min(K, 30)))
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -603,33 +571,134 @@ def main():
             units += u
             reps += 1
         note = _cpu_only_bench(w, args.prefill).sample_note + f", {reps} repetition(s)"
-        cpu = {"value": units / tot, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": note}
+        cpu = {"value": units / tot, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": note,
+               "host_cores": os.cpu_count(), "host_cores_usable": len(os.sched_getaffinity(0))}
+
+    # The metric names two lengths: the default run measures L = 128k (c3) in the same process, after
+    # the L = 8k workload has been released, and reports it beside the headline value.
+    also = None
+    if base == "c2" and not variant and not args.heads and not args.batch and not args.io_dtype and not args.no_also:
+        del bench
+        torch.cuda.empty_cache()
+        w3 = W.CONFIGS["c3"]
+        b3 = make_bench(w3, dev, None)
+        K3 = max(3, min(K, 30))
+        m3 = measure(b3, K3, 3, local_rank, dev, e2e_steps=3)
+        also = {"c3": result_block(w3, b3, m3, K3, 3, world, None)}
+        del b3
+        bench = None
 
     if rank == 0:
-        peak, peak_src = measured_peak()
-        achieved = bench.alg_bytes / (kern_ms * 1e-3) / 1e9
-        out = {
-            "metric": METRIC, "value": tot_units / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
-            "steps": K, "warmup": Wm, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(w) + (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + (" - prefill of the whole window" if args.prefill else "") + (" + backward" if args.backward else "") + (" with token projections in front (gate from their sum_q)" if args.project else "") + (", gate shared across heads" if args.shared_gates else ""), "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
-                       "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
-                       "l2": f"{bench.nsets} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
-                             if bench.nsets > 1 else "one pass touches more bytes than L2 holds"},
-            "clocks": clocks,
-            "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": bench.h2d,
-                    "d2h_bytes_per_step": bench.d2h, "steps": Ke},
-            "gpu_launches": bench.launches_per_step * K,
-            "roofline": {"bound": "hbm", "kernel": bench.kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": bench.alg_bytes,
-                         "kernel_ms": kern_ms, "kernel_timed_steps": len([e for e in e0 if e is not None]),
-                         "frac_of_8000": achieved / 8000.0,
-                         "kernel_tokens_per_s": bench.units_per_step / (kern_ms * 1e-3),
-                         "traffic": None if (args.project or args.backward or args.decode or args.prefill) else NCU_TRAFFIC_BYTES.get(w.name)},   # None for reduced cases and variant legs
-            "cpu_baseline": cpu,
-        }
+        out = {"metric": METRIC}
+        label = (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + \
+                (" - prefill of the whole window" if args.prefill else "") + (" + backward" if args.backward else "") + \
+                (" with token projections in front (gate from their sum_q)" if args.project else "") + \
+                (", gate shared across heads" if args.shared_gates else "")
+        out.update(result_block(w, m["bench_info"], m, K, Wm, world, cpu, label=label, variant=variant))
+        if also is not None:
+            out["also"] = also
         print(json.dumps(out))
     R.finish()
+
+
+def arithmetic_dtype(w) -> str:
+    """What the dominant kernel computes in (not a precision claim about the I/O)."""
+    if w.N_max or w.dtype == "f32":
+        return "f32"
+    tc = w.n == 196 or (w.n >= 4096 and (w.n & (w.n - 1)) == 0)
+    return "f16 tensor-core operands, f32 accumulate (" + w.dtype + " I/O)" if tc else "f32 (" + w.dtype + " I/O)"
+
+
+def measure(bench, K, Wm, local_rank, dev, e2e_steps):
+    """Wm warm-up steps, then windows of exactly K steps each (one window when it lasts >= 50 ms, up to
+    15 otherwise; the median window is reported), then the end-to-end leg."""
+    for k in range(Wm):
+        bench.step(k)
+    torch.cuda.synchronize()
+    # The dominant call is bracketed by events on every ev_stride-th timed step only: an event between
+    # two kernels keeps the second from starting as the first one's programmatic dependent, so
+    # bracketing every step would change what is measured.
+    ev_stride = 8 if K >= 64 else 1
+    sampler = ClockSampler(local_rank)
+    R.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    windows, kern = [], []
+    step0 = Wm
+    while True:
+        e0 = [torch.cuda.Event(enable_timing=True) if k % ev_stride == 0 else None for k in range(K)]
+        e1 = [torch.cuda.Event(enable_timing=True) if k % ev_stride == 0 else None for k in range(K)]
+        ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev_a.record()
+        for k in range(K):
+            bench.step(step0 + k, e0[k], e1[k])
+        ev_b.record()
+        torch.cuda.synchronize()
+        R.barrier()
+        step0 += K
+        ms = ev_a.elapsed_time(ev_b)
+        tot_ms, tot_units = R.aggregate(ms, bench.units_per_step * K, dev)      # max over ranks, summed units
+        windows.append((tot_ms, tot_units))
+        kern.append(statistics.mean(a.elapsed_time(b) for a, b in zip(e0, e1) if a is not None))
+        total = sum(x[0] for x in windows)
+        if len(windows) >= 15 or (len(windows) == 1 and tot_ms >= 50.0) or total >= 400.0:
+            break
+    clocks = sampler.stop()
+    order = sorted(range(len(windows)), key=lambda i: windows[i][0])
+    mid = order[len(order) // 2]
+    tot_ms, tot_units = windows[mid]
+    kern_ms = statistics.median(kern)
+
+    # end to end: host buffers, copies inside the timed region
+    Ke = e2e_steps
+    bench.e2e_prepare()
+    for k in range(3):
+        bench.e2e_step(k)
+    torch.cuda.synchronize()
+    R.barrier()
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev_a.record()
+    for k in range(Ke):
+        bench.e2e_step(3 + k)
+    bench.e2e_finish()
+    ev_b.record()
+    torch.cuda.synchronize()
+    R.barrier()
+    e2e_ms, e2e_units = R.aggregate(ev_a.elapsed_time(ev_b), bench.units_per_step * Ke, dev)
+    info = {k: getattr(bench, k) for k in ("alg_bytes", "kernel_name", "launches_per_step", "h2d", "d2h", "nsets", "units_per_step")}
+    return {"tot_ms": tot_ms, "tot_units": tot_units, "kern_ms": kern_ms, "clocks": clocks, "windows": len(windows),
+            "window_ms": [round(x[0], 4) for x in windows], "kern_events": len([e for e in e0 if e is not None]) * len(windows),
+            "e2e_ms": e2e_ms, "e2e_units": e2e_units, "e2e_steps": Ke, "bench_info": info}
+
+
+def result_block(w, info, m, K, Wm, world, cpu, label="", variant=False):
+    if not isinstance(info, dict):
+        info = m["bench_info"]
+    peak, peak_src = measured_peak()
+    achieved = info["alg_bytes"] / (m["kern_ms"] * 1e-3) / 1e9
+    traffic = None if variant else NCU_TRAFFIC.get(w.name)        # None for reduced cases and variant legs
+    return {
+        "value": m["tot_units"] / (m["tot_ms"] * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        "steps": K, "warmup": Wm, "ms_per_step": m["tot_ms"] / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": arithmetic_dtype(w), "data": "synthetic",
+        "timed_windows": {"count": m["windows"], "steps_each": K, "reported": "median window", "ms": m["window_ms"]},
+        "config": {"workload": describe(w) + label, "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
+                   "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",
+                   "l2": f"{info['nsets']} rotating buffer set(s); inputs+outputs+weights per rotation exceed L2"
+                         if info["nsets"] > 1 else "one pass touches more bytes than L2 holds"},
+        "clocks": m["clocks"],
+        "e2e": {"value": m["e2e_units"] / (m["e2e_ms"] * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": info["h2d"],
+                "d2h_bytes_per_step": info["d2h"], "steps": m["e2e_steps"]},
+        "gpu_launches": info["launches_per_step"] * K * m["windows"],
+        "roofline": {"bound": "hbm", "kernel": info["kernel_name"], "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": info["alg_bytes"],
+                     "kernel_ms": m["kern_ms"], "kernel_timed_steps": m["kern_events"],
+                     "frac_of_8000": achieved / 8000.0,
+                     "kernel_tokens_per_s": info["units_per_step"] / (m["kern_ms"] * 1e-3),
+                     "traffic": traffic[0] if traffic else None,
+                     "traffic_source": traffic[1] if traffic else None},
+        "cpu_baseline": cpu,
+    }
 
 
 if __name__ == "__main__":

@@ -11,8 +11,7 @@ Notation follows the paper: ``n`` transform length, ``K = floor(n/2)+1`` bins,
 ``d`` channels per head, ``g`` the complex spectral gate of one head,
 ``N`` = ``N_max`` the cache window.
 
-Readings taken where the paper is silent or garbled (all listed in the design
-notes of the repository):
+Readings taken where the paper is silent or garbled:
   * modReLU (Sec. 3.2 step 3c prints no formula): the standard definition
     ``max(|z| + beta, 0) * z/|z|`` with a real bias per bin, 0 at ``z = 0``.
     Parity for the *choice* of this definition is unpinned.

@@ -7,6 +7,8 @@
 //   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
 #include "common.cuh"
 
+#include <atomic>
+#include <string>
 #include <type_traits>
 
 namespace spectre {
@@ -688,19 +690,20 @@ static __device__ __align__(256) unsigned char g_gate_static_scratch[SPECTRE_GAT
 
 namespace spectre {
 static const int kMaxDevices = 64;
-static void* g_static_ptr[kMaxDevices] = {};     // device address of the array, per device ordinal
+static std::atomic<void*> g_static_ptr[kMaxDevices];     // device address of the array, per device ordinal
 
-// With `device` current: resolves (once) the device address of the static scratch.
+// With `device` current: resolves (once) the device address of the static scratch.  Host threads
+// that race on the first call of a device each look the address up and store the same value.
 static int static_scratch_address(int device, void** out) {
   if (device < 0 || device >= kMaxDevices) return fail(SPECTRE_ERR_UNSUPPORTED, "device ordinal beyond 63");
-  if (!g_static_ptr[device]) {
-    void* p = nullptr;
+  void* p = g_static_ptr[device].load(std::memory_order_acquire);
+  if (!p) {
     cudaError_t e = cudaGetSymbolAddress(&p, g_gate_static_scratch);
     if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(gate static scratch)");
     if (!p) return fail(SPECTRE_ERR_CUDA, "static scratch has no device address");
-    g_static_ptr[device] = p;
+    g_static_ptr[device].store(p, std::memory_order_release);
   }
-  *out = g_static_ptr[device];
+  *out = p;
   return SPECTRE_OK;
 }
 }  // namespace spectre
@@ -712,8 +715,11 @@ extern "C" int spectre_gate_static(spectre_ctx* ctx, void* stream, const spectre
                                    const int64_t* shift, int64_t shift_all, float* g_out, float* qbar_out) {
   if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
   if (!gp) return fail(SPECTRE_ERR_INVALID_ARG, "gate parameters are NULL");
-  if (B < 1 || H < 1 || D < 1 || n_fft < 1 || gp->toeplitz_r < 0)
-    return fail(SPECTRE_ERR_INVALID_ARG, "B, H, D, n_fft must be positive");
+  if (B < 1 || H < 1 || D < 1 || D > 1024) return fail(SPECTRE_ERR_INVALID_ARG, "B, H, D must be positive (D <= 1024)");
+  if (n_fft < 1 || n_fft > (1 << 24)) return fail(SPECTRE_ERR_INVALID_ARG, "n_fft out of range");
+  // the widths that size the scratch are range-checked before the size is computed from them
+  if (gp->hidden < 1 || gp->hidden > 1024) return fail(SPECTRE_ERR_UNSUPPORTED, "hidden width must be in 1..1024");
+  if (gp->toeplitz_r < 0 || gp->toeplitz_r > 64) return fail(SPECTRE_ERR_UNSUPPORTED, "toeplitz_r must be in 0..64");
   size_t off_a, off_b;
   const size_t need = gate_ws_layout(B, H, D, n_fft, gp->toeplitz_r, gp->hidden, 1, &off_a, &off_b);   // one copy of the sums
   if (need > SPECTRE_GATE_STATIC_BYTES)

@@ -24,8 +24,6 @@
 // images per head); larger groups measured faster than groups small enough to stay in L2.
 #include <cuda_fp16.h>
 
-#include <cstdlib>
-
 #include "tc_stage.cuh"
 
 namespace spectre {
@@ -41,43 +39,6 @@ constexpr int k4EpiWarps = 16;
 constexpr int k4EpiThreads = 32 * k4EpiWarps;
 constexpr int k4CoreThreads = k4EpiThreads + 32;    // + producer / MMA-issuing warp
 constexpr int k4CoreSmem = k4FBytes + 2 * k4BBytes + 2 * k4GBytes + 64;
-constexpr uint32_t k4SpinLimit = 1u << 24;
-
-__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint64_t desc4(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
-  uint64_t d = (uint64_t)((saddr >> 4) & 0x3fff);
-  d |= (uint64_t)((lbo >> 4) & 0x3fff) << 16;
-  d |= (uint64_t)((sbo >> 4) & 0x3fff) << 32;
-  d |= (uint64_t)1 << 46;
-  return d;
-}
-__device__ __forceinline__ bool wait4(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < k4SpinLimit; ++it) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-__device__ __forceinline__ uint32_t h2pack(float lo, float hi) {
-  __half2 h = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
-__device__ __forceinline__ float2 h2unpack(uint32_t u) {
-  __half2 h = *reinterpret_cast<__half2*>(&u);
-  return __half22float2(h);
-}
-__device__ __forceinline__ void ld16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void ld_wait4() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // XOR skew of the low five bits of a staged word's index: the 8 tiles x 4 pairs a warp writes at once
 // land in 32 different banks
@@ -136,7 +97,7 @@ __device__ __forceinline__ void tc_gate_body(const TcGateParams& p, int sk, floa
     uint32_t v = 0u;
     if (k1 < 64) {
       const float2 gv2 = vals[k1 + 64 * k2];
-      v = h2pack(gv2.x * inv, gv2.y * inv);
+      v = pack_h2(gv2.x * inv, gv2.y * inv);
     }
     img[idx] = v;
   }
@@ -198,7 +159,7 @@ __global__ void __launch_bounds__(256, 3) tc_in_kernel(const TcInParams p, const
 #pragma unroll
       for (int n1 = 0; n1 < R; ++n1) {
         const uint32_t v = n1 < nvalid ? __ldg(pl + n1 * lstride) : 0u;
-        x[n1] = F16 ? h2unpack(v) : make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+        x[n1] = F16 ? unpack_h2(v) : make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
       }
       Dft<R, false>::run(x);
       const float2 w1 = tws[rs];
@@ -211,7 +172,7 @@ __global__ void __launch_bounds__(256, 3) tc_in_kernel(const TcInParams p, const
 #pragma unroll
         for (int k1 = 0; k1 < R; ++k1) {
           const float2 v = cmul(x[k1], w);
-          ps[k1 * sstride] = h2pack(v.x, v.y);
+          ps[k1 * sstride] = pack_h2(v.x, v.y);
           w = cmul(w, w1);
         }
       }
@@ -238,18 +199,6 @@ __global__ void __launch_bounds__(256, 3) tc_in_kernel(const TcInParams p, const
   }
 }
 
-#ifdef SPECTRE_TC_TIMING
-__device__ long long g_core_timing[256][16];
-#define CORE_STAMP(slot) do { if (T == 0 && warp == 0 && blockIdx.x < 256) g_core_timing[blockIdx.x][slot] = clock64(); } while (0)
-__device__ long long g_core_wait[256][8];       // per CTA: cycles warp 0 spent waiting for the MMAs, per (stage, slot)
-#define CORE_WAIT_BEGIN() long long wt0_ = clock64()
-#define CORE_WAIT_END(idx) do { if (T == 0 && warp == 0 && blockIdx.x < 256) g_core_wait[blockIdx.x][idx] += clock64() - wt0_; } while (0)
-#else
-#define CORE_STAMP(slot) do { } while (0)
-#define CORE_WAIT_BEGIN() do { } while (0)
-#define CORE_WAIT_END(idx) do { } while (0)
-#endif
-
 // =====================================================================================
 // core: 4096-point units on the tensor cores
 // =====================================================================================
@@ -270,15 +219,15 @@ __device__ __forceinline__ void core_store(uint32_t tmem_d, unsigned char* out, 
   const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
-  ld16x256b_x4(taddr0, r[0]);
+  tmem_ld_16x256b_x4(taddr0, r[0]);
 #pragma unroll
   for (int step = 0; step < 4; ++step) {                        // step = 2 j + chunk
     const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
-    ld_wait4();
+    tmem_ld_wait();
     if (step < 3) {
       const int ns = step + 1;
-      ld16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 1)) << 16) + 32 * (ns & 1), r[ns & 1]);
+      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 1)) << 16) + 32 * (ns & 1), r[ns & 1]);
     }
     const uint32_t (&rr)[16] = r[step & 1];
     const int grp0 = 8 * cq + 4 * chunk;                        // first 8-column group of the chunk
@@ -286,15 +235,11 @@ __device__ __forceinline__ void core_store(uint32_t tmem_d, unsigned char* out, 
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
       uint2 o;
-      o.x = h2pack(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
-      o.y = h2pack(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
+      o.x = pack_h2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
+      o.y = pack_h2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
       *reinterpret_cast<uint2*>(out + base + x * 32) = o;
     }
   }
-}
-
-__device__ __forceinline__ void arrive4(uint32_t bar) {
-  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" :: "r"(bar) : "memory");
 }
 
 // Persistent: a CTA takes pairs of units (2 pair, 2 pair + 1).  16 epilogue warps alternate
@@ -314,10 +259,10 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
   __shared__ uint32_t tmem_slot;
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
   uint32_t barL[2], barD[2], barB[2];
-  for (int s2 = 0; s2 < 2; ++s2) { barL[s2] = s_u32(&bars[s2]); barD[s2] = s_u32(&bars[2 + s2]); barB[s2] = s_u32(&bars[4 + s2]); }
+  for (int s2 = 0; s2 < 2; ++s2) { barL[s2] = smem_u32(&bars[s2]); barD[s2] = smem_u32(&bars[2 + s2]); barB[s2] = smem_u32(&bars[4 + s2]); }
 
   if (warp == k4EpiWarps) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s_u32(&tmem_slot)), "r"(512));
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(512));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
   if (tid == 0) {
@@ -339,7 +284,6 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
   const uint32_t tmem = tmem_slot;
   const int npairs = (p.nunits + 1) / 2;
   bool ok = true;
-  CORE_STAMP(0);
 
   if (warp == k4EpiWarps) {
     // ---- producer + MMA issuer ----
@@ -352,9 +296,9 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
         const unsigned char* gim = p.gimg + (size_t)(unit / p.ntile) * k4GBytes;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL[s2]), "r"(k4ImgBytes + k4GBytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(s_u32(Bsm[s2])), "l"(img), "r"(k4ImgBytes), "r"(barL[s2]) : "memory");
+                     :: "r"(smem_u32(Bsm[s2])), "l"(img), "r"(k4ImgBytes), "r"(barL[s2]) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(s_u32(Gsm[s2])), "l"(gim), "r"(k4GBytes), "r"(barL[s2]) : "memory");
+                     :: "r"(smem_u32(Gsm[s2])), "l"(gim), "r"(k4GBytes), "r"(barL[s2]) : "memory");
       } else {
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(barL[s2]) : "memory");   // odd tail: nothing to fetch
       }
@@ -366,21 +310,21 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
       for (int stage = 0; stage < 4 && ok; ++stage) {
         for (int s2 = 0; s2 < 2 && ok; ++s2) {
           if (stage == 0) {
-            ok = wait4(barL[s2], iter & 1);                         // operand landed
-            if (ok && iter > 0) ok = wait4(barB[s2], 1);            // previous result of this slot left TMEM
+            ok = mbar_wait(barL[s2], iter & 1);                         // operand landed
+            if (ok && iter > 0) ok = mbar_wait(barB[s2], 1);            // previous result of this slot left TMEM
           } else {
-            ok = wait4(barB[s2], (stage - 1) & 1);
+            ok = mbar_wait(barB[s2], (stage - 1) & 1);
           }
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           if (T == 0) {
-            const uint32_t a0 = s_u32(Fsm), b0 = s_u32(Bsm[s2]);
+            const uint32_t a0 = smem_u32(Fsm), b0 = smem_u32(Bsm[s2]);
             const uint32_t lbo = stage == 0 ? k8Lbo0 : (stage == 1 ? k8Lbo1 : (stage == 2 ? k8Lbo2 : k8Lbo3));
             const uint32_t sbo = stage == 0 ? k8Sbo0 : (stage == 1 ? k8Sbo1 : (stage == 2 ? k8Sbo2 : k8Sbo3));
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-              const uint64_t da = desc4(a0 + ks * 256, 128, 2048);
-              const uint64_t db = desc4(b0 + ks * 2 * lbo, lbo, sbo);
+              const uint64_t da = umma_desc(a0 + ks * 256, 128, 2048);
+              const uint64_t db = umma_desc(b0 + ks * 2 * lbo, lbo, sbo);
               const uint32_t acc = ks > 0;
               asm volatile(
                   "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
@@ -396,7 +340,7 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
       const int next = pair + gridDim.x;
       if (next < npairs) {
         for (int s2 = 0; s2 < 2 && ok; ++s2) {
-          ok = wait4(barD[s2], 1);
+          ok = mbar_wait(barD[s2], 1);
           if (ok && T == 0) fetch(next, s2);
           __syncwarp();
         }
@@ -410,11 +354,8 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
       for (int stage = 0; stage < 4 && ok; ++stage) {
 #pragma unroll 1
         for (int s2 = 0; s2 < 2 && ok; ++s2) {
-          CORE_WAIT_BEGIN();
-          ok = wait4(barD[s2], stage & 1);
-          CORE_WAIT_END(2 * stage + s2);
+          ok = mbar_wait(barD[s2], stage & 1);
           if (!ok) break;
-          if (pair == blockIdx.x && stage == 0 && s2 == 0) CORE_STAMP(1);
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t td = tmem + 256 * s2;
           const int unit = 2 * pair + s2;
@@ -424,8 +365,7 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
           else if (unit < p.nunits) core_store(td, p.ws_out + (size_t)unit * k4OutBytes, q, cq, T);
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          if (pair == blockIdx.x) CORE_STAMP(2 + 2 * stage + s2);
-          arrive4(barB[s2]);
+          mbar_arrive(barB[s2]);
         }
       }
     }
@@ -481,7 +421,7 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
     float2 x[R];
 #pragma unroll
     for (int k1 = 0; k1 < R; ++k1) {
-      float2 f = h2unpack(__ldg(pu + k1 * ustride));
+      float2 f = unpack_h2(__ldg(pu + k1 * ustride));
       x[k1] = make_float2(f.x * gsc[k1], -f.y * gsc[k1]);       // result of conj(FFT(conj(.))), scaled
     }
     const float2 w1 = tws[tl];
@@ -497,7 +437,7 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
 #pragma unroll
     for (int n1 = 0; n1 < R; ++n1) {
       if (F16) {
-        ps[n1 * NT * npair] = h2pack(x[n1].x, x[n1].y);
+        ps[n1 * NT * npair] = pack_h2(x[n1].x, x[n1].y);
       } else {
         __nv_bfloat162 o = __floats2bfloat162_rn(x[n1].x, x[n1].y);
         ps[n1 * NT * npair] = *reinterpret_cast<uint32_t*>(&o);
@@ -538,7 +478,6 @@ size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
   // heads per group: measured on B200, larger groups win (fewer, fuller launches) although the
   // intermediates then no longer stay in L2; the preferred workspace is capped at 1.25 GiB
   size_t budget = (size_t)1280 << 20;
-  if (const char* e = std::getenv("SPECTRE_TC_L2_FRACTION_PCT")) budget = ctx->l2_bytes / 100 * (size_t)atoi(e);
   size_t g = budget / per;
   if (g < 1) g = 1;
   if (g > (size_t)nslab) g = nslab;

@@ -9,9 +9,10 @@ run that stops at the first failure has already run every other test."""
 import pytest
 import torch
 
+from oracle import spectre_oracle as O
 from paper_2502_18394_b200 import binding as S
 from paper_2502_18394_b200 import workloads as W
-from util import gate_to_complex, rel_err, to_dev
+from util import GATE_TOL, gate_params_np, gate_to_complex, rel_err, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -34,6 +35,17 @@ def test_static_gate_matches_workspace_gate_twice_in_a_row():
             assert torch.cuda.mem_get_info()[0] == free_before   # no device memory was taken
         assert rel_err(gate_to_complex(got), gate_to_complex(ref)) < 1e-5   # pooled sums use float atomics
         assert rel_err(W.to_f64(qbar), W.to_f64(qbar_ref)) < 1e-5
+        # and against the oracle, like every other gate test
+        gref = O.gate(W.to_f64(x).sum(axis=1), 1.0 / w.L, w.n, shift=[5] * w.B, **gate_params_np(p))
+        assert rel_err(gate_to_complex(got), gref) < GATE_TOL["16bit"]
+    # Toeplitz update on: the pre-update gate sits at the start of the array, the sums behind it
+    pt = W.gate_params(w, modrelu_bias_std=0.05, toeplitz_r=2, bias_std=0.1)
+    x = W.activations(w, stream=7).cuda()
+    ref = S.spectre_gate(ctx, to_dev(pt), w.n, q=x, shift_all=3)
+    got = S.spectre_gate_static(ctx, to_dev(pt), w.n, g_out, q=x, shift_all=3)
+    assert rel_err(gate_to_complex(got), gate_to_complex(ref)) < 1e-5
+    gref = O.gate(W.to_f64(x).sum(axis=1), 1.0 / w.L, w.n, shift=[3] * w.B, **gate_params_np(pt))
+    assert rel_err(gate_to_complex(got), gref) < GATE_TOL["16bit"]
     # the running-sum form (decode) and the size limit
     sum_q = torch.randn(w.B, w.H, w.D, device="cuda") * 3
     ref = S.spectre_gate(ctx, p, w.n, sum_q=sum_q, inv_count=1.0 / w.n)
