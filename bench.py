@@ -207,7 +207,7 @@ class MixerBench:
             self.kernel_name, nk = "mixer_tc196_kernel (single-kernel tcgen05 mixer, refinement in the store phase) + level_gates_kernel", (2 if fused_wrm else 1)
         elif w.dtype in ("bf16", "f16") and ws_mix and w.n >= 4096:
             R, ntile = w.n // 4096, w.D // 8
-            per = R * ntile * (65536 + 65536) + R * 18432 + 256
+            per = R * ntile * (65536 + 65536) + R * 16384 + 256
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
             self.kernel_name, nk = "mixer, staged tcgen05 path (tc_in incl. gate images + tc_core + tc_out per group)", 3 * groups
         elif ws_mix:

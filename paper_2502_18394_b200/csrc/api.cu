@@ -12,6 +12,8 @@ int build_dft64(__half* F, cudaStream_t st);   // mixer_tc.cu
 int build_tw8192(float2* tab, cudaStream_t st);
 int build_dft49(__half* F, cudaStream_t st);
 int build_tw64x64(float4* tab, cudaStream_t st);
+int build_tw_staged(float2* tab, cudaStream_t st);   // mixer_tc4k.cu
+int build_dft32(void* mats, cudaStream_t st);        // mixer_tc32.cu
 
 static thread_local std::string g_last_error;
 
@@ -97,6 +99,8 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
   c->tw8192 = nullptr;
   c->dft49 = nullptr;
   c->tw64x64 = nullptr;
+  c->tw_staged = nullptr;
+  c->dft32 = nullptr;
   c->status_host = nullptr;
   c->status_dev = nullptr;
   cudaError_t e2 = cudaSetDevice(device);
@@ -104,6 +108,8 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw8192, 2049 * sizeof(float2));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft49, 128 * 128 * sizeof(__half));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw64x64, 2048 * sizeof(float4));
+  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw_staged, 63 * 128 * sizeof(float2));
+  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft32, 4 * 16384);
   if (e2 == cudaSuccess) e2 = cudaHostAlloc(reinterpret_cast<void**>(&c->status_host), sizeof(int), cudaHostAllocMapped);
   if (e2 == cudaSuccess) {
     *c->status_host = 0;
@@ -114,6 +120,8 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
     if (rc == SPECTRE_OK) rc = build_tw8192(reinterpret_cast<float2*>(c->tw8192), 0);
     if (rc == SPECTRE_OK) rc = build_dft49(reinterpret_cast<__half*>(c->dft49), 0);
     if (rc == SPECTRE_OK) rc = build_tw64x64(reinterpret_cast<float4*>(c->tw64x64), 0);
+    if (rc == SPECTRE_OK) rc = build_tw_staged(reinterpret_cast<float2*>(c->tw_staged), 0);
+    if (rc == SPECTRE_OK) rc = build_dft32(c->dft32, 0);
     if (rc == SPECTRE_OK) e2 = cudaStreamSynchronize(0);
     else e2 = cudaErrorUnknown;
   }
@@ -131,6 +139,8 @@ extern "C" int spectre_destroy(spectre_ctx* ctx) {
     if (ctx->tw8192) cudaFree(ctx->tw8192);
     if (ctx->dft49) cudaFree(ctx->dft49);
     if (ctx->tw64x64) cudaFree(ctx->tw64x64);
+    if (ctx->tw_staged) cudaFree(ctx->tw_staged);
+    if (ctx->dft32) cudaFree(ctx->dft32);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
   }
   delete ctx;

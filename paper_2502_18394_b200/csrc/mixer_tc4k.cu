@@ -29,16 +29,17 @@
 namespace spectre {
 
 // ---- shared with mixer_tc.cu (same conventions) ------------------------------------
-constexpr int k4BBytes = k8BBytes;               // one 256-column operand buffer (largest of the four stage layouts)
-constexpr int k4ImgBytes = 16 * k8Lbo0;          // stage-0 operand image in the workspace (dense: columns 64 c + t2, K = t1)
+constexpr int k4Lbo = 4096, k4Sbo = 128;         // every operand image of the core is dense: 4096 bytes between K groups, 128 between 8-column groups
+constexpr int k4BBytes = 16 * k4Lbo;             // one 256-column operand buffer
+constexpr int k4ImgBytes = k4BBytes;             // stage-0 operand image in the workspace (columns 64 c + t2, K = t1)
 constexpr int k4FBytes = 128 * 128 * 2;
-constexpr int k4GStride = k8GStride;             // gate table: entry (k1, k2) at 72 k2 + k1, bin kM = k1 + 64 k2
-constexpr int k4GBytes = k8GBytes;
-constexpr int k4OutBytes = 4096 * 4 * 4;         // unit result: [t'][4 pairs] half2
-constexpr int k4EpiWarps = 16;
+constexpr int k4GBytes = 4096 * 4;               // gate table: bin kM = k1 + 64 k2 at 64 k2 + (k1 ^ 8 (k2 % 4)), fp16 (re, im)
+constexpr int k4OutBytes = 4096 * 4 * 4;         // unit result: [unit_row_slot(t')][4 pairs] half2
+constexpr int k4EpiWarps = 8;                    // 2 per TMEM lane quadrant, one column half each
 constexpr int k4EpiThreads = 32 * k4EpiWarps;
 constexpr int k4CoreThreads = k4EpiThreads + 32;    // + producer / MMA-issuing warp
-constexpr int k4CoreSmem = k4FBytes + 2 * k4BBytes + 2 * k4GBytes + 64;
+constexpr int k4CoreSmem = k4FBytes + k4BBytes + k4GBytes + 64;
+static_assert(2 * (k4CoreSmem + 1024) <= 233472, "two core CTAs per SM");
 
 // XOR skew of the low five bits of a staged word's index: the 8 tiles x 4 pairs a warp writes at once
 // land in 32 different banks
@@ -47,6 +48,23 @@ __device__ __forceinline__ int stage_skew(int tile, int c4) { return (tile & 7) 
 // forward-scale of the radix-R step (keeps fp16 magnitudes near the input's)
 __host__ __device__ constexpr float in_scale(int R) {
   return R <= 2 ? 1.0f : (R <= 8 ? 0.5f : (R == 16 ? 0.25f : 0.125f));
+}
+
+// Twiddles of the four-step split for every supported R: row R - 1 + k1 (k1 < R) holds W_n^{64 k1 t1} for
+// t1 < 64 and then W_n^{k1 t2} for t2 < 64, n = 4096 R (angles reduced in integers).
+__global__ void build_tw_staged_kernel(float2* tab) {
+  const int row = blockIdx.x, e = threadIdx.x;                 // 63 rows x 128 entries
+  int R = 1;
+  while (2 * R - 1 <= row) R *= 2;
+  const int k1 = row - (R - 1);
+  const unsigned n = 4096u * (unsigned)R;
+  const unsigned m = e < 64 ? (64u * (unsigned)k1 * (unsigned)e) % n : ((unsigned)k1 * (unsigned)(e - 64)) % n;
+  tab[row * 128 + e] = twiddle_fwd(m, n);
+}
+int build_tw_staged(float2* tab, cudaStream_t st) {
+  build_tw_staged_kernel<<<63, 128, 0, st>>>(tab);
+  SPECTRE_LAUNCH_OK("build_tw_staged_kernel");
+  return SPECTRE_OK;
 }
 
 // =====================================================================================
@@ -92,14 +110,10 @@ __device__ __forceinline__ void tc_gate_body(const TcGateParams& p, int sk, floa
   const float inv = m > 0.f ? 1.0f / m : 0.f;
   if (threadIdx.x == 0) p.gscale[sk] = m;
   uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * k4GBytes);
-  for (int idx = threadIdx.x; idx < 64 * k4GStride; idx += 256) {
-    const int k2 = idx / k4GStride, k1 = idx - k2 * k4GStride;        // kM = k1 + 64 k2
-    uint32_t v = 0u;
-    if (k1 < 64) {
-      const float2 gv2 = vals[k1 + 64 * k2];
-      v = pack_h2(gv2.x * inv, gv2.y * inv);
-    }
-    img[idx] = v;
+  for (int idx = threadIdx.x; idx < 4096; idx += 256) {
+    const int k2 = idx >> 6, k1 = idx & 63;                            // kM = k1 + 64 k2
+    const float2 gv2 = vals[idx];
+    img[64 * k2 + (k1 ^ (8 * (k2 & 3)))] = pack_h2(gv2.x * inv, gv2.y * inv);
   }
 }
 
@@ -208,69 +222,101 @@ struct TcCoreParams {
   unsigned char* ws_out;
   const __half* F;
   const float4* tw64;       // stage twiddles W_4096^{row d} in epilogue order
-  int nunits, ntile;
+  const float2* twr;        // [R][128]: W_n^{64 k1 t1}, W_n^{k1 t2} (the rows of this R in the context's table)
+  const float* gscale;      // [slab_local * R + k1] gate scale of the unit's (head, k1)
+  float out_scale;          // 1 / (R * forward scale of the radix-R step)
+  int nunits, ntile, R;
   int* status;
 };
 
-// Last epilogue of a unit for one warp (TMEM lane quadrant q, 64-column quarter cq): the accumulator
-// has rows s2 and columns 4 s1 + c (tc_stage.cuh); the unit's result [t' = 64 row + s1][pair] goes to
-// the workspace as half2, two pairs per 8-byte store.  TMEM loads run one 32-column chunk ahead.
-__device__ __forceinline__ void core_store(uint32_t tmem_d, unsigned char* out, int q, int cq, int T) {
-  const int i = T >> 2, p = (T >> 1) & 1, cp = T & 1;
+// Where row t' of a unit's result lies, in 16-byte units (the four pairs of a row stay together): rows
+// are ordered (s1 / 4, t' / 64, s1 % 4) with s1 = t' % 64, the order in which the core's last epilogue
+// holds them (8 lanes = 8 values of t' / 64, 4 lanes = 4 values of s1 % 4), so one of its store
+// instructions writes 512 contiguous bytes.
+__host__ __device__ __forceinline__ int unit_row_slot(int tp) {
+  const int row = tp >> 6, s1 = tp & 63;
+  return ((s1 >> 2) * 64 + row) * 4 + (s1 & 3);
+}
+
+// Last epilogue of a unit for one warp (TMEM lane quadrant q, column half ch): the accumulator has rows
+// s2 and columns 16 (s1 / 4) + 8 (c / 2) + 2 (s1 % 4) + c % 2 (tc_stage.cuh, COLS = 2): D = the inverse
+// stages' conj(FFT(conj(.))) of the unit at t' = 64 row + s1, all four pairs of two values of s1 per
+// 32-column chunk in one thread.  What leaves is ready for the inverse radix-R step over k1:
+// conj(D W_n^{k1 t'}) times the gate scale and 1 / (R s_in), as half2 [unit_row_slot(t')][pair], one
+// 16-byte store per row.  tw = this k1's 128 table entries.  TMEM loads run one chunk ahead.
+__device__ __forceinline__ void core_store(uint32_t tmem_d, unsigned char* out, int q, int ch, int T,
+                                           const float2* __restrict__ tw, float gsc) {
+  const int i = T >> 2, tq = T & 3;
+  float2 fa[2], fb[8];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const float2 t = __ldg(tw + 8 * (2 * q + j) + i);
+    fa[j] = make_float2(t.x * gsc, t.y * gsc);
+  }
+#pragma unroll
+  for (int k = 0; k < 8; ++k) fb[k] = __ldg(tw + 64 + 4 * (8 * ch + k) + tq);   // s1 = 4 (8 ch + k) + tq
   uint32_t r[2][16];
-  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * cq;
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 128 * ch;
   tmem_ld_16x256b_x4(taddr0, r[0]);
 #pragma unroll
-  for (int step = 0; step < 4; ++step) {                        // step = 2 j + chunk
-    const int j = step >> 1, chunk = step & 1;
+  for (int step = 0; step < 8; ++step) {                        // step = 2 cc + j: columns 128 ch + 32 cc .. + 31
+    const int cc = step >> 1, j = step & 1;
     const int row = 8 * (2 * q + j) + i;
     tmem_ld_wait();
-    if (step < 3) {
+    if (step < 7) {
       const int ns = step + 1;
-      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 1)) << 16) + 32 * (ns & 1), r[ns & 1]);
+      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * (ns & 1)) << 16) + 32 * (ns >> 1), r[ns & 1]);
     }
     const uint32_t (&rr)[16] = r[step & 1];
-    const int grp0 = 8 * cq + 4 * chunk;                        // first 8-column group of the chunk
-    const uint32_t base = (uint32_t)(((64 * row + 2 * grp0 + p) * 4 + 2 * cp) * 4);
 #pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      uint2 o;
-      o.x = pack_h2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2]));
-      o.y = pack_h2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3]));
-      *reinterpret_cast<uint2*>(out + base + x * 32) = o;
+    for (int s = 0; s < 2; ++s) {                               // s1 / 4 = 8 ch + 2 cc + s; 8-column groups 2 s, 2 s + 1 = pairs 0-1, 2-3
+      const float2 w = cmul(fa[j], fb[2 * cc + s]);
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {                             // pair e: group 2 s + e / 2, column e % 2
+        const int b0 = 4 * (2 * s + (e >> 1)) + (e & 1);
+        const float2 pz = cmul(make_float2(__uint_as_float(rr[b0]), __uint_as_float(rr[b0 + 2])), w);
+        o[e] = pack_h2(pz.x, -pz.y);
+      }
+      const int k = 8 * ch + 2 * cc + s;                        // s1 / 4
+      *reinterpret_cast<uint4*>(out + (size_t)((k * 64 + row) * 4 + tq) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
 }
 
-// Persistent: a CTA takes pairs of units (2 pair, 2 pair + 1).  16 epilogue warps alternate
-// between the two units of the pair; one more warp fetches operands and issues the MMAs, so
-// while the ALUs run one unit's epilogue the tensor core runs the other unit's stage.
-//   barL[s]  operand + gate table of slot s landed (bulk copies, transaction count)
-//   barD[s]  the stage's MMAs of slot s completed                    (4 phases per pair)
-//   barB[s]  all epilogue threads finished with slot s: next operand written (stages 0-2) or
-//            result stored and the slot free again (stage 3)         (4 phases per pair)
-__global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreParams p) {
-  extern __shared__ __align__(128) unsigned char smem[];
+// Persistent, two CTAs per SM (112 KB of shared memory, 256 TMEM columns, 8 epilogue warps + 1 warp that
+// fetches and issues).  A CTA works through a contiguous range of units, one at a time: operand image
+// (64 KB, one bulk copy) and, when the (head, k1) changes, the gate table (16 KB) -> 4 x [MMA -> epilogue]
+// in place on one operand buffer -> result to the workspace.  The next unit's image is fetched as soon
+// as the last MMAs of the current one have read the buffer, under the last epilogue.  One CTA's MMAs and
+// copies run under the other CTA's epilogues.  (Splitting a unit into two 128-column halves that
+// ping-pong inside the CTA measured slower: an MMA of N = 128 re-reads the DFT matrix per half and the
+// stage becomes bound by shared-memory reads.)
+//   barL  operand image (+ gate table) landed (transaction count)       1 phase per unit
+//   barD  the stage's MMAs completed                                     4 phases per unit
+//   barB  all epilogue threads done with the stage: next operand written (stages 0-2) or the
+//         accumulator drained (stage 3)                                  4 phases per unit
+// Operand images (tc_stage.cuh): stages 0-2 have columns 64 c + digit, the last operand has columns
+// 16 (s1 / 4) + 8 (c / 2) + 2 (s1 % 4) + c % 2.
+__global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* Fsm = smem;
-  unsigned char* Bsm[2] = {smem + k4FBytes, smem + k4FBytes + k4BBytes};
-  uint32_t* Gsm[2] = {reinterpret_cast<uint32_t*>(smem + k4FBytes + 2 * k4BBytes),
-                      reinterpret_cast<uint32_t*>(smem + k4FBytes + 2 * k4BBytes + k4GBytes)};
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + k4FBytes + 2 * k4BBytes + 2 * k4GBytes);
-  __shared__ uint32_t tmem_slot;
+  unsigned char* Bsm = smem + k4FBytes;
+  uint32_t* Gsm = reinterpret_cast<uint32_t*>(smem + k4FBytes + k4BBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + k4FBytes + k4BBytes + k4GBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6);
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
-  uint32_t barL[2], barD[2], barB[2];
-  for (int s2 = 0; s2 < 2; ++s2) { barL[s2] = smem_u32(&bars[s2]); barD[s2] = smem_u32(&bars[2 + s2]); barB[s2] = smem_u32(&bars[4 + s2]); }
+  const uint32_t barL = smem_u32(&bars[0]);
+  const uint32_t barD = smem_u32(&bars[1]), barB = smem_u32(&bars[2]);
 
   if (warp == k4EpiWarps) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(512));
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(tmem_slot)), "r"(256));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
   if (tid == 0) {
-    for (int s2 = 0; s2 < 2; ++s2) {
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barL[s2]), "r"(1));
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barD[s2]), "r"(1));
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(barB[s2]), "r"(k4EpiThreads));
-    }
+    mbar_init(barL, 1);
+    mbar_init(barD, 1);
+    mbar_init(barB, k4EpiThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < k4EpiThreads) {
@@ -281,101 +327,94 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem = tmem_slot;
-  const int npairs = (p.nunits + 1) / 2;
+  const uint32_t tmem = *tmem_slot;
+  // this CTA's units: a contiguous range, so that consecutive units mostly share the gate table
+  const int per = (p.nunits + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int u0 = (int)blockIdx.x * per, u1 = min(p.nunits, u0 + per);
   bool ok = true;
 
   if (warp == k4EpiWarps) {
     // ---- producer + MMA issuer ----
-    const uint32_t idesc = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
-    // fetch(pair, slot): one bulk copy for the operand image, one for the gate table
-    auto fetch = [&](int pair, int s2) {
-      const int unit = 2 * pair + s2;
-      if (unit < p.nunits) {
-        const unsigned char* img = p.ws_in + (size_t)unit * k4ImgBytes;
-        const unsigned char* gim = p.gimg + (size_t)(unit / p.ntile) * k4GBytes;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL[s2]), "r"(k4ImgBytes + k4GBytes) : "memory");
+    const uint32_t idesc = umma_idesc_128x256();
+    auto fetch = [&](int unit) {
+      const bool new_gate = unit == u0 || unit / p.ntile != (unit - 1) / p.ntile;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL), "r"(k4ImgBytes + (new_gate ? k4GBytes : 0)) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   :: "r"(smem_u32(Bsm)), "l"(p.ws_in + (size_t)unit * k4ImgBytes), "r"(k4ImgBytes), "r"(barL) : "memory");
+      if (new_gate)
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(smem_u32(Bsm[s2])), "l"(img), "r"(k4ImgBytes), "r"(barL[s2]) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(smem_u32(Gsm[s2])), "l"(gim), "r"(k4GBytes), "r"(barL[s2]) : "memory");
-      } else {
-        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(barL[s2]) : "memory");   // odd tail: nothing to fetch
-      }
+                     :: "r"(smem_u32(Gsm)), "l"(p.gimg + (size_t)(unit / p.ntile) * k4GBytes), "r"(k4GBytes), "r"(barL) : "memory");
     };
-    int iter = 0;
-    if (T == 0 && blockIdx.x < npairs) { fetch(blockIdx.x, 0); fetch(blockIdx.x, 1); }
+    if (T == 0 && u0 < u1) fetch(u0);
     __syncwarp();
-    for (int pair = blockIdx.x; pair < npairs && ok; pair += gridDim.x, ++iter) {
+    for (int unit = u0, it = 0; unit < u1 && ok; ++unit, ++it) {
       for (int stage = 0; stage < 4 && ok; ++stage) {
-        for (int s2 = 0; s2 < 2 && ok; ++s2) {
-          if (stage == 0) {
-            ok = mbar_wait(barL[s2], iter & 1);                         // operand landed
-            if (ok && iter > 0) ok = mbar_wait(barB[s2], 1);            // previous result of this slot left TMEM
-          } else {
-            ok = mbar_wait(barB[s2], (stage - 1) & 1);
-          }
-          if (!ok) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          if (T == 0) {
-            const uint32_t a0 = smem_u32(Fsm), b0 = smem_u32(Bsm[s2]);
-            const uint32_t lbo = stage == 0 ? k8Lbo0 : (stage == 1 ? k8Lbo1 : (stage == 2 ? k8Lbo2 : k8Lbo3));
-            const uint32_t sbo = stage == 0 ? k8Sbo0 : (stage == 1 ? k8Sbo1 : (stage == 2 ? k8Sbo2 : k8Sbo3));
+        if (stage == 0) {
+          ok = mbar_wait(barL, it & 1);                         // operand landed
+          if (ok && it > 0) ok = mbar_wait(barB, 1);            // previous result has left TMEM
+        } else {
+          ok = mbar_wait(barB, (stage - 1) & 1);
+        }
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (T == 0) {
+          const uint32_t a0 = smem_u32(Fsm), b0 = smem_u32(Bsm);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              const uint64_t da = umma_desc(a0 + ks * 256, 128, 2048);
-              const uint64_t db = umma_desc(b0 + ks * 2 * lbo, lbo, sbo);
-              const uint32_t acc = ks > 0;
-              asm volatile(
-                  "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                  :: "r"(tmem + 256 * s2), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barD[s2]) : "memory");
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t da = umma_desc(a0 + ks * 256, 128, 2048);
+            const uint64_t db = umma_desc(b0 + ks * 2 * k4Lbo, k4Lbo, k4Sbo);
+            const uint32_t acc = ks > 0;
+            asm volatile(
+                "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                :: "r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
           }
-          __syncwarp();
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barD) : "memory");
         }
+        __syncwarp();
       }
-      // the slot's shared memory is free once its last MMAs completed: prefetch the next pair
-      // while the epilogue warps still drain the accumulators
-      const int next = pair + gridDim.x;
-      if (next < npairs) {
-        for (int s2 = 0; s2 < 2 && ok; ++s2) {
-          ok = mbar_wait(barD[s2], 1);
-          if (ok && T == 0) fetch(next, s2);
-          __syncwarp();
-        }
+      // the operand buffer is free once the last MMAs completed: fetch the next unit under the last epilogues
+      if (ok && unit + 1 < u1) {
+        ok = mbar_wait(barD, 1);
+        if (ok && T == 0) fetch(unit + 1);
+        __syncwarp();
       }
     }
+    if (!ok) mbar_wait(barL, 0);                                // do not leave with a copy into this CTA still in flight
   } else {
-    // ---- epilogue warps ----
-    const int q = warp & 3, cq = warp >> 2;
-    for (int pair = blockIdx.x; pair < npairs && ok; pair += gridDim.x) {
+    // ---- epilogue warps: quadrant q, the two 64-column quarters of column half wh ----
+    const int q = warp & 3, wh = warp >> 2;
+    for (int unit = u0; unit < u1 && ok; ++unit) {
 #pragma unroll 1
       for (int stage = 0; stage < 4 && ok; ++stage) {
+        ok = mbar_wait(barD, stage & 1);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (stage == 3) {
+          const int gi = unit / p.ntile;                         // slab_local * R + k1
+          core_store(tmem, p.ws_out + (size_t)unit * k4OutBytes, q, wh, T, p.twr + 128 * (gi % p.R),
+                     __ldg(p.gscale + gi) * p.out_scale);
+        } else {
 #pragma unroll 1
-        for (int s2 = 0; s2 < 2 && ok; ++s2) {
-          ok = mbar_wait(barD[s2], stage & 1);
-          if (!ok) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t td = tmem + 256 * s2;
-          const int unit = 2 * pair + s2;
-          if (stage == 0) epilogue_twiddle<k8Lbo1, k8Sbo1, true>(td, Bsm[s2], q, cq, T, p.tw64);
-          else if (stage == 1) epilogue_gate(td, Bsm[s2], q, cq, T, Gsm[s2]);
-          else if (stage == 2) epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bsm[s2], q, cq, T, p.tw64);
-          else if (unit < p.nunits) core_store(td, p.ws_out + (size_t)unit * k4OutBytes, q, cq, T);
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          mbar_arrive(barB[s2]);
+          for (int cc = 0; cc < 2; ++cc) {
+            const int cq = 2 * wh + cc;
+            if (stage == 0) epilogue_twiddle<k4Lbo, k4Sbo, 1>(tmem, Bsm, q, cq, T, p.tw64);
+            else if (stage == 1) epilogue_gate_t<k4Lbo, k4Sbo, 64, true>(tmem, Bsm, q, cq, T, Gsm);
+            else epilogue_twiddle<k4Lbo, k4Sbo, 2>(tmem, Bsm, q, cq, T, p.tw64);
+          }
         }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(barB);
       }
     }
   }
   if (!ok && T == 0) atomicExch(p.status, 1);
+  __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == k4EpiWarps) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(512));
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(256));
   }
 }
 
@@ -383,14 +422,14 @@ __global__ void __launch_bounds__(k4CoreThreads, 1) tc_core_kernel(const TcCoreP
 // transpose-out
 // =====================================================================================
 struct TcOutParams {
-  const unsigned char* ws_out;   // [unit][t'][4] half2
-  const float* gscale;           // [slab_local * R + k1]
+  const unsigned char* ws_out;   // [unit][unit_row_slot(t')][4] half2
   bf16* dst;
   int64_t d_sb, d_sl, d_sh;
   int H, D, L, n, ntile, slab0;
 };
 
-// CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.
+// CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.  The units'
+// results arrive ready for the inverse radix-R step (conjugated, scaled, times conj(W_n^{k1 t'})).
 template <int R, bool F16>
 __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
   constexpr int NT = 512 / R;
@@ -401,15 +440,8 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t8 = lane >> 2, c4 = lane & 3;
   const int npair = p.D / 2;
-  const float base_scale = 1.0f / ((float)R * in_scale(R));
   const int skew_mask = (p.ntile & (p.ntile - 1)) == 0 ? min(p.ntile, 8) - 1 : 0;   // XOR stays inside the row
 
-  // gate scales of this head's R units, times 1 / (R s_in)
-  __shared__ float gsc[R];
-  __shared__ float2 tws[NT];                                   // W_n^{t'} of this CTA's t'
-  if (threadIdx.x < R) gsc[threadIdx.x] = __ldg(p.gscale + slab_local * R + threadIdx.x) * base_scale;
-  for (int tl = threadIdx.x; tl < NT; tl += 256) tws[tl] = twiddle_fwd((unsigned)(tb * NT + tl), (unsigned)p.n);
-  __syncthreads();
   // phase 1: a warp takes (tile, 8 consecutive t'); lane = (t' % 8, pair within the tile)
   const int nitems = p.ntile * (NT / 8);
   const uint32_t* wsl = reinterpret_cast<const uint32_t*>(p.ws_out + (size_t)slab_local * R * p.ntile * k4OutBytes);
@@ -417,20 +449,10 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
   for (int item = warp; item < nitems; item += 8) {
     const int tile = item % p.ntile, tl = (item / p.ntile) * 8 + t8;
     const int tp = tb * NT + tl;
-    const uint32_t* pu = wsl + tile * (k4OutBytes / 4) + tp * 4 + c4;
+    const uint32_t* pu = wsl + tile * (k4OutBytes / 4) + unit_row_slot(tp) * 4 + c4;
     float2 x[R];
 #pragma unroll
-    for (int k1 = 0; k1 < R; ++k1) {
-      float2 f = unpack_h2(__ldg(pu + k1 * ustride));
-      x[k1] = make_float2(f.x * gsc[k1], -f.y * gsc[k1]);       // result of conj(FFT(conj(.))), scaled
-    }
-    const float2 w1 = tws[tl];
-    float2 w = w1;
-#pragma unroll
-    for (int k = 1; k < R; ++k) {
-      x[k] = cmulc(x[k], w);                                    // times conj(W_n^{k1 t'})
-      w = cmul(w, w1);
-    }
+    for (int k1 = 0; k1 < R; ++k1) x[k1] = unpack_h2(__ldg(pu + k1 * ustride));   // scaled and twiddled by the core
     Dft<R, true>::run(x);
     const int word = (tile * 4 + c4) ^ ((tl & skew_mask) << 2);   // skew: the 8 rows of a warp hit 8 bank groups
     uint32_t* ps = stage + tl * npair + word;
@@ -517,15 +539,17 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   SPECTRE_LAUNCH_OK("tc_in_kernel");
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
-                     reinterpret_cast<const float4*>(ctx->tw64x64), (int)nunits, ntile, ctx->status_dev};
+                     reinterpret_cast<const float4*>(ctx->tw64x64),
+                     reinterpret_cast<const float2*>(ctx->tw_staged) + (size_t)(R - 1) * 128, gscale,
+                     1.0f / ((float)R * in_scale(R)), (int)nunits, ntile, R, ctx->status_dev};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
-  int grid = (int)((nunits + 1) / 2);               // pairs of units
-  if (grid > ctx->sm_count) grid = ctx->sm_count;
+  int grid = 2 * ctx->sm_count;                     // two resident CTAs per SM, a contiguous range of units each
+  if ((size_t)grid > nunits) grid = (int)nunits;
   tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
   SPECTRE_LAUNCH_OK("tc_core_kernel");
 
   constexpr int NT = 512 / R;
-  TcOutParams op = {ws_out, gscale, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
+  TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
                     y->H, D, y->L, n, ntile, slab0};
   const size_t smem_out = (size_t)R * NT * (D / 2) * 4;
   if (smem_out > 48 * 1024)

@@ -25,8 +25,11 @@ constexpr int k8GBytes = 64 * k8GStride * 4;     // per half, fp16 (re, im)
 // + {0, 1}.  It multiplies by W_4096^{row d} (read from a table laid out in this thread order, one
 // 16-byte load per x) and writes the transposed operand (row -> column index, d -> K) as one
 // 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
-//   COLS64: output columns 64 c + row (else 4 row + c).
-template <int LBO, int SBO, bool COLS64>
+//   COLS: order of the output columns.  1: 64 c + row.  0: 4 row + c.  2: 16 (row / 4) + 8 (c / 2) +
+//   2 (row % 4) + c % 2, which keeps the four rows a half-warp writes at once in four different
+//   16-byte slots of a core matrix even when LBO and SBO are multiples of 128 (dense images), and
+//   leaves all four pairs of a row in one thread of the epilogue that reads the next accumulator.
+template <int LBO, int SBO, int COLS>
 __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
                                                  const float4* __restrict__ tw) {
   const int i = T >> 2, tq = T & 3;
@@ -40,30 +43,42 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
     const int row = 8 * (2 * q + j) + i;
     float4 w[4];
 #pragma unroll
+#ifdef VAR_NOTW
+    for (int x = 0; x < 4; ++x) w[x] = make_float4(0.9f, 0.1f, 0.8f, 0.2f);
+#else
     for (int x = 0; x < 4; ++x) w[x] = __ldg(tw + (4 * step + x) * 32);
+#endif
     tmem_ld_wait();
     if (step < 3) {
       const int nj = (step + 1) >> 1, nchunk = (step + 1) & 1;
       tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * nj) << 16) + 32 * nchunk, r[(step + 1) & 1]);
     }
     const uint32_t (&rr)[16] = r[step & 1];
-    const uint32_t colpart = COLS64 ? (uint32_t)((8 * c + (row >> 3)) * SBO + (row & 7) * 16)
-                                    : (uint32_t)((row >> 1) * SBO + (4 * (row & 1) + c) * 16);
+    const uint32_t colpart = COLS == 1 ? (uint32_t)((8 * c + (row >> 3)) * SBO + (row & 7) * 16)
+                           : COLS == 0 ? (uint32_t)((row >> 1) * SBO + (4 * (row & 1) + c) * 16)
+                                       : (uint32_t)((2 * (row >> 2) + (c >> 1)) * SBO + (2 * (row & 3) + (c & 1)) * 16);
     const uint32_t base = colpart + (uint32_t)((8 * chunk + (tq >> 1)) * LBO + 8 * (tq & 1));
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
       const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), make_float2(w[x].x, w[x].y));
       const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), make_float2(w[x].z, w[x].w));
+#ifdef VAR_NOST
+      if (v0.x == 123.456f) *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
+#else
       *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
+#endif
     }
   }
 }
 
 // Epilogue after the second forward stage: rows k2, columns 64 c + k1; bin 2 (k1 + 64 k2) + parity
 // of the half.  Gate, conjugate (for the inverse by the conj trick) and write the operand with
-// the same columns and K = k2.
-__device__ __forceinline__ void epilogue_gate(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
-                                              const uint32_t* __restrict__ Gtab) {
+// the same columns and K = k2.  GXOR: the table is dense (64 entries per k2) with k1 XOR 8 (k2 % 4)
+// as the column, which spreads the four rows of a half-warp over the banks without padding;
+// otherwise entry (k1, k2) sits at GSTRIDE k2 + k1.
+template <int LBO, int SBO, int GSTRIDE, bool GXOR>
+__device__ __forceinline__ void epilogue_gate_t(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
+                                                const uint32_t* __restrict__ Gtab) {
   const int i = T >> 2, tq = T & 3;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * c;
@@ -78,17 +93,21 @@ __device__ __forceinline__ void epilogue_gate(uint32_t tmem_d, unsigned char* Bo
       tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * nj) << 16) + 32 * nchunk, r[(step + 1) & 1]);
     }
     const uint32_t (&rr)[16] = r[step & 1];
-    const uint32_t base = (uint32_t)((8 * c + 4 * chunk) * k8Sbo2 + (2 * tq) * 16 + (row >> 2) * k8Lbo2 + (row & 3) * 4);
-    const uint32_t* grow = Gtab + k8GStride * row + 32 * chunk + 2 * tq;
+    const uint32_t base = (uint32_t)((8 * c + 4 * chunk) * SBO + (2 * tq) * 16 + (row >> 2) * LBO + (row & 3) * 4);
+    const uint32_t* grow = Gtab + GSTRIDE * row + 32 * chunk + 2 * tq;
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
-      const uint2 gp = *reinterpret_cast<const uint2*>(grow + 8 * x);
+      const uint2 gp = *reinterpret_cast<const uint2*>(grow + 8 * (GXOR ? (x ^ (row & 3)) : x));
       const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), unpack_h2(gp.x));
       const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), unpack_h2(gp.y));
-      *reinterpret_cast<uint32_t*>(Bout + base + x * k8Sbo2) = pack_h2(v0.x, -v0.y);
-      *reinterpret_cast<uint32_t*>(Bout + base + x * k8Sbo2 + 16) = pack_h2(v1.x, -v1.y);
+      *reinterpret_cast<uint32_t*>(Bout + base + x * SBO) = pack_h2(v0.x, -v0.y);
+      *reinterpret_cast<uint32_t*>(Bout + base + x * SBO + 16) = pack_h2(v1.x, -v1.y);
     }
   }
+}
+__device__ __forceinline__ void epilogue_gate(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
+                                              const uint32_t* __restrict__ Gtab) {
+  epilogue_gate_t<k8Lbo2, k8Sbo2, k8GStride, false>(tmem_d, Bout, q, c, T, Gtab);
 }
 
 }  // namespace spectre
