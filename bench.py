@@ -209,7 +209,9 @@ class MixerBench:
             R, ntile = w.n // 4096, w.D // 8
             per = R * ntile * (65536 + 65536) + R * 16384 + 256
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))
-            self.kernel_name, nk = "mixer, staged tcgen05 path (tc_in incl. gate images + tc_core + tc_out per group)", 3 * groups
+            tc32 = R == 32 and w.D == 64 and w.L % 4096 == 0
+            self.kernel_name, nk = ("mixer, staged tcgen05 path (" + ("tc_in32 incl. gate images + tc_core + tc_out32" if tc32 else
+                                    "tc_in incl. gate images + tc_core + tc_out") + " per group)"), 3 * groups
         elif ws_mix:
             per = w.n * (w.D // 2) * 8
             groups = math.ceil(w.B * w.H / max(1, ws_mix // per))

@@ -9,14 +9,6 @@ constexpr int kTcLbo = 144;                    // bytes between core matrices al
 constexpr int kTcSbo = 2320;                   // bytes between 8-column groups (16 * 144 + 16 pad)
 constexpr int kTcBBytes = 32 * kTcSbo;         // one 256-column B operand
 constexpr int kTcFBytes = 128 * 128 * 2;
-// Optional phase stamps (SM clock), compiled in only for profiling builds.
-#ifdef SPECTRE_TC_TIMING
-__device__ long long g_tc_timing[1024][16];
-#define TC_STAMP(slot) do { if (T == 0 && warp == 0 && blockIdx.x < 1024) g_tc_timing[blockIdx.x][slot] = clock64(); } while (0)
-#else
-#define TC_STAMP(slot) do { } while (0)
-#endif
-
 // Byte offset of element (column nu, K index kappa) in a B operand.
 __device__ __forceinline__ uint32_t b_off(int nu, int kappa) {
   return (uint32_t)((nu >> 3) * kTcSbo + (kappa >> 3) * kTcLbo + (nu & 7) * 16 + (kappa & 7) * 2);
@@ -236,7 +228,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
 
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
   const int nwork = p.H * ((p.B + NH - 1) / NH);     // work items: NH batch entries of one head index
-  TC_STAMP(0);
 
   if (warp == EW) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(256 * NHALF));
@@ -268,7 +259,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = tmem_slot;
-  TC_STAMP(1);
 
   if (warp == EW) {
     // ---- MMA issuer: per work item 2 stages x NH / 2 halves, 7 K-steps each ----
@@ -373,7 +363,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");     // the previous item's accumulator reads are done
-    TC_STAMP(2);
     mbar_arrive(smem_u32(&bars[0]));
     if (NHALF == 2) mbar_arrive(smem_u32(&bars[1]));
 
@@ -434,7 +423,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
     // the column quarter is fixed, with 2 heads the one half's quarters 2 (warp >> 2) + unit
     const int q = warp & 3;
     const int i = T >> 2, t4 = T & 3;
-    TC_STAMP(3);
     // ---- gate epilogue: rows kM, columns (head, k1, pair) unchanged; next operand has K = kM ----
 #pragma unroll 1
     for (int unit = 0; unit < 2 && ok; ++unit) {
@@ -468,7 +456,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      TC_STAMP(4 + unit);
       if (NH == 4 || unit == 1) mbar_arrive(smem_u32(&bars[half]));
     }
     // ---- final: rows t', inverse radix-4 over k1 (columns 32 apart), bf16 rows t' + 49 n1 ----
@@ -528,7 +515,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
         }
       }
     }
-    TC_STAMP(6);
     if (J > 0) {
       // ---- wavelet refinement on the staged bf16 rows (Sec. 3.5): Haar over aligned blocks of 2^J
       //      tokens, bands scaled by 1 + s, synthesis; a thread takes 8 channels of one block and
@@ -610,7 +596,6 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
         }
       }
     }
-    TC_STAMP(7);
     // end of the item: the staged rows and level gates are free again; a wait that ran out ends the loop for all
     if (!ok) abort_s = 1;
     asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");

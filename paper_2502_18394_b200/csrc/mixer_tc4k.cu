@@ -506,6 +506,12 @@ size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
   return g * per;
 }
 
+// mixer_tc32.cu: the radix-32 steps on the tensor cores (n = 131072, d_head = 64)
+bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_act* y, int n);
+int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
+                   unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc);
+int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int slab0, int cnt);
+
 template <int R, bool F16>
 static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                       const spectre_act* y, int n, int slab0, int cnt, unsigned char* ws) {
@@ -516,8 +522,13 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   unsigned char* gimg = ws_out + nunits * k4OutBytes;
   float* gscale = reinterpret_cast<float*>(gimg + (size_t)cnt * R * k4GBytes);
 
+  const bool tc32 = R == 32 && tc32_supported(ctx, v, y, n);      // radix-32 steps on the tensor cores
   TcGateParams gp = {reinterpret_cast<const float2*>(g), gimg, gscale, n, n / 2 + 1, R, slab0};
 
+  if (tc32) {
+    int rc = launch_tc_in32(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, in_scale(R));
+    if (rc != SPECTRE_OK) return rc;
+  } else {
   constexpr int NT2 = (R <= 2) ? 64 : 128 / R;
   TcInParams ip = {reinterpret_cast<const bf16*>(v->ptr), v->stride_b, v->stride_l, v->stride_h, ws_in,
                    v->H, D, v->L, n, ntile, slab0};
@@ -537,6 +548,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   cfg.numAttrs = 1;
   SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_in_kernel<R, F16>, ip, gp, cnt * R));
   SPECTRE_LAUNCH_OK("tc_in_kernel");
+  }
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
                      reinterpret_cast<const float4*>(ctx->tw64x64),
@@ -548,6 +560,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
   SPECTRE_LAUNCH_OK("tc_core_kernel");
 
+  if (tc32) return launch_tc_out32(ctx, st, ws_out, y, slab0, cnt);
   constexpr int NT = 512 / R;
   TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
                     y->H, D, y->L, n, ntile, slab0};

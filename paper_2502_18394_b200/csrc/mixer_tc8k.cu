@@ -40,13 +40,6 @@ constexpr int k8EpiThreads = 32 * k8EpiWarps;
 constexpr int k8Threads = k8EpiThreads + 32;     // + 1 warp issuing copies and MMAs
 static_assert(16 * k8Lbo1 <= k8BBytes && 16 * k8Lbo2 <= k8BBytes && k8Smem <= 232448, "shared memory layout");
 
-#ifdef SPECTRE_TC_TIMING
-__device__ long long g_tc8k_timing[1024][16];
-#define TC8K_STAMP(slot) do { if (T == 0 && warp == 0 && blockIdx.x < 1024) g_tc8k_timing[blockIdx.x][slot] = clock64(); } while (0)
-#else
-#define TC8K_STAMP(slot) do { } while (0)
-#endif
-
 struct Tc8kParams {
   const float2* g;        // [B*H][4097]
   const __half* F;        // 64-point DFT matrix, canonical smem layout
@@ -102,7 +95,6 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
   const int col0 = tile * 8;
   const float2* g = p.g + (size_t)slab * 4097;
 
-  TC8K_STAMP(0);
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), k8EpiThreads);
     mbar_init(smem_u32(&bars[1]), k8EpiThreads);
@@ -121,7 +113,6 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
   // run while that kernel finishes (if it triggers early, as the gate kernels do); nothing of V or g
   // is read before its writes are visible.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  TC8K_STAMP(1);
 
   if (warp == k8EpiWarps) {
     bool ok = true;
@@ -191,7 +182,6 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
       Gsm[0][(k & 1) * (k8GBytes / 4) + k8GStride * (m >> 6) + (m & 63)] = pack_h2(gv[i].x * ginv, gv[i].y * ginv);
     }
     asm volatile("bar.sync 1, %0;" :: "r"(k8EpiThreads) : "memory");
-    TC8K_STAMP(2);
 
     // ---- radix-2 step in place: rows t (landed in Bsm[0]) and t + 4096 (Bsm[1]) -> e, o in fp16.
     //      A thread takes t1 = 4a..4a+3 at one t2: four 16-byte chunks (one row each, 4 pairs) in,
@@ -236,7 +226,6 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
       }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    TC8K_STAMP(3);
     mbar_arrive(smem_u32(&bars[0]));
     mbar_arrive(smem_u32(&bars[1]));
 
@@ -256,7 +245,6 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
         else epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bh, q, cq, T, p.tw64);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        TC8K_STAMP(4 + 2 * stage + half);
         mbar_arrive(smem_u32(&bars[half]));
       }
     }
@@ -265,7 +253,6 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
     //      ((s1 & 7) * 64 + t1) * 16; each column quarter hands its boxes to the TMA engine ----
     if (ok) ok = mbar_wait(smem_u32(&bars[2]), 1);
     if (ok) ok = mbar_wait(smem_u32(&bars[3]), 1);
-    TC8K_STAMP(10);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int i = T >> 2, pp = (T >> 1) & 1, cp = T & 1;
@@ -315,12 +302,10 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
       }
       if (q == 0 && T == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
-    TC8K_STAMP(11);
     if (!ok && T == 0) atomicExch(p.status, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  TC8K_STAMP(12);
   if (warp == k8EpiWarps) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(512));

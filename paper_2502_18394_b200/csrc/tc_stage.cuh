@@ -43,11 +43,7 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
     const int row = 8 * (2 * q + j) + i;
     float4 w[4];
 #pragma unroll
-#ifdef VAR_NOTW
-    for (int x = 0; x < 4; ++x) w[x] = make_float4(0.9f, 0.1f, 0.8f, 0.2f);
-#else
     for (int x = 0; x < 4; ++x) w[x] = __ldg(tw + (4 * step + x) * 32);
-#endif
     tmem_ld_wait();
     if (step < 3) {
       const int nj = (step + 1) >> 1, nchunk = (step + 1) & 1;
@@ -62,11 +58,7 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
     for (int x = 0; x < 4; ++x) {
       const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), make_float2(w[x].x, w[x].y));
       const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), make_float2(w[x].z, w[x].w));
-#ifdef VAR_NOST
-      if (v0.x == 123.456f) *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
-#else
       *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
-#endif
     }
   }
 }
