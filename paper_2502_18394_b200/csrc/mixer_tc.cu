@@ -42,7 +42,7 @@ __global__ void build_tw8192_kernel(float2* tab) {
 
 // Twiddles between the two 64-point stages of a 4096-point transform, in the order the epilogue
 // threads use them: entry ((((q 2 + j) 2 + chunk) 4 + x) 32 + lane) holds W_4096^{row d} and
-// W_4096^{row (d + 1)} for row = 8 (2q + j) + lane / 4 and d = 32 chunk + 8 x + 2 (lane % 4).
+// W_4096^{row (d + 1)} (real parts first, then imaginary parts) for row = 8 (2q + j) + lane / 4 and d = 32 chunk + 8 x + 2 (lane % 4).
 __global__ void build_tw64x64_kernel(float4* tab) {
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= 2048) return;
@@ -51,7 +51,7 @@ __global__ void build_tw64x64_kernel(float4* tab) {
   float s0, c0, s1, c1;
   sincospif((float)((row * d) & 4095) / 2048.0f, &s0, &c0);
   sincospif((float)((row * (d + 1)) & 4095) / 2048.0f, &s1, &c1);
-  tab[idx] = make_float4(c0, -s0, c1, -s1);
+  tab[idx] = make_float4(c0, c1, -s0, -s1);             // (re, re, im, im) of the two: operands of the packed products
 }
 
 int build_tw64x64(float4* tab, cudaStream_t st) {

@@ -270,16 +270,24 @@ __device__ __forceinline__ void core_store(uint32_t tmem_d, unsigned char* out, 
     const uint32_t (&rr)[16] = r[step & 1];
 #pragma unroll
     for (int s = 0; s < 2; ++s) {                               // s1 / 4 = 8 ch + 2 cc + s; 8-column groups 2 s, 2 s + 1 = pairs 0-1, 2-3
+      // conj(D w) = D conj-multiplied: (re, -im) of D w, with the sign folded into the second factor
       const float2 w = cmul(fa[j], fb[2 * cc + s]);
-      uint32_t o[4];
+      const uint64_t WX = pk2(w.x, w.x), WYn = pk2(-w.y, -w.y);
+      uint2 o[2];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {                             // pair e: group 2 s + e / 2, column e % 2
-        const int b0 = 4 * (2 * s + (e >> 1)) + (e & 1);
-        const float2 pz = cmul(make_float2(__uint_as_float(rr[b0]), __uint_as_float(rr[b0 + 2])), w);
-        o[e] = pack_h2(pz.x, -pz.y);
+      for (int e2 = 0; e2 < 2; ++e2) {                          // pairs 2 e2, 2 e2 + 1: 8-column group 2 s + e2
+        const int b0 = 4 * (2 * s + e2);
+        const uint64_t RE = pk2u(rr[b0], rr[b0 + 1]), IM = pk2u(rr[b0 + 2], rr[b0 + 3]);
+        // D w = (re w.x - im w.y) + j (re w.y + im w.x); stored: (real, -imag)
+        const uint64_t X = fma2(IM, WYn, mul2(RE, WX));
+        const uint64_t Yn = sub2(mul2(RE, WYn), mul2(IM, WX));
+        float x0, x1, y0, y1;
+        upk2(X, x0, x1);
+        upk2(Yn, y0, y1);
+        o[e2] = make_uint2(pack_h2(x0, y0), pack_h2(x1, y1));
       }
       const int k = 8 * ch + 2 * cc + s;                        // s1 / 4
-      *reinterpret_cast<uint4*>(out + (size_t)((k * 64 + row) * 4 + tq) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(out + (size_t)((k * 64 + row) * 4 + tq) * 16) = make_uint4(o[0].x, o[0].y, o[1].x, o[1].y);
     }
   }
 }

@@ -64,6 +64,46 @@ __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d)
   return make_uint2(pack_bf2(a, b), pack_bf2(c, d));
 }
 
+// ---- packed fp32 pairs (sm_100: one instruction works on two fp32 values in a 64-bit register) ----
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pk2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+// Two complex products at once: (re0 + j im0) w0 and (re1 + j im1) w1 with RE = (re0, re1), IM = (im0, im1),
+// WX = (w0.x, w1.x), WY = (w0.y, w1.y); results as half2 (re, im) each.
+__device__ __forceinline__ uint2 cmul2_pack_h2(uint64_t RE, uint64_t IM, uint64_t WX, uint64_t WY) {
+  const uint64_t X = sub2(mul2(RE, WX), mul2(IM, WY));
+  const uint64_t Y = fma2(RE, WY, mul2(IM, WX));
+  float x0, x1, y0, y1;
+  upk2(X, x0, x1);
+  upk2(Y, y0, y1);
+  return make_uint2(pack_h2(x0, y0), pack_h2(x1, y1));
+}
+
 // 16 lanes x 32 columns of fp32: thread T gets, per 8-column group x, rows T/4 (r[4x], r[4x+1])
 // and T/4 + 8 (r[4x+2], r[4x+3]) at columns 8x + 2(T%4) + {0, 1}.
 __device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {

@@ -23,7 +23,7 @@ constexpr int k8GBytes = 64 * k8GStride * 4;     // per half, fp16 (re, im)
 // contracted), for one warp: TMEM lane quadrant q, pair c.  A thread owns rows (new digit)
 // 16 q' + T/4 for the two lane groups q' = 2q, 2q+1 and the columns d = 32 chunk + 8 x + 2 (T%4)
 // + {0, 1}.  It multiplies by W_4096^{row d} (read from a table laid out in this thread order, one
-// 16-byte load per x) and writes the transposed operand (row -> column index, d -> K) as one
+// 16-byte load per x; the two products of an x run as packed fp32 pairs) and writes the transposed operand (row -> column index, d -> K) as one
 // 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
 //   COLS: order of the output columns.  1: 64 c + row.  0: 4 row + c.  2: 16 (row / 4) + 8 (c / 2) +
 //   2 (row % 4) + c % 2, which keeps the four rows a half-warp writes at once in four different
@@ -56,9 +56,9 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
     const uint32_t base = colpart + (uint32_t)((8 * chunk + (tq >> 1)) * LBO + 8 * (tq & 1));
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
-      const float2 v0 = cmul(make_float2(__uint_as_float(rr[4 * x]), __uint_as_float(rr[4 * x + 2])), make_float2(w[x].x, w[x].y));
-      const float2 v1 = cmul(make_float2(__uint_as_float(rr[4 * x + 1]), __uint_as_float(rr[4 * x + 3])), make_float2(w[x].z, w[x].w));
-      *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) = make_uint2(pack_h2(v0.x, v0.y), pack_h2(v1.x, v1.y));
+      // table entry: (w0.x, w1.x, w0.y, w1.y) for the two columns of the thread
+      *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) =
+          cmul2_pack_h2(pk2u(rr[4 * x], rr[4 * x + 1]), pk2u(rr[4 * x + 2], rr[4 * x + 3]), pk2(w[x].x, w[x].y), pk2(w[x].z, w[x].w));
     }
   }
 }
