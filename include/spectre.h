@@ -40,7 +40,8 @@ typedef enum {
   SPECTRE_ERR_UNSUPPORTED = 2,   /* valid request outside the supported set              */
   SPECTRE_ERR_WORKSPACE = 3,     /* workspace missing or smaller than the query result   */
   SPECTRE_ERR_CUDA = 4,          /* a CUDA runtime call or launch failed                 */
-  SPECTRE_ERR_TIMEOUT = 5        /* a bounded on-chip wait ran out (spectre_poll_status) */
+  SPECTRE_ERR_TIMEOUT = 5,       /* a bounded on-chip wait ran out (spectre_poll_status) */
+  SPECTRE_ERR_RANGE = 6          /* a 16-bit tensor-core mixer overflowed (spectre_poll_status) */
 } spectre_status;
 
 /* Element types of activations and ring buffers; weights are SPECTRE_F32 or SPECTRE_BF16. */
@@ -54,11 +55,22 @@ typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch l
  * pinned status word, all released by spectre_destroy.  No other call allocates. */
 int spectre_create(spectre_ctx** out, int device);
 int spectre_destroy(spectre_ctx* ctx);
-/* The tensor-core mixer hands tiles between its warps through on-chip barriers whose waits
- * are bounded; a wait that runs out makes the kernel finish early and record it.  Call this
- * after synchronising the stream: SPECTRE_OK, or SPECTRE_ERR_TIMEOUT (and the record is
- * cleared) if any kernel since the last poll gave up, in which case its output is invalid. */
+/* The tensor-core mixers record two kinds of trouble in a status word instead of failing on
+ * the device.  (1) They hand tiles between their warps through on-chip barriers whose waits are
+ * bounded; a wait that runs out makes the kernel finish early.  (2) Their intermediates are
+ * fp16 (see spectre_mixer_forward for the amplitude range this allows); a call whose input
+ * leaves that range ends in Inf / NaN outputs, which the last epilogue notices.  Call this
+ * after synchronising the stream: SPECTRE_OK, or - the record is cleared - SPECTRE_ERR_TIMEOUT
+ * if any kernel since the last poll gave up on a wait (its output is invalid), else
+ * SPECTRE_ERR_RANGE if one produced non-finite values (rerun that call on the fp32 path:
+ * environment variable SPECTRE_FORCE_PATH=alu). */
 int spectre_poll_status(spectre_ctx* ctx);
+/* Diagnostic (the paper has no counterpart): enqueues a one-warp kernel whose bounded wait
+ * runs out by construction - a barrier nobody arrives on, 4096 polls, no copy or MMA in
+ * flight - and which reports it the way the mixers do, so that the path wait -> status word ->
+ * spectre_poll_status can be exercised without disturbing a real kernel.  After the stream
+ * is synchronised the next spectre_poll_status returns SPECTRE_ERR_TIMEOUT once. */
+int spectre_selftest_wait_timeout(spectre_ctx* ctx, void* stream);
 /* Static description of a status code. */
 const char* spectre_status_string(int status);
 /* Text of the most recent failure on the calling thread ("" if none). */
@@ -201,6 +213,16 @@ typedef struct {
  *              n_fft = 196, D = 64 the workspace only holds the level gates that
  *              wrm's MLP produces for the refinement fused into the mixer kernel
  *              (B H 3 D floats): with less, the refinement runs as its own kernel
+ * Amplitude range of the 16-bit paths.  bf16 / fp16 activations at n_fft = 196 (D = 64) and
+ * n_fft = 4096 ... 131072 run on the tensor cores with fp16 operands between the stages and
+ * fixed power-of-two stage scales (unitary overall), fp32 accumulation.  Noise-like data passes
+ * at any plausible magnitude, but a column with a constant or periodic component of amplitude A
+ * concentrates A sqrt(n_fft) in one bin: beyond A of about 250 at n_fft = 131072, 500 at 8192 and
+ * 1000 at 196 an intermediate exceeds 65504, the outputs turn into Inf / NaN, and
+ * spectre_poll_status reports SPECTRE_ERR_RANGE.  Data whose magnitude is below about 1e-3
+ * gradually loses accuracy in fp16 subnormals, without a report.  f32 activations, and any
+ * activations with the environment variable SPECTRE_FORCE_PATH=alu, take the fp32 path, which has
+ * neither limit.
  */
 size_t spectre_mixer_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t L, int32_t H,
                                      int32_t D, int32_t n_fft, int32_t dtype);

@@ -22,12 +22,14 @@ SPECTRE_ERR_UNSUPPORTED = 2
 SPECTRE_ERR_WORKSPACE = 3
 SPECTRE_ERR_CUDA = 4
 SPECTRE_ERR_TIMEOUT = 5
+SPECTRE_ERR_RANGE = 6
 SPECTRE_F32 = 0
 SPECTRE_BF16 = 1
 SPECTRE_F16 = 2
 
 EXPORTS = [
     "spectre_create", "spectre_destroy", "spectre_status_string", "spectre_last_error", "spectre_poll_status",
+    "spectre_selftest_wait_timeout",
     "spectre_gate_workspace_bytes", "spectre_gate", "spectre_gate_static_max_bytes", "spectre_gate_static",
     "spectre_mixer_workspace_bytes", "spectre_mixer_forward",
     "spectre_wavelet_refine",
@@ -84,6 +86,8 @@ def lib():
     L.spectre_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
     L.spectre_destroy.argtypes = [C.c_void_p]
     L.spectre_poll_status.argtypes = [C.c_void_p]
+    L.spectre_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_void_p]
+    L.spectre_selftest_wait_timeout.restype = C.c_int
     L.spectre_status_string.argtypes = [C.c_int]
     L.spectre_status_string.restype = C.c_char_p
     L.spectre_last_error.restype = C.c_char_p
@@ -168,8 +172,13 @@ class Context:
         self.device = device
 
     def poll_status(self):
-        """Raises SpectreError(SPECTRE_ERR_TIMEOUT) if a kernel gave up on a bounded wait (call after a sync)."""
+        """Raises SpectreError(SPECTRE_ERR_TIMEOUT) if a kernel gave up on a bounded wait, or
+        SpectreError(SPECTRE_ERR_RANGE) if a 16-bit tensor-core mixer overflowed (call after a sync)."""
         _check(lib().spectre_poll_status(self.handle))
+
+    def selftest_wait_timeout(self):
+        """Enqueues the diagnostic kernel whose bounded wait runs out by construction."""
+        _check(lib().spectre_selftest_wait_timeout(self.handle, _stream()))
 
     def close(self):
         if self.handle:

@@ -2,9 +2,7 @@
 #include <cstdio>
 #include <new>
 
-#include "common.cuh"
-
-#include <cuda_fp16.h>
+#include "tc_common.cuh"
 
 namespace spectre {
 
@@ -152,8 +150,33 @@ extern "C" int spectre_poll_status(spectre_ctx* ctx) {
   int v = *reinterpret_cast<volatile int*>(ctx->status_host);
   if (v != 0) {
     *reinterpret_cast<volatile int*>(ctx->status_host) = 0;
-    return fail(SPECTRE_ERR_TIMEOUT, "a kernel gave up on a bounded on-chip wait; its outputs are undefined");
+    if (v & 1) return fail(SPECTRE_ERR_TIMEOUT, "a kernel gave up on a bounded on-chip wait; its outputs are undefined");
+    return fail(SPECTRE_ERR_RANGE,
+                "a tensor-core mixer produced non-finite values: its fp16 intermediates overflowed (input amplitude beyond "
+                "the documented range); rerun that call with SPECTRE_FORCE_PATH=alu");
   }
+  return SPECTRE_OK;
+}
+
+// One warp, one barrier nobody arrives on, a short poll limit: the wait runs out by construction (no copy,
+// no MMA in flight), the kernel records it like the mixers do and returns normally.
+__global__ void wait_selftest_kernel(int* status) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const bool ok = mbar_wait_limit(b, 0, 4096);
+  if (!ok && threadIdx.x == 0) report_timeout(status);
+}
+
+extern "C" int spectre_selftest_wait_timeout(spectre_ctx* ctx, void* stream) {
+  if (!ctx) return fail(SPECTRE_ERR_INVALID_ARG, "ctx is NULL");
+  SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
+  wait_selftest_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(ctx->status_dev);
+  SPECTRE_LAUNCH_OK("wait_selftest_kernel");
   return SPECTRE_OK;
 }
 
@@ -165,6 +188,7 @@ extern "C" const char* spectre_status_string(int status) {
     case SPECTRE_ERR_WORKSPACE: return "workspace missing or too small";
     case SPECTRE_ERR_CUDA: return "CUDA error";
     case SPECTRE_ERR_TIMEOUT: return "device-side wait timed out";
+    case SPECTRE_ERR_RANGE: return "input amplitude outside the range of the 16-bit tensor-core path";
     default: return "unknown status";
   }
 }

@@ -287,11 +287,12 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
         __syncwarp();
       }
     }
-    if (!ok && T == 0) atomicExch(p.status, 1);
+    if (!ok && T == 0) report_timeout(p.status);
   } else {
     // The CTA keeps its DFT matrix, accumulators and barriers over all its work items: the barriers
     // complete two phases per item, so every item sees the same parities.
     bool ok = true;
+    bool bad = false;                                 // a non-finite result: the fp16 intermediates overflowed
 #pragma unroll 1
     for (int work = blockIdx.x; work < nwork; work += gridDim.x) {
     // the item's heads are batch entries bg NH .. bg NH + NH - 1 of ONE head index hh: they share the
@@ -508,6 +509,7 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
               const int row = tp + 49 * n1;
               const uint2 out = F16 ? make_uint2(pack_h2(gs * y0[n1].x, gs * y0[n1].y), pack_h2(gs * y1[n1].x, gs * y1[n1].y))
                                     : pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y);
+              bad |= nonfinite16x2<F16>(out.x) | nonfinite16x2<F16>(out.y);
               if (J > 0) *reinterpret_cast<uint2*>(Bsm[half] + ((hl & 1) * 196 + row) * k196StageRow + 2 * col) = out;
               else if (row < p.L) __stcs(reinterpret_cast<uint2*>(dst + (int64_t)row * p.d_sl + col), out);
             }
@@ -601,7 +603,8 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
     asm volatile("bar.sync 1, %0;" :: "r"(ET) : "memory");
     if (abort_s) break;
     }
-    if (!ok && T == 0) atomicExch(p.status, 1);
+    if (!ok && T == 0) report_timeout(p.status);
+    if (__any_sync(0xffffffffu, bad) && T == 0) report_range(p.status);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

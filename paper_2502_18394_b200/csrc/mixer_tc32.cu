@@ -297,7 +297,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
     }
   }
   if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-  if (!ok && T == 0) atomicExch(p.status, 1);
+  if (!ok && T == 0) report_timeout(p.status);
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -391,6 +391,7 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
     // ---- epilogue warps: lane quadrant q: tiles 4 (q / 2) .. + 3, n1 = 16 (q % 2) + 8 j + i; column half wh ----
     const int q = warp & 3, wh = (warp >> 2) & 1, j = warp >> 3, i = T >> 2, tq = T & 3, gq = q >> 1;
     const int n1 = 16 * (q & 1) + 8 * j + i;
+    bool bad = false;                                            // a non-finite result: the fp16 intermediates overflowed
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
       const int slab = p.slab0 + item % p.cnt, blk = item / p.cnt;
@@ -420,7 +421,9 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
               // rows (n1, C) and (n1, S) applied to the columns (re, im): y = (C re - S im) + j (S re + C im)
               const float ya = __uint_as_float(rr[4 * x]) - __uint_as_float(rr[4 * x + 3]);
               const float yb = __uint_as_float(rr[4 * x + 2]) + __uint_as_float(rr[4 * x + 1]);
-              *reinterpret_cast<uint32_t*>(prow + (4 * wh + x) * 4096) = F16 ? pack_h2(ya, yb) : pack_bf2(ya, yb);
+              const uint32_t yo = F16 ? pack_h2(ya, yb) : pack_bf2(ya, yb);
+              bad |= nonfinite16x2<F16>(yo);
+              *reinterpret_cast<uint32_t*>(prow + (4 * wh + x) * 4096) = yo;
             }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -438,8 +441,9 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
       }
     }
     if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (__any_sync(0xffffffffu, bad) && T == 0) report_range(p.status);
   }
-  if (!ok && T == 0) atomicExch(p.status, 1);
+  if (!ok && T == 0) report_timeout(p.status);
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

@@ -416,7 +416,7 @@ __global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreP
       }
     }
   }
-  if (!ok && T == 0) atomicExch(p.status, 1);
+  if (!ok && T == 0) report_timeout(p.status);
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -434,6 +434,7 @@ struct TcOutParams {
   bf16* dst;
   int64_t d_sb, d_sl, d_sh;
   int H, D, L, n, ntile, slab0;
+  int* status;
 };
 
 // CTA = (slab, block of NT consecutive t'); rows n1 * 4096 + t' for all n1 are produced.  The units'
@@ -452,6 +453,7 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
 
   // phase 1: a warp takes (tile, 8 consecutive t'); lane = (t' % 8, pair within the tile)
   const int nitems = p.ntile * (NT / 8);
+  bool bad = false;                                             // a non-finite result: the fp16 intermediates overflowed
   const uint32_t* wsl = reinterpret_cast<const uint32_t*>(p.ws_out + (size_t)slab_local * R * p.ntile * k4OutBytes);
   const int ustride = p.ntile * (k4OutBytes / 4);               // words between consecutive k1 (same tile)
   for (int item = warp; item < nitems; item += 8) {
@@ -466,14 +468,12 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
     uint32_t* ps = stage + tl * npair + word;
 #pragma unroll
     for (int n1 = 0; n1 < R; ++n1) {
-      if (F16) {
-        ps[n1 * NT * npair] = pack_h2(x[n1].x, x[n1].y);
-      } else {
-        __nv_bfloat162 o = __floats2bfloat162_rn(x[n1].x, x[n1].y);
-        ps[n1 * NT * npair] = *reinterpret_cast<uint32_t*>(&o);
-      }
+      const uint32_t o = F16 ? pack_h2(x[n1].x, x[n1].y) : pack_bf2(x[n1].x, x[n1].y);
+      bad |= nonfinite16x2<F16>(o);
+      ps[n1 * NT * npair] = o;
     }
   }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) report_range(p.status);
   __syncthreads();
   // phase 2: whole rows
   bf16* dst = p.dst + b * p.d_sb + h * p.d_sh;
@@ -571,7 +571,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   if (tc32) return launch_tc_out32(ctx, st, ws_out, y, slab0, cnt);
   constexpr int NT = 512 / R;
   TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
-                    y->H, D, y->L, n, ntile, slab0};
+                    y->H, D, y->L, n, ntile, slab0, ctx->status_dev};
   const size_t smem_out = (size_t)R * NT * (D / 2) * 4;
   if (smem_out > 48 * 1024)
     SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel<R, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_out));

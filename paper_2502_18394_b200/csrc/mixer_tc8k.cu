@@ -158,7 +158,13 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
         __syncwarp();
       }
     }
-    if (!ok && T == 0) atomicExch(p.status, 1);
+    if (!ok) {
+      if (T == 0) report_timeout(p.status);
+      // do not leave with copies into this CTA's shared memory still in flight (bounded again)
+      mbar_wait(smem_u32(&bars[4]), 0);
+      mbar_wait(smem_u32(&bars[5]), 0);
+      mbar_wait(smem_u32(&bars[6]), 0);
+    }
   } else {
     // ---- gate tables (while the rows are in flight): Hermitian extension, normalised by a bound
     //      on max |g| so that the gated spectrum stays in fp16 range; bin 2 (k1 + 64 k2) + parity ----
@@ -260,6 +266,7 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
       const float2 wstep = twiddle8192(p.tw, 2u);
       const uint32_t taddr0 = tmem + ((uint32_t)(32 * q) << 16) + 64 * cq;
       uint32_t re[2][16], ro[2][16];
+      bool bad = false;                                          // a non-finite result: the fp16 intermediates overflowed
       tmem_ld_16x256b_x4(taddr0, re[0]);
       tmem_ld_16x256b_x4(taddr0 + 256, ro[0]);
 #pragma unroll
@@ -284,10 +291,11 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
           const float2 o0 = cmul(make_float2(__uint_as_float(xo[4 * x]), __uint_as_float(xo[4 * x + 2])), w);
           const float2 o1 = cmul(make_float2(__uint_as_float(xo[4 * x + 1]), __uint_as_float(xo[4 * x + 3])), w);
           if (x < 3) w = cmul(w, wstep);
-          *reinterpret_cast<uint2*>(Bsm[0] + base + 2048 * x) =
-              pack_io4<F16>(gs * (e0.x + o0.x), -gs * (e0.y + o0.y), gs * (e1.x + o1.x), -gs * (e1.y + o1.y));
-          *reinterpret_cast<uint2*>(Bsm[1] + base + 2048 * x) =
-              pack_io4<F16>(gs * (e0.x - o0.x), -gs * (e0.y - o0.y), gs * (e1.x - o1.x), -gs * (e1.y - o1.y));
+          const uint2 ylo = pack_io4<F16>(gs * (e0.x + o0.x), -gs * (e0.y + o0.y), gs * (e1.x + o1.x), -gs * (e1.y + o1.y));
+          const uint2 yhi = pack_io4<F16>(gs * (e0.x - o0.x), -gs * (e0.y - o0.y), gs * (e1.x - o1.x), -gs * (e1.y - o1.y));
+          bad |= nonfinite16x2<F16>(ylo.x) | nonfinite16x2<F16>(ylo.y) | nonfinite16x2<F16>(yhi.x) | nonfinite16x2<F16>(yhi.y);
+          *reinterpret_cast<uint2*>(Bsm[0] + base + 2048 * x) = ylo;
+          *reinterpret_cast<uint2*>(Bsm[1] + base + 2048 * x) = yhi;
         }
         if (j == 1) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -301,8 +309,9 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
         }
       }
       if (q == 0 && T == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      if (__any_sync(0xffffffffu, bad) && T == 0) report_range(p.status);
     }
-    if (!ok && T == 0) atomicExch(p.status, 1);
+    if (!ok && T == 0) report_timeout(p.status);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(kPjThreads, 3) project_qv_kernel(const ProjPar
             }
       }
     }
-    if (!ok && T == 0) atomicExch(p.status, 1);
+    if (!ok && T == 0) report_timeout(p.status);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

@@ -26,8 +26,9 @@ __device__ __forceinline__ uint32_t umma_idesc_128x256() {
   return (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kTcSpinLimit; ++it) {
+// Bounded wait: false once `limit` polls have passed without the phase completing.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
@@ -35,6 +36,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (ok) return true;
   }
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_limit(bar, parity, kTcSpinLimit); }
+
+// The status word the host polls: bit 0 = a bounded wait ran out, bit 1 = a result left the fp16 range
+// of the tensor-core path's intermediates (non-finite output).
+__device__ __forceinline__ void report_timeout(int* status) { atomicOr(status, 1); }
+__device__ __forceinline__ void report_range(int* status) { atomicOr(status, 2); }
+// two packed 16-bit outputs (bf16 or fp16): is either one Inf or NaN
+template <bool F16> __device__ __forceinline__ bool nonfinite16x2(uint32_t u) {
+  const uint32_t m = F16 ? 0x7c007c00u : 0x7f807f80u, e = u & m;
+  return (e & 0xffffu) == (m & 0xffffu) || (e >> 16) == (m >> 16);
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" :: "r"(bar) : "memory");

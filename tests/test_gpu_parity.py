@@ -706,3 +706,51 @@ def test_invalid_arguments_are_rejected_before_launch(ctx):
         S.spectre_wavelet_refine(ctx, x[:, :62].contiguous(), {"levels": 2, "level_gates": torch.zeros(1, 2, 3, 16, device="cuda")})
     torch.cuda.synchronize()                                   # context still healthy
     assert float(S.spectre_mixer_forward(ctx, x, g).abs().max()) == 0.0
+
+
+# ------------------------------------------------------------------ status word: waits that run out, range
+def test_bounded_wait_that_runs_out_is_reported_once_and_the_context_stays_usable(ctx):
+    # a kernel whose wait runs out by construction (barrier nobody arrives on, nothing in flight): the
+    # status word is set, the poll reports it once and clears it, and the next real call is correct
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ctx.selftest_wait_timeout()
+    torch.cuda.synchronize()
+    with pytest.raises(S.SpectreError) as e:
+        ctx.poll_status()
+    assert e.value.status == S.SPECTRE_ERR_TIMEOUT
+    ctx.poll_status()                                        # cleared
+    w = W.Workload("t", B=1, L=8192, H=2, D=64, dtype="bf16", seed=4)
+    assert run_mixer(ctx, w) < TOL["bf16"]
+    torch.cuda.synchronize()
+    ctx.poll_status()
+
+
+@pytest.mark.parametrize("n,H", [(8192, 2), (131072, 1), (196, 3), (16384, 2)])
+def test_16bit_paths_report_overflow_and_small_inputs_keep_their_accuracy(ctx, n, H, monkeypatch):
+    # the tensor-core paths keep fp16 intermediates: a constant channel far beyond the documented
+    # amplitude must not pass silently (non-finite outputs are reported by the poll), the fp32 path
+    # takes the same tensor, and a whole tensor scaled down by 1e-2 still meets the bound
+    w = W.Workload("t", B=1, L=n, H=H, D=64, dtype="bf16", seed=n)
+    x = W.activations(w)
+    g = W.random_gate(w)
+    gc = gate_to_complex(g)
+    big = x.clone()
+    big[:, :, 0, 3] = 30000.0                                # constant column: A sqrt(n) far beyond fp16
+    y = S.spectre_mixer_forward(ctx, big.cuda(), g.cuda())
+    torch.cuda.synchronize()
+    with pytest.raises(S.SpectreError) as e:
+        ctx.poll_status()
+    assert e.value.status == S.SPECTRE_ERR_RANGE
+    ctx.poll_status()                                        # cleared
+    monkeypatch.setenv("SPECTRE_FORCE_PATH", "alu")
+    y = S.spectre_mixer_forward(ctx, big.cuda(), g.cuda())
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    assert slab_err(W.to_f64(y), O.mixer(W.to_f64(big), gc)) < TOL["bf16"]
+    monkeypatch.delenv("SPECTRE_FORCE_PATH")
+    small = (x.float() * 1e-2).to(torch.bfloat16)
+    y = S.spectre_mixer_forward(ctx, small.cuda(), g.cuda())
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    assert slab_err(W.to_f64(y), O.mixer(W.to_f64(small), gc)) < TOL["bf16"]
