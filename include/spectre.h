@@ -201,8 +201,9 @@ typedef struct {
  *   v, y     activations of identical shape and dtype; y may alias v where the
  *            transform is one kernel (the workspace query returns 0, and the
  *            bf16 / fp16 tensor-core paths n_fft = 196 with D = 64 and
- *            n_fft = 8192); on a multi-pass path an aliased call is refused
- *            with SPECTRE_ERR_INVALID_ARG
+ *            n_fft = 8192); on a multi-pass path a call whose v and y overlap
+ *            anywhere between their first and last byte is refused with
+ *            SPECTRE_ERR_INVALID_ARG
  *   g        [B, H, K, 2] float32, K = n_fft/2 + 1; one gain per bin per head,
  *            applied to all D columns; Im of the DC / Nyquist gains is ignored
  *   n_fft    == L: exact circular transform of Eq. 1;  > L: rows L..n_fft-1 are

@@ -733,8 +733,19 @@ extern "C" int spectre_mixer_forward(spectre_ctx* ctx, void* stream, const spect
     if (workspace_bytes < slab_ws_bytes(n_fft, v->D))
       return fail(SPECTRE_ERR_WORKSPACE, "mixer workspace smaller than one (batch, head) slab");
   }
-  if ((staged || pl.N1 > 1) && v->ptr == y->ptr)
-    return fail(SPECTRE_ERR_INVALID_ARG, "y may not alias v on the multi-pass path");
+  if (staged || pl.N1 > 1) {
+    // any overlap of the two views' byte extents counts, not only equal base pointers
+    auto extent = [](const spectre_act* a, const char** lo, const char** hi) {
+      const int64_t es = io_elem_bytes(a->dtype);
+      const int64_t last = (a->B - 1) * a->stride_b + (a->L - 1) * a->stride_l + (a->H - 1) * a->stride_h + a->D;
+      *lo = reinterpret_cast<const char*>(a->ptr);
+      *hi = *lo + last * es;
+    };
+    const char *vl, *vh, *yl, *yh;
+    extent(v, &vl, &vh);
+    extent(y, &yl, &yh);
+    if (vl < yh && yl < vh) return fail(SPECTRE_ERR_INVALID_ARG, "y may not overlap v on the multi-pass path");
+  }
   if (wrm) {
     if (wrm->levels < 1 || wrm->levels > 10 || (v->L % (1 << wrm->levels)) != 0)
       return fail(SPECTRE_ERR_INVALID_ARG, "wavelet levels: 2^J must divide L");
