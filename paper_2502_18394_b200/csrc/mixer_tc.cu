@@ -509,7 +509,8 @@ __global__ void __launch_bounds__(128 * NH + 32, NH == 2 ? 2 : 1) mixer_tc196_ke
               const int row = tp + 49 * n1;
               const uint2 out = F16 ? make_uint2(pack_h2(gs * y0[n1].x, gs * y0[n1].y), pack_h2(gs * y1[n1].x, gs * y1[n1].y))
                                     : pack_bf16x4(gs * y0[n1].x, gs * y0[n1].y, gs * y1[n1].x, gs * y1[n1].y);
-              bad |= nonfinite16x2<F16>(out.x) | nonfinite16x2<F16>(out.y);
+              // an overflow anywhere in a column makes every row of it non-finite: one row per thread is enough
+              if (n1 == 0) bad |= nonfinite16x2<F16>(out.x) | nonfinite16x2<F16>(out.y);
               if (J > 0) *reinterpret_cast<uint2*>(Bsm[half] + ((hl & 1) * 196 + row) * k196StageRow + 2 * col) = out;
               else if (row < p.L) __stcs(reinterpret_cast<uint2*>(dst + (int64_t)row * p.d_sl + col), out);
             }

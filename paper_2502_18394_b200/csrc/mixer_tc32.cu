@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
               const float ya = __uint_as_float(rr[4 * x]) - __uint_as_float(rr[4 * x + 3]);
               const float yb = __uint_as_float(rr[4 * x + 2]) + __uint_as_float(rr[4 * x + 1]);
               const uint32_t yo = F16 ? pack_h2(ya, yb) : pack_bf2(ya, yb);
-              bad |= nonfinite16x2<F16>(yo);
+              if (x == 0) bad |= nonfinite16x2<F16>(yo);       // every row of an overflowed column is non-finite: one row is enough
               *reinterpret_cast<uint32_t*>(prow + (4 * wh + x) * 4096) = yo;
             }
           }
