@@ -211,6 +211,16 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
       const int slab_local = item >> 8, a = (item >> 4) & 15, t2b = item & 15;
+      // One gate image with every 8th item (there are 8 items per image): its strided reads are issued
+      // here and consumed after the item's epilogues, so their latency hides under them.
+      const int sk = (int)blockIdx.x + (it >> 3) * (int)gridDim.x;
+      const bool gate_item = (it & 7) == 0 && sk < p.cnt * 32;
+      float2 gvv[8];
+      if (gate_item) {
+        const float2* g = p.g + (size_t)(p.slab0 + (sk >> 5)) * p.K;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) gvv[t] = gate_ext(g, (sk & 31) + 32 * (tid + kXEpiThreads * t), p.n);
+      }
       // sc W_n^{64 k1 (4a + u)} and W_n^{k1 t2} of this thread's two k1 and this item's rows
       float2 wA[4];
 #pragma unroll
@@ -262,37 +272,27 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
-      // ---- one gate image after every 8th item (there are 8 items per image): per (head, k1) the 4096
-      //      gate values the core needs, normalised by a bound on their maximum, fp16, entry
-      //      kM = kl + 64 k2 at 64 k2 + (kl ^ 8 (k2 % 4)).  The strided reads wait under the item
-      //      the producer has already fetched ----
-      if ((it & 7) == 0) {
-        const int sk = (int)blockIdx.x + (it >> 3) * (int)gridDim.x;
-        if (sk < p.cnt * 32) {
-          const int gk1 = sk & 31;
-          const float2* g = p.g + (size_t)(p.slab0 + (sk >> 5)) * p.K;
-          float2 v[8];
+      // ---- the gate image: per (head, k1) the 4096 gate values the core needs, normalised by a bound on
+      //      their maximum, fp16, entry kM = kl + 64 k2 at 64 k2 + (kl ^ 8 (k2 % 4)) ----
+      if (gate_item) {
+        float mx = 0.f;
 #pragma unroll
-          for (int t = 0; t < 8; ++t) v[t] = gate_ext(g, gk1 + 32 * (tid + kXEpiThreads * t), p.n);
-          float mx = 0.f;
+        for (int t = 0; t < 8; ++t) mx = fmaxf(mx, fmaxf(fabsf(gvv[t].x), fabsf(gvv[t].y)));
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (T == 0) red[warp] = mx;
+        asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");
+        mx = 0.f;
+        for (int w8 = 0; w8 < kXEpiWarps; ++w8) mx = fmaxf(mx, red[w8]);
+        mx *= 1.41421356f;
+        const float inv = mx > 0.f ? 1.0f / mx : 0.f;
+        uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * kXGBytes);
 #pragma unroll
-          for (int t = 0; t < 8; ++t) mx = fmaxf(mx, fmaxf(fabsf(v[t].x), fabsf(v[t].y)));
-          for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-          if (T == 0) red[warp] = mx;
-          asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");
-          mx = 0.f;
-          for (int w8 = 0; w8 < kXEpiWarps; ++w8) mx = fmaxf(mx, red[w8]);
-          mx *= 1.41421356f;
-          const float inv = mx > 0.f ? 1.0f / mx : 0.f;
-          uint32_t* img = reinterpret_cast<uint32_t*>(p.gimg + (size_t)sk * kXGBytes);
-#pragma unroll
-          for (int t = 0; t < 8; ++t) {
-            const int idx = tid + kXEpiThreads * t, k2 = idx >> 6, kl = idx & 63;
-            img[64 * k2 + (kl ^ (8 * (k2 & 3)))] = pack_h2(v[t].x * inv, v[t].y * inv);
-          }
-          if (tid == 0) p.gscale[sk] = mx;
-          asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");   // red[] may be rewritten
+        for (int t = 0; t < 8; ++t) {
+          const int idx = tid + kXEpiThreads * t, k2 = idx >> 6, kl = idx & 63;
+          img[64 * k2 + (kl ^ (8 * (k2 & 3)))] = pack_h2(gvv[t].x * inv, gvv[t].y * inv);
         }
+        if (tid == 0) p.gscale[sk] = mx;
+        asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");   // red[] may be rewritten
       }
     }
   }
