@@ -39,14 +39,14 @@ L2_BYTES = 126e6
 # captures summarised under profiles/ (None until a capture exists for that workload).
 # c2: mixer_tc8192_kernel 35.0 MB read + 1.2 MB written inside the launch (its 33.6 MB output was still
 #     dirty in L2 when the launch ended, so this understates the traffic; nothing is re-read)
-# c3: the four kernels of one staged mixer call at full size (intermediates spill from L2)
+# c3: the three kernels of one staged mixer call at full size (intermediates spill from L2)
 # c4: append_spectrum_kernel measured at B = 2 (1015.3 MB), scaled by 4 to B = 8
 # c5: mixer_tc196_kernel at full size: 82.0 MB read + 27.6 MB written by the end of the launch (the rest of
 #     the 77 MB output is still in L2 then)
 # Not measured by this run: each entry names the committed summary it was read from.
 NCU_TRAFFIC = {"c1": None,
                "c2": (36.9e6, "profiles/mixer_tc8192_kernel_c2.md (ncu capture, not this run)"),
-               "c3": (3126e6, "profiles/launches_c3_gate_mixer.md (ncu capture, not this run)"),
+               "c3": (3120e6, "profiles/launches_c3_gate_mixer.md (ncu capture, not this run)"),
                "c4": (4061e6, "profiles/append_spectrum_kernel_c4_batch2.md (ncu capture at B = 2, x4; not this run)"),
                "c5": (109.6e6, "profiles/launches_c5_and_kernels.md (ncu capture, not this run)")}
 
