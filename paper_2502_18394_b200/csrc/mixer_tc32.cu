@@ -21,7 +21,7 @@
 //                    TMA stores.
 //
 // Both are persistent, one CTA per SM: a producer warp runs TMA loads one work item ahead and issues
-// the MMAs, 8 epilogue warps drain the two accumulators of an item in turn.  Every wait is bounded
+// the MMAs, 16 epilogue warps drain the two accumulators of an item in turn.  Every wait is bounded
 // and reports through the status word.
 #include <cuda.h>
 
