@@ -88,6 +88,24 @@ def test_mixer_131072_radix32_on_tensor_cores(ctx, dt, L, H):
     assert bool((ybig[:, L:] == 7.0).all())
 
 
+def test_mixer_131072_radix32_in_head_groups_and_batches(ctx):
+    # a workspace that holds one head only: the heads run group by group (slab offsets of every kernel),
+    # with two batch entries and a head slice of a wider buffer as input and output views
+    w = W.Workload("t", B=2, L=131072, H=2, D=64, dtype="bf16", seed=77)
+    big = W.activations(W.scaled(w, H=3)).cuda()
+    x = big[:, :, 1:3, :]
+    g = W.random_gate(w).cuda()
+    per_head = S.spectre_mixer_workspace_bytes(ctx, 1, w.L, 1, 64, w.L, S.SPECTRE_BF16)
+    ws = torch.empty(per_head + 64, dtype=torch.uint8, device="cuda")
+    ybig = torch.zeros_like(big)
+    S.spectre_mixer_forward(ctx, x, g, y=ybig[:, :, 0:2, :], workspace=ws)
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ref = O.mixer(W.to_f64(x), gate_to_complex(g))
+    assert_close(W.to_f64(ybig[:, :, 0:2, :]), ref, "bf16")
+    assert float(ybig[:, :, 2].abs().max()) == 0.0
+
+
 def test_mixer_bf16_tensor_core_zero_pad_and_strides(ctx):
     w = W.Workload("t", B=2, L=6000, H=2, D=64, dtype="bf16", n_fft=8192, seed=61)
     assert run_mixer(ctx, w, n_fft=8192) < TOL["bf16"]
