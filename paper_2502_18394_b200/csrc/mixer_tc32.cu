@@ -3,7 +3,7 @@
 // kernels of mixer_tc4k.cu around the same core:
 //
 //   tc_in32_kernel   rows n1 * 4096 + t' of [B, L, H, D] are whole 128-byte lines.  A TMA box
-//                    (64 columns, 1 t', 32 n1; 128-byte swizzle) lands them as an MN-major B operand
+//                    (64 columns, 32 n1, 2 t'; 128-byte swizzle) lands them as two MN-major B operands
 //                    with K = n1 and N = the 64 real columns, straight from HBM, no conversion.  One
 //                    MMA does the real-input 32-point DFT over n1 for 8 values of t' at once:
 //                    A (128 x 64) is block diagonal, two copies of [C; -S], so lanes 0-63 hold (k1,
@@ -20,9 +20,11 @@
 //                    x 32 n1 complete 128-byte output rows, staged (128-byte swizzle) and written by
 //                    TMA stores.
 //
-// Both are persistent, one CTA per SM: a producer warp runs TMA loads one work item ahead and issues
-// the MMAs, 16 epilogue warps drain the two accumulators of an item in turn.  Every wait is bounded
-// and reports through the status word.
+// Both are persistent, one CTA per SM, four roles joined by mbarriers: a load warp keeps up to three
+// half items (32 KB of operands each) in flight through a ring of four slots, an MMA warp starts an
+// accumulator as soon as its slot has landed and the accumulator is drained, 16 epilogue warps drain the
+// two accumulators of an item in turn into two store boxes, a store warp hands each box to TMA stores.
+// Every wait is bounded and reports through the status word.
 #include <cuda.h>
 
 #include <string>
@@ -32,14 +34,15 @@
 namespace spectre {
 
 constexpr int kXBox = 32 * 128;                   // one landed box: 32 rows of 128 bytes
-constexpr int kXItemOp = 16 * kXBox;              // operands of one work item: 2 MMAs x 2 lane groups x 4 blocks
+constexpr int kXItemOp = 16 * kXBox;              // operands of one work item: 2 accumulators x 2 lane groups x 4 blocks
+constexpr int kXHalfOp = 8 * kXBox;               // one accumulator's operands: a slot of the four-deep load ring
 constexpr int kXMat = 128 * 64 * 2;               // one 128 x 64 matrix
 constexpr int kXEpiWarps = 16, kXEpiThreads = 512;  // per TMEM lane quadrant: 2 column halves x 2 sixteen-lane halves
-constexpr int kXInThreads = kXEpiThreads + 32;    // + producer warp
-constexpr int kXOutThreads = kXEpiThreads + 32;
+constexpr int kXInThreads = kXEpiThreads + 96;    // + MMA warp + store warp + load warp
+constexpr int kXOutThreads = kXEpiThreads + 96;
 constexpr int kXInStage = 65536;                  // two store boxes of [tile (8)][k1 (32)][pair (4)][t2 (2)][4 t1], fp16 (re, im)
-constexpr int kXInSmem = 2 * kXMat + 2 * kXItemOp + kXInStage + 160;
-constexpr int kXOutSmem = kXMat + 2 * kXItemOp + 2 * 32768 + 128;
+constexpr int kXInSmem = 2 * kXMat + 2 * kXItemOp + kXInStage + 256;
+constexpr int kXOutSmem = kXMat + 2 * kXItemOp + 2 * 32768 + 192;
 constexpr int kXImgBytes = 65536, kXGBytes = 16384, kXOutBytes = 65536;   // as in mixer_tc4k.cu
 static_assert(kXInSmem <= 232448 && kXOutSmem <= 232448, "shared memory");
 
@@ -93,17 +96,83 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* tm, int c0, int 
 }
 
 // one item's MMAs for accumulator m: npass passes (matrix 0, then matrix 1 on top) x 4 K steps
-__device__ __forceinline__ void issue_item_mmas(uint32_t tmem_d, uint32_t a_base, int npass, uint32_t op_m, uint32_t idesc) {
+// op_m: the accumulator's first box; `grp` bytes between the boxes of the two lane groups, `lbo` bytes between
+// the boxes of the four 64-column blocks
+__device__ __forceinline__ void issue_item_mmas(uint32_t tmem_d, uint32_t a_base, int npass, uint32_t op_m, uint32_t grp, uint32_t lbo,
+                                                uint32_t idesc) {
   for (int pass = 0; pass < npass; ++pass) {
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks) {
       const uint64_t da = umma_desc(a_base + pass * kXMat + ks * 256, 128, 1024);
-      const uint64_t db = umma_desc_mn_sw128(op_m + (ks >> 1) * 4 * kXBox + (ks & 1) * 2048, kXBox, 1024);
+      const uint64_t db = umma_desc_mn_sw128(op_m + (ks >> 1) * grp + (ks & 1) * 2048, lbo, 1024);
       const uint32_t acc = (pass | ks) != 0;
       asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                    :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
     }
   }
+}
+
+// The 16 mbarriers of a CTA.  Operands travel through a ring of four half-item slots (one accumulator's
+// operands each): the load warp fills a slot when its last MMAs are done, the MMA warp starts an
+// accumulator when its slot is full and the epilogue has drained it, the epilogue warps fill a store box
+// when its last TMA store has read it, and the store warp sends it off.  Three half items can be in
+// flight while one is consumed: a single 64 KB item in flight per SM does not cover HBM latency.
+struct XBars {
+  uint32_t base;
+  __device__ explicit XBars(uint32_t b) : base(b) {}
+  __device__ uint32_t slotFull(int s) const { return base + 8u * s; }          // TMA bytes landed (count 1 + tx)
+  __device__ uint32_t slotFree(int s) const { return base + 32u + 8u * s; }    // its MMAs committed
+  __device__ uint32_t accFull(int m) const { return base + 64u + 8u * m; }     // accumulator complete
+  __device__ uint32_t accFree(int m) const { return base + 80u + 8u * m; }     // every epilogue thread has read it
+  __device__ uint32_t boxFull(int m) const { return base + 96u + 8u * m; }     // every epilogue warp has written its part
+  __device__ uint32_t boxFree(int m) const { return base + 112u + 8u * m; }    // the store has read the box
+  __device__ void init() const {
+    for (int s = 0; s < 4; ++s) { mbar_init(slotFull(s), 1); mbar_init(slotFree(s), 1); }
+    for (int m = 0; m < 2; ++m) {
+      mbar_init(accFull(m), 1); mbar_init(accFree(m), kXEpiThreads); mbar_init(boxFull(m), kXEpiWarps); mbar_init(boxFree(m), 1);
+    }
+  }
+};
+
+// MMA warp: half item hseq = 2 it + m takes ring slot hseq % 4 and accumulator m
+template <typename Issue>
+__device__ __forceinline__ bool mma_warp_loop(const XBars& bar, int nitems, int T, bool ok, Issue issue) {
+  int hseq = 0, it = 0;
+  for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
+    for (int m = 0; m < 2 && ok; ++m, ++hseq) {
+      const int slot = hseq & 3;
+      ok = mbar_wait(bar.slotFull(slot), (hseq >> 2) & 1);
+      if (ok && it > 0) ok = mbar_wait(bar.accFree(m), (it - 1) & 1);   // the epilogue has drained this accumulator
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (T == 0) {
+        issue(m, slot);
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar.accFull(m)) : "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar.slotFree(slot)) : "memory");
+      }
+      __syncwarp();
+    }
+  }
+  return ok;
+}
+
+// load warp: fills the ring up to three half items ahead of the MMAs
+template <typename Fetch>
+__device__ __forceinline__ bool load_warp_loop(const XBars& bar, int nitems, int T, bool ok, Fetch fetch) {
+  int hseq = 0;
+  for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
+    for (int m = 0; m < 2 && ok; ++m) {
+      const int slot = hseq & 3;
+      if (hseq >= 4) ok = mbar_wait(bar.slotFree(slot), ((hseq >> 2) - 1) & 1);
+      if (!ok) break;
+      if (T == 0) { mbar_expect_tx(bar.slotFull(slot), kXHalfOp); fetch(item, m, slot); }
+      __syncwarp();
+      ++hseq;
+    }
+  }
+  if (!ok)                                                      // leave no copy into this CTA in flight
+    for (int back = 1; back <= 4 && back <= hseq; ++back) mbar_wait(bar.slotFull((hseq - back) & 3), ((hseq - back) >> 2) & 1);
+  return ok;
 }
 
 // =====================================================================================
@@ -138,14 +207,13 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
   unsigned char* Op = smem + 2 * kXMat;                        // two item slots
   uint32_t* Stg = reinterpret_cast<uint32_t*>(smem + 2 * kXMat + 2 * kXItemOp);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kXMat + 2 * kXItemOp + kXInStage);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  float* red = reinterpret_cast<float*>(bars + 9);             // 16 floats
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  float* red = reinterpret_cast<float*>(bars + 17);            // 16 floats
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
-  const uint32_t barFull[2] = {smem_u32(&bars[0]), smem_u32(&bars[1])}, barFree[2] = {smem_u32(&bars[2]), smem_u32(&bars[3])};
-  const uint32_t accFull[2] = {smem_u32(&bars[4]), smem_u32(&bars[5])}, accFree[2] = {smem_u32(&bars[6]), smem_u32(&bars[7])};
+  const XBars bar(smem_u32(bars));
 
   if (tid == 0) {
-    for (int s = 0; s < 2; ++s) { mbar_init(barFull[s], 1); mbar_init(barFree[s], 1); mbar_init(accFull[s], 1); mbar_init(accFree[s], kXEpiThreads); }
+    bar.init();
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kXEpiWarps) {
@@ -166,51 +234,56 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
   bool ok = (smem_u32(smem) & 1023u) == 0;                      // the swizzled boxes need 1024-byte aligned slots
 
   if (warp == kXEpiWarps) {
-    // ---- producer + MMA issuer ----
+    // ---- MMA warp ----
     const uint32_t idesc = umma_idesc_x(F16 ? 0u : 1u);
-    auto fetch = [&](int item, int slot) {
+    ok = mma_warp_loop(bar, nitems, T, ok, [&](int m, int slot) {
+      issue_item_mmas(tmem + 256 * m, smem_u32(Asm), F16 ? 1 : 2, smem_u32(Op) + slot * kXHalfOp, kXBox, 2 * kXBox, idesc);
+    });
+  } else if (warp == kXEpiWarps + 2) {
+    // ---- load warp: per u one box of rows t' = 64 (4 a + u) + 4 t2b + 2 m + {0, 1} (lane groups), all 32 n1 of each ----
+    ok = load_warp_loop(bar, nitems, T, ok, [&](int item, int m, int slot) {
       const int slab = p.slab0 + (item >> 8), a = (item >> 4) & 15, t2b = item & 15;
       const int b = slab / p.H, h = slab - b * p.H;
-      mbar_expect_tx(barFull[slot], kXItemOp);
-      for (int m = 0; m < 2; ++m)
-        for (int gq = 0; gq < 2; ++gq)
-          for (int u = 0; u < 4; ++u)
-            tma_load_5d(smem_u32(Op) + slot * kXItemOp + ((m * 2 + gq) * 4 + u) * kXBox, &tm_in, 0,
-                        64 * (4 * a + u) + 4 * t2b + 2 * m + gq, 0, h, b, barFull[slot]);
-    };
-    if (T == 0 && (int)blockIdx.x < nitems) fetch(blockIdx.x, 0);
-    __syncwarp();
+      for (int u = 0; u < 4; ++u)
+        tma_load_5d(smem_u32(Op) + slot * kXHalfOp + u * 2 * kXBox, &tm_in, 0, 0, 64 * (4 * a + u) + 4 * t2b + 2 * m, h, b,
+                    bar.slotFull(slot));
+    });
+  } else if (warp == kXEpiWarps + 1) {
+    // ---- store warp: hands each filled box to one TMA store, frees it once the copy has read it ----
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
-      const int slot = it & 1, next = item + gridDim.x;
-      if (next < nitems) {                                      // the other slot: free once the MMAs of item it - 1 are done
-        if (it >= 1) ok = mbar_wait(barFree[slot ^ 1], ((it - 1) >> 1) & 1);
-        if (ok && T == 0) fetch(next, slot ^ 1);
-        __syncwarp();
-      }
-      if (ok) ok = mbar_wait(barFull[slot], (it >> 1) & 1);
+      const int slab_local = item >> 8, a = (item >> 4) & 15, t2b = item & 15;
       for (int m = 0; m < 2 && ok; ++m) {
-        if (it > 0) ok = mbar_wait(accFree[m], (it - 1) & 1);   // the epilogue has drained this accumulator
-        if (!ok) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (T == 0) {
-          issue_item_mmas(tmem + 256 * m, smem_u32(Asm), F16 ? 1 : 2, smem_u32(Op) + slot * kXItemOp + m * 8 * kXBox, idesc);
-          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(accFull[m]) : "memory");
+        ok = mbar_wait(bar.boxFull(m), it & 1);
+        if (ok && T == 0) {
+          // every unit (k1, tile) of the head gets, per pair, two consecutive t2 = 32 bytes of its image
+          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                       :: "l"(&tm_img), "r"(8 * (4 * t2b + 2 * m)), "r"(4 * a), "r"(32 * slab_local), "r"(0),
+                          "r"(smem_u32(Stg) + 32768 * m) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          mbar_arrive(bar.boxFree(m));
         }
         __syncwarp();
       }
-      if (ok && T == 0)
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barFree[slot]) : "memory");
-      __syncwarp();
     }
-    if (!ok) { mbar_wait(barFull[0], 0); mbar_wait(barFull[1], 0); }   // no copy into this CTA left in flight
+    if (T == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   } else {
     // ---- epilogue warps: lane quadrant q = lane group q / 2, k1 = 16 (q % 2) + 8 j + i; column half wh ----
     const int q = warp & 3, wh = (warp >> 2) & 1, j = warp >> 3, i = T >> 2, tq = T & 3, gq = q >> 1;
     const int k1 = 16 * (q & 1) + 8 * j + i;
+    // twiddles of an item's rows, fetched one item ahead: W_n^{64 k1 (4a + u)} and W_n^{k1 t2}
+    float2 nA[4], nB0, nB1;
+    auto fetch_tw = [&](int item) {
+      const int a = (item >> 4) & 15, t2b = item & 15;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) nA[u] = __ldg(p.twr + 128 * k1 + 4 * a + u);
+      nB0 = __ldg(p.twr + 128 * k1 + 64 + 4 * t2b + gq);
+      nB1 = __ldg(p.twr + 128 * k1 + 64 + 4 * t2b + 2 + gq);
+    };
+    if ((int)blockIdx.x < nitems) fetch_tw(blockIdx.x);
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
-      const int slab_local = item >> 8, a = (item >> 4) & 15, t2b = item & 15;
       // One gate image with every 8th item (there are 8 items per image): its strided reads are issued
       // here and consumed after the item's epilogues, so their latency hides under them.
       const int sk = (int)blockIdx.x + (it >> 3) * (int)gridDim.x;
@@ -221,18 +294,18 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
 #pragma unroll
         for (int t = 0; t < 8; ++t) gvv[t] = gate_ext(g, (sk & 31) + 32 * (tid + kXEpiThreads * t), p.n);
       }
-      // sc W_n^{64 k1 (4a + u)} and W_n^{k1 t2} of this thread's two k1 and this item's rows
+      // sc W_n^{64 k1 (4a + u)} and W_n^{k1 t2} of this thread's k1 and this item's rows
       float2 wA[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) { const float2 t = __ldg(p.twr + 128 * k1 + 4 * a + u); wA[u] = make_float2(t.x * p.sc, t.y * p.sc); }
+      for (int u = 0; u < 4; ++u) wA[u] = make_float2(nA[u].x * p.sc, nA[u].y * p.sc);
+      const float2 wB0 = nB0, wB1 = nB1;
+      if (item + (int)gridDim.x < nitems) fetch_tw(item + gridDim.x);
 #pragma unroll 1
       for (int m = 0; m < 2 && ok; ++m) {
-        // the store that last read this box must be done with it
-        if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-        asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");
         unsigned char* box = reinterpret_cast<unsigned char*>(Stg) + 32768 * m;   // [tile (8)][k1 (32)][pair c4 (4)][t2 (2)][4 t1 = 16 bytes]
-        const float2 wB = __ldg(p.twr + 128 * k1 + 64 + 4 * t2b + 2 * m + gq);
-        ok = mbar_wait(accFull[m], it & 1);
+        const float2 wB = m ? wB1 : wB0;
+        if (it > 0) ok = mbar_wait(bar.boxFree(m), (it - 1) & 1);   // the store that last read this box is done with it
+        if (ok) ok = mbar_wait(bar.accFull(m), it & 1);
         if (ok) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t taddr0 = tmem + 256 * m + ((uint32_t)(32 * q + 16 * j) << 16) + 32 * wh;
@@ -261,15 +334,10 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
             }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          mbar_arrive(accFree[m]);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");
-        if (tid == 0 && ok) {
-          // every unit (k1, tile) of the head gets, per pair, two consecutive t2 = 32 bytes of its image
-          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                       :: "l"(&tm_img), "r"(8 * (4 * t2b + 2 * m)), "r"(4 * a), "r"(32 * slab_local), "r"(0), "r"(smem_u32(box)) : "memory");
-          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          mbar_arrive(bar.accFree(m));
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (T == 0) mbar_arrive(bar.boxFull(m));
         }
       }
       // ---- the gate image: per (head, k1) the 4096 gate values the core needs, normalised by a bound on
@@ -296,7 +364,6 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
       }
     }
   }
-  if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   if (!ok && T == 0) report_timeout(p.status);
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -324,13 +391,12 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
   unsigned char* Stg = smem + 2 * kXItemOp;                    // two boxes of [t'l (8)][n1 (32)][128 bytes], swizzled
   unsigned char* Asm = smem + 2 * kXItemOp + 65536;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kXItemOp + 65536 + kXMat);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   const int tid = threadIdx.x, warp = tid >> 5, T = tid & 31;
-  const uint32_t barFull[2] = {smem_u32(&bars[0]), smem_u32(&bars[1])}, barFree[2] = {smem_u32(&bars[2]), smem_u32(&bars[3])};
-  const uint32_t accFull[2] = {smem_u32(&bars[4]), smem_u32(&bars[5])}, accFree[2] = {smem_u32(&bars[6]), smem_u32(&bars[7])};
+  const XBars bar(smem_u32(bars));
 
   if (tid == 0) {
-    for (int s = 0; s < 2; ++s) { mbar_init(barFull[s], 1); mbar_init(barFree[s], 1); mbar_init(accFull[s], 1); mbar_init(accFree[s], kXEpiThreads); }
+    bar.init();
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kXEpiWarps) {
@@ -350,43 +416,42 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
   bool ok = (smem_u32(smem) & 1023u) == 0;                      // the swizzled boxes need 1024-byte aligned slots
 
   if (warp == kXEpiWarps) {
-    // ---- producer + MMA issuer ----
+    // ---- MMA warp ----
     const uint32_t idesc = umma_idesc_x(0u);
-    auto fetch = [&](int item, int slot) {
+    ok = mma_warp_loop(bar, nitems, T, ok, [&](int m, int slot) {
+      issue_item_mmas(tmem + 256 * m, smem_u32(Asm), 1, smem_u32(Op) + slot * kXHalfOp, 4 * kXBox, kXBox, idesc);
+    });
+  } else if (warp == kXEpiWarps + 2) {
+    // ---- load warp: per lane group and tile one box of 8 row slots x 32 k1 ----
+    ok = load_warp_loop(bar, nitems, T, ok, [&](int item, int m, int slot) {
       const int slab_local = item % p.cnt, blk = item / p.cnt;
-      mbar_expect_tx(barFull[slot], kXItemOp);
-      for (int m = 0; m < 2; ++m)
-        for (int gq = 0; gq < 2; ++gq)
-          for (int jb = 0; jb < 4; ++jb)
-            tma_load_4d(smem_u32(Op) + slot * kXItemOp + ((m * 2 + gq) * 4 + jb) * kXBox, &tm_res, 128 * blk + 64 * m,
-                        4 * gq + jb, 0, slab_local, barFull[slot]);
-    };
-    if (T == 0 && (int)blockIdx.x < nitems) fetch(blockIdx.x, 0);
-    __syncwarp();
+      for (int gq = 0; gq < 2; ++gq)
+        for (int jb = 0; jb < 4; ++jb)
+          tma_load_4d(smem_u32(Op) + slot * kXHalfOp + (gq * 4 + jb) * kXBox, &tm_res, 128 * blk + 64 * m, 4 * gq + jb, 0, slab_local,
+                      bar.slotFull(slot));
+    });
+  } else if (warp == kXEpiWarps + 1) {
+    // ---- store warp: two TMA stores per filled box, the box is free once they have read it ----
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
-      const int slot = it & 1, next = item + gridDim.x;
-      if (next < nitems) {
-        if (it >= 1) ok = mbar_wait(barFree[slot ^ 1], ((it - 1) >> 1) & 1);
-        if (ok && T == 0) fetch(next, slot ^ 1);
-        __syncwarp();
-      }
-      if (ok) ok = mbar_wait(barFull[slot], (it >> 1) & 1);
+      const int slab = p.slab0 + item % p.cnt, blk = item / p.cnt;
+      const int b = slab / p.H, h = slab - b * p.H;
+      const int k4 = blk >> 4, row0 = 4 * (blk & 15);
       for (int m = 0; m < 2 && ok; ++m) {
-        if (it > 0) ok = mbar_wait(accFree[m], (it - 1) & 1);
-        if (!ok) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (T == 0) {
-          issue_item_mmas(tmem + 256 * m, smem_u32(Asm), 1, smem_u32(Op) + slot * kXItemOp + m * 8 * kXBox, idesc);
-          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(accFull[m]) : "memory");
+        ok = mbar_wait(bar.boxFull(m), it & 1);
+        if (ok && T == 0) {
+          // box rows t'l = 0..3: t' = 64 (row0 + 2m) + 4 k4 + {0..3}; t'l = 4..7: the next t' / 64
+          const int tp = 64 * (row0 + 2 * m) + 4 * k4;
+          tma_store_5d(&tm_out, 0, 0, tp, h, b, smem_u32(Stg) + 32768 * m);
+          tma_store_5d(&tm_out, 0, 0, tp + 64, h, b, smem_u32(Stg) + 32768 * m + 16384);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          mbar_arrive(bar.boxFree(m));
         }
         __syncwarp();
       }
-      if (ok && T == 0)
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(barFree[slot]) : "memory");
-      __syncwarp();
     }
-    if (!ok) { mbar_wait(barFull[0], 0); mbar_wait(barFull[1], 0); }
+    if (T == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   } else {
     // ---- epilogue warps: lane quadrant q: tiles 4 (q / 2) .. + 3, n1 = 16 (q % 2) + 8 j + i; column half wh ----
     const int q = warp & 3, wh = (warp >> 2) & 1, j = warp >> 3, i = T >> 2, tq = T & 3, gq = q >> 1;
@@ -394,17 +459,12 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
     bool bad = false;                                            // a non-finite result: the fp16 intermediates overflowed
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
-      const int slab = p.slab0 + item % p.cnt, blk = item / p.cnt;
-      const int b = slab / p.H, h = slab - b * p.H;
       // row slots 16 blk .. + 15 of every unit: s1 / 4 = blk / 16, rows t' / 64 = 4 (blk % 16) + {0..3}, s1 % 4 = {0..3}
-      const int k4 = blk >> 4, row0 = 4 * (blk & 15);
 #pragma unroll 1
       for (int m = 0; m < 2 && ok; ++m) {
-        // the stores that last read this box must be done with it
-        if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-        asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");
         unsigned char* box = Stg + 32768 * m;
-        ok = mbar_wait(accFull[m], it & 1);
+        if (it > 0) ok = mbar_wait(bar.boxFree(m), (it - 1) & 1);   // the stores that last read this box are done with it
+        if (ok) ok = mbar_wait(bar.accFull(m), it & 1);
         if (ok) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t taddr0 = tmem + 256 * m + ((uint32_t)(32 * q + 16 * j) << 16) + 32 * wh;
@@ -427,20 +487,13 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
             }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          mbar_arrive(accFree[m]);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("bar.sync 1, %0;" :: "r"(kXEpiThreads) : "memory");
-        if (tid == 0 && ok) {
-          // box rows t'l = 0..3: t' = 64 (row0 + 2m) + 4 k4 + {0..3}; t'l = 4..7: the next t' / 64
-          const int tp = 64 * (row0 + 2 * m) + 4 * k4;
-          tma_store_5d(&tm_out, 0, 0, tp, h, b, smem_u32(box));
-          tma_store_5d(&tm_out, 0, 0, tp + 64, h, b, smem_u32(box) + 16384);
-          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          mbar_arrive(bar.accFree(m));
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (T == 0) mbar_arrive(bar.boxFull(m));
         }
       }
     }
-    if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (__any_sync(0xffffffffu, bad) && T == 0) report_range(p.status);
   }
   if (!ok && T == 0) report_timeout(p.status);
@@ -480,17 +533,13 @@ bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_
          encode_fn32() != nullptr;
 }
 
-// dims (column, A, B, head, batch) over [B, L, H, 64]: row = 4096 n1 + t'; n1_second puts n1 before t'
-static int make_act_map(CUtensorMap* tm, const spectre_act* a, bool n1_second, unsigned box_n1, unsigned box_tp) {
+// dims (column, n1, t', head, batch) over [B, L, H, 64]: row = 4096 n1 + t'
+static int make_act_map(CUtensorMap* tm, const spectre_act* a, unsigned box_n1, unsigned box_tp) {
   const cuuint64_t sl = (cuuint64_t)a->stride_l * 2, sh = (cuuint64_t)a->stride_h * 2, sb = (cuuint64_t)a->stride_b * 2;
   const cuuint64_t nb = (cuuint64_t)(a->L / 4096);
-  cuuint64_t dims[5] = {64, 4096, nb, (cuuint64_t)a->H, (cuuint64_t)a->B};
-  cuuint64_t strides[4] = {sl, 4096 * sl, sh, sb};
-  cuuint32_t box[5] = {64, box_tp, box_n1, 1, 1};
-  if (n1_second) {
-    dims[1] = nb; dims[2] = 4096; strides[0] = 4096 * sl; strides[1] = sl;
-    box[1] = box_n1; box[2] = box_tp;
-  }
+  cuuint64_t dims[5] = {64, nb, 4096, (cuuint64_t)a->H, (cuuint64_t)a->B};
+  cuuint64_t strides[4] = {4096 * sl, sl, sh, sb};
+  cuuint32_t box[5] = {64, box_n1, box_tp, 1, 1};
   cuuint32_t es[5] = {1, 1, 1, 1, 1};
   CUresult r = encode_fn32()(tm, a->dtype == SPECTRE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr,
                              dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -502,7 +551,7 @@ static int make_act_map(CUtensorMap* tm, const spectre_act* a, bool n1_second, u
 int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
                    unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc) {
   CUtensorMap tm;
-  int rc = make_act_map(&tm, v, false, 32, 1);
+  int rc = make_act_map(&tm, v, 32, 2);
   if (rc != SPECTRE_OK) return rc;
   CUtensorMap tm_img;
   {
@@ -541,7 +590,7 @@ int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v
 
 int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int slab0, int cnt) {
   CUtensorMap tm_res, tm_out;
-  int rc = make_act_map(&tm_out, y, true, 32, 4);
+  int rc = make_act_map(&tm_out, y, 32, 4);
   if (rc != SPECTRE_OK) return rc;
   {
     // the units' results as fp16: (one unit, tile, k1, slab of the group)
