@@ -5,7 +5,7 @@
 //                      stream over W2, 1-8 batch entries per pass; with the Toeplitz update off it also applies modReLU and
 //                      the positional phase
 //   gate_post_kernel Toeplitz update, modReLU, phase (only when r > 0)
-#include "common.cuh"
+#include "tc_common.cuh"
 
 #include <atomic>
 #include <string>
@@ -444,6 +444,12 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
   float2 acc[BB];
 #pragma unroll
   for (int bb = 0; bb < BB; ++bb) acc[bb] = make_float2(b2[2 * k], b2[2 * k + 1]);
+  // BB >= 4: the sums of two batch entries share a packed fp32 pair (one instruction per pair and
+  // component; each half rounds like a scalar fmaf, so the results do not change)
+  constexpr int NP = BB >= 4 ? BB / 2 : 1;
+  uint64_t ax[NP], ay[NP];
+#pragma unroll
+  for (int pp = 0; pp < NP; ++pp) { ax[pp] = pk2(acc[0].x, acc[0].x); ay[pp] = pk2(acc[0].y, acc[0].y); }
   auto rows = [&](int j, auto full) {                    // rows j .. j + R - 1 (all present when `full`)
     constexpr bool kFull = decltype(full)::value;
     const int nr = kFull ? R : min(R, p.hidden - j);
@@ -457,21 +463,20 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
       if (kFull || i < nr) {
         const float2 wv = wraw<WT>::cvt(w[i]);
         const float* ur = u + (j + i) * BB;             // entries of absent batch rows hold stale values, never stored
-        float ub[BB];
         if (BB >= 4) {
+          const uint64_t wx = pk2(wv.x, wv.x), wy = pk2(wv.y, wv.y);
 #pragma unroll
           for (int v = 0; v < BB / 4; ++v) {
-            const float4 t = *reinterpret_cast<const float4*>(ur + 4 * v);
-            ub[4 * v] = t.x; ub[4 * v + 1] = t.y; ub[4 * v + 2] = t.z; ub[4 * v + 3] = t.w;
+            const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(ur + 4 * v);   // entries 4v .. 4v + 3
+            ax[2 * v] = fma2(t.x, wx, ax[2 * v]);         ay[2 * v] = fma2(t.x, wy, ay[2 * v]);
+            ax[2 * v + 1] = fma2(t.y, wx, ax[2 * v + 1]); ay[2 * v + 1] = fma2(t.y, wy, ay[2 * v + 1]);
           }
         } else {
 #pragma unroll
-          for (int bb = 0; bb < BB; ++bb) ub[bb] = ur[bb];
-        }
-#pragma unroll
-        for (int bb = 0; bb < BB; ++bb) {
-          acc[bb].x = fmaf(ub[bb], wv.x, acc[bb].x);
-          acc[bb].y = fmaf(ub[bb], wv.y, acc[bb].y);
+          for (int bb = 0; bb < BB; ++bb) {
+            acc[bb].x = fmaf(ur[bb], wv.x, acc[bb].x);
+            acc[bb].y = fmaf(ur[bb], wv.y, acc[bb].y);
+          }
         }
       }
     }
@@ -480,6 +485,13 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
     for (int j = 0; j < p.hidden; j += R) rows(j, std::true_type());
   } else {
     for (int j = 0; j < p.hidden; j += R) rows(j, std::false_type());
+  }
+  if (BB >= 4) {
+#pragma unroll
+    for (int pp = 0; pp < NP; ++pp) {
+      upk2(ax[pp], acc[2 * pp].x, acc[2 * pp + 1].x);
+      upk2(ay[pp], acc[2 * pp].y, acc[2 * pp + 1].y);
+    }
   }
   const float bias = (!p.post && p.modrelu_bias) ? p.modrelu_bias[h * p.hs_mb + k] : 0.f;
   // one positional phase for the whole batch unless per-entry shifts are given

@@ -610,6 +610,31 @@ def test_project_qv(ctx, B, L, H, wdt):
     assert rel_err(gate_to_complex(g1), gate_to_complex(g2)) < 2e-2
 
 
+@pytest.mark.parametrize("L", [8192, 16384])
+def test_value_projection_commutes_with_the_mixer(ctx, L):
+    # Eq. 2-4: the gate is one complex number per (head, bin) and the transforms act along the sequence only,
+    # so the per-head d x d value projection commutes with the whole mixer: irFFT(g . rFFT(X W^(v))) =
+    # irFFT(g . rFFT(X)) W^(v).  The mixer can therefore read X as it lies in memory and W^(v) be applied
+    # to its output (or folded into the output projection's weights): no projected copy of V crosses HBM
+    # before the transform.  Both orders are run through the library and compared with the oracle.
+    w = W.Workload("t", B=1, L=L, H=2, D=64, dtype="bf16", seed=L + 5)
+    x = W.activations(w, structured=True)
+    gen = torch.Generator().manual_seed(L + 1)
+    Wq = (torch.randn(2, 64, 64, generator=gen) / 8).to(torch.bfloat16)
+    Wv = (torch.randn(2, 64, 64, generator=gen) / 8).to(torch.bfloat16)
+    g = W.random_gate(w)
+    _, v, _ = S.spectre_project_qv(ctx, x.cuda(), Wq.cuda(), Wv.cuda())
+    y_a = S.spectre_mixer_forward(ctx, v, g.cuda(), n_fft=L)                 # project, then mix
+    y0 = S.spectre_mixer_forward(ctx, x.cuda(), g.cuda(), n_fft=L)           # mix the raw tokens ...
+    _, y_b, _ = S.spectre_project_qv(ctx, y0, Wq.cuda(), Wv.cuda())          # ... then project
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    _, rv, _ = O.project_qv(W.to_f64(x), W.to_f64(Wq), W.to_f64(Wv))
+    ref = O.mixer(rv, gate_to_complex(g), n_fft=L)
+    assert_close(W.to_f64(y_a), ref, "bf16")
+    assert_close(W.to_f64(y_b), ref, "bf16")
+
+
 # ------------------------------------------------------------------ backward
 @pytest.mark.parametrize("dt,L,n,D", [("f32", 64, 64, 16), ("f32", 196, 196, 24), ("f32", 50, 64, 16), ("bf16", 1024, 1024, 32),
                                       ("f32", 4096, 4096, 16), ("bf16", 8192, 8192, 64), ("f32", 16384, 16384, 16),
