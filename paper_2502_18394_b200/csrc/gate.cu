@@ -388,6 +388,68 @@ __global__ void __launch_bounds__(256) gate_hidden_kernel(const GateMlpParams p)
     }
 }
 
+// ---- the output layer's stream over W2: blocks of rows of one column (bin) per thread ----
+// rows j .. j + N - 1 (all present when FULL) held in wc[o .. o + N - 1], added to the sums of BB batch entries
+template <typename WT, int BB, bool FULL, int N>
+__device__ __forceinline__ void gate_use_rows(const typename wraw<WT>::type (&wc)[wraw<WT>::kRows], int o, int j, int hidden,
+                                              const float* __restrict__ u, float2 (&acc)[BB],
+                                              uint64_t (&ax)[BB >= 4 ? BB / 2 : 1], uint64_t (&ay)[BB >= 4 ? BB / 2 : 1]) {
+  const int nr = FULL ? N : min(N, hidden - j);
+#pragma unroll
+  for (int i = 0; i < N; ++i) {
+    if (FULL || i < nr) {
+      const float2 wv = wraw<WT>::cvt(wc[o + i]);
+      const float* ur = u + (j + i) * BB;                 // entries of absent batch rows hold stale values, never stored
+      if (BB >= 4) {
+        const uint64_t wx = pk2(wv.x, wv.x), wy = pk2(wv.y, wv.y);
+#pragma unroll
+        for (int v = 0; v < BB / 4; ++v) {
+          const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(ur + 4 * v);   // entries 4v .. 4v + 3
+          ax[2 * v] = fma2(t.x, wx, ax[2 * v]);         ay[2 * v] = fma2(t.x, wy, ay[2 * v]);
+          ax[2 * v + 1] = fma2(t.y, wx, ax[2 * v + 1]); ay[2 * v + 1] = fma2(t.y, wy, ay[2 * v + 1]);
+        }
+      } else {
+#pragma unroll
+        for (int bb = 0; bb < BB; ++bb) {
+          acc[bb].x = fmaf(ur[bb], wv.x, acc[bb].x);
+          acc[bb].y = fmaf(ur[bb], wv.y, acc[bb].y);
+        }
+      }
+    }
+  }
+}
+template <typename WT, bool FULL, int N>
+__device__ __forceinline__ void gate_fetch_rows(typename wraw<WT>::type (&wc)[wraw<WT>::kRows], int o, const WT* __restrict__ col,
+                                                size_t ld, int j, int hidden) {
+  const int nr = FULL ? N : min(N, hidden - j);
+#pragma unroll
+  for (int i = 0; i < N; ++i)
+    if (FULL || i < nr) wc[o + i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
+}
+// w holds rows 0 .. R - 1 on entry.  One batch entry per pass: a block of R rows is requested when the
+// one before it has been used.  Several entries per pass (a thread then spends long enough on a row for
+// the latency of a whole block to show): the two halves of w alternate, each refilled with the rows R
+// further on as soon as it has been used, so R / 2 to R rows are in flight throughout.
+template <typename WT, int BB, bool FULL>
+__device__ __forceinline__ void gate_stream(typename wraw<WT>::type (&w)[wraw<WT>::kRows], const WT* __restrict__ col, size_t ld,
+                                            int hidden, const float* __restrict__ u, float2 (&acc)[BB],
+                                            uint64_t (&ax)[BB >= 4 ? BB / 2 : 1], uint64_t (&ay)[BB >= 4 ? BB / 2 : 1]) {
+  constexpr int R = wraw<WT>::kRows, Hf = R / 2;
+  if (BB >= 4) {
+    for (int j = 0; j < hidden; j += R) {
+      gate_use_rows<WT, BB, FULL, Hf>(w, 0, j, hidden, u, acc, ax, ay);
+      if (j + R < hidden) gate_fetch_rows<WT, FULL, Hf>(w, 0, col, ld, j + R, hidden);
+      if (j + Hf < hidden) gate_use_rows<WT, BB, FULL, Hf>(w, Hf, j + Hf, hidden, u, acc, ax, ay);
+      if (j + R + Hf < hidden) gate_fetch_rows<WT, FULL, Hf>(w, Hf, col, ld, j + R + Hf, hidden);
+    }
+  } else {
+    for (int j = 0; j < hidden; j += R) {
+      if (j > 0) gate_fetch_rows<WT, FULL, R>(w, 0, col, ld, j, hidden);
+      gate_use_rows<WT, BB, FULL, R>(w, 0, j, hidden, u, acc, ax, ay);
+    }
+  }
+}
+
 // PRE: the hidden activations were computed once per (head, batch entry) by gate_hidden_kernel
 // (long transforms: hundreds of CTAs per head would otherwise repeat that work).
 template <typename WT, int BB, bool PRE>
@@ -450,42 +512,8 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
   uint64_t ax[NP], ay[NP];
 #pragma unroll
   for (int pp = 0; pp < NP; ++pp) { ax[pp] = pk2(acc[0].x, acc[0].x); ay[pp] = pk2(acc[0].y, acc[0].y); }
-  auto rows = [&](int j, auto full) {                    // rows j .. j + R - 1 (all present when `full`)
-    constexpr bool kFull = decltype(full)::value;
-    const int nr = kFull ? R : min(R, p.hidden - j);
-    if (j > 0) {
-#pragma unroll
-      for (int i = 0; i < R; ++i)
-        if (kFull || i < nr) w[i] = wraw<WT>::load(col + (size_t)(j + i) * ld);
-    }
-#pragma unroll
-    for (int i = 0; i < R; ++i) {
-      if (kFull || i < nr) {
-        const float2 wv = wraw<WT>::cvt(w[i]);
-        const float* ur = u + (j + i) * BB;             // entries of absent batch rows hold stale values, never stored
-        if (BB >= 4) {
-          const uint64_t wx = pk2(wv.x, wv.x), wy = pk2(wv.y, wv.y);
-#pragma unroll
-          for (int v = 0; v < BB / 4; ++v) {
-            const ulonglong2 t = *reinterpret_cast<const ulonglong2*>(ur + 4 * v);   // entries 4v .. 4v + 3
-            ax[2 * v] = fma2(t.x, wx, ax[2 * v]);         ay[2 * v] = fma2(t.x, wy, ay[2 * v]);
-            ax[2 * v + 1] = fma2(t.y, wx, ax[2 * v + 1]); ay[2 * v + 1] = fma2(t.y, wy, ay[2 * v + 1]);
-          }
-        } else {
-#pragma unroll
-          for (int bb = 0; bb < BB; ++bb) {
-            acc[bb].x = fmaf(ur[bb], wv.x, acc[bb].x);
-            acc[bb].y = fmaf(ur[bb], wv.y, acc[bb].y);
-          }
-        }
-      }
-    }
-  };
-  if (p.hidden % R == 0) {
-    for (int j = 0; j < p.hidden; j += R) rows(j, std::true_type());
-  } else {
-    for (int j = 0; j < p.hidden; j += R) rows(j, std::false_type());
-  }
+  if (p.hidden % R == 0) gate_stream<WT, BB, true>(w, col, ld, p.hidden, u, acc, ax, ay);
+  else gate_stream<WT, BB, false>(w, col, ld, p.hidden, u, acc, ax, ay);
   if (BB >= 4) {
 #pragma unroll
     for (int pp = 0; pp < NP; ++pp) {
@@ -503,7 +531,7 @@ __global__ void __launch_bounds__(256, BB == 1 ? 4 : 2) gate_out_kernel(const Ga
       const int b = b0 + bb;
       float2 a = acc[bb];
       if (!p.post) {
-        a = modrelu(a, bias);
+        if (p.modrelu_bias) a = modrelu(a, bias);         // without a bias modReLU is the identity (|z| z / |z| = z, exactly, in this arithmetic too)
         a = cmul(a, p.shift ? phase_factor(k, p.n, p.shift_all + p.shift[b]) : ph);
       }
       p.g_out[((size_t)b * p.H + h) * p.K + k] = a;
