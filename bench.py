@@ -46,7 +46,7 @@ L2_BYTES = 126e6
 # Not measured by this run: each entry names the committed summary it was read from.
 NCU_TRAFFIC = {"c1": None,
                "c2": (36.9e6, "profiles/mixer_tc8192_kernel_c2.md (ncu capture, not this run)"),
-               "c3": (3120e6, "profiles/launches_c3_gate_mixer.md (ncu capture, not this run)"),
+               "c3": (3125e6, "profiles/launches_c3_gate_mixer.md (ncu capture, not this run)"),
                "c4": (4061e6, "profiles/append_spectrum_kernel_c4_batch2.md (ncu capture at B = 2, x4; not this run)"),
                "c5": (109.6e6, "profiles/launches_c5_and_kernels.md (ncu capture, not this run)")}
 

@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
             if (u == 3) {
 #pragma unroll
               for (int x = 0; x < 4; ++x)
-                *reinterpret_cast<uint4*>(box + (((4 * wh + x) * 32 + k1) * 4 + tq) * 32 + 16 * gq) =
+                *reinterpret_cast<uint4*>(box + (((4 * wh + x) * 32 + k1) * 4 + tq) * 32 + 16 * (gq ^ (k1 & 1))) =
                     make_uint4(chunk[x][0], chunk[x][1], chunk[x][2], chunk[x][3]);
             }
           }
@@ -561,7 +561,7 @@ int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v
     cuuint32_t box[4] = {16, 4, 32, 8};
     cuuint32_t es[4] = {1, 1, 1, 1};
     CUresult r = encode_fn32()(&tm_img, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, ws_in, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                               CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
   }
   TcIn32Params p = {};
