@@ -329,9 +329,9 @@ class MixerBench:
 class AppendBench:
     """One Prefix-FFT cache append per step (decode)."""
 
-    def __init__(self, w: W.Workload, dev, nsets=None, decode=False, prefill=False):
+    def __init__(self, w: W.Workload, dev, nsets=None, decode=False, prefill=False, readout=False):
         from paper_2502_18394_b200 import binding as S
-        self.S, self.w, self.dev, self.decode, self.prefill = S, w, dev, decode, prefill
+        self.S, self.w, self.dev, self.decode, self.prefill, self.readout = S, w, dev, decode, prefill, readout
         self.ctx = S.Context(dev.index)
         self.cache = S.PrefixCache(w.B, w.H, w.D, w.N_max, dtype=W.torch_dtype(w.dtype), device=dev)
         # state: a full window of random tokens (prefill through the library)
@@ -353,6 +353,26 @@ class AppendBench:
             groups = -(-(w.B * w.H) // max(1, min(w.B * w.H, ws.numel() // per)))
             self.launches_per_step = 3 * groups + 3                       # (strided, on-chip, split) per group; 2 ring fills; pooling
             self.h2d, self.d2h = 2 * tok, w.B * w.H * w.D * 4
+            self.q_host = self.v_host = None
+            return
+        if readout:
+            # the timed call is the read-out of the whole window from the cached spectrum (Sec. 3.3.2 step (e))
+            del ws, q
+            es = 4 if w.dtype == "f32" else 2
+            N, K = w.N_max, w.N_max // 2 + 1
+            self.ro_g = W.random_gate(W.scaled(w, n_fft=N)).to(dev)
+            self.ro_y = torch.empty((w.B, N, w.H, w.D), dtype=W.torch_dtype(w.dtype), device=dev)
+            self.ro_ws = torch.empty(max(S.spectre_readout_workspace_bytes(self.ctx, w.B, w.H, w.D, N), 16), dtype=torch.uint8, device=dev)
+            self.units_per_step = w.B * N
+            self.alg_bytes = w.B * w.H * K * w.D * 8 + w.B * N * w.H * w.D * es + w.B * w.H * K * 8   # read spectrum, write rows, read g
+            if w.dtype != "f32":
+                self.arith_dtype = "f16 tensor-core operands, f32 accumulate (f32 spectrum in, " + w.dtype + " rows out)"
+            self.kernel_name = ("spectre_prefix_cache_readout (gated operand images from the fp32 spectra, inverse half of the staged "
+                                "tcgen05 path)" if w.dtype != "f32" else "spectre_prefix_cache_readout (fp32 transform kernels)")
+            per = 2 * (N // 4096) * (w.D // 8) * 65536
+            groups = -(-(w.B * w.H) // max(1, min(w.B * w.H, self.ro_ws.numel() // max(per, 1))))
+            self.launches_per_step = 4 * groups                           # (gate maximum, spectrum-in, core, transpose-out) per group
+            self.h2d, self.d2h = w.B * w.H * K * 8, w.B * N * w.H * w.D * es
             self.q_host = self.v_host = None
             return
         del ws, q
@@ -391,6 +411,13 @@ class AppendBench:
         return self.S.prepare_append(self.ctx, self.cache, self.qd[i], self.vd[i], self.t0 + k)
 
     def step(self, k: int, e0=None, e1=None):
+        if self.readout:
+            if e0 is not None:
+                e0.record()
+            self.S.spectre_prefix_cache_readout(self.ctx, self.cache, self.ro_g, y=self.ro_y, workspace=self.ro_ws)
+            if e1 is not None:
+                e1.record()
+            return
         if self.prefill:
             if e0 is not None:
                 e0.record()
@@ -406,6 +433,10 @@ class AppendBench:
             e1.record()
 
     def e2e_prepare(self):
+        if self.readout:
+            self.pin_g = self.ro_g.cpu().pin_memory()
+            self.pin_y = torch.empty_like(self.ro_y, device="cpu").pin_memory()
+            return
         if self.prefill:
             self.pin_q = self.pf_q.cpu().pin_memory()
             self.pin_v = self.pf_v.cpu().pin_memory()
@@ -418,6 +449,11 @@ class AppendBench:
             self.pin_s = torch.empty_like(self.y_rows, device="cpu").pin_memory()
 
     def e2e_step(self, k: int):
+        if self.readout:
+            self.ro_g.copy_(self.pin_g, non_blocking=True)
+            self.S.spectre_prefix_cache_readout(self.ctx, self.cache, self.ro_g, y=self.ro_y, workspace=self.ro_ws)
+            self.pin_y.copy_(self.ro_y, non_blocking=True)
+            return
         if self.prefill:
             self.pf_q.copy_(self.pin_q, non_blocking=True)
             self.pf_v.copy_(self.pin_v, non_blocking=True)
@@ -440,6 +476,13 @@ class AppendBench:
         w = self.w
         rng = np.random.default_rng(0)
         N, K = w.N_max, w.N_max // 2 + 1
+        if getattr(self, "readout", False):
+            # bounded sample: the read-out of one head of one batch entry (N_max rows), scaled to tokens/s
+            st = {"N": N, "prefix_fft": rng.standard_normal((1, 1, K, w.D)) + 1j * rng.standard_normal((1, 1, K, w.D))}
+            gg = rng.standard_normal((1, 1, K)) + 1j * rng.standard_normal((1, 1, K))
+            t0 = time.perf_counter()
+            O.decode_readout(st, gg)
+            return time.perf_counter() - t0, N / w.H
         if getattr(self, "prefill", False):
             # bounded sample: the prefill of one head of one batch entry (N_max tokens), scaled to tokens/s
             qs = rng.standard_normal((1, N, 1, w.D))
@@ -462,8 +505,8 @@ class AppendBench:
         return time.perf_counter() - t0, 1
 
 
-def make_bench(w, dev, nsets, decode=False, backward=False, project=False, shared_gates=False, prefill=False):
-    return AppendBench(w, dev, nsets, decode, prefill) if w.N_max else MixerBench(w, dev, nsets, backward, project, shared_gates)
+def make_bench(w, dev, nsets, decode=False, backward=False, project=False, shared_gates=False, prefill=False, readout=False):
+    return AppendBench(w, dev, nsets, decode, prefill, readout) if w.N_max else MixerBench(w, dev, nsets, backward, project, shared_gates)
 
 
 # --------------------------------------------------------------------------- arms
@@ -473,7 +516,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     torch.set_num_threads(1)
-    bench = _cpu_only_bench(w, getattr(args, "prefill", False))
+    bench = _cpu_only_bench(w, getattr(args, "prefill", False), getattr(args, "readout", False))
     for _ in range(min(args.warmup, 1)):
         bench.cpu_step()
     tot, units = 0.0, 0
@@ -494,13 +537,16 @@ def run_reference(args, w):
     print(json.dumps(out))
 
 
-def _cpu_only_bench(w, prefill=False):
+def _cpu_only_bench(w, prefill=False, readout=False):
     """A bench object whose GPU side is never built (the reference arm runs without the library)."""
     cls = AppendBench if w.N_max else MixerBench
     b = cls.__new__(cls)
     b.w = w
     b.prefill = prefill
-    if w.N_max and prefill:
+    b.readout = readout
+    if w.N_max and readout:
+        b.sample_note = "the read-out of one head of one batch entry (N_max rows), scaled to tokens/s"
+    elif w.N_max and prefill:
         b.sample_note = "the prefill of one head of one batch entry (N_max tokens), scaled to tokens/s"
     elif w.N_max:
         qs, vs = W.decode_tokens(w, 1)
@@ -531,6 +577,7 @@ def main():
     ap.add_argument("--backward", action="store_true", help="mixer workloads: step = gate + forward + backward; the timed call is the backward")
     ap.add_argument("--decode", action="store_true", help="c4: time the whole decode step (gate + fused update/read-out)")
     ap.add_argument("--prefill", action="store_true", help="c4: time the prefill of the whole window (N_max tokens per batch entry)")
+    ap.add_argument("--readout", action="store_true", help="c4: time the read-out of the whole window from the cached spectrum")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
     if args.heads:
@@ -553,14 +600,14 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     base = args.workload
     default_steps = {"c1": 2000, "c2": 2000, "c3": 100, "c4": 200, "c5": 500}[base]
-    K = args.steps if args.steps is not None else (30 if getattr(args, "prefill", False) else default_steps)
+    K = args.steps if args.steps is not None else (30 if (args.prefill or args.readout) else default_steps)
     Wm = max(3, args.warmup if args.warmup is not None else 10)
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     R.init()
-    variant = args.decode or args.backward or args.project or args.shared_gates or args.prefill
-    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project, args.shared_gates, args.prefill)
-    m = measure(bench, K, Wm, local_rank, dev, e2e_steps=3 if args.prefill else max(3, min(K, 30)))
+    variant = args.decode or args.backward or args.project or args.shared_gates or args.prefill or args.readout
+    bench = make_bench(w, dev, args.sets, args.decode, args.backward, args.project, args.shared_gates, args.prefill, args.readout)
+    m = measure(bench, K, Wm, local_rank, dev, e2e_steps=3 if (args.prefill or args.readout) else max(3, min(K, 30)))
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -572,7 +619,7 @@ def main():
             tot += dt
             units += u
             reps += 1
-        note = _cpu_only_bench(w, args.prefill).sample_note + f", {reps} repetition(s)"
+        note = _cpu_only_bench(w, args.prefill, args.readout).sample_note + f", {reps} repetition(s)"
         cpu = {"value": units / tot, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": note,
                "host_cores": os.cpu_count(), "host_cores_usable": len(os.sched_getaffinity(0))}
 
@@ -594,6 +641,7 @@ def main():
         out = {"metric": METRIC}
         label = (" - whole decode step (gate + update + read-out of row N-1)" if args.decode else "") + \
                 (" - prefill of the whole window" if args.prefill else "") + (" + backward" if args.backward else "") + \
+                (" - read-out of the whole window from the cached spectrum" if args.readout else "") + \
                 (" with token projections in front (gate from their sum_q)" if args.project else "") + \
                 (", gate shared across heads" if args.shared_gates else "")
         out.update(result_block(w, m["bench_info"], m, K, Wm, world, cpu, label=label, variant=variant))
@@ -668,6 +716,7 @@ def measure(bench, K, Wm, local_rank, dev, e2e_steps):
     R.barrier()
     e2e_ms, e2e_units = R.aggregate(ev_a.elapsed_time(ev_b), bench.units_per_step * Ke, dev)
     info = {k: getattr(bench, k) for k in ("alg_bytes", "kernel_name", "launches_per_step", "h2d", "d2h", "nsets", "units_per_step")}
+    info["arith_dtype"] = getattr(bench, "arith_dtype", None)
     return {"tot_ms": tot_ms, "tot_units": tot_units, "kern_ms": kern_ms, "clocks": clocks, "windows": len(windows),
             "window_ms": [round(x[0], 4) for x in windows], "kern_events": len([e for e in e0 if e is not None]) * len(windows),
             "e2e_ms": e2e_ms, "e2e_units": e2e_units, "e2e_steps": Ke, "bench_info": info}
@@ -682,7 +731,7 @@ def result_block(w, info, m, K, Wm, world, cpu, label="", variant=False):
     return {
         "value": m["tot_units"] / (m["tot_ms"] * 1e-3), "unit": "tokens/s", "n_gpus": world,
         "steps": K, "warmup": Wm, "ms_per_step": m["tot_ms"] / K, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": arithmetic_dtype(w), "data": "synthetic",
+        "vs_baseline": None, "dtype": info.get("arith_dtype") or arithmetic_dtype(w), "data": "synthetic",
         "timed_windows": {"count": m["windows"], "steps_each": K, "reported": "median window", "ms": m["window_ms"]},
         "config": {"workload": describe(w) + label, "io_dtype": w.dtype, "B": w.B, "L": w.L, "H": w.H, "d_head": w.D,
                    "n_fft": w.n if not w.N_max else w.N_max, "parallelism": f"replicas x{world} (no sharding)",

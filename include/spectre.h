@@ -329,6 +329,11 @@ int spectre_prefix_cache_decode_step(spectre_ctx* ctx, void* stream, const spect
  * N_max must be a supported transform length.  The same rows equal
  * spectre_mixer_forward(V_buf, g) because prefix_fft = R(V_buf); this entry
  * point does half the work and does not need the ring buffer.
+ * bf16 / fp16 rows with N_max = 4096 * 2^r (r <= 5) and D <= 64 take the tensor
+ * cores: the gated spectra become fp16 operand images and the inverse stages of
+ * spectre_mixer_forward's long-sequence path run on them (same amplitude range and
+ * SPECTRE_ERR_RANGE report as there; SPECTRE_FORCE_PATH=alu, fp32 rows, or a workspace
+ * too small for the operand images of one (batch, head) keep the fp32 kernels).
  */
 size_t spectre_readout_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
                                        int32_t N_max);

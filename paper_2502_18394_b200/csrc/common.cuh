@@ -76,6 +76,16 @@ __device__ __forceinline__ float2 twiddle_fwd(unsigned num, unsigned den) {
   return make_float2(c, -s);
 }
 
+// Full-spectrum value of a column pair (a, b) from their half spectra and the gate (read-out from a cached spectrum):
+// Z_k = X^a_k + j X^b_k with X = g * P completed by Hermitian symmetry; at DC and Nyquist only
+// the real parts of the two products survive the real inverse (App. B).
+__device__ __forceinline__ float2 pair_from_half(float2 gk, float4 ab, int k, int kk, int n) {
+  const float2 xa = cmul(gk, make_float2(ab.x, ab.y)), xb = cmul(gk, make_float2(ab.z, ab.w));
+  if (k == 0 || 2 * k == n) return make_float2(xa.x, xb.x);
+  if (kk == k) return make_float2(xa.x - xb.y, xa.y + xb.x);
+  return make_float2(xa.x + xb.y, xb.x - xa.y);
+}
+
 // exp(-j 2 pi m / 8192) from the quarter-wave table (cos, sin)(2 pi r / 8192), r = 0..2048
 __device__ __forceinline__ float2 twiddle8192(const float2* __restrict__ tab, unsigned m) {
   const unsigned q = (m >> 11) & 3u, r = m & 2047u;

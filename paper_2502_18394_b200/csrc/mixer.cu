@@ -38,6 +38,10 @@ size_t tc196_level_gate_bytes(int B, int H);
 bool tc4k_supported(int n, int D);                                                     // mixer_tc4k.cu
 size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
 size_t tc4k_min_workspace(int n, int D);
+bool tc4k_readout_supported(const spectre_ctx* ctx, const spectre_act* y, int n);
+size_t tc4k_readout_workspace_bytes(int n, int D, int nslab);
+int launch_readout_tc4k(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y, int n,
+                        void* ws, size_t ws_bytes);
 int launch_mixer_tc4k(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
                       const spectre_act* y, int n, void* ws, size_t ws_bytes);
 
@@ -189,16 +193,6 @@ __device__ __forceinline__ void run_stage(int R, float4* sm, const float2* tw, i
     case 3: stage<3, INV>(sm, tw, Mloc, S); break;
     default: break;
   }
-}
-
-// Full-spectrum value of a column pair (a, b) from their half spectra and the gate (mode 2):
-// Z_k = X^a_k + j X^b_k with X = g * P completed by Hermitian symmetry; at DC and Nyquist only
-// the real parts of the two products survive the real inverse (App. B).
-__device__ __forceinline__ float2 pair_from_half(float2 gk, float4 ab, int k, int kk, int n) {
-  const float2 xa = cmul(gk, make_float2(ab.x, ab.y)), xb = cmul(gk, make_float2(ab.z, ab.w));
-  if (k == 0 || 2 * k == n) return make_float2(xa.x, xb.x);
-  if (kk == k) return make_float2(xa.x - xb.y, xa.y + xb.x);
-  return make_float2(xa.x + xb.y, xb.x - xa.y);
 }
 
 // Last forward stage (block size = radix, no twiddles) fused with the gate and,
@@ -664,10 +658,16 @@ static int inverse_typed(const spectre_ctx* ctx, cudaStream_t st, const float2* 
   return SPECTRE_OK;
 }
 
+// Enough for either route of inverse_from_spectrum (the output dtype is not known here)
 size_t inverse_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
   TransformPlan pl;
-  if (!make_plan(ctx, n, &pl) || pl.N1 == 1) return 0;
-  return (size_t)preferred_group(ctx, n, D, nslab) * slab_ws_bytes(n, D);
+  if (!make_plan(ctx, n, &pl)) return 0;
+  size_t a = pl.N1 == 1 ? 0 : (size_t)preferred_group(ctx, n, D, nslab) * slab_ws_bytes(n, D);
+  if (ctx->dft64 && tc4k_supported(n, D) && D <= 64 && forced_path() != kPathAlu) {
+    const size_t b = tc4k_readout_workspace_bytes(n, D, nslab);
+    if (b > a) a = b;
+  }
+  return a;
 }
 
 int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y,
@@ -677,6 +677,11 @@ int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* 
   if (pl.N1 > 1) {
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 15)) return fail(SPECTRE_ERR_WORKSPACE, "workspace is NULL or not 16-byte aligned");
   }
+  // 16-bit outputs of a staged length: gated operand images from the spectra, then the inverse half of the
+  // tensor-core path (the fp16 intermediates meet the 16-bit output bound; fp32 outputs stay on the fp32 kernels)
+  if (forced_path() != kPathAlu && tc4k_readout_supported(ctx, y, n) && ws && !(reinterpret_cast<uintptr_t>(ws) & 15) &&
+      ws_bytes >= tc4k_min_workspace(n, y->D))
+    return launch_readout_tc4k(ctx, st, spec, g, y, n, ws, ws_bytes);
   const float2* sp = reinterpret_cast<const float2*>(spec);
   SPECTRE_IO_DISPATCH(y->dtype, return inverse_typed<T>(ctx, st, sp, g, y, pl, ws, ws_bytes));
 }

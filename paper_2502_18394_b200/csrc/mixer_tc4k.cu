@@ -227,6 +227,8 @@ struct TcCoreParams {
   float out_scale;          // 1 / (R * forward scale of the radix-R step)
   int nunits, ntile, R;
   int* status;
+  int first_stage;          // 0: whole units.  2: the images are third-stage operands (gated spectra, see
+                            // tc_spec_in_kernel): only the two inverse stages run, no gate table is read
 };
 
 // Where row t' of a unit's result lies, in 16-byte units (the four pairs of a row stay together): rows
@@ -345,7 +347,7 @@ __global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreP
     // ---- producer + MMA issuer ----
     const uint32_t idesc = umma_idesc_128x256();
     auto fetch = [&](int unit) {
-      const bool new_gate = unit == u0 || unit / p.ntile != (unit - 1) / p.ntile;
+      const bool new_gate = p.first_stage == 0 && (unit == u0 || unit / p.ntile != (unit - 1) / p.ntile);
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(barL), "r"(k4ImgBytes + (new_gate ? k4GBytes : 0)) : "memory");
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                    :: "r"(smem_u32(Bsm)), "l"(p.ws_in + (size_t)unit * k4ImgBytes), "r"(k4ImgBytes), "r"(barL) : "memory");
@@ -356,8 +358,8 @@ __global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreP
     if (T == 0 && u0 < u1) fetch(u0);
     __syncwarp();
     for (int unit = u0, it = 0; unit < u1 && ok; ++unit, ++it) {
-      for (int stage = 0; stage < 4 && ok; ++stage) {
-        if (stage == 0) {
+      for (int stage = p.first_stage; stage < 4 && ok; ++stage) {
+        if (stage == p.first_stage) {
           ok = mbar_wait(barL, it & 1);                         // operand landed
           if (ok && it > 0) ok = mbar_wait(barB, 1);            // previous result has left TMEM
         } else {
@@ -393,7 +395,7 @@ __global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreP
     const int q = warp & 3, wh = warp >> 2;
     for (int unit = u0; unit < u1 && ok; ++unit) {
 #pragma unroll 1
-      for (int stage = 0; stage < 4 && ok; ++stage) {
+      for (int stage = p.first_stage; stage < 4 && ok; ++stage) {
         ok = mbar_wait(barD, stage & 1);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -491,6 +493,82 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
 // =====================================================================================
 // host
 // =====================================================================================
+// =====================================================================================
+// whole-window read-out from cached half spectra (Sec. 3.3.2 step (e)): the inverse half of the path.
+// tc_spec_in_kernel writes, per unit (head, k1, tile), what the core's gate epilogue would have left:
+// the operand of the third stage, conj(s Z_k g_k / m) as fp16 with columns 64 c + kA and K = kB, bin
+// k = k1 + R (kA + 64 kB), Z = the pair's full-spectrum value from the two half spectra (Hermitian
+// completion, real DC / Nyquist products), s = the forward scale the transforms would have applied
+// (in_scale(R) / 64) and m = sqrt(2) max |g| of the head, which the core's last epilogue undoes.
+// =====================================================================================
+struct TcSpecParams {
+  const float2* spec;       // [B*H][K][D] half spectra, fp32
+  const float2* g;          // [B*H][K]
+  unsigned char* ws_in;     // [unit][k4ImgBytes]
+  float* gscale;            // [slab_local * R + k1]
+  int n, K, R, D, ntile, slab0;
+  float sc;
+};
+
+// one CTA per head of the group: m for all its R units
+__global__ void __launch_bounds__(256) tc_gate_amax_kernel(const TcSpecParams p) {
+  __shared__ float red[8];
+  const float2* g = p.g + (size_t)(p.slab0 + blockIdx.x) * p.K;
+  float m = 0.f;
+  for (int k = threadIdx.x; k < p.K; k += 256) {
+    const float2 v = __ldg(g + k);
+    m = fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y)));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = 0.f;
+  for (int i = 0; i < 8; ++i) m = fmaxf(m, red[i]);
+  if ((int)threadIdx.x < p.R) p.gscale[blockIdx.x * p.R + threadIdx.x] = m * 1.41421356f;
+}
+
+// CTA = (head, k1, K group j): the 256 bins kA < 64, kB = 4 j .. 4 j + 3 of the unit row.  A warp reads a
+// bin as one 512-byte row (lane = column pair: two float2), multiplies, and drops its fp16 value into a
+// staging array [pair][kA][kB % 4] (pair stride 260 words: 16-byte aligned rows, 4-way conflicts on the
+// 4-byte stores only); the CTA then writes each tile's 4096 contiguous bytes of K group j.
+constexpr int kSpecPitch = 260;
+__global__ void __launch_bounds__(256, 3) tc_spec_in_kernel(const TcSpecParams p) {
+  extern __shared__ __align__(16) uint32_t spec_stage[];        // [D / 2][kSpecPitch]
+  const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31;
+  const int j = blockIdx.x & 15, sk = blockIdx.x >> 4;
+  const int slab_local = sk / p.R, k1 = sk - slab_local * p.R, slab = p.slab0 + slab_local;
+  const int npair = p.D / 2;
+  const float m = p.gscale[sk];
+  const float s = m > 0.f ? p.sc / m : 0.f;
+  const float2* spec = p.spec + (size_t)slab * p.K * p.D;
+  const float2* g = p.g + (size_t)slab * p.K;
+#pragma unroll 1
+  for (int r0 = 0; r0 < 32; r0 += 8) {
+    float4 ab[8];
+    float2 gk[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {                               // 8 bins in flight per warp
+      const int bin = warp + 8 * (r0 + u), kA = bin & 63, kB = 4 * j + (bin >> 6);
+      const int k = k1 + p.R * (kA + 64 * kB), kk = (2 * k <= p.n) ? k : p.n - k;
+      ab[u] = l < npair ? __ldg(reinterpret_cast<const float4*>(spec + (size_t)kk * p.D + 2 * l)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      gk[u] = __ldg(g + kk);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int bin = warp + 8 * (r0 + u), kA = bin & 63, kB = 4 * j + (bin >> 6);
+      const int k = k1 + p.R * (kA + 64 * kB), kk = (2 * k <= p.n) ? k : p.n - k;
+      const float2 z = pair_from_half(cscale(gk[u], s), ab[u], k, kk, p.n);
+      if (l < npair) spec_stage[l * kSpecPitch + 4 * kA + (bin >> 6)] = pack_h2(z.x, -z.y);   // conjugate: inverse by the conj trick
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < p.ntile * 256; e += 256) {
+    const int tile = e >> 8, pc = e & 255;                      // pc = 64 c + kA
+    const uint4 v = *reinterpret_cast<const uint4*>(spec_stage + (4 * tile + (pc >> 6)) * kSpecPitch + 4 * (pc & 63));
+    *reinterpret_cast<uint4*>(p.ws_in + (size_t)(sk * p.ntile + tile) * k4ImgBytes + j * 4096 + pc * 16) = v;
+  }
+}
+
 static size_t tc4k_slab_bytes(int R, int D) {
   const int ntile = D / 8;
   return (size_t)R * ntile * (k4ImgBytes + k4OutBytes) + (size_t)R * k4GBytes + 256;
@@ -561,7 +639,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
                      reinterpret_cast<const float4*>(ctx->tw64x64),
                      reinterpret_cast<const float2*>(ctx->tw_staged) + (size_t)(R - 1) * 128, gscale,
-                     1.0f / ((float)R * in_scale(R)), (int)nunits, ntile, R, ctx->status_dev};
+                     1.0f / ((float)R * in_scale(R)), (int)nunits, ntile, R, ctx->status_dev, 0};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
   int grid = 2 * ctx->sm_count;                     // two resident CTAs per SM, a contiguous range of units each
   if ((size_t)grid > nunits) grid = (int)nunits;
@@ -610,5 +688,88 @@ int launch_mixer_tc4k(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
 }
 
 size_t tc4k_min_workspace(int n, int D) { return tc4k_slab_bytes(n / 4096, D); }
+
+// ---- whole-window read-out: cached half spectra -> gated operand images -> inverse stages -> rows ----
+bool tc4k_readout_supported(const spectre_ctx* ctx, const spectre_act* y, int n) {
+  return (y->dtype == SPECTRE_BF16 || y->dtype == SPECTRE_F16) && ctx->dft64 != nullptr && ctx->tw_staged != nullptr &&
+         tc4k_supported(n, y->D) && y->D <= 64;
+}
+// preferred workspace: groups of heads worth about 320 MB (the launches are full long before that)
+size_t tc4k_readout_workspace_bytes(int n, int D, int nslab) {
+  const size_t per = tc4k_slab_bytes(n / 4096, D);
+  size_t g = ((size_t)320 << 20) / per;
+  if (g < 1) g = 1;
+  if (g > (size_t)nslab) g = nslab;
+  return g * per;
+}
+
+template <int R, bool F16>
+static int tc4k_readout_group(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y,
+                              int n, int slab0, int cnt, unsigned char* ws) {
+  const int D = y->D, ntile = D / 8;
+  const size_t nunits = (size_t)cnt * R * ntile;
+  unsigned char* ws_in = ws;
+  unsigned char* ws_out = ws_in + nunits * k4ImgBytes;
+  unsigned char* gimg = ws_out + nunits * k4OutBytes;          // unused here: the gate is already in the images
+  float* gscale = reinterpret_cast<float*>(gimg + (size_t)cnt * R * k4GBytes);
+
+  TcSpecParams sp = {reinterpret_cast<const float2*>(spec), reinterpret_cast<const float2*>(g), ws_in, gscale,
+                     n, n / 2 + 1, R, D, ntile, slab0, in_scale(R) / 64.0f};
+  tc_gate_amax_kernel<<<cnt, 256, 0, st>>>(sp);
+  SPECTRE_LAUNCH_OK("tc_gate_amax_kernel");
+  const size_t smem_spec = (size_t)(D / 2) * kSpecPitch * 4;
+  tc_spec_in_kernel<<<cnt * R * 16, 256, smem_spec, st>>>(sp);
+  SPECTRE_LAUNCH_OK("tc_spec_in_kernel");
+
+  TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
+                     reinterpret_cast<const float4*>(ctx->tw64x64),
+                     reinterpret_cast<const float2*>(ctx->tw_staged) + (size_t)(R - 1) * 128, gscale,
+                     1.0f / ((float)R * in_scale(R)), (int)nunits, ntile, R, ctx->status_dev, 2};
+  SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
+  int grid = 2 * ctx->sm_count;
+  if ((size_t)grid > nunits) grid = (int)nunits;
+  tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
+  SPECTRE_LAUNCH_OK("tc_core_kernel");
+
+  if (R == 32 && tc32_supported(ctx, y, y, n)) return launch_tc_out32(ctx, st, ws_out, y, slab0, cnt);
+  constexpr int NT = 512 / R;
+  TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
+                    y->H, D, y->L, n, ntile, slab0, ctx->status_dev};
+  const size_t smem_out = (size_t)R * NT * (D / 2) * 4;
+  if (smem_out > 48 * 1024)
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel<R, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_out));
+  tc_out_kernel<R, F16><<<cnt * (4096 / NT), 256, smem_out, st>>>(op);
+  SPECTRE_LAUNCH_OK("tc_out_kernel");
+  return SPECTRE_OK;
+}
+
+int launch_readout_tc4k(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y, int n,
+                        void* ws, size_t ws_bytes) {
+  const int R = n / 4096, nslab = y->B * y->H;
+  const size_t per = tc4k_slab_bytes(R, y->D);
+  int group = (int)(ws_bytes / per);
+  const int pref = (int)(tc4k_readout_workspace_bytes(n, y->D, nslab) / per);
+  if (group > pref) group = pref;
+  if (group < 1) return fail(SPECTRE_ERR_WORKSPACE, "read-out workspace smaller than one (batch, head) slab");
+  unsigned char* w = reinterpret_cast<unsigned char*>(ws);
+  const bool f16 = y->dtype == SPECTRE_F16;
+  for (int s0 = 0; s0 < nslab; s0 += group) {
+    const int cnt = nslab - s0 < group ? nslab - s0 : group;
+    int rc;
+#define SPECTRE_TC4K_READOUT(RR) (f16 ? tc4k_readout_group<RR, true>(ctx, st, spec, g, y, n, s0, cnt, w) : tc4k_readout_group<RR, false>(ctx, st, spec, g, y, n, s0, cnt, w))
+    switch (R) {
+      case 1: rc = SPECTRE_TC4K_READOUT(1); break;
+      case 2: rc = SPECTRE_TC4K_READOUT(2); break;
+      case 4: rc = SPECTRE_TC4K_READOUT(4); break;
+      case 8: rc = SPECTRE_TC4K_READOUT(8); break;
+      case 16: rc = SPECTRE_TC4K_READOUT(16); break;
+      case 32: rc = SPECTRE_TC4K_READOUT(32); break;
+      default: return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported by the tensor-core path");
+    }
+#undef SPECTRE_TC4K_READOUT
+    if (rc != SPECTRE_OK) return rc;
+  }
+  return SPECTRE_OK;
+}
 
 }  // namespace spectre
