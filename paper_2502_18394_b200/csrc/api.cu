@@ -9,7 +9,7 @@ namespace spectre {
 int build_dft64(__half* F, cudaStream_t st);   // mixer_tc.cu
 int build_tw8192(float2* tab, cudaStream_t st);
 int build_dft49(__half* F, cudaStream_t st);
-int build_tw64x64(float4* tab, cudaStream_t st);
+int build_tw64x64(float2* tab, cudaStream_t st);
 int build_tw_staged(float2* tab, cudaStream_t st);   // mixer_tc4k.cu
 int build_dft32(void* mats, cudaStream_t st);        // mixer_tc32.cu
 
@@ -105,7 +105,7 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft64, 128 * 128 * sizeof(__half));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw8192, 2049 * sizeof(float2));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft49, 128 * 128 * sizeof(__half));
-  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw64x64, 2048 * sizeof(float4));
+  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw64x64, 2048 * sizeof(float2));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw_staged, 63 * 128 * sizeof(float2));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft32, 4 * 16384);
   if (e2 == cudaSuccess) e2 = cudaHostAlloc(reinterpret_cast<void**>(&c->status_host), sizeof(int), cudaHostAllocMapped);
@@ -117,7 +117,7 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
     int rc = build_dft64(reinterpret_cast<__half*>(c->dft64), 0);
     if (rc == SPECTRE_OK) rc = build_tw8192(reinterpret_cast<float2*>(c->tw8192), 0);
     if (rc == SPECTRE_OK) rc = build_dft49(reinterpret_cast<__half*>(c->dft49), 0);
-    if (rc == SPECTRE_OK) rc = build_tw64x64(reinterpret_cast<float4*>(c->tw64x64), 0);
+    if (rc == SPECTRE_OK) rc = build_tw64x64(reinterpret_cast<float2*>(c->tw64x64), 0);
     if (rc == SPECTRE_OK) rc = build_tw_staged(reinterpret_cast<float2*>(c->tw_staged), 0);
     if (rc == SPECTRE_OK) rc = build_dft32(c->dft32, 0);
     if (rc == SPECTRE_OK) e2 = cudaStreamSynchronize(0);

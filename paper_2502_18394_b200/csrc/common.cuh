@@ -20,7 +20,7 @@ struct spectre_ctx {
   void* dft64;            // device: 64-point DFT matrix (fp16, MMA operand layout), 32 KiB
   void* dft49;            // device: 49-point DFT matrix, same format (n = 196 path), 32 KiB
   void* tw8192;           // device: (cos, sin)(2 pi r / 8192), r = 0..2048 (quarter wave), 16 KiB
-  void* tw64x64;          // device: W_4096^{row d} pairs in the epilogue threads' own order (float4), 32 KiB
+  void* tw64x64;          // device: W_4096^{row d}, even columns d, in the epilogue threads' own order (float2), 16 KiB
   void* tw_staged;        // device: twiddles of the four-step split n = 4096 R, R = 1..32 (float2): rows R - 1 + k1 of
                           // 128 entries, W_n^{64 k1 t1} (t1 < 64) then W_n^{k1 t2} (t2 < 64); 63 KiB
   void* dft32;            // device: 32-point DFT matrices of the radix-32 kernels (MMA operand layout), 4 x 16 KiB

@@ -41,20 +41,19 @@ __global__ void build_tw8192_kernel(float2* tab) {
 }
 
 // Twiddles between the two 64-point stages of a 4096-point transform, in the order the epilogue
-// threads use them: entry ((((q 2 + j) 2 + chunk) 4 + x) 32 + lane) holds W_4096^{row d} and
-// W_4096^{row (d + 1)} (real parts first, then imaginary parts) for row = 8 (2q + j) + lane / 4 and d = 32 chunk + 8 x + 2 (lane % 4).
-__global__ void build_tw64x64_kernel(float4* tab) {
+// threads use them: entry ((((q 2 + j) 2 + chunk) 4 + x) 32 + lane) holds W_4096^{row d} for
+// row = 8 (2q + j) + lane / 4 and the even column d = 32 chunk + 8 x + 2 (lane % 4).
+__global__ void build_tw64x64_kernel(float2* tab) {
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= 2048) return;
   int lane = idx & 31, x = (idx >> 5) & 3, chunk = (idx >> 7) & 1, j = (idx >> 8) & 1, q = idx >> 9;
   int row = 8 * (2 * q + j) + (lane >> 2), d = 32 * chunk + 8 * x + 2 * (lane & 3);
-  float s0, c0, s1, c1;
+  float s0, c0;
   sincospif((float)((row * d) & 4095) / 2048.0f, &s0, &c0);
-  sincospif((float)((row * (d + 1)) & 4095) / 2048.0f, &s1, &c1);
-  tab[idx] = make_float4(c0, c1, -s0, -s1);             // (re, re, im, im) of the two: operands of the packed products
+  tab[idx] = make_float2(c0, -s0);
 }
 
-int build_tw64x64(float4* tab, cudaStream_t st) {
+int build_tw64x64(float2* tab, cudaStream_t st) {
   build_tw64x64_kernel<<<8, 256, 0, st>>>(tab);
   SPECTRE_LAUNCH_OK("build_tw64x64_kernel");
   return SPECTRE_OK;

@@ -221,7 +221,7 @@ struct TcCoreParams {
   const unsigned char* gimg;
   unsigned char* ws_out;
   const __half* F;
-  const float4* tw64;       // stage twiddles W_4096^{row d} in epilogue order
+  const float2* tw64;       // stage twiddles W_4096^{row d} (even d) in epilogue order
   const float2* twr;        // [R][128]: W_n^{64 k1 t1}, W_n^{k1 t2} (the rows of this R in the context's table)
   const float* gscale;      // [slab_local * R + k1] gate scale of the unit's (head, k1)
   float out_scale;          // 1 / (R * forward scale of the radix-R step)
@@ -393,6 +393,9 @@ __global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreP
   } else {
     // ---- epilogue warps: quadrant q, the two 64-column quarters of column half wh ----
     const int q = warp & 3, wh = warp >> 2;
+    // W_4096^{row} of this thread's two accumulator rows (8 (2q + j) + T / 4): odd columns' stage twiddles
+    const float2* twh = p.tw64;
+    const float2 wr0 = twiddle_fwd((unsigned)(16 * q + (T >> 2)), 4096u), wr1 = twiddle_fwd((unsigned)(16 * q + 8 + (T >> 2)), 4096u);
     for (int unit = u0; unit < u1 && ok; ++unit) {
 #pragma unroll 1
       for (int stage = p.first_stage; stage < 4 && ok; ++stage) {
@@ -404,12 +407,11 @@ __global__ void __launch_bounds__(k4CoreThreads, 2) tc_core_kernel(const TcCoreP
           core_store(tmem, p.ws_out + (size_t)unit * k4OutBytes, q, wh, T, p.twr + 128 * (gi % p.R),
                      __ldg(p.gscale + gi) * p.out_scale);
         } else {
+          if (stage == 0) epilogue_twiddle2<k4Lbo, k4Sbo, 1>(tmem, Bsm, q, 2 * wh, T, twh, wr0, wr1);
+          else if (stage == 2) epilogue_twiddle2<k4Lbo, k4Sbo, 2>(tmem, Bsm, q, 2 * wh, T, twh, wr0, wr1);
+          else {
 #pragma unroll 1
-          for (int cc = 0; cc < 2; ++cc) {
-            const int cq = 2 * wh + cc;
-            if (stage == 0) epilogue_twiddle<k4Lbo, k4Sbo, 1>(tmem, Bsm, q, cq, T, p.tw64);
-            else if (stage == 1) epilogue_gate_t<k4Lbo, k4Sbo, 64, true>(tmem, Bsm, q, cq, T, Gsm);
-            else epilogue_twiddle<k4Lbo, k4Sbo, 2>(tmem, Bsm, q, cq, T, p.tw64);
+            for (int cc = 0; cc < 2; ++cc) epilogue_gate_t<k4Lbo, k4Sbo, 64, true>(tmem, Bsm, q, 2 * wh + cc, T, Gsm);
           }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -637,7 +639,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   }
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
-                     reinterpret_cast<const float4*>(ctx->tw64x64),
+                     reinterpret_cast<const float2*>(ctx->tw64x64),
                      reinterpret_cast<const float2*>(ctx->tw_staged) + (size_t)(R - 1) * 128, gscale,
                      1.0f / ((float)R * in_scale(R)), (int)nunits, ntile, R, ctx->status_dev, 0};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));
@@ -722,7 +724,7 @@ static int tc4k_readout_group(const spectre_ctx* ctx, cudaStream_t st, const flo
   SPECTRE_LAUNCH_OK("tc_spec_in_kernel");
 
   TcCoreParams cp = {ws_in, gimg, ws_out, reinterpret_cast<const __half*>(ctx->dft64),
-                     reinterpret_cast<const float4*>(ctx->tw64x64),
+                     reinterpret_cast<const float2*>(ctx->tw64x64),
                      reinterpret_cast<const float2*>(ctx->tw_staged) + (size_t)(R - 1) * 128, gscale,
                      1.0f / ((float)R * in_scale(R)), (int)nunits, ntile, R, ctx->status_dev, 2};
   SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_core_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k4CoreSmem));

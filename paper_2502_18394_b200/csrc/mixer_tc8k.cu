@@ -44,7 +44,7 @@ struct Tc8kParams {
   const float2* g;        // [B*H][4097]
   const __half* F;        // 64-point DFT matrix, canonical smem layout
   const float2* tw;       // quarter-wave twiddle table (8192nds)
-  const float4* tw64;     // stage twiddles W_4096^{row d} in epilogue order
+  const float2* tw64;     // stage twiddles W_4096^{row d} (even d) in epilogue order
   int H, ntile;
   int* status;            // host-mapped status word (0 = fine)
 };
@@ -236,6 +236,8 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
     mbar_arrive(smem_u32(&bars[1]));
 
     const int q = warp & 3, cq = warp >> 2;
+    // W_4096^{row} of this thread's two accumulator rows (8 (2q + j) + T / 4): the odd columns' stage twiddles
+    const float2 wr0 = twiddle_fwd((unsigned)(16 * q + (T >> 2)), 4096u), wr1 = twiddle_fwd((unsigned)(16 * q + 8 + (T >> 2)), 4096u);
     // ---- stages 1..3: wait for D, transform, hand the next operand to the issuer ----
 #pragma unroll 1
     for (int stage = 0; stage < 3 && ok; ++stage) {
@@ -246,9 +248,9 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t td = tmem + 256 * half;
         unsigned char* Bh = Bsm[0] + half * k8BBytes;
-        if (stage == 0) epilogue_twiddle<k8Lbo1, k8Sbo1, true>(td, Bh, q, cq, T, p.tw64);
+        if (stage == 0) epilogue_twiddle<k8Lbo1, k8Sbo1, true>(td, Bh, q, cq, T, p.tw64, wr0, wr1);
         else if (stage == 1) epilogue_gate(td, Bh, q, cq, T, Gsm[0] + half * (k8GBytes / 4));
-        else epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bh, q, cq, T, p.tw64);
+        else epilogue_twiddle<k8Lbo3, k8Sbo3, false>(td, Bh, q, cq, T, p.tw64, wr0, wr1);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(smem_u32(&bars[half]));
@@ -378,7 +380,7 @@ int launch_mixer_tc8192(const spectre_ctx* ctx, cudaStream_t st, const spectre_a
   p.g = reinterpret_cast<const float2*>(g);
   p.F = reinterpret_cast<const __half*>(ctx->dft64);
   p.tw = reinterpret_cast<const float2*>(ctx->tw8192);
-  p.tw64 = reinterpret_cast<const float4*>(ctx->tw64x64);
+  p.tw64 = reinterpret_cast<const float2*>(ctx->tw64x64);
   p.H = v->H; p.ntile = v->D / 8;
   p.status = ctx->status_dev;
   const unsigned grid = (unsigned)((size_t)v->B * v->H * p.ntile);

@@ -22,16 +22,19 @@ constexpr int k8GBytes = 64 * k8GStride * 4;     // per half, fp16 (re, im)
 // Epilogue after a stage whose accumulator has columns 64 c + d (d = the digit still to be
 // contracted), for one warp: TMEM lane quadrant q, pair c.  A thread owns rows (new digit)
 // 16 q' + T/4 for the two lane groups q' = 2q, 2q+1 and the columns d = 32 chunk + 8 x + 2 (T%4)
-// + {0, 1}.  It multiplies by W_4096^{row d} (read from a table laid out in this thread order, one
-// 16-byte load per x; the two products of an x run as packed fp32 pairs) and writes the transposed operand (row -> column index, d -> K) as one
-// 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
+// + {0, 1}.  It multiplies by W_4096^{row d}: the even column's factor comes from a table laid out in
+// this thread order (one 8-byte load per x; 16 KiB in all, which stays in the 28 KB of L1 that 228 KB of
+// shared memory leave: a table with both columns' factors does not, and its reads were L2 traffic of
+// the size of the operands), the odd column's is that times W_4096^{row} (wr0, wr1: the thread's two
+// rows).  The two products of an x run as packed fp32 pairs; the transposed operand (row -> column index,
+// d -> K) leaves as one 8-byte store per x.  TMEM loads run one 32-column chunk ahead.
 //   COLS: order of the output columns.  1: 64 c + row.  0: 4 row + c.  2: 16 (row / 4) + 8 (c / 2) +
 //   2 (row % 4) + c % 2, which keeps the four rows a half-warp writes at once in four different
 //   16-byte slots of a core matrix even when LBO and SBO are multiples of 128 (dense images), and
 //   leaves all four pairs of a row in one thread of the epilogue that reads the next accumulator.
 template <int LBO, int SBO, int COLS>
 __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char* Bout, int q, int c, int T,
-                                                 const float4* __restrict__ tw) {
+                                                 const float2* __restrict__ tw, float2 wr0, float2 wr1) {
   const int i = T >> 2, tq = T & 3;
   uint32_t r[2][16];
   const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * c;
@@ -41,7 +44,7 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
   for (int step = 0; step < 4; ++step) {                      // step = 2 j + chunk
     const int j = step >> 1, chunk = step & 1;
     const int row = 8 * (2 * q + j) + i;
-    float4 w[4];
+    float2 w[4];
 #pragma unroll
     for (int x = 0; x < 4; ++x) w[x] = __ldg(tw + (4 * step + x) * 32);
     tmem_ld_wait();
@@ -56,9 +59,49 @@ __device__ __forceinline__ void epilogue_twiddle(uint32_t tmem_d, unsigned char*
     const uint32_t base = colpart + (uint32_t)((8 * chunk + (tq >> 1)) * LBO + 8 * (tq & 1));
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
-      // table entry: (w0.x, w1.x, w0.y, w1.y) for the two columns of the thread
+      const float2 w1 = cmul(w[x], j ? wr1 : wr0);
       *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) =
-          cmul2_pack_h2(pk2u(rr[4 * x], rr[4 * x + 1]), pk2u(rr[4 * x + 2], rr[4 * x + 3]), pk2(w[x].x, w[x].y), pk2(w[x].z, w[x].w));
+          cmul2_pack_h2(pk2u(rr[4 * x], rr[4 * x + 1]), pk2u(rr[4 * x + 2], rr[4 * x + 3]), pk2(w[x].x, w1.x), pk2(w[x].y, w1.y));
+    }
+  }
+}
+
+// The same for the two pairs c0 and c0 + 1 of one warp: the twiddles depend on (row, d) only, so each
+// table entry is fetched once and used for both pairs.  The eight (step, pair) accumulator chunks are
+// walked in the order (step, pair) with the TMEM loads one chunk ahead.
+template <int LBO, int SBO, int COLS>
+__device__ __forceinline__ void epilogue_twiddle2(uint32_t tmem_d, unsigned char* Bout, int q, int c0, int T,
+                                                  const float2* __restrict__ tw, float2 wr0, float2 wr1) {
+  const int i = T >> 2, tq = T & 3;
+  uint32_t r[2][16];
+  const uint32_t taddr0 = tmem_d + ((uint32_t)(32 * q) << 16) + 64 * c0;
+  tmem_ld_16x256b_x4(taddr0, r[0]);
+  tw += q * 512 + T;
+  float2 w[4];
+#pragma unroll
+  for (int s8 = 0; s8 < 8; ++s8) {                            // s8 = 2 step + cc, step = 2 j + chunk
+    const int step = s8 >> 1, cc = s8 & 1, c = c0 + cc;
+    const int j = step >> 1, chunk = step & 1;
+    const int row = 8 * (2 * q + j) + i;
+    if (cc == 0) {
+#pragma unroll
+      for (int x = 0; x < 4; ++x) w[x] = __ldg(tw + (4 * step + x) * 32);
+    }
+    tmem_ld_wait();
+    if (s8 < 7) {
+      const int ns = (s8 + 1) >> 1, ncc = (s8 + 1) & 1;
+      tmem_ld_16x256b_x4(taddr0 + ((uint32_t)(16 * (ns >> 1)) << 16) + 32 * (ns & 1) + 64 * ncc, r[(s8 + 1) & 1]);
+    }
+    const uint32_t (&rr)[16] = r[s8 & 1];
+    const uint32_t colpart = COLS == 1 ? (uint32_t)((8 * c + (row >> 3)) * SBO + (row & 7) * 16)
+                           : COLS == 0 ? (uint32_t)((row >> 1) * SBO + (4 * (row & 1) + c) * 16)
+                                       : (uint32_t)((2 * (row >> 2) + (c >> 1)) * SBO + (2 * (row & 3) + (c & 1)) * 16);
+    const uint32_t base = colpart + (uint32_t)((8 * chunk + (tq >> 1)) * LBO + 8 * (tq & 1));
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const float2 w1 = cmul(w[x], j ? wr1 : wr0);
+      *reinterpret_cast<uint2*>(Bout + base + 2 * x * LBO) =
+          cmul2_pack_h2(pk2u(rr[4 * x], rr[4 * x + 1]), pk2u(rr[4 * x + 2], rr[4 * x + 3]), pk2(w[x].x, w1.x), pk2(w[x].y, w1.y));
     }
   }
 }
