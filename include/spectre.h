@@ -50,8 +50,8 @@ typedef enum { SPECTRE_F32 = 0, SPECTRE_BF16 = 1, SPECTRE_F16 = 2 } spectre_dtyp
 typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch limits */
 
 /* Creates a context for CUDA device `device`.  Besides host memory it owns six small device
- * tables (the 64-point and 49-point DFT matrices of the tensor-core mixers and the twiddles
- * between two 64-point stages, 32 KiB each; a quarter-wave twiddle table, 16 KiB; the twiddles
+ * tables (the 64-point and 49-point DFT matrices of the tensor-core mixers, 32 KiB each; the
+ * twiddles between two 64-point stages and a quarter-wave twiddle table, 16 KiB each; the twiddles
  * of the four-step splits n = 4096 R, 63 KiB; the four 32-point DFT matrices of the radix-32
  * kernels, 64 KiB) and one pinned status word, all released by spectre_destroy.  No other
  * call allocates. */
