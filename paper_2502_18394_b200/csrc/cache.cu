@@ -20,27 +20,41 @@ int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* 
 // ws[slab_local][k1][kM][D/2], bin k = k1 + N1 kM.  The half spectra of the two
 // real columns follow from Hermitian symmetry (App. B):
 //   A_k = (Z_k + conj(Z_{n-k})) / 2,   B_k = (Z_k - conj(Z_{n-k})) / (2j).
+// A thread takes kSplitBins consecutive bins of one column pair, all their loads in flight together.
+constexpr int kSplitBins = 4;
 __global__ void __launch_bounds__(256) split_kernel(const float2* __restrict__ ws, float* __restrict__ prefix, int n,
                                                     int K, int D, int N1, int M, int slab0, int nslab) {
   const int half = D / 2;
-  const size_t total = (size_t)nslab * K * half;
+  const int kblocks = (K + kSplitBins - 1) / kSplitBins;
+  const size_t total = (size_t)nslab * kblocks * half;
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
-  int c = (int)(idx % half);
-  size_t r = idx / half;
-  int k = (int)(r % K);
-  int slab_local = (int)(r / K);
-  int km = (n - k) % n;
-  size_t rk = ((size_t)slab_local * N1 + (k % N1)) * M + k / N1;
-  size_t rm = ((size_t)slab_local * N1 + (km % N1)) * M + km / N1;
-  float2 z = ws[rk * half + c], zm = ws[rm * half + c];
-  float4 out;
-  out.x = 0.5f * (z.x + zm.x);
-  out.y = 0.5f * (z.y - zm.y);
-  out.z = 0.5f * (z.y + zm.y);
-  out.w = -0.5f * (z.x - zm.x);
-  size_t o = (((size_t)(slab0 + slab_local) * K + k) * D + 2 * c) * 2;
-  *reinterpret_cast<float4*>(prefix + o) = out;
+  const int c = (int)(idx % half);
+  const size_t r = idx / half;
+  const int k0 = (int)(r % kblocks) * kSplitBins;
+  const int slab_local = (int)(r / kblocks);
+  float2 z[kSplitBins], zm[kSplitBins];
+#pragma unroll
+  for (int u = 0; u < kSplitBins; ++u) {
+    const int k = min(k0 + u, K - 1), km = (n - k) % n;
+    const size_t rk = ((size_t)slab_local * N1 + (k % N1)) * M + k / N1;
+    const size_t rm = ((size_t)slab_local * N1 + (km % N1)) * M + km / N1;
+    z[u] = ws[rk * half + c];
+    zm[u] = ws[rm * half + c];
+  }
+#pragma unroll
+  for (int u = 0; u < kSplitBins; ++u) {
+    const int k = k0 + u;
+    if (k < K) {
+      float4 out;
+      out.x = 0.5f * (z[u].x + zm[u].x);
+      out.y = 0.5f * (z[u].y - zm[u].y);
+      out.z = 0.5f * (z[u].y + zm[u].y);
+      out.w = -0.5f * (z[u].x - zm[u].x);
+      const size_t o = (((size_t)(slab0 + slab_local) * K + k) * D + 2 * c) * 2;
+      *reinterpret_cast<float4*>(prefix + o) = out;
+    }
+  }
 }
 
 // Ring buffers: rows 0..L-1 <- tokens, rows L..N-1 <- 0 (Alg. 1 PreFill).  A CTA copies kRingRows
@@ -317,7 +331,7 @@ extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, cons
     int N1 = 1, M = N;
     rc = forward_spectrum(ctx, st, v, N, s0, cnt, ws, &N1, &M);
     if (rc != SPECTRE_OK) return rc;
-    size_t total = (size_t)cnt * K * (D / 2);
+    size_t total = (size_t)cnt * ((K + kSplitBins - 1) / kSplitBins) * (D / 2);
     split_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, cache->prefix_fft, N, K, D, N1, M, s0, cnt);
     SPECTRE_LAUNCH_OK("split_kernel");
   }

@@ -284,35 +284,52 @@ __device__ __forceinline__ void cross_stage(const OnchipParams& p, const TileCoo
   float4* remote[C];
 #pragma unroll
   for (int q = 0; q < C; ++q) remote[q] = cluster.map_shared_rank(sm, q);
-  for (int w = threadIdx.x; w < nwork; w += blockDim.x) {
-    int pg = w & 3, m = tc.rank * per + (w >> 2);
-    float2 xa[C], xb[C];
-    float2 w1 = twiddle_fwd((unsigned)m, (unsigned)p.M);
-    float2 wq[C];
-    wq[0] = make_float2(1.f, 0.f);
+  // forward: the global loads of two work items are issued before either is used
+  constexpr int UN = INV ? 1 : 2;
+  for (int w0 = threadIdx.x; w0 < nwork; w0 += UN * blockDim.x) {
+    float4 vin[UN][C];
 #pragma unroll
-    for (int q = 1; q < C; ++q) wq[q] = (q == 1) ? w1 : cmul(wq[q / 2], wq[q - q / 2]);
+    for (int u = 0; u < UN; ++u) {
+      const int w = w0 + u * blockDim.x;
+      if (w < nwork) {
+        const int pg = w & 3, m = tc.rank * per + (w >> 2);
 #pragma unroll
-    for (int q = 0; q < C; ++q) {
-      float4 v = INV ? remote[q][(size_t)m * 4 + pg] : load_elem<T>(p, tc, m + q * p.Mloc, pg);
-      xa[q] = make_float2(v.x, v.y);
-      xb[q] = make_float2(v.z, v.w);
-      if (INV && q > 0) {
-        xa[q] = cmulc(xa[q], wq[q]);
-        xb[q] = cmulc(xb[q], wq[q]);
+        for (int q = 0; q < C; ++q) vin[u][q] = INV ? remote[q][(size_t)m * 4 + pg] : load_elem<T>(p, tc, m + q * p.Mloc, pg);
       }
     }
-    Dft<C, INV>::run(xa);
-    Dft<C, INV>::run(xb);
 #pragma unroll
-    for (int q = 0; q < C; ++q) {
-      if (!INV && q > 0) {
-        xa[q] = cmul(xa[q], wq[q]);
-        xb[q] = cmul(xb[q], wq[q]);
+    for (int u = 0; u < UN; ++u) {
+      const int w = w0 + u * blockDim.x;
+      if (w >= nwork) break;
+      const int pg = w & 3, m = tc.rank * per + (w >> 2);
+      float2 xa[C], xb[C];
+      float2 w1 = twiddle_fwd((unsigned)m, (unsigned)p.M);
+      float2 wq[C];
+      wq[0] = make_float2(1.f, 0.f);
+#pragma unroll
+      for (int q = 1; q < C; ++q) wq[q] = (q == 1) ? w1 : cmul(wq[q / 2], wq[q - q / 2]);
+#pragma unroll
+      for (int q = 0; q < C; ++q) {
+        const float4 v = vin[u][q];
+        xa[q] = make_float2(v.x, v.y);
+        xb[q] = make_float2(v.z, v.w);
+        if (INV && q > 0) {
+          xa[q] = cmulc(xa[q], wq[q]);
+          xb[q] = cmulc(xb[q], wq[q]);
+        }
       }
-      float4 v = make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y);
-      if (INV) store_elem<T>(p, tc, m + q * p.Mloc, pg, v);
-      else remote[q][(size_t)m * 4 + pg] = v;
+      Dft<C, INV>::run(xa);
+      Dft<C, INV>::run(xb);
+#pragma unroll
+      for (int q = 0; q < C; ++q) {
+        if (!INV && q > 0) {
+          xa[q] = cmul(xa[q], wq[q]);
+          xb[q] = cmul(xb[q], wq[q]);
+        }
+        float4 v = make_float4(xa[q].x, xa[q].y, xb[q].x, xb[q].y);
+        if (INV) store_elem<T>(p, tc, m + q * p.Mloc, pg, v);
+        else remote[q][(size_t)m * 4 + pg] = v;
+      }
     }
   }
 }
