@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
                                                                  const __grid_constant__ CUtensorMap tm_img, const TcIn32Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* Asm = smem;                                   // hi, lo (bf16) or the fp16 matrix
-  unsigned char* Op = smem + 2 * kXMat;                        // two item slots
+  unsigned char* Op = smem + 2 * kXMat;                        // ring of four half-item slots
   uint32_t* Stg = reinterpret_cast<uint32_t*>(smem + 2 * kXMat + 2 * kXItemOp);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kXMat + 2 * kXItemOp + kXInStage);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
@@ -387,7 +387,7 @@ template <bool F16>
 __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_constant__ CUtensorMap tm_res,
                                                                   const __grid_constant__ CUtensorMap tm_out, const TcOut32Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
-  unsigned char* Op = smem;                                    // two item slots
+  unsigned char* Op = smem;                                    // ring of four half-item slots
   unsigned char* Stg = smem + 2 * kXItemOp;                    // two boxes of [t'l (8)][n1 (32)][128 bytes], swizzled
   unsigned char* Asm = smem + 2 * kXItemOp + 65536;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kXItemOp + 65536 + kXMat);
