@@ -460,21 +460,38 @@ __global__ void __launch_bounds__(256, 3) tc_out_kernel(const TcOutParams p) {
   bool bad = false;                                             // a non-finite result: the fp16 intermediates overflowed
   const uint32_t* wsl = reinterpret_cast<const uint32_t*>(p.ws_out + (size_t)slab_local * R * p.ntile * k4OutBytes);
   const int ustride = p.ntile * (k4OutBytes / 4);               // words between consecutive k1 (same tile)
-  for (int item = warp; item < nitems; item += 8) {
-    const int tile = item % p.ntile, tl = (item / p.ntile) * 8 + t8;
-    const int tp = tb * NT + tl;
-    const uint32_t* pu = wsl + tile * (k4OutBytes / 4) + unit_row_slot(tp) * 4 + c4;
-    float2 x[R];
+  // the 4-byte loads of UN items (R each) are issued before the first butterfly: short radices alone leave
+  // too few bytes in flight per SM
+  constexpr int UN = R >= 16 ? 1 : (R == 8 ? 2 : 4);
+  for (int item0 = warp; item0 < nitems; item0 += 8 * UN) {
+    uint32_t raw[UN][R];
 #pragma unroll
-    for (int k1 = 0; k1 < R; ++k1) x[k1] = unpack_h2(__ldg(pu + k1 * ustride));   // scaled and twiddled by the core
-    Dft<R, true>::run(x);
-    const int word = (tile * 4 + c4) ^ ((tl & skew_mask) << 2);   // skew: the 8 rows of a warp hit 8 bank groups
-    uint32_t* ps = stage + tl * npair + word;
+    for (int u = 0; u < UN; ++u) {
+      const int item = item0 + 8 * u;
+      if (item < nitems) {
+        const int tile = item % p.ntile, tl = (item / p.ntile) * 8 + t8;
+        const uint32_t* pu = wsl + tile * (k4OutBytes / 4) + unit_row_slot(tb * NT + tl) * 4 + c4;
 #pragma unroll
-    for (int n1 = 0; n1 < R; ++n1) {
-      const uint32_t o = F16 ? pack_h2(x[n1].x, x[n1].y) : pack_bf2(x[n1].x, x[n1].y);
-      if (n1 == 0) bad |= nonfinite16x2<F16>(o);                // every row of an overflowed column is non-finite: one row is enough
-      ps[n1 * NT * npair] = o;
+        for (int k1 = 0; k1 < R; ++k1) raw[u][k1] = __ldg(pu + k1 * ustride);   // scaled and twiddled by the core
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      const int item = item0 + 8 * u;
+      if (item >= nitems) break;
+      const int tile = item % p.ntile, tl = (item / p.ntile) * 8 + t8;
+      float2 x[R];
+#pragma unroll
+      for (int k1 = 0; k1 < R; ++k1) x[k1] = unpack_h2(raw[u][k1]);
+      Dft<R, true>::run(x);
+      const int word = (tile * 4 + c4) ^ ((tl & skew_mask) << 2);   // skew: the 8 rows of a warp hit 8 bank groups
+      uint32_t* ps = stage + tl * npair + word;
+#pragma unroll
+      for (int n1 = 0; n1 < R; ++n1) {
+        const uint32_t o = F16 ? pack_h2(x[n1].x, x[n1].y) : pack_bf2(x[n1].x, x[n1].y);
+        if (n1 == 0) bad |= nonfinite16x2<F16>(o);              // every row of an overflowed column is non-finite: one row is enough
+        ps[n1 * NT * npair] = o;
+      }
     }
   }
   if (__any_sync(0xffffffffu, bad) && lane == 0) report_range(p.status);
