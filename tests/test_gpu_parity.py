@@ -638,6 +638,32 @@ def test_value_projection_commutes_with_the_mixer(ctx, L):
     assert_close(W.to_f64(y_b), ref, "bf16")
 
 
+def test_cache_readout_workspace_sizes(ctx):
+    # 16-bit rows of a staged length: the full query (all heads in one group), a workspace for one
+    # (batch, head) only (one group per head through the tensor-core kernels), and none at all (the
+    # fp32 kernels, which need no workspace at this length) must give the same rows
+    N = 8192
+    w = W.Workload("t", B=2, L=N, H=3, D=32, dtype="bf16", n_fft=N, seed=77, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    cache = S.PrefixCache(w.B, w.H, w.D, N, dtype=torch.bfloat16)
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    st = O.cache_prefill(W.to_f64(q), W.to_f64(v), N)
+    g = W.random_gate(w)
+    ref = O.decode_readout(st, gate_to_complex(g))
+    full = S.spectre_readout_workspace_bytes(ctx, w.B, w.H, w.D, N)
+    one = full // (w.B * w.H)
+    assert one * w.B * w.H == full                                # the query is a whole number of heads
+    outs = []
+    for nbytes in (full, one, 0):
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda") if nbytes else torch.empty(0, dtype=torch.uint8, device="cuda")
+        y = S.spectre_prefix_cache_readout(ctx, cache, g.cuda(), workspace=ws)
+        torch.cuda.synchronize()
+        ctx.poll_status()
+        assert_close(W.to_f64(y), ref, "bf16")
+        outs.append(y)
+    assert torch.equal(outs[0], outs[1])                          # grouping does not change a bit
+
+
 # ------------------------------------------------------------------ backward
 @pytest.mark.parametrize("dt,L,n,D", [("f32", 64, 64, 16), ("f32", 196, 196, 24), ("f32", 50, 64, 16), ("bf16", 1024, 1024, 32),
                                       ("f32", 4096, 4096, 16), ("bf16", 8192, 8192, 64), ("f32", 16384, 16384, 16),
