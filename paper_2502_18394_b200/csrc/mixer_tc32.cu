@@ -1,6 +1,6 @@
-// The radix-32 steps of the four-step split n = 32 * 4096 (Sec. 3.2 steps 2 and 4 at n = 131072) on
-// the tensor cores, for bf16 or fp16 activations with d_head = 64.  They replace the transposing ALU
-// kernels of mixer_tc4k.cu around the same core:
+// The radix-R steps of the four-step split n = R * 4096 for R = 32, 16, 8 (Sec. 3.2 steps 2 and 4 at
+// n = 131072, 65536, 32768) on the tensor cores, for bf16 or fp16 activations with d_head = 64.  They
+// replace the transposing ALU kernels of mixer_tc4k.cu around the same core.  Described for R = 32:
 //
 //   tc_in32_kernel   rows n1 * 4096 + t' of [B, L, H, D] are whole 128-byte lines.  A TMA box
 //                    (64 columns, 32 n1, 2 t'; 128-byte swizzle) lands them as two MN-major B operands
@@ -19,6 +19,11 @@
 //                    lanes 0-63 serve tiles 0-3, lanes 64-127 tiles 4-7, so one MMA yields 8 rows t'
 //                    x 32 n1 complete 128-byte output rows, staged (128-byte swizzle) and written by
 //                    TMA stores.
+//
+// R = 16 and 8 use the same MMA shape: the 32 contracted rows of a lane group are S = 32 / R independent
+// sets of R rows (boxes of R rows, one 1024-byte swizzle atom per 8), the matrices are block diagonal
+// within a group as well (an R-point DFT per set), and a set stands for another t' (tc_in32: S times
+// as many t2 per item, store runs of 32 S bytes) or another block of row slots (tc_out32).
 //
 // Both are persistent, one CTA per SM, four roles joined by mbarriers: a load warp keeps up to three
 // half items (32 KB of operands each) in flight through a ring of four slots, an MMA warp starts an
@@ -46,20 +51,25 @@ constexpr int kXOutSmem = kXMat + 2 * kXItemOp + 2 * 32768 + 192;
 constexpr int kXImgBytes = 65536, kXGBytes = 16384, kXOutBytes = 65536;   // as in mixer_tc4k.cu
 static_assert(kXInSmem <= 232448 && kXOutSmem <= 232448, "shared memory");
 
-// ---- the four matrices ------------------------------------------------------------------------
+// ---- the matrices: four per radix R = 32, 16, 8 (in this order) -----------------------------------
 // Row m of a matrix: lane group m / 64, then 16-lane blocks of 8 indices with part 0 in the lower 8
 // lanes and part 1 in the upper 8 (where a 16x256b TMEM load puts both into one thread); column kk:
-// group kk / 32, contracted index kk % 32; zero unless the groups agree.  K-major canonical layout.
-__global__ void build_dft32_kernel(unsigned char* mats) {
+// group kk / 32, contracted index kk % 32; zero unless the groups agree.  For R < 32 the 32 indices of
+// a group are 32 / R independent sets of R (index = R set + k): an R-point DFT per set, zero across sets.
+// K-major canonical layout.
+__global__ void build_dft32_kernel(unsigned char* mats_all) {
+  const int R = 32 >> blockIdx.y;
+  unsigned char* mats = mats_all + (size_t)blockIdx.y * 4 * kXMat;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= 128 * 64) return;
   const int m = idx >> 6, kk = idx & 63;
   const int g = m >> 6, blk = (m >> 4) & 3, l = m & 15, a = 8 * blk + (l & 7), part = l >> 3;
   const int gk = kk >> 5, c = kk & 31;
+  const bool on = g == gk && a / R == c / R;
   float s, co;
-  sincospif((float)((a * c) & 31) / 16.0f, &s, &co);
-  const float fwd = g == gk ? (part == 0 ? co : -s) : 0.f;      // [C; -S]: X[k1] = sum x (cos - j sin)
-  const float inv = g == gk ? (part == 0 ? co : s) : 0.f;       // [C;  S]: W^{-k n} = cos + j sin
+  sincospif((float)(((a % R) * (c % R)) % R) * 2.0f / (float)R, &s, &co);
+  const float fwd = on ? (part == 0 ? co : -s) : 0.f;           // [C; -S]: X[k1] = sum x (cos - j sin)
+  const float inv = on ? (part == 0 ? co : s) : 0.f;            // [C;  S]: W^{-k n} = cos + j sin
   const size_t off = (size_t)((m >> 3) * 1024 + (kk >> 3) * 128 + (m & 7) * 16 + (kk & 7) * 2);
   const __nv_bfloat16 hi = __float2bfloat16(fwd);
   *reinterpret_cast<__nv_bfloat16*>(mats + off) = hi;
@@ -68,7 +78,7 @@ __global__ void build_dft32_kernel(unsigned char* mats) {
   *reinterpret_cast<__half*>(mats + 3 * kXMat + off) = __float2half(inv);
 }
 int build_dft32(void* mats, cudaStream_t st) {
-  build_dft32_kernel<<<32, 256, 0, st>>>(reinterpret_cast<unsigned char*>(mats));
+  build_dft32_kernel<<<dim3(32, 3), 256, 0, st>>>(reinterpret_cast<unsigned char*>(mats));
   SPECTRE_LAUNCH_OK("build_dft32_kernel");
   return SPECTRE_OK;
 }
@@ -183,14 +193,14 @@ struct TcIn32Params {
   const float2* twr;            // [32][128]: W_n^{64 k1 t1}, W_n^{k1 t2}
   unsigned char* ws_in;         // [unit][kXImgBytes]
   const float2* g;              // [B*H][K]
-  unsigned char* gimg;          // [slab_local * 32 + k1][kXGBytes]
-  float* gscale;                // [slab_local * 32 + k1]
+  unsigned char* gimg;          // [slab_local * R + k1][kXGBytes]
+  float* gscale;                // [slab_local * R + k1]
   int H, slab0, cnt, n, K;
-  float sc;                     // forward scale of the radix-32 step
+  float sc;                     // forward scale of the radix-R step
   int* status;
 };
 
-// bins k = k1 + 32 kM, kM < 4096, of the Hermitian extension of one head's gate
+// bins k = k1 + R kM, kM < 4096, of the Hermitian extension of one head's gate
 __device__ __forceinline__ float2 gate_ext(const float2* __restrict__ g, int k, int n) {
   const int kk = (2 * k <= n) ? k : n - k;
   float2 v = __ldg(g + kk);
@@ -199,9 +209,13 @@ __device__ __forceinline__ float2 gate_ext(const float2* __restrict__ g, int k, 
   return v;
 }
 
-template <bool F16>
+// R = 32, 16 or 8 (n = 4096 R).  The 32 contracted rows of a lane group hold S = 32 / R sets of R rows n1:
+// set s of lane group gq is row t' = 64 (4 a + u) + t2 with t2 = 4 S t2b + 2 S m + 2 s + gq, so an
+// accumulator m covers 2 S consecutive t2 and a store box row (tile, k1, pair) is a run of 32 S bytes.
+template <bool F16, int R>
 __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_constant__ CUtensorMap tm_in,
                                                                  const __grid_constant__ CUtensorMap tm_img, const TcIn32Params p) {
+  constexpr int S = 32 / R, T2B = 16 / S;                      // sets per lane group; t2 blocks (of 4 S) per unit row
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* Asm = smem;                                   // hi, lo (bf16) or the fp16 matrix
   unsigned char* Op = smem + 2 * kXMat;                        // ring of four half-item slots
@@ -230,7 +244,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
   asm volatile("griddepcontrol.wait;" ::: "memory");           // launched as a programmatic dependent
-  const int nitems = p.cnt * 256;                               // (slab, 16 groups of 4 t1, 16 blocks of 4 t2): one head's images are written while L2 holds them
+  const int nitems = p.cnt * 16 * T2B;                          // (slab, 16 groups of 4 t1, blocks of 4 S t2): one head's images are written while L2 holds them
   bool ok = (smem_u32(smem) & 1023u) == 0;                      // the swizzled boxes need 1024-byte aligned slots
 
   if (warp == kXEpiWarps) {
@@ -240,25 +254,34 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
       issue_item_mmas(tmem + 256 * m, smem_u32(Asm), F16 ? 1 : 2, smem_u32(Op) + slot * kXHalfOp, kXBox, 2 * kXBox, idesc);
     });
   } else if (warp == kXEpiWarps + 2) {
-    // ---- load warp: per u one box of rows t' = 64 (4 a + u) + 4 t2b + 2 m + {0, 1} (lane groups), all 32 n1 of each ----
+    // ---- load warp: R = 32: per u one box of the rows of both lane groups (t' and t' + 1), all 32 n1 of each;
+    //      R < 32: per (u, lane group, set) one box of R rows n1 ----
     ok = load_warp_loop(bar, nitems, T, ok, [&](int item, int m, int slot) {
-      const int slab = p.slab0 + (item >> 8), a = (item >> 4) & 15, t2b = item & 15;
+      const int slab = p.slab0 + item / (16 * T2B), a = (item / T2B) & 15, t2b = item % T2B;
       const int b = slab / p.H, h = slab - b * p.H;
-      for (int u = 0; u < 4; ++u)
-        tma_load_5d(smem_u32(Op) + slot * kXHalfOp + u * 2 * kXBox, &tm_in, 0, 0, 64 * (4 * a + u) + 4 * t2b + 2 * m, h, b,
-                    bar.slotFull(slot));
+      for (int u = 0; u < 4; ++u) {
+        const int tp = 64 * (4 * a + u) + 4 * S * t2b + 2 * S * m;
+        if (S == 1) {
+          tma_load_5d(smem_u32(Op) + slot * kXHalfOp + u * 2 * kXBox, &tm_in, 0, 0, tp, h, b, bar.slotFull(slot));
+        } else {
+          for (int gq = 0; gq < 2; ++gq)
+            for (int s = 0; s < S; ++s)
+              tma_load_5d(smem_u32(Op) + slot * kXHalfOp + (u * 2 + gq) * kXBox + s * R * 128, &tm_in, 0, 0, tp + 2 * s + gq, h, b,
+                          bar.slotFull(slot));
+        }
+      }
     });
   } else if (warp == kXEpiWarps + 1) {
     // ---- store warp: hands each filled box to one TMA store, frees it once the copy has read it ----
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
-      const int slab_local = item >> 8, a = (item >> 4) & 15, t2b = item & 15;
+      const int slab_local = item / (16 * T2B), a = (item / T2B) & 15, t2b = item % T2B;
       for (int m = 0; m < 2 && ok; ++m) {
         ok = mbar_wait(bar.boxFull(m), it & 1);
         if (ok && T == 0) {
-          // every unit (k1, tile) of the head gets, per pair, two consecutive t2 = 32 bytes of its image
+          // every unit (k1, tile) of the head gets, per pair, 2 S consecutive t2 = 32 S bytes of its image
           asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                       :: "l"(&tm_img), "r"(8 * (4 * t2b + 2 * m)), "r"(4 * a), "r"(32 * slab_local), "r"(0),
+                       :: "l"(&tm_img), "r"(8 * (4 * S * t2b + 2 * S * m)), "r"(4 * a), "r"(R * slab_local), "r"(0),
                           "r"(smem_u32(Stg) + 32768 * m) : "memory");
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -269,17 +292,17 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
     }
     if (T == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   } else {
-    // ---- epilogue warps: lane quadrant q = lane group q / 2, k1 = 16 (q % 2) + 8 j + i; column half wh ----
+    // ---- epilogue warps: lane quadrant q = lane group q / 2, index 16 (q % 2) + 8 j + i = R set + k1; column half wh ----
     const int q = warp & 3, wh = (warp >> 2) & 1, j = warp >> 3, i = T >> 2, tq = T & 3, gq = q >> 1;
-    const int k1 = 16 * (q & 1) + 8 * j + i;
+    const int set = (16 * (q & 1) + 8 * j + i) / R, k1 = (16 * (q & 1) + 8 * j + i) % R;
     // twiddles of an item's rows, fetched one item ahead: W_n^{64 k1 (4a + u)} and W_n^{k1 t2}
     float2 nA[4], nB0, nB1;
     auto fetch_tw = [&](int item) {
-      const int a = (item >> 4) & 15, t2b = item & 15;
+      const int a = (item / T2B) & 15, t2b = item % T2B;
 #pragma unroll
       for (int u = 0; u < 4; ++u) nA[u] = __ldg(p.twr + 128 * k1 + 4 * a + u);
-      nB0 = __ldg(p.twr + 128 * k1 + 64 + 4 * t2b + gq);
-      nB1 = __ldg(p.twr + 128 * k1 + 64 + 4 * t2b + 2 + gq);
+      nB0 = __ldg(p.twr + 128 * k1 + 64 + 4 * S * t2b + 2 * set + gq);
+      nB1 = __ldg(p.twr + 128 * k1 + 64 + 4 * S * t2b + 2 * S + 2 * set + gq);
     };
     if ((int)blockIdx.x < nitems) fetch_tw(blockIdx.x);
     int it = 0;
@@ -287,12 +310,12 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
       // One gate image with every 8th item (there are 8 items per image): its strided reads are issued
       // here and consumed after the item's epilogues, so their latency hides under them.
       const int sk = (int)blockIdx.x + (it >> 3) * (int)gridDim.x;
-      const bool gate_item = (it & 7) == 0 && sk < p.cnt * 32;
+      const bool gate_item = (it & 7) == 0 && sk < p.cnt * R;
       float2 gvv[8];
       if (gate_item) {
-        const float2* g = p.g + (size_t)(p.slab0 + (sk >> 5)) * p.K;
+        const float2* g = p.g + (size_t)(p.slab0 + sk / R) * p.K;
 #pragma unroll
-        for (int t = 0; t < 8; ++t) gvv[t] = gate_ext(g, (sk & 31) + 32 * (tid + kXEpiThreads * t), p.n);
+        for (int t = 0; t < 8; ++t) gvv[t] = gate_ext(g, sk % R + R * (tid + kXEpiThreads * t), p.n);
       }
       // sc W_n^{64 k1 (4a + u)} and W_n^{k1 t2} of this thread's k1 and this item's rows
       float2 wA[4];
@@ -302,7 +325,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
       if (item + (int)gridDim.x < nitems) fetch_tw(item + gridDim.x);
 #pragma unroll 1
       for (int m = 0; m < 2 && ok; ++m) {
-        unsigned char* box = reinterpret_cast<unsigned char*>(Stg) + 32768 * m;   // [tile (8)][k1 (32)][pair c4 (4)][t2 (2)][4 t1 = 16 bytes]
+        unsigned char* box = reinterpret_cast<unsigned char*>(Stg) + 32768 * m;   // [tile (8)][k1 (R)][pair c4 (4)][t2 (2 S)][4 t1 = 16 bytes]
         const float2 wB = m ? wB1 : wB0;
         if (it > 0) ok = mbar_wait(bar.boxFree(m), (it - 1) & 1);   // the store that last read this box is done with it
         if (ok) ok = mbar_wait(bar.accFull(m), it & 1);
@@ -329,7 +352,8 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
             if (u == 3) {
 #pragma unroll
               for (int x = 0; x < 4; ++x)
-                *reinterpret_cast<uint4*>(box + (((4 * wh + x) * 32 + k1) * 4 + tq) * 32 + 16 * (gq ^ (k1 & 1))) =
+                *reinterpret_cast<uint4*>(box + (((4 * wh + x) * R + k1) * 4 + tq) * (32 * S) +
+                                          16 * (S == 1 ? (gq ^ (k1 & 1)) : 2 * set + gq)) =        // R = 32: 32-byte swizzle of the box
                     make_uint4(chunk[x][0], chunk[x][1], chunk[x][2], chunk[x][3]);
             }
           }
@@ -383,12 +407,15 @@ struct TcOut32Params {
   int* status;
 };
 
-template <bool F16>
+// R = 32, 16 or 8.  The 32 contracted rows of a lane group hold S = 32 / R sets of R rows k1: set s takes
+// the row slots of block S blk + s, so an item covers 16 S values of t' and R output rows n1 for each.
+template <bool F16, int R>
 __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_constant__ CUtensorMap tm_res,
                                                                   const __grid_constant__ CUtensorMap tm_out, const TcOut32Params p) {
+  constexpr int S = 32 / R;
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* Op = smem;                                    // ring of four half-item slots
-  unsigned char* Stg = smem + 2 * kXItemOp;                    // two boxes of [t'l (8)][n1 (32)][128 bytes], swizzled
+  unsigned char* Stg = smem + 2 * kXItemOp;                    // two boxes of [set (S)][t'l (8)][n1 (R)][128 bytes], swizzled
   unsigned char* Asm = smem + 2 * kXItemOp + 65536;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kXItemOp + 65536 + kXMat);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
@@ -412,7 +439,7 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
-  const int nitems = p.cnt * 256;                               // (16 consecutive row slots of every unit, slab)
+  const int nitems = p.cnt * (256 / S);                         // (S blocks of 16 consecutive row slots of every unit, slab)
   bool ok = (smem_u32(smem) & 1023u) == 0;                      // the swizzled boxes need 1024-byte aligned slots
 
   if (warp == kXEpiWarps) {
@@ -422,13 +449,14 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
       issue_item_mmas(tmem + 256 * m, smem_u32(Asm), 1, smem_u32(Op) + slot * kXHalfOp, 4 * kXBox, kXBox, idesc);
     });
   } else if (warp == kXEpiWarps + 2) {
-    // ---- load warp: per lane group and tile one box of 8 row slots x 32 k1 ----
+    // ---- load warp: per lane group, tile and set one box of 8 row slots x R k1 ----
     ok = load_warp_loop(bar, nitems, T, ok, [&](int item, int m, int slot) {
       const int slab_local = item % p.cnt, blk = item / p.cnt;
       for (int gq = 0; gq < 2; ++gq)
         for (int jb = 0; jb < 4; ++jb)
-          tma_load_4d(smem_u32(Op) + slot * kXHalfOp + (gq * 4 + jb) * kXBox, &tm_res, 128 * blk + 64 * m, 4 * gq + jb, 0, slab_local,
-                      bar.slotFull(slot));
+          for (int s = 0; s < S; ++s)
+            tma_load_4d(smem_u32(Op) + slot * kXHalfOp + (gq * 4 + jb) * kXBox + s * R * 128, &tm_res, 128 * (S * blk + s) + 64 * m,
+                        4 * gq + jb, 0, slab_local, bar.slotFull(slot));
     });
   } else if (warp == kXEpiWarps + 1) {
     // ---- store warp: two TMA stores per filled box, the box is free once they have read it ----
@@ -436,14 +464,18 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
       const int slab = p.slab0 + item % p.cnt, blk = item / p.cnt;
       const int b = slab / p.H, h = slab - b * p.H;
-      const int k4 = blk >> 4, row0 = 4 * (blk & 15);
       for (int m = 0; m < 2 && ok; ++m) {
         ok = mbar_wait(bar.boxFull(m), it & 1);
         if (ok && T == 0) {
-          // box rows t'l = 0..3: t' = 64 (row0 + 2m) + 4 k4 + {0..3}; t'l = 4..7: the next t' / 64
-          const int tp = 64 * (row0 + 2 * m) + 4 * k4;
-          tma_store_5d(&tm_out, 0, 0, tp, h, b, smem_u32(Stg) + 32768 * m);
-          tma_store_5d(&tm_out, 0, 0, tp + 64, h, b, smem_u32(Stg) + 32768 * m + 16384);
+          for (int s = 0; s < S; ++s) {
+            // row slots 16 bs .. + 15 of every unit: s1 / 4 = bs / 16, rows t' / 64 = 4 (bs % 16) + {0..3}, s1 % 4 = {0..3}
+            const int bs = S * blk + s, k4 = bs >> 4, row0 = 4 * (bs & 15);
+            // box rows t'l = 0..3: t' = 64 (row0 + 2m) + 4 k4 + {0..3}; t'l = 4..7: the next t' / 64
+            const int tp = 64 * (row0 + 2 * m) + 4 * k4;
+            const uint32_t src = smem_u32(Stg) + 32768 * m + s * (8 * R * 128);
+            tma_store_5d(&tm_out, 0, 0, tp, h, b, src);
+            tma_store_5d(&tm_out, 0, 0, tp + 64, h, b, src + 4 * R * 128);
+          }
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
           mbar_arrive(bar.boxFree(m));
@@ -453,13 +485,12 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
     }
     if (T == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   } else {
-    // ---- epilogue warps: lane quadrant q: tiles 4 (q / 2) .. + 3, n1 = 16 (q % 2) + 8 j + i; column half wh ----
+    // ---- epilogue warps: lane quadrant q: tiles 4 (q / 2) .. + 3, index 16 (q % 2) + 8 j + i = R set + n1; column half wh ----
     const int q = warp & 3, wh = (warp >> 2) & 1, j = warp >> 3, i = T >> 2, tq = T & 3, gq = q >> 1;
-    const int n1 = 16 * (q & 1) + 8 * j + i;
+    const int set = (16 * (q & 1) + 8 * j + i) / R, n1 = (16 * (q & 1) + 8 * j + i) % R;
     bool bad = false;                                            // a non-finite result: the fp16 intermediates overflowed
     int it = 0;
     for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++it) {
-      // row slots 16 blk .. + 15 of every unit: s1 / 4 = blk / 16, rows t' / 64 = 4 (blk % 16) + {0..3}, s1 % 4 = {0..3}
 #pragma unroll 1
       for (int m = 0; m < 2 && ok; ++m) {
         unsigned char* box = Stg + 32768 * m;
@@ -475,7 +506,7 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
             tmem_ld_wait();
             if (jb < 3) tmem_ld_16x256b_x4(taddr0 + 64 * (jb + 1), r[(jb + 1) & 1]);
             const uint32_t (&rr)[16] = r[jb & 1];
-            unsigned char* prow = box + n1 * 128 + (((4 * gq + jb) ^ (n1 & 7)) * 16) + 4 * tq;
+            unsigned char* prow = box + (set * 8 * R + n1) * 128 + (((4 * gq + jb) ^ (n1 & 7)) * 16) + 4 * tq;
 #pragma unroll
             for (int x = 0; x < 4; ++x) {                       // row slot t'l = 4 wh + x of the box, pair tq
               // rows (n1, C) and (n1, S) applied to the columns (re, im): y = (C re - S im) + j (S re + C im)
@@ -483,7 +514,7 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
               const float yb = __uint_as_float(rr[4 * x + 2]) + __uint_as_float(rr[4 * x + 1]);
               const uint32_t yo = F16 ? pack_h2(ya, yb) : pack_bf2(ya, yb);
               if (x == 0) bad |= nonfinite16x2<F16>(yo);       // every row of an overflowed column is non-finite: one row is enough
-              *reinterpret_cast<uint32_t*>(prow + (4 * wh + x) * 4096) = yo;
+              *reinterpret_cast<uint32_t*>(prow + (4 * wh + x) * (R * 128)) = yo;
             }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -522,15 +553,15 @@ static EncodeTiledFn32 encode_fn32() {
   return fn;
 }
 
-// Shapes the radix-32 tensor-core kernels take: n = 131072, 64 channels per head (one 128-byte line per
-// row and head), whole 4096-row blocks, 16-byte aligned strides.
+// Shapes the tensor-core transpose kernels take: n = 4096 R with R = 32, 16 or 8, 64 channels per head (one
+// 128-byte line per row and head), whole 4096-row blocks, 16-byte aligned strides.
 bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_act* y, int n) {
   auto ok = [](const spectre_act* a) {
     return (reinterpret_cast<uintptr_t>(a->ptr) & 15) == 0 && a->stride_l % 8 == 0 && a->stride_h % 8 == 0 &&
            a->stride_b % 8 == 0 && a->stride_l > 0 && a->stride_h > 0 && a->stride_b > 0;
   };
-  return n == 131072 && v->D == 64 && v->L % 4096 == 0 && ok(v) && ok(y) && ctx->dft32 != nullptr && ctx->tw_staged != nullptr &&
-         encode_fn32() != nullptr;
+  return (n == 131072 || n == 65536 || n == 32768) && v->D == 64 && v->L % 4096 == 0 && ok(v) && ok(y) && ctx->dft32 != nullptr &&
+         ctx->tw_staged != nullptr && encode_fn32() != nullptr;
 }
 
 // dims (column, n1, t', head, batch) over [B, L, H, 64]: row = 4096 n1 + t'
@@ -548,29 +579,35 @@ static int make_act_map(CUtensorMap* tm, const spectre_act* a, unsigned box_n1, 
   return SPECTRE_OK;
 }
 
-int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
-                   unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc) {
+static int radix_index(int R) { return R == 32 ? 0 : (R == 16 ? 1 : 2); }       // order of the matrix sets in the context
+
+template <int R>
+static int launch_tc_in_r(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
+                          unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc) {
+  constexpr int S = 32 / R;
   CUtensorMap tm;
-  int rc = make_act_map(&tm, v, 32, 2);
+  int rc = make_act_map(&tm, v, R, S == 1 ? 2 : 1);
   if (rc != SPECTRE_OK) return rc;
   CUtensorMap tm_img;
   {
-    // the operand images as fp16: (t2 x 4 t1 of one pair and K group: 1024 bytes; 4 a + c4; slab * 32 + k1; tile)
-    cuuint64_t dims[4] = {512, 64, (cuuint64_t)cnt * 32, 8};
+    // the operand images as fp16: (t2 x 4 t1 of one pair and K group: 1024 bytes; 4 a + c4; slab * R + k1; tile)
+    cuuint64_t dims[4] = {512, 64, (cuuint64_t)cnt * R, 8};
     cuuint64_t strides[3] = {1024, 8 * (cuuint64_t)kXImgBytes, (cuuint64_t)kXImgBytes};
-    cuuint32_t box[4] = {16, 4, 32, 8};
+    cuuint32_t box[4] = {16 * S, 4, R, 8};
     cuuint32_t es[4] = {1, 1, 1, 1};
     CUresult r = encode_fn32()(&tm_img, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, ws_in, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                               CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                               S == 1 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
   }
   TcIn32Params p = {};
-  p.mats = reinterpret_cast<const unsigned char*>(ctx->dft32);
-  p.twr = reinterpret_cast<const float2*>(ctx->tw_staged) + 31 * 128;
+  p.mats = reinterpret_cast<const unsigned char*>(ctx->dft32) + (size_t)radix_index(R) * 4 * kXMat;
+  p.twr = reinterpret_cast<const float2*>(ctx->tw_staged) + (size_t)(R - 1) * 128;
   p.ws_in = ws_in; p.g = reinterpret_cast<const float2*>(g); p.gimg = gimg; p.gscale = gscale;
   p.H = v->H; p.slab0 = slab0; p.cnt = cnt; p.n = n; p.K = n / 2 + 1; p.sc = sc;
   p.status = ctx->status_dev;
-  int grid = cnt * 256 < ctx->sm_count ? cnt * 256 : ctx->sm_count;
+  const int nitems = cnt * (256 / S);
+  int grid = nitems < ctx->sm_count ? nitems : ctx->sm_count;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -578,25 +615,37 @@ int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kXInThreads); cfg.dynamicSmemBytes = kXInSmem; cfg.stream = st;
   cfg.attrs = attr; cfg.numAttrs = 1;
   if (v->dtype == SPECTRE_F16) {
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in32_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXInSmem));
-    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_in32_kernel<true>, tm, tm_img, p));
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in32_kernel<true, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXInSmem));
+    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_in32_kernel<true, R>, tm, tm_img, p));
   } else {
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXInSmem));
-    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_in32_kernel<false>, tm, tm_img, p));
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_in32_kernel<false, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXInSmem));
+    SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_in32_kernel<false, R>, tm, tm_img, p));
   }
   SPECTRE_LAUNCH_OK("tc_in32_kernel");
   return SPECTRE_OK;
 }
 
-int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int slab0, int cnt) {
+int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
+                   unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc) {
+  switch (n / 4096) {
+    case 32: return launch_tc_in_r<32>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
+    case 16: return launch_tc_in_r<16>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
+    case 8: return launch_tc_in_r<8>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
+    default: return fail(SPECTRE_ERR_UNSUPPORTED, "radix not supported by the tensor-core transpose kernels");
+  }
+}
+
+template <int R>
+static int launch_tc_out_r(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int slab0, int cnt) {
+  constexpr int S = 32 / R;
   CUtensorMap tm_res, tm_out;
-  int rc = make_act_map(&tm_out, y, 32, 4);
+  int rc = make_act_map(&tm_out, y, R, 4);
   if (rc != SPECTRE_OK) return rc;
   {
     // the units' results as fp16: (one unit, tile, k1, slab of the group)
-    cuuint64_t dims[4] = {(cuuint64_t)kXOutBytes / 2, 8, 32, (cuuint64_t)cnt};
-    cuuint64_t strides[3] = {(cuuint64_t)kXOutBytes, 8 * (cuuint64_t)kXOutBytes, 256 * (cuuint64_t)kXOutBytes};
-    cuuint32_t box[4] = {64, 1, 32, 1};
+    cuuint64_t dims[4] = {(cuuint64_t)kXOutBytes / 2, 8, R, (cuuint64_t)cnt};
+    cuuint64_t strides[3] = {(cuuint64_t)kXOutBytes, 8 * (cuuint64_t)kXOutBytes, 8 * R * (cuuint64_t)kXOutBytes};
+    cuuint32_t box[4] = {64, 1, R, 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
     CUresult r = encode_fn32()(&tm_res, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<unsigned char*>(ws_out), dims, strides, box, es,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -604,18 +653,28 @@ int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char
     if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
   }
   TcOut32Params p = {};
-  p.mats = reinterpret_cast<const unsigned char*>(ctx->dft32);
+  p.mats = reinterpret_cast<const unsigned char*>(ctx->dft32) + (size_t)radix_index(R) * 4 * kXMat;
   p.H = y->H; p.slab0 = slab0; p.cnt = cnt; p.status = ctx->status_dev;
-  int grid = cnt * 256 < ctx->sm_count ? cnt * 256 : ctx->sm_count;
+  const int nitems = cnt * (256 / S);
+  int grid = nitems < ctx->sm_count ? nitems : ctx->sm_count;
   if (y->dtype == SPECTRE_F16) {
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out32_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXOutSmem));
-    tc_out32_kernel<true><<<grid, kXOutThreads, kXOutSmem, st>>>(tm_res, tm_out, p);
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out32_kernel<true, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXOutSmem));
+    tc_out32_kernel<true, R><<<grid, kXOutThreads, kXOutSmem, st>>>(tm_res, tm_out, p);
   } else {
-    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXOutSmem));
-    tc_out32_kernel<false><<<grid, kXOutThreads, kXOutSmem, st>>>(tm_res, tm_out, p);
+    SPECTRE_CUDA_OK(cudaFuncSetAttribute(tc_out32_kernel<false, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, kXOutSmem));
+    tc_out32_kernel<false, R><<<grid, kXOutThreads, kXOutSmem, st>>>(tm_res, tm_out, p);
   }
   SPECTRE_LAUNCH_OK("tc_out32_kernel");
   return SPECTRE_OK;
+}
+
+int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int n, int slab0, int cnt) {
+  switch (n / 4096) {
+    case 32: return launch_tc_out_r<32>(ctx, st, ws_out, y, slab0, cnt);
+    case 16: return launch_tc_out_r<16>(ctx, st, ws_out, y, slab0, cnt);
+    case 8: return launch_tc_out_r<8>(ctx, st, ws_out, y, slab0, cnt);
+    default: return fail(SPECTRE_ERR_UNSUPPORTED, "radix not supported by the tensor-core transpose kernels");
+  }
 }
 
 }  // namespace spectre

@@ -615,7 +615,7 @@ size_t tc4k_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab) {
 bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_act* y, int n);
 int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
                    unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc);
-int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int slab0, int cnt);
+int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char* ws_out, const spectre_act* y, int n, int slab0, int cnt);
 
 template <int R, bool F16>
 static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g,
@@ -627,7 +627,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   unsigned char* gimg = ws_out + nunits * k4OutBytes;
   float* gscale = reinterpret_cast<float*>(gimg + (size_t)cnt * R * k4GBytes);
 
-  const bool tc32 = R == 32 && tc32_supported(ctx, v, y, n);      // radix-32 steps on the tensor cores
+  const bool tc32 = R >= 8 && tc32_supported(ctx, v, y, n);       // radix-32 / 16 / 8 steps on the tensor cores
   TcGateParams gp = {reinterpret_cast<const float2*>(g), gimg, gscale, n, n / 2 + 1, R, slab0};
 
   if (tc32) {
@@ -665,7 +665,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
   SPECTRE_LAUNCH_OK("tc_core_kernel");
 
-  if (tc32) return launch_tc_out32(ctx, st, ws_out, y, slab0, cnt);
+  if (tc32) return launch_tc_out32(ctx, st, ws_out, y, n, slab0, cnt);
   constexpr int NT = 512 / R;
   TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
                     y->H, D, y->L, n, ntile, slab0, ctx->status_dev};
@@ -750,7 +750,7 @@ static int tc4k_readout_group(const spectre_ctx* ctx, cudaStream_t st, const flo
   tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
   SPECTRE_LAUNCH_OK("tc_core_kernel");
 
-  if (R == 32 && tc32_supported(ctx, y, y, n)) return launch_tc_out32(ctx, st, ws_out, y, slab0, cnt);
+  if (R >= 8 && tc32_supported(ctx, y, y, n)) return launch_tc_out32(ctx, st, ws_out, y, n, slab0, cnt);
   constexpr int NT = 512 / R;
   TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
                     y->H, D, y->L, n, ntile, slab0, ctx->status_dev};

@@ -72,18 +72,21 @@ def test_mixer_bf16_tensor_core_staged_lengths(ctx, n, H, D):
     ctx.poll_status()
 
 
-@pytest.mark.parametrize("dt,L,H", [("bf16", 131072, 2), ("f16", 131072, 1), ("bf16", 3 * 4096, 3)])
-def test_mixer_131072_radix32_on_tensor_cores(ctx, dt, L, H):
-    # n = 131072 with d_head = 64: both radix-32 steps are tensor-core kernels fed by whole-row TMA boxes;
-    # a short sequence (whole 4096-row blocks) reads the missing blocks as zero and writes none of them
-    w = W.Workload("t", B=1, L=L, H=H, D=64, dtype=dt, n_fft=131072, seed=L + H)
+@pytest.mark.parametrize("dt,n,L,H", [("bf16", 131072, 131072, 2), ("f16", 131072, 131072, 1), ("bf16", 131072, 3 * 4096, 3),
+                                      ("bf16", 65536, 65536, 2), ("f16", 65536, 5 * 4096, 3), ("bf16", 32768, 32768, 3),
+                                      ("f16", 32768, 32768, 2), ("bf16", 32768, 2 * 4096, 2)])
+def test_mixer_131072_radix32_on_tensor_cores(ctx, dt, n, L, H):
+    # n = 4096 R, R = 32, 16, 8, with d_head = 64: both radix-R steps are tensor-core kernels fed by whole-row
+    # TMA boxes (R < 32: 32 / R sets of rows share a lane group); a short sequence (whole 4096-row blocks) reads
+    # the missing blocks as zero and writes none of them
+    w = W.Workload("t", B=1, L=L, H=H, D=64, dtype=dt, n_fft=n, seed=L + H)
     x = W.activations(w, structured=True).cuda()
     g = W.random_gate(w).cuda()
     ybig = torch.full((1, L + 8, H, 64), 7.0, dtype=W.torch_dtype(dt), device="cuda")
-    S.spectre_mixer_forward(ctx, x, g, y=ybig[:, :L], n_fft=131072)
+    S.spectre_mixer_forward(ctx, x, g, y=ybig[:, :L], n_fft=n)
     torch.cuda.synchronize()
     ctx.poll_status()
-    ref = O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=131072)
+    ref = O.mixer(W.to_f64(x), gate_to_complex(g), n_fft=n)
     assert_close(W.to_f64(ybig[:, :L]), ref, dt)
     assert bool((ybig[:, L:] == 7.0).all())
 
