@@ -52,8 +52,8 @@ typedef struct spectre_ctx spectre_ctx;   /* opaque: device properties, launch l
 /* Creates a context for CUDA device `device`.  Besides host memory it owns six small device
  * tables (the 64-point and 49-point DFT matrices of the tensor-core mixers, 32 KiB each; the
  * twiddles between two 64-point stages and a quarter-wave twiddle table, 16 KiB each; the twiddles
- * of the four-step splits n = 4096 R, 63 KiB; the four 32-point DFT matrices of the radix-32
- * kernels, 64 KiB) and one pinned status word, all released by spectre_destroy.  No other
+ * of the four-step splits n = 4096 R, 63 KiB; the DFT matrices of the tensor-core radix-32 ... 2
+ * kernels, 320 KiB) and one pinned status word, all released by spectre_destroy.  No other
  * call allocates. */
 int spectre_create(spectre_ctx** out, int device);
 int spectre_destroy(spectre_ctx* ctx);

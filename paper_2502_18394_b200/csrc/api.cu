@@ -107,7 +107,7 @@ extern "C" int spectre_create(spectre_ctx** out, int device) {
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft49, 128 * 128 * sizeof(__half));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw64x64, 2048 * sizeof(float2));
   if (e2 == cudaSuccess) e2 = cudaMalloc(&c->tw_staged, 63 * 128 * sizeof(float2));
-  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft32, 3 * 4 * 16384);
+  if (e2 == cudaSuccess) e2 = cudaMalloc(&c->dft32, 5 * 4 * 16384);
   if (e2 == cudaSuccess) e2 = cudaHostAlloc(reinterpret_cast<void**>(&c->status_host), sizeof(int), cudaHostAllocMapped);
   if (e2 == cudaSuccess) {
     *c->status_host = 0;

@@ -23,7 +23,7 @@ struct spectre_ctx {
   void* tw64x64;          // device: W_4096^{row d}, even columns d, in the epilogue threads' own order (float2), 16 KiB
   void* tw_staged;        // device: twiddles of the four-step split n = 4096 R, R = 1..32 (float2): rows R - 1 + k1 of
                           // 128 entries, W_n^{64 k1 t1} (t1 < 64) then W_n^{k1 t2} (t2 < 64); 63 KiB
-  void* dft32;            // device: DFT matrices of the tensor-core radix-32 / 16 / 8 kernels (MMA operand layout), 3 x 4 x 16 KiB
+  void* dft32;            // device: DFT matrices of the tensor-core radix-32 ... 2 kernels (MMA operand layout), 5 x 4 x 16 KiB
   int* status_host;       // pinned, device-mapped status word written by kernels whose waits ran out
   int* status_dev;
 };

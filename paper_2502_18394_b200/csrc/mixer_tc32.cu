@@ -1,5 +1,5 @@
-// The radix-R steps of the four-step split n = R * 4096 for R = 32, 16, 8 (Sec. 3.2 steps 2 and 4 at
-// n = 131072, 65536, 32768) on the tensor cores, for bf16 or fp16 activations with d_head = 64.  They
+// The radix-R steps of the four-step split n = R * 4096 for R = 32 ... 2 (Sec. 3.2 steps 2 and 4 at
+// n = 131072 ... 8192) on the tensor cores, for bf16 or fp16 activations with d_head = 64.  They
 // replace the transposing ALU kernels of mixer_tc4k.cu around the same core.  Described for R = 32:
 //
 //   tc_in32_kernel   rows n1 * 4096 + t' of [B, L, H, D] are whole 128-byte lines.  A TMA box
@@ -20,10 +20,11 @@
 //                    x 32 n1 complete 128-byte output rows, staged (128-byte swizzle) and written by
 //                    TMA stores.
 //
-// R = 16 and 8 use the same MMA shape: the 32 contracted rows of a lane group are S = 32 / R independent
-// sets of R rows (boxes of R rows, one 1024-byte swizzle atom per 8), the matrices are block diagonal
+// R < 32 uses the same MMA shape: the 32 contracted rows of a lane group are S = 32 / R independent
+// sets of R rows (one TMA box of R rows x S sets lands them set by set), the matrices are block diagonal
 // within a group as well (an R-point DFT per set), and a set stands for another t' (tc_in32: S times
-// as many t2 per item, store runs of 32 S bytes) or another block of row slots (tc_out32).
+// as many t2 per item, store runs of 32 S bytes) or another 128-byte piece of the units' results
+// (tc_out32).
 //
 // Both are persistent, one CTA per SM, four roles joined by mbarriers: a load warp keeps up to three
 // half items (32 KB of operands each) in flight through a ring of four slots, an MMA warp starts an
@@ -51,7 +52,7 @@ constexpr int kXOutSmem = kXMat + 2 * kXItemOp + 2 * 32768 + 192;
 constexpr int kXImgBytes = 65536, kXGBytes = 16384, kXOutBytes = 65536;   // as in mixer_tc4k.cu
 static_assert(kXInSmem <= 232448 && kXOutSmem <= 232448, "shared memory");
 
-// ---- the matrices: four per radix R = 32, 16, 8 (in this order) -----------------------------------
+// ---- the matrices: four per radix R = 32, 16, 8, 4, 2 (in this order) -----------------------------
 // Row m of a matrix: lane group m / 64, then 16-lane blocks of 8 indices with part 0 in the lower 8
 // lanes and part 1 in the upper 8 (where a 16x256b TMEM load puts both into one thread); column kk:
 // group kk / 32, contracted index kk % 32; zero unless the groups agree.  For R < 32 the 32 indices of
@@ -78,7 +79,7 @@ __global__ void build_dft32_kernel(unsigned char* mats_all) {
   *reinterpret_cast<__half*>(mats + 3 * kXMat + off) = __float2half(inv);
 }
 int build_dft32(void* mats, cudaStream_t st) {
-  build_dft32_kernel<<<dim3(32, 3), 256, 0, st>>>(reinterpret_cast<unsigned char*>(mats));
+  build_dft32_kernel<<<dim3(32, 5), 256, 0, st>>>(reinterpret_cast<unsigned char*>(mats));
   SPECTRE_LAUNCH_OK("build_dft32_kernel");
   return SPECTRE_OK;
 }
@@ -209,13 +210,15 @@ __device__ __forceinline__ float2 gate_ext(const float2* __restrict__ g, int k, 
   return v;
 }
 
-// R = 32, 16 or 8 (n = 4096 R).  The 32 contracted rows of a lane group hold S = 32 / R sets of R rows n1:
-// set s of lane group gq is row t' = 64 (4 a + u) + t2 with t2 = 4 S t2b + 2 S m + 2 s + gq, so an
-// accumulator m covers 2 S consecutive t2 and a store box row (tile, k1, pair) is a run of 32 S bytes.
+// R = 32 ... 2 (n = 4096 R).  The 32 contracted rows of a lane group hold S = 32 / R sets of R rows n1:
+// set s of lane group gq is row t' = 64 (4 a + u) + t2 with t2 = 4 S t2b + 2 S m + S gq + s (one TMA box of
+// R n1 x S t' lands a lane group's 32 rows set by set), so an accumulator m covers 2 S consecutive t2 and a
+// store box row (tile, k1, pair) is a run of 32 S bytes (at most 256: R = 2 stores two boxes of 128).
 template <bool F16, int R>
 __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_constant__ CUtensorMap tm_in,
                                                                  const __grid_constant__ CUtensorMap tm_img, const TcIn32Params p) {
   constexpr int S = 32 / R, T2B = 16 / S;                      // sets per lane group; t2 blocks (of 4 S) per unit row
+  static_assert(R == 32 || R == 16 || R == 8 || R == 4 || R == 2, "radix");
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* Asm = smem;                                   // hi, lo (bf16) or the fp16 matrix
   unsigned char* Op = smem + 2 * kXMat;                        // ring of four half-item slots
@@ -255,7 +258,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
     });
   } else if (warp == kXEpiWarps + 2) {
     // ---- load warp: R = 32: per u one box of the rows of both lane groups (t' and t' + 1), all 32 n1 of each;
-    //      R < 32: per (u, lane group, set) one box of R rows n1 ----
+    //      R < 32: per (u, lane group) one box of S consecutive t' x R rows n1 ----
     ok = load_warp_loop(bar, nitems, T, ok, [&](int item, int m, int slot) {
       const int slab = p.slab0 + item / (16 * T2B), a = (item / T2B) & 15, t2b = item % T2B;
       const int b = slab / p.H, h = slab - b * p.H;
@@ -265,9 +268,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
           tma_load_5d(smem_u32(Op) + slot * kXHalfOp + u * 2 * kXBox, &tm_in, 0, 0, tp, h, b, bar.slotFull(slot));
         } else {
           for (int gq = 0; gq < 2; ++gq)
-            for (int s = 0; s < S; ++s)
-              tma_load_5d(smem_u32(Op) + slot * kXHalfOp + (u * 2 + gq) * kXBox + s * R * 128, &tm_in, 0, 0, tp + 2 * s + gq, h, b,
-                          bar.slotFull(slot));
+            tma_load_5d(smem_u32(Op) + slot * kXHalfOp + (u * 2 + gq) * kXBox, &tm_in, 0, 0, tp + S * gq, h, b, bar.slotFull(slot));
         }
       }
     });
@@ -301,8 +302,8 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
       const int a = (item / T2B) & 15, t2b = item % T2B;
 #pragma unroll
       for (int u = 0; u < 4; ++u) nA[u] = __ldg(p.twr + 128 * k1 + 4 * a + u);
-      nB0 = __ldg(p.twr + 128 * k1 + 64 + 4 * S * t2b + 2 * set + gq);
-      nB1 = __ldg(p.twr + 128 * k1 + 64 + 4 * S * t2b + 2 * S + 2 * set + gq);
+      nB0 = __ldg(p.twr + 128 * k1 + 64 + 4 * S * t2b + S * gq + set);
+      nB1 = __ldg(p.twr + 128 * k1 + 64 + 4 * S * t2b + 2 * S + S * gq + set);
     };
     if ((int)blockIdx.x < nitems) fetch_tw(blockIdx.x);
     int it = 0;
@@ -353,7 +354,7 @@ __global__ void __launch_bounds__(kXInThreads, 1) tc_in32_kernel(const __grid_co
 #pragma unroll
               for (int x = 0; x < 4; ++x)
                 *reinterpret_cast<uint4*>(box + (((4 * wh + x) * R + k1) * 4 + tq) * (32 * S) +
-                                          16 * (S == 1 ? (gq ^ (k1 & 1)) : 2 * set + gq)) =        // R = 32: 32-byte swizzle of the box
+                                          16 * (S == 1 ? (gq ^ (k1 & 1)) : S * gq + set)) =        // R = 32: 32-byte swizzle of the box
                     make_uint4(chunk[x][0], chunk[x][1], chunk[x][2], chunk[x][3]);
             }
           }
@@ -407,12 +408,15 @@ struct TcOut32Params {
   int* status;
 };
 
-// R = 32, 16 or 8.  The 32 contracted rows of a lane group hold S = 32 / R sets of R rows k1: set s takes
-// the row slots of block S blk + s, so an item covers 16 S values of t' and R output rows n1 for each.
+// R = 32 ... 2.  A unit's result is 512 pieces of 128 bytes (8 row slots x 4 pairs; piece e2 holds rows
+// t' / 64 = 2 (e2 % 32) + {0, 1}, s1 / 4 = e2 / 32, s1 % 4 = 0..3).  The 32 contracted rows of a lane group
+// hold S = 32 / R sets of R rows k1: set s of accumulator m is piece e2 = 2 S blk + S m + s (one TMA box of
+// R k1 x S pieces per lane group and tile), so an item covers 16 S values of t' and R output rows n1 for each.
 template <bool F16, int R>
 __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_constant__ CUtensorMap tm_res,
                                                                   const __grid_constant__ CUtensorMap tm_out, const TcOut32Params p) {
   constexpr int S = 32 / R;
+  static_assert(R == 32 || R == 16 || R == 8 || R == 4 || R == 2, "radix");
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* Op = smem;                                    // ring of four half-item slots
   unsigned char* Stg = smem + 2 * kXItemOp;                    // two boxes of [set (S)][t'l (8)][n1 (R)][128 bytes], swizzled
@@ -449,14 +453,13 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
       issue_item_mmas(tmem + 256 * m, smem_u32(Asm), 1, smem_u32(Op) + slot * kXHalfOp, 4 * kXBox, kXBox, idesc);
     });
   } else if (warp == kXEpiWarps + 2) {
-    // ---- load warp: per lane group, tile and set one box of 8 row slots x R k1 ----
+    // ---- load warp: per lane group and tile one box of S pieces x R k1 ----
     ok = load_warp_loop(bar, nitems, T, ok, [&](int item, int m, int slot) {
       const int slab_local = item % p.cnt, blk = item / p.cnt;
       for (int gq = 0; gq < 2; ++gq)
         for (int jb = 0; jb < 4; ++jb)
-          for (int s = 0; s < S; ++s)
-            tma_load_4d(smem_u32(Op) + slot * kXHalfOp + (gq * 4 + jb) * kXBox + s * R * 128, &tm_res, 128 * (S * blk + s) + 64 * m,
-                        4 * gq + jb, 0, slab_local, bar.slotFull(slot));
+          tma_load_5d(smem_u32(Op) + slot * kXHalfOp + (gq * 4 + jb) * kXBox, &tm_res, 0, 0, 2 * S * blk + S * m, 4 * gq + jb, slab_local,
+                      bar.slotFull(slot));
     });
   } else if (warp == kXEpiWarps + 1) {
     // ---- store warp: two TMA stores per filled box, the box is free once they have read it ----
@@ -468,10 +471,9 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
         ok = mbar_wait(bar.boxFull(m), it & 1);
         if (ok && T == 0) {
           for (int s = 0; s < S; ++s) {
-            // row slots 16 bs .. + 15 of every unit: s1 / 4 = bs / 16, rows t' / 64 = 4 (bs % 16) + {0..3}, s1 % 4 = {0..3}
-            const int bs = S * blk + s, k4 = bs >> 4, row0 = 4 * (bs & 15);
-            // box rows t'l = 0..3: t' = 64 (row0 + 2m) + 4 k4 + {0..3}; t'l = 4..7: the next t' / 64
-            const int tp = 64 * (row0 + 2 * m) + 4 * k4;
+            // box rows t'l = 0..3: t' = 64 row + 4 k4 + {0..3}; t'l = 4..7: the next t' / 64
+            const int e2 = 2 * S * blk + S * m + s, k4 = e2 >> 5, row = 2 * (e2 & 31);
+            const int tp = 64 * row + 4 * k4;
             const uint32_t src = smem_u32(Stg) + 32768 * m + s * (8 * R * 128);
             tma_store_5d(&tm_out, 0, 0, tp, h, b, src);
             tma_store_5d(&tm_out, 0, 0, tp + 64, h, b, src + 4 * R * 128);
@@ -506,7 +508,7 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
             tmem_ld_wait();
             if (jb < 3) tmem_ld_16x256b_x4(taddr0 + 64 * (jb + 1), r[(jb + 1) & 1]);
             const uint32_t (&rr)[16] = r[jb & 1];
-            unsigned char* prow = box + (set * 8 * R + n1) * 128 + (((4 * gq + jb) ^ (n1 & 7)) * 16) + 4 * tq;
+            unsigned char* pcol = box + (set * 8 * R + n1) * 128 + 4 * tq;          // + t'l R rows, + the swizzled 16-byte chunk
 #pragma unroll
             for (int x = 0; x < 4; ++x) {                       // row slot t'l = 4 wh + x of the box, pair tq
               // rows (n1, C) and (n1, S) applied to the columns (re, im): y = (C re - S im) + j (S re + C im)
@@ -514,7 +516,8 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
               const float yb = __uint_as_float(rr[4 * x + 2]) + __uint_as_float(rr[4 * x + 1]);
               const uint32_t yo = F16 ? pack_h2(ya, yb) : pack_bf2(ya, yb);
               if (x == 0) bad |= nonfinite16x2<F16>(yo);       // every row of an overflowed column is non-finite: one row is enough
-              *reinterpret_cast<uint32_t*>(prow + (4 * wh + x) * (R * 128)) = yo;
+              const int srow = (4 * wh + x) * R + n1;                      // row of the set's block: the swizzle key is row % 8
+              *reinterpret_cast<uint32_t*>(pcol + (4 * wh + x) * (R * 128) + (((4 * gq + jb) ^ (srow & 7)) * 16)) = yo;
             }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -560,7 +563,7 @@ bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_
     return (reinterpret_cast<uintptr_t>(a->ptr) & 15) == 0 && a->stride_l % 8 == 0 && a->stride_h % 8 == 0 &&
            a->stride_b % 8 == 0 && a->stride_l > 0 && a->stride_h > 0 && a->stride_b > 0;
   };
-  return (n == 131072 || n == 65536 || n == 32768) && v->D == 64 && v->L % 4096 == 0 && ok(v) && ok(y) && ctx->dft32 != nullptr &&
+  return n >= 8192 && n <= 131072 && (n & (n - 1)) == 0 && v->D == 64 && v->L % 4096 == 0 && ok(v) && ok(y) && ctx->dft32 != nullptr &&
          ctx->tw_staged != nullptr && encode_fn32() != nullptr;
 }
 
@@ -579,14 +582,14 @@ static int make_act_map(CUtensorMap* tm, const spectre_act* a, unsigned box_n1, 
   return SPECTRE_OK;
 }
 
-static int radix_index(int R) { return R == 32 ? 0 : (R == 16 ? 1 : 2); }       // order of the matrix sets in the context
+static int radix_index(int R) { return R == 32 ? 0 : (R == 16 ? 1 : (R == 8 ? 2 : (R == 4 ? 3 : 4))); }   // order of the matrix sets in the context
 
 template <int R>
 static int launch_tc_in_r(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, const float* g, int n, int slab0, int cnt,
                           unsigned char* ws_in, unsigned char* gimg, float* gscale, float sc) {
   constexpr int S = 32 / R;
   CUtensorMap tm;
-  int rc = make_act_map(&tm, v, R, S == 1 ? 2 : 1);
+  int rc = make_act_map(&tm, v, R, S == 1 ? 2 : S);
   if (rc != SPECTRE_OK) return rc;
   CUtensorMap tm_img;
   {
@@ -631,6 +634,8 @@ int launch_tc_in32(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v
     case 32: return launch_tc_in_r<32>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
     case 16: return launch_tc_in_r<16>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
     case 8: return launch_tc_in_r<8>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
+    case 4: return launch_tc_in_r<4>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
+    case 2: return launch_tc_in_r<2>(ctx, st, v, g, n, slab0, cnt, ws_in, gimg, gscale, sc);
     default: return fail(SPECTRE_ERR_UNSUPPORTED, "radix not supported by the tensor-core transpose kernels");
   }
 }
@@ -642,12 +647,12 @@ static int launch_tc_out_r(const spectre_ctx* ctx, cudaStream_t st, const unsign
   int rc = make_act_map(&tm_out, y, R, 4);
   if (rc != SPECTRE_OK) return rc;
   {
-    // the units' results as fp16: (one unit, tile, k1, slab of the group)
-    cuuint64_t dims[4] = {(cuuint64_t)kXOutBytes / 2, 8, R, (cuuint64_t)cnt};
-    cuuint64_t strides[3] = {(cuuint64_t)kXOutBytes, 8 * (cuuint64_t)kXOutBytes, 8 * R * (cuuint64_t)kXOutBytes};
-    cuuint32_t box[4] = {64, 1, R, 1};
-    cuuint32_t es[4] = {1, 1, 1, 1};
-    CUresult r = encode_fn32()(&tm_res, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<unsigned char*>(ws_out), dims, strides, box, es,
+    // the units' results as fp16: (128-byte piece, k1, piece index within the unit, tile, slab of the group)
+    cuuint64_t dims[5] = {64, R, 512, 8, (cuuint64_t)cnt};
+    cuuint64_t strides[4] = {8 * (cuuint64_t)kXOutBytes, 128, (cuuint64_t)kXOutBytes, 8 * R * (cuuint64_t)kXOutBytes};
+    cuuint32_t box[5] = {64, R, S, 1, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    CUresult r = encode_fn32()(&tm_res, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<unsigned char*>(ws_out), dims, strides, box, es,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
@@ -673,6 +678,8 @@ int launch_tc_out32(const spectre_ctx* ctx, cudaStream_t st, const unsigned char
     case 32: return launch_tc_out_r<32>(ctx, st, ws_out, y, slab0, cnt);
     case 16: return launch_tc_out_r<16>(ctx, st, ws_out, y, slab0, cnt);
     case 8: return launch_tc_out_r<8>(ctx, st, ws_out, y, slab0, cnt);
+    case 4: return launch_tc_out_r<4>(ctx, st, ws_out, y, slab0, cnt);
+    case 2: return launch_tc_out_r<2>(ctx, st, ws_out, y, slab0, cnt);
     default: return fail(SPECTRE_ERR_UNSUPPORTED, "radix not supported by the tensor-core transpose kernels");
   }
 }

@@ -627,7 +627,7 @@ static int tc4k_group(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   unsigned char* gimg = ws_out + nunits * k4OutBytes;
   float* gscale = reinterpret_cast<float*>(gimg + (size_t)cnt * R * k4GBytes);
 
-  const bool tc32 = R >= 8 && tc32_supported(ctx, v, y, n);       // radix-32 / 16 / 8 steps on the tensor cores
+  const bool tc32 = R >= 2 && tc32_supported(ctx, v, y, n);       // radix-32 ... 2 steps on the tensor cores
   TcGateParams gp = {reinterpret_cast<const float2*>(g), gimg, gscale, n, n / 2 + 1, R, slab0};
 
   if (tc32) {
@@ -750,7 +750,7 @@ static int tc4k_readout_group(const spectre_ctx* ctx, cudaStream_t st, const flo
   tc_core_kernel<<<grid, k4CoreThreads, k4CoreSmem, st>>>(cp);
   SPECTRE_LAUNCH_OK("tc_core_kernel");
 
-  if (R >= 8 && tc32_supported(ctx, y, y, n)) return launch_tc_out32(ctx, st, ws_out, y, n, slab0, cnt);
+  if (R >= 2 && tc32_supported(ctx, y, y, n)) return launch_tc_out32(ctx, st, ws_out, y, n, slab0, cnt);
   constexpr int NT = 512 / R;
   TcOutParams op = {ws_out, reinterpret_cast<bf16*>(y->ptr), y->stride_b, y->stride_l, y->stride_h,
                     y->H, D, y->L, n, ntile, slab0, ctx->status_dev};

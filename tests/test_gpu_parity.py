@@ -74,11 +74,15 @@ def test_mixer_bf16_tensor_core_staged_lengths(ctx, n, H, D):
 
 @pytest.mark.parametrize("dt,n,L,H", [("bf16", 131072, 131072, 2), ("f16", 131072, 131072, 1), ("bf16", 131072, 3 * 4096, 3),
                                       ("bf16", 65536, 65536, 2), ("f16", 65536, 5 * 4096, 3), ("bf16", 32768, 32768, 3),
-                                      ("f16", 32768, 32768, 2), ("bf16", 32768, 2 * 4096, 2)])
-def test_mixer_131072_radix32_on_tensor_cores(ctx, dt, n, L, H):
-    # n = 4096 R, R = 32, 16, 8, with d_head = 64: both radix-R steps are tensor-core kernels fed by whole-row
+                                      ("f16", 32768, 32768, 2), ("bf16", 32768, 2 * 4096, 2), ("bf16", 16384, 16384, 3),
+                                      ("f16", 16384, 3 * 4096, 2), ("bf16", 8192, 4096, 2)])
+def test_mixer_131072_radix32_on_tensor_cores(ctx, dt, n, L, H, monkeypatch):
+    # n = 4096 R, R = 32 ... 2, with d_head = 64: both radix-R steps are tensor-core kernels fed by whole-row
     # TMA boxes (R < 32: 32 / R sets of rows share a lane group); a short sequence (whole 4096-row blocks) reads
-    # the missing blocks as zero and writes none of them
+    # the missing blocks as zero and writes none of them (n = 8192 takes this path when L is a whole block
+    # but the single-kernel path is switched off)
+    if n == 8192:
+        monkeypatch.setenv("SPECTRE_FORCE_PATH", "staged")
     w = W.Workload("t", B=1, L=L, H=H, D=64, dtype=dt, n_fft=n, seed=L + H)
     x = W.activations(w, structured=True).cuda()
     g = W.random_gate(w).cuda()
