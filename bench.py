@@ -224,7 +224,7 @@ class MixerBench:
         self.d2h = self.h2d
         if project:
             es = 2
-            self.kernel_name = "spectre_project_qv (proj_weights_kernel + project_qv_kernel, tcgen05)"
+            self.kernel_name = "spectre_project_qv (proj_weights_kernel + project_qv_persistent_kernel, tcgen05 + TMA)"
             self.alg_bytes = 3 * w.B * w.L * w.H * w.D * es + 2 * w.H * w.D * w.D * es     # read X, write Q and V, read weights
             self.launches_per_step += 1          # weights transpose + projection replace the pooling pass
         if backward:

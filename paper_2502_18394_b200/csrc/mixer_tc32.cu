@@ -84,28 +84,10 @@ int build_dft32(void* mats, cudaStream_t st) {
   return SPECTRE_OK;
 }
 
-// B operand landed by a 128-byte-swizzled TMA box: MN-major, 64 N elements (128 bytes) per K row, 8 K rows
-// per 1024-byte atom; lbo = bytes between 64-element N blocks, sbo = bytes between 8-row K groups.
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
-  return umma_desc(saddr, lbo, sbo) | ((uint64_t)2 << 61);
-}
 // kind::f16, A K-major, B MN-major, fp32 accumulator, M = 128, N = 256; fmt 0 = fp16, 1 = bf16 (both operands)
 __device__ __forceinline__ uint32_t umma_idesc_x(uint32_t fmt) {
   return (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-               :: "r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.5d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-               :: "r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_store_5d(const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4, %5}], [%6];"
-               :: "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(src) : "memory");
-}
-
 // one item's MMAs for accumulator m: npass passes (matrix 0, then matrix 1 on top) x 4 K steps
 // op_m: the accumulator's first box; `grp` bytes between the boxes of the two lane groups, `lbo` bytes between
 // the boxes of the four 64-column blocks
@@ -541,21 +523,6 @@ __global__ void __launch_bounds__(kXOutThreads, 1) tc_out32_kernel(const __grid_
 }
 
 // ---- host side ---------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn32)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn32 encode_fn32() {
-  static EncodeTiledFn32 fn = [] {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      ptr = nullptr;
-    return reinterpret_cast<EncodeTiledFn32>(ptr);
-  }();
-  return fn;
-}
-
 // Shapes the tensor-core transpose kernels take: n = 4096 R with R = 32, 16 or 8, 64 channels per head (one
 // 128-byte line per row and head), whole 4096-row blocks, 16-byte aligned strides.
 bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_act* y, int n) {
@@ -564,7 +531,7 @@ bool tc32_supported(const spectre_ctx* ctx, const spectre_act* v, const spectre_
            a->stride_b % 8 == 0 && a->stride_l > 0 && a->stride_h > 0 && a->stride_b > 0;
   };
   return n >= 8192 && n <= 131072 && (n & (n - 1)) == 0 && v->D == 64 && v->L % 4096 == 0 && ok(v) && ok(y) && ctx->dft32 != nullptr &&
-         ctx->tw_staged != nullptr && encode_fn32() != nullptr;
+         ctx->tw_staged != nullptr && tensor_map_encoder() != nullptr;
 }
 
 // dims (column, n1, t', head, batch) over [B, L, H, 64]: row = 4096 n1 + t'
@@ -575,7 +542,7 @@ static int make_act_map(CUtensorMap* tm, const spectre_act* a, unsigned box_n1, 
   cuuint64_t strides[4] = {4096 * sl, sl, sh, sb};
   cuuint32_t box[5] = {64, box_n1, box_tp, 1, 1};
   cuuint32_t es[5] = {1, 1, 1, 1, 1};
-  CUresult r = encode_fn32()(tm, a->dtype == SPECTRE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr,
+  CUresult r = tensor_map_encoder()(tm, a->dtype == SPECTRE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr,
                              dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
@@ -598,7 +565,7 @@ static int launch_tc_in_r(const spectre_ctx* ctx, cudaStream_t st, const spectre
     cuuint64_t strides[3] = {1024, 8 * (cuuint64_t)kXImgBytes, (cuuint64_t)kXImgBytes};
     cuuint32_t box[4] = {16 * S, 4, R, 8};
     cuuint32_t es[4] = {1, 1, 1, 1};
-    CUresult r = encode_fn32()(&tm_img, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, ws_in, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    CUresult r = tensor_map_encoder()(&tm_img, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, ws_in, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                S == 1 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
@@ -652,7 +619,7 @@ static int launch_tc_out_r(const spectre_ctx* ctx, cudaStream_t st, const unsign
     cuuint64_t strides[4] = {8 * (cuuint64_t)kXOutBytes, 128, (cuuint64_t)kXOutBytes, 8 * R * (cuuint64_t)kXOutBytes};
     cuuint32_t box[5] = {64, R, S, 1, 1};
     cuuint32_t es[5] = {1, 1, 1, 1, 1};
-    CUresult r = encode_fn32()(&tm_res, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<unsigned char*>(ws_out), dims, strides, box, es,
+    CUresult r = tensor_map_encoder()(&tm_res, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<unsigned char*>(ws_out), dims, strides, box, es,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");

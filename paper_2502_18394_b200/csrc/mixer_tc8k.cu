@@ -326,29 +326,13 @@ __global__ void __launch_bounds__(k8Threads, 1) mixer_tc8192_kernel(const __grid
 
 // ---- host side ---------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      ptr = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(ptr);
-  }();
-  return fn;
-}
-
 // The tensor maps need 16-byte aligned bases and strides and whole 64-row blocks.
 bool tc8192_supported(const spectre_act* v, const spectre_act* y) {
   auto ok = [](const spectre_act* a) {
     return (reinterpret_cast<uintptr_t>(a->ptr) & 15) == 0 && a->stride_l % 8 == 0 && a->stride_h % 8 == 0 &&
            a->stride_b % 8 == 0 && a->stride_l > 0 && a->stride_h > 0 && a->stride_b > 0;
   };
-  return v->L % 64 == 0 && v->D % 8 == 0 && ok(v) && ok(y) && encode_tiled_fn() != nullptr;
+  return v->L % 64 == 0 && v->D % 8 == 0 && ok(v) && ok(y) && tensor_map_encoder() != nullptr;
 }
 
 // dims (column, row digit A, row digit B, head, batch); t1_fastest puts t1 (stride 64 rows) second.
@@ -362,7 +346,7 @@ static int make_row_map(CUtensorMap* tm, const spectre_act* a, bool t1_fastest, 
   }
   cuuint32_t box[5] = {8, box1, box2, 1, 1};
   cuuint32_t es[5] = {1, 1, 1, 1, 1};
-  CUresult r = encode_tiled_fn()(tm, a->dtype == SPECTRE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr, dims, strides, box, es,
+  CUresult r = tensor_map_encoder()(tm, a->dtype == SPECTRE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a->ptr, dims, strides, box, es,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(SPECTRE_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");

@@ -1,6 +1,7 @@
 // Helpers shared by the tcgen05 kernels: shared-memory matrix descriptors, mbarrier waits with an
 // iteration limit, TMEM loads, fp16 / bf16 packing.
 #pragma once
+#include <cuda.h>
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -130,5 +131,50 @@ __device__ __forceinline__ void tmem_ld_16x256b_x1(uint32_t taddr, uint32_t (&r)
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- tensor maps ------------------------------------------------------------------------------------
+// Operand landed by a 128-byte-swizzled TMA box (rows of 128 bytes, 8 rows per 1024-byte atom), as an
+// MN-major operand (the 64 elements of a row run along M / N, the rows along K: lbo = bytes between
+// 64-element blocks, sbo = bytes between 8-row K groups) or as a K-major operand (the row is 64 elements
+// of K, the rows run along M / N: sbo = bytes between 8-row groups, a K step of 16 elements advances the
+// start address by 32 bytes inside the swizzled row; lbo is not used).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  return umma_desc(saddr, lbo, sbo) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t saddr, uint32_t sbo) {
+  return umma_desc(saddr, 16, sbo) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+               :: "r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.5d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+               :: "r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+               :: "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4, %5}], [%6];"
+               :: "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(src) : "memory");
+}
+
+// cuTensorMapEncodeTiled through the runtime (no link against libcuda); NULL if the driver lacks it
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline TensorMapEncodeFn tensor_map_encoder() {
+  static TensorMapEncodeFn fn = [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      ptr = nullptr;
+    return reinterpret_cast<TensorMapEncodeFn>(ptr);
+  }();
+  return fn;
+}
 
 }  // namespace spectre
