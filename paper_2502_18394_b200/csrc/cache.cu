@@ -118,14 +118,22 @@ __global__ void __launch_bounds__(256) append_spectrum_kernel(float* __restrict_
         d1 -= io<T>::load1(old + 1);
       }
     }
-    for (int i = 0; i < nb; ++i) {
-      float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
-      if (live) {
-        float4* p = reinterpret_cast<float4*>(base + ((size_t)i * D + 2 * c) * 2);
-        float4 v = *p;
-        v.x = fmaf(d0, wr, v.x); v.y = fmaf(d0, wi, v.y);
-        v.z = fmaf(d1, wr, v.z); v.w = fmaf(d1, wi, v.w);
-        *p = v;
+    // four bins per round, their loads issued together (the compiler cannot move a load of this array
+    // above the store before it)
+    for (int i0 = 0; i0 < nb; i0 += 4) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (live && i0 + u < nb) v[u] = *reinterpret_cast<const float4*>(base + ((size_t)(i0 + u) * D + 2 * c) * 2);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = min(i0 + u, 31);
+        const float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
+        if (live && i0 + u < nb) {
+          v[u].x = fmaf(d0, wr, v[u].x); v[u].y = fmaf(d0, wi, v[u].y);
+          v[u].z = fmaf(d1, wr, v[u].z); v[u].w = fmaf(d1, wi, v[u].w);
+          *reinterpret_cast<float4*>(base + ((size_t)(i0 + u) * D + 2 * c) * 2) = v[u];
+        }
       }
     }
   }
@@ -217,21 +225,33 @@ __global__ void __launch_bounds__(256) decode_spectrum_kernel(float* __restrict_
     float acc[NR][2];
 #pragma unroll
     for (int r = 0; r < NR; ++r) acc[r][0] = acc[r][1] = 0.f;
-    for (int i = 0; i < nb; ++i) {
-      const float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (live) {
-        float4* p = reinterpret_cast<float4*>(base + ((size_t)i * D + 2 * c) * 2);
-        v = *p;
-        v.x = fmaf(d0, wr, v.x); v.y = fmaf(d0, wi, v.y);
-        v.z = fmaf(d1, wr, v.z); v.w = fmaf(d1, wi, v.w);
-        *p = v;
+    // four bins per round, their loads issued together (the compiler cannot move a load of this array
+    // above the store before it)
+    for (int i0 = 0; i0 < nb; i0 += 4) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (live && i0 + u < nb) v[u] = *reinterpret_cast<const float4*>(base + ((size_t)(i0 + u) * D + 2 * c) * 2);
       }
 #pragma unroll
-      for (int r = 0; r < NR; ++r) {
-        const float cr = __shfl_sync(0xffffffffu, coef[r].x, i), ci = __shfl_sync(0xffffffffu, coef[r].y, i);
-        acc[r][0] = fmaf(cr, v.x, fmaf(-ci, v.y, acc[r][0]));
-        acc[r][1] = fmaf(cr, v.z, fmaf(-ci, v.w, acc[r][1]));
+      for (int u = 0; u < 4; ++u) {
+        const int i = min(i0 + u, 31);
+        const bool in = i0 + u < nb;                          // uniform over the warp
+        const float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
+        if (live && in) {
+          v[u].x = fmaf(d0, wr, v[u].x); v[u].y = fmaf(d0, wi, v[u].y);
+          v[u].z = fmaf(d1, wr, v[u].z); v[u].w = fmaf(d1, wi, v[u].w);
+          *reinterpret_cast<float4*>(base + ((size_t)(i0 + u) * D + 2 * c) * 2) = v[u];
+        }
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+          const float cr = __shfl_sync(0xffffffffu, coef[r].x, i), ci = __shfl_sync(0xffffffffu, coef[r].y, i);
+          if (in) {
+            acc[r][0] = fmaf(cr, v[u].x, fmaf(-ci, v[u].y, acc[r][0]));
+            acc[r][1] = fmaf(cr, v[u].z, fmaf(-ci, v[u].w, acc[r][1]));
+          }
+        }
       }
     }
 #pragma unroll
