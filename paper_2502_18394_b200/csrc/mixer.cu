@@ -349,7 +349,20 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
     for (int s = 0; s + 1 < p.nstage; ++s) S /= p.radix[s];     // where the forward stages would have left off
   } else {
     if (C == 1) {
-      for (int i = threadIdx.x; i < Mloc * 4; i += blockDim.x) sm[i] = load_elem<T>(p, tc, i >> 2, i & 3);
+      // four elements per thread and round, their loads issued together
+      for (int i0 = threadIdx.x; i0 < Mloc * 4; i0 += 4 * blockDim.x) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * blockDim.x;
+          if (i < Mloc * 4) v[u] = load_elem<T>(p, tc, i >> 2, i & 3);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * blockDim.x;
+          if (i < Mloc * 4) sm[i] = v[u];
+        }
+      }
       __syncthreads();
     } else {
       cg::cluster_group cluster = cg::this_cluster();
