@@ -225,17 +225,17 @@ __global__ void __launch_bounds__(256) decode_spectrum_kernel(float* __restrict_
     float acc[NR][2];
 #pragma unroll
     for (int r = 0; r < NR; ++r) acc[r][0] = acc[r][1] = 0.f;
-    // four bins per round, their loads issued together (the compiler cannot move a load of this array
+    // eight bins per round, their loads issued together (the compiler cannot move a load of this array
     // above the store before it)
-    for (int i0 = 0; i0 < nb; i0 += 4) {
-      float4 v[4];
+    for (int i0 = 0; i0 < nb; i0 += 8) {
+      float4 v[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live && i0 + u < nb) v[u] = *reinterpret_cast<const float4*>(base + ((size_t)(i0 + u) * D + 2 * c) * 2);
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         const int i = min(i0 + u, 31);
         const bool in = i0 + u < nb;                          // uniform over the warp
         const float wr = __shfl_sync(0xffffffffu, my.x, i), wi = __shfl_sync(0xffffffffu, my.y, i);
