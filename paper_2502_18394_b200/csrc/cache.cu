@@ -5,25 +5,36 @@
 namespace spectre {
 
 // from mixer.cu / gate.cu
-int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
-                     float2* ws, int* N1_out, int* M_out);
+int forward_decimated(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
+                      float2* ws, int* N1_out, int* M_out, void* ring, int* ring_done);
 bool transform_supported(const spectre_ctx* ctx, int n);
 size_t transform_slab_bytes(int n, int D);
 int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy_max, int* ncopy_used);
+int pool_sum_ring(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, void* ring, int N);
 size_t gate_min_workspace(int B, int H, int D, int n_fft, int r);
 size_t inverse_workspace_bytes(const spectre_ctx* ctx, int n, int D, int nslab);
 int inverse_from_spectrum(const spectre_ctx* ctx, cudaStream_t st, const float* spec, const float* g, const spectre_act* y,
                           int n, void* ws, size_t ws_bytes);
 
 // ---- prefill -----------------------------------------------------------------
-// The forward pass leaves Z = fft_n(a + jb) for each column pair (a, b) in
-// ws[slab_local][k1][kM][D/2], bin k = k1 + N1 kM.  The half spectra of the two
-// real columns follow from Hermitian symmetry (App. B):
+// With Z = fft_n(a + jb) for each column pair (a, b), the half spectra of the two real columns follow
+// from Hermitian symmetry (App. B):
 //   A_k = (Z_k + conj(Z_{n-k})) / 2,   B_k = (Z_k - conj(Z_{n-k})) / (2j).
-// A thread takes kSplitBins consecutive bins of one column pair, all their loads in flight together.
+__device__ __forceinline__ void store_split(float* __restrict__ prefix, size_t slab, int K, int D, int k, int c, float2 z,
+                                            float2 zm) {
+  float4 out;
+  out.x = 0.5f * (z.x + zm.x);
+  out.y = 0.5f * (z.y - zm.y);
+  out.z = 0.5f * (z.y + zm.y);
+  out.w = -0.5f * (z.x - zm.x);
+  *reinterpret_cast<float4*>(prefix + ((slab * K + k) * D + 2 * c) * 2) = out;
+}
+
+// Transforms that fit the on-chip kernel (N1 = 1) leave Z in ws[slab_local][k][D/2].  A thread takes
+// kSplitBins consecutive bins of one column pair, all their loads in flight together.
 constexpr int kSplitBins = 4;
 __global__ void __launch_bounds__(256) split_kernel(const float2* __restrict__ ws, float* __restrict__ prefix, int n,
-                                                    int K, int D, int N1, int M, int slab0, int nslab) {
+                                                    int K, int D, int slab0, int nslab) {
   const int half = D / 2;
   const int kblocks = (K + kSplitBins - 1) / kSplitBins;
   const size_t total = (size_t)nslab * kblocks * half;
@@ -37,24 +48,69 @@ __global__ void __launch_bounds__(256) split_kernel(const float2* __restrict__ w
 #pragma unroll
   for (int u = 0; u < kSplitBins; ++u) {
     const int k = min(k0 + u, K - 1), km = (n - k) % n;
-    const size_t rk = ((size_t)slab_local * N1 + (k % N1)) * M + k / N1;
-    const size_t rm = ((size_t)slab_local * N1 + (km % N1)) * M + km / N1;
-    z[u] = ws[rk * half + c];
-    zm[u] = ws[rm * half + c];
+    z[u] = ws[((size_t)slab_local * n + k) * half + c];
+    zm[u] = ws[((size_t)slab_local * n + km) * half + c];
   }
 #pragma unroll
   for (int u = 0; u < kSplitBins; ++u) {
     const int k = k0 + u;
-    if (k < K) {
-      float4 out;
-      out.x = 0.5f * (z[u].x + zm[u].x);
-      out.y = 0.5f * (z[u].y - zm[u].y);
-      out.z = 0.5f * (z[u].y + zm[u].y);
-      out.w = -0.5f * (z[u].x - zm[u].x);
-      const size_t o = (((size_t)(slab0 + slab_local) * K + k) * D + 2 * c) * 2;
-      *reinterpret_cast<float4*>(prefix + o) = out;
-    }
+    if (k < K) store_split(prefix, (size_t)(slab0 + slab_local), K, D, k, c, z[u], zm[u]);
   }
+}
+
+// Longer transforms, n = N1 M with token t = N1 n2 + n1: the forward pass leaves the M-point spectra of the
+// N1 decimated sequences, Y[n1][k2] in ws[slab_local][n1][k2][D/2], and the last radix-N1 step runs here,
+//   Z[k2 + M k1] = sum_n1 W_N1^{n1 k1} ( W_n^{n1 k2} Y[n1][k2] ).
+// Z[n - k] for k = k2 + M k1 is Z[(M - k2) + M (N1 - 1 - k1)] (k2 > 0), so the thread that owns k2 and
+// M - k2 of one column pair holds both sides of every Hermitian pair it stores: the bins k2 + M k1 and
+// (M - k2) + M k1 for k1 < N1/2 (and, at k2 = 0, bin n/2); the packed spectrum never goes back to memory.
+template <int N1>
+__global__ void __launch_bounds__(256) combine_split_kernel(const float2* __restrict__ ws, float* __restrict__ prefix, int n,
+                                                            int K, int D, int M, int slab0, int nslab) {
+  const int half = D / 2;
+  const int nk2 = M / 2 + 1;
+  const size_t total = (size_t)nslab * nk2 * half;
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int c = (int)(idx % half);
+  const size_t r = idx / half;
+  const int k2 = (int)(r % nk2);
+  const int slab_local = (int)(r / nk2);
+  const int m2 = (M - k2) % M;
+  float2 xa[N1], xb[N1];
+#pragma unroll
+  for (int n1 = 0; n1 < N1; ++n1) {
+    const size_t row = ((size_t)slab_local * N1 + n1) * M;
+    xa[n1] = ws[(row + k2) * half + c];
+    xb[n1] = ws[(row + m2) * half + c];
+  }
+  const float2 wa1 = twiddle_fwd((unsigned)k2, (unsigned)n), wb1 = twiddle_fwd((unsigned)m2, (unsigned)n);
+  float2 wa[N1], wb[N1];
+  wa[0] = wb[0] = make_float2(1.f, 0.f);
+#pragma unroll
+  for (int q = 1; q < N1; ++q) {
+    wa[q] = (q == 1) ? wa1 : cmul(wa[q / 2], wa[q - q / 2]);
+    wb[q] = (q == 1) ? wb1 : cmul(wb[q / 2], wb[q - q / 2]);
+    xa[q] = cmul(xa[q], wa[q]);
+    xb[q] = cmul(xb[q], wb[q]);
+  }
+  Dft<N1, false>::run(xa);
+  Dft<N1, false>::run(xb);
+  const size_t slab = (size_t)(slab0 + slab_local);
+  const bool own = k2 == 0 || k2 == m2;       // k2 = 0 and k2 = M/2 are their own mirror
+#pragma unroll
+  for (int k1 = 0; k1 < N1 / 2; ++k1) {
+    store_split(prefix, slab, K, D, k2 + M * k1, c, xa[k1], k2 == 0 ? xa[(N1 - k1) % N1] : xb[N1 - 1 - k1]);
+    if (!own) store_split(prefix, slab, K, D, m2 + M * k1, c, xb[k1], xa[N1 - 1 - k1]);
+  }
+  if (k2 == 0) store_split(prefix, slab, K, D, M * (N1 / 2), c, xa[N1 / 2], xa[N1 / 2]);
+}
+
+template <int N1>
+static void launch_combine_split(cudaStream_t st, const float2* ws, float* prefix, int n, int K, int D, int M, int slab0,
+                                 int cnt) {
+  const size_t total = (size_t)cnt * (M / 2 + 1) * (D / 2);
+  combine_split_kernel<N1><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, prefix, n, K, D, M, slab0, cnt);
 }
 
 // Ring buffers: rows 0..L-1 <- tokens, rows L..N-1 <- 0 (Alg. 1 PreFill).  A CTA copies kRingRows
@@ -346,27 +402,38 @@ extern "C" int spectre_prefix_cache_prefill(spectre_ctx* ctx, void* stream, cons
   size_t gmax = workspace_bytes / per;
   int group = gmax > (size_t)nslab ? nslab : (int)gmax;
   float2* ws = reinterpret_cast<float2*>(workspace);
+  int v_ring_done = 0;                 // the transform's load pass can fill V_buf on its way
   for (int s0 = 0; s0 < nslab; s0 += group) {
     int cnt = nslab - s0 < group ? nslab - s0 : group;
     int N1 = 1, M = N;
-    rc = forward_spectrum(ctx, st, v, N, s0, cnt, ws, &N1, &M);
+    rc = forward_decimated(ctx, st, v, N, s0, cnt, ws, &N1, &M, cache->V_buf, &v_ring_done);
     if (rc != SPECTRE_OK) return rc;
-    size_t total = (size_t)cnt * ((K + kSplitBins - 1) / kSplitBins) * (D / 2);
-    split_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, cache->prefix_fft, N, K, D, N1, M, s0, cnt);
-    SPECTRE_LAUNCH_OK("split_kernel");
+    switch (N1) {
+      case 1: {
+        size_t total = (size_t)cnt * ((K + kSplitBins - 1) / kSplitBins) * (D / 2);
+        split_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ws, cache->prefix_fft, N, K, D, s0, cnt);
+        break;
+      }
+      case 2: launch_combine_split<2>(st, ws, cache->prefix_fft, N, K, D, M, s0, cnt); break;
+      case 4: launch_combine_split<4>(st, ws, cache->prefix_fft, N, K, D, M, s0, cnt); break;
+      case 8: launch_combine_split<8>(st, ws, cache->prefix_fft, N, K, D, M, s0, cnt); break;
+      case 16: launch_combine_split<16>(st, ws, cache->prefix_fft, N, K, D, M, s0, cnt); break;
+      default: return fail(SPECTRE_ERR_UNSUPPORTED, "outer factor not supported");
+    }
+    SPECTRE_LAUNCH_OK("split kernel");
   }
   const size_t nblocks = (size_t)B * ((N + kRingRows - 1) / kRingRows);
   if (nblocks > 0x7fffffffu) return fail(SPECTRE_ERR_UNSUPPORTED, "B * N_max too large for the ring copy");
   unsigned blocks = (unsigned)nblocks;
-  SPECTRE_IO_DISPATCH(cache->buf_dtype, {
-    ring_fill_kernel<T><<<blocks, 256, 0, st>>>(reinterpret_cast<const T*>(v->ptr), v->stride_b, v->stride_l, v->stride_h,
-                                                reinterpret_cast<T*>(cache->V_buf), B, N, H, D, v->L);
-    ring_fill_kernel<T><<<blocks, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
-                                                reinterpret_cast<T*>(cache->Q_buf), B, N, H, D, q->L);
-  });
-  SPECTRE_LAUNCH_OK("ring_fill_kernel");
-  int used = 1;
-  return pool_sum(ctx, st, q, cache->sum_q, 1, &used);
+  if (!v_ring_done) {
+    SPECTRE_IO_DISPATCH(cache->buf_dtype, {
+      ring_fill_kernel<T><<<blocks, 256, 0, st>>>(reinterpret_cast<const T*>(v->ptr), v->stride_b, v->stride_l, v->stride_h,
+                                                  reinterpret_cast<T*>(cache->V_buf), B, N, H, D, v->L);
+    });
+    SPECTRE_LAUNCH_OK("ring_fill_kernel");
+  }
+  // q is read once: its sum over the sequence and its ring copy come from the same pass
+  return pool_sum_ring(ctx, st, q, cache->sum_q, cache->Q_buf, N);
 }
 
 extern "C" int spectre_prefix_cache_append(spectre_ctx* ctx, void* stream, const spectre_cache* cache, const void* q_t,

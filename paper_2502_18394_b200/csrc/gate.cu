@@ -71,10 +71,12 @@ template <> struct vec8<float> {
   }
 };
 
-template <typename T>
+// RING: the rows also go, as loaded, into the dense copy ring[B][N][H][D]; rows L..N-1 of it are zeroed
+// (the ring buffer of the Prefix-FFT cache, Alg. 1 PreFill), and the slices cover N rows instead of L.
+template <typename T, bool RING>
 __global__ void __launch_bounds__(256, 4) pool_kernel(const T* __restrict__ q, int64_t sb, int64_t sl, int64_t sh, int L,
                                                    int H, int D, int rows_per, int ncopy, size_t copy_stride,
-                                                   float* __restrict__ sums) {
+                                                   float* __restrict__ sums, T* __restrict__ ring, int N) {
   __shared__ float red[8][8][32];                              // [warp][channel][lane]
   // the gate kernels behind this one may start early: they stream weights before they need the sums
   asm volatile("griddepcontrol.launch_dependents;");
@@ -86,17 +88,21 @@ __global__ void __launch_bounds__(256, 4) pool_kernel(const T* __restrict__ q, i
   const bool live = vi < nvec;
   const int h = live ? vi / vec_per_head : 0, c = live ? (vi - h * vec_per_head) * 8 : 0;
   const T* base = q + b * sb + h * sh + c;
-  const int r0 = blockIdx.y * rows_per, r1 = min(L, r0 + rows_per);
+  const int r0 = blockIdx.y * rows_per, r1 = min(L, r0 + rows_per), r2 = RING ? min(N, r0 + rows_per) : r1;
   float acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.f;
   if (live) {
-    for (int r = r0 + warp; r < r1; r += 8 * R) {
+    T* out = RING ? ring + ((size_t)b * N * H + h) * D + c : nullptr;
+    for (int r = r0 + warp; r < r2; r += 8 * R) {
       typename vec8<T>::raw v[R];
 #pragma unroll
       for (int u = 0; u < R; ++u) v[u] = (r + 8 * u < r1) ? vec8<T>::load(base + (int64_t)(r + 8 * u) * sl) : vec8<T>::zero();
 #pragma unroll
-      for (int u = 0; u < R; ++u) vec8<T>::add(v[u], acc);
+      for (int u = 0; u < R; ++u) {
+        vec8<T>::add(v[u], acc);
+        if (RING && r + 8 * u < r2) *reinterpret_cast<typename vec8<T>::raw*>(out + (size_t)(r + 8 * u) * H * D) = v[u];
+      }
     }
   }
 #pragma unroll
@@ -112,8 +118,11 @@ __global__ void __launch_bounds__(256, 4) pool_kernel(const T* __restrict__ q, i
   }
 }
 
-// Sums of q over the sequence into *ncopy_used <= ncopy_max partial copies (the consumer adds them up).
-int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy_max, int* ncopy_used) {
+// Sums of q over the sequence into *ncopy_used <= ncopy_max partial copies (the consumer adds them up);
+// with `ring`, also the copy of q into ring[B][N][H][D] (zero rows from L on).
+static int pool_launch(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy_max,
+                       int* ncopy_used, void* ring, int N) {
+  const int rows = ring ? N : q->L;
   const size_t copy_stride = (size_t)q->B * q->H * q->D;
   const int groups = (q->H * (q->D / 8) + 31) / 32;
   if (q->B > 65535) return fail(SPECTRE_ERR_UNSUPPORTED, "B exceeds 65535");
@@ -122,9 +131,9 @@ int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, floa
   const long long per_slice = (long long)groups * q->B;
   long long slices = (4LL * ctx->sm_count) / per_slice;
   if (slices < 1) slices = 1;
-  int rows_per = (int)((q->L + slices - 1) / slices);
+  int rows_per = (int)((rows + slices - 1) / slices);
   if (rows_per < 8) rows_per = 8;
-  const int nslice = (q->L + rows_per - 1) / rows_per;
+  const int nslice = (rows + rows_per - 1) / rows_per;
   int ncopy = (nslice + 15) / 16;                              // <= 16 CTAs add into one address
   if (ncopy > 8) ncopy = 8;                                    // one batch of loads for the consumer
   if (ncopy > ncopy_max) ncopy = ncopy_max;
@@ -132,11 +141,27 @@ int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, floa
   *ncopy_used = ncopy;
   if (nslice > 1) SPECTRE_CUDA_OK(cudaMemsetAsync(sums, 0, copy_stride * ncopy * sizeof(float), st));
   dim3 grid((unsigned)groups, (unsigned)nslice, (unsigned)q->B);
-  SPECTRE_IO_DISPATCH(q->dtype, pool_kernel<T><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l,
-                                                                     q->stride_h, q->L, q->H, q->D, rows_per, ncopy,
-                                                                     copy_stride, sums));
+  SPECTRE_IO_DISPATCH(q->dtype, {
+    if (ring)
+      pool_kernel<T, true><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
+                                                 q->L, q->H, q->D, rows_per, ncopy, copy_stride, sums,
+                                                 reinterpret_cast<T*>(ring), N);
+    else
+      pool_kernel<T, false><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(q->ptr), q->stride_b, q->stride_l, q->stride_h,
+                                                  q->L, q->H, q->D, rows_per, ncopy, copy_stride, sums, nullptr, 0);
+  });
   SPECTRE_LAUNCH_OK("pool_kernel");
   return SPECTRE_OK;
+}
+
+int pool_sum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, int ncopy_max, int* ncopy_used) {
+  return pool_launch(ctx, st, q, sums, ncopy_max, ncopy_used, nullptr, 0);
+}
+
+// Prefill of the cache's query side in one pass over q: sum over the sequence into sums[B,H,D] and the ring copy.
+int pool_sum_ring(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* q, float* sums, void* ring, int N) {
+  int used = 1;
+  return pool_launch(ctx, st, q, sums, 1, &used, ring, N);
 }
 
 // ---- MLP ---------------------------------------------------------------------

@@ -82,6 +82,9 @@ struct OnchipParams {
   int mode;              // 0: forward, gate, inverse   1: forward only -> spectrum in ws
                          // 2: inverse only, from the gated half spectra in `spec`
   int src_ws, dst_ws;
+  int decim;             // src_ws = 0 only: element j of sequence k1 is token N1 j + k1 (decimated input)
+  int share;             // C = 1 only: the ntile CTAs of a (slab, k1) form a cluster that loads whole head rows
+  void* ring;            // share only: dense [B][n][H][D] copy of the (zero-padded) input written while loading, or NULL
   float scale;           // 1/n, folded into the gate
 };
 
@@ -111,8 +114,9 @@ __device__ __forceinline__ float4 load_elem(const OnchipParams& p, const TileCoo
     size_t row = ((size_t)tc.slab_local * p.N1 + tc.k1) * p.M + j;
     return *reinterpret_cast<const float4*>(p.ws + row * (p.D / 2) + col / 2);
   }
-  if (j >= p.L) return make_float4(0.f, 0.f, 0.f, 0.f);
-  const T* ptr = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + (int64_t)j * p.s_sl + tc.h * p.s_sh + col;
+  const int t = p.decim ? j * p.N1 + tc.k1 : j;
+  if (t >= p.L) return make_float4(0.f, 0.f, 0.f, 0.f);
+  const T* ptr = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + (int64_t)t * p.s_sl + tc.h * p.s_sh + col;
   return io<T>::load4(ptr);
 }
 
@@ -334,6 +338,74 @@ __device__ __forceinline__ void cross_stage(const OnchipParams& p, const TileCoo
   }
 }
 
+// Input of the ntile single-CTA transforms of one (slab, k1), loaded as whole head rows: the CTAs form a
+// cluster, CTA `tile` reads rows [tile Mloc/ntile, (tile+1) Mloc/ntile) across all D columns (a warp
+// covers whole contiguous rows, 16 bytes per lane, all of a thread's loads in flight together) and writes
+// each 4-column group into the shared memory of the CTA that owns its tile.
+// 16 bytes of a row as float4 groups of 4 columns: one group for fp32, two for the 16-bit types
+template <typename T> struct RowPiece;
+template <> struct RowPiece<float> {
+  static constexpr int kGroups = 1;
+  static __device__ __forceinline__ float4 group(const uint4& r, int) {
+    return make_float4(__uint_as_float(r.x), __uint_as_float(r.y), __uint_as_float(r.z), __uint_as_float(r.w));
+  }
+};
+template <> struct RowPiece<bf16> {
+  static constexpr int kGroups = 2;
+  static __device__ __forceinline__ float4 group(const uint4& r, int g) {
+    const unsigned lo = g ? r.z : r.x, hi = g ? r.w : r.y;
+    return make_float4(__uint_as_float(lo << 16), __uint_as_float(lo & 0xffff0000u), __uint_as_float(hi << 16),
+                       __uint_as_float(hi & 0xffff0000u));
+  }
+};
+template <> struct RowPiece<f16> {
+  static constexpr int kGroups = 2;
+  static __device__ __forceinline__ float4 group(const uint4& r, int g) {
+    const unsigned lo = g ? r.z : r.x, hi = g ? r.w : r.y;
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&lo));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&hi));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+};
+
+template <typename T>
+__device__ __forceinline__ void shared_rows_load(const OnchipParams& p, const TileCoord& tc, float4* sm,
+                                                 cg::cluster_group& cluster) {
+  constexpr int G = RowPiece<T>::kGroups;
+  constexpr int kInFlight = 8;                       // 16-byte loads per thread and round
+  const int npc = p.ntile * 4 / G;                   // 16-byte pieces of a row (D = 16 ntile columns)
+  const int per = p.Mloc / p.ntile;
+  const int total = per * npc;
+  const T* src = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + tc.h * p.s_sh;
+  T* ring = p.ring ? reinterpret_cast<T*>(p.ring) + ((size_t)tc.b * p.n * p.H + tc.h) * p.D : nullptr;
+  for (int i0 = threadIdx.x; i0 < total; i0 += kInFlight * blockDim.x) {
+    uint4 v[kInFlight];
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+      const int i = i0 + u * blockDim.x;
+      v[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (i < total) {
+        const int j = tc.tile * per + i / npc, pc = i % npc;
+        const int t = p.decim ? j * p.N1 + tc.k1 : j;
+        if (t < p.L) v[u] = __ldcs(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl + 4 * G * pc));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+      const int i = i0 + u * blockDim.x;
+      if (i < total) {
+        const int j = tc.tile * per + i / npc, pc = i % npc;
+        if (ring) __stcs(reinterpret_cast<uint4*>(ring + (size_t)(p.decim ? j * p.N1 + tc.k1 : j) * p.H * p.D + 4 * G * pc), v[u]);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const int pgx = pc * G + g;
+          cluster.map_shared_rank(sm, pgx >> 2)[(size_t)j * 4 + (pgx & 3)] = RowPiece<T>::group(v[u], g);
+        }
+      }
+    }
+  }
+}
+
 template <typename T, int C>
 __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -348,7 +420,12 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
   if (p.mode == 2) {
     for (int s = 0; s + 1 < p.nstage; ++s) S /= p.radix[s];     // where the forward stages would have left off
   } else {
-    if (C == 1) {
+    if (C == 1 && p.share) {
+      cg::cluster_group cluster = cg::this_cluster();
+      cluster.sync();                       // every CTA of the cluster is resident before remote writes
+      shared_rows_load<T>(p, tc, sm, cluster);
+      cluster.sync();
+    } else if (C == 1) {
       // four elements per thread and round, their loads issued together
       for (int i0 = threadIdx.x; i0 < Mloc * 4; i0 += 4 * blockDim.x) {
         float4 v[4];
@@ -523,11 +600,11 @@ static int launch_onchip_c(const OnchipParams& p, const TransformPlan& pl, int n
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.x = (C == 1 && p.share) ? p.ntile : C;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (C > 1) ? 1 : 0;
+  cfg.numAttrs = (C > 1 || p.share) ? 1 : 0;
   SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
   return SPECTRE_OK;
 }
@@ -646,6 +723,38 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
   SPECTRE_IO_DISPATCH(v->dtype, rc = (launch_strided<T, false>(sp, pl.N1, st)));
   if (rc != SPECTRE_OK) return rc;
   p.src_ws = 1;
+  SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
+}
+
+// Forward transforms of the decimated sequences (used by the cache prefill): with n = N1 M and token
+// t = N1 n2 + n1, ws[slab_local][n1][k2][D/2] = sum_n2 z[N1 n2 + n1] W_M^{n2 k2}, read straight from the
+// activations.  The radix-N1 step over n1 (bin k2 + M k1 = sum_n1 W_N1^{n1 k1} W_n^{n1 k2} ws[n1][k2]) is
+// left to the caller, which can fuse it with what follows.  N1 = 1: the spectrum itself.  With `ring`
+// (dense [B][n][H][D], the activations' dtype) the pass also writes the zero-padded input there when its
+// load path can (rows of whole heads); *ring_done tells the caller whether it did.
+int forward_decimated(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
+                      float2* ws, int* N1_out, int* M_out, void* ring, int* ring_done) {
+  TransformPlan pl;
+  if (!make_plan(ctx, n, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
+  // Up to 16 sequences of kLocalMax tokens: single-CTA transforms whose tiles share whole-row loads.
+  const int ntile = (v->D + 15) / 16;
+  const bool share = n > kLocalMax && n <= 16 * kLocalMax && v->D % 16 == 0 && (ntile == 2 || ntile == 4 || ntile == 8);
+  if (share) {
+    TransformPlan one;
+    if (!make_plan(ctx, kLocalMax, &one)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
+    pl = one;
+    pl.n = n;
+    pl.N1 = n / kLocalMax;
+  }
+  *N1_out = pl.N1; *M_out = pl.M;
+  OnchipParams p = {};
+  fill_common(p, pl, v->H, v->D, v->L);
+  p.src = v->ptr;
+  p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
+  p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
+  p.src_ws = 0; p.decim = pl.N1 > 1; p.share = share;
+  p.ring = share ? ring : nullptr;
+  *ring_done = share && ring != nullptr;
   SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
 }
 
