@@ -436,6 +436,22 @@ def test_cache_prefill_and_append(ctx, dt, N, L, steps):
     assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
 
 
+@pytest.mark.parametrize("dt,N,L,D", [("bf16", 4096, 4001, 64), ("f32", 8192, 8192, 32), ("f16", 16384, 9000, 128),
+                                       ("bf16", 32768, 32761, 64), ("bf16", 65536, 65536, 32), ("f32", 32768, 5, 48)])
+def test_cache_prefill_long_windows(ctx, dt, N, L, D):
+    # windows beyond one CTA's 2048 rows: decimated transforms, last radix step fused with the Hermitian
+    # split; where a head's rows are whole 16-column tiles the transform's load pass also fills V_buf
+    w = W.Workload("t", B=2, L=L, H=3, D=D, dtype=dt, seed=N + L + D, N_max=N)
+    q, v = W.activations(w, stream=1), W.activations(w, stream=2)
+    cache = S.PrefixCache(w.B, w.H, w.D, N, dtype=W.torch_dtype(dt))
+    cache.V_buf.fill_(7.0); cache.Q_buf.fill_(7.0); cache.prefix_fft.fill_(7.0); cache.sum_q.fill_(7.0)
+    S.spectre_prefix_cache_prefill(ctx, cache, q.cuda(), v.cuda())
+    st = O.cache_prefill(W.to_f64(q), W.to_f64(v), N)
+    e_p, e_s = cache_err(cache, st)
+    assert e_p < TOL["f32"] and e_s < TOL["f32"], (e_p, e_s)
+    assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
+
+
 def test_cache_non_power_of_two_window_append(ctx):
     # append works for any window length; prefill the state by hand (zeros)
     N = 100
