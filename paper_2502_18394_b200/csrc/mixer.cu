@@ -203,9 +203,13 @@ __device__ __forceinline__ void run_stage(int R, float4* sm, const float2* tw, i
 // in mode 0, the first inverse stage.  Local position blk*R + q' holds local
 // frequency kl = rev(blk) + (Mloc/R) q'.  Mode 2 starts here: the values come from
 // the gated half spectra instead of the forward stages.
-template <typename T, int R>
+// FIX: the plan is known at compile time (Mloc = 2048 as 16 x 16 x 8), so the index arithmetic of the
+// stages is shifts and masks instead of divisions by run-time values.
+constexpr int kFixMloc = 2048;
+template <typename T, int R, bool FIX>
 __device__ __forceinline__ void middle(const OnchipParams& p, const TileCoord& tc, float4* sm) {
-  const int nwork = (p.Mloc / R) * 4;
+  const int Mloc = FIX ? kFixMloc : p.Mloc;
+  const int nwork = (Mloc / R) * 4;
   const int nst = p.nstage;
   const int slab = p.slab0 + tc.slab_local;
   const float2* g = p.g + (size_t)slab * p.K;
@@ -224,12 +228,16 @@ __device__ __forceinline__ void middle(const OnchipParams& p, const TileCoord& t
       Dft<R, false>::run(xb);
     }
     int rev = 0, tmp = blk;
-    for (int i = nst - 2; i >= 0; --i) {
-      int d = tmp % p.radix[i];
-      tmp /= p.radix[i];
-      rev += d * p.prefix[i];
+    if (FIX) {
+      rev = ((blk & 15) << 4) | (blk >> 4);          // blk < 256: two radix-16 digits swapped
+    } else {
+      for (int i = nst - 2; i >= 0; --i) {
+        int d = tmp % p.radix[i];
+        tmp /= p.radix[i];
+        rev += d * p.prefix[i];
+      }
     }
-    const int kstep = p.Mloc / R;
+    const int kstep = Mloc / R;
 #pragma unroll
     for (int q = 0; q < R; ++q) {
       int kl = rev + kstep * q;
@@ -265,14 +273,14 @@ __device__ __forceinline__ void middle(const OnchipParams& p, const TileCoord& t
 template <typename T>
 __device__ __forceinline__ void run_middle(int R, const OnchipParams& p, const TileCoord& tc, float4* sm) {
   switch (R) {
-    case 16: middle<T, 16>(p, tc, sm); break;
-    case 8: middle<T, 8>(p, tc, sm); break;
-    case 4: middle<T, 4>(p, tc, sm); break;
-    case 2: middle<T, 2>(p, tc, sm); break;
-    case 7: middle<T, 7>(p, tc, sm); break;
-    case 5: middle<T, 5>(p, tc, sm); break;
-    case 3: middle<T, 3>(p, tc, sm); break;
-    default: middle<T, 1>(p, tc, sm); break;
+    case 16: middle<T, 16, false>(p, tc, sm); break;
+    case 8: middle<T, 8, false>(p, tc, sm); break;
+    case 4: middle<T, 4, false>(p, tc, sm); break;
+    case 2: middle<T, 2, false>(p, tc, sm); break;
+    case 7: middle<T, 7, false>(p, tc, sm); break;
+    case 5: middle<T, 5, false>(p, tc, sm); break;
+    case 3: middle<T, 3, false>(p, tc, sm); break;
+    default: middle<T, 1, false>(p, tc, sm); break;
   }
 }
 
@@ -373,7 +381,8 @@ __device__ __forceinline__ void shared_rows_load(const OnchipParams& p, const Ti
                                                  cg::cluster_group& cluster) {
   constexpr int G = RowPiece<T>::kGroups;
   constexpr int kInFlight = 8;                       // 16-byte loads per thread and round
-  const int npc = p.ntile * 4 / G;                   // 16-byte pieces of a row (D = 16 ntile columns)
+  const int npc = p.ntile * 4 / G;                   // 16-byte pieces of a row (D = 16 ntile columns), a power of two
+  const int lg = __ffs(npc) - 1;
   const int per = p.Mloc / p.ntile;
   const int total = per * npc;
   const T* src = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + tc.h * p.s_sh;
@@ -385,7 +394,7 @@ __device__ __forceinline__ void shared_rows_load(const OnchipParams& p, const Ti
       const int i = i0 + u * blockDim.x;
       v[u] = make_uint4(0u, 0u, 0u, 0u);
       if (i < total) {
-        const int j = tc.tile * per + i / npc, pc = i % npc;
+        const int j = tc.tile * per + (i >> lg), pc = i & (npc - 1);
         const int t = p.decim ? j * p.N1 + tc.k1 : j;
         if (t < p.L) v[u] = __ldcs(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl + 4 * G * pc));
       }
@@ -394,7 +403,7 @@ __device__ __forceinline__ void shared_rows_load(const OnchipParams& p, const Ti
     for (int u = 0; u < kInFlight; ++u) {
       const int i = i0 + u * blockDim.x;
       if (i < total) {
-        const int j = tc.tile * per + i / npc, pc = i % npc;
+        const int j = tc.tile * per + (i >> lg), pc = i & (npc - 1);
         if (ring) __stcs(reinterpret_cast<uint4*>(ring + (size_t)(p.decim ? j * p.N1 + tc.k1 : j) * p.H * p.D + 4 * G * pc), v[u]);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -406,19 +415,20 @@ __device__ __forceinline__ void shared_rows_load(const OnchipParams& p, const Ti
   }
 }
 
-template <typename T, int C>
+template <typename T, int C, bool FIX>
 __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int Mloc = FIX ? kFixMloc : p.Mloc;
   float4* sm = reinterpret_cast<float4*>(smem_raw);                       // [Mloc][4] (8 complex pairs per row)
-  float2* tw = reinterpret_cast<float2*>(smem_raw + (size_t)p.Mloc * 64);  // [Mloc] exp(-j 2 pi i / Mloc)
+  float2* tw = reinterpret_cast<float2*>(smem_raw + (size_t)Mloc * 64);    // [Mloc] exp(-j 2 pi i / Mloc)
   const TileCoord tc = tile_coord(p);
-  const int Mloc = p.Mloc;
 
   for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = twiddle_fwd((unsigned)i, (unsigned)Mloc);
 
   int S = Mloc;
   if (p.mode == 2) {
-    for (int s = 0; s + 1 < p.nstage; ++s) S /= p.radix[s];     // where the forward stages would have left off
+    if (FIX) S = 8;
+    else for (int s = 0; s + 1 < p.nstage; ++s) S /= p.radix[s];   // where the forward stages would have left off
   } else {
     if (C == 1 && p.share) {
       cg::cluster_group cluster = cg::this_cluster();
@@ -448,19 +458,34 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
       cluster.sync();
     }
     // forward stages (all but the last), the fused middle, inverse stages mirrored
-    for (int s = 0; s + 1 < p.nstage; ++s) {
-      run_stage<false>(p.radix[s], sm, tw, Mloc, S);
-      S /= p.radix[s];
+    if (FIX) {
+      stage<16, false>(sm, tw, kFixMloc, 2048);
       __syncthreads();
+      stage<16, false>(sm, tw, kFixMloc, 128);
+      __syncthreads();
+    } else {
+      for (int s = 0; s + 1 < p.nstage; ++s) {
+        run_stage<false>(p.radix[s], sm, tw, Mloc, S);
+        S /= p.radix[s];
+        __syncthreads();
+      }
     }
   }
-  run_middle<T>(p.nstage > 0 ? p.radix[p.nstage - 1] : 1, p, tc, sm);
+  if (FIX) middle<T, 8, true>(p, tc, sm);
+  else run_middle<T>(p.nstage > 0 ? p.radix[p.nstage - 1] : 1, p, tc, sm);
   if (p.mode == 1) return;                // forward only: spectrum already written
   __syncthreads();
-  for (int s = p.nstage - 2; s >= 0; --s) {
-    S *= p.radix[s];
-    run_stage<true>(p.radix[s], sm, tw, Mloc, S);
+  if (FIX) {
+    stage<16, true>(sm, tw, kFixMloc, 128);
     __syncthreads();
+    stage<16, true>(sm, tw, kFixMloc, 2048);
+    __syncthreads();
+  } else {
+    for (int s = p.nstage - 2; s >= 0; --s) {
+      S *= p.radix[s];
+      run_stage<true>(p.radix[s], sm, tw, Mloc, S);
+      __syncthreads();
+    }
   }
 
   if (C == 1) {
@@ -588,9 +613,9 @@ static bool make_plan(const spectre_ctx* ctx, int n, TransformPlan* pl) {
   return pl->smem <= (size_t)ctx->max_smem_optin;
 }
 
-template <typename T, int C>
-static int launch_onchip_c(const OnchipParams& p, const TransformPlan& pl, int nslab, cudaStream_t st) {
-  auto kern = onchip_kernel<T, C>;
+template <typename T, int C, bool FIX>
+static int launch_onchip_cf(const OnchipParams& p, const TransformPlan& pl, int nslab, cudaStream_t st) {
+  auto kern = onchip_kernel<T, C, FIX>;
   if (pl.smem > 48 * 1024)
     SPECTRE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
   cudaLaunchConfig_t cfg = {};
@@ -607,6 +632,12 @@ static int launch_onchip_c(const OnchipParams& p, const TransformPlan& pl, int n
   cfg.numAttrs = (C > 1 || p.share) ? 1 : 0;
   SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
   return SPECTRE_OK;
+}
+
+template <typename T, int C>
+static int launch_onchip_c(const OnchipParams& p, const TransformPlan& pl, int nslab, cudaStream_t st) {
+  const bool fix = pl.Mloc == kFixMloc && pl.nstage == 3 && pl.radix[0] == 16 && pl.radix[1] == 16 && pl.radix[2] == 8;
+  return fix ? launch_onchip_cf<T, C, true>(p, pl, nslab, st) : launch_onchip_cf<T, C, false>(p, pl, nslab, st);
 }
 
 template <typename T>
