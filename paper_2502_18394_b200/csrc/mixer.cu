@@ -83,8 +83,8 @@ struct OnchipParams {
                          // 2: inverse only, from the gated half spectra in `spec`
   int src_ws, dst_ws;
   int decim;             // src_ws = 0 only: element j of sequence k1 is token N1 j + k1 (decimated input)
-  int share;             // C = 1 only: the ntile CTAs of a (slab, k1) form a cluster that loads whole head rows
-  void* ring;            // share only: dense [B][n][H][D] copy of the (zero-padded) input written while loading, or NULL
+  int direct;            // C = 1, 2048 rows, 512 threads: the tile is fetched in one round of 16-byte loads
+  void* ring;            // direct only: dense [B][n][H][D] copy of the (zero-padded) input written while loading, or NULL
   float scale;           // 1/n, folded into the gate
 };
 
@@ -346,10 +346,6 @@ __device__ __forceinline__ void cross_stage(const OnchipParams& p, const TileCoo
   }
 }
 
-// Input of the ntile single-CTA transforms of one (slab, k1), loaded as whole head rows: the CTAs form a
-// cluster, CTA `tile` reads rows [tile Mloc/ntile, (tile+1) Mloc/ntile) across all D columns (a warp
-// covers whole contiguous rows, 16 bytes per lane, all of a thread's loads in flight together) and writes
-// each 4-column group into the shared memory of the CTA that owns its tile.
 // 16 bytes of a row as float4 groups of 4 columns: one group for fp32, two for the 16-bit types
 template <typename T> struct RowPiece;
 template <> struct RowPiece<float> {
@@ -376,44 +372,53 @@ template <> struct RowPiece<f16> {
   }
 };
 
+// Input of a single-CTA transform of 2048 rows, 512 threads: the tile's 16 columns of a row are 4 / G
+// 16-byte pieces, exactly kPieces per thread, fetched in one round with all loads in flight: fetch() issues
+// them (first thing in the kernel, so their latency runs under the set-up), place() converts them into the
+// shared-memory tile, ring() stores the raw pieces into a dense copy of the input, if one is wanted.
 template <typename T>
-__device__ __forceinline__ void shared_rows_load(const OnchipParams& p, const TileCoord& tc, float4* sm,
-                                                 cg::cluster_group& cluster) {
-  constexpr int G = RowPiece<T>::kGroups;
-  constexpr int kInFlight = 8;                       // 16-byte loads per thread and round
-  const int npc = p.ntile * 4 / G;                   // 16-byte pieces of a row (D = 16 ntile columns), a power of two
-  const int lg = __ffs(npc) - 1;
-  const int per = p.Mloc / p.ntile;
-  const int total = per * npc;
-  const T* src = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + tc.h * p.s_sh;
-  T* ring = p.ring ? reinterpret_cast<T*>(p.ring) + ((size_t)tc.b * p.n * p.H + tc.h) * p.D : nullptr;
-  for (int i0 = threadIdx.x; i0 < total; i0 += kInFlight * blockDim.x) {
-    uint4 v[kInFlight];
+struct TileRows {
+  static constexpr int G = RowPiece<T>::kGroups;
+  static constexpr int kPieces = 16 / G;
+  static constexpr int kPerRow = 4 / G;              // pieces of a row that belong to the tile
+  uint4 v[kPieces];
+
+  static __device__ __forceinline__ int token(const OnchipParams& p, const TileCoord& tc, int i) {
+    const int j = i / kPerRow;
+    return p.decim ? j * p.N1 + tc.k1 : j;
+  }
+  __device__ __forceinline__ void fetch(const OnchipParams& p, const TileCoord& tc) {
+    const T* src = reinterpret_cast<const T*>(p.src) + tc.b * p.s_sb + tc.h * p.s_sh + tc.tile * 16;
 #pragma unroll
-    for (int u = 0; u < kInFlight; ++u) {
-      const int i = i0 + u * blockDim.x;
+    for (int u = 0; u < kPieces; ++u) {
+      const int i = threadIdx.x + u * blockDim.x;
+      const int t = token(p, tc, i), col = 4 * G * (i % kPerRow);
       v[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (i < total) {
-        const int j = tc.tile * per + (i >> lg), pc = i & (npc - 1);
-        const int t = p.decim ? j * p.N1 + tc.k1 : j;
-        if (t < p.L) v[u] = __ldcs(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl + 4 * G * pc));
-      }
+      if (i < p.Mloc * kPerRow && t < p.L && tc.tile * 16 + col < p.D)
+        v[u] = __ldcs(reinterpret_cast<const uint4*>(src + (int64_t)t * p.s_sl + col));
     }
+  }
+  __device__ __forceinline__ void place(const OnchipParams& p, float4* sm) const {
 #pragma unroll
-    for (int u = 0; u < kInFlight; ++u) {
-      const int i = i0 + u * blockDim.x;
-      if (i < total) {
-        const int j = tc.tile * per + (i >> lg), pc = i & (npc - 1);
-        if (ring) __stcs(reinterpret_cast<uint4*>(ring + (size_t)(p.decim ? j * p.N1 + tc.k1 : j) * p.H * p.D + 4 * G * pc), v[u]);
+    for (int u = 0; u < kPieces; ++u) {
+      const int i = threadIdx.x + u * blockDim.x;
+      if (i < p.Mloc * kPerRow) {
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-          const int pgx = pc * G + g;
-          cluster.map_shared_rank(sm, pgx >> 2)[(size_t)j * 4 + (pgx & 3)] = RowPiece<T>::group(v[u], g);
-        }
+        for (int g = 0; g < G; ++g) sm[(size_t)(i / kPerRow) * 4 + (i % kPerRow) * G + g] = RowPiece<T>::group(v[u], g);
       }
     }
   }
-}
+  __device__ __forceinline__ void ring(const OnchipParams& p, const TileCoord& tc) const {
+    T* dst = reinterpret_cast<T*>(p.ring) + ((size_t)tc.b * p.n * p.H + tc.h) * p.D + tc.tile * 16;
+#pragma unroll
+    for (int u = 0; u < kPieces; ++u) {
+      const int i = threadIdx.x + u * blockDim.x;
+      const int col = 4 * G * (i % kPerRow);
+      if (i < p.Mloc * kPerRow && tc.tile * 16 + col < p.D)
+        __stcs(reinterpret_cast<uint4*>(dst + (size_t)token(p, tc, i) * p.H * p.D + col), v[u]);
+    }
+  }
+};
 
 template <typename T, int C, bool FIX>
 __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
@@ -422,6 +427,9 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
   float4* sm = reinterpret_cast<float4*>(smem_raw);                       // [Mloc][4] (8 complex pairs per row)
   float2* tw = reinterpret_cast<float2*>(smem_raw + (size_t)Mloc * 64);    // [Mloc] exp(-j 2 pi i / Mloc)
   const TileCoord tc = tile_coord(p);
+  const bool direct = C == 1 && p.direct && p.mode != 2;
+  TileRows<T> rows;
+  if (direct) rows.fetch(p, tc);
 
   for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = twiddle_fwd((unsigned)i, (unsigned)Mloc);
 
@@ -430,11 +438,10 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
     if (FIX) S = 8;
     else for (int s = 0; s + 1 < p.nstage; ++s) S /= p.radix[s];   // where the forward stages would have left off
   } else {
-    if (C == 1 && p.share) {
-      cg::cluster_group cluster = cg::this_cluster();
-      cluster.sync();                       // every CTA of the cluster is resident before remote writes
-      shared_rows_load<T>(p, tc, sm, cluster);
-      cluster.sync();
+    if (direct) {
+      rows.place(p, sm);
+      if (p.ring) rows.ring(p, tc);
+      __syncthreads();
     } else if (C == 1) {
       // four elements per thread and round, their loads issued together
       for (int i0 = threadIdx.x; i0 < Mloc * 4; i0 += 4 * blockDim.x) {
@@ -625,11 +632,11 @@ static int launch_onchip_cf(const OnchipParams& p, const TransformPlan& pl, int 
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (C == 1 && p.share) ? p.ntile : C;
+  attr[0].val.clusterDim.x = C;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (C > 1 || p.share) ? 1 : 0;
+  cfg.numAttrs = (C > 1) ? 1 : 0;
   SPECTRE_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
   return SPECTRE_OK;
 }
@@ -762,15 +769,14 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
 // activations.  The radix-N1 step over n1 (bin k2 + M k1 = sum_n1 W_N1^{n1 k1} W_n^{n1 k2} ws[n1][k2]) is
 // left to the caller, which can fuse it with what follows.  N1 = 1: the spectrum itself.  With `ring`
 // (dense [B][n][H][D], the activations' dtype) the pass also writes the zero-padded input there when its
-// load path can (rows of whole heads); *ring_done tells the caller whether it did.
+// load path can; *ring_done tells the caller whether it did.
 int forward_decimated(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
                       float2* ws, int* N1_out, int* M_out, void* ring, int* ring_done) {
   TransformPlan pl;
   if (!make_plan(ctx, n, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
-  // Up to 16 sequences of kLocalMax tokens: single-CTA transforms whose tiles share whole-row loads.
-  const int ntile = (v->D + 15) / 16;
-  const bool share = n > kLocalMax && n <= 16 * kLocalMax && v->D % 16 == 0 && (ntile == 2 || ntile == 4 || ntile == 8);
-  if (share) {
+  // Up to 16 sequences of kLocalMax tokens: single-CTA transforms, no exchange between CTAs.
+  const bool direct = n > kLocalMax && n <= 16 * kLocalMax && v->D % 8 == 0;
+  if (direct) {
     TransformPlan one;
     if (!make_plan(ctx, kLocalMax, &one)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
     pl = one;
@@ -783,9 +789,9 @@ int forward_decimated(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   p.src = v->ptr;
   p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
   p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
-  p.src_ws = 0; p.decim = pl.N1 > 1; p.share = share;
-  p.ring = share ? ring : nullptr;
-  *ring_done = share && ring != nullptr;
+  p.src_ws = 0; p.decim = pl.N1 > 1; p.direct = direct;
+  p.ring = direct ? ring : nullptr;
+  *ring_done = direct && ring != nullptr;
   SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
 }
 
