@@ -85,6 +85,7 @@ struct OnchipParams {
   int decim;             // src_ws = 0 only: element j of sequence k1 is token N1 j + k1 (decimated input)
   int direct;            // C = 1, 2048 rows, 512 threads: the tile is fetched in one round of 16-byte loads
   void* ring;            // direct only: dense [B][n][H][D] copy of the (zero-padded) input written while loading, or NULL
+  const float2* twq;     // (cos, sin)(2 pi r / 8192), r = 0..2048 (quarter wave): source of the twiddles of the fixed plan
   float scale;           // 1/n, folded into the gate
 };
 
@@ -146,7 +147,10 @@ __device__ __forceinline__ float2 gate_at(const float2* __restrict__ g, int k, i
 // One radix-R stage on block size S of the tile in shared memory.
 //   forward (decimation in frequency): y_q'[m] = W_S^{m q'} sum_q x[m + q S/R] W_R^{q q'}
 //   inverse (decimation in time):      x[m + q S/R] = sum_q' conj(W_R^{q q'}) conj(W_S^{m q'}) y_q'[m]
-template <int R, bool INV>
+// COMPACT: tw holds only this stage's factors, W_S^{m q} at [q * (S/R) + m], so that the lanes of a warp
+// (consecutive m) read consecutive words; the strided reads of the full table collide on a few banks when
+// S is small.
+template <int R, bool INV, bool COMPACT = false>
 __device__ __forceinline__ void stage(float4* sm, const float2* tw, int Mloc, int S) {
   const int sub = S / R;
   const int step = Mloc / S;
@@ -165,7 +169,7 @@ __device__ __forceinline__ void stage(float4* sm, const float2* tw, int Mloc, in
     if (INV) {
 #pragma unroll
       for (int q = 1; q < R; ++q) {
-        float2 t = tw[m * q * step];
+        float2 t = COMPACT ? tw[q * sub + m] : tw[m * q * step];
         xa[q] = cmulc(xa[q], t);
         xb[q] = cmulc(xb[q], t);
       }
@@ -175,7 +179,7 @@ __device__ __forceinline__ void stage(float4* sm, const float2* tw, int Mloc, in
     if (!INV) {
 #pragma unroll
       for (int q = 1; q < R; ++q) {
-        float2 t = tw[m * q * step];
+        float2 t = COMPACT ? tw[q * sub + m] : tw[m * q * step];
         xa[q] = cmul(xa[q], t);
         xb[q] = cmul(xb[q], t);
       }
@@ -426,12 +430,28 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
   const int Mloc = FIX ? kFixMloc : p.Mloc;
   float4* sm = reinterpret_cast<float4*>(smem_raw);                       // [Mloc][4] (8 complex pairs per row)
   float2* tw = reinterpret_cast<float2*>(smem_raw + (size_t)Mloc * 64);    // [Mloc] exp(-j 2 pi i / Mloc)
+  float2* tw128 = tw + Mloc;                                               // FIX: [16][8] W_128^{m q}, the second stage's factors
   const TileCoord tc = tile_coord(p);
   const bool direct = C == 1 && p.direct && p.mode != 2;
   TileRows<T> rows;
   if (direct) rows.fetch(p, tc);
 
-  for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = twiddle_fwd((unsigned)i, (unsigned)Mloc);
+  if (FIX) {
+    // W_2048^i = exp(-j(quadrant pi/2 + 2 pi 4 (i % 512) / 8192)) from the quarter-wave table: one load serves
+    // the four quadrants; 512 threads
+    auto rot = [](float2 cs, int qd) {
+      return qd == 0 ? make_float2(cs.x, -cs.y) : qd == 1 ? make_float2(-cs.y, -cs.x)
+           : qd == 2 ? make_float2(-cs.x, cs.y) : make_float2(cs.y, cs.x);
+    };
+    const float2 cs = __ldg(p.twq + 4 * (threadIdx.x & 511));
+    float2 cs2 = make_float2(1.f, 0.f);
+    const int i2 = 16 * (threadIdx.x >> 3) * (threadIdx.x & 7);          // threads 0..127: q = tid / 8, m = tid % 8
+    if (threadIdx.x < 128) cs2 = __ldg(p.twq + 4 * (i2 & 511));
+    for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = rot(cs, i >> 9);
+    if (threadIdx.x < 128) tw128[threadIdx.x] = rot(cs2, i2 >> 9);
+  } else {
+    for (int i = threadIdx.x; i < Mloc; i += blockDim.x) tw[i] = twiddle_fwd((unsigned)i, (unsigned)Mloc);
+  }
 
   int S = Mloc;
   if (p.mode == 2) {
@@ -468,7 +488,7 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
     if (FIX) {
       stage<16, false>(sm, tw, kFixMloc, 2048);
       __syncthreads();
-      stage<16, false>(sm, tw, kFixMloc, 128);
+      stage<16, false, true>(sm, tw128, kFixMloc, 128);
       __syncthreads();
     } else {
       for (int s = 0; s + 1 < p.nstage; ++s) {
@@ -483,7 +503,7 @@ __global__ void __launch_bounds__(512, 1) onchip_kernel(const OnchipParams p) {
   if (p.mode == 1) return;                // forward only: spectrum already written
   __syncthreads();
   if (FIX) {
-    stage<16, true>(sm, tw, kFixMloc, 128);
+    stage<16, true, true>(sm, tw128, kFixMloc, 128);
     __syncthreads();
     stage<16, true>(sm, tw, kFixMloc, 2048);
     __syncthreads();
@@ -616,7 +636,7 @@ static bool make_plan(const spectre_ctx* ctx, int n, TransformPlan* pl) {
   int want = pl->Mloc * 4 / 8;
   int thr = (want + 31) / 32 * 32;
   pl->threads = thr < 64 ? 64 : (thr > 512 ? 512 : thr);
-  pl->smem = (size_t)pl->Mloc * 64 + (size_t)pl->Mloc * 8;
+  pl->smem = (size_t)pl->Mloc * 64 + (size_t)pl->Mloc * 8 + 128 * sizeof(float2);
   return pl->smem <= (size_t)ctx->max_smem_optin;
 }
 
@@ -672,7 +692,8 @@ static int launch_strided(const StridedParams& p, int N1, cudaStream_t st) {
   return SPECTRE_OK;
 }
 
-static void fill_common(OnchipParams& p, const TransformPlan& pl, int H, int D, int L) {
+static void fill_common(const spectre_ctx* ctx, OnchipParams& p, const TransformPlan& pl, int H, int D, int L) {
+  p.twq = reinterpret_cast<const float2*>(ctx->tw8192);
   p.H = H; p.D = D; p.L = L;
   p.n = pl.n; p.K = pl.n / 2 + 1;
   p.M = pl.M; p.Mloc = pl.Mloc; p.C = pl.C; p.N1 = pl.N1;
@@ -700,7 +721,7 @@ static int mixer_typed(const spectre_ctx* ctx, cudaStream_t st, const spectre_ac
                        const spectre_act* y, const TransformPlan& pl, void* ws, size_t ws_bytes) {
   const int nslab = v->B * v->H;
   OnchipParams p = {};
-  fill_common(p, pl, v->H, v->D, v->L);
+  fill_common(ctx, p, pl, v->H, v->D, v->L);
   p.src = v->ptr; p.dst = y->ptr;
   p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
   p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
@@ -744,7 +765,7 @@ int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act*
   if (!make_plan(ctx, n, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
   *N1_out = pl.N1; *M_out = pl.M;
   OnchipParams p = {};
-  fill_common(p, pl, v->H, v->D, v->L);
+  fill_common(ctx, p, pl, v->H, v->D, v->L);
   p.src = v->ptr;
   p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
   p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
@@ -785,7 +806,7 @@ int forward_decimated(const spectre_ctx* ctx, cudaStream_t st, const spectre_act
   }
   *N1_out = pl.N1; *M_out = pl.M;
   OnchipParams p = {};
-  fill_common(p, pl, v->H, v->D, v->L);
+  fill_common(ctx, p, pl, v->H, v->D, v->L);
   p.src = v->ptr;
   p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
   p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
@@ -802,7 +823,7 @@ static int inverse_typed(const spectre_ctx* ctx, cudaStream_t st, const float2* 
                          const TransformPlan& pl, void* ws, size_t ws_bytes) {
   const int nslab = y->B * y->H;
   OnchipParams p = {};
-  fill_common(p, pl, y->H, y->D, y->L);
+  fill_common(ctx, p, pl, y->H, y->D, y->L);
   p.dst = y->ptr;
   p.d_sb = y->stride_b; p.d_sl = y->stride_l; p.d_sh = y->stride_h;
   p.g = reinterpret_cast<const float2*>(g);
