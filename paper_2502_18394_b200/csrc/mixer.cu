@@ -756,36 +756,7 @@ static int mixer_typed(const spectre_ctx* ctx, cudaStream_t st, const spectre_ac
   return SPECTRE_OK;
 }
 
-// Forward transform only (used by the cache prefill): complex spectrum of the
-// pair-packed columns for slabs [slab0, slab0+cnt) into ws, laid out
-// ws[slab_local][k1][kM][D/2] with bin k = k1 + N1 * kM.
-int forward_spectrum(const spectre_ctx* ctx, cudaStream_t st, const spectre_act* v, int n, int slab0, int cnt,
-                     float2* ws, int* N1_out, int* M_out) {
-  TransformPlan pl;
-  if (!make_plan(ctx, n, &pl)) return fail(SPECTRE_ERR_UNSUPPORTED, "transform length not supported");
-  *N1_out = pl.N1; *M_out = pl.M;
-  OnchipParams p = {};
-  fill_common(ctx, p, pl, v->H, v->D, v->L);
-  p.src = v->ptr;
-  p.s_sb = v->stride_b; p.s_sl = v->stride_l; p.s_sh = v->stride_h;
-  p.ws = ws; p.mode = 1; p.dst_ws = 1; p.slab0 = slab0;
-  if (pl.N1 == 1) {
-    p.src_ws = 0;
-    SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
-  }
-  StridedParams sp = {};
-  sp.src = v->ptr; sp.ws = ws;
-  sp.s_sb = v->stride_b; sp.s_sl = v->stride_l; sp.s_sh = v->stride_h;
-  sp.H = v->H; sp.D = v->D; sp.L = v->L; sp.n = pl.n; sp.M = pl.M;
-  sp.slab0 = slab0; sp.nslab = cnt;
-  int rc = SPECTRE_OK;
-  SPECTRE_IO_DISPATCH(v->dtype, rc = (launch_strided<T, false>(sp, pl.N1, st)));
-  if (rc != SPECTRE_OK) return rc;
-  p.src_ws = 1;
-  SPECTRE_IO_DISPATCH(v->dtype, return launch_onchip<T>(p, pl, cnt, st));
-}
-
-// Forward transforms of the decimated sequences (used by the cache prefill): with n = N1 M and token
+// Forward transforms of the decimated sequences (used by the cache prefill and the gate gradient): with n = N1 M and token
 // t = N1 n2 + n1, ws[slab_local][n1][k2][D/2] = sum_n2 z[N1 n2 + n1] W_M^{n2 k2}, read straight from the
 // activations.  The radix-N1 step over n1 (bin k2 + M k1 = sum_n1 W_N1^{n1 k1} W_n^{n1 k2} ws[n1][k2]) is
 // left to the caller, which can fuse it with what follows.  N1 = 1: the spectrum itself.  With `ring`
