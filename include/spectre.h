@@ -260,6 +260,8 @@ typedef struct {
  * rows 0..L-1 <- tokens and rows L..N_max-1 <- 0, sum_q = sum_i q_i.
  * q, v: [B, L, H, D] with L <= N_max, dtype == buf_dtype.  N_max must be a
  * supported n.  workspace >= spectre_prefill_workspace_bytes(...) bytes.
+ * The ring buffers are written by the passes that read q and v (q and v must
+ * not overlap V_buf or Q_buf).
  */
 size_t spectre_prefill_workspace_bytes(const spectre_ctx* ctx, int32_t B, int32_t H, int32_t D,
                                        int32_t N_max);
