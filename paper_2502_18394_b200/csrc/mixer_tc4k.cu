@@ -546,10 +546,13 @@ __global__ void __launch_bounds__(256) tc_gate_amax_kernel(const TcSpecParams p)
   if ((int)threadIdx.x < p.R) p.gscale[blockIdx.x * p.R + threadIdx.x] = m * 1.41421356f;
 }
 
-// CTA = (head, k1, K group j): the 256 bins kA < 64, kB = 4 j .. 4 j + 3 of the unit row.  A warp reads a
-// bin as one 512-byte row (lane = column pair: two float2), multiplies, and drops its fp16 value into a
-// staging array [pair][kA][kB % 4] (pair stride 260 words: 16-byte aligned rows, 4-way conflicts on the
-// 4-byte stores only); the CTA then writes each tile's 4096 contiguous bytes of K group j.
+// CTA = (head, k1, K group j): the 256 bins kA < 64, kB = 4 j .. 4 j + 3 of the unit row.  A warp takes
+// the four bins kB of one kA at a time, two kA per round (8 rows of 512 bytes in flight; lane = column pair:
+// two float2).  With A, B the pair's half-spectrum values, the value to store is conj(Z) with
+//   Z = g (A + jB) for a bin of the lower half, Z = conj(g) (conj(A) + j conj(B)) for a mirrored one
+// (one complex product per bin; at DC and Nyquist only the real parts of gA and gB survive, App. B).  The
+// four fp16 results of a (pair, kA) go into the staging array [pair][kA][kB % 4] as one 16-byte store (pair
+// stride 260 words: no bank conflicts); the CTA then writes each tile's 4096 contiguous bytes of K group j.
 constexpr int kSpecPitch = 260;
 __global__ void __launch_bounds__(256, 3) tc_spec_in_kernel(const TcSpecParams p) {
   extern __shared__ __align__(16) uint32_t spec_stage[];        // [D / 2][kSpecPitch]
@@ -557,27 +560,45 @@ __global__ void __launch_bounds__(256, 3) tc_spec_in_kernel(const TcSpecParams p
   const int j = blockIdx.x & 15, sk = blockIdx.x >> 4;
   const int slab_local = sk / p.R, k1 = sk - slab_local * p.R, slab = p.slab0 + slab_local;
   const int npair = p.D / 2;
+  const bool live = l < npair;
   const float m = p.gscale[sk];
   const float s = m > 0.f ? p.sc / m : 0.f;
-  const float2* spec = p.spec + (size_t)slab * p.K * p.D;
+  const float4* spec = reinterpret_cast<const float4*>(p.spec + (size_t)slab * p.K * p.D) + (live ? l : 0);
   const float2* g = p.g + (size_t)slab * p.K;
+  const int rowq = p.D / 2;                                     // float4 per bin row
 #pragma unroll 1
-  for (int r0 = 0; r0 < 32; r0 += 8) {
-    float4 ab[8];
-    float2 gk[8];
+  for (int it = 0; it < 8; it += 2) {
+    float4 ab[2][4];
+    float2 gk[2][4];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {                               // 8 bins in flight per warp
-      const int bin = warp + 8 * (r0 + u), kA = bin & 63, kB = 4 * j + (bin >> 6);
-      const int k = k1 + p.R * (kA + 64 * kB), kk = (2 * k <= p.n) ? k : p.n - k;
-      ab[u] = l < npair ? __ldg(reinterpret_cast<const float4*>(spec + (size_t)kk * p.D + 2 * l)) : make_float4(0.f, 0.f, 0.f, 0.f);
-      gk[u] = __ldg(g + kk);
+    for (int a = 0; a < 2; ++a) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int k = k1 + p.R * (warp + 8 * (it + a) + 64 * (4 * j + u));
+        const unsigned kk = (unsigned)((2 * k <= p.n) ? k : p.n - k);
+        ab[a][u] = __ldg(spec + kk * (unsigned)rowq);
+        gk[a][u] = __ldg(g + kk);
+      }
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int bin = warp + 8 * (r0 + u), kA = bin & 63, kB = 4 * j + (bin >> 6);
-      const int k = k1 + p.R * (kA + 64 * kB), kk = (2 * k <= p.n) ? k : p.n - k;
-      const float2 z = pair_from_half(cscale(gk[u], s), ab[u], k, kk, p.n);
-      if (l < npair) spec_stage[l * kSpecPitch + 4 * kA + (bin >> 6)] = pack_h2(z.x, -z.y);   // conjugate: inverse by the conj trick
+    for (int a = 0; a < 2; ++a) {
+      uint32_t h[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int k = k1 + p.R * (warp + 8 * (it + a) + 64 * (4 * j + u));
+        const float4 v = ab[a][u];
+        const float2 gs = cscale(gk[a][u], s);
+        float2 cz;                                              // conj(Z)
+        if (k == 0 || 2 * k == p.n) {
+          cz = make_float2(gs.x * v.x - gs.y * v.y, -(gs.x * v.z - gs.y * v.w));
+        } else if (2 * k < p.n) {
+          cz = cmul(make_float2(gs.x, -gs.y), make_float2(v.x - v.w, -(v.y + v.z)));   // conj(g) conj(A + jB)
+        } else {
+          cz = cmul(gs, make_float2(v.x + v.w, v.y - v.z));                             // g conj(conj A + j conj B)
+        }
+        h[u] = pack_h2(cz.x, cz.y);
+      }
+      if (live) *reinterpret_cast<uint4*>(spec_stage + l * kSpecPitch + 4 * (warp + 8 * (it + a))) = make_uint4(h[0], h[1], h[2], h[3]);
     }
   }
   __syncthreads();
