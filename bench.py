@@ -51,6 +51,15 @@ NCU_TRAFFIC = {"c1": None,
                "c5": (109.6e6, "profiles/launches_c5_and_kernels.md (ncu capture, not this run)")}
 
 
+def pool_launches(B, rows, H, D, sm_count=148):
+    """Kernels of one pooling pass: the pass itself and, when it runs in several slices of the sequence that add
+    into the same sums (the library's rule, restated), the small kernel that clears them."""
+    groups = (H * (D // 8) + 31) // 32
+    slices = max(1, (4 * sm_count) // (groups * B))
+    rows_per = max(8, -(-rows // slices))
+    return 1 + (1 if -(-rows // rows_per) > 1 else 0)
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -218,24 +227,26 @@ class MixerBench:
             self.kernel_name, nk = "mixer (strided + onchip + strided per group)", 3 * groups
         else:
             self.kernel_name, nk = "mixer (onchip_kernel)", 1
-        # pool, gate_out (+ gate_hidden when a head's bins span >= 32 CTAs), mixer kernels, wavelet
-        self.launches_per_step = 2 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk + (1 if w.wavelet_levels and not fused_wrm else 0)
+        # pool (+ the kernel that clears its partial sums when it runs in several slices), gate_out (+ gate_hidden when a
+        # head's bins span >= 32 CTAs), mixer kernels, wavelet
+        self.launches_per_step = (pool_launches(w.B, w.L, w.H, w.D) + 1 + (1 if (w.K + 255) // 256 >= 32 else 0) + nk +
+                                  (1 if w.wavelet_levels and not fused_wrm else 0))
         self.h2d = w.B * w.L * w.H * w.D * (4 if w.dtype == "f32" else 2)
         self.d2h = self.h2d
         if project:
             es = 2
             self.kernel_name = "spectre_project_qv (proj_weights_kernel + project_qv_persistent_kernel, tcgen05 + TMA)"
             self.alg_bytes = 3 * w.B * w.L * w.H * w.D * es + 2 * w.H * w.D * w.D * es     # read X, write Q and V, read weights
-            self.launches_per_step += 1          # weights transpose + projection replace the pooling pass
+            # weights transpose + projection replace the pooling pass
+            self.launches_per_step += 2 - pool_launches(w.B, w.L, w.H, w.D)
         if backward:
             # timed call = spectre_mixer_backward: dV (read dY, write dV, read g) + gate gradient (read V and dY, write dg)
             self.kernel_name = "spectre_mixer_backward (dV through the forward kernels, dg through two fp32 transforms)"
             self.alg_bytes = 2 * mixer_algorithmic_bytes(w)
             per = w.n * (w.D // 2) * 8
             gb = math.ceil(w.B * w.H / max(1, min(w.B * w.H, (128 << 20) // per)))
-            # conjugate gate + forward kernels on dY; per group of heads two forward-only transforms
-            # (one kernel each up to n = 8192, two beyond) and the reduction
-            self.launches_per_step += 1 + nk + gb * (3 if w.n <= 8192 else 5)
+            # conjugate gate + forward kernels on dY; per group of heads two forward-only transforms and the reduction
+            self.launches_per_step += 1 + nk + gb * 3
 
     def step(self, k: int, e0=None, e1=None):
         d = self.sets[k % self.nsets]
@@ -348,10 +359,11 @@ class AppendBench:
             self.units_per_step = w.B * w.N_max
             tok = w.B * w.N_max * w.H * w.D * es
             self.alg_bytes = 4 * tok + w.B * w.H * K * w.D * 8            # read q, v; write both rings; write the spectrum
-            self.kernel_name = "spectre_prefix_cache_prefill (fp32 transforms per group of heads + split, ring fills, pooling)"
+            self.kernel_name = "spectre_prefix_cache_prefill (per group of heads fp32 transforms of the decimated sequences, filling V_buf, + last radix step with the Hermitian split; one pass over q for sum_q and Q_buf)"
             per = w.N_max * (w.D // 2) * 8
             groups = -(-(w.B * w.H) // max(1, min(w.B * w.H, ws.numel() // per)))
-            self.launches_per_step = 3 * groups + 3                       # (strided, on-chip, split) per group; 2 ring fills; pooling
+            # (transforms, combine + split) per group; the query pass (pooling + ring) and the kernel that clears its sums
+            self.launches_per_step = 2 * groups + pool_launches(w.B, w.N_max, w.H, w.D)
             self.h2d, self.d2h = 2 * tok, w.B * w.H * w.D * 4
             self.q_host = self.v_host = None
             return
