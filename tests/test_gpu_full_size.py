@@ -90,6 +90,9 @@ def test_c4_full_size_append_sampled_bins(ctx):
     q = torch.cat([W.activations(one, stream=10 + b) for b in range(w.B)], dim=0).cuda()
     v = torch.cat([W.activations(one, stream=30 + b) for b in range(w.B)], dim=0).cuda()
     S.spectre_prefix_cache_prefill(ctx, cache, q, v)
+    # the ring buffers are written by the passes that read the tokens: bit for bit the inputs, at full size
+    assert torch.equal(cache.V_buf, v) and torch.equal(cache.Q_buf, q)
+    assert rel_err(W.to_f64(cache.sum_q), W.to_f64(q.double().sum(dim=1))) < TOL["f32"]
     del q, v
     steps = w.appends
     qs, vs = W.decode_tokens(w, steps)
