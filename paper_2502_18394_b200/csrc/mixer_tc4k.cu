@@ -554,6 +554,46 @@ __global__ void __launch_bounds__(256) tc_gate_amax_kernel(const TcSpecParams p)
 // four fp16 results of a (pair, kA) go into the staging array [pair][kA][kB % 4] as one 16-byte store (pair
 // stride 260 words: no bank conflicts); the CTA then writes each tile's 4096 contiguous bytes of K group j.
 constexpr int kSpecPitch = 260;
+
+// The bins of a CTA lie on one side of the Nyquist bin: k = k1 + R kA + (n / 64) kB with kB = 4 j + u, so
+// j < 8 means k < n/2 and j >= 8 means k > n/2, except for the two real bins k = 0 (j = 0) and k = n/2 (j = 8)
+// of the first unit row, which the caller patches.  MIRROR is therefore a property of the CTA.
+template <bool MIRROR>
+__device__ __forceinline__ void spec_in_bins(const TcSpecParams& p, const float4* __restrict__ spec, const float2* __restrict__ g,
+                                             uint32_t* spec_stage, int j, int k1, int warp, int l, bool live, float s) {
+  const unsigned rowq = (unsigned)(p.D / 2);                    // float4 per bin row
+  const int kbase = k1 + p.R * (warp + 256 * j), r8 = 8 * p.R, r64 = 64 * p.R;
+#pragma unroll 1
+  for (int it = 0; it < 8; it += 2) {
+    float4 ab[2][4];
+    float2 gk[2][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int k = kbase + (it + a) * r8 + u * r64;
+        const unsigned kk = (unsigned)(MIRROR ? p.n - k : k);
+        ab[a][u] = __ldg(spec + kk * rowq);
+        gk[a][u] = __ldg(g + kk);
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      uint32_t h[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float4 v = ab[a][u];
+        const float2 gs = cscale(gk[a][u], s);
+        // conj(Z): conj(g) conj(A + jB) below the Nyquist bin, g conj(conj A + j conj B) above it
+        const float2 cz = MIRROR ? cmul(gs, make_float2(v.x + v.w, v.y - v.z))
+                                 : cmul(make_float2(gs.x, -gs.y), make_float2(v.x - v.w, -(v.y + v.z)));
+        h[u] = pack_h2(cz.x, cz.y);
+      }
+      if (live) *reinterpret_cast<uint4*>(spec_stage + l * kSpecPitch + 4 * (warp + 8 * (it + a))) = make_uint4(h[0], h[1], h[2], h[3]);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(256, 3) tc_spec_in_kernel(const TcSpecParams p) {
   extern __shared__ __align__(16) uint32_t spec_stage[];        // [D / 2][kSpecPitch]
   const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31;
@@ -565,41 +605,14 @@ __global__ void __launch_bounds__(256, 3) tc_spec_in_kernel(const TcSpecParams p
   const float s = m > 0.f ? p.sc / m : 0.f;
   const float4* spec = reinterpret_cast<const float4*>(p.spec + (size_t)slab * p.K * p.D) + (live ? l : 0);
   const float2* g = p.g + (size_t)slab * p.K;
-  const int rowq = p.D / 2;                                     // float4 per bin row
-#pragma unroll 1
-  for (int it = 0; it < 8; it += 2) {
-    float4 ab[2][4];
-    float2 gk[2][4];
-#pragma unroll
-    for (int a = 0; a < 2; ++a) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int k = k1 + p.R * (warp + 8 * (it + a) + 64 * (4 * j + u));
-        const unsigned kk = (unsigned)((2 * k <= p.n) ? k : p.n - k);
-        ab[a][u] = __ldg(spec + kk * (unsigned)rowq);
-        gk[a][u] = __ldg(g + kk);
-      }
-    }
-#pragma unroll
-    for (int a = 0; a < 2; ++a) {
-      uint32_t h[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int k = k1 + p.R * (warp + 8 * (it + a) + 64 * (4 * j + u));
-        const float4 v = ab[a][u];
-        const float2 gs = cscale(gk[a][u], s);
-        float2 cz;                                              // conj(Z)
-        if (k == 0 || 2 * k == p.n) {
-          cz = make_float2(gs.x * v.x - gs.y * v.y, -(gs.x * v.z - gs.y * v.w));
-        } else if (2 * k < p.n) {
-          cz = cmul(make_float2(gs.x, -gs.y), make_float2(v.x - v.w, -(v.y + v.z)));   // conj(g) conj(A + jB)
-        } else {
-          cz = cmul(gs, make_float2(v.x + v.w, v.y - v.z));                             // g conj(conj A + j conj B)
-        }
-        h[u] = pack_h2(cz.x, cz.y);
-      }
-      if (live) *reinterpret_cast<uint4*>(spec_stage + l * kSpecPitch + 4 * (warp + 8 * (it + a))) = make_uint4(h[0], h[1], h[2], h[3]);
-    }
+  if (j >= 8) spec_in_bins<true>(p, spec, g, spec_stage, j, k1, warp, l, live, s);
+  else spec_in_bins<false>(p, spec, g, spec_stage, j, k1, warp, l, live, s);
+  if (k1 == 0 && warp == 0 && (j == 0 || j == 8) && live) {
+    // the real bins k = 0 and k = n/2 (kA = 0, first kB of the group): only Re(gA) and Re(gB) survive (App. B)
+    const unsigned kk = j == 0 ? 0u : (unsigned)(p.n / 2);
+    const float4 v = __ldg(spec + kk * (unsigned)(p.D / 2));
+    const float2 gs = cscale(__ldg(g + kk), s);
+    spec_stage[l * kSpecPitch] = pack_h2(gs.x * v.x - gs.y * v.y, -(gs.x * v.z - gs.y * v.w));
   }
   __syncthreads();
   for (int e = tid; e < p.ntile * 256; e += 256) {
