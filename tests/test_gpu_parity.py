@@ -452,6 +452,30 @@ def test_cache_prefill_long_windows(ctx, dt, N, L, D):
     assert np.array_equal(W.to_f64(cache.V_buf), st["V_buf"]) and np.array_equal(W.to_f64(cache.Q_buf), st["Q_buf"])
 
 
+@pytest.mark.parametrize("dt,N,D", [("bf16", 8192, 32), ("f32", 1024, 16)])
+def test_cache_prefill_workspace_grouping(ctx, dt, N, D):
+    # a smaller workspace only changes how many (batch, head) slabs go through the transforms together
+    w = W.Workload("t", B=2, L=N - 5, H=3, D=D, dtype=dt, seed=N + D, N_max=N)
+    q, v = W.activations(w, stream=1).cuda(), W.activations(w, stream=2).cuda()
+    per = N * (D // 2) * 8                                  # one slab of pair-packed fp32 spectra
+    full = S.spectre_prefill_workspace_bytes(ctx, w.B, w.H, w.D, N)
+    assert full >= per
+    outs = []
+    for nbytes in (full, per, 2 * per + 100, 4 * per):
+        cache = S.PrefixCache(w.B, w.H, w.D, N, dtype=W.torch_dtype(dt))
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        S.spectre_prefix_cache_prefill(ctx, cache, q, v, workspace=ws)
+        torch.cuda.synchronize()
+        outs.append((cache.prefix_fft.clone(), cache.V_buf.clone(), cache.Q_buf.clone()))
+    for o in outs[1:]:
+        assert torch.equal(o[0], outs[0][0]) and torch.equal(o[1], outs[0][1]) and torch.equal(o[2], outs[0][2])
+    st = O.cache_prefill(W.to_f64(q.cpu()), W.to_f64(v.cpu()), N)
+    P = W.to_f64(outs[1][0]); P = P[..., 0] + 1j * P[..., 1]
+    assert rel_err(P, st["prefix_fft"]) < TOL["f32"]
+    with pytest.raises(S.SpectreError):
+        S.spectre_prefix_cache_prefill(ctx, cache, q, v, workspace=torch.empty(per - 16, dtype=torch.uint8, device="cuda"))
+
+
 def test_cache_non_power_of_two_window_append(ctx):
     # append works for any window length; prefill the state by hand (zeros)
     N = 100
