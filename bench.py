@@ -51,6 +51,12 @@ NCU_TRAFFIC = {"c1": None,
                "c5": (109.6e6, "profiles/launches_c5_and_kernels.md (ncu capture, not this run)")}
 
 
+# The same for the variant legs of c4 that have a capture (per call; both taken at B = 2 and scaled by 4, the
+# traffic being proportional to the batch).
+NCU_TRAFFIC_VARIANT = {("c4", "prefill"): (10208e6, "profiles/launches_c4_prefill.md (ncu capture at B = 2, x4; not this run)"),
+                       ("c4", "readout"): (7015e6, "profiles/launches_c4_readout.md (ncu capture at B = 2, x4; not this run)")}
+
+
 def pool_launches(B, rows, H, D, sm_count=148):
     """Kernels of one pooling pass: the pass itself and, when it runs in several slices of the sequence that add
     into the same sums (the library's rule, restated), the small kernel that clears them."""
@@ -656,7 +662,10 @@ def main():
                 (" - read-out of the whole window from the cached spectrum" if args.readout else "") + \
                 (" with token projections in front (gate from their sum_q)" if args.project else "") + \
                 (", gate shared across heads" if args.shared_gates else "")
-        out.update(result_block(w, m["bench_info"], m, K, Wm, world, cpu, label=label, variant=variant))
+        vname = "prefill" if args.prefill else ("readout" if args.readout else None)
+        reduced = bool(args.heads or args.batch or args.io_dtype)
+        out.update(result_block(w, m["bench_info"], m, K, Wm, world, cpu, label=label, variant=variant,
+                                variant_traffic=None if reduced else NCU_TRAFFIC_VARIANT.get((base, vname))))
         if also is not None:
             out["also"] = also
         print(json.dumps(out))
@@ -734,12 +743,12 @@ def measure(bench, K, Wm, local_rank, dev, e2e_steps):
             "e2e_ms": e2e_ms, "e2e_units": e2e_units, "e2e_steps": Ke, "bench_info": info}
 
 
-def result_block(w, info, m, K, Wm, world, cpu, label="", variant=False):
+def result_block(w, info, m, K, Wm, world, cpu, label="", variant=False, variant_traffic=None):
     if not isinstance(info, dict):
         info = m["bench_info"]
     peak, peak_src = measured_peak()
     achieved = info["alg_bytes"] / (m["kern_ms"] * 1e-3) / 1e9
-    traffic = None if variant else NCU_TRAFFIC.get(w.name)        # None for reduced cases and variant legs
+    traffic = variant_traffic if variant else NCU_TRAFFIC.get(w.name)   # None for reduced cases and legs without a capture
     return {
         "value": m["tot_units"] / (m["tot_ms"] * 1e-3), "unit": "tokens/s", "n_gpus": world,
         "steps": K, "warmup": Wm, "ms_per_step": m["tot_ms"] / K, "higher_is_better": True, "scaling": "weak",
