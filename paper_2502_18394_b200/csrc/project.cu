@@ -25,9 +25,10 @@ template <> __device__ __forceinline__ float pj_wload<bf16>(const bf16* p) { ret
 // [H][d_in][d_out] (x @ W) for q and v  ->  wt[H][2 * 64][64] bf16 (output-major)
 template <typename WT>
 __global__ void __launch_bounds__(256) proj_weights_kernel(const WT* __restrict__ Wq, const WT* __restrict__ Wv,
-                                                           bf16* __restrict__ wt, int H) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= H * 128 * 64) return;
+                                                           bf16* __restrict__ wt, int H, float* __restrict__ sum_q, size_t nsum) {
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < nsum) sum_q[idx] = 0.f;             // the projection kernel adds its token sums into these (no memset node in the stream)
+  if (idx >= (size_t)H * 128 * 64) return;
   const int i = idx & 63, o = (idx >> 6) & 127, h = idx >> 13;
   const WT* W = o < 64 ? Wq : Wv;
   const float w = pj_wload<WT>(W + ((size_t)h * 64 + i) * 64 + (o & 63));
@@ -301,13 +302,15 @@ extern "C" int spectre_project_qv(spectre_ctx* ctx, void* stream, const spectre_
   SPECTRE_CUDA_OK(cudaSetDevice(ctx->device));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   bf16* wt = reinterpret_cast<bf16*>(workspace);
-  const unsigned wblocks = (unsigned)((x->H * 128 * 64 + 255) / 256);
+  const size_t nsum = sum_q ? (size_t)x->B * x->H * 64 : 0, nw = (size_t)x->H * 128 * 64;
+  const unsigned wblocks = (unsigned)(((nsum > nw ? nsum : nw) + 255) / 256);
   if (wdtype == SPECTRE_BF16)
-    proj_weights_kernel<bf16><<<wblocks, 256, 0, st>>>(reinterpret_cast<const bf16*>(Wq), reinterpret_cast<const bf16*>(Wv), wt, x->H);
+    proj_weights_kernel<bf16><<<wblocks, 256, 0, st>>>(reinterpret_cast<const bf16*>(Wq), reinterpret_cast<const bf16*>(Wv), wt, x->H,
+                                                       sum_q, nsum);
   else
-    proj_weights_kernel<float><<<wblocks, 256, 0, st>>>(reinterpret_cast<const float*>(Wq), reinterpret_cast<const float*>(Wv), wt, x->H);
+    proj_weights_kernel<float><<<wblocks, 256, 0, st>>>(reinterpret_cast<const float*>(Wq), reinterpret_cast<const float*>(Wv), wt, x->H,
+                                                        sum_q, nsum);
   SPECTRE_LAUNCH_OK("proj_weights_kernel");
-  if (sum_q) SPECTRE_CUDA_OK(cudaMemsetAsync(sum_q, 0, (size_t)x->B * x->H * 64 * sizeof(float), st));
   if (tensor_map_encoder() == nullptr) return fail(SPECTRE_ERR_UNSUPPORTED, "the driver does not provide cuTensorMapEncodeTiled");
   CUtensorMap tm_x, tm_q, tm_v;
   rc = make_tile_map(&tm_x, x);
