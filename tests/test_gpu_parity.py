@@ -714,7 +714,8 @@ def test_cache_readout_workspace_sizes(ctx):
 # ------------------------------------------------------------------ backward
 @pytest.mark.parametrize("dt,L,n,D", [("f32", 64, 64, 16), ("f32", 196, 196, 24), ("f32", 50, 64, 16), ("bf16", 1024, 1024, 32),
                                       ("f32", 4096, 4096, 16), ("bf16", 8192, 8192, 64), ("f32", 16384, 16384, 16),
-                                      ("bf16", 3000, 4096, 64), ("bf16", 30000, 32768, 32), ("f16", 65536, 65536, 24)])
+                                      ("bf16", 3000, 4096, 64), ("bf16", 30000, 32768, 32), ("f16", 65536, 65536, 24),
+                                      ("bf16", 8192, 8192, 128), ("f32", 2048, 2048, 40)])
 def test_mixer_backward(ctx, dt, L, n, D):
     # dv = mixer(dy, conj g), dg_k = (w_k / n) sum_c conj(Vhat) Ghat against the oracle's gradients
     w = W.Workload("t", B=2, L=L, H=2, D=D, dtype=dt, n_fft=n, seed=3 * n + L)
